@@ -1,0 +1,173 @@
+/*
+ * coral_lmhead.h - C ABI of the weight-grouped LM-head draft step (sm_100a).
+ *
+ * The operation is the "LM Head Router" of the CORAL paper (Section 3.3): the
+ * draft model's LM head W_vocab [V x H] is divided equally into N groups of
+ * v = V/N tokens; per query row a router scores the groups, only the top-n
+ * groups are activated, logits are computed for the tokens of the activated
+ * groups only, a softmax is taken over them, and the best k_tokens candidates
+ * (Appendix B, "Tree decoding": top 10 candidates per node) are returned.
+ *
+ * Conventions
+ *  - Every function returns an int status: CORAL_OK (0) or a negative
+ *    CORAL_ERR_* code.  Nothing throws, aborts or prints.
+ *  - "dev" pointers are CUDA device pointers of the current device, "host"
+ *    pointers are ordinary host memory.  bf16 tensors are raw 16-bit patterns.
+ *  - All matrices are row-major and densely packed.
+ *  - `stream` is a cudaStream_t passed as void* (NULL = default stream).
+ *  - One draft call may be in flight per handle (the workspace is per handle);
+ *    different handles are independent.
+ */
+#ifndef CORAL_LMHEAD_H_
+#define CORAL_LMHEAD_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define CORAL_LMHEAD_ABI_VERSION 1
+
+#define CORAL_OK 0
+#define CORAL_ERR_INVALID (-1)     /* bad argument (NULL, out of range, unsupported shape) */
+#define CORAL_ERR_GROUPING (-2)    /* group_map does not split V into N equal groups */
+#define CORAL_ERR_CUDA (-3)        /* a CUDA runtime call failed */
+#define CORAL_ERR_NOMEM (-4)       /* host or device allocation failed */
+#define CORAL_ERR_TIMEOUT (-5)     /* a bounded device-side wait gave up (device status word) */
+#define CORAL_ERR_BOUNDS (-6)      /* a device-side index check failed (device status word) */
+
+/* Limits of this build. */
+#define CORAL_MAX_GROUPS 256       /* n_groups <= 256 */
+#define CORAL_MAX_K_TOKENS 32      /* k_tokens <= 32 */
+
+/* Execution paths (coral_lmhead_set_path / coral_lmhead_stats.path). */
+#define CORAL_PATH_AUTO 0          /* chosen from (M, k_groups) */
+#define CORAL_PATH_SIMT 1          /* gathered GEMV: weight streaming + fp32 FMA */
+#define CORAL_PATH_TCGEN05 2       /* routed grouped GEMM on tcgen05 / TMEM tiles */
+
+typedef struct coral_lmhead_s *coral_lmhead_handle;
+
+typedef struct coral_lmhead_config {
+    uint32_t struct_size;   /* sizeof(coral_lmhead_config), for versioning */
+    int32_t H;              /* hidden size d; multiple of 8 (128-bit loads) */
+    int32_t V;              /* vocabulary size; multiple of n_groups */
+    int32_t n_groups;       /* N, 1..CORAL_MAX_GROUPS */
+    int32_t max_M;          /* largest number of query rows per draft call */
+    int32_t max_k_groups;   /* largest top-n, 1..n_groups */
+    int32_t max_k_tokens;   /* largest number of candidates, 1..CORAL_MAX_K_TOKENS */
+    uint32_t flags;         /* reserved, 0 */
+} coral_lmhead_config;
+
+typedef struct coral_lmhead_stats {
+    int32_t path;            /* CORAL_PATH_* taken by the last draft call */
+    int32_t M, k_groups, k_tokens;
+    int32_t groups_touched;  /* |U|: size of the union of selected groups over the rows */
+    int32_t kernel_launches; /* kernels the last draft call enqueued */
+    int64_t weight_bytes;    /* |U| * v * H * 2: LM-head bytes the step has to read */
+    int64_t algorithmic_bytes; /* weight_bytes + gate N*H*2 + hidden M*H*2 + outputs M*k_tokens*8 */
+} coral_lmhead_stats;
+
+/* ABI version of the loaded library (CORAL_LMHEAD_ABI_VERSION). */
+int coral_lmhead_version(void);
+
+/*
+ * Sizes of the two device buffers a handle needs, so that the caller can
+ * allocate them (Section 3.3: N groups of v = V/N tokens fixes the packed
+ * copy's size; the workspace holds the gate, tables and per-call partials).
+ * CORAL_ERR_INVALID if cfg is NULL/inconsistent: V % n_groups != 0,
+ * H % 8 != 0, a field < 1, or a limit above is exceeded.
+ */
+int coral_lmhead_query_sizes(const coral_lmhead_config *cfg, size_t *packed_bytes, size_t *workspace_bytes);
+
+/*
+ * Build a handle (Section 3.3: "divide the LM head equally into N groups").
+ *   W_vocab_dev    [V x H] bf16, device.  Frozen LM head of the draft model.
+ *   group_map_host [V] int32, host.  token -> group in [0, N); every group
+ *                  must hold exactly V/N tokens, else CORAL_ERR_GROUPING.
+ *   W_gate_dev     [N x H] bf16, device.  Router matrix (the W2 of Eq. 7).
+ *   packed_buf_dev / workspace_dev: device buffers of at least the sizes
+ *                  coral_lmhead_query_sizes reports, 256-byte aligned, owned by
+ *                  the caller and alive until destroy.  Either may be NULL:
+ *                  the library then allocates (cudaMalloc) and owns that one.
+ * The weights are copied group-contiguously (tokens of a group in ascending
+ * token id) into packed_buf; W_gate and the tables go to the workspace.  The
+ * call synchronises `stream` before returning, so the inputs may be freed.
+ */
+int coral_lmhead_create(coral_lmhead_handle *out, const coral_lmhead_config *cfg, const void *W_vocab_dev,
+                        const int32_t *group_map_host, const void *W_gate_dev, void *packed_buf_dev,
+                        void *workspace_dev, void *stream);
+
+/*
+ * One draft step for M query rows (Section 3.3 and Appendix B, tree decoding):
+ *   gate scores g = W_gate h per row; the k_groups best groups per row
+ *   (descending score, equal scores -> lower group index); logits of the
+ *   tokens of those groups (bf16 inputs, fp32 accumulation); log-softmax over
+ *   the row's active logits; the k_tokens best tokens per row (descending,
+ *   equal -> lower token id).
+ *   hidden_dev       [M x H] bf16, device
+ *   out_ids_dev      [M x k_tokens] int32, device: global token ids
+ *   out_logprobs_dev [M x k_tokens] float, device: natural-log probabilities
+ * Asynchronous on `stream`: no allocation, no host synchronisation.
+ * CORAL_ERR_INVALID (nothing enqueued) for NULL pointers, M < 1 or > max_M,
+ * k_groups outside [1, min(N, max_k_groups)], k_tokens outside
+ * [1, min(max_k_tokens, k_groups * v)].  Device-side problems are reported by
+ * coral_lmhead_status.
+ */
+int coral_lmhead_draft(coral_lmhead_handle h, const void *hidden_dev, int M, int k_groups, int k_tokens,
+                       int32_t *out_ids_dev, float *out_logprobs_dev, void *stream);
+
+/*
+ * Same step with optional taps for checking each stage (all device, any may
+ * be NULL):
+ *   forced_groups_dev [M x k_groups] int32: use these groups (distinct, in
+ *                     [0, N)) instead of the router's choice
+ *   out_groups_dev    [M x k_groups] int32: selected groups in selection order
+ *   out_gate_dev      [M x N] float: router scores
+ *   out_logits_dev    [M x k_groups x v] float: slot s of row m holds the
+ *                     logits of the tokens of group out_groups[m][s] in
+ *                     ascending token id
+ *   out_lse_dev       [M] float: log-sum-exp over the row's active logits
+ */
+int coral_lmhead_draft_ex(coral_lmhead_handle h, const void *hidden_dev, int M, int k_groups, int k_tokens,
+                          const int32_t *forced_groups_dev, int32_t *out_groups_dev, float *out_gate_dev,
+                          float *out_logits_dev, float *out_lse_dev, int32_t *out_ids_dev,
+                          float *out_logprobs_dev, void *stream);
+
+/*
+ * The same draft step for callers that hold HOST buffers (hidden_host
+ * [M x H] bf16; out_ids_host / out_logprobs_host [M x k_tokens]).  Copies the
+ * rows to the device, runs coral_lmhead_draft, copies the results back and
+ * synchronises `stream` before returning.  Pinned host memory makes the copies
+ * asynchronous up to that final synchronisation.
+ */
+int coral_lmhead_draft_host(coral_lmhead_handle h, const void *hidden_host, int M, int k_groups, int k_tokens,
+                            int32_t *out_ids_host, float *out_logprobs_host, void *stream);
+
+/* Force an execution path (CORAL_PATH_*) for later draft calls; AUTO restores the default choice. */
+int coral_lmhead_set_path(coral_lmhead_handle h, int path);
+
+/*
+ * Synchronise `stream`, return the device status word of the handle (CORAL_OK,
+ * CORAL_ERR_TIMEOUT, CORAL_ERR_BOUNDS) and clear it.
+ */
+int coral_lmhead_status(coral_lmhead_handle h, void *stream);
+
+/*
+ * Facts about the last draft call (Appendix B: in tree decoding all the groups
+ * involved by any candidate are activated; groups_touched is that union).
+ * Synchronises `stream` to read the union size back.
+ */
+int coral_lmhead_last_stats(coral_lmhead_handle h, coral_lmhead_stats *out, void *stream);
+
+/* Static, NUL-terminated description of a status code. */
+const char *coral_lmhead_error_string(int code);
+
+/* Free what the library allocated.  NULL is accepted. */
+int coral_lmhead_destroy(coral_lmhead_handle h);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CORAL_LMHEAD_H_ */

@@ -1,0 +1,87 @@
+// Shared device helpers for the grouped LM-head kernels (sm_100a).
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace coral {
+
+constexpr int kTileRows = 128;        // vocab rows per work tile
+constexpr int kMaxKTokens = 32;       // CORAL_MAX_K_TOKENS
+constexpr int kMaxGroups = 256;       // CORAL_MAX_GROUPS
+constexpr float kNegInf = -__builtin_huge_valf();
+constexpr int kNoToken = 0x7fffffff;
+
+// Device-resident per-handle state written by the kernels.
+struct DeviceState {
+    int status;        // 0 or a CORAL_ERR_* code (first error wins)
+    int n_union;       // groups touched by the last call
+};
+
+// Per-call view of the workspace handed to the kernels.
+struct CallView {
+    int M, H, V, N, v, T;          // T = tiles per group = ceil(v / kTileRows)
+    int k_groups, k_tokens;
+    const uint16_t* packed;        // [N][v][H] bf16, group-contiguous
+    const uint16_t* w_gate;        // [N][H] bf16
+    const int32_t* group_tokens;   // [N][v] global token id of packed row
+    const uint16_t* hidden;        // [M][H] bf16
+    float* gate;                   // [M][N]
+    int32_t* sel;                  // [M][k_groups]
+    int16_t* slot_of;              // [M][N] slot of group n in row m, -1 if not selected
+    int32_t* group_count;          // [N]
+    int32_t* group_offset;         // [N+1]
+    int32_t* bucket_row;           // [M*k_groups] rows that selected a group, ascending per group
+    int32_t* bucket_slot;          // [M*k_groups] the slot the group has in that row
+    float* part_max;               // [M][k_groups][T]
+    float* part_sum;               // [M][k_groups][T]
+    float* part_val;               // [M][k_groups][T][k_tokens]
+    int32_t* part_id;              // [M][k_groups][T][k_tokens]
+    DeviceState* state;
+};
+
+__device__ __forceinline__ float bf16_lo(uint32_t u) { return __uint_as_float(u << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t u) { return __uint_as_float(u & 0xffff0000u); }
+
+// fp32 dot product of 8 bf16 pairs held in two 128-bit words.
+__device__ __forceinline__ float dot8(const uint4& a, const uint4& b, float acc) {
+    acc = fmaf(bf16_lo(a.x), bf16_lo(b.x), acc);
+    acc = fmaf(bf16_hi(a.x), bf16_hi(b.x), acc);
+    acc = fmaf(bf16_lo(a.y), bf16_lo(b.y), acc);
+    acc = fmaf(bf16_hi(a.y), bf16_hi(b.y), acc);
+    acc = fmaf(bf16_lo(a.z), bf16_lo(b.z), acc);
+    acc = fmaf(bf16_hi(a.z), bf16_hi(b.z), acc);
+    acc = fmaf(bf16_lo(a.w), bf16_lo(b.w), acc);
+    acc = fmaf(bf16_hi(a.w), bf16_hi(b.w), acc);
+    return acc;
+}
+
+__device__ __forceinline__ float warp_sum(float x) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
+    return x;
+}
+
+__device__ __forceinline__ float warp_max(float x) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) x = fmaxf(x, __shfl_xor_sync(0xffffffffu, x, o));
+    return x;
+}
+
+// Order used everywhere: larger value first, equal values -> smaller key first.
+__device__ __forceinline__ bool better(float va, int ka, float vb, int kb) {
+    return va > vb || (va == vb && ka < kb);
+}
+
+// All lanes receive the best (value, key) pair of the warp.
+__device__ __forceinline__ void warp_argbest(float& v, int& k) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        float ov = __shfl_xor_sync(0xffffffffu, v, o);
+        int ok = __shfl_xor_sync(0xffffffffu, k, o);
+        if (better(ov, ok, v, k)) { v = ov; k = ok; }
+    }
+}
+
+__device__ __forceinline__ void set_status(DeviceState* st, int code) { atomicCAS(&st->status, 0, code); }
+
+}  // namespace coral

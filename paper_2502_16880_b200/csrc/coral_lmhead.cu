@@ -1,0 +1,332 @@
+// C ABI of the grouped LM-head draft step: handle management, argument checks,
+// workspace layout and kernel launches.  See include/coral_lmhead.h.
+#include "coral_lmhead.h"
+
+#include <cuda_runtime.h>
+
+#include <new>
+#include <vector>
+
+#include "common.cuh"
+#include "head_simt.cuh"
+#include "merge.cuh"
+#include "route.cuh"
+
+using namespace coral;
+
+namespace {
+
+constexpr size_t kAlign = 256;
+inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
+
+// Offsets of the workspace sections (bytes from the workspace base).
+struct Layout {
+    size_t w_gate, group_tokens, state, gate, sel, slot_of, group_count, group_offset, bucket_row, bucket_slot,
+        part_max, part_sum, part_val, part_id, stage_hidden, stage_ids, stage_logprobs, total;
+    size_t packed_bytes;
+    int v, T;
+};
+
+bool config_ok(const coral_lmhead_config* c) {
+    if (!c || c->struct_size != sizeof(coral_lmhead_config)) return false;
+    if (c->H < 8 || c->H % 8 != 0 || c->V < 1 || c->n_groups < 1 || c->n_groups > CORAL_MAX_GROUPS) return false;
+    if (c->V % c->n_groups != 0) return false;
+    if (c->max_M < 1 || c->max_k_groups < 1 || c->max_k_groups > c->n_groups) return false;
+    if (c->max_k_tokens < 1 || c->max_k_tokens > CORAL_MAX_K_TOKENS) return false;
+    return true;
+}
+
+Layout make_layout(const coral_lmhead_config& c) {
+    Layout L{};
+    L.v = c.V / c.n_groups;
+    L.T = (L.v + kTileRows - 1) / kTileRows;
+    const size_t M = c.max_M, N = c.n_groups, H = c.H, kg = c.max_k_groups, kt = c.max_k_tokens, T = L.T;
+    size_t o = 0;
+    auto take = [&](size_t bytes) { size_t at = o; o = align_up(o + bytes); return at; };
+    L.w_gate = take(N * H * 2);
+    L.group_tokens = take((size_t)c.V * 4);
+    L.state = take(sizeof(DeviceState));
+    L.gate = take(M * N * 4);
+    L.sel = take(M * kg * 4);
+    L.slot_of = take(M * N * 2);
+    L.group_count = take(N * 4);
+    L.group_offset = take((N + 1) * 4);
+    L.bucket_row = take(M * kg * 4);
+    L.bucket_slot = take(M * kg * 4);
+    L.part_max = take(M * kg * T * 4);
+    L.part_sum = take(M * kg * T * 4);
+    L.part_val = take(M * kg * T * kt * 4);
+    L.part_id = take(M * kg * T * kt * 4);
+    L.stage_hidden = take(M * H * 2);
+    L.stage_ids = take(M * kt * 4);
+    L.stage_logprobs = take(M * kt * 4);
+    L.total = o;
+    L.packed_bytes = (size_t)c.V * H * 2;
+    return L;
+}
+
+// packed[n][i][:] = W_vocab[group_tokens[n][i]][:]; one block per packed row.
+__global__ void pack_rows_kernel(const uint16_t* __restrict__ W, const int32_t* __restrict__ group_tokens,
+                                 uint16_t* __restrict__ packed, int H) {
+    const size_t row = blockIdx.x;
+    const uint4* src = reinterpret_cast<const uint4*>(W + (size_t)group_tokens[row] * H);
+    uint4* dst = reinterpret_cast<uint4*>(packed + row * H);
+    for (int ch = threadIdx.x; ch < (H >> 3); ch += blockDim.x) dst[ch] = __ldg(src + ch);
+}
+
+}  // namespace
+
+struct coral_lmhead_s {
+    coral_lmhead_config cfg;
+    Layout L;
+    unsigned char* packed;
+    unsigned char* ws;
+    bool own_packed, own_ws;
+    int forced_path;
+    int simt_smem;
+    // facts about the last draft call
+    int last_path, last_M, last_kg, last_kt, last_launches;
+};
+
+namespace {
+
+CallView make_view(const coral_lmhead_s* h, const void* hidden, int M, int kg, int kt) {
+    CallView c{};
+    const Layout& L = h->L;
+    unsigned char* ws = h->ws;
+    c.M = M; c.H = h->cfg.H; c.V = h->cfg.V; c.N = h->cfg.n_groups; c.v = L.v; c.T = L.T;
+    c.k_groups = kg; c.k_tokens = kt;
+    c.packed = reinterpret_cast<const uint16_t*>(h->packed);
+    c.w_gate = reinterpret_cast<const uint16_t*>(ws + L.w_gate);
+    c.group_tokens = reinterpret_cast<const int32_t*>(ws + L.group_tokens);
+    c.hidden = reinterpret_cast<const uint16_t*>(hidden);
+    c.gate = reinterpret_cast<float*>(ws + L.gate);
+    c.sel = reinterpret_cast<int32_t*>(ws + L.sel);
+    c.slot_of = reinterpret_cast<int16_t*>(ws + L.slot_of);
+    c.group_count = reinterpret_cast<int32_t*>(ws + L.group_count);
+    c.group_offset = reinterpret_cast<int32_t*>(ws + L.group_offset);
+    c.bucket_row = reinterpret_cast<int32_t*>(ws + L.bucket_row);
+    c.bucket_slot = reinterpret_cast<int32_t*>(ws + L.bucket_slot);
+    c.part_max = reinterpret_cast<float*>(ws + L.part_max);
+    c.part_sum = reinterpret_cast<float*>(ws + L.part_sum);
+    c.part_val = reinterpret_cast<float*>(ws + L.part_val);
+    c.part_id = reinterpret_cast<int32_t*>(ws + L.part_id);
+    c.state = reinterpret_cast<DeviceState*>(ws + L.state);
+    return c;
+}
+
+int choose_path(const coral_lmhead_s* h, int M, int kg) {
+    (void)M; (void)kg;
+    if (h->forced_path != CORAL_PATH_AUTO) return h->forced_path;
+    return CORAL_PATH_SIMT;
+}
+
+}  // namespace
+
+extern "C" {
+
+int coral_lmhead_version(void) { return CORAL_LMHEAD_ABI_VERSION; }
+
+const char* coral_lmhead_error_string(int code) {
+    switch (code) {
+        case CORAL_OK: return "ok";
+        case CORAL_ERR_INVALID: return "invalid argument";
+        case CORAL_ERR_GROUPING: return "group_map does not split the vocabulary into equal groups";
+        case CORAL_ERR_CUDA: return "CUDA runtime error";
+        case CORAL_ERR_NOMEM: return "out of memory";
+        case CORAL_ERR_TIMEOUT: return "device-side wait timed out";
+        case CORAL_ERR_BOUNDS: return "device-side index check failed";
+        default: return "unknown status";
+    }
+}
+
+int coral_lmhead_query_sizes(const coral_lmhead_config* cfg, size_t* packed_bytes, size_t* workspace_bytes) {
+    if (!config_ok(cfg) || !packed_bytes || !workspace_bytes) return CORAL_ERR_INVALID;
+    const Layout L = make_layout(*cfg);
+    *packed_bytes = L.packed_bytes;
+    *workspace_bytes = L.total;
+    return CORAL_OK;
+}
+
+int coral_lmhead_create(coral_lmhead_handle* out, const coral_lmhead_config* cfg, const void* W_vocab_dev,
+                        const int32_t* group_map_host, const void* W_gate_dev, void* packed_buf_dev,
+                        void* workspace_dev, void* stream) {
+    if (!out) return CORAL_ERR_INVALID;
+    *out = nullptr;
+    if (!config_ok(cfg) || !W_vocab_dev || !group_map_host || !W_gate_dev) return CORAL_ERR_INVALID;
+    if ((reinterpret_cast<uintptr_t>(W_vocab_dev) & 15) || (reinterpret_cast<uintptr_t>(W_gate_dev) & 15) ||
+        (reinterpret_cast<uintptr_t>(packed_buf_dev) & (kAlign - 1)) ||
+        (reinterpret_cast<uintptr_t>(workspace_dev) & (kAlign - 1)))
+        return CORAL_ERR_INVALID;
+    const int N = cfg->n_groups, V = cfg->V, v = V / N;
+
+    // token -> group must be in range and split V into N equal groups (Section 3.3)
+    std::vector<int32_t> group_tokens;
+    std::vector<int32_t> fill;
+    try {
+        group_tokens.resize((size_t)V);
+        fill.assign((size_t)N, 0);
+    } catch (const std::bad_alloc&) {
+        return CORAL_ERR_NOMEM;
+    }
+    for (int x = 0; x < V; ++x) {
+        const int g = group_map_host[x];
+        if (g < 0 || g >= N) return CORAL_ERR_INVALID;
+        if (fill[g] >= v) return CORAL_ERR_GROUPING;
+        group_tokens[(size_t)g * v + fill[g]++] = x;   // ascending token id inside a group
+    }
+    for (int n = 0; n < N; ++n)
+        if (fill[n] != v) return CORAL_ERR_GROUPING;
+
+    coral_lmhead_s* h = new (std::nothrow) coral_lmhead_s();
+    if (!h) return CORAL_ERR_NOMEM;
+    h->cfg = *cfg;
+    h->L = make_layout(*cfg);
+    h->forced_path = CORAL_PATH_AUTO;
+    h->packed = static_cast<unsigned char*>(packed_buf_dev);
+    h->ws = static_cast<unsigned char*>(workspace_dev);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int rc = CORAL_OK;
+    do {
+        if (!h->packed) {
+            if (cudaMalloc(&h->packed, h->L.packed_bytes) != cudaSuccess) { h->packed = nullptr; rc = CORAL_ERR_NOMEM; break; }
+            h->own_packed = true;
+        }
+        if (!h->ws) {
+            if (cudaMalloc(&h->ws, h->L.total) != cudaSuccess) { h->ws = nullptr; rc = CORAL_ERR_NOMEM; break; }
+            h->own_ws = true;
+        }
+        h->simt_smem = kSimtRowBlock * cfg->H * 2 + kSimtRowBlock * kTileRows * 4;
+        // The attribute is per kernel, not per handle: always raise it to the device's opt-in limit.
+        int dev = 0, smem_optin = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess) {
+            rc = CORAL_ERR_CUDA; break;
+        }
+        if (h->simt_smem > smem_optin) { rc = CORAL_ERR_INVALID; break; }
+        if (cudaFuncSetAttribute(head_simt_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_optin) !=
+            cudaSuccess) { rc = CORAL_ERR_CUDA; break; }
+        if (cudaMemcpyAsync(h->ws + h->L.group_tokens, group_tokens.data(), (size_t)V * 4, cudaMemcpyHostToDevice, st) !=
+            cudaSuccess) { rc = CORAL_ERR_CUDA; break; }
+        if (cudaMemcpyAsync(h->ws + h->L.w_gate, W_gate_dev, (size_t)N * cfg->H * 2, cudaMemcpyDeviceToDevice, st) !=
+            cudaSuccess) { rc = CORAL_ERR_CUDA; break; }
+        if (cudaMemsetAsync(h->ws + h->L.state, 0, sizeof(DeviceState), st) != cudaSuccess) { rc = CORAL_ERR_CUDA; break; }
+        pack_rows_kernel<<<V, 128, 0, st>>>(static_cast<const uint16_t*>(W_vocab_dev),
+                                            reinterpret_cast<const int32_t*>(h->ws + h->L.group_tokens),
+                                            reinterpret_cast<uint16_t*>(h->packed), cfg->H);
+        if (cudaGetLastError() != cudaSuccess) { rc = CORAL_ERR_CUDA; break; }
+        if (cudaStreamSynchronize(st) != cudaSuccess) { rc = CORAL_ERR_CUDA; break; }
+    } while (0);
+    if (rc != CORAL_OK) {
+        coral_lmhead_destroy(h);
+        return rc;
+    }
+    *out = h;
+    return CORAL_OK;
+}
+
+int coral_lmhead_destroy(coral_lmhead_handle h) {
+    if (!h) return CORAL_OK;
+    if (h->own_packed && h->packed) cudaFree(h->packed);
+    if (h->own_ws && h->ws) cudaFree(h->ws);
+    delete h;
+    return CORAL_OK;
+}
+
+int coral_lmhead_set_path(coral_lmhead_handle h, int path) {
+    if (!h || path < CORAL_PATH_AUTO || path > CORAL_PATH_TCGEN05) return CORAL_ERR_INVALID;
+    if (path == CORAL_PATH_TCGEN05) return CORAL_ERR_INVALID;   // not built yet
+    h->forced_path = path;
+    return CORAL_OK;
+}
+
+int coral_lmhead_draft_ex(coral_lmhead_handle h, const void* hidden_dev, int M, int k_groups, int k_tokens,
+                          const int32_t* forced_groups_dev, int32_t* out_groups_dev, float* out_gate_dev,
+                          float* out_logits_dev, float* out_lse_dev, int32_t* out_ids_dev, float* out_logprobs_dev,
+                          void* stream) {
+    if (!h || !hidden_dev || !out_ids_dev || !out_logprobs_dev) return CORAL_ERR_INVALID;
+    if (reinterpret_cast<uintptr_t>(hidden_dev) & 15) return CORAL_ERR_INVALID;
+    const coral_lmhead_config& cfg = h->cfg;
+    if (M < 1 || M > cfg.max_M) return CORAL_ERR_INVALID;
+    if (k_groups < 1 || k_groups > cfg.max_k_groups) return CORAL_ERR_INVALID;
+    if (k_tokens < 1 || k_tokens > cfg.max_k_tokens || (long long)k_tokens > (long long)k_groups * h->L.v)
+        return CORAL_ERR_INVALID;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const CallView c = make_view(h, hidden_dev, M, k_groups, k_tokens);
+    const int path = choose_path(h, M, k_groups);
+    int launches = 0;
+
+    gate_kernel<<<dim3(c.N, (M + kGateRows - 1) / kGateRows), kGateThreads, 0, st>>>(c, out_gate_dev);
+    ++launches;
+    select_kernel<<<(M + kSelectWarps - 1) / kSelectWarps, kSelectWarps * 32, 0, st>>>(c, forced_groups_dev,
+                                                                                      out_groups_dev);
+    ++launches;
+    bucket_kernel<<<1, kBucketThreads, 0, st>>>(c);
+    ++launches;
+    head_simt_kernel<<<dim3(c.T, c.N), kSimtThreads, h->simt_smem, st>>>(c, out_logits_dev);
+    ++launches;
+    merge_kernel<<<M, kMergeThreads, 0, st>>>(c, out_ids_dev, out_logprobs_dev, out_lse_dev);
+    ++launches;
+    if (cudaGetLastError() != cudaSuccess) return CORAL_ERR_CUDA;
+
+    h->last_path = path; h->last_M = M; h->last_kg = k_groups; h->last_kt = k_tokens; h->last_launches = launches;
+    return CORAL_OK;
+}
+
+int coral_lmhead_draft(coral_lmhead_handle h, const void* hidden_dev, int M, int k_groups, int k_tokens,
+                       int32_t* out_ids_dev, float* out_logprobs_dev, void* stream) {
+    return coral_lmhead_draft_ex(h, hidden_dev, M, k_groups, k_tokens, nullptr, nullptr, nullptr, nullptr, nullptr,
+                                 out_ids_dev, out_logprobs_dev, stream);
+}
+
+int coral_lmhead_draft_host(coral_lmhead_handle h, const void* hidden_host, int M, int k_groups, int k_tokens,
+                            int32_t* out_ids_host, float* out_logprobs_host, void* stream) {
+    if (!h || !hidden_host || !out_ids_host || !out_logprobs_host) return CORAL_ERR_INVALID;
+    if (M < 1 || M > h->cfg.max_M || k_tokens < 1 || k_tokens > h->cfg.max_k_tokens) return CORAL_ERR_INVALID;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    unsigned char* ws = h->ws;
+    void* d_hidden = ws + h->L.stage_hidden;
+    int32_t* d_ids = reinterpret_cast<int32_t*>(ws + h->L.stage_ids);
+    float* d_lp = reinterpret_cast<float*>(ws + h->L.stage_logprobs);
+    if (cudaMemcpyAsync(d_hidden, hidden_host, (size_t)M * h->cfg.H * 2, cudaMemcpyHostToDevice, st) != cudaSuccess)
+        return CORAL_ERR_CUDA;
+    const int rc = coral_lmhead_draft(h, d_hidden, M, k_groups, k_tokens, d_ids, d_lp, stream);
+    if (rc != CORAL_OK) return rc;
+    if (cudaMemcpyAsync(out_ids_host, d_ids, (size_t)M * k_tokens * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        return CORAL_ERR_CUDA;
+    if (cudaMemcpyAsync(out_logprobs_host, d_lp, (size_t)M * k_tokens * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        return CORAL_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return CORAL_ERR_CUDA;
+    return CORAL_OK;
+}
+
+int coral_lmhead_status(coral_lmhead_handle h, void* stream) {
+    if (!h) return CORAL_ERR_INVALID;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    DeviceState s{};
+    DeviceState* d = reinterpret_cast<DeviceState*>(h->ws + h->L.state);
+    if (cudaMemcpyAsync(&s, d, sizeof s, cudaMemcpyDeviceToHost, st) != cudaSuccess) return CORAL_ERR_CUDA;
+    if (cudaMemsetAsync(&d->status, 0, sizeof(int), st) != cudaSuccess) return CORAL_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return CORAL_ERR_CUDA;
+    return s.status;
+}
+
+int coral_lmhead_last_stats(coral_lmhead_handle h, coral_lmhead_stats* out, void* stream) {
+    if (!h || !out) return CORAL_ERR_INVALID;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    DeviceState s{};
+    if (cudaMemcpyAsync(&s, h->ws + h->L.state, sizeof s, cudaMemcpyDeviceToHost, st) != cudaSuccess) return CORAL_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return CORAL_ERR_CUDA;
+    out->path = h->last_path;
+    out->M = h->last_M;
+    out->k_groups = h->last_kg;
+    out->k_tokens = h->last_kt;
+    out->groups_touched = s.n_union;
+    out->kernel_launches = h->last_launches;
+    out->weight_bytes = (int64_t)s.n_union * h->L.v * h->cfg.H * 2;
+    out->algorithmic_bytes = out->weight_bytes + (int64_t)h->cfg.n_groups * h->cfg.H * 2 +
+                             (int64_t)h->last_M * h->cfg.H * 2 + (int64_t)h->last_M * h->last_kt * 8;
+    return CORAL_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,245 @@
+"""Thin ctypes binding of the C ABI in include/coral_lmhead.h.
+
+Argument marshalling only: every step of the draft path runs in the CUDA
+library.  torch is used for device memory and streams.  There is no CPU
+fallback: if the compiled library is missing, loading fails with an error.
+The function names are those of the C ABI; `LMHead` is a small convenience
+wrapper that owns the device buffers.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libcoral_lmhead.so")
+
+CORAL_OK = 0
+CORAL_ERR_INVALID = -1
+CORAL_ERR_GROUPING = -2
+CORAL_ERR_CUDA = -3
+CORAL_ERR_NOMEM = -4
+CORAL_ERR_TIMEOUT = -5
+CORAL_ERR_BOUNDS = -6
+CORAL_PATH_AUTO, CORAL_PATH_SIMT, CORAL_PATH_TCGEN05 = 0, 1, 2
+
+
+class coral_lmhead_config(ctypes.Structure):
+    _fields_ = [("struct_size", ctypes.c_uint32), ("H", ctypes.c_int32), ("V", ctypes.c_int32),
+                ("n_groups", ctypes.c_int32), ("max_M", ctypes.c_int32), ("max_k_groups", ctypes.c_int32),
+                ("max_k_tokens", ctypes.c_int32), ("flags", ctypes.c_uint32)]
+
+
+class coral_lmhead_stats(ctypes.Structure):
+    _fields_ = [("path", ctypes.c_int32), ("M", ctypes.c_int32), ("k_groups", ctypes.c_int32),
+                ("k_tokens", ctypes.c_int32), ("groups_touched", ctypes.c_int32),
+                ("kernel_launches", ctypes.c_int32), ("weight_bytes", ctypes.c_int64),
+                ("algorithmic_bytes", ctypes.c_int64)]
+
+
+_lib = None
+_vp, _i = ctypes.c_void_p, ctypes.c_int
+
+_SIGNATURES = {
+    "coral_lmhead_version": (_i, []),
+    "coral_lmhead_query_sizes": (_i, [ctypes.POINTER(coral_lmhead_config), ctypes.POINTER(ctypes.c_size_t),
+                                      ctypes.POINTER(ctypes.c_size_t)]),
+    "coral_lmhead_create": (_i, [ctypes.POINTER(_vp), ctypes.POINTER(coral_lmhead_config), _vp, _vp, _vp, _vp, _vp, _vp]),
+    "coral_lmhead_draft": (_i, [_vp, _vp, _i, _i, _i, _vp, _vp, _vp]),
+    "coral_lmhead_draft_ex": (_i, [_vp, _vp, _i, _i, _i, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
+    "coral_lmhead_draft_host": (_i, [_vp, _vp, _i, _i, _i, _vp, _vp, _vp]),
+    "coral_lmhead_set_path": (_i, [_vp, _i]),
+    "coral_lmhead_status": (_i, [_vp, _vp]),
+    "coral_lmhead_last_stats": (_i, [_vp, ctypes.POINTER(coral_lmhead_stats), _vp]),
+    "coral_lmhead_error_string": (ctypes.c_char_p, [_i]),
+    "coral_lmhead_destroy": (_i, [_vp]),
+}
+
+
+def load_library(path: str = LIB_PATH):
+    """Load the compiled CUDA library.  Raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(path):
+            raise RuntimeError(
+                f"{path} is missing: build it with `python -m paper_2502_16880_b200.build` "
+                "(nvcc, sm_100a). There is no fallback path.")
+        lib = ctypes.CDLL(path)
+        for name, (res, args) in _SIGNATURES.items():
+            fn = getattr(lib, name)
+            fn.restype, fn.argtypes = res, args
+        _lib = lib
+    return _lib
+
+
+class CoralError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {coral_lmhead_error_string(code)} ({code})")
+
+
+def _check(code: int, where: str) -> None:
+    if code != CORAL_OK:
+        raise CoralError(code, where)
+
+
+def _dev_ptr(t, dtype=None, allow_none=True):
+    if t is None:
+        if allow_none:
+            return None
+        raise ValueError("tensor required")
+    if not t.is_cuda or not t.is_contiguous():
+        raise ValueError("expected a contiguous CUDA tensor")
+    if dtype is not None and t.dtype != dtype:
+        raise ValueError(f"expected dtype {dtype}, got {t.dtype}")
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def _stream_ptr(stream):
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return ctypes.c_void_p(stream.cuda_stream)
+
+
+def make_config(H, V, n_groups, max_M, max_k_groups, max_k_tokens) -> coral_lmhead_config:
+    return coral_lmhead_config(ctypes.sizeof(coral_lmhead_config), H, V, n_groups, max_M, max_k_groups,
+                               max_k_tokens, 0)
+
+
+# ---- functions named as in the C ABI -------------------------------------------------
+def coral_lmhead_version() -> int:
+    return int(load_library().coral_lmhead_version())
+
+
+def coral_lmhead_error_string(code: int) -> str:
+    return load_library().coral_lmhead_error_string(int(code)).decode()
+
+
+def coral_lmhead_query_sizes(cfg: coral_lmhead_config):
+    pb, wb = ctypes.c_size_t(0), ctypes.c_size_t(0)
+    _check(load_library().coral_lmhead_query_sizes(ctypes.byref(cfg), ctypes.byref(pb), ctypes.byref(wb)),
+           "coral_lmhead_query_sizes")
+    return int(pb.value), int(wb.value)
+
+
+def coral_lmhead_create(cfg, W_vocab, group_map_host, W_gate, packed_buf=None, workspace=None, stream=None):
+    """W_vocab/W_gate: CUDA bf16 tensors; group_map_host: CPU int32 tensor [V]. Returns an opaque handle."""
+    if group_map_host.is_cuda or group_map_host.dtype != torch.int32 or not group_map_host.is_contiguous():
+        raise ValueError("group_map_host must be a contiguous CPU int32 tensor")
+    if group_map_host.numel() != cfg.V:
+        raise ValueError("group_map_host must have V entries")
+    h = ctypes.c_void_p()
+    _check(load_library().coral_lmhead_create(
+        ctypes.byref(h), ctypes.byref(cfg), _dev_ptr(W_vocab, torch.bfloat16, False),
+        ctypes.c_void_p(group_map_host.data_ptr()), _dev_ptr(W_gate, torch.bfloat16, False),
+        _dev_ptr(packed_buf), _dev_ptr(workspace), _stream_ptr(stream)), "coral_lmhead_create")
+    return h
+
+
+def coral_lmhead_draft(handle, hidden, k_groups, k_tokens, out_ids, out_logprobs, stream=None):
+    M = hidden.shape[0]
+    _check(load_library().coral_lmhead_draft(
+        handle, _dev_ptr(hidden, torch.bfloat16, False), M, int(k_groups), int(k_tokens),
+        _dev_ptr(out_ids, torch.int32, False), _dev_ptr(out_logprobs, torch.float32, False), _stream_ptr(stream)),
+        "coral_lmhead_draft")
+
+
+def coral_lmhead_draft_ex(handle, hidden, k_groups, k_tokens, out_ids, out_logprobs, forced_groups=None,
+                          out_groups=None, out_gate=None, out_logits=None, out_lse=None, stream=None):
+    M = hidden.shape[0]
+    _check(load_library().coral_lmhead_draft_ex(
+        handle, _dev_ptr(hidden, torch.bfloat16, False), M, int(k_groups), int(k_tokens),
+        _dev_ptr(forced_groups, torch.int32), _dev_ptr(out_groups, torch.int32), _dev_ptr(out_gate, torch.float32),
+        _dev_ptr(out_logits, torch.float32), _dev_ptr(out_lse, torch.float32),
+        _dev_ptr(out_ids, torch.int32, False), _dev_ptr(out_logprobs, torch.float32, False), _stream_ptr(stream)),
+        "coral_lmhead_draft_ex")
+
+
+def coral_lmhead_draft_host(handle, hidden_host, k_groups, k_tokens, out_ids_host, out_logprobs_host, stream=None):
+    """Host (ideally pinned) buffers in and out; returns after the results are in host memory."""
+    for t in (hidden_host, out_ids_host, out_logprobs_host):
+        if t.is_cuda or not t.is_contiguous():
+            raise ValueError("expected contiguous CPU tensors")
+    M = hidden_host.shape[0]
+    _check(load_library().coral_lmhead_draft_host(
+        handle, ctypes.c_void_p(hidden_host.data_ptr()), M, int(k_groups), int(k_tokens),
+        ctypes.c_void_p(out_ids_host.data_ptr()), ctypes.c_void_p(out_logprobs_host.data_ptr()),
+        _stream_ptr(stream)), "coral_lmhead_draft_host")
+
+
+def coral_lmhead_set_path(handle, path: int) -> None:
+    _check(load_library().coral_lmhead_set_path(handle, int(path)), "coral_lmhead_set_path")
+
+
+def coral_lmhead_status(handle, stream=None) -> int:
+    return int(load_library().coral_lmhead_status(handle, _stream_ptr(stream)))
+
+
+def coral_lmhead_last_stats(handle, stream=None) -> coral_lmhead_stats:
+    s = coral_lmhead_stats()
+    _check(load_library().coral_lmhead_last_stats(handle, ctypes.byref(s), _stream_ptr(stream)),
+           "coral_lmhead_last_stats")
+    return s
+
+
+def coral_lmhead_destroy(handle) -> None:
+    _check(load_library().coral_lmhead_destroy(handle), "coral_lmhead_destroy")
+
+
+# ---- convenience wrapper ---------------------------------------------------------------
+class LMHead:
+    """Owns the packed weights and workspace (torch allocations) of one handle."""
+
+    def __init__(self, W_vocab, group_map_host, W_gate, max_M, max_k_groups, max_k_tokens=10):
+        V, H = W_vocab.shape
+        N = W_gate.shape[0]
+        self.cfg = make_config(H, V, N, max_M, max_k_groups, max_k_tokens)
+        pb, wb = coral_lmhead_query_sizes(self.cfg)
+        dev = W_vocab.device
+        self.packed = torch.empty(pb, dtype=torch.uint8, device=dev)
+        self.workspace = torch.empty(wb, dtype=torch.uint8, device=dev)
+        self.handle = coral_lmhead_create(self.cfg, W_vocab, group_map_host, W_gate, self.packed, self.workspace)
+        self.device = dev
+
+    def draft(self, hidden, k_groups, k_tokens, taps=False, forced_groups=None, stream=None):
+        M = hidden.shape[0]
+        dev = self.device
+        ids = torch.empty((M, k_tokens), dtype=torch.int32, device=dev)
+        lps = torch.empty((M, k_tokens), dtype=torch.float32, device=dev)
+        if not taps and forced_groups is None:
+            coral_lmhead_draft(self.handle, hidden, k_groups, k_tokens, ids, lps, stream)
+            return ids, lps
+        v = self.cfg.V // self.cfg.n_groups
+        out = {
+            "groups": torch.empty((M, k_groups), dtype=torch.int32, device=dev),
+            "gate": torch.empty((M, self.cfg.n_groups), dtype=torch.float32, device=dev),
+            "logits": torch.empty((M, k_groups, v), dtype=torch.float32, device=dev),
+            "lse": torch.empty((M,), dtype=torch.float32, device=dev),
+        }
+        coral_lmhead_draft_ex(self.handle, hidden, k_groups, k_tokens, ids, lps, forced_groups=forced_groups,
+                              out_groups=out["groups"], out_gate=out["gate"], out_logits=out["logits"],
+                              out_lse=out["lse"], stream=stream)
+        out["ids"], out["logprobs"] = ids, lps
+        return out
+
+    def set_path(self, path):
+        coral_lmhead_set_path(self.handle, path)
+
+    def status(self):
+        return coral_lmhead_status(self.handle)
+
+    def stats(self):
+        return coral_lmhead_last_stats(self.handle)
+
+    def close(self):
+        if self.handle is not None:
+            coral_lmhead_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

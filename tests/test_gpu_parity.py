@@ -1,0 +1,183 @@
+"""GPU parity: the CUDA path through the C ABI against the CPU oracle."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2502_16880_b200 import lmhead, synth
+from tests import parity_harness as ph
+
+pytestmark = pytest.mark.gpu
+
+PATHS = [lmhead.CORAL_PATH_SIMT]
+
+
+def _head(cfg, W, gm, Wg, max_M=None, max_kg=None, max_kt=None):
+    return lmhead.LMHead(ph.to_dev_bf16(W), torch.from_numpy(gm), ph.to_dev_bf16(Wg),
+                         max_M or cfg.M, max_kg or cfg.N, max_kt or 32)
+
+
+_cache = {}
+
+
+def _weights(name):
+    """Weights are expensive to draw at the Llama3/Qwen shapes: one set per config per session."""
+    if name not in _cache:
+        _cache.clear()
+        cfg = synth.CONFIGS[name]
+        W, gm, Wg = synth.make_w_vocab(cfg), synth.make_group_map(cfg), synth.make_w_gate(cfg)
+        _cache[name] = (cfg, W, gm, Wg, _head(cfg, W, gm, Wg, max_M=max(cfg.M, 64)))
+    return _cache[name]
+
+
+def _check(head, W, gm, Wg, hb, kg, kt, path, forced=None):
+    head.set_path(path)
+    out = ph.gpu_draft_numpy(head, hb, kg, kt, forced_groups=forced)
+    assert head.status() == 0
+    rep = ph.compare(W, gm, Wg, hb, kg, kt, out, forced_groups=forced)
+    assert rep.ok, rep.errors
+    return rep, out
+
+
+@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("M,kg,kt", [(4, 4, 10), (1, 1, 1), (1, 4, 10), (3, 16, 32), (16, 2, 10), (40, 16, 7)])
+def test_tiny(path, M, kg, kt):
+    cfg, W, gm, Wg, head = _weights("tiny")
+    hb = synth.make_hidden(cfg, M)
+    rep, out = _check(head, W, gm, Wg, hb, kg, kt, path)
+    st = head.stats()
+    assert st.groups_touched == len(set(out["groups"].ravel().tolist()))
+    assert st.weight_bytes == st.groups_touched * cfg.v * cfg.H * 2
+
+
+@pytest.mark.parametrize("path", PATHS)
+def test_ragged_shape(path):
+    # v = 300 (two full tiles + a tail of 44), H = 328 (not a multiple of 256)
+    cfg = synth.HeadConfig("ragged", H=328, V=1800, N=6, k_groups=3, k_tokens=10, M=13, seed=5, w_std=0.05)
+    W, gm, Wg, hb = synth.make_all(cfg)
+    head = _head(cfg, W, gm, Wg)
+    for kg, kt in [(3, 10), (6, 32), (1, 5)]:
+        _check(head, W, gm, Wg, hb, kg, kt, path)
+    head.close()
+
+
+@pytest.mark.parametrize("path", PATHS)
+def test_small_group_fewer_rows_than_k_tokens(path):
+    # v = 6 < k_tokens: per-tile candidate lists are padded
+    cfg = synth.HeadConfig("small_v", H=64, V=48, N=8, k_groups=4, k_tokens=20, M=5, seed=9, w_std=0.3)
+    W, gm, Wg, hb = synth.make_all(cfg)
+    head = _head(cfg, W, gm, Wg)
+    _check(head, W, gm, Wg, hb, 4, 20, path)
+    _check(head, W, gm, Wg, hb, 8, 32, path)
+    head.close()
+
+
+@pytest.mark.parametrize("path", PATHS)
+def test_forced_groups(path):
+    cfg, W, gm, Wg, head = _weights("tiny")
+    hb = synth.make_hidden(cfg, 5)
+    forced = np.tile(np.array([7, 0, 15], np.int32), (5, 1))
+    rep, out = _check(head, W, gm, Wg, hb, 3, 10, path, forced=forced)
+    assert np.array_equal(out["groups"], forced)
+
+
+@pytest.mark.parametrize("path", PATHS)
+def test_exact_ties_zero_weights(path):
+    cfg = synth.HeadConfig("zeros", H=64, V=640, N=5, k_groups=2, k_tokens=10, M=3, seed=1)
+    gm, hb = synth.make_group_map(cfg), synth.make_hidden(cfg)
+    W = np.zeros((cfg.V, cfg.H), np.uint16)
+    Wg = np.zeros((cfg.N, cfg.H), np.uint16)
+    head = _head(cfg, W, gm, Wg)
+    head.set_path(path)
+    out = ph.gpu_draft_numpy(head, hb, 2, 10)
+    assert out["groups"].tolist() == [[0, 1]] * cfg.M                 # equal scores -> lower index
+    assert out["ids"].tolist() == [np.flatnonzero(gm < 2)[:10].tolist()] * cfg.M   # equal logits -> lower id
+    np.testing.assert_allclose(out["logprobs"], -np.log(2 * cfg.v), atol=1e-5)
+    head.close()
+
+
+@pytest.mark.parametrize("path", PATHS)
+def test_deterministic_bitwise(path):
+    cfg, W, gm, Wg, head = _weights("tiny")
+    hb = synth.make_hidden(cfg, 33)
+    head.set_path(path)
+    a = ph.gpu_draft_numpy(head, hb, 4, 10)
+    b = ph.gpu_draft_numpy(head, hb, 4, 10)
+    for k in a:
+        assert np.array_equal(a[k], b[k]), k
+
+
+def test_argument_errors_return_codes():
+    cfg, W, gm, Wg, head = _weights("tiny")
+    h = ph.to_dev_bf16(synth.make_hidden(cfg, 4))
+    ids = torch.empty((4, 10), dtype=torch.int32, device="cuda")
+    lps = torch.empty((4, 10), dtype=torch.float32, device="cuda")
+    lib = lmhead.load_library()
+    import ctypes
+    hp, ip, lp = (ctypes.c_void_p(t.data_ptr()) for t in (h, ids, lps))
+    assert lib.coral_lmhead_draft(head.handle, hp, 0, 4, 10, ip, lp, None) == lmhead.CORAL_ERR_INVALID
+    assert lib.coral_lmhead_draft(head.handle, hp, 10 ** 6, 4, 10, ip, lp, None) == lmhead.CORAL_ERR_INVALID
+    assert lib.coral_lmhead_draft(head.handle, hp, 4, 0, 10, ip, lp, None) == lmhead.CORAL_ERR_INVALID
+    assert lib.coral_lmhead_draft(head.handle, hp, 4, cfg.N + 1, 10, ip, lp, None) == lmhead.CORAL_ERR_INVALID
+    assert lib.coral_lmhead_draft(head.handle, hp, 4, 4, 33, ip, lp, None) == lmhead.CORAL_ERR_INVALID
+    assert lib.coral_lmhead_draft(head.handle, None, 4, 4, 10, ip, lp, None) == lmhead.CORAL_ERR_INVALID
+    assert lib.coral_lmhead_draft(head.handle, hp, 4, 4, 10, None, lp, None) == lmhead.CORAL_ERR_INVALID
+    assert lib.coral_lmhead_draft(None, hp, 4, 4, 10, ip, lp, None) == lmhead.CORAL_ERR_INVALID
+    # unequal groups are rejected at create, before anything touches the device
+    bad = gm.copy()
+    bad[0] = (bad[0] + 1) % cfg.N
+    with pytest.raises(lmhead.CoralError) as e:
+        lmhead.LMHead(ph.to_dev_bf16(W), torch.from_numpy(bad), ph.to_dev_bf16(Wg), 4, 4, 10)
+    assert e.value.code == lmhead.CORAL_ERR_GROUPING
+    assert head.status() == 0
+
+
+def test_library_owned_buffers_and_host_entry():
+    cfg = synth.CONFIGS["tiny"]
+    W, gm, Wg, hb = synth.make_all(cfg)
+    c = lmhead.make_config(cfg.H, cfg.V, cfg.N, 8, cfg.N, 10)
+    handle = lmhead.coral_lmhead_create(c, ph.to_dev_bf16(W), torch.from_numpy(gm), ph.to_dev_bf16(Wg))
+    hh = torch.from_numpy(hb.view(np.int16)).pin_memory()
+    ids = torch.empty((cfg.M, 10), dtype=torch.int32).pin_memory()
+    lps = torch.empty((cfg.M, 10), dtype=torch.float32).pin_memory()
+    lmhead.coral_lmhead_draft_host(handle, hh, cfg.k_groups, 10, ids, lps)
+    rep = ph.compare(W, gm, Wg, hb, cfg.k_groups, 10, {"ids": ids.numpy(), "logprobs": lps.numpy()})
+    assert rep.ok, rep.errors
+    assert lmhead.coral_lmhead_status(handle) == 0
+    lmhead.coral_lmhead_destroy(handle)
+
+
+@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("name,Ms", [("llama2_7b", (1, 8, 60)), ("llama3_8b", (1, 8, 60))])
+def test_paper_shapes(path, name, Ms):
+    cfg, W, gm, Wg, head = _weights(name)
+    for M in Ms:
+        hb = synth.make_hidden(cfg, M)
+        head.set_path(path)
+        out = ph.gpu_draft_numpy(head, hb, cfg.k_groups, cfg.k_tokens)
+        assert head.status() == 0
+        # the oracle checks all rows for M <= 8 and a spread sample of rows beyond
+        rows = np.arange(M) if M <= 8 else np.unique(np.linspace(0, M - 1, 6).astype(int))
+        rep = ph.compare(W, gm, Wg, hb[rows], cfg.k_groups, cfg.k_tokens, {k: v[rows] for k, v in out.items()})
+        assert rep.ok, rep.errors
+        st = head.stats()
+        assert st.groups_touched == len(set(out["groups"].ravel().tolist()))
+
+
+@pytest.mark.parametrize("path", PATHS)
+def test_qwen_shape_group_sweep_and_dense_equivalence(path):
+    cfg, W, gm, Wg, head = _weights("qwen25_7b")
+    hb = synth.make_hidden(cfg, 60)
+    rows = np.array([0, 29, 59])
+    for kg in (2, 4, 8, 16, 64):
+        head.set_path(path)
+        out = ph.gpu_draft_numpy(head, hb, kg, cfg.k_tokens)
+        assert head.status() == 0
+        rep = ph.compare(W, gm, Wg, hb[rows], kg, cfg.k_tokens, {k: v[rows] for k, v in out.items()})
+        assert rep.ok, (kg, rep.errors)
+    # k_groups = N is the dense head: every row's ids/log-probs equal a dense log-softmax (library, fp32 on GPU)
+    Wd, hd = ph.to_dev_bf16(W), ph.to_dev_bf16(hb)
+    dense = torch.log_softmax((hd.float() @ Wd.float().T), dim=1)
+    top = torch.topk(dense, cfg.k_tokens, dim=1)
+    same = (top.indices.cpu().numpy() == out["ids"]).mean()
+    assert same > 0.99
+    np.testing.assert_allclose(out["logprobs"], top.values.cpu().numpy(), atol=2e-3)
