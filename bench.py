@@ -1,0 +1,355 @@
+#!/usr/bin/env python
+"""Benchmark of the grouped LM-head draft step on B200.
+
+One "step" is one draft call (gate -> top-k groups -> gathered GEMV of the
+selected groups -> log-sum-exp -> top-k tokens) over one batch of M query rows.
+Headline workload: the Llama3-8B-shaped draft head of the paper's Table 1
+(H=4096, V=128256) in 64 groups with the top 8 active (the N=64/top8 cell of
+its Table 4), M=8 tree-node rows, 10 candidates per row; seeded synthetic
+bf16 weights N(0, 0.02) and hidden states N(0, 1).
+
+value = algorithmic bytes of the step (bytes of the groups actually touched +
+gate + hidden + outputs) / step time, summed over ranks: achieved HBM GB/s.
+The same line carries the step latency, the dense head (all groups active and
+a torch matmul comparator), other M, the dominant kernel's roofline fraction,
+an end-to-end number through the host-buffer entry point, and the CPU oracle
+timed on the host cores.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "grouped LM-head draft-step HBM GB/s (algorithmic bytes of touched groups / step time)"
+UNIT = "GB/s"
+WORKLOAD = "llama3_8b"
+N_BATCHES = 8            # distinct hidden batches rotated through the steps
+FLUSH_BYTES = 512 << 20  # > 2x the 126 MB L2, written between timed steps
+
+
+def _peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            d = json.load(f)
+        return float(d["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+
+    Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.rows = []
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                 "-lms", "50"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            if len(r) < 6:
+                continue
+            try:
+                sm.append(float(r[0]))
+                mx.append(float(r[1]))
+            except ValueError:
+                continue
+            for n, val in zip(names, r[2:6]):
+                if val.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def _visible_index(local_rank: int) -> int:
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local_rank])
+        except (ValueError, IndexError):
+            return local_rank
+    return local_rank
+
+
+def aggregate_over_ranks(dist, local_ms: float, local_bytes: float, device=None):
+    """Whole-job figures: time = max over ranks, bytes = sum over ranks (no data-path collective)."""
+    import torch
+    t = torch.tensor([local_ms], dtype=torch.float64, device=device)
+    b = torch.tensor([local_bytes], dtype=torch.float64, device=device)
+    if dist is not None and dist.is_initialized() and dist.get_world_size() > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        dist.all_reduce(b, op=dist.ReduceOp.SUM)
+    return float(t.item()), float(b.item())
+
+
+def batches_for_rank(rank: int, world: int, n_batches: int = N_BATCHES):
+    """Every rank drafts for its own sequences: disjoint hidden batches per rank."""
+    return [rank * n_batches + i for i in range(n_batches)]
+
+
+def run_oracle_baseline(cfg, W, gm, Wg, hidden_batches, steps, warmup=0):
+    """Times the CPU oracle, as it stands, on whole draft steps of the same workload."""
+    from oracle import lmhead_oracle as orc
+    times, touched = [], []
+    for i in range(warmup + steps):
+        hb = hidden_batches[i % len(hidden_batches)]
+        t0 = time.perf_counter()
+        r = orc.draft(W, gm, Wg, hb, cfg.k_groups, cfg.k_tokens, want_logits=False)
+        dt = time.perf_counter() - t0
+        if i >= warmup:
+            times.append(dt)
+            touched.append(len(set(r.groups.ravel().tolist())))
+    return times, touched, orc.threads()
+
+
+def algorithmic_bytes(cfg, groups_touched, M):
+    return groups_touched * cfg.v * cfg.H * 2 + cfg.N * cfg.H * 2 + M * cfg.H * 2 + M * cfg.k_tokens * 8
+
+
+def main_reference(args, rank):
+    """--impl reference: the CPU oracle on the host cores (rank 0 only)."""
+    if rank != 0:
+        return
+    from paper_2502_16880_b200 import synth
+    cfg = synth.CONFIGS[WORKLOAD].with_(M=args.rows)
+    W, gm, Wg = synth.make_w_vocab(cfg), synth.make_group_map(cfg), synth.make_w_gate(cfg)
+    hbs = [synth.make_hidden(cfg, cfg.M, batch=b) for b in range(N_BATCHES)]
+    times, touched, cores = run_oracle_baseline(cfg, W, gm, Wg, hbs, args.steps, args.warmup)
+    total = sum(times)
+    byts = sum(algorithmic_bytes(cfg, u, cfg.M) for u in touched)
+    val = byts / total / 1e9
+    sample = f"whole draft steps, M={cfg.M}, {args.steps} steps"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": total / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": f"{WORKLOAD}: H={cfg.H} V={cfg.V} N={cfg.N} top-{cfg.k_groups} M={cfg.M} "
+                               f"k_tokens={cfg.k_tokens}"},
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--rows", type=int, default=8, help="M of the headline workload")
+    ap.add_argument("--quick", action="store_true", help="headline only: skip the other M, dense and CPU legs")
+    args = ap.parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+
+    if args.impl == "reference":
+        main_reference(args, rank)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2502_16880_b200 import lmhead, synth
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU path)")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    lmhead.load_library()
+
+    cfg = synth.CONFIGS[WORKLOAD].with_(M=args.rows)
+    W, gm, Wg = synth.make_w_vocab(cfg), synth.make_group_map(cfg), synth.make_w_gate(cfg)
+
+    def dev_bf16(bits):
+        return torch.from_numpy(bits.view(np.int16)).to(dev).view(torch.bfloat16)
+
+    Wd = dev_bf16(W)
+    head = lmhead.LMHead(Wd, torch.from_numpy(gm), dev_bf16(Wg), max_M=64, max_k_groups=cfg.N, max_k_tokens=cfg.k_tokens)
+    flush = torch.empty(FLUSH_BYTES, dtype=torch.uint8, device=dev)
+    stream = torch.cuda.current_stream()
+
+    def time_steps(M, k_groups, steps, warmup, batches, kernel_timing=False):
+        """Per-step CUDA-event times (ms) with an L2 flush before every step, outside the event pair."""
+        hb_bits = [synth.make_hidden(cfg, M, batch=b) for b in batches]
+        hds = [dev_bf16(b) for b in hb_bits]
+        ids = torch.empty((M, cfg.k_tokens), dtype=torch.int32, device=dev)
+        lps = torch.empty((M, cfg.k_tokens), dtype=torch.float32, device=dev)
+        lmhead.coral_lmhead_set_kernel_timing(head.handle, kernel_timing)
+        ms, kms, touched, launches = [], [], [], 0
+        ev0 = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
+        ev1 = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
+        for i in range(warmup):
+            flush.fill_(i & 0xFF)
+            lmhead.coral_lmhead_draft(head.handle, hds[i % len(hds)], k_groups, cfg.k_tokens, ids, lps, stream)
+        # union size per batch (the stats call synchronises; done outside the timed steps)
+        per_batch_union = []
+        for hd in hds:
+            lmhead.coral_lmhead_draft(head.handle, hd, k_groups, cfg.k_tokens, ids, lps, stream)
+            st = head.stats()
+            per_batch_union.append(st.groups_touched)
+            per_launch = st.kernel_launches
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+        for i in range(steps):
+            flush.fill_(i & 0xFF)
+            ev0[i].record(stream)
+            lmhead.coral_lmhead_draft(head.handle, hds[i % len(hds)], k_groups, cfg.k_tokens, ids, lps, stream)
+            ev1[i].record(stream)
+            launches += per_launch
+            touched.append(per_batch_union[i % len(hds)])
+            if kernel_timing:
+                kms.append(lmhead.coral_lmhead_head_kernel_ms(head.handle))
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        ms = [a.elapsed_time(b) for a, b in zip(ev0, ev1)]
+        lmhead.coral_lmhead_set_kernel_timing(head.handle, False)
+        assert head.status() == 0
+        return ms, kms, touched, launches, hb_bits
+
+    my_batches = batches_for_rank(rank, world)
+    sampler = ClockSampler(_visible_index(local_rank))
+    sampler.start()            # runs across every timed GPU leg below
+    ms, _, touched, launches, hb_bits = time_steps(cfg.M, cfg.k_groups, args.steps, max(args.warmup, 3), my_batches)
+    local_ms = float(sum(ms))
+    local_bytes = float(sum(algorithmic_bytes(cfg, u, cfg.M) for u in touched))
+    tot_ms, tot_bytes = aggregate_over_ranks(dist if world > 1 else None, local_ms, local_bytes, dev)
+    value = tot_bytes / (tot_ms * 1e-3) / 1e9
+
+    # dominant kernel: the weight-streaming kernel, timed alone with events inside the library call
+    peak, peak_kind = _peaks()
+    ksteps = min(args.steps, 100)
+    _, kms, ktouched, _, _ = time_steps(cfg.M, cfg.k_groups, ksteps, 3, my_batches, kernel_timing=True)
+    k_bytes = float(np.mean([u * cfg.v * cfg.H * 2 + cfg.M * cfg.H * 2 for u in ktouched]))
+    k_ms = float(np.mean(kms))
+    achieved = k_bytes / (k_ms * 1e-3) / 1e9
+    roofline = {"bound": "hbm", "kernel": "head_simt_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "traffic": None,
+                "avg_launch_us": k_ms * 1e3, "algorithmic_bytes_per_launch": k_bytes}
+
+    # end to end through the host-buffer entry point (pinned host memory; copies inside the timed region)
+    hh = [torch.from_numpy(b.view(np.int16)).pin_memory() for b in hb_bits]
+    ids_h = torch.empty((cfg.M, cfg.k_tokens), dtype=torch.int32).pin_memory()
+    lps_h = torch.empty((cfg.M, cfg.k_tokens), dtype=torch.float32).pin_memory()
+    e2e_steps = min(args.steps, 100)
+    for i in range(3):
+        lmhead.coral_lmhead_draft_host(head.handle, hh[i % len(hh)], cfg.k_groups, cfg.k_tokens, ids_h, lps_h, stream)
+    e2e_t = 0.0
+    for i in range(e2e_steps):
+        flush.fill_(i & 0xFF)
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        lmhead.coral_lmhead_draft_host(head.handle, hh[i % len(hh)], cfg.k_groups, cfg.k_tokens, ids_h, lps_h, stream)
+        e2e_t += time.perf_counter() - t0
+    e2e_bytes = float(sum(algorithmic_bytes(cfg, touched[i % len(touched)], cfg.M) for i in range(e2e_steps)))
+    e2e_ms, e2e_tot_bytes = aggregate_over_ranks(dist if world > 1 else None, e2e_t * 1e3, e2e_bytes, dev)
+    e2e = {"value": e2e_tot_bytes / (e2e_ms * 1e-3) / 1e9, "unit": UNIT, "us_per_step": e2e_ms / e2e_steps * 1e3,
+           "h2d_bytes_per_step": cfg.M * cfg.H * 2, "d2h_bytes_per_step": cfg.M * cfg.k_tokens * 8}
+
+    out = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": tot_ms / args.steps, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16 inputs, f32 accumulate", "data": "synthetic",
+        "config": {"workload": f"{WORKLOAD}: H={cfg.H} V={cfg.V} N={cfg.N} top-{cfg.k_groups} M={cfg.M} "
+                               f"k_tokens={cfg.k_tokens}, seed {cfg.seed}",
+                   "l2": f"flush: {FLUSH_BYTES >> 20} MiB written before every timed step; {N_BATCHES} hidden batches "
+                         "rotated", "parallelism": f"replicas x{world}, rows sharded by sequence, no collective"},
+        "us_per_step": tot_ms / args.steps * 1e3,
+        "us_per_step_median": float(np.median(ms)) * 1e3,
+        "groups_touched_mean": float(np.mean(touched)),
+        "hbm_frac_whole_step": value / (peak * world),
+        "roofline": roofline, "e2e": e2e, "gpu_launches": launches,
+    }
+
+    if rank == 0 and world == 1 and not args.quick:
+        extra_steps = min(args.steps, 50)
+        also = []
+        for M in (1, 60):
+            ms_m, _, t_m, _, _ = time_steps(M, cfg.k_groups, extra_steps, 3, my_batches)
+            c2 = cfg.with_(M=M)
+            b_m = float(np.mean([algorithmic_bytes(c2, u, M) for u in t_m]))
+            us = float(np.mean(ms_m)) * 1e3
+            also.append({"M": M, "us_per_step": us, "GBps": b_m / us / 1e3, "hbm_frac": b_m / us / 1e3 / peak,
+                         "groups_touched_mean": float(np.mean(t_m))})
+        out["other_M"] = also
+        # dense head on the same GPU: (i) this library with every group active, (ii) torch bf16 matmul comparator
+        ms_d, _, t_d, _, _ = time_steps(cfg.M, cfg.N, extra_steps, 3, my_batches)
+        dense_bytes = algorithmic_bytes(cfg, cfg.N, cfg.M)
+        hd = dev_bf16(hb_bits[0])
+        tms = []
+        for i in range(extra_steps + 3):
+            flush.fill_(i & 0xFF)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            z = torch.matmul(hd, Wd.T).float()
+            torch.topk(torch.log_softmax(z, dim=1), cfg.k_tokens, dim=1)
+            b.record()
+            torch.cuda.synchronize()
+            if i >= 3:
+                tms.append(a.elapsed_time(b))
+        out["dense_head"] = {
+            "all_groups_active_us": float(np.mean(ms_d)) * 1e3,
+            "all_groups_active_GBps": dense_bytes / (float(np.mean(ms_d)) * 1e-3) / 1e9,
+            "torch_matmul_logsoftmax_topk_us": float(np.mean(tms)) * 1e3,
+            "grouped_vs_dense_speedup": float(np.mean(ms_d)) / (tot_ms / args.steps),
+        }
+        out["clocks"] = sampler.stop()
+        # CPU oracle on the host cores: whole steps of the same workload, bounded
+        o_steps = 3
+        times, o_touched, cores = run_oracle_baseline(cfg, W, gm, Wg, hb_bits, o_steps, warmup=1)
+        o_bytes = sum(algorithmic_bytes(cfg, u, cfg.M) for u in o_touched)
+        out["cpu_baseline"] = {"value": o_bytes / sum(times) / 1e9, "unit": UNIT, "cores": cores, "kind": "oracle",
+                               "sample": f"{o_steps} whole draft steps of the same workload (M={cfg.M})",
+                               "us_per_step": sum(times) / o_steps * 1e6}
+    if "clocks" not in out:
+        out["clocks"] = sampler.stop()
+    if rank == 0:
+        print(json.dumps(out))
+    head.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

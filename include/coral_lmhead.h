@@ -149,6 +149,17 @@ int coral_lmhead_draft_host(coral_lmhead_handle h, const void *hidden_host, int 
 int coral_lmhead_set_path(coral_lmhead_handle h, int path);
 
 /*
+ * Measurement aid for the dominant kernel (the one that streams the selected
+ * groups' weights; Section 3.3 names the LM head as the drafter's main cost).
+ * With timing on, every draft call records a CUDA event before and after that
+ * kernel on the call's stream; coral_lmhead_head_kernel_ms waits for the last
+ * call's second event and returns the elapsed milliseconds between the two.
+ * Timing is off by default.  CORAL_ERR_INVALID if timing was never switched on.
+ */
+int coral_lmhead_set_kernel_timing(coral_lmhead_handle h, int on);
+int coral_lmhead_head_kernel_ms(coral_lmhead_handle h, float *ms);
+
+/*
  * Synchronise `stream`, return the device status word of the handle (CORAL_OK,
  * CORAL_ERR_TIMEOUT, CORAL_ERR_BOUNDS) and clear it.
  */

@@ -84,6 +84,8 @@ struct coral_lmhead_s {
     bool own_packed, own_ws;
     int forced_path;
     int simt_smem;
+    cudaEvent_t ev_head0, ev_head1;   // around the weight-streaming kernel when kernel timing is on
+    bool timing;
     // facts about the last draft call
     int last_path, last_M, last_kg, last_kt, last_launches;
 };
@@ -229,6 +231,8 @@ int coral_lmhead_destroy(coral_lmhead_handle h) {
     if (!h) return CORAL_OK;
     if (h->own_packed && h->packed) cudaFree(h->packed);
     if (h->own_ws && h->ws) cudaFree(h->ws);
+    if (h->ev_head0) cudaEventDestroy(h->ev_head0);
+    if (h->ev_head1) cudaEventDestroy(h->ev_head1);
     delete h;
     return CORAL_OK;
 }
@@ -263,8 +267,10 @@ int coral_lmhead_draft_ex(coral_lmhead_handle h, const void* hidden_dev, int M, 
     ++launches;
     bucket_kernel<<<1, kBucketThreads, 0, st>>>(c);
     ++launches;
+    if (h->timing) cudaEventRecord(h->ev_head0, st);
     head_simt_kernel<<<dim3(c.T, c.N), kSimtThreads, h->simt_smem, st>>>(c, out_logits_dev);
     ++launches;
+    if (h->timing) cudaEventRecord(h->ev_head1, st);
     merge_kernel<<<M, kMergeThreads, 0, st>>>(c, out_ids_dev, out_logprobs_dev, out_lse_dev);
     ++launches;
     if (cudaGetLastError() != cudaSuccess) return CORAL_ERR_CUDA;
@@ -297,6 +303,23 @@ int coral_lmhead_draft_host(coral_lmhead_handle h, const void* hidden_host, int 
     if (cudaMemcpyAsync(out_logprobs_host, d_lp, (size_t)M * k_tokens * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess)
         return CORAL_ERR_CUDA;
     if (cudaStreamSynchronize(st) != cudaSuccess) return CORAL_ERR_CUDA;
+    return CORAL_OK;
+}
+
+int coral_lmhead_set_kernel_timing(coral_lmhead_handle h, int on) {
+    if (!h) return CORAL_ERR_INVALID;
+    if (on && !h->ev_head0) {
+        if (cudaEventCreate(&h->ev_head0) != cudaSuccess || cudaEventCreate(&h->ev_head1) != cudaSuccess)
+            return CORAL_ERR_CUDA;
+    }
+    h->timing = on != 0;
+    return CORAL_OK;
+}
+
+int coral_lmhead_head_kernel_ms(coral_lmhead_handle h, float* ms) {
+    if (!h || !ms || !h->ev_head0) return CORAL_ERR_INVALID;
+    if (cudaEventSynchronize(h->ev_head1) != cudaSuccess) return CORAL_ERR_CUDA;
+    if (cudaEventElapsedTime(ms, h->ev_head0, h->ev_head1) != cudaSuccess) return CORAL_ERR_CUDA;
     return CORAL_OK;
 }
 

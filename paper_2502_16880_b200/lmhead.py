@@ -51,6 +51,8 @@ _SIGNATURES = {
     "coral_lmhead_draft_ex": (_i, [_vp, _vp, _i, _i, _i, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "coral_lmhead_draft_host": (_i, [_vp, _vp, _i, _i, _i, _vp, _vp, _vp]),
     "coral_lmhead_set_path": (_i, [_vp, _i]),
+    "coral_lmhead_set_kernel_timing": (_i, [_vp, _i]),
+    "coral_lmhead_head_kernel_ms": (_i, [_vp, ctypes.POINTER(ctypes.c_float)]),
     "coral_lmhead_status": (_i, [_vp, _vp]),
     "coral_lmhead_last_stats": (_i, [_vp, ctypes.POINTER(coral_lmhead_stats), _vp]),
     "coral_lmhead_error_string": (ctypes.c_char_p, [_i]),
@@ -171,6 +173,16 @@ def coral_lmhead_draft_host(handle, hidden_host, k_groups, k_tokens, out_ids_hos
 
 def coral_lmhead_set_path(handle, path: int) -> None:
     _check(load_library().coral_lmhead_set_path(handle, int(path)), "coral_lmhead_set_path")
+
+
+def coral_lmhead_set_kernel_timing(handle, on: bool) -> None:
+    _check(load_library().coral_lmhead_set_kernel_timing(handle, int(bool(on))), "coral_lmhead_set_kernel_timing")
+
+
+def coral_lmhead_head_kernel_ms(handle) -> float:
+    ms = ctypes.c_float(0.0)
+    _check(load_library().coral_lmhead_head_kernel_ms(handle, ctypes.byref(ms)), "coral_lmhead_head_kernel_ms")
+    return float(ms.value)
 
 
 def coral_lmhead_status(handle, stream=None) -> int:
