@@ -37,10 +37,12 @@ extern "C" {
 #define CORAL_ERR_NOMEM (-4)       /* host or device allocation failed */
 #define CORAL_ERR_TIMEOUT (-5)     /* a bounded device-side wait gave up (device status word) */
 #define CORAL_ERR_BOUNDS (-6)      /* a device-side index check failed (device status word) */
+#define CORAL_ERR_TOO_LARGE (-7)   /* request exceeds the fixed scratch of coral_lmhead_route_static */
 
 /* Limits of this build. */
 #define CORAL_MAX_GROUPS 256       /* n_groups <= 256 */
 #define CORAL_MAX_K_TOKENS 32      /* k_tokens <= 32 */
+#define CORAL_ROUTE_STATIC_MAX_ROWS 64 /* M <= 64 for coral_lmhead_route_static */
 
 /* Execution paths (coral_lmhead_set_path / coral_lmhead_stats.path). */
 #define CORAL_PATH_AUTO 0          /* chosen from (M, k_groups) */
@@ -171,6 +173,43 @@ int coral_lmhead_status(coral_lmhead_handle h, void *stream);
  * Synchronises `stream` to read the union size back.
  */
 int coral_lmhead_last_stats(coral_lmhead_handle h, coral_lmhead_stats *out, void *stream);
+
+/*
+ * Router step (gate scores and the k_groups best groups per row) for callers
+ * that must not allocate.  The paper has no counterpart to this entry point;
+ * it computes the same scores and selections as coral_lmhead_draft_ex reports
+ * through out_gate_dev / out_groups_dev.
+ *
+ * Who needs it: code that runs where device allocation is off limits, for
+ * example a serving loop whose memory pool is fixed up front and audited, a
+ * plug-in that is handed a stream but no allocator, or a latency-critical
+ * section where cudaMalloc's implicit device synchronisation is unacceptable.
+ * Such callers cannot create a handle (that needs a workspace).  Here they pass
+ * only inputs and outputs; the scratch the router kernels need lives in a fixed
+ * array inside the library's device image, CORAL_ROUTE_STATIC_MAX_ROWS rows x
+ * CORAL_MAX_GROUPS groups (about 160 KiB), which every GPU that loads the
+ * library keeps until the process exits.  The call makes no cudaMalloc,
+ * cudaFree or other allocating call.
+ *
+ *   W_gate_dev     [n_groups x H] bf16, device, 16-byte aligned
+ *   hidden_dev     [M x H] bf16, device, 16-byte aligned
+ *   out_groups_dev [M x k_groups] int32, device: groups in selection order
+ *                  (descending score, equal scores -> lower index)
+ *   out_gate_dev   [M x n_groups] float, device, or NULL
+ * Asynchronous on `stream`.  CORAL_ERR_TOO_LARGE if M exceeds
+ * CORAL_ROUTE_STATIC_MAX_ROWS; CORAL_ERR_INVALID for NULL/misaligned pointers,
+ * H not a positive multiple of 8, n_groups outside [1, CORAL_MAX_GROUPS] or
+ * k_groups outside [1, n_groups].
+ *
+ * The first call on each device looks up the array's device address (a
+ * runtime query, made with that device current); make that first call before
+ * starting any stream capture.  All calls on a device share the one array and
+ * it keeps the previous call's contents (the call clears what has to start at
+ * zero): two calls whose kernels may overlap on the GPU (different streams,
+ * no ordering between them) race and give undefined results.
+ */
+int coral_lmhead_route_static(const void *W_gate_dev, const void *hidden_dev, int M, int H, int n_groups,
+                              int k_groups, int32_t *out_groups_dev, float *out_gate_dev, void *stream);
 
 /* Static, NUL-terminated description of a status code. */
 const char *coral_lmhead_error_string(int code);

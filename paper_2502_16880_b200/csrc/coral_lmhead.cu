@@ -138,6 +138,7 @@ const char* coral_lmhead_error_string(int code) {
         case CORAL_ERR_NOMEM: return "out of memory";
         case CORAL_ERR_TIMEOUT: return "device-side wait timed out";
         case CORAL_ERR_BOUNDS: return "device-side index check failed";
+        case CORAL_ERR_TOO_LARGE: return "size exceeds the built-in scratch of the no-allocation entry point";
         default: return "unknown status";
     }
 }
@@ -353,3 +354,72 @@ int coral_lmhead_last_stats(coral_lmhead_handle h, coral_lmhead_stats* out, void
 }
 
 }  // extern "C"
+
+// ---------------------------------------------------------------------------------------------
+// Router step without any allocation (see coral_lmhead_route_static in the header).
+// The gate scores, the per-row slot table and the status word that the router kernels use as
+// scratch live in this file-scope device array instead of a caller- or library-allocated
+// workspace.  Every GPU that loads the library holds one copy of it until the process exits.
+// ---------------------------------------------------------------------------------------------
+namespace {
+
+constexpr int kStaticMaxRows = CORAL_ROUTE_STATIC_MAX_ROWS;
+constexpr size_t kStaticGateOff = 0;                                                       // float [rows][N]
+constexpr size_t kStaticSelOff = kStaticGateOff + (size_t)kStaticMaxRows * kMaxGroups * 4;  // int32 [rows][k]
+constexpr size_t kStaticSlotOff = kStaticSelOff + (size_t)kStaticMaxRows * kMaxGroups * 4;  // int16 [rows][N]
+constexpr size_t kStaticStateOff = kStaticSlotOff + (size_t)kStaticMaxRows * kMaxGroups * 2;
+constexpr size_t kStaticBytes = kStaticStateOff + 256;
+
+static __device__ __align__(256) unsigned char g_route_scratch[kStaticBytes];
+
+// In host code `g_route_scratch` is only a handle for the runtime, not a device address.  The
+// address is looked up once per device, with that device current, and cached here.
+constexpr int kMaxDevices = 64;
+unsigned char* g_route_scratch_addr[kMaxDevices] = {};
+
+int route_scratch_for_current_device(unsigned char** out) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) return CORAL_ERR_CUDA;
+    if (dev < 0 || dev >= kMaxDevices) return CORAL_ERR_INVALID;
+    unsigned char* p = __atomic_load_n(&g_route_scratch_addr[dev], __ATOMIC_ACQUIRE);
+    if (!p) {
+        if (cudaGetSymbolAddress(reinterpret_cast<void**>(&p), g_route_scratch) != cudaSuccess || !p)
+            return CORAL_ERR_CUDA;
+        __atomic_store_n(&g_route_scratch_addr[dev], p, __ATOMIC_RELEASE);   // same value from any thread
+    }
+    *out = p;
+    return CORAL_OK;
+}
+
+}  // namespace
+
+extern "C" int coral_lmhead_route_static(const void* W_gate_dev, const void* hidden_dev, int M, int H, int n_groups,
+                                         int k_groups, int32_t* out_groups_dev, float* out_gate_dev, void* stream) {
+    if (!W_gate_dev || !hidden_dev || !out_groups_dev) return CORAL_ERR_INVALID;
+    if ((reinterpret_cast<uintptr_t>(W_gate_dev) & 15) || (reinterpret_cast<uintptr_t>(hidden_dev) & 15))
+        return CORAL_ERR_INVALID;
+    if (H < 8 || H % 8 != 0 || n_groups < 1 || n_groups > CORAL_MAX_GROUPS) return CORAL_ERR_INVALID;
+    if (k_groups < 1 || k_groups > n_groups) return CORAL_ERR_INVALID;
+    if (M < 1) return CORAL_ERR_INVALID;
+    if (M > kStaticMaxRows) return CORAL_ERR_TOO_LARGE;   // the built-in scratch holds at most that many rows
+    unsigned char* scratch = nullptr;
+    const int rc = route_scratch_for_current_device(&scratch);
+    if (rc != CORAL_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+
+    CallView c{};
+    c.M = M; c.H = H; c.N = n_groups; c.k_groups = k_groups;
+    c.w_gate = static_cast<const uint16_t*>(W_gate_dev);
+    c.hidden = static_cast<const uint16_t*>(hidden_dev);
+    c.gate = reinterpret_cast<float*>(scratch + kStaticGateOff);
+    c.sel = reinterpret_cast<int32_t*>(scratch + kStaticSelOff);
+    c.slot_of = reinterpret_cast<int16_t*>(scratch + kStaticSlotOff);
+    c.state = reinterpret_cast<DeviceState*>(scratch + kStaticStateOff);
+    // The array keeps the previous call's contents.  The status word must start at zero; the gate,
+    // selection and slot tables are fully rewritten for rows < M before anything reads them.
+    if (cudaMemsetAsync(c.state, 0, sizeof(DeviceState), st) != cudaSuccess) return CORAL_ERR_CUDA;
+    gate_kernel<<<dim3(c.N, (M + kGateRows - 1) / kGateRows), kGateThreads, 0, st>>>(c, out_gate_dev);
+    select_kernel<<<(M + kSelectWarps - 1) / kSelectWarps, kSelectWarps * 32, 0, st>>>(c, nullptr, out_groups_dev);
+    if (cudaGetLastError() != cudaSuccess) return CORAL_ERR_CUDA;
+    return CORAL_OK;
+}

@@ -23,6 +23,8 @@ CORAL_ERR_CUDA = -3
 CORAL_ERR_NOMEM = -4
 CORAL_ERR_TIMEOUT = -5
 CORAL_ERR_BOUNDS = -6
+CORAL_ERR_TOO_LARGE = -7
+CORAL_ROUTE_STATIC_MAX_ROWS = 64
 CORAL_PATH_AUTO, CORAL_PATH_SIMT, CORAL_PATH_TCGEN05 = 0, 1, 2
 
 
@@ -55,6 +57,7 @@ _SIGNATURES = {
     "coral_lmhead_head_kernel_ms": (_i, [_vp, ctypes.POINTER(ctypes.c_float)]),
     "coral_lmhead_status": (_i, [_vp, _vp]),
     "coral_lmhead_last_stats": (_i, [_vp, ctypes.POINTER(coral_lmhead_stats), _vp]),
+    "coral_lmhead_route_static": (_i, [_vp, _vp, _i, _i, _i, _i, _vp, _vp, _vp]),
     "coral_lmhead_error_string": (ctypes.c_char_p, [_i]),
     "coral_lmhead_destroy": (_i, [_vp]),
 }
@@ -194,6 +197,18 @@ def coral_lmhead_last_stats(handle, stream=None) -> coral_lmhead_stats:
     _check(load_library().coral_lmhead_last_stats(handle, ctypes.byref(s), _stream_ptr(stream)),
            "coral_lmhead_last_stats")
     return s
+
+
+def coral_lmhead_route_static(W_gate, hidden, k_groups, out_groups, out_gate=None, stream=None) -> None:
+    """Gate scores and top-k groups without a handle and without any allocation inside the library
+    (for callers that are not allowed to allocate device memory); at most CORAL_ROUTE_STATIC_MAX_ROWS rows.
+    The tensors passed in are the only memory the caller provides; scratch is built into the library."""
+    N, H = W_gate.shape
+    M = hidden.shape[0]
+    _check(load_library().coral_lmhead_route_static(
+        _dev_ptr(W_gate, torch.bfloat16, False), _dev_ptr(hidden, torch.bfloat16, False), M, H, N, int(k_groups),
+        _dev_ptr(out_groups, torch.int32, False), _dev_ptr(out_gate, torch.float32), _stream_ptr(stream)),
+        "coral_lmhead_route_static")
 
 
 def coral_lmhead_destroy(handle) -> None:

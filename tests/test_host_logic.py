@@ -37,7 +37,7 @@ def test_library_exports_every_declared_symbol(lib):
 
 def test_error_strings_and_host_only_argument_checks(lib):
     assert lmhead.coral_lmhead_error_string(0) == "ok"
-    for code in range(-6, 0):
+    for code in range(-7, 0):
         assert lmhead.coral_lmhead_error_string(code) not in ("ok", "unknown status")
     ok = lmhead.make_config(4096, 128256, 64, 960, 8, 10)
     pb, wb = lmhead.coral_lmhead_query_sizes(ok)
