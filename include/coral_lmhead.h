@@ -46,8 +46,9 @@ extern "C" {
 
 /* Execution paths (coral_lmhead_set_path / coral_lmhead_stats.path). */
 #define CORAL_PATH_AUTO 0          /* chosen from (M, k_groups) */
-#define CORAL_PATH_SIMT 1          /* gathered GEMV: weight streaming + fp32 FMA */
+#define CORAL_PATH_SIMT 1          /* gathered GEMV, M <= 8: bulk-copy weight streaming + fp32 FMA */
 #define CORAL_PATH_TCGEN05 2       /* routed grouped GEMM on tcgen05 / TMEM tiles */
+#define CORAL_PATH_SIMT_PLAIN 3    /* gathered GEMV with plain 128-bit loads, any M */
 
 typedef struct coral_lmhead_s *coral_lmhead_handle;
 
@@ -147,7 +148,11 @@ int coral_lmhead_draft_ex(coral_lmhead_handle h, const void *hidden_dev, int M, 
 int coral_lmhead_draft_host(coral_lmhead_handle h, const void *hidden_host, int M, int k_groups, int k_tokens,
                             int32_t *out_ids_host, float *out_logprobs_host, void *stream);
 
-/* Force an execution path (CORAL_PATH_*) for later draft calls; AUTO restores the default choice. */
+/*
+ * Force an execution path (CORAL_PATH_*) for later draft calls; AUTO restores the default choice.
+ * A draft call that the forced path cannot run (e.g. CORAL_PATH_SIMT with M > 8) returns
+ * CORAL_ERR_INVALID.
+ */
 int coral_lmhead_set_path(coral_lmhead_handle h, int path);
 
 /*

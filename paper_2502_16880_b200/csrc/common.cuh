@@ -32,6 +32,9 @@ struct CallView {
     int32_t* group_offset;         // [N+1]
     int32_t* bucket_row;           // [M*k_groups] rows that selected a group, ascending per group
     int32_t* bucket_slot;          // [M*k_groups] the slot the group has in that row
+    int32_t* bucket_pos;           // [M][k_groups] position of row m in the bucket of its slot's group
+    int32_t* union_list;           // [N] touched groups in ascending order (first n_union entries)
+    int32_t* union_rank;           // [N] index of group n in union_list, -1 if untouched
     float* part_max;               // [M][k_groups][T]
     float* part_sum;               // [M][k_groups][T]
     float* part_val;               // [M][k_groups][T][k_tokens]

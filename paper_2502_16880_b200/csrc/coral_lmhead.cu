@@ -9,6 +9,7 @@
 
 #include "common.cuh"
 #include "head_simt.cuh"
+#include "head_stream.cuh"
 #include "merge.cuh"
 #include "route.cuh"
 
@@ -22,8 +23,9 @@ inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 // Offsets of the workspace sections (bytes from the workspace base).
 struct Layout {
     size_t w_gate, group_tokens, state, gate, sel, slot_of, group_count, group_offset, bucket_row, bucket_slot,
-        part_max, part_sum, part_val, part_id, stage_hidden, stage_ids, stage_logprobs, total;
-    size_t packed_bytes;
+        bucket_pos, union_list, union_rank, part_max, part_sum, part_val, part_id, sp_max, sp_sum, sp_val, sp_id,
+        cand_val, cand_id, stage_hidden, stage_ids, stage_logprobs, total;
+    size_t packed_bytes, cand_cap;
     int v, T;
 };
 
@@ -35,6 +37,40 @@ bool config_ok(const coral_lmhead_config* c) {
     if (c->max_k_tokens < 1 || c->max_k_tokens > CORAL_MAX_K_TOKENS) return false;
     return true;
 }
+
+// Geometry of the streaming path.  The workspace layout must not depend on the device (sizes are
+// queried before a device is chosen), so it is sized for any grid in [kStreamGridMin, kStreamGridCap];
+// the launch geometry is fixed at create from the device's SM count and shared-memory limit.
+constexpr int kStreamGridMin = 64, kStreamGridCap = 160;
+
+int stream_seg_max(int n_groups, int T, int grid) {
+    const long per_max = ((long)n_groups * T + grid - 1) / grid;
+    return (int)((per_max + T - 1) / T) + 1;
+}
+
+StreamGeom make_stream_geom(const coral_lmhead_config& c, int sms, int smem_optin) {
+    StreamGeom g{};
+    const int v = c.V / c.n_groups;
+    g.grid = sms < kStreamGridCap ? sms : kStreamGridCap;
+    g.T = (v + kStreamTile - 1) / kStreamTile;
+    int sr = 1;
+    while (sr < kStreamTile && (size_t)(sr * 2) * c.H * 2 <= 16384) sr *= 2;
+    g.stage_rows = sr;
+    const size_t stage_bytes = (size_t)sr * c.H * 2;
+    const size_t fixed = sizeof(float) * (kStreamWarps * kStreamTile * kStreamMaxR + kStreamMaxR * kStreamTile) + 1024;
+    long ns = ((long)smem_optin - (long)fixed) / (long)stage_bytes;
+    g.n_stages = (int)(ns > 8 ? 8 : ns);
+    g.seg_max = stream_seg_max(c.n_groups, g.T, g.grid);
+    return g;
+}
+
+size_t stream_smem_bytes(const StreamGeom& g, int H) {
+    return (size_t)g.n_stages * g.stage_rows * H * 2 +
+           sizeof(float) * (kStreamWarps * kStreamTile * kStreamMaxR + kStreamMaxR * kStreamTile) +
+           sizeof(uint64_t) * 2 * g.n_stages + 16;
+}
+
+constexpr int kMergeSmemCands = 4096;   // candidates the streaming merge keeps in shared memory
 
 Layout make_layout(const coral_lmhead_config& c) {
     Layout L{};
@@ -53,6 +89,19 @@ Layout make_layout(const coral_lmhead_config& c) {
     L.group_offset = take((N + 1) * 4);
     L.bucket_row = take(M * kg * 4);
     L.bucket_slot = take(M * kg * 4);
+    L.bucket_pos = take(M * kg * 4);
+    L.union_list = take(N * 4);
+    L.union_rank = take(N * 4);
+    const int T16 = (L.v + kStreamTile - 1) / kStreamTile;
+    const size_t sp = (size_t)kStreamGridCap * stream_seg_max(c.n_groups, T16, kStreamGridMin) * kStreamMaxR;
+    L.sp_max = take(sp * 4);
+    L.sp_sum = take(sp * 4);
+    L.sp_val = take(sp * kt * 4);
+    L.sp_id = take(sp * kt * 4);
+    const size_t cand_rows = M < (size_t)kStreamMaxR ? M : (size_t)kStreamMaxR;
+    L.cand_cap = ((size_t)kStreamGridCap + 2 * kg) * kt;
+    L.cand_val = take(cand_rows * L.cand_cap * 4);
+    L.cand_id = take(cand_rows * L.cand_cap * 4);
     L.part_max = take(M * kg * T * 4);
     L.part_sum = take(M * kg * T * 4);
     L.part_val = take(M * kg * T * kt * 4);
@@ -84,6 +133,8 @@ struct coral_lmhead_s {
     bool own_packed, own_ws;
     int forced_path;
     int simt_smem;
+    StreamGeom sg;
+    int stream_smem;     // 0 if the streaming path is not available for this shape/device
     cudaEvent_t ev_head0, ev_head1;   // around the weight-streaming kernel when kernel timing is on
     bool timing;
     // facts about the last draft call
@@ -109,6 +160,9 @@ CallView make_view(const coral_lmhead_s* h, const void* hidden, int M, int kg, i
     c.group_offset = reinterpret_cast<int32_t*>(ws + L.group_offset);
     c.bucket_row = reinterpret_cast<int32_t*>(ws + L.bucket_row);
     c.bucket_slot = reinterpret_cast<int32_t*>(ws + L.bucket_slot);
+    c.bucket_pos = reinterpret_cast<int32_t*>(ws + L.bucket_pos);
+    c.union_list = reinterpret_cast<int32_t*>(ws + L.union_list);
+    c.union_rank = reinterpret_cast<int32_t*>(ws + L.union_rank);
     c.part_max = reinterpret_cast<float*>(ws + L.part_max);
     c.part_sum = reinterpret_cast<float*>(ws + L.part_sum);
     c.part_val = reinterpret_cast<float*>(ws + L.part_val);
@@ -117,10 +171,15 @@ CallView make_view(const coral_lmhead_s* h, const void* hidden, int M, int kg, i
     return c;
 }
 
+bool stream_ok(const coral_lmhead_s* h, int M) { return h->stream_smem > 0 && M <= kStreamMaxR; }
+
+// CORAL_PATH_SIMT: streaming kernel (needs M <= 8); CORAL_PATH_SIMT_PLAIN: any M.  Returns 0 if the
+// forced path cannot run this call.
 int choose_path(const coral_lmhead_s* h, int M, int kg) {
-    (void)M; (void)kg;
+    (void)kg;
+    if (h->forced_path == CORAL_PATH_SIMT) return stream_ok(h, M) ? CORAL_PATH_SIMT : 0;
     if (h->forced_path != CORAL_PATH_AUTO) return h->forced_path;
-    return CORAL_PATH_SIMT;
+    return stream_ok(h, M) ? CORAL_PATH_SIMT : CORAL_PATH_SIMT_PLAIN;
 }
 
 }  // namespace
@@ -209,6 +268,17 @@ int coral_lmhead_create(coral_lmhead_handle* out, const coral_lmhead_config* cfg
         if (h->simt_smem > smem_optin) { rc = CORAL_ERR_INVALID; break; }
         if (cudaFuncSetAttribute(head_simt_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_optin) !=
             cudaSuccess) { rc = CORAL_ERR_CUDA; break; }
+        int sms = 0;
+        if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) { rc = CORAL_ERR_CUDA; break; }
+        h->sg = make_stream_geom(*cfg, sms, smem_optin);
+        h->stream_smem = 0;
+        if (cfg->H <= kStreamMaxH && sms >= kStreamGridMin && h->sg.n_stages >= 2) {
+            h->stream_smem = (int)stream_smem_bytes(h->sg, cfg->H);
+            if (cudaFuncSetAttribute(head_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_optin) !=
+                cudaSuccess) { rc = CORAL_ERR_CUDA; break; }
+            if (cudaFuncSetAttribute(merge_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     kMergeSmemCands * 8) != cudaSuccess) { rc = CORAL_ERR_CUDA; break; }
+        }
         if (cudaMemcpyAsync(h->ws + h->L.group_tokens, group_tokens.data(), (size_t)V * 4, cudaMemcpyHostToDevice, st) !=
             cudaSuccess) { rc = CORAL_ERR_CUDA; break; }
         if (cudaMemcpyAsync(h->ws + h->L.w_gate, W_gate_dev, (size_t)N * cfg->H * 2, cudaMemcpyDeviceToDevice, st) !=
@@ -239,7 +309,7 @@ int coral_lmhead_destroy(coral_lmhead_handle h) {
 }
 
 int coral_lmhead_set_path(coral_lmhead_handle h, int path) {
-    if (!h || path < CORAL_PATH_AUTO || path > CORAL_PATH_TCGEN05) return CORAL_ERR_INVALID;
+    if (!h || path < CORAL_PATH_AUTO || path > CORAL_PATH_SIMT_PLAIN) return CORAL_ERR_INVALID;
     if (path == CORAL_PATH_TCGEN05) return CORAL_ERR_INVALID;   // not built yet
     h->forced_path = path;
     return CORAL_OK;
@@ -259,6 +329,7 @@ int coral_lmhead_draft_ex(coral_lmhead_handle h, const void* hidden_dev, int M, 
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const CallView c = make_view(h, hidden_dev, M, k_groups, k_tokens);
     const int path = choose_path(h, M, k_groups);
+    if (path == 0) return CORAL_ERR_INVALID;   // the forced path does not support this call
     int launches = 0;
 
     gate_kernel<<<dim3(c.N, (M + kGateRows - 1) / kGateRows), kGateThreads, 0, st>>>(c, out_gate_dev);
@@ -269,11 +340,24 @@ int coral_lmhead_draft_ex(coral_lmhead_handle h, const void* hidden_dev, int M, 
     bucket_kernel<<<1, kBucketThreads, 0, st>>>(c);
     ++launches;
     if (h->timing) cudaEventRecord(h->ev_head0, st);
-    head_simt_kernel<<<dim3(c.T, c.N), kSimtThreads, h->simt_smem, st>>>(c, out_logits_dev);
-    ++launches;
-    if (h->timing) cudaEventRecord(h->ev_head1, st);
-    merge_kernel<<<M, kMergeThreads, 0, st>>>(c, out_ids_dev, out_logprobs_dev, out_lse_dev);
-    ++launches;
+    if (path == CORAL_PATH_SIMT) {
+        const Layout& L = h->L;
+        StreamPartials pp{reinterpret_cast<float*>(h->ws + L.sp_max), reinterpret_cast<float*>(h->ws + L.sp_sum),
+                          reinterpret_cast<float*>(h->ws + L.sp_val), reinterpret_cast<int32_t*>(h->ws + L.sp_id)};
+        head_stream_kernel<<<h->sg.grid, kStreamThreads, h->stream_smem, st>>>(c, h->sg, pp, out_logits_dev);
+        ++launches;
+        if (h->timing) cudaEventRecord(h->ev_head1, st);
+        merge_stream_kernel<<<M, kMergeStreamThreads, kMergeSmemCands * 8, st>>>(
+            c, h->sg, pp, reinterpret_cast<float*>(h->ws + L.cand_val), reinterpret_cast<int32_t*>(h->ws + L.cand_id),
+            (int)L.cand_cap, kMergeSmemCands, out_ids_dev, out_logprobs_dev, out_lse_dev);
+        ++launches;
+    } else {
+        head_simt_kernel<<<dim3(c.T, c.N), kSimtThreads, h->simt_smem, st>>>(c, out_logits_dev);
+        ++launches;
+        if (h->timing) cudaEventRecord(h->ev_head1, st);
+        merge_kernel<<<M, kMergeThreads, 0, st>>>(c, out_ids_dev, out_logprobs_dev, out_lse_dev);
+        ++launches;
+    }
     if (cudaGetLastError() != cudaSuccess) return CORAL_ERR_CUDA;
 
     h->last_path = path; h->last_M = M; h->last_kg = k_groups; h->last_kt = k_tokens; h->last_launches = launches;

@@ -125,7 +125,11 @@ __global__ void __launch_bounds__(kBucketThreads) bucket_kernel(CallView c) {
         for (int n = 0; n < c.N; ++n) {
             s_offset[n] = run;
             run += s_count[n];
-            uni += s_count[n] > 0;
+            if (c.union_rank) c.union_rank[n] = s_count[n] > 0 ? uni : -1;
+            if (s_count[n] > 0) {
+                if (c.union_list) c.union_list[uni] = n;
+                ++uni;
+            }
         }
         s_offset[c.N] = run;
         c.state->n_union = uni;
@@ -145,6 +149,7 @@ __global__ void __launch_bounds__(kBucketThreads) bucket_kernel(CallView c) {
                 const int p = pos + __popc(bal & ((1u << lane) - 1u));
                 c.bucket_row[p] = m;
                 c.bucket_slot[p] = sl;
+                if (c.bucket_pos) c.bucket_pos[(size_t)m * c.k_groups + sl] = p - s_offset[n];
             }
             pos += __popc(bal);
         }

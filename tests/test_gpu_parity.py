@@ -8,7 +8,12 @@ from tests import parity_harness as ph
 
 pytestmark = pytest.mark.gpu
 
-PATHS = [lmhead.CORAL_PATH_SIMT]
+PATHS = [lmhead.CORAL_PATH_SIMT, lmhead.CORAL_PATH_SIMT_PLAIN]
+
+
+def _supported(path, M):
+    return path != lmhead.CORAL_PATH_SIMT or M <= 8
+
 
 
 def _head(cfg, W, gm, Wg, max_M=None, max_kg=None, max_kt=None):
@@ -30,6 +35,8 @@ def _weights(name):
 
 
 def _check(head, W, gm, Wg, hb, kg, kt, path, forced=None):
+    if not _supported(path, hb.shape[0]):
+        pytest.skip("streaming path takes M <= 8")
     head.set_path(path)
     out = ph.gpu_draft_numpy(head, hb, kg, kt, forced_groups=forced)
     assert head.status() == 0
@@ -52,7 +59,8 @@ def test_tiny(path, M, kg, kt):
 @pytest.mark.parametrize("path", PATHS)
 def test_ragged_shape(path):
     # v = 300 (two full tiles + a tail of 44), H = 328 (not a multiple of 256)
-    cfg = synth.HeadConfig("ragged", H=328, V=1800, N=6, k_groups=3, k_tokens=10, M=13, seed=5, w_std=0.05)
+    cfg = synth.HeadConfig("ragged", H=328, V=1800, N=6, k_groups=3, k_tokens=10,
+                           M=13 if path != lmhead.CORAL_PATH_SIMT else 7, seed=5, w_std=0.05)
     W, gm, Wg, hb = synth.make_all(cfg)
     head = _head(cfg, W, gm, Wg)
     for kg, kt in [(3, 10), (6, 32), (1, 5)]:
@@ -98,7 +106,7 @@ def test_exact_ties_zero_weights(path):
 @pytest.mark.parametrize("path", PATHS)
 def test_deterministic_bitwise(path):
     cfg, W, gm, Wg, head = _weights("tiny")
-    hb = synth.make_hidden(cfg, 33)
+    hb = synth.make_hidden(cfg, 33 if path != lmhead.CORAL_PATH_SIMT else 8)
     head.set_path(path)
     a = ph.gpu_draft_numpy(head, hb, 4, 10)
     b = ph.gpu_draft_numpy(head, hb, 4, 10)
@@ -122,6 +130,12 @@ def test_argument_errors_return_codes():
     assert lib.coral_lmhead_draft(head.handle, None, 4, 4, 10, ip, lp, None) == lmhead.CORAL_ERR_INVALID
     assert lib.coral_lmhead_draft(head.handle, hp, 4, 4, 10, None, lp, None) == lmhead.CORAL_ERR_INVALID
     assert lib.coral_lmhead_draft(None, hp, 4, 4, 10, ip, lp, None) == lmhead.CORAL_ERR_INVALID
+    # a forced path that cannot take the call is refused, not silently replaced
+    h9 = ph.to_dev_bf16(synth.make_hidden(cfg, 9))
+    head.set_path(lmhead.CORAL_PATH_SIMT)
+    assert lib.coral_lmhead_draft(head.handle, ctypes.c_void_p(h9.data_ptr()), 9, 4, 10, ip, lp, None) == \
+        lmhead.CORAL_ERR_INVALID
+    head.set_path(lmhead.CORAL_PATH_AUTO)
     # unequal groups are rejected at create, before anything touches the device
     bad = gm.copy()
     bad[0] = (bad[0] + 1) % cfg.N
@@ -151,6 +165,8 @@ def test_library_owned_buffers_and_host_entry():
 def test_paper_shapes(path, name, Ms):
     cfg, W, gm, Wg, head = _weights(name)
     for M in Ms:
+        if not _supported(path, M):
+            continue
         hb = synth.make_hidden(cfg, M)
         head.set_path(path)
         out = ph.gpu_draft_numpy(head, hb, cfg.k_groups, cfg.k_tokens)
@@ -166,8 +182,9 @@ def test_paper_shapes(path, name, Ms):
 @pytest.mark.parametrize("path", PATHS)
 def test_qwen_shape_group_sweep_and_dense_equivalence(path):
     cfg, W, gm, Wg, head = _weights("qwen25_7b")
-    hb = synth.make_hidden(cfg, 60)
-    rows = np.array([0, 29, 59])
+    M = 60 if _supported(path, 60) else 8
+    hb = synth.make_hidden(cfg, M)
+    rows = np.array([0, M // 2, M - 1])
     for kg in (2, 4, 8, 16, 64):
         head.set_path(path)
         out = ph.gpu_draft_numpy(head, hb, kg, cfg.k_tokens)
