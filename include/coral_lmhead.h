@@ -46,7 +46,7 @@ extern "C" {
 
 /* Execution paths (coral_lmhead_set_path / coral_lmhead_stats.path). */
 #define CORAL_PATH_AUTO 0          /* chosen from (M, k_groups) */
-#define CORAL_PATH_SIMT 1          /* gathered GEMV, M <= 8: bulk-copy weight streaming + fp32 FMA */
+#define CORAL_PATH_STREAM 1        /* bulk-copy weight streaming + warp MMA (fp32 accumulate); M <= 128, H % 256 == 0, H <= 4096 */
 #define CORAL_PATH_TCGEN05 2       /* routed grouped GEMM on tcgen05 / TMEM tiles */
 #define CORAL_PATH_SIMT_PLAIN 3    /* gathered GEMV with plain 128-bit loads, any M */
 
@@ -150,7 +150,7 @@ int coral_lmhead_draft_host(coral_lmhead_handle h, const void *hidden_host, int 
 
 /*
  * Force an execution path (CORAL_PATH_*) for later draft calls; AUTO restores the default choice.
- * A draft call that the forced path cannot run (e.g. CORAL_PATH_SIMT with M > 8) returns
+ * A draft call that the forced path cannot run (e.g. CORAL_PATH_STREAM with M > 128) returns
  * CORAL_ERR_INVALID.
  */
 int coral_lmhead_set_path(coral_lmhead_handle h, int path);

@@ -15,12 +15,15 @@ constexpr int kNoToken = 0x7fffffff;
 struct DeviceState {
     int status;        // 0 or a CORAL_ERR_* code (first error wins)
     int n_union;       // groups touched by the last call
+    int n_virtual;     // (group, pass) entries of the union list; equals n_union when no group needs a second pass
 };
 
 // Per-call view of the workspace handed to the kernels.
 struct CallView {
     int M, H, V, N, v, T;          // T = tiles per group = ceil(v / kTileRows)
     int k_groups, k_tokens;
+    int union_cap;                 // capacity of union_list
+    int pass_rows;                 // rows of a group handled per pass over its weights (0: one pass for any count)
     const uint16_t* packed;        // [N][v][H] bf16, group-contiguous
     const uint16_t* w_gate;        // [N][H] bf16
     const int32_t* group_tokens;   // [N][v] global token id of packed row
@@ -33,8 +36,8 @@ struct CallView {
     int32_t* bucket_row;           // [M*k_groups] rows that selected a group, ascending per group
     int32_t* bucket_slot;          // [M*k_groups] the slot the group has in that row
     int32_t* bucket_pos;           // [M][k_groups] position of row m in the bucket of its slot's group
-    int32_t* union_list;           // [N] touched groups in ascending order (first n_union entries)
-    int32_t* union_rank;           // [N] index of group n in union_list, -1 if untouched
+    int32_t* union_list;           // [n_virtual] group | pass << 16, ascending (group, pass)
+    int32_t* union_rank;           // [N] index of (group n, pass 0) in union_list, -1 if untouched
     float* part_max;               // [M][k_groups][T]
     float* part_sum;               // [M][k_groups][T]
     float* part_val;               // [M][k_groups][T][k_tokens]

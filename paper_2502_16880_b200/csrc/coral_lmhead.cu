@@ -42,10 +42,12 @@ bool config_ok(const coral_lmhead_config* c) {
 // queried before a device is chosen), so it is sized for any grid in [kStreamGridMin, kStreamGridCap];
 // the launch geometry is fixed at create from the device's SM count and shared-memory limit.
 constexpr int kStreamGridMin = 64, kStreamGridCap = 160;
+constexpr int kStreamMaxPasses = kStreamMaxM / kStreamPassRows;
 
-int stream_seg_max(int n_groups, int T, int grid) {
-    const long per_max = ((long)n_groups * T + grid - 1) / grid;
-    return (int)((per_max + T - 1) / T) + 1;
+// Most (group, pass) entries a CTA's run of ceil(n_virtual * T / grid) items can overlap.
+int stream_seg_max(int n_groups, int grid) {
+    const long n_virtual_max = (long)n_groups * kStreamMaxPasses;
+    return (int)((n_virtual_max + grid - 1) / grid) + 1;
 }
 
 StreamGeom make_stream_geom(const coral_lmhead_config& c, int sms, int smem_optin) {
@@ -53,20 +55,19 @@ StreamGeom make_stream_geom(const coral_lmhead_config& c, int sms, int smem_opti
     const int v = c.V / c.n_groups;
     g.grid = sms < kStreamGridCap ? sms : kStreamGridCap;
     g.T = (v + kStreamTile - 1) / kStreamTile;
-    int sr = 1;
-    while (sr < kStreamTile && (size_t)(sr * 2) * c.H * 2 <= 16384) sr *= 2;
-    g.stage_rows = sr;
-    const size_t stage_bytes = (size_t)sr * c.H * 2;
-    const size_t fixed = sizeof(float) * (kStreamWarps * kStreamTile * kStreamMaxR + kStreamMaxR * kStreamTile) + 1024;
-    long ns = ((long)smem_optin - (long)fixed) / (long)stage_bytes;
-    g.n_stages = (int)(ns > 8 ? 8 : ns);
-    g.seg_max = stream_seg_max(c.n_groups, g.T, g.grid);
+    g.kc = (c.H % 512 == 0) ? 512 : 256;
+    g.kstages = c.H / g.kc;
+    g.row_stride = g.kc * 2 + kStreamRowPad;
+    g.stage_bytes = kStreamTile * g.row_stride;
+    const long fixed = (long)sizeof(float) * 2 * kStreamWarps * kStreamTile * kStreamPassRows + 1024;
+    long ns = ((long)smem_optin - fixed) / g.stage_bytes;
+    g.n_stages = (int)(ns > 12 ? 12 : ns);
+    g.seg_max = stream_seg_max(c.n_groups, g.grid);
     return g;
 }
 
-size_t stream_smem_bytes(const StreamGeom& g, int H) {
-    return (size_t)g.n_stages * g.stage_rows * H * 2 +
-           sizeof(float) * (kStreamWarps * kStreamTile * kStreamMaxR + kStreamMaxR * kStreamTile) +
+size_t stream_smem_bytes(const StreamGeom& g) {
+    return (size_t)g.n_stages * g.stage_bytes + sizeof(float) * 2 * kStreamWarps * kStreamTile * kStreamPassRows +
            sizeof(uint64_t) * 2 * g.n_stages + 16;
 }
 
@@ -90,15 +91,14 @@ Layout make_layout(const coral_lmhead_config& c) {
     L.bucket_row = take(M * kg * 4);
     L.bucket_slot = take(M * kg * 4);
     L.bucket_pos = take(M * kg * 4);
-    L.union_list = take(N * 4);
+    L.union_list = take(N * kStreamMaxPasses * 4);
     L.union_rank = take(N * 4);
-    const int T16 = (L.v + kStreamTile - 1) / kStreamTile;
-    const size_t sp = (size_t)kStreamGridCap * stream_seg_max(c.n_groups, T16, kStreamGridMin) * kStreamMaxR;
+    const size_t sp = (size_t)kStreamGridCap * stream_seg_max(c.n_groups, kStreamGridMin) * kStreamPassRows;
     L.sp_max = take(sp * 4);
     L.sp_sum = take(sp * 4);
     L.sp_val = take(sp * kt * 4);
     L.sp_id = take(sp * kt * 4);
-    const size_t cand_rows = M < (size_t)kStreamMaxR ? M : (size_t)kStreamMaxR;
+    const size_t cand_rows = M < (size_t)kStreamMaxM ? M : (size_t)kStreamMaxM;
     L.cand_cap = ((size_t)kStreamGridCap + 2 * kg) * kt;
     L.cand_val = take(cand_rows * L.cand_cap * 4);
     L.cand_id = take(cand_rows * L.cand_cap * 4);
@@ -163,6 +163,7 @@ CallView make_view(const coral_lmhead_s* h, const void* hidden, int M, int kg, i
     c.bucket_pos = reinterpret_cast<int32_t*>(ws + L.bucket_pos);
     c.union_list = reinterpret_cast<int32_t*>(ws + L.union_list);
     c.union_rank = reinterpret_cast<int32_t*>(ws + L.union_rank);
+    c.union_cap = h->cfg.n_groups * kStreamMaxPasses;
     c.part_max = reinterpret_cast<float*>(ws + L.part_max);
     c.part_sum = reinterpret_cast<float*>(ws + L.part_sum);
     c.part_val = reinterpret_cast<float*>(ws + L.part_val);
@@ -171,15 +172,15 @@ CallView make_view(const coral_lmhead_s* h, const void* hidden, int M, int kg, i
     return c;
 }
 
-bool stream_ok(const coral_lmhead_s* h, int M) { return h->stream_smem > 0 && M <= kStreamMaxR; }
+bool stream_ok(const coral_lmhead_s* h, int M) { return h->stream_smem > 0 && M <= kStreamMaxM; }
 
-// CORAL_PATH_SIMT: streaming kernel (needs M <= 8); CORAL_PATH_SIMT_PLAIN: any M.  Returns 0 if the
+// CORAL_PATH_STREAM: streaming kernel (M <= 128, H a multiple of 256, <= 4096); CORAL_PATH_SIMT_PLAIN: any shape.  Returns 0 if the
 // forced path cannot run this call.
 int choose_path(const coral_lmhead_s* h, int M, int kg) {
     (void)kg;
-    if (h->forced_path == CORAL_PATH_SIMT) return stream_ok(h, M) ? CORAL_PATH_SIMT : 0;
+    if (h->forced_path == CORAL_PATH_STREAM) return stream_ok(h, M) ? CORAL_PATH_STREAM : 0;
     if (h->forced_path != CORAL_PATH_AUTO) return h->forced_path;
-    return stream_ok(h, M) ? CORAL_PATH_SIMT : CORAL_PATH_SIMT_PLAIN;
+    return stream_ok(h, M) ? CORAL_PATH_STREAM : CORAL_PATH_SIMT_PLAIN;
 }
 
 }  // namespace
@@ -272,10 +273,12 @@ int coral_lmhead_create(coral_lmhead_handle* out, const coral_lmhead_config* cfg
         if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) { rc = CORAL_ERR_CUDA; break; }
         h->sg = make_stream_geom(*cfg, sms, smem_optin);
         h->stream_smem = 0;
-        if (cfg->H <= kStreamMaxH && sms >= kStreamGridMin && h->sg.n_stages >= 2) {
-            h->stream_smem = (int)stream_smem_bytes(h->sg, cfg->H);
-            if (cudaFuncSetAttribute(head_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_optin) !=
-                cudaSuccess) { rc = CORAL_ERR_CUDA; break; }
+        if (cfg->H <= kStreamMaxH && cfg->H % 256 == 0 && sms >= kStreamGridMin && h->sg.n_stages >= 2) {
+            h->stream_smem = (int)stream_smem_bytes(h->sg);
+            if (cudaFuncSetAttribute(head_stream_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_optin) !=
+                    cudaSuccess ||
+                cudaFuncSetAttribute(head_stream_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_optin) !=
+                    cudaSuccess) { rc = CORAL_ERR_CUDA; break; }
             if (cudaFuncSetAttribute(merge_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      kMergeSmemCands * 8) != cudaSuccess) { rc = CORAL_ERR_CUDA; break; }
         }
@@ -327,9 +330,10 @@ int coral_lmhead_draft_ex(coral_lmhead_handle h, const void* hidden_dev, int M, 
     if (k_tokens < 1 || k_tokens > cfg.max_k_tokens || (long long)k_tokens > (long long)k_groups * h->L.v)
         return CORAL_ERR_INVALID;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const CallView c = make_view(h, hidden_dev, M, k_groups, k_tokens);
+    CallView c = make_view(h, hidden_dev, M, k_groups, k_tokens);
     const int path = choose_path(h, M, k_groups);
     if (path == 0) return CORAL_ERR_INVALID;   // the forced path does not support this call
+    c.pass_rows = path == CORAL_PATH_STREAM ? kStreamPassRows : 0;
     int launches = 0;
 
     gate_kernel<<<dim3(c.N, (M + kGateRows - 1) / kGateRows), kGateThreads, 0, st>>>(c, out_gate_dev);
@@ -340,11 +344,14 @@ int coral_lmhead_draft_ex(coral_lmhead_handle h, const void* hidden_dev, int M, 
     bucket_kernel<<<1, kBucketThreads, 0, st>>>(c);
     ++launches;
     if (h->timing) cudaEventRecord(h->ev_head0, st);
-    if (path == CORAL_PATH_SIMT) {
+    if (path == CORAL_PATH_STREAM) {
         const Layout& L = h->L;
         StreamPartials pp{reinterpret_cast<float*>(h->ws + L.sp_max), reinterpret_cast<float*>(h->ws + L.sp_sum),
                           reinterpret_cast<float*>(h->ws + L.sp_val), reinterpret_cast<int32_t*>(h->ws + L.sp_id)};
-        head_stream_kernel<<<h->sg.grid, kStreamThreads, h->stream_smem, st>>>(c, h->sg, pp, out_logits_dev);
+        if (h->sg.kc == 512)
+            head_stream_kernel<2><<<h->sg.grid, kStreamThreads, h->stream_smem, st>>>(c, h->sg, pp, out_logits_dev);
+        else
+            head_stream_kernel<1><<<h->sg.grid, kStreamThreads, h->stream_smem, st>>>(c, h->sg, pp, out_logits_dev);
         ++launches;
         if (h->timing) cudaEventRecord(h->ev_head1, st);
         merge_stream_kernel<<<M, kMergeStreamThreads, kMergeSmemCands * 8, st>>>(

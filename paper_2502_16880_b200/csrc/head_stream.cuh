@@ -1,43 +1,51 @@
-// Gathered GEMV for few query rows (M <= 8), streaming version.
+// Gathered GEMV / small grouped GEMM for the draft step, streaming version.
 //
-// Every touched group's vocab rows are read exactly once: a producer thread
-// issues bulk asynchronous copies (cp.async.bulk, mbarrier completion) of whole
-// packed rows into a shared-memory ring; eight consumer warps split the hidden
-// dimension between them, keep their slice of the group's hidden rows in fp32
-// registers, and accumulate the dot products with fp32 FMAs.  Per 16-row item
-// the warps' partial sums are combined in shared memory, and one warp per
-// hidden row folds the 16 logits into a running (max, sum-exp, top-k) that is
-// written once per (CTA, group) segment.  (CORAL Section 3.3: logits only for
-// the activated groups, softmax over them; Appendix B: top candidates per row.)
+// Every touched group's vocab rows are read exactly once per pass: the producer
+// warp issues bulk asynchronous copies (cp.async.bulk, mbarrier completion) of
+// 16-row x kc-column slabs into a shared-memory ring; eight consumer warps split
+// each slab's columns between them and multiply it with their slice of the
+// group's hidden rows, which they keep in registers as bf16 MMA operands
+// (mma.sync m16n8k16, fp32 accumulators: vocab rows on the M axis, up to 16
+// hidden rows on the N axis).  Per 16-row item the warps' partial sums meet in
+// shared memory, and one warp per hidden row folds the 16 logits into a running
+// (max, sum-exp, top-k) that is written once per (CTA, group) segment.
+// (CORAL Section 3.3: logits only for the activated groups, softmax over them;
+// Appendix B: top candidates per row, union of the rows' groups.)
 //
-// Work split: the touched groups' rows form n_union * T items of 16 rows; CTA b
-// owns the contiguous run [b*per, (b+1)*per), so it changes group at most
-// seg_max - 1 times and all CTAs stream the same number of bytes.
+// A group selected by more than 16 rows is streamed in ceil(R/16) passes; each
+// (group, pass) is a "virtual group" of the union list.
+// Work split: the virtual groups' rows form n_virtual * T items of 16 rows; CTA b
+// owns the contiguous run [b*per, (b+1)*per), so all CTAs stream the same bytes.
 #pragma once
 #include "common.cuh"
 
 namespace coral {
 
-constexpr int kStreamTile = 16;                 // vocab rows per item
+constexpr int kStreamTile = 16;                 // vocab rows per item (the MMA's M)
 constexpr int kStreamWarps = 8;                 // consumer warps
 constexpr int kStreamConsumers = kStreamWarps * 32;
 constexpr int kStreamThreads = 32 + kStreamConsumers;   // warp 0 = producer
-constexpr int kStreamMaxR = 8;                  // hidden rows per group on this path (M <= 8)
-constexpr int kStreamMaxH = 4096;               // two 16-byte chunks per consumer thread
+constexpr int kStreamPassRows = 16;             // hidden rows per pass (two n-tiles of 8)
+constexpr int kStreamMaxH = 4096;               // 16 k-blocks of 32 columns per warp
+constexpr int kStreamMaxM = 128;                // beyond this the pass count makes the path pointless
+constexpr int kStreamRowPad = 64;               // bytes after each slab row: rows alternate bank halves
 constexpr int kStreamSpin = 1 << 20;            // bound of every mbarrier wait
 constexpr int kStreamSpinAfterAbort = 1 << 8;
 
 struct StreamGeom {
     int grid;         // CTAs launched
-    int stage_rows;   // vocab rows per ring stage (divides kStreamTile)
+    int kc;           // columns per slab (512, or 256 when H is not a multiple of 512)
+    int kstages;      // slabs per item = H / kc
     int n_stages;     // ring depth
-    int seg_max;      // most groups one CTA's run can overlap
+    int seg_max;      // most virtual groups one CTA's run can overlap
     int T;            // items per group = ceil(v / kStreamTile)
+    int row_stride;   // bytes between slab rows in shared memory = kc * 2 + kStreamRowPad
+    int stage_bytes;  // kStreamTile * row_stride
 };
 
-// One partial per (CTA, segment, hidden row of the group).
+// One partial per (CTA, segment, hidden row of the pass).
 struct StreamPartials {
-    float* pmax;      // [grid][seg_max][kStreamMaxR]
+    float* pmax;      // [grid][seg_max][kStreamPassRows]
     float* psum;
     float* pval;      // [...][k_tokens]
     int32_t* pid;
@@ -81,164 +89,185 @@ __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t
 }
 __device__ __forceinline__ void consumer_bar() { asm volatile("bar.sync 1, %0;" ::"n"(kStreamConsumers) : "memory"); }
 
-__device__ __forceinline__ void unpack8(const uint4& q, float* f) {
-    f[0] = bf16_lo(q.x); f[1] = bf16_hi(q.x); f[2] = bf16_lo(q.y); f[3] = bf16_hi(q.y);
-    f[4] = bf16_lo(q.z); f[5] = bf16_hi(q.z); f[6] = bf16_lo(q.w); f[7] = bf16_hi(q.w);
+
+__device__ __forceinline__ uint4 lds128(uint32_t addr) {
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+    return v;
+}
+
+// D += A(16x16, bf16, row) * B(16x8, bf16, col), fp32 accumulate.
+__device__ __forceinline__ void mma_bf16_16816(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                               uint32_t b0, uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
+        "{%0, %1, %2, %3};"
+        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
 struct StreamShared {
     unsigned char* ring;      // n_stages * stage_bytes
-    float* zpart;             // [kStreamWarps][kStreamTile][kStreamMaxR]
-    float* z;                 // [kStreamMaxR][kStreamTile]
+    float* zpart;             // [2][kStreamWarps][kStreamTile][kStreamPassRows]
     uint64_t* full;           // [n_stages]
     uint64_t* empty;          // [n_stages]
     volatile int* abort_flag;
 };
 
-// Consumer side of one segment: items [lo, hi) of the run, all inside union group j (group n, R hidden rows).
-template <int R>
+// Fold the 16 logits of one item (lane i < rows holds z of tile row i and its token id) into a warp's
+// running statistics of one hidden row: online max / sum-exp and the sorted top-k list (entry i in lane i).
+__device__ __forceinline__ void fold_item(float zv, int tok, bool have, int k_tokens, int lane, float& run_max,
+                                          float& run_sum, float& lv, int& lid) {
+    const float tmax = warp_max(zv);
+    const float nmax = fmaxf(run_max, tmax);
+    const float add = warp_sum(have ? __expf(zv - nmax) : 0.f);
+    run_sum = run_sum * __expf(run_max - nmax) + add;     // exp(-inf) = 0 on the first item
+    run_max = nmax;
+    const float kth = __shfl_sync(0xffffffffu, lv, k_tokens - 1);
+    const int kth_id = __shfl_sync(0xffffffffu, lid, k_tokens - 1);
+    if (kth_id == kNoToken || tmax >= kth) {
+        float a = lv, b = zv;
+        int ai = lid, bi = tok;
+        float ov = kNegInf;
+        int oi = kNoToken;
+        for (int k = 0; k < k_tokens; ++k) {
+            float bv;
+            int bk;
+            if (better(a, ai, b, bi)) { bv = a; bk = ai; } else { bv = b; bk = bi; }
+            warp_argbest(bv, bk);
+            if (bk != kNoToken) {
+                if (ai == bk) { a = kNegInf; ai = kNoToken; }
+                if (bi == bk) { b = kNegInf; bi = kNoToken; }
+            }
+            if (lane == k) { ov = bv; oi = bk; }
+        }
+        lv = ov;
+        lid = oi;
+    }
+}
+
+// Consumer side of one segment: items [lo, hi) of the run, all inside virtual group j = (group n, pass).
+// NT n-tiles of 8 hidden rows; KBW k-blocks (32 columns) per warp per slab.
+template <int NT, int KBW>
 __device__ __forceinline__ void stream_segment(const CallView& c, const StreamGeom& g, const StreamShared& sh,
                                                const StreamPartials& pp, float* __restrict__ logits_tap, int n,
-                                               int j, int lo, int hi, int seg, int& stage, uint32_t& phase) {
+                                               int pass, int R, int j, int lo, int hi, int seg, int& stage,
+                                               uint32_t& phase, int& zbuf) {
+    constexpr int KSMAX = 16 / KBW;
     const int ct = threadIdx.x - 32, cw = ct >> 5, lane = ct & 31;
-    const int chunks = c.H >> 3;
-    const int off = c.group_offset[n];
-    const bool v0 = ct < chunks, v1 = ct + kStreamConsumers < chunks;
-    const int stage_bytes = g.stage_rows * c.H * 2;
-    const int row_bytes = c.H * 2;
+    const int gq = lane >> 2, tq = lane & 3;
+    const int off = c.group_offset[n] + pass * kStreamPassRows;
+    const int col0 = (cw * KBW) * 32 + tq * 8;          // first column of this lane inside a slab
 
-    float hreg[R][16];
+    // B operands: hidden row (nt*8 + gq), the lane's 8 columns of every k-block of this warp
+    uint4 breg[NT][16];
 #pragma unroll
-    for (int r = 0; r < R; ++r) {
-        const uint4* hp = reinterpret_cast<const uint4*>(c.hidden + (size_t)c.bucket_row[off + r] * c.H);
-        uint4 q0 = make_uint4(0, 0, 0, 0), q1 = make_uint4(0, 0, 0, 0);
-        if (v0) q0 = __ldg(hp + ct);
-        if (v1) q1 = __ldg(hp + ct + kStreamConsumers);
-        unpack8(q0, &hreg[r][0]);
-        unpack8(q1, &hreg[r][8]);
+    for (int nt = 0; nt < NT; ++nt) {
+        const int rr = nt * 8 + gq;
+        const bool valid = rr < R;
+        const uint16_t* hp = c.hidden + (size_t)(valid ? c.bucket_row[off + rr] : 0) * c.H;
+#pragma unroll
+        for (int ks = 0; ks < KSMAX; ++ks)
+#pragma unroll
+            for (int i = 0; i < KBW; ++i) {
+                uint4 q = make_uint4(0, 0, 0, 0);
+                if (valid && ks < g.kstages) q = __ldg(reinterpret_cast<const uint4*>(hp + ks * g.kc + col0 + i * 32));
+                breg[nt][ks * KBW + i] = q;
+            }
     }
-    // running statistics of hidden row r = cw (warps cw < R); list entry i lives in lane i
-    float run_max = kNegInf, run_sum = 0.f, lv = kNegInf;
-    int lid = kNoToken;
-    const int my_m = (cw < R) ? c.bucket_row[off + cw] : 0;
-    const int my_slot = (cw < R) ? c.bucket_slot[off + cw] : 0;
+    // running statistics: warp cw owns hidden rows cw and cw + 8 of the pass
+    float run_max[NT], run_sum[NT], lv[NT];
+    int lid[NT], my_m[NT], my_slot[NT];
+#pragma unroll
+    for (int q = 0; q < NT; ++q) {
+        run_max[q] = kNegInf; run_sum[q] = 0.f; lv[q] = kNegInf; lid[q] = kNoToken;
+        const int r = cw + 8 * q;
+        my_m[q] = r < R ? c.bucket_row[off + r] : 0;
+        my_slot[q] = r < R ? c.bucket_slot[off + r] : 0;
+    }
+    const uint32_t ring = smem_u32(sh.ring);
 
     for (int item = lo; item < hi; ++item) {
-        const int t = item - j * g.T;
-        const int row0 = t * kStreamTile;
+        const int row0 = (item - j * g.T) * kStreamTile;
         const int rows = min(kStreamTile, c.v - row0);
-        for (int s0 = 0; s0 < rows; s0 += g.stage_rows) {
-            const int nrows = min(g.stage_rows, rows - s0);
-            mbar_wait(smem_u32(&sh.full[stage]), phase, sh.abort_flag, c.state);
-            const unsigned char* sp = sh.ring + (size_t)stage * stage_bytes;
-            for (int rr = 0; rr < nrows; rr += 2) {
-                const bool two = rr + 1 < nrows;
-                float acc0[R], acc1[R];
+        float acc[NT][2][4];
 #pragma unroll
-                for (int r = 0; r < R; ++r) { acc0[r] = 0.f; acc1[r] = 0.f; }
-                const uint4* w0p = reinterpret_cast<const uint4*>(sp + (size_t)rr * row_bytes);
-                const uint4* w1p = reinterpret_cast<const uint4*>(sp + (size_t)(rr + (two ? 1 : 0)) * row_bytes);
-                if (v0) {
-                    float a[8], b[8];
-                    unpack8(w0p[ct], a);
-                    unpack8(w1p[ct], b);
+        for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
-                    for (int r = 0; r < R; ++r)
+            for (int e = 0; e < 4; ++e) { acc[nt][0][e] = 0.f; acc[nt][1][e] = 0.f; }
 #pragma unroll
-                        for (int e = 0; e < 8; ++e) {
-                            acc0[r] = fmaf(a[e], hreg[r][e], acc0[r]);
-                            acc1[r] = fmaf(b[e], hreg[r][e], acc1[r]);
-                        }
-                }
-                if (v1) {
-                    float a[8], b[8];
-                    unpack8(w0p[ct + kStreamConsumers], a);
-                    unpack8(w1p[ct + kStreamConsumers], b);
+        for (int ks = 0; ks < KSMAX; ++ks) {
+            if (ks < g.kstages) {
+                mbar_wait(smem_u32(&sh.full[stage]), phase, sh.abort_flag, c.state);
+                const uint32_t sp = ring + (uint32_t)stage * g.stage_bytes;
 #pragma unroll
-                    for (int r = 0; r < R; ++r)
+                for (int i = 0; i < KBW; ++i) {
+                    const uint32_t cb = (uint32_t)(col0 + i * 32) * 2;
+                    const uint4 wg = lds128(sp + gq * g.row_stride + cb);
+                    const uint4 wh = lds128(sp + (gq + 8) * g.row_stride + cb);
 #pragma unroll
-                        for (int e = 0; e < 8; ++e) {
-                            acc0[r] = fmaf(a[e], hreg[r][8 + e], acc0[r]);
-                            acc1[r] = fmaf(b[e], hreg[r][8 + e], acc1[r]);
-                        }
-                }
-#pragma unroll
-                for (int r = 0; r < R; ++r) {
-                    const float s0v = warp_sum(acc0[r]);
-                    const float s1v = warp_sum(acc1[r]);
-                    if (lane == 0) {
-                        sh.zpart[(cw * kStreamTile + s0 + rr) * kStreamMaxR + r] = s0v;
-                        if (two) sh.zpart[(cw * kStreamTile + s0 + rr + 1) * kStreamMaxR + r] = s1v;
+                    for (int nt = 0; nt < NT; ++nt) {
+                        const uint4 b = breg[nt][ks * KBW + i];
+                        mma_bf16_16816(acc[nt][0], wg.x, wh.x, wg.y, wh.y, b.x, b.y);
+                        mma_bf16_16816(acc[nt][1], wg.z, wh.z, wg.w, wh.w, b.z, b.w);
                     }
                 }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&sh.empty[stage]));
+                if (++stage == g.n_stages) { stage = 0; phase ^= 1u; }
             }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&sh.empty[stage]));
-            if (++stage == g.n_stages) { stage = 0; phase ^= 1u; }
         }
-        consumer_bar();
-        if (ct < R * kStreamTile) {
-            const int r = ct / kStreamTile, row = ct - r * kStreamTile;
-            float s = 0.f;
+        // this warp's partial sums over its columns: rows gq, gq+8; hidden rows nt*8 + 2*tq, +1
+        float* zp = sh.zpart + ((size_t)(zbuf * kStreamWarps + cw) * kStreamTile) * kStreamPassRows;
 #pragma unroll
-            for (int w = 0; w < kStreamWarps; ++w) s += sh.zpart[(w * kStreamTile + row) * kStreamMaxR + r];
-            sh.z[r * kStreamTile + row] = s;
+        for (int nt = 0; nt < NT; ++nt) {
+            *reinterpret_cast<float2*>(zp + gq * kStreamPassRows + nt * 8 + 2 * tq) =
+                make_float2(acc[nt][0][0] + acc[nt][1][0], acc[nt][0][1] + acc[nt][1][1]);
+            *reinterpret_cast<float2*>(zp + (gq + 8) * kStreamPassRows + nt * 8 + 2 * tq) =
+                make_float2(acc[nt][0][2] + acc[nt][1][2], acc[nt][0][3] + acc[nt][1][3]);
         }
         consumer_bar();
-        if (cw < R) {
-            const bool have = lane < rows;
-            const float zv = have ? sh.z[cw * kStreamTile + lane] : kNegInf;
-            const int tok = have ? __ldg(c.group_tokens + (size_t)n * c.v + row0 + lane) : kNoToken;
-            if (logits_tap && have) logits_tap[((size_t)my_m * c.k_groups + my_slot) * c.v + row0 + lane] = zv;
-            const float tmax = warp_max(zv);
-            const float nmax = fmaxf(run_max, tmax);
-            const float add = warp_sum(have ? __expf(zv - nmax) : 0.f);
-            run_sum = run_sum * __expf(run_max - nmax) + add;     // exp(-inf) = 0 on the first item
-            run_max = nmax;
-            const float kth = __shfl_sync(0xffffffffu, lv, c.k_tokens - 1);
-            const int kth_id = __shfl_sync(0xffffffffu, lid, c.k_tokens - 1);
-            if (kth_id == kNoToken || tmax >= kth) {
-                // merge the sorted list (lane i: entry i) with the new values (lane i: row i)
-                float a = lv, b = zv;
-                int ai = lid, bi = tok;
-                float ov = kNegInf;
-                int oi = kNoToken;
-                for (int k = 0; k < c.k_tokens; ++k) {
-                    float bv;
-                    int bk;
-                    if (better(a, ai, b, bi)) { bv = a; bk = ai; } else { bv = b; bk = bi; }
-                    warp_argbest(bv, bk);
-                    if (bk != kNoToken) {
-                        if (ai == bk) { a = kNegInf; ai = kNoToken; }
-                        if (bi == bk) { b = kNegInf; bi = kNoToken; }
-                    }
-                    if (lane == k) { ov = bv; oi = bk; }
+        const bool have = lane < rows;
+        const int tok = have ? __ldg(c.group_tokens + (size_t)n * c.v + row0 + lane) : kNoToken;
+#pragma unroll
+        for (int q = 0; q < NT; ++q) {
+            const int r = cw + 8 * q;
+            if (r < R) {
+                float zv = kNegInf;
+                if (have) {
+                    const float* zr = sh.zpart + ((size_t)(zbuf * kStreamWarps) * kStreamTile + lane) * kStreamPassRows + r;
+                    zv = 0.f;
+#pragma unroll
+                    for (int w = 0; w < kStreamWarps; ++w) zv += zr[(size_t)w * kStreamTile * kStreamPassRows];
+                    if (logits_tap) logits_tap[((size_t)my_m[q] * c.k_groups + my_slot[q]) * c.v + row0 + lane] = zv;
                 }
-                lv = ov;
-                lid = oi;
+                fold_item(zv, tok, have, c.k_tokens, lane, run_max[q], run_sum[q], lv[q], lid[q]);
             }
         }
+        zbuf ^= 1;
     }
-    if (cw < R) {
-        const size_t p = ((size_t)blockIdx.x * g.seg_max + seg) * kStreamMaxR + cw;
-        if (lane == 0) { pp.pmax[p] = run_max; pp.psum[p] = run_sum; }
-        if (lane < c.k_tokens) { pp.pval[p * c.k_tokens + lane] = lv; pp.pid[p * c.k_tokens + lane] = lid; }
+#pragma unroll
+    for (int q = 0; q < NT; ++q) {
+        const int r = cw + 8 * q;
+        if (r < R) {
+            const size_t p = ((size_t)blockIdx.x * g.seg_max + seg) * kStreamPassRows + r;
+            if (lane == 0) { pp.pmax[p] = run_max[q]; pp.psum[p] = run_sum[q]; }
+            if (lane < c.k_tokens) { pp.pval[p * c.k_tokens + lane] = lv[q]; pp.pid[p * c.k_tokens + lane] = lid[q]; }
+        }
     }
 }
 
 // grid = g.grid CTAs of kStreamThreads threads; dynamic shared memory laid out as StreamShared.
+template <int KBW>
 __global__ void __launch_bounds__(kStreamThreads, 1) head_stream_kernel(CallView c, StreamGeom g, StreamPartials pp,
                                                                         float* __restrict__ logits_tap) {
     extern __shared__ __align__(128) unsigned char stream_smem_raw[];
     unsigned char* smem_raw = stream_smem_raw;
-    const int stage_bytes = g.stage_rows * c.H * 2;
     StreamShared sh;
     sh.ring = smem_raw;
-    size_t o = (size_t)g.n_stages * stage_bytes;
+    size_t o = (size_t)g.n_stages * g.stage_bytes;
     sh.zpart = reinterpret_cast<float*>(smem_raw + o);
-    o += sizeof(float) * kStreamWarps * kStreamTile * kStreamMaxR;
-    sh.z = reinterpret_cast<float*>(smem_raw + o);
-    o += sizeof(float) * kStreamMaxR * kStreamTile;
+    o += sizeof(float) * 2 * kStreamWarps * kStreamTile * kStreamPassRows;
     sh.full = reinterpret_cast<uint64_t*>(smem_raw + o);
     o += sizeof(uint64_t) * g.n_stages;
     sh.empty = reinterpret_cast<uint64_t*>(smem_raw + o);
@@ -256,57 +285,54 @@ __global__ void __launch_bounds__(kStreamThreads, 1) head_stream_kernel(CallView
     }
     __syncthreads();
 
-    const int n_union = c.state->n_union;
-    const int n_items = n_union * g.T;
+    const int n_items = c.state->n_virtual * g.T;
     const int per = (n_items + g.grid - 1) / g.grid;
     const int lo = min(n_items, (int)blockIdx.x * per);
     const int hi = min(n_items, lo + per);
     if (lo >= hi) return;
 
     if (threadIdx.x < 32) {
-        if (threadIdx.x != 0) return;
-        // producer: one bulk copy per ring stage, rows of one group are contiguous in the packed copy
+        // producer warp: lane 0 waits for the slot and posts the byte count, lanes < rows copy one slab row each
+        const int lane = threadIdx.x;
         int stage = 0;
         uint32_t phase = 0;
+        const uint32_t row_bytes = (uint32_t)g.kc * 2;
         for (int item = lo; item < hi; ++item) {
-            const int j = item / g.T, t = item - j * g.T;
-            const int n = c.union_list[j];
-            const int row0 = t * kStreamTile;
+            const int j = item / g.T;
+            const int n = c.union_list[j] & 0xffff;
+            const int row0 = (item - j * g.T) * kStreamTile;
             const int rows = min(kStreamTile, c.v - row0);
-            for (int s0 = 0; s0 < rows; s0 += g.stage_rows) {
-                const int nrows = min(g.stage_rows, rows - s0);
-                mbar_wait(smem_u32(&sh.empty[stage]), phase ^ 1u, sh.abort_flag, c.state);
-                const uint32_t bytes = (uint32_t)nrows * c.H * 2;
+            const uint16_t* src = c.packed + ((size_t)n * c.v + row0 + lane) * c.H;
+            for (int ks = 0; ks < g.kstages; ++ks) {
                 const uint32_t bar = smem_u32(&sh.full[stage]);
-                mbar_expect_tx(bar, bytes);
-                bulk_g2s(smem_u32(sh.ring + (size_t)stage * stage_bytes),
-                         c.packed + ((size_t)n * c.v + row0 + s0) * c.H, bytes, bar);
+                if (lane == 0) {
+                    mbar_wait(smem_u32(&sh.empty[stage]), phase ^ 1u, sh.abort_flag, c.state);
+                    mbar_expect_tx(bar, (uint32_t)rows * row_bytes);
+                }
+                __syncwarp();
+                if (lane < rows)
+                    bulk_g2s(smem_u32(sh.ring + (size_t)stage * g.stage_bytes + (size_t)lane * g.row_stride),
+                             src + (size_t)ks * g.kc, row_bytes, bar);
                 if (++stage == g.n_stages) { stage = 0; phase ^= 1u; }
             }
         }
         return;
     }
 
-    // consumers: walk the run segment by segment (one union group each)
-    int stage = 0;
+    // consumers: walk the run segment by segment (one virtual group each)
+    int stage = 0, zbuf = 0;
     uint32_t phase = 0;
     const int j_first = lo / g.T;
     for (int pos = lo; pos < hi;) {
         const int j = pos / g.T;
         const int seg_hi = min(hi, (j + 1) * g.T);
-        const int n = c.union_list[j];
-        const int R = min(c.group_count[n], kStreamMaxR);
-        const int seg = j - j_first;
-        switch (R) {
-            case 1: stream_segment<1>(c, g, sh, pp, logits_tap, n, j, pos, seg_hi, seg, stage, phase); break;
-            case 2: stream_segment<2>(c, g, sh, pp, logits_tap, n, j, pos, seg_hi, seg, stage, phase); break;
-            case 3: stream_segment<3>(c, g, sh, pp, logits_tap, n, j, pos, seg_hi, seg, stage, phase); break;
-            case 4: stream_segment<4>(c, g, sh, pp, logits_tap, n, j, pos, seg_hi, seg, stage, phase); break;
-            case 5: stream_segment<5>(c, g, sh, pp, logits_tap, n, j, pos, seg_hi, seg, stage, phase); break;
-            case 6: stream_segment<6>(c, g, sh, pp, logits_tap, n, j, pos, seg_hi, seg, stage, phase); break;
-            case 7: stream_segment<7>(c, g, sh, pp, logits_tap, n, j, pos, seg_hi, seg, stage, phase); break;
-            default: stream_segment<8>(c, g, sh, pp, logits_tap, n, j, pos, seg_hi, seg, stage, phase); break;
-        }
+        const int entry = c.union_list[j];
+        const int n = entry & 0xffff, pass = entry >> 16;
+        const int R = min(c.group_count[n] - pass * kStreamPassRows, kStreamPassRows);
+        if (R <= 8)
+            stream_segment<1, KBW>(c, g, sh, pp, logits_tap, n, pass, R, j, pos, seg_hi, j - j_first, stage, phase, zbuf);
+        else
+            stream_segment<2, KBW>(c, g, sh, pp, logits_tap, n, pass, R, j, pos, seg_hi, j - j_first, stage, phase, zbuf);
         pos = seg_hi;
     }
 }
@@ -330,18 +356,18 @@ __global__ void __launch_bounds__(kMergeStreamThreads) merge_stream_kernel(CallV
     __shared__ float s_lse;
     __shared__ int s_first[kMaxGroups], s_cnt[kMaxGroups], s_base[kMaxGroups + 1], s_rpos[kMaxGroups], s_j[kMaxGroups];
 
-    const int n_union = c.state->n_union;
-    const int n_items = n_union * g.T;
+    const int n_items = c.state->n_virtual * g.T;
     const int per = (n_items + g.grid - 1) / g.grid;
     for (int s = threadIdx.x; s < c.k_groups; s += kMergeStreamThreads) {
         const int n = c.sel[(size_t)m * c.k_groups + s];
-        const int j = c.union_rank[n];
+        const int pos_in_bucket = c.bucket_pos[(size_t)m * c.k_groups + s];
+        const int j = c.union_rank[n] + pos_in_bucket / kStreamPassRows;
         const int fb = (j * g.T) / per;
         const int lb = ((j + 1) * g.T - 1) / per;
         s_first[s] = fb;
         s_cnt[s] = lb - fb + 1;
         s_j[s] = j;
-        s_rpos[s] = c.bucket_pos[(size_t)m * c.k_groups + s];
+        s_rpos[s] = pos_in_bucket % kStreamPassRows;
     }
     __syncthreads();
     if (threadIdx.x == 0) {
@@ -363,7 +389,7 @@ __global__ void __launch_bounds__(kMergeStreamThreads) merge_stream_kernel(CallV
         while (s + 1 < c.k_groups && s_base[s + 1] <= q) ++s;
         const int b = s_first[s] + (q - s_base[s]);
         const int seg = s_j[s] - (b * per) / g.T;
-        const size_t p = ((size_t)b * g.seg_max + seg) * kStreamMaxR + s_rpos[s];
+        const size_t p = ((size_t)b * g.seg_max + seg) * kStreamPassRows + s_rpos[s];
         mx = fmaxf(mx, pp.pmax[p]);
         for (int i = 0; i < c.k_tokens; ++i) {
             cv[q * c.k_tokens + i] = pp.pval[p * c.k_tokens + i];
@@ -383,7 +409,7 @@ __global__ void __launch_bounds__(kMergeStreamThreads) merge_stream_kernel(CallV
         while (s + 1 < c.k_groups && s_base[s + 1] <= q) ++s;
         const int b = s_first[s] + (q - s_base[s]);
         const int seg = s_j[s] - (b * per) / g.T;
-        const size_t p = ((size_t)b * g.seg_max + seg) * kStreamMaxR + s_rpos[s];
+        const size_t p = ((size_t)b * g.seg_max + seg) * kStreamPassRows + s_rpos[s];
         sum += pp.psum[p] * expf(pp.pmax[p] - mx);
     }
     sum = warp_sum(sum);

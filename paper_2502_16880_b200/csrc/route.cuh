@@ -121,18 +121,22 @@ __global__ void __launch_bounds__(kBucketThreads) bucket_kernel(CallView c) {
     }
     __syncthreads();
     if (threadIdx.x == 0) {
-        int run = 0, uni = 0;
+        int run = 0, uni = 0, virt = 0;
         for (int n = 0; n < c.N; ++n) {
             s_offset[n] = run;
             run += s_count[n];
-            if (c.union_rank) c.union_rank[n] = s_count[n] > 0 ? uni : -1;
+            if (c.union_rank) c.union_rank[n] = s_count[n] > 0 ? virt : -1;
             if (s_count[n] > 0) {
-                if (c.union_list) c.union_list[uni] = n;
+                const int passes = c.pass_rows > 0 ? (s_count[n] + c.pass_rows - 1) / c.pass_rows : 1;
+                for (int p = 0; p < passes; ++p)
+                    if (c.union_list && virt + p < c.union_cap) c.union_list[virt + p] = n | (p << 16);
+                virt += passes;
                 ++uni;
             }
         }
         s_offset[c.N] = run;
         c.state->n_union = uni;
+        c.state->n_virtual = min(virt, c.union_cap);
     }
     __syncthreads();
     for (int n = threadIdx.x; n <= c.N; n += kBucketThreads) {

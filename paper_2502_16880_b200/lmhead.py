@@ -25,7 +25,7 @@ CORAL_ERR_TIMEOUT = -5
 CORAL_ERR_BOUNDS = -6
 CORAL_ERR_TOO_LARGE = -7
 CORAL_ROUTE_STATIC_MAX_ROWS = 64
-CORAL_PATH_AUTO, CORAL_PATH_SIMT, CORAL_PATH_TCGEN05, CORAL_PATH_SIMT_PLAIN = 0, 1, 2, 3
+CORAL_PATH_AUTO, CORAL_PATH_STREAM, CORAL_PATH_TCGEN05, CORAL_PATH_SIMT_PLAIN = 0, 1, 2, 3
 
 
 class coral_lmhead_config(ctypes.Structure):

@@ -8,11 +8,11 @@ from tests import parity_harness as ph
 
 pytestmark = pytest.mark.gpu
 
-PATHS = [lmhead.CORAL_PATH_SIMT, lmhead.CORAL_PATH_SIMT_PLAIN]
+PATHS = [lmhead.CORAL_PATH_STREAM, lmhead.CORAL_PATH_SIMT_PLAIN]
 
 
-def _supported(path, M):
-    return path != lmhead.CORAL_PATH_SIMT or M <= 8
+def _supported(path, M, H=256):
+    return path != lmhead.CORAL_PATH_STREAM or (M <= 128 and H % 256 == 0 and H <= 4096)
 
 
 
@@ -30,13 +30,13 @@ def _weights(name):
         _cache.clear()
         cfg = synth.CONFIGS[name]
         W, gm, Wg = synth.make_w_vocab(cfg), synth.make_group_map(cfg), synth.make_w_gate(cfg)
-        _cache[name] = (cfg, W, gm, Wg, _head(cfg, W, gm, Wg, max_M=max(cfg.M, 64)))
+        _cache[name] = (cfg, W, gm, Wg, _head(cfg, W, gm, Wg, max_M=max(cfg.M, 128)))
     return _cache[name]
 
 
 def _check(head, W, gm, Wg, hb, kg, kt, path, forced=None):
-    if not _supported(path, hb.shape[0]):
-        pytest.skip("streaming path takes M <= 8")
+    if not _supported(path, hb.shape[0], hb.shape[1]):
+        pytest.skip("streaming path takes M <= 128 and H a multiple of 256")
     head.set_path(path)
     out = ph.gpu_draft_numpy(head, hb, kg, kt, forced_groups=forced)
     assert head.status() == 0
@@ -46,7 +46,8 @@ def _check(head, W, gm, Wg, hb, kg, kt, path, forced=None):
 
 
 @pytest.mark.parametrize("path", PATHS)
-@pytest.mark.parametrize("M,kg,kt", [(4, 4, 10), (1, 1, 1), (1, 4, 10), (3, 16, 32), (16, 2, 10), (40, 16, 7)])
+@pytest.mark.parametrize("M,kg,kt", [(4, 4, 10), (1, 1, 1), (1, 4, 10), (3, 16, 32), (16, 2, 10), (40, 16, 7),
+                                     (128, 3, 10), (9, 16, 10), (17, 16, 5)])
 def test_tiny(path, M, kg, kt):
     cfg, W, gm, Wg, head = _weights("tiny")
     hb = synth.make_hidden(cfg, M)
@@ -59,8 +60,9 @@ def test_tiny(path, M, kg, kt):
 @pytest.mark.parametrize("path", PATHS)
 def test_ragged_shape(path):
     # v = 300 (two full tiles + a tail of 44), H = 328 (not a multiple of 256)
-    cfg = synth.HeadConfig("ragged", H=328, V=1800, N=6, k_groups=3, k_tokens=10,
-                           M=13 if path != lmhead.CORAL_PATH_SIMT else 7, seed=5, w_std=0.05)
+    # v = 300 is 18 items of 16 rows + a tail of 12; H = 328 only runs on the plain path, H = 768 on both
+    H = 328 if path == lmhead.CORAL_PATH_SIMT_PLAIN else 768
+    cfg = synth.HeadConfig("ragged", H=H, V=1800, N=6, k_groups=3, k_tokens=10, M=13, seed=5, w_std=0.05)
     W, gm, Wg, hb = synth.make_all(cfg)
     head = _head(cfg, W, gm, Wg)
     for kg, kt in [(3, 10), (6, 32), (1, 5)]:
@@ -71,7 +73,7 @@ def test_ragged_shape(path):
 @pytest.mark.parametrize("path", PATHS)
 def test_small_group_fewer_rows_than_k_tokens(path):
     # v = 6 < k_tokens: per-tile candidate lists are padded
-    cfg = synth.HeadConfig("small_v", H=64, V=48, N=8, k_groups=4, k_tokens=20, M=5, seed=9, w_std=0.3)
+    cfg = synth.HeadConfig("small_v", H=256, V=48, N=8, k_groups=4, k_tokens=20, M=5, seed=9, w_std=0.3)
     W, gm, Wg, hb = synth.make_all(cfg)
     head = _head(cfg, W, gm, Wg)
     _check(head, W, gm, Wg, hb, 4, 20, path)
@@ -90,7 +92,7 @@ def test_forced_groups(path):
 
 @pytest.mark.parametrize("path", PATHS)
 def test_exact_ties_zero_weights(path):
-    cfg = synth.HeadConfig("zeros", H=64, V=640, N=5, k_groups=2, k_tokens=10, M=3, seed=1)
+    cfg = synth.HeadConfig("zeros", H=256, V=640, N=5, k_groups=2, k_tokens=10, M=3, seed=1)
     gm, hb = synth.make_group_map(cfg), synth.make_hidden(cfg)
     W = np.zeros((cfg.V, cfg.H), np.uint16)
     Wg = np.zeros((cfg.N, cfg.H), np.uint16)
@@ -106,7 +108,7 @@ def test_exact_ties_zero_weights(path):
 @pytest.mark.parametrize("path", PATHS)
 def test_deterministic_bitwise(path):
     cfg, W, gm, Wg, head = _weights("tiny")
-    hb = synth.make_hidden(cfg, 33 if path != lmhead.CORAL_PATH_SIMT else 8)
+    hb = synth.make_hidden(cfg, 33)
     head.set_path(path)
     a = ph.gpu_draft_numpy(head, hb, 4, 10)
     b = ph.gpu_draft_numpy(head, hb, 4, 10)
@@ -131,11 +133,15 @@ def test_argument_errors_return_codes():
     assert lib.coral_lmhead_draft(head.handle, hp, 4, 4, 10, None, lp, None) == lmhead.CORAL_ERR_INVALID
     assert lib.coral_lmhead_draft(None, hp, 4, 4, 10, ip, lp, None) == lmhead.CORAL_ERR_INVALID
     # a forced path that cannot take the call is refused, not silently replaced
-    h9 = ph.to_dev_bf16(synth.make_hidden(cfg, 9))
-    head.set_path(lmhead.CORAL_PATH_SIMT)
-    assert lib.coral_lmhead_draft(head.handle, ctypes.c_void_p(h9.data_ptr()), 9, 4, 10, ip, lp, None) == \
+    big = lmhead.LMHead(ph.to_dev_bf16(W), torch.from_numpy(gm), ph.to_dev_bf16(Wg), 200, 4, 10)
+    h200 = ph.to_dev_bf16(synth.make_hidden(cfg, 200))
+    i200 = torch.empty((200, 10), dtype=torch.int32, device="cuda")
+    l200 = torch.empty((200, 10), dtype=torch.float32, device="cuda")
+    big.set_path(lmhead.CORAL_PATH_STREAM)
+    assert lib.coral_lmhead_draft(big.handle, ctypes.c_void_p(h200.data_ptr()), 200, 4, 10,
+                                  ctypes.c_void_p(i200.data_ptr()), ctypes.c_void_p(l200.data_ptr()), None) == \
         lmhead.CORAL_ERR_INVALID
-    head.set_path(lmhead.CORAL_PATH_AUTO)
+    big.close()
     # unequal groups are rejected at create, before anything touches the device
     bad = gm.copy()
     bad[0] = (bad[0] + 1) % cfg.N
@@ -165,8 +171,6 @@ def test_library_owned_buffers_and_host_entry():
 def test_paper_shapes(path, name, Ms):
     cfg, W, gm, Wg, head = _weights(name)
     for M in Ms:
-        if not _supported(path, M):
-            continue
         hb = synth.make_hidden(cfg, M)
         head.set_path(path)
         out = ph.gpu_draft_numpy(head, hb, cfg.k_groups, cfg.k_tokens)
@@ -182,7 +186,7 @@ def test_paper_shapes(path, name, Ms):
 @pytest.mark.parametrize("path", PATHS)
 def test_qwen_shape_group_sweep_and_dense_equivalence(path):
     cfg, W, gm, Wg, head = _weights("qwen25_7b")
-    M = 60 if _supported(path, 60) else 8
+    M = 60
     hb = synth.make_hidden(cfg, M)
     rows = np.array([0, M // 2, M - 1])
     for kg in (2, 4, 8, 16, 64):
