@@ -24,7 +24,8 @@ struct CallView {
     int k_groups, k_tokens;
     int union_cap;                 // capacity of union_list
     int pass_rows;                 // rows of a group handled per pass over its weights (0: one pass for any count)
-    const uint16_t* packed;        // [N][v][H] bf16, group-contiguous
+    const uint16_t* packed;        // blocked copy of W_vocab, see packed_chunk_offset
+    int kc, kstages, swz, T16;     // packed layout: columns per slab, slabs per row, chunk swizzle, 16-row items per group
     const uint16_t* w_gate;        // [N][H] bf16
     const int32_t* group_tokens;   // [N][v] global token id of packed row
     const uint16_t* hidden;        // [M][H] bf16
@@ -44,6 +45,20 @@ struct CallView {
     int32_t* part_id;              // [M][k_groups][T][k_tokens]
     DeviceState* state;
 };
+
+// Packed layout of the LM head: per group, per item of 16 vocab rows (ascending token id), per slab of kc
+// columns: a contiguous [16 rows][kc] bf16 block, so that one slab is one contiguous bulk copy.  With swz
+// the 16-byte chunks of odd rows have bit 2 of their index flipped (the two 64-byte halves of every 128
+// bytes swapped), which keeps 128-bit shared-memory reads of two adjacent rows on disjoint banks.
+// Returns the offset, in 16-byte units, of logical chunk `ch` (8 columns) of row `j` of group `n`.
+__host__ __device__ __forceinline__ size_t packed_chunk_offset(int n, int j, int ch, int kc, int kstages, int swz,
+                                                               int T16) {
+    const int cpr = kc >> 3;                       // chunks per slab row
+    const int ks = ch / cpr, cc = ch - ks * cpr;
+    const int item = j >> 4, r = j & 15;
+    const int phys = swz ? (cc ^ ((r & 1) << 2)) : cc;
+    return ((((size_t)n * T16 + item) * kstages + ks) * 16 + r) * cpr + phys;
+}
 
 __device__ __forceinline__ float bf16_lo(uint32_t u) { return __uint_as_float(u << 16); }
 __device__ __forceinline__ float bf16_hi(uint32_t u) { return __uint_as_float(u & 0xffff0000u); }

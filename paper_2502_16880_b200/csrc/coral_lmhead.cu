@@ -27,6 +27,7 @@ struct Layout {
         cand_val, cand_id, stage_hidden, stage_ids, stage_logprobs, total;
     size_t packed_bytes, cand_cap;
     int v, T;
+    int kc, kstages, swz, T16;   // packed layout (see packed_chunk_offset)
 };
 
 bool config_ok(const coral_lmhead_config* c) {
@@ -57,9 +58,9 @@ StreamGeom make_stream_geom(const coral_lmhead_config& c, int sms, int smem_opti
     g.T = (v + kStreamTile - 1) / kStreamTile;
     g.kc = (c.H % 512 == 0) ? 512 : 256;
     g.kstages = c.H / g.kc;
-    g.row_stride = g.kc * 2 + kStreamRowPad;
+    g.row_stride = g.kc * 2;
     g.stage_bytes = kStreamTile * g.row_stride;
-    const long fixed = (long)sizeof(float) * 2 * kStreamWarps * kStreamTile * kStreamPassRows + 1024;
+    const long fixed = (long)sizeof(float) * kStreamZBufs * kStreamWarps * kStreamTile * kStreamPassRows + 1024;
     long ns = ((long)smem_optin - fixed) / g.stage_bytes;
     g.n_stages = (int)(ns > 12 ? 12 : ns);
     g.seg_max = stream_seg_max(c.n_groups, g.grid);
@@ -67,8 +68,10 @@ StreamGeom make_stream_geom(const coral_lmhead_config& c, int sms, int smem_opti
 }
 
 size_t stream_smem_bytes(const StreamGeom& g) {
-    return (size_t)g.n_stages * g.stage_bytes + sizeof(float) * 2 * kStreamWarps * kStreamTile * kStreamPassRows +
-           sizeof(uint64_t) * 2 * g.n_stages + 16;
+    return (size_t)g.n_stages * g.stage_bytes +
+           sizeof(float) * kStreamZBufs * kStreamWarps * kStreamTile * kStreamPassRows +
+           sizeof(uint64_t) * 2 * g.n_stages + sizeof(uint64_t) * 2 * kStreamZBufs +
+           sizeof(int) * kStreamSegTab + 16;
 }
 
 constexpr int kMergeSmemCands = 4096;   // candidates the streaming merge keeps in shared memory
@@ -110,17 +113,23 @@ Layout make_layout(const coral_lmhead_config& c) {
     L.stage_ids = take(M * kt * 4);
     L.stage_logprobs = take(M * kt * 4);
     L.total = o;
-    L.packed_bytes = (size_t)c.V * H * 2;
+    L.T16 = (L.v + 15) / 16;
+    L.kc = (c.H % 512 == 0) ? 512 : (c.H % 256 == 0) ? 256 : c.H;
+    L.kstages = c.H / L.kc;
+    L.swz = (L.kc % 64 == 0) ? 1 : 0;
+    L.packed_bytes = (size_t)c.n_groups * L.T16 * 16 * H * 2;
     return L;
 }
 
-// packed[n][i][:] = W_vocab[group_tokens[n][i]][:]; one block per packed row.
+// Row i of group n of the packed copy = W_vocab[group_tokens[n][i]], in the blocked layout; one block per row.
 __global__ void pack_rows_kernel(const uint16_t* __restrict__ W, const int32_t* __restrict__ group_tokens,
-                                 uint16_t* __restrict__ packed, int H) {
-    const size_t row = blockIdx.x;
+                                 uint16_t* __restrict__ packed, int H, int v, int kc, int kstages, int swz, int T16) {
+    const int row = blockIdx.x;
+    const int n = row / v, j = row - n * v;
     const uint4* src = reinterpret_cast<const uint4*>(W + (size_t)group_tokens[row] * H);
-    uint4* dst = reinterpret_cast<uint4*>(packed + row * H);
-    for (int ch = threadIdx.x; ch < (H >> 3); ch += blockDim.x) dst[ch] = __ldg(src + ch);
+    uint4* dst = reinterpret_cast<uint4*>(packed);
+    for (int ch = threadIdx.x; ch < (H >> 3); ch += blockDim.x)
+        dst[packed_chunk_offset(n, j, ch, kc, kstages, swz, T16)] = __ldg(src + ch);
 }
 
 }  // namespace
@@ -150,6 +159,7 @@ CallView make_view(const coral_lmhead_s* h, const void* hidden, int M, int kg, i
     c.M = M; c.H = h->cfg.H; c.V = h->cfg.V; c.N = h->cfg.n_groups; c.v = L.v; c.T = L.T;
     c.k_groups = kg; c.k_tokens = kt;
     c.packed = reinterpret_cast<const uint16_t*>(h->packed);
+    c.kc = L.kc; c.kstages = L.kstages; c.swz = L.swz; c.T16 = L.T16;
     c.w_gate = reinterpret_cast<const uint16_t*>(ws + L.w_gate);
     c.group_tokens = reinterpret_cast<const int32_t*>(ws + L.group_tokens);
     c.hidden = reinterpret_cast<const uint16_t*>(hidden);
@@ -289,7 +299,8 @@ int coral_lmhead_create(coral_lmhead_handle* out, const coral_lmhead_config* cfg
         if (cudaMemsetAsync(h->ws + h->L.state, 0, sizeof(DeviceState), st) != cudaSuccess) { rc = CORAL_ERR_CUDA; break; }
         pack_rows_kernel<<<V, 128, 0, st>>>(static_cast<const uint16_t*>(W_vocab_dev),
                                             reinterpret_cast<const int32_t*>(h->ws + h->L.group_tokens),
-                                            reinterpret_cast<uint16_t*>(h->packed), cfg->H);
+                                            reinterpret_cast<uint16_t*>(h->packed), cfg->H, v, h->L.kc, h->L.kstages,
+                                            h->L.swz, h->L.T16);
         if (cudaGetLastError() != cudaSuccess) { rc = CORAL_ERR_CUDA; break; }
         if (cudaStreamSynchronize(st) != cudaSuccess) { rc = CORAL_ERR_CUDA; break; }
     } while (0);

@@ -60,17 +60,17 @@ __device__ __forceinline__ void tile_partials(const CallView& c, const float* z,
 }
 
 template <int R>
-__device__ __forceinline__ void simt_tile_dots(const uint16_t* __restrict__ wt, const uint16_t* hs, float* zs,
+__device__ __forceinline__ void simt_tile_dots(const CallView& c, int n, int row0, const uint16_t* hs, float* zs,
                                                int rows, int H, int warp, int lane) {
     const int chunks = H >> 3;
+    const uint4* __restrict__ wbase = reinterpret_cast<const uint4*>(c.packed);
     for (int j = warp; j < rows; j += kSimtWarps) {
-        const uint4* __restrict__ wrow = reinterpret_cast<const uint4*>(wt + (size_t)j * H);
         float acc[R];
 #pragma unroll
         for (int r = 0; r < R; ++r) acc[r] = 0.f;
 #pragma unroll 4
         for (int ch = lane; ch < chunks; ch += 32) {
-            const uint4 w = __ldg(wrow + ch);
+            const uint4 w = __ldg(wbase + packed_chunk_offset(n, row0 + j, ch, c.kc, c.kstages, c.swz, c.T16));
 #pragma unroll
             for (int r = 0; r < R; ++r)
                 acc[r] = dot8(w, *reinterpret_cast<const uint4*>(hs + (size_t)r * H + ch * 8), acc[r]);
@@ -95,7 +95,6 @@ __global__ void __launch_bounds__(kSimtThreads) head_simt_kernel(CallView c, flo
     const int off = c.group_offset[n];
     const int row0 = t * kTileRows;
     const int rows = min(kTileRows, c.v - row0);
-    const uint16_t* __restrict__ wt = c.packed + ((size_t)n * c.v + row0) * c.H;
     const int32_t* __restrict__ tokens = c.group_tokens + (size_t)n * c.v + row0;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int chunks = c.H >> 3;
@@ -110,14 +109,14 @@ __global__ void __launch_bounds__(kSimtThreads) head_simt_kernel(CallView c, flo
         }
         __syncthreads();
         switch (rb) {
-            case 1: simt_tile_dots<1>(wt, hs, zs, rows, c.H, warp, lane); break;
-            case 2: simt_tile_dots<2>(wt, hs, zs, rows, c.H, warp, lane); break;
-            case 3: simt_tile_dots<3>(wt, hs, zs, rows, c.H, warp, lane); break;
-            case 4: simt_tile_dots<4>(wt, hs, zs, rows, c.H, warp, lane); break;
-            case 5: simt_tile_dots<5>(wt, hs, zs, rows, c.H, warp, lane); break;
-            case 6: simt_tile_dots<6>(wt, hs, zs, rows, c.H, warp, lane); break;
-            case 7: simt_tile_dots<7>(wt, hs, zs, rows, c.H, warp, lane); break;
-            default: simt_tile_dots<8>(wt, hs, zs, rows, c.H, warp, lane); break;
+            case 1: simt_tile_dots<1>(c, n, row0, hs, zs, rows, c.H, warp, lane); break;
+            case 2: simt_tile_dots<2>(c, n, row0, hs, zs, rows, c.H, warp, lane); break;
+            case 3: simt_tile_dots<3>(c, n, row0, hs, zs, rows, c.H, warp, lane); break;
+            case 4: simt_tile_dots<4>(c, n, row0, hs, zs, rows, c.H, warp, lane); break;
+            case 5: simt_tile_dots<5>(c, n, row0, hs, zs, rows, c.H, warp, lane); break;
+            case 6: simt_tile_dots<6>(c, n, row0, hs, zs, rows, c.H, warp, lane); break;
+            case 7: simt_tile_dots<7>(c, n, row0, hs, zs, rows, c.H, warp, lane); break;
+            default: simt_tile_dots<8>(c, n, row0, hs, zs, rows, c.H, warp, lane); break;
         }
         __syncthreads();
         for (int r = warp; r < rb; r += kSimtWarps) {

@@ -1,14 +1,17 @@
 // Gathered GEMV / small grouped GEMM for the draft step, streaming version.
 //
-// Every touched group's vocab rows are read exactly once per pass: the producer
-// warp issues bulk asynchronous copies (cp.async.bulk, mbarrier completion) of
-// 16-row x kc-column slabs into a shared-memory ring; eight consumer warps split
-// each slab's columns between them and multiply it with their slice of the
+// Every touched group's vocab rows are read exactly once per pass: a producer
+// warp issues one bulk asynchronous copy (cp.async.bulk, mbarrier completion)
+// per 16-row x kc-column slab (16 KiB, contiguous in the packed layout) into a
+// shared-memory ring.  Eight MMA warps split each slab's columns between them and
+// multiply it with their slice of the
 // group's hidden rows, which they keep in registers as bf16 MMA operands
 // (mma.sync m16n8k16, fp32 accumulators: vocab rows on the M axis, up to 16
-// hidden rows on the N axis).  Per 16-row item the warps' partial sums meet in
-// shared memory, and one warp per hidden row folds the 16 logits into a running
-// (max, sum-exp, top-k) that is written once per (CTA, group) segment.
+// hidden rows on the N axis).  Per 16-row item the MMA warps drop their partial
+// sums into one of four shared-memory buffers and carry on; three further warps
+// pick the buffers up, add the eight partials and fold the 16 logits of every
+// hidden row into a running (max, sum-exp, top-k) that is written once per
+// (CTA, group) segment.  The MMA warps therefore never wait for the statistics.
 // (CORAL Section 3.3: logits only for the activated groups, softmax over them;
 // Appendix B: top candidates per row, union of the rows' groups.)
 //
@@ -22,13 +25,14 @@
 namespace coral {
 
 constexpr int kStreamTile = 16;                 // vocab rows per item (the MMA's M)
-constexpr int kStreamWarps = 8;                 // consumer warps
-constexpr int kStreamConsumers = kStreamWarps * 32;
-constexpr int kStreamThreads = 32 + kStreamConsumers;   // warp 0 = producer
+constexpr int kStreamWarps = 8;                 // MMA warps (warps 0..7)
+constexpr int kStreamStatWarps = 3;             // statistics warps (warps 8..10); warp 11 is the producer
+constexpr int kStreamThreads = (kStreamWarps + kStreamStatWarps + 1) * 32;
+constexpr int kStreamZBufs = 4;                 // buffers of per-item partial sums between the two roles
+constexpr int kStreamSegTab = 64;               // capacity of the per-CTA segment table
 constexpr int kStreamPassRows = 16;             // hidden rows per pass (two n-tiles of 8)
 constexpr int kStreamMaxH = 4096;               // 16 k-blocks of 32 columns per warp
 constexpr int kStreamMaxM = 128;                // beyond this the pass count makes the path pointless
-constexpr int kStreamRowPad = 64;               // bytes after each slab row: rows alternate bank halves
 constexpr int kStreamSpin = 1 << 20;            // bound of every mbarrier wait
 constexpr int kStreamSpinAfterAbort = 1 << 8;
 
@@ -39,8 +43,8 @@ struct StreamGeom {
     int n_stages;     // ring depth
     int seg_max;      // most virtual groups one CTA's run can overlap
     int T;            // items per group = ceil(v / kStreamTile)
-    int row_stride;   // bytes between slab rows in shared memory = kc * 2 + kStreamRowPad
-    int stage_bytes;  // kStreamTile * row_stride
+    int row_stride;   // bytes between slab rows = kc * 2
+    int stage_bytes;  // kStreamTile * row_stride: one slab, contiguous in the packed copy
 };
 
 // One partial per (CTA, segment, hidden row of the pass).
@@ -87,7 +91,6 @@ __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                  ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
 }
-__device__ __forceinline__ void consumer_bar() { asm volatile("bar.sync 1, %0;" ::"n"(kStreamConsumers) : "memory"); }
 
 
 __device__ __forceinline__ uint4 lds128(uint32_t addr) {
@@ -108,16 +111,20 @@ __device__ __forceinline__ void mma_bf16_16816(float (&d)[4], uint32_t a0, uint3
 
 struct StreamShared {
     unsigned char* ring;      // n_stages * stage_bytes
-    float* zpart;             // [2][kStreamWarps][kStreamTile][kStreamPassRows]
-    uint64_t* full;           // [n_stages]
-    uint64_t* empty;          // [n_stages]
+    float* zpart;             // [kStreamZBufs][kStreamWarps][kStreamTile][kStreamPassRows]
+    uint64_t* full;           // [n_stages] completion of the copy into a slot
+    uint64_t* empty;          // [n_stages] all MMA warps have finished reading the slot
+    uint64_t* zfull;          // [kStreamZBufs] all MMA warps have written the buffer
+    uint64_t* zfree;          // [kStreamZBufs] all statistics warps have read the buffer
+    int* segtab;              // [kStreamSegTab] union_list entries of this CTA's run
     volatile int* abort_flag;
+    int lo, hi, j_first;      // this CTA's run of items and its first virtual group
 };
 
 // Fold the 16 logits of one item (lane i < rows holds z of tile row i and its token id) into a warp's
 // running statistics of one hidden row: online max / sum-exp and the sorted top-k list (entry i in lane i).
-__device__ __forceinline__ void fold_item(float zv, int tok, bool have, int k_tokens, int lane, float& run_max,
-                                          float& run_sum, float& lv, int& lid) {
+__device__ __forceinline__ void fold_item(float zv, const int32_t* __restrict__ tokens, bool have, int k_tokens,
+                                          int lane, float& run_max, float& run_sum, float& lv, int& lid) {
     const float tmax = warp_max(zv);
     const float nmax = fmaxf(run_max, tmax);
     const float add = warp_sum(have ? __expf(zv - nmax) : 0.f);
@@ -127,7 +134,7 @@ __device__ __forceinline__ void fold_item(float zv, int tok, bool have, int k_to
     const int kth_id = __shfl_sync(0xffffffffu, lid, k_tokens - 1);
     if (kth_id == kNoToken || tmax >= kth) {
         float a = lv, b = zv;
-        int ai = lid, bi = tok;
+        int ai = lid, bi = have ? __ldg(tokens + lane) : kNoToken;
         float ov = kNegInf;
         int oi = kNoToken;
         for (int k = 0; k < k_tokens; ++k) {
@@ -146,15 +153,14 @@ __device__ __forceinline__ void fold_item(float zv, int tok, bool have, int k_to
     }
 }
 
-// Consumer side of one segment: items [lo, hi) of the run, all inside virtual group j = (group n, pass).
-// NT n-tiles of 8 hidden rows; KBW k-blocks (32 columns) per warp per slab.
+// MMA side of one segment: items [lo, hi) of the run, all inside virtual group j = (group n, pass) with R
+// hidden rows.  NT n-tiles of 8 hidden rows; KBW k-blocks (32 columns) per warp per slab.
 template <int NT, int KBW>
-__device__ __forceinline__ void stream_segment(const CallView& c, const StreamGeom& g, const StreamShared& sh,
-                                               const StreamPartials& pp, float* __restrict__ logits_tap, int n,
-                                               int pass, int R, int j, int lo, int hi, int seg, int& stage,
-                                               uint32_t& phase, int& zbuf) {
+__device__ __forceinline__ void stream_segment_mma(const CallView& c, const StreamGeom& g, const StreamShared& sh,
+                                                   int n, int pass, int R, int lo, int hi, int& stage,
+                                                   uint32_t& phase, int& it) {
     constexpr int KSMAX = 16 / KBW;
-    const int ct = threadIdx.x - 32, cw = ct >> 5, lane = ct & 31;
+    const int cw = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int gq = lane >> 2, tq = lane & 3;
     const int off = c.group_offset[n] + pass * kStreamPassRows;
     const int col0 = (cw * KBW) * 32 + tq * 8;          // first column of this lane inside a slab
@@ -170,26 +176,14 @@ __device__ __forceinline__ void stream_segment(const CallView& c, const StreamGe
         for (int ks = 0; ks < KSMAX; ++ks)
 #pragma unroll
             for (int i = 0; i < KBW; ++i) {
-                uint4 q = make_uint4(0, 0, 0, 0);
-                if (valid && ks < g.kstages) q = __ldg(reinterpret_cast<const uint4*>(hp + ks * g.kc + col0 + i * 32));
-                breg[nt][ks * KBW + i] = q;
+                uint4 hv = make_uint4(0, 0, 0, 0);
+                if (valid && ks < g.kstages) hv = __ldg(reinterpret_cast<const uint4*>(hp + ks * g.kc + col0 + i * 32));
+                breg[nt][ks * KBW + i] = hv;
             }
-    }
-    // running statistics: warp cw owns hidden rows cw and cw + 8 of the pass
-    float run_max[NT], run_sum[NT], lv[NT];
-    int lid[NT], my_m[NT], my_slot[NT];
-#pragma unroll
-    for (int q = 0; q < NT; ++q) {
-        run_max[q] = kNegInf; run_sum[q] = 0.f; lv[q] = kNegInf; lid[q] = kNoToken;
-        const int r = cw + 8 * q;
-        my_m[q] = r < R ? c.bucket_row[off + r] : 0;
-        my_slot[q] = r < R ? c.bucket_slot[off + r] : 0;
     }
     const uint32_t ring = smem_u32(sh.ring);
 
-    for (int item = lo; item < hi; ++item) {
-        const int row0 = (item - j * g.T) * kStreamTile;
-        const int rows = min(kStreamTile, c.v - row0);
+    for (int item = lo; item < hi; ++item, ++it) {
         float acc[NT][2][4];
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt)
@@ -202,7 +196,7 @@ __device__ __forceinline__ void stream_segment(const CallView& c, const StreamGe
                 const uint32_t sp = ring + (uint32_t)stage * g.stage_bytes;
 #pragma unroll
                 for (int i = 0; i < KBW; ++i) {
-                    const uint32_t cb = (uint32_t)(col0 + i * 32) * 2;
+                    const uint32_t cb = ((uint32_t)(col0 + i * 32) * 2) ^ ((uint32_t)(gq & 1) << 6);   // chunk swizzle
                     const uint4 wg = lds128(sp + gq * g.row_stride + cb);
                     const uint4 wh = lds128(sp + (gq + 8) * g.row_stride + cb);
 #pragma unroll
@@ -218,7 +212,9 @@ __device__ __forceinline__ void stream_segment(const CallView& c, const StreamGe
             }
         }
         // this warp's partial sums over its columns: rows gq, gq+8; hidden rows nt*8 + 2*tq, +1
-        float* zp = sh.zpart + ((size_t)(zbuf * kStreamWarps + cw) * kStreamTile) * kStreamPassRows;
+        const int zb = it % kStreamZBufs;
+        mbar_wait(smem_u32(&sh.zfree[zb]), ((uint32_t)(it / kStreamZBufs) & 1u) ^ 1u, sh.abort_flag, c.state);
+        float* zp = sh.zpart + ((size_t)(zb * kStreamWarps + cw) * kStreamTile) * kStreamPassRows;
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt) {
             *reinterpret_cast<float2*>(zp + gq * kStreamPassRows + nt * 8 + 2 * tq) =
@@ -226,33 +222,66 @@ __device__ __forceinline__ void stream_segment(const CallView& c, const StreamGe
             *reinterpret_cast<float2*>(zp + (gq + 8) * kStreamPassRows + nt * 8 + 2 * tq) =
                 make_float2(acc[nt][0][2] + acc[nt][1][2], acc[nt][0][3] + acc[nt][1][3]);
         }
-        consumer_bar();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&sh.zfull[zb]));
+    }
+}
+
+// Statistics side of one segment.  Warp sw (0..2) owns hidden rows sw, sw+3, sw+6, ... of the pass.
+__device__ __forceinline__ void stream_segment_stats(const CallView& c, const StreamGeom& g, const StreamShared& sh,
+                                                     const StreamPartials& pp, float* __restrict__ logits_tap, int n,
+                                                     int pass, int R, int j, int lo, int hi, int seg, int& it) {
+    constexpr int kOwn = (kStreamPassRows + kStreamStatWarps - 1) / kStreamStatWarps;
+    const int sw = (threadIdx.x >> 5) - kStreamWarps, lane = threadIdx.x & 31;
+    const int off = c.group_offset[n] + pass * kStreamPassRows;
+    float run_max[kOwn], run_sum[kOwn], lv[kOwn];
+    int lid[kOwn], my_m[kOwn], my_slot[kOwn];
+#pragma unroll
+    for (int u = 0; u < kOwn; ++u) {
+        run_max[u] = kNegInf; run_sum[u] = 0.f; lv[u] = kNegInf; lid[u] = kNoToken;
+        const int r = sw + kStreamStatWarps * u;
+        my_m[u] = r < R ? c.bucket_row[off + r] : 0;
+        my_slot[u] = r < R ? c.bucket_slot[off + r] : 0;
+    }
+    for (int item = lo; item < hi; ++item, ++it) {
+        const int row0 = (item - j * g.T) * kStreamTile;
+        const int rows = min(kStreamTile, c.v - row0);
         const bool have = lane < rows;
-        const int tok = have ? __ldg(c.group_tokens + (size_t)n * c.v + row0 + lane) : kNoToken;
+        const int32_t* tokens = c.group_tokens + (size_t)n * c.v + row0;
+        const int zb = it % kStreamZBufs;
+        mbar_wait(smem_u32(&sh.zfull[zb]), (uint32_t)(it / kStreamZBufs) & 1u, sh.abort_flag, c.state);
+        float zv[kOwn];
 #pragma unroll
-        for (int q = 0; q < NT; ++q) {
-            const int r = cw + 8 * q;
-            if (r < R) {
-                float zv = kNegInf;
-                if (have) {
-                    const float* zr = sh.zpart + ((size_t)(zbuf * kStreamWarps) * kStreamTile + lane) * kStreamPassRows + r;
-                    zv = 0.f;
+        for (int u = 0; u < kOwn; ++u) {
+            const int r = sw + kStreamStatWarps * u;
+            zv[u] = kNegInf;
+            if (r < R && have) {
+                const float* zr = sh.zpart + ((size_t)(zb * kStreamWarps) * kStreamTile + lane) * kStreamPassRows + r;
+                float z = 0.f;
 #pragma unroll
-                    for (int w = 0; w < kStreamWarps; ++w) zv += zr[(size_t)w * kStreamTile * kStreamPassRows];
-                    if (logits_tap) logits_tap[((size_t)my_m[q] * c.k_groups + my_slot[q]) * c.v + row0 + lane] = zv;
-                }
-                fold_item(zv, tok, have, c.k_tokens, lane, run_max[q], run_sum[q], lv[q], lid[q]);
+                for (int w = 0; w < kStreamWarps; ++w) z += zr[(size_t)w * kStreamTile * kStreamPassRows];
+                zv[u] = z;
             }
         }
-        zbuf ^= 1;
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&sh.zfree[zb]));      // the buffer is in registers now
+#pragma unroll
+        for (int u = 0; u < kOwn; ++u) {
+            const int r = sw + kStreamStatWarps * u;
+            if (r < R) {
+                if (logits_tap && have)
+                    logits_tap[((size_t)my_m[u] * c.k_groups + my_slot[u]) * c.v + row0 + lane] = zv[u];
+                fold_item(zv[u], tokens, have, c.k_tokens, lane, run_max[u], run_sum[u], lv[u], lid[u]);
+            }
+        }
     }
 #pragma unroll
-    for (int q = 0; q < NT; ++q) {
-        const int r = cw + 8 * q;
+    for (int u = 0; u < kOwn; ++u) {
+        const int r = sw + kStreamStatWarps * u;
         if (r < R) {
             const size_t p = ((size_t)blockIdx.x * g.seg_max + seg) * kStreamPassRows + r;
-            if (lane == 0) { pp.pmax[p] = run_max[q]; pp.psum[p] = run_sum[q]; }
-            if (lane < c.k_tokens) { pp.pval[p * c.k_tokens + lane] = lv[q]; pp.pid[p * c.k_tokens + lane] = lid[q]; }
+            if (lane == 0) { pp.pmax[p] = run_max[u]; pp.psum[p] = run_sum[u]; }
+            if (lane < c.k_tokens) { pp.pval[p * c.k_tokens + lane] = lv[u]; pp.pid[p * c.k_tokens + lane] = lid[u]; }
         }
     }
 }
@@ -267,72 +296,88 @@ __global__ void __launch_bounds__(kStreamThreads, 1) head_stream_kernel(CallView
     sh.ring = smem_raw;
     size_t o = (size_t)g.n_stages * g.stage_bytes;
     sh.zpart = reinterpret_cast<float*>(smem_raw + o);
-    o += sizeof(float) * 2 * kStreamWarps * kStreamTile * kStreamPassRows;
+    o += sizeof(float) * kStreamZBufs * kStreamWarps * kStreamTile * kStreamPassRows;
     sh.full = reinterpret_cast<uint64_t*>(smem_raw + o);
     o += sizeof(uint64_t) * g.n_stages;
+    sh.zfull = reinterpret_cast<uint64_t*>(smem_raw + o);
+    o += sizeof(uint64_t) * kStreamZBufs;
+    sh.zfree = reinterpret_cast<uint64_t*>(smem_raw + o);
+    o += sizeof(uint64_t) * kStreamZBufs;
     sh.empty = reinterpret_cast<uint64_t*>(smem_raw + o);
     o += sizeof(uint64_t) * g.n_stages;
+    sh.segtab = reinterpret_cast<int*>(smem_raw + o);
+    o += sizeof(int) * kStreamSegTab;
     sh.abort_flag = reinterpret_cast<volatile int*>(smem_raw + o);
+
+    const int n_items = c.state->n_virtual * g.T;
+    const int per = (n_items + g.grid - 1) / g.grid;
+    sh.lo = min(n_items, (int)blockIdx.x * per);
+    sh.hi = min(n_items, sh.lo + per);
+    if (sh.lo >= sh.hi) return;
+    sh.j_first = sh.lo / g.T;
+    const int n_segs = min((sh.hi - 1) / g.T - sh.j_first + 1, kStreamSegTab);
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < g.n_stages; ++s) {
             mbar_init(smem_u32(&sh.full[s]), 1);
             mbar_init(smem_u32(&sh.empty[s]), kStreamWarps);
         }
+        for (int b = 0; b < kStreamZBufs; ++b) {
+            mbar_init(smem_u32(&sh.zfull[b]), kStreamWarps);
+            mbar_init(smem_u32(&sh.zfree[b]), kStreamStatWarps);
+        }
         *sh.abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
+    if (threadIdx.x < n_segs) sh.segtab[threadIdx.x] = c.union_list[sh.j_first + threadIdx.x];
     __syncthreads();
 
-    const int n_items = c.state->n_virtual * g.T;
-    const int per = (n_items + g.grid - 1) / g.grid;
-    const int lo = min(n_items, (int)blockIdx.x * per);
-    const int hi = min(n_items, lo + per);
-    if (lo >= hi) return;
-
-    if (threadIdx.x < 32) {
-        // producer warp: lane 0 waits for the slot and posts the byte count, lanes < rows copy one slab row each
-        const int lane = threadIdx.x;
+    const int cw = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (cw == kStreamWarps + kStreamStatWarps) {
+        // producer: one contiguous copy per slab; a slab's valid rows are a prefix of its 16 rows
+        if (lane != 0) return;
         int stage = 0;
         uint32_t phase = 0;
-        const uint32_t row_bytes = (uint32_t)g.kc * 2;
-        for (int item = lo; item < hi; ++item) {
-            const int j = item / g.T;
-            const int n = c.union_list[j] & 0xffff;
-            const int row0 = (item - j * g.T) * kStreamTile;
-            const int rows = min(kStreamTile, c.v - row0);
-            const uint16_t* src = c.packed + ((size_t)n * c.v + row0 + lane) * c.H;
-            for (int ks = 0; ks < g.kstages; ++ks) {
-                const uint32_t bar = smem_u32(&sh.full[stage]);
-                if (lane == 0) {
+        for (int pos = sh.lo; pos < sh.hi;) {
+            const int j = pos / g.T;
+            const int seg_hi = min(sh.hi, (j + 1) * g.T);
+            const int n = sh.segtab[min(j - sh.j_first, kStreamSegTab - 1)] & 0xffff;
+            int t = pos - j * g.T;
+            const uint16_t* src = c.packed + ((((size_t)n * g.T + t) * g.kstages) * kStreamTile) * g.kc;
+            for (int item = pos; item < seg_hi; ++item, ++t) {
+                const uint32_t bytes = (uint32_t)min(kStreamTile, c.v - t * kStreamTile) * g.row_stride;
+                for (int ks = 0; ks < g.kstages; ++ks) {
                     mbar_wait(smem_u32(&sh.empty[stage]), phase ^ 1u, sh.abort_flag, c.state);
-                    mbar_expect_tx(bar, (uint32_t)rows * row_bytes);
+                    const uint32_t bar = smem_u32(&sh.full[stage]);
+                    mbar_expect_tx(bar, bytes);
+                    bulk_g2s(smem_u32(sh.ring + (size_t)stage * g.stage_bytes), src, bytes, bar);
+                    src += (size_t)kStreamTile * g.kc;
+                    if (++stage == g.n_stages) { stage = 0; phase ^= 1u; }
                 }
-                __syncwarp();
-                if (lane < rows)
-                    bulk_g2s(smem_u32(sh.ring + (size_t)stage * g.stage_bytes + (size_t)lane * g.row_stride),
-                             src + (size_t)ks * g.kc, row_bytes, bar);
-                if (++stage == g.n_stages) { stage = 0; phase ^= 1u; }
             }
+            pos = seg_hi;
         }
         return;
     }
+    const bool mma_role = cw < kStreamWarps;
 
-    // consumers: walk the run segment by segment (one virtual group each)
-    int stage = 0, zbuf = 0;
+    // both roles walk the run segment by segment (one virtual group each)
+    int stage = 0, it = 0;
     uint32_t phase = 0;
-    const int j_first = lo / g.T;
-    for (int pos = lo; pos < hi;) {
+    for (int pos = sh.lo; pos < sh.hi;) {
         const int j = pos / g.T;
-        const int seg_hi = min(hi, (j + 1) * g.T);
-        const int entry = c.union_list[j];
+        const int seg = min(j - sh.j_first, kStreamSegTab - 1);
+        const int seg_hi = min(sh.hi, (j + 1) * g.T);
+        const int entry = sh.segtab[seg];
         const int n = entry & 0xffff, pass = entry >> 16;
-        const int R = min(c.group_count[n] - pass * kStreamPassRows, kStreamPassRows);
-        if (R <= 8)
-            stream_segment<1, KBW>(c, g, sh, pp, logits_tap, n, pass, R, j, pos, seg_hi, j - j_first, stage, phase, zbuf);
+        const int R = max(1, min(c.group_count[n] - pass * kStreamPassRows, kStreamPassRows));
+        if (!mma_role)
+            stream_segment_stats(c, g, sh, pp, logits_tap, n, pass, R, j, pos, seg_hi, seg, it);
+        else if (R <= 8)
+            stream_segment_mma<1, KBW>(c, g, sh, n, pass, R, pos, seg_hi, stage, phase, it);
         else
-            stream_segment<2, KBW>(c, g, sh, pp, logits_tap, n, pass, R, j, pos, seg_hi, j - j_first, stage, phase, zbuf);
+            stream_segment_mma<2, KBW>(c, g, sh, n, pass, R, pos, seg_hi, stage, phase, it);
         pos = seg_hi;
     }
 }
