@@ -165,6 +165,8 @@ int coral_lmhead_set_path(coral_lmhead_handle h, int path);
  */
 int coral_lmhead_set_kernel_timing(coral_lmhead_handle h, int on);
 int coral_lmhead_head_kernel_ms(coral_lmhead_handle h, float *ms);
+/* Same aid, three spans of the last timed call: router stage, weight-streaming kernel, merge. */
+int coral_lmhead_stage_ms(coral_lmhead_handle h, float *route_ms, float *head_ms, float *merge_ms);
 
 /*
  * Synchronise `stream`, return the device status word of the handle (CORAL_OK,

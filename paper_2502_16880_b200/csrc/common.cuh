@@ -15,6 +15,7 @@ constexpr int kNoToken = 0x7fffffff;
 struct DeviceState {
     int status;        // 0 or a CORAL_ERR_* code (first error wins)
     int n_union;       // groups touched by the last call
+    int ticket;        // arrival counter of the fused router kernel; zero between calls
     int n_virtual;     // (group, pass) entries of the union list; equals n_union when no group needs a second pass
 };
 
@@ -102,6 +103,12 @@ __device__ __forceinline__ void warp_argbest(float& v, int& k) {
         if (better(ov, ok, v, k)) { v = ov; k = ok; }
     }
 }
+
+// Programmatic dependent launch: a kernel launched with the programmatic-serialisation attribute may start
+// while its predecessor in the stream still runs; pdl_wait() blocks until the predecessor has completed
+// and its writes are visible (no-op without the attribute).  pdl_launch_dependents() lets the successor start.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
 __device__ __forceinline__ void set_status(DeviceState* st, int code) { atomicCAS(&st->status, 0, code); }
 

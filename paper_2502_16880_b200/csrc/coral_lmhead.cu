@@ -145,6 +145,7 @@ struct coral_lmhead_s {
     StreamGeom sg;
     int stream_smem;     // 0 if the streaming path is not available for this shape/device
     cudaEvent_t ev_head0, ev_head1;   // around the weight-streaming kernel when kernel timing is on
+    cudaEvent_t ev_begin, ev_end;     // before the router stage / after the merge
     bool timing;
     // facts about the last draft call
     int last_path, last_M, last_kg, last_kt, last_launches;
@@ -180,6 +181,23 @@ CallView make_view(const coral_lmhead_s* h, const void* hidden, int M, int kg, i
     c.part_id = reinterpret_cast<int32_t*>(ws + L.part_id);
     c.state = reinterpret_cast<DeviceState*>(ws + L.state);
     return c;
+}
+
+// Launch with the programmatic-serialisation attribute: the kernel may begin while the previous kernel of
+// the stream is still running and synchronises with it through pdl_wait().
+template <typename... KArgs, typename... Args>
+cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args) {
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
 }
 
 bool stream_ok(const coral_lmhead_s* h, int M) { return h->stream_smem > 0 && M <= kStreamMaxM; }
@@ -318,6 +336,8 @@ int coral_lmhead_destroy(coral_lmhead_handle h) {
     if (h->own_ws && h->ws) cudaFree(h->ws);
     if (h->ev_head0) cudaEventDestroy(h->ev_head0);
     if (h->ev_head1) cudaEventDestroy(h->ev_head1);
+    if (h->ev_begin) cudaEventDestroy(h->ev_begin);
+    if (h->ev_end) cudaEventDestroy(h->ev_end);
     delete h;
     return CORAL_OK;
 }
@@ -347,27 +367,31 @@ int coral_lmhead_draft_ex(coral_lmhead_handle h, const void* hidden_dev, int M, 
     c.pass_rows = path == CORAL_PATH_STREAM ? kStreamPassRows : 0;
     int launches = 0;
 
-    gate_kernel<<<dim3(c.N, (M + kGateRows - 1) / kGateRows), kGateThreads, 0, st>>>(c, out_gate_dev);
-    ++launches;
-    select_kernel<<<(M + kSelectWarps - 1) / kSelectWarps, kSelectWarps * 32, 0, st>>>(c, forced_groups_dev,
-                                                                                      out_groups_dev);
-    ++launches;
-    bucket_kernel<<<1, kBucketThreads, 0, st>>>(c);
-    ++launches;
+    if (h->timing) cudaEventRecord(h->ev_begin, st);
+    if (M <= kRouteFusedMaxM) {
+        route_fused_kernel<<<c.N, kRouteThreads, 0, st>>>(c, forced_groups_dev, out_groups_dev, out_gate_dev);
+        ++launches;
+    } else {
+        gate_kernel<<<dim3(c.N, (M + kGateRows - 1) / kGateRows), kGateThreads, 0, st>>>(c, out_gate_dev);
+        ++launches;
+        select_kernel<<<(M + kSelectWarps - 1) / kSelectWarps, kSelectWarps * 32, 0, st>>>(c, forced_groups_dev,
+                                                                                          out_groups_dev);
+        ++launches;
+        bucket_kernel<<<1, kBucketThreads, 0, st>>>(c);
+        ++launches;
+    }
     if (h->timing) cudaEventRecord(h->ev_head0, st);
     if (path == CORAL_PATH_STREAM) {
         const Layout& L = h->L;
         StreamPartials pp{reinterpret_cast<float*>(h->ws + L.sp_max), reinterpret_cast<float*>(h->ws + L.sp_sum),
                           reinterpret_cast<float*>(h->ws + L.sp_val), reinterpret_cast<int32_t*>(h->ws + L.sp_id)};
-        if (h->sg.kc == 512)
-            head_stream_kernel<2><<<h->sg.grid, kStreamThreads, h->stream_smem, st>>>(c, h->sg, pp, out_logits_dev);
-        else
-            head_stream_kernel<1><<<h->sg.grid, kStreamThreads, h->stream_smem, st>>>(c, h->sg, pp, out_logits_dev);
+        launch_pdl(h->sg.kc == 512 ? head_stream_kernel<2> : head_stream_kernel<1>, dim3(h->sg.grid),
+                   dim3(kStreamThreads), (size_t)h->stream_smem, st, c, h->sg, pp, out_logits_dev);
         ++launches;
         if (h->timing) cudaEventRecord(h->ev_head1, st);
-        merge_stream_kernel<<<M, kMergeStreamThreads, kMergeSmemCands * 8, st>>>(
-            c, h->sg, pp, reinterpret_cast<float*>(h->ws + L.cand_val), reinterpret_cast<int32_t*>(h->ws + L.cand_id),
-            (int)L.cand_cap, kMergeSmemCands, out_ids_dev, out_logprobs_dev, out_lse_dev);
+        launch_pdl(merge_stream_kernel, dim3(M), dim3(kMergeStreamThreads), (size_t)kMergeSmemCands * 8, st, c, h->sg, pp,
+                   reinterpret_cast<float*>(h->ws + L.cand_val), reinterpret_cast<int32_t*>(h->ws + L.cand_id),
+                   (int)L.cand_cap, (int)kMergeSmemCands, out_ids_dev, out_logprobs_dev, out_lse_dev);
         ++launches;
     } else {
         head_simt_kernel<<<dim3(c.T, c.N), kSimtThreads, h->simt_smem, st>>>(c, out_logits_dev);
@@ -376,6 +400,7 @@ int coral_lmhead_draft_ex(coral_lmhead_handle h, const void* hidden_dev, int M, 
         merge_kernel<<<M, kMergeThreads, 0, st>>>(c, out_ids_dev, out_logprobs_dev, out_lse_dev);
         ++launches;
     }
+    if (h->timing) cudaEventRecord(h->ev_end, st);
     if (cudaGetLastError() != cudaSuccess) return CORAL_ERR_CUDA;
 
     h->last_path = path; h->last_M = M; h->last_kg = k_groups; h->last_kt = k_tokens; h->last_launches = launches;
@@ -412,7 +437,8 @@ int coral_lmhead_draft_host(coral_lmhead_handle h, const void* hidden_host, int 
 int coral_lmhead_set_kernel_timing(coral_lmhead_handle h, int on) {
     if (!h) return CORAL_ERR_INVALID;
     if (on && !h->ev_head0) {
-        if (cudaEventCreate(&h->ev_head0) != cudaSuccess || cudaEventCreate(&h->ev_head1) != cudaSuccess)
+        if (cudaEventCreate(&h->ev_head0) != cudaSuccess || cudaEventCreate(&h->ev_head1) != cudaSuccess ||
+            cudaEventCreate(&h->ev_begin) != cudaSuccess || cudaEventCreate(&h->ev_end) != cudaSuccess)
             return CORAL_ERR_CUDA;
     }
     h->timing = on != 0;
@@ -423,6 +449,16 @@ int coral_lmhead_head_kernel_ms(coral_lmhead_handle h, float* ms) {
     if (!h || !ms || !h->ev_head0) return CORAL_ERR_INVALID;
     if (cudaEventSynchronize(h->ev_head1) != cudaSuccess) return CORAL_ERR_CUDA;
     if (cudaEventElapsedTime(ms, h->ev_head0, h->ev_head1) != cudaSuccess) return CORAL_ERR_CUDA;
+    return CORAL_OK;
+}
+
+int coral_lmhead_stage_ms(coral_lmhead_handle h, float* route_ms, float* head_ms, float* merge_ms) {
+    if (!h || !route_ms || !head_ms || !merge_ms || !h->ev_head0) return CORAL_ERR_INVALID;
+    if (cudaEventSynchronize(h->ev_end) != cudaSuccess) return CORAL_ERR_CUDA;
+    if (cudaEventElapsedTime(route_ms, h->ev_begin, h->ev_head0) != cudaSuccess ||
+        cudaEventElapsedTime(head_ms, h->ev_head0, h->ev_head1) != cudaSuccess ||
+        cudaEventElapsedTime(merge_ms, h->ev_head1, h->ev_end) != cudaSuccess)
+        return CORAL_ERR_CUDA;
     return CORAL_OK;
 }
 

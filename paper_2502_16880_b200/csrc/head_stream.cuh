@@ -309,6 +309,8 @@ __global__ void __launch_bounds__(kStreamThreads, 1) head_stream_kernel(CallView
     o += sizeof(int) * kStreamSegTab;
     sh.abort_flag = reinterpret_cast<volatile int*>(smem_raw + o);
 
+    pdl_launch_dependents();
+    pdl_wait();                   // the router stage's outputs are complete from here on
     const int n_items = c.state->n_virtual * g.T;
     const int per = (n_items + g.grid - 1) / g.grid;
     sh.lo = min(n_items, (int)blockIdx.x * per);
@@ -385,6 +387,7 @@ __global__ void __launch_bounds__(kStreamThreads, 1) head_stream_kernel(CallView
 // Merge for the streaming path: block per row.  The pieces of row m, slot s are the partials that the
 // CTAs overlapping that slot's group wrote for the row's position in the group's bucket.
 constexpr int kMergeStreamThreads = 256;
+constexpr int kMergeMaxPieces = 1024;         // >= grid + 2 * k_groups for every supported shape
 __global__ void __launch_bounds__(kMergeStreamThreads) merge_stream_kernel(CallView c, StreamGeom g, StreamPartials pp,
                                                                            float* __restrict__ cand_val_scratch,
                                                                            int32_t* __restrict__ cand_id_scratch,
@@ -401,6 +404,7 @@ __global__ void __launch_bounds__(kMergeStreamThreads) merge_stream_kernel(CallV
     __shared__ float s_lse;
     __shared__ int s_first[kMaxGroups], s_cnt[kMaxGroups], s_base[kMaxGroups + 1], s_rpos[kMaxGroups], s_j[kMaxGroups];
 
+    pdl_wait();                   // partials of the streaming kernel are complete from here on
     const int n_items = c.state->n_virtual * g.T;
     const int per = (n_items + g.grid - 1) / g.grid;
     for (int s = threadIdx.x; s < c.k_groups; s += kMergeStreamThreads) {
@@ -427,19 +431,23 @@ __global__ void __launch_bounds__(kMergeStreamThreads) merge_stream_kernel(CallV
     int32_t* ci = (C <= smem_cands) ? reinterpret_cast<int32_t*>(msm + sizeof(float) * smem_cands)
                                     : cand_id_scratch + (size_t)m * cand_cap;
 
-    // piece q -> (slot s, CTA b) by search over the (few) slots; gather max/sum and the candidate lists
-    float mx = kNegInf;
+    // piece q -> index of its partial; P <= grid + 2 * k_groups
+    __shared__ int s_piece[kMergeMaxPieces];
     for (int q = threadIdx.x; q < P; q += kMergeStreamThreads) {
         int s = 0;
         while (s + 1 < c.k_groups && s_base[s + 1] <= q) ++s;
         const int b = s_first[s] + (q - s_base[s]);
         const int seg = s_j[s] - (b * per) / g.T;
-        const size_t p = ((size_t)b * g.seg_max + seg) * kStreamPassRows + s_rpos[s];
-        mx = fmaxf(mx, pp.pmax[p]);
-        for (int i = 0; i < c.k_tokens; ++i) {
-            cv[q * c.k_tokens + i] = pp.pval[p * c.k_tokens + i];
-            ci[q * c.k_tokens + i] = pp.pid[p * c.k_tokens + i];
-        }
+        s_piece[min(q, kMergeMaxPieces - 1)] = (int)(((size_t)b * g.seg_max + seg) * kStreamPassRows + s_rpos[s]);
+    }
+    __syncthreads();
+    float mx = kNegInf;
+    for (int q = threadIdx.x; q < P; q += kMergeStreamThreads) mx = fmaxf(mx, pp.pmax[s_piece[min(q, kMergeMaxPieces - 1)]]);
+    for (int idx = threadIdx.x; idx < C; idx += kMergeStreamThreads) {
+        const int q = idx / c.k_tokens, i = idx - q * c.k_tokens;
+        const size_t p = (size_t)s_piece[min(q, kMergeMaxPieces - 1)];
+        cv[idx] = pp.pval[p * c.k_tokens + i];
+        ci[idx] = pp.pid[p * c.k_tokens + i];
     }
     mx = warp_max(mx);
     if (lane == 0) s_f[warp] = mx;
@@ -450,11 +458,7 @@ __global__ void __launch_bounds__(kMergeStreamThreads) merge_stream_kernel(CallV
     __syncthreads();
     float sum = 0.f;
     for (int q = threadIdx.x; q < P; q += kMergeStreamThreads) {
-        int s = 0;
-        while (s + 1 < c.k_groups && s_base[s + 1] <= q) ++s;
-        const int b = s_first[s] + (q - s_base[s]);
-        const int seg = s_j[s] - (b * per) / g.T;
-        const size_t p = ((size_t)b * g.seg_max + seg) * kStreamPassRows + s_rpos[s];
+        const int p = s_piece[min(q, kMergeMaxPieces - 1)];
         sum += pp.psum[p] * expf(pp.pmax[p] - mx);
     }
     sum = warp_sum(sum);

@@ -160,4 +160,192 @@ __global__ void __launch_bounds__(kBucketThreads) bucket_kernel(CallView c) {
     }
 }
 
+
+// Router stage in one launch for few rows (M <= kRouteFusedMaxM).  grid = N CTAs: CTA n computes the gate
+// scores of group n (threads split H), then takes a ticket; the CTA that draws the last ticket - nobody
+// waits for anybody - selects the groups of every row, buckets the rows by group and writes the union
+// list.  Same outputs as gate_kernel + select_kernel + bucket_kernel.
+// Selection is by rank: a group's slot is the number of groups that beat it (higher score, or equal score
+// and lower index), so the cost does not grow with k_groups.
+constexpr int kRouteFusedMaxM = 32;
+constexpr int kRouteThreads = 256;
+
+__global__ void __launch_bounds__(kRouteThreads)
+    route_fused_kernel(CallView c, const int32_t* __restrict__ forced, int32_t* __restrict__ groups_tap,
+                       float* __restrict__ gate_tap) {
+    __shared__ int16_t s_slot[kRouteFusedMaxM][kMaxGroups];
+    __shared__ float s_val[kRouteThreads / 32][kMaxGroups];
+    __shared__ int s_count[kMaxGroups];
+    __shared__ int s_offset[kMaxGroups + 1];
+    __shared__ float s_red[kRouteThreads / 32][8];
+    __shared__ int s_last;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    constexpr int kWarps = kRouteThreads / 32;
+    const int chunks = c.H >> 3;
+    pdl_launch_dependents();      // the next kernel may set itself up; it waits for this grid before reading
+
+    {
+        const int n = blockIdx.x;
+        const uint4* __restrict__ wg = reinterpret_cast<const uint4*>(c.w_gate + (size_t)n * c.H);
+        for (int m0 = 0; m0 < c.M; m0 += 8) {
+            const int rows = min(8, c.M - m0);
+            const uint4* __restrict__ hid = reinterpret_cast<const uint4*>(c.hidden + (size_t)m0 * c.H);
+            float acc[8];
+#pragma unroll
+            for (int r = 0; r < 8; ++r) acc[r] = 0.f;
+            for (int ch = threadIdx.x; ch < chunks; ch += kRouteThreads) {
+                const uint4 w = __ldg(wg + ch);
+#pragma unroll
+                for (int r = 0; r < 8; ++r)
+                    if (r < rows) acc[r] = dot8(w, __ldg(hid + (size_t)r * chunks + ch), acc[r]);
+            }
+#pragma unroll
+            for (int r = 0; r < 8; ++r) {
+                const float sum = warp_sum(acc[r]);
+                if (lane == 0) s_red[warp][r] = sum;
+            }
+            __syncthreads();
+            if (threadIdx.x < rows) {
+                float sum = 0.f;
+#pragma unroll
+                for (int w = 0; w < kWarps; ++w) sum += s_red[w][threadIdx.x];
+                c.gate[(size_t)(m0 + threadIdx.x) * c.N + n] = sum;
+                if (gate_tap) gate_tap[(size_t)(m0 + threadIdx.x) * c.N + n] = sum;
+            }
+            __syncthreads();
+        }
+    }
+    // ticket: the scores above are published before the ticket is drawn; the last CTA sees all of them
+    if (threadIdx.x == 0) {
+        __threadfence();
+        const int ticket = atomicAdd(&c.state->ticket, 1);
+        s_last = ticket == (int)gridDim.x - 1;
+        if (s_last) c.state->ticket = 0;          // ready for the next call on this handle
+        __threadfence();
+    }
+    __syncthreads();
+    if (!s_last) return;
+
+    // groups of every row: one warp per row
+    constexpr int kPer = kMaxGroups / 32;
+    for (int m = warp; m < c.M; m += kWarps) {
+        int slot[kPer];
+#pragma unroll
+        for (int i = 0; i < kPer; ++i) slot[i] = -1;
+        if (forced) {
+            for (int s = 0; s < c.k_groups; ++s) {
+                int pick = forced[(size_t)m * c.k_groups + s];
+                if (pick < 0 || pick >= c.N) {           // never index with it; report and fall back to group 0
+                    if (lane == 0) set_status(c.state, -6);
+                    pick = 0;
+                }
+#pragma unroll
+                for (int i = 0; i < kPer; ++i) {
+                    if (lane + 32 * i == pick) {
+                        if (slot[i] >= 0) set_status(c.state, -6);   // a forced group named twice
+                        slot[i] = s;
+                    }
+                }
+            }
+        } else {
+            float val[kPer];
+#pragma unroll
+            for (int i = 0; i < kPer; ++i) {
+                const int n = lane + 32 * i;
+                val[i] = (n < c.N) ? __ldcg(c.gate + (size_t)m * c.N + n) : kNegInf;
+                if (n < c.N) s_val[warp][n] = val[i];
+            }
+            __syncwarp();
+            int rank[kPer];
+#pragma unroll
+            for (int i = 0; i < kPer; ++i) rank[i] = 0;
+            for (int j = 0; j < c.N; ++j) {
+                const float vj = s_val[warp][j];
+#pragma unroll
+                for (int i = 0; i < kPer; ++i) rank[i] += better(vj, j, val[i], lane + 32 * i) ? 1 : 0;
+            }
+#pragma unroll
+            for (int i = 0; i < kPer; ++i)
+                if (lane + 32 * i < c.N && rank[i] < c.k_groups) slot[i] = rank[i];
+            __syncwarp();
+        }
+#pragma unroll
+        for (int i = 0; i < kPer; ++i) {
+            const int n = lane + 32 * i;
+            if (n < c.N) {
+                s_slot[m][n] = (int16_t)slot[i];
+                c.slot_of[(size_t)m * c.N + n] = (int16_t)slot[i];
+                if (slot[i] >= 0) {
+                    c.sel[(size_t)m * c.k_groups + slot[i]] = n;
+                    if (groups_tap) groups_tap[(size_t)m * c.k_groups + slot[i]] = n;
+                }
+            }
+        }
+    }
+    __syncthreads();
+
+    // rows per group (M <= 32: one ballot per group)
+    for (int n = warp; n < c.N; n += kWarps) {
+        const bool in = lane < c.M && s_slot[lane][n] >= 0;
+        const unsigned bal = __ballot_sync(0xffffffffu, in);
+        if (lane == 0) s_count[n] = __popc(bal);
+    }
+    __syncthreads();
+    if (warp == 0) {
+        // exclusive scan of the counts and numbering of the (group, pass) entries, 8 consecutive groups per lane
+        int cnt[kPer], passes[kPer], tot = 0, vtot = 0, utot = 0;
+#pragma unroll
+        for (int i = 0; i < kPer; ++i) {
+            const int n = lane * kPer + i;
+            cnt[i] = n < c.N ? s_count[n] : 0;
+            passes[i] = cnt[i] == 0 ? 0 : (c.pass_rows > 0 ? (cnt[i] + c.pass_rows - 1) / c.pass_rows : 1);
+            tot += cnt[i];
+            vtot += passes[i];
+            utot += cnt[i] > 0;
+        }
+        int ex = tot, vex = vtot, uex = utot;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int a = __shfl_up_sync(0xffffffffu, ex, o), b = __shfl_up_sync(0xffffffffu, vex, o);
+            const int d = __shfl_up_sync(0xffffffffu, uex, o);
+            if (lane >= o) { ex += a; vex += b; uex += d; }
+        }
+        const int all = __shfl_sync(0xffffffffu, ex, 31), vall = __shfl_sync(0xffffffffu, vex, 31);
+        const int uall = __shfl_sync(0xffffffffu, uex, 31);
+        int run = ex - tot, virt = vex - vtot;
+#pragma unroll
+        for (int i = 0; i < kPer; ++i) {
+            const int n = lane * kPer + i;
+            if (n < c.N) {
+                s_offset[n] = run;
+                c.group_offset[n] = run;
+                c.group_count[n] = cnt[i];
+                c.union_rank[n] = cnt[i] > 0 ? virt : -1;
+                for (int p = 0; p < passes[i]; ++p)
+                    if (virt + p < c.union_cap) c.union_list[virt + p] = n | (p << 16);
+                run += cnt[i];
+                virt += passes[i];
+            }
+        }
+        if (lane == 0) {
+            s_offset[c.N] = all;
+            c.group_offset[c.N] = all;
+            c.state->n_union = uall;
+            c.state->n_virtual = min(vall, c.union_cap);
+        }
+    }
+    __syncthreads();
+    for (int n = warp; n < c.N; n += kWarps) {
+        const int sl = lane < c.M ? (int)s_slot[lane][n] : -1;
+        const unsigned bal = __ballot_sync(0xffffffffu, sl >= 0);
+        if (sl >= 0) {
+            const int pos = __popc(bal & ((1u << lane) - 1u));
+            const int p = s_offset[n] + pos;
+            c.bucket_row[p] = lane;
+            c.bucket_slot[p] = sl;
+            c.bucket_pos[(size_t)lane * c.k_groups + sl] = pos;
+        }
+    }
+}
+
 }  // namespace coral

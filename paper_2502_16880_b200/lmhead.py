@@ -55,6 +55,7 @@ _SIGNATURES = {
     "coral_lmhead_set_path": (_i, [_vp, _i]),
     "coral_lmhead_set_kernel_timing": (_i, [_vp, _i]),
     "coral_lmhead_head_kernel_ms": (_i, [_vp, ctypes.POINTER(ctypes.c_float)]),
+    "coral_lmhead_stage_ms": (_i, [_vp] + [ctypes.POINTER(ctypes.c_float)] * 3),
     "coral_lmhead_status": (_i, [_vp, _vp]),
     "coral_lmhead_last_stats": (_i, [_vp, ctypes.POINTER(coral_lmhead_stats), _vp]),
     "coral_lmhead_route_static": (_i, [_vp, _vp, _i, _i, _i, _i, _vp, _vp, _vp]),
@@ -186,6 +187,14 @@ def coral_lmhead_head_kernel_ms(handle) -> float:
     ms = ctypes.c_float(0.0)
     _check(load_library().coral_lmhead_head_kernel_ms(handle, ctypes.byref(ms)), "coral_lmhead_head_kernel_ms")
     return float(ms.value)
+
+
+def coral_lmhead_stage_ms(handle):
+    """(route_ms, head_ms, merge_ms) of the last call made with kernel timing on."""
+    a, b, c = ctypes.c_float(0.0), ctypes.c_float(0.0), ctypes.c_float(0.0)
+    _check(load_library().coral_lmhead_stage_ms(handle, ctypes.byref(a), ctypes.byref(b), ctypes.byref(c)),
+           "coral_lmhead_stage_ms")
+    return float(a.value), float(b.value), float(c.value)
 
 
 def coral_lmhead_status(handle, stream=None) -> int:
