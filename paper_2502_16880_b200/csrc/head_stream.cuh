@@ -121,36 +121,37 @@ struct StreamShared {
     int lo, hi, j_first;      // this CTA's run of items and its first virtual group
 };
 
-// Fold the 16 logits of one item (lane i < rows holds z of tile row i and its token id) into a warp's
-// running statistics of one hidden row: online max / sum-exp and the sorted top-k list (entry i in lane i).
+// Fold the 16 logits of one item into a warp's running statistics of one hidden row.  Lane i < rows holds
+// the logit of tile row i.  Softmax part: every lane keeps an online (max, sum-exp) over the values it has
+// seen, combined across lanes once per segment.  Top-k part: the sorted list lives one entry per lane
+// (entry i in lane i < k_tokens); a value that can beat the current k-th entry is inserted by shifting the
+// tail of the list one lane up, so the common case (no candidate) costs one ballot.
 __device__ __forceinline__ void fold_item(float zv, const int32_t* __restrict__ tokens, bool have, int k_tokens,
-                                          int lane, float& run_max, float& run_sum, float& lv, int& lid) {
-    const float tmax = warp_max(zv);
-    const float nmax = fmaxf(run_max, tmax);
-    const float add = warp_sum(have ? __expf(zv - nmax) : 0.f);
-    run_sum = run_sum * __expf(run_max - nmax) + add;     // exp(-inf) = 0 on the first item
-    run_max = nmax;
-    const float kth = __shfl_sync(0xffffffffu, lv, k_tokens - 1);
-    const int kth_id = __shfl_sync(0xffffffffu, lid, k_tokens - 1);
-    if (kth_id == kNoToken || tmax >= kth) {
-        float a = lv, b = zv;
-        int ai = lid, bi = have ? __ldg(tokens + lane) : kNoToken;
-        float ov = kNegInf;
-        int oi = kNoToken;
-        for (int k = 0; k < k_tokens; ++k) {
-            float bv;
-            int bk;
-            if (better(a, ai, b, bi)) { bv = a; bk = ai; } else { bv = b; bk = bi; }
-            warp_argbest(bv, bk);
-            if (bk != kNoToken) {
-                if (ai == bk) { a = kNegInf; ai = kNoToken; }
-                if (bi == bk) { b = kNegInf; bi = kNoToken; }
-            }
-            if (lane == k) { ov = bv; oi = bk; }
-        }
-        lv = ov;
-        lid = oi;
+                                          int lane, float& lane_max, float& lane_sum, float& lv, int& lid,
+                                          float& kth, int& kth_id) {
+    if (have) {
+        const float nmax = fmaxf(lane_max, zv);
+        lane_sum = lane_sum * __expf(lane_max - nmax) + __expf(zv - nmax);   // exp(-inf) = 0 the first time
+        lane_max = nmax;
     }
+    unsigned cand = __ballot_sync(0xffffffffu, have && (kth_id == kNoToken || zv >= kth));
+    if (cand == 0) return;
+    const int tok = ((cand >> lane) & 1u) ? __ldg(tokens + lane) : kNoToken;
+    while (cand) {
+        const int src = __ffs(cand) - 1;
+        cand &= cand - 1;
+        const float v = __shfl_sync(0xffffffffu, zv, src);
+        const int id = __shfl_sync(0xffffffffu, tok, src);
+        const int pos = __popc(__ballot_sync(0xffffffffu, better(lv, lid, v, id)));   // entries that stay ahead
+        const float up_v = __shfl_up_sync(0xffffffffu, lv, 1);
+        const int up_id = __shfl_up_sync(0xffffffffu, lid, 1);
+        if (pos < k_tokens) {
+            if (lane == pos) { lv = v; lid = id; }
+            else if (lane > pos && lane < k_tokens) { lv = up_v; lid = up_id; }
+        }
+    }
+    kth = __shfl_sync(0xffffffffu, lv, k_tokens - 1);
+    kth_id = __shfl_sync(0xffffffffu, lid, k_tokens - 1);
 }
 
 // MMA side of one segment: items [lo, hi) of the run, all inside virtual group j = (group n, pass) with R
@@ -234,11 +235,12 @@ __device__ __forceinline__ void stream_segment_stats(const CallView& c, const St
     constexpr int kOwn = (kStreamPassRows + kStreamStatWarps - 1) / kStreamStatWarps;
     const int sw = (threadIdx.x >> 5) - kStreamWarps, lane = threadIdx.x & 31;
     const int off = c.group_offset[n] + pass * kStreamPassRows;
-    float run_max[kOwn], run_sum[kOwn], lv[kOwn];
-    int lid[kOwn], my_m[kOwn], my_slot[kOwn];
+    float run_max[kOwn], run_sum[kOwn], lv[kOwn], kth[kOwn];
+    int lid[kOwn], kth_id[kOwn], my_m[kOwn], my_slot[kOwn];
 #pragma unroll
     for (int u = 0; u < kOwn; ++u) {
         run_max[u] = kNegInf; run_sum[u] = 0.f; lv[u] = kNegInf; lid[u] = kNoToken;
+        kth[u] = kNegInf; kth_id[u] = kNoToken;
         const int r = sw + kStreamStatWarps * u;
         my_m[u] = r < R ? c.bucket_row[off + r] : 0;
         my_slot[u] = r < R ? c.bucket_slot[off + r] : 0;
@@ -271,7 +273,7 @@ __device__ __forceinline__ void stream_segment_stats(const CallView& c, const St
             if (r < R) {
                 if (logits_tap && have)
                     logits_tap[((size_t)my_m[u] * c.k_groups + my_slot[u]) * c.v + row0 + lane] = zv[u];
-                fold_item(zv[u], tokens, have, c.k_tokens, lane, run_max[u], run_sum[u], lv[u], lid[u]);
+                fold_item(zv[u], tokens, have, c.k_tokens, lane, run_max[u], run_sum[u], lv[u], lid[u], kth[u], kth_id[u]);
             }
         }
     }
@@ -280,7 +282,9 @@ __device__ __forceinline__ void stream_segment_stats(const CallView& c, const St
         const int r = sw + kStreamStatWarps * u;
         if (r < R) {
             const size_t p = ((size_t)blockIdx.x * g.seg_max + seg) * kStreamPassRows + r;
-            if (lane == 0) { pp.pmax[p] = run_max[u]; pp.psum[p] = run_sum[u]; }
+            const float mx = warp_max(run_max[u]);                       // combine the lanes' online softmax states
+            const float sm = warp_sum(run_sum[u] * __expf(run_max[u] - mx));
+            if (lane == 0) { pp.pmax[p] = mx; pp.psum[p] = sm; }
             if (lane < c.k_tokens) { pp.pval[p * c.k_tokens + lane] = lv[u]; pp.pid[p * c.k_tokens + lane] = lid[u]; }
         }
     }
@@ -400,7 +404,6 @@ __global__ void __launch_bounds__(kMergeStreamThreads) merge_stream_kernel(CallV
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     constexpr int kWarps = kMergeStreamThreads / 32;
     __shared__ float s_f[kWarps];
-    __shared__ int s_i[kWarps];
     __shared__ float s_lse;
     __shared__ int s_first[kMaxGroups], s_cnt[kMaxGroups], s_base[kMaxGroups + 1], s_rpos[kMaxGroups], s_j[kMaxGroups];
 
@@ -474,31 +477,51 @@ __global__ void __launch_bounds__(kMergeStreamThreads) merge_stream_kernel(CallV
     __syncthreads();
     const float lse = s_lse;
 
-    float last_v = __builtin_huge_valf();
-    int last_id = -1;
-    for (int k = 0; k < c.k_tokens; ++k) {
-        float bv = kNegInf;
-        int bk = kNoToken;
-        for (int i = threadIdx.x; i < C; i += kMergeStreamThreads) {
-            const float v = cv[i];
-            const int id = ci[i];
-            const bool after = v < last_v || (v == last_v && id > last_id);
-            if (after && better(v, id, bv, bk)) { bv = v; bk = id; }
+    // Token ids are unique across the candidates, so "strictly after the last pick in (value desc, id asc)
+    // order" selects the next one without marking.  Two levels: every warp picks the k_tokens best of its
+    // strided share, then warp 0 picks the k_tokens best of those.
+    __shared__ float s_wv[kWarps][kMaxKTokens];
+    __shared__ int s_wi[kWarps][kMaxKTokens];
+    {
+        float last_v = __builtin_huge_valf();
+        int last_id = -1;
+        for (int k = 0; k < c.k_tokens; ++k) {
+            float bv = kNegInf;
+            int bk = kNoToken;
+            for (int i = threadIdx.x; i < C; i += kMergeStreamThreads) {
+                const float v = cv[i];
+                const int id = ci[i];
+                const bool after = v < last_v || (v == last_v && id > last_id);
+                if (after && better(v, id, bv, bk)) { bv = v; bk = id; }
+            }
+            warp_argbest(bv, bk);
+            if (lane == k) { s_wv[warp][k] = bv; s_wi[warp][k] = bk; }
+            last_v = bv;
+            last_id = bk;
         }
-        warp_argbest(bv, bk);
-        __syncthreads();
-        if (lane == 0) { s_f[warp] = bv; s_i[warp] = bk; }
-        __syncthreads();
-        bv = s_f[0]; bk = s_i[0];
-#pragma unroll
-        for (int w = 1; w < kWarps; ++w)
-            if (better(s_f[w], s_i[w], bv, bk)) { bv = s_f[w]; bk = s_i[w]; }
-        if (threadIdx.x == 0) {
-            out_ids[(size_t)m * c.k_tokens + k] = bk;
-            out_logprobs[(size_t)m * c.k_tokens + k] = bv - lse;
+    }
+    __syncthreads();
+    if (warp == 0) {
+        const int C2 = kWarps * c.k_tokens;
+        float last_v = __builtin_huge_valf();
+        int last_id = -1;
+        for (int k = 0; k < c.k_tokens; ++k) {
+            float bv = kNegInf;
+            int bk = kNoToken;
+            for (int i = lane; i < C2; i += 32) {
+                const float v = s_wv[i / c.k_tokens][i % c.k_tokens];
+                const int id = s_wi[i / c.k_tokens][i % c.k_tokens];
+                const bool after = v < last_v || (v == last_v && id > last_id);
+                if (after && better(v, id, bv, bk)) { bv = v; bk = id; }
+            }
+            warp_argbest(bv, bk);
+            if (lane == 0) {
+                out_ids[(size_t)m * c.k_tokens + k] = bk;
+                out_logprobs[(size_t)m * c.k_tokens + k] = bv - lse;
+            }
+            last_v = bv;
+            last_id = bk;
         }
-        last_v = bv;
-        last_id = bk;
     }
 }
 

@@ -161,6 +161,67 @@ __global__ void __launch_bounds__(kBucketThreads) bucket_kernel(CallView c) {
 }
 
 
+// Groups of row m by one warp (NPER = groups per lane).  Rank selection: slot of a group = number of groups
+// that beat it (higher score, or equal score and lower index).  Forced groups take their listed order.
+template <int NPER>
+__device__ __forceinline__ void route_select_row(const CallView& c, const int32_t* __restrict__ forced,
+                                                 int32_t* __restrict__ groups_tap, int m, int lane, float* s_val,
+                                                 int16_t* s_slot_row) {
+    int slot[NPER];
+#pragma unroll
+    for (int i = 0; i < NPER; ++i) slot[i] = -1;
+    if (forced) {
+        for (int s = 0; s < c.k_groups; ++s) {
+            int pick = forced[(size_t)m * c.k_groups + s];
+            if (pick < 0 || pick >= c.N) {           // never index with it; report and fall back to group 0
+                if (lane == 0) set_status(c.state, -6);
+                pick = 0;
+            }
+#pragma unroll
+            for (int i = 0; i < NPER; ++i) {
+                if (lane + 32 * i == pick) {
+                    if (slot[i] >= 0) set_status(c.state, -6);   // a forced group named twice
+                    slot[i] = s;
+                }
+            }
+        }
+    } else {
+        float val[NPER];
+#pragma unroll
+        for (int i = 0; i < NPER; ++i) {
+            const int n = lane + 32 * i;
+            val[i] = (n < c.N) ? __ldcg(c.gate + (size_t)m * c.N + n) : kNegInf;
+            if (n < c.N) s_val[n] = val[i];
+        }
+        __syncwarp();
+        int rank[NPER];
+#pragma unroll
+        for (int i = 0; i < NPER; ++i) rank[i] = 0;
+#pragma unroll 4
+        for (int j = 0; j < c.N; ++j) {
+            const float vj = s_val[j];
+#pragma unroll
+            for (int i = 0; i < NPER; ++i) rank[i] += better(vj, j, val[i], lane + 32 * i) ? 1 : 0;
+        }
+#pragma unroll
+        for (int i = 0; i < NPER; ++i)
+            if (lane + 32 * i < c.N && rank[i] < c.k_groups) slot[i] = rank[i];
+        __syncwarp();
+    }
+#pragma unroll
+    for (int i = 0; i < NPER; ++i) {
+        const int n = lane + 32 * i;
+        if (n < c.N) {
+            s_slot_row[n] = (int16_t)slot[i];
+            c.slot_of[(size_t)m * c.N + n] = (int16_t)slot[i];
+            if (slot[i] >= 0) {
+                c.sel[(size_t)m * c.k_groups + slot[i]] = n;
+                if (groups_tap) groups_tap[(size_t)m * c.k_groups + slot[i]] = n;
+            }
+        }
+    }
+}
+
 // Router stage in one launch for few rows (M <= kRouteFusedMaxM).  grid = N CTAs: CTA n computes the gate
 // scores of group n (threads split H), then takes a ticket; the CTA that draws the last ticket - nobody
 // waits for anybody - selects the groups of every row, buckets the rows by group and writes the union
@@ -195,9 +256,12 @@ __global__ void __launch_bounds__(kRouteThreads)
             for (int r = 0; r < 8; ++r) acc[r] = 0.f;
             for (int ch = threadIdx.x; ch < chunks; ch += kRouteThreads) {
                 const uint4 w = __ldg(wg + ch);
+                uint4 hv[8];                       // all loads first, so they are in flight together
 #pragma unroll
                 for (int r = 0; r < 8; ++r)
-                    if (r < rows) acc[r] = dot8(w, __ldg(hid + (size_t)r * chunks + ch), acc[r]);
+                    hv[r] = r < rows ? __ldg(hid + (size_t)r * chunks + ch) : make_uint4(0, 0, 0, 0);
+#pragma unroll
+                for (int r = 0; r < 8; ++r) acc[r] = dot8(w, hv[r], acc[r]);
             }
 #pragma unroll
             for (int r = 0; r < 8; ++r) {
@@ -227,63 +291,15 @@ __global__ void __launch_bounds__(kRouteThreads)
     if (!s_last) return;
 
     // groups of every row: one warp per row
-    constexpr int kPer = kMaxGroups / 32;
     for (int m = warp; m < c.M; m += kWarps) {
-        int slot[kPer];
-#pragma unroll
-        for (int i = 0; i < kPer; ++i) slot[i] = -1;
-        if (forced) {
-            for (int s = 0; s < c.k_groups; ++s) {
-                int pick = forced[(size_t)m * c.k_groups + s];
-                if (pick < 0 || pick >= c.N) {           // never index with it; report and fall back to group 0
-                    if (lane == 0) set_status(c.state, -6);
-                    pick = 0;
-                }
-#pragma unroll
-                for (int i = 0; i < kPer; ++i) {
-                    if (lane + 32 * i == pick) {
-                        if (slot[i] >= 0) set_status(c.state, -6);   // a forced group named twice
-                        slot[i] = s;
-                    }
-                }
-            }
-        } else {
-            float val[kPer];
-#pragma unroll
-            for (int i = 0; i < kPer; ++i) {
-                const int n = lane + 32 * i;
-                val[i] = (n < c.N) ? __ldcg(c.gate + (size_t)m * c.N + n) : kNegInf;
-                if (n < c.N) s_val[warp][n] = val[i];
-            }
-            __syncwarp();
-            int rank[kPer];
-#pragma unroll
-            for (int i = 0; i < kPer; ++i) rank[i] = 0;
-            for (int j = 0; j < c.N; ++j) {
-                const float vj = s_val[warp][j];
-#pragma unroll
-                for (int i = 0; i < kPer; ++i) rank[i] += better(vj, j, val[i], lane + 32 * i) ? 1 : 0;
-            }
-#pragma unroll
-            for (int i = 0; i < kPer; ++i)
-                if (lane + 32 * i < c.N && rank[i] < c.k_groups) slot[i] = rank[i];
-            __syncwarp();
-        }
-#pragma unroll
-        for (int i = 0; i < kPer; ++i) {
-            const int n = lane + 32 * i;
-            if (n < c.N) {
-                s_slot[m][n] = (int16_t)slot[i];
-                c.slot_of[(size_t)m * c.N + n] = (int16_t)slot[i];
-                if (slot[i] >= 0) {
-                    c.sel[(size_t)m * c.k_groups + slot[i]] = n;
-                    if (groups_tap) groups_tap[(size_t)m * c.k_groups + slot[i]] = n;
-                }
-            }
-        }
+        if (c.N <= 32) route_select_row<1>(c, forced, groups_tap, m, lane, s_val[warp], s_slot[m]);
+        else if (c.N <= 64) route_select_row<2>(c, forced, groups_tap, m, lane, s_val[warp], s_slot[m]);
+        else if (c.N <= 128) route_select_row<4>(c, forced, groups_tap, m, lane, s_val[warp], s_slot[m]);
+        else route_select_row<8>(c, forced, groups_tap, m, lane, s_val[warp], s_slot[m]);
     }
     __syncthreads();
 
+    constexpr int kPer = kMaxGroups / 32;
     // rows per group (M <= 32: one ballot per group)
     for (int n = warp; n < c.N; n += kWarps) {
         const bool in = lane < c.M && s_slot[lane][n] >= 0;
