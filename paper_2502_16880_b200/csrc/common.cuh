@@ -37,7 +37,7 @@ struct CallView {
     int32_t* group_offset;         // [N+1]
     int32_t* bucket_row;           // [M*k_groups] rows that selected a group, ascending per group
     int32_t* bucket_slot;          // [M*k_groups] the slot the group has in that row
-    int32_t* bucket_pos;           // [M][k_groups] position of row m in the bucket of its slot's group
+    int32_t* slot_desc;            // [M][k_groups] (index in union_list of the slot's (group, pass)) << 8 | row's position in the pass
     int32_t* union_list;           // [n_virtual] group | pass << 16, ascending (group, pass)
     int32_t* union_rank;           // [N] index of (group n, pass 0) in union_list, -1 if untouched
     float* part_max;               // [M][k_groups][T]

@@ -23,7 +23,7 @@ inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 // Offsets of the workspace sections (bytes from the workspace base).
 struct Layout {
     size_t w_gate, group_tokens, state, gate, sel, slot_of, group_count, group_offset, bucket_row, bucket_slot,
-        bucket_pos, union_list, union_rank, part_max, part_sum, part_val, part_id, sp_max, sp_sum, sp_val, sp_id,
+        slot_desc, union_list, union_rank, part_max, part_sum, part_val, part_id, sp_max, sp_sum, sp_val, sp_id,
         cand_val, cand_id, stage_hidden, stage_ids, stage_logprobs, total;
     size_t packed_bytes, cand_cap;
     int v, T;
@@ -93,7 +93,7 @@ Layout make_layout(const coral_lmhead_config& c) {
     L.group_offset = take((N + 1) * 4);
     L.bucket_row = take(M * kg * 4);
     L.bucket_slot = take(M * kg * 4);
-    L.bucket_pos = take(M * kg * 4);
+    L.slot_desc = take(M * kg * 4);
     L.union_list = take(N * kStreamMaxPasses * 4);
     L.union_rank = take(N * 4);
     const size_t sp = (size_t)kStreamGridCap * stream_seg_max(c.n_groups, kStreamGridMin) * kStreamPassRows;
@@ -171,7 +171,7 @@ CallView make_view(const coral_lmhead_s* h, const void* hidden, int M, int kg, i
     c.group_offset = reinterpret_cast<int32_t*>(ws + L.group_offset);
     c.bucket_row = reinterpret_cast<int32_t*>(ws + L.bucket_row);
     c.bucket_slot = reinterpret_cast<int32_t*>(ws + L.bucket_slot);
-    c.bucket_pos = reinterpret_cast<int32_t*>(ws + L.bucket_pos);
+    c.slot_desc = reinterpret_cast<int32_t*>(ws + L.slot_desc);
     c.union_list = reinterpret_cast<int32_t*>(ws + L.union_list);
     c.union_rank = reinterpret_cast<int32_t*>(ws + L.union_rank);
     c.union_cap = h->cfg.n_groups * kStreamMaxPasses;

@@ -313,8 +313,8 @@ __global__ void __launch_bounds__(kStreamThreads, 1) head_stream_kernel(CallView
     o += sizeof(int) * kStreamSegTab;
     sh.abort_flag = reinterpret_cast<volatile int*>(smem_raw + o);
 
-    pdl_launch_dependents();
     pdl_wait();                   // the router stage's outputs are complete from here on
+    pdl_launch_dependents();      // the merge kernel may start reading the router's outputs
     const int n_items = c.state->n_virtual * g.T;
     const int per = (n_items + g.grid - 1) / g.grid;
     sh.lo = min(n_items, (int)blockIdx.x * per);
@@ -388,10 +388,13 @@ __global__ void __launch_bounds__(kStreamThreads, 1) head_stream_kernel(CallView
     }
 }
 
-// Merge for the streaming path: block per row.  The pieces of row m, slot s are the partials that the
-// CTAs overlapping that slot's group wrote for the row's position in the group's bucket.
+// Merge for the streaming path: block per row.  The pieces of row m, slot s are the partials that the CTAs
+// overlapping that slot's (group, pass) wrote for the row's position in the pass.  Every piece holds a
+// sorted top-k list, so the largest of the pieces' k-th values is a lower bound of the row's k-th value:
+// only candidates at or above it are kept, and those few are ranked by counting.
 constexpr int kMergeStreamThreads = 256;
 constexpr int kMergeMaxPieces = 1024;         // >= grid + 2 * k_groups for every supported shape
+constexpr int kMergeRankMax = 256;            // survivors ranked by counting; more fall back to k rounds
 __global__ void __launch_bounds__(kMergeStreamThreads) merge_stream_kernel(CallView c, StreamGeom g, StreamPartials pp,
                                                                            float* __restrict__ cand_val_scratch,
                                                                            int32_t* __restrict__ cand_id_scratch,
@@ -403,69 +406,87 @@ __global__ void __launch_bounds__(kMergeStreamThreads) merge_stream_kernel(CallV
     const int m = blockIdx.x;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     constexpr int kWarps = kMergeStreamThreads / 32;
-    __shared__ float s_f[kWarps];
+    __shared__ float s_f[kWarps], s_t[kWarps];
     __shared__ float s_lse;
-    __shared__ int s_first[kMaxGroups], s_cnt[kMaxGroups], s_base[kMaxGroups + 1], s_rpos[kMaxGroups], s_j[kMaxGroups];
+    __shared__ int s_n;
+    __shared__ int s_first[kMaxGroups], s_base[kMaxGroups + 1], s_rpos[kMaxGroups], s_j[kMaxGroups];
+    __shared__ int s_piece[kMergeMaxPieces];
 
-    pdl_wait();                   // partials of the streaming kernel are complete from here on
+    // The router's outputs were complete before the streaming kernel let this grid start.
     const int n_items = c.state->n_virtual * g.T;
     const int per = (n_items + g.grid - 1) / g.grid;
     for (int s = threadIdx.x; s < c.k_groups; s += kMergeStreamThreads) {
-        const int n = c.sel[(size_t)m * c.k_groups + s];
-        const int pos_in_bucket = c.bucket_pos[(size_t)m * c.k_groups + s];
-        const int j = c.union_rank[n] + pos_in_bucket / kStreamPassRows;
+        const int desc = c.slot_desc[(size_t)m * c.k_groups + s];
+        const int j = desc >> 8;
         const int fb = (j * g.T) / per;
         const int lb = ((j + 1) * g.T - 1) / per;
         s_first[s] = fb;
-        s_cnt[s] = lb - fb + 1;
+        s_base[s] = lb - fb + 1;       // piece count, turned into an exclusive prefix below
         s_j[s] = j;
-        s_rpos[s] = pos_in_bucket % kStreamPassRows;
+        s_rpos[s] = desc & 255;
     }
+    if (threadIdx.x == 0) s_n = 0;
     __syncthreads();
     if (threadIdx.x == 0) {
         int run = 0;
-        for (int s = 0; s < c.k_groups; ++s) { s_base[s] = run; run += s_cnt[s]; }
+        for (int s = 0; s < c.k_groups; ++s) { const int cnt = s_base[s]; s_base[s] = run; run += cnt; }
         s_base[c.k_groups] = run;
     }
     __syncthreads();
-    const int P = s_base[c.k_groups];
-    const int C = P * c.k_tokens;
-    float* cv = (C <= smem_cands) ? reinterpret_cast<float*>(msm) : cand_val_scratch + (size_t)m * cand_cap;
-    int32_t* ci = (C <= smem_cands) ? reinterpret_cast<int32_t*>(msm + sizeof(float) * smem_cands)
-                                    : cand_id_scratch + (size_t)m * cand_cap;
-
-    // piece q -> index of its partial; P <= grid + 2 * k_groups
-    __shared__ int s_piece[kMergeMaxPieces];
+    const int P = min(s_base[c.k_groups], kMergeMaxPieces);
     for (int q = threadIdx.x; q < P; q += kMergeStreamThreads) {
         int s = 0;
         while (s + 1 < c.k_groups && s_base[s + 1] <= q) ++s;
         const int b = s_first[s] + (q - s_base[s]);
         const int seg = s_j[s] - (b * per) / g.T;
-        s_piece[min(q, kMergeMaxPieces - 1)] = (int)(((size_t)b * g.seg_max + seg) * kStreamPassRows + s_rpos[s]);
+        s_piece[q] = (int)(((size_t)b * g.seg_max + seg) * kStreamPassRows + s_rpos[s]);
     }
     __syncthreads();
-    float mx = kNegInf;
-    for (int q = threadIdx.x; q < P; q += kMergeStreamThreads) mx = fmaxf(mx, pp.pmax[s_piece[min(q, kMergeMaxPieces - 1)]]);
-    for (int idx = threadIdx.x; idx < C; idx += kMergeStreamThreads) {
-        const int q = idx / c.k_tokens, i = idx - q * c.k_tokens;
-        const size_t p = (size_t)s_piece[min(q, kMergeMaxPieces - 1)];
-        cv[idx] = pp.pval[p * c.k_tokens + i];
-        ci[idx] = pp.pid[p * c.k_tokens + i];
+
+    pdl_wait();                   // partials of the streaming kernel are complete from here on
+
+    // pass 1 over the pieces: joint log-sum-exp and the candidate threshold
+    float mx = kNegInf, thr = kNegInf;
+    for (int q = threadIdx.x; q < P; q += kMergeStreamThreads) {
+        const size_t p = (size_t)s_piece[q];
+        mx = fmaxf(mx, pp.pmax[p]);
+        thr = fmaxf(thr, pp.pval[p * c.k_tokens + c.k_tokens - 1]);
     }
     mx = warp_max(mx);
-    if (lane == 0) s_f[warp] = mx;
+    thr = warp_max(thr);
+    if (lane == 0) { s_f[warp] = mx; s_t[warp] = thr; }
     __syncthreads();
     mx = s_f[0];
+    thr = s_t[0];
 #pragma unroll
-    for (int w = 1; w < kWarps; ++w) mx = fmaxf(mx, s_f[w]);
+    for (int w = 1; w < kWarps; ++w) { mx = fmaxf(mx, s_f[w]); thr = fmaxf(thr, s_t[w]); }
     __syncthreads();
     float sum = 0.f;
     for (int q = threadIdx.x; q < P; q += kMergeStreamThreads) {
-        const int p = s_piece[min(q, kMergeMaxPieces - 1)];
+        const int p = s_piece[q];
         sum += pp.psum[p] * expf(pp.pmax[p] - mx);
     }
     sum = warp_sum(sum);
     if (lane == 0) s_f[warp] = sum;
+
+    // pass 2: keep the candidates at or above the threshold (order of arrival does not matter: the
+    // ranking below is by the total order (value desc, token id asc))
+    const int C = P * c.k_tokens;
+    const int cap = (C <= smem_cands) ? smem_cands : cand_cap;
+    float* cv = (C <= smem_cands) ? reinterpret_cast<float*>(msm) : cand_val_scratch + (size_t)m * cand_cap;
+    int32_t* ci = (C <= smem_cands) ? reinterpret_cast<int32_t*>(msm + sizeof(float) * smem_cands)
+                                    : cand_id_scratch + (size_t)m * cand_cap;
+    for (int q = warp; q < P; q += kWarps) {
+        const size_t p = (size_t)s_piece[q];
+        if (lane < c.k_tokens) {
+            const float v = pp.pval[p * c.k_tokens + lane];
+            const int id = pp.pid[p * c.k_tokens + lane];
+            if (id != kNoToken && v >= thr) {
+                const int at = atomicAdd(&s_n, 1);
+                if (at < cap) { cv[at] = v; ci[at] = id; }
+            }
+        }
+    }
     __syncthreads();
     if (threadIdx.x == 0) {
         float tot = 0.f;
@@ -476,52 +497,49 @@ __global__ void __launch_bounds__(kMergeStreamThreads) merge_stream_kernel(CallV
     }
     __syncthreads();
     const float lse = s_lse;
+    const int S = min(s_n, cap);
 
-    // Token ids are unique across the candidates, so "strictly after the last pick in (value desc, id asc)
-    // order" selects the next one without marking.  Two levels: every warp picks the k_tokens best of its
-    // strided share, then warp 0 picks the k_tokens best of those.
-    __shared__ float s_wv[kWarps][kMaxKTokens];
-    __shared__ int s_wi[kWarps][kMaxKTokens];
-    {
-        float last_v = __builtin_huge_valf();
-        int last_id = -1;
-        for (int k = 0; k < c.k_tokens; ++k) {
-            float bv = kNegInf;
-            int bk = kNoToken;
-            for (int i = threadIdx.x; i < C; i += kMergeStreamThreads) {
-                const float v = cv[i];
-                const int id = ci[i];
-                const bool after = v < last_v || (v == last_v && id > last_id);
-                if (after && better(v, id, bv, bk)) { bv = v; bk = id; }
+    if (S <= kMergeRankMax) {
+        // rank by counting: survivor i goes to output position (number of survivors that beat it)
+        if (threadIdx.x < S) {
+            const float v = cv[threadIdx.x];
+            const int id = ci[threadIdx.x];
+            int rank = 0;
+            for (int i = 0; i < S; ++i) rank += better(cv[i], ci[i], v, id) ? 1 : 0;
+            if (rank < c.k_tokens) {
+                out_ids[(size_t)m * c.k_tokens + rank] = id;
+                out_logprobs[(size_t)m * c.k_tokens + rank] = v - lse;
             }
-            warp_argbest(bv, bk);
-            if (lane == k) { s_wv[warp][k] = bv; s_wi[warp][k] = bk; }
-            last_v = bv;
-            last_id = bk;
         }
+        return;
     }
-    __syncthreads();
-    if (warp == 0) {
-        const int C2 = kWarps * c.k_tokens;
-        float last_v = __builtin_huge_valf();
-        int last_id = -1;
-        for (int k = 0; k < c.k_tokens; ++k) {
-            float bv = kNegInf;
-            int bk = kNoToken;
-            for (int i = lane; i < C2; i += 32) {
-                const float v = s_wv[i / c.k_tokens][i % c.k_tokens];
-                const int id = s_wi[i / c.k_tokens][i % c.k_tokens];
-                const bool after = v < last_v || (v == last_v && id > last_id);
-                if (after && better(v, id, bv, bk)) { bv = v; bk = id; }
-            }
-            warp_argbest(bv, bk);
-            if (lane == 0) {
-                out_ids[(size_t)m * c.k_tokens + k] = bk;
-                out_logprobs[(size_t)m * c.k_tokens + k] = bv - lse;
-            }
-            last_v = bv;
-            last_id = bk;
+    // many survivors (short or tied lists): k rounds of "best strictly after the last pick"
+    __shared__ int s_i[kWarps];
+    float last_v = __builtin_huge_valf();
+    int last_id = -1;
+    for (int k = 0; k < c.k_tokens; ++k) {
+        float bv = kNegInf;
+        int bk = kNoToken;
+        for (int i = threadIdx.x; i < S; i += kMergeStreamThreads) {
+            const float v = cv[i];
+            const int id = ci[i];
+            const bool after = v < last_v || (v == last_v && id > last_id);
+            if (after && better(v, id, bv, bk)) { bv = v; bk = id; }
         }
+        warp_argbest(bv, bk);
+        __syncthreads();
+        if (lane == 0) { s_f[warp] = bv; s_i[warp] = bk; }
+        __syncthreads();
+        bv = s_f[0]; bk = s_i[0];
+#pragma unroll
+        for (int w = 1; w < kWarps; ++w)
+            if (better(s_f[w], s_i[w], bv, bk)) { bv = s_f[w]; bk = s_i[w]; }
+        if (threadIdx.x == 0) {
+            out_ids[(size_t)m * c.k_tokens + k] = bk;
+            out_logprobs[(size_t)m * c.k_tokens + k] = bv - lse;
+        }
+        last_v = bv;
+        last_id = bk;
     }
 }
 

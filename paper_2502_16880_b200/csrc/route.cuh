@@ -108,6 +108,7 @@ constexpr int kBucketThreads = 1024;
 __global__ void __launch_bounds__(kBucketThreads) bucket_kernel(CallView c) {
     __shared__ int s_count[kMaxGroups];
     __shared__ int s_offset[kMaxGroups + 1];
+    __shared__ int s_rank[kMaxGroups];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     constexpr int kWarps = kBucketThreads / 32;
     for (int n = warp; n < c.N; n += kWarps) {
@@ -125,6 +126,7 @@ __global__ void __launch_bounds__(kBucketThreads) bucket_kernel(CallView c) {
         for (int n = 0; n < c.N; ++n) {
             s_offset[n] = run;
             run += s_count[n];
+            s_rank[n] = virt;
             if (c.union_rank) c.union_rank[n] = s_count[n] > 0 ? virt : -1;
             if (s_count[n] > 0) {
                 const int passes = c.pass_rows > 0 ? (s_count[n] + c.pass_rows - 1) / c.pass_rows : 1;
@@ -153,7 +155,12 @@ __global__ void __launch_bounds__(kBucketThreads) bucket_kernel(CallView c) {
                 const int p = pos + __popc(bal & ((1u << lane) - 1u));
                 c.bucket_row[p] = m;
                 c.bucket_slot[p] = sl;
-                if (c.bucket_pos) c.bucket_pos[(size_t)m * c.k_groups + sl] = p - s_offset[n];
+                if (c.slot_desc) {
+                    const int pos_in_group = p - s_offset[n];
+                    const int pass = c.pass_rows > 0 ? pos_in_group / c.pass_rows : 0;
+                    c.slot_desc[(size_t)m * c.k_groups + sl] =
+                        ((s_rank[n] + pass) << 8) | ((pos_in_group - pass * max(c.pass_rows, 1)) & 255);
+                }
             }
             pos += __popc(bal);
         }
@@ -166,7 +173,7 @@ __global__ void __launch_bounds__(kBucketThreads) bucket_kernel(CallView c) {
 template <int NPER>
 __device__ __forceinline__ void route_select_row(const CallView& c, const int32_t* __restrict__ forced,
                                                  int32_t* __restrict__ groups_tap, int m, int lane, float* s_val,
-                                                 int16_t* s_slot_row) {
+                                                 int16_t* s_slot_row, unsigned* s_rowmask) {
     int slot[NPER];
 #pragma unroll
     for (int i = 0; i < NPER; ++i) slot[i] = -1;
@@ -215,6 +222,7 @@ __device__ __forceinline__ void route_select_row(const CallView& c, const int32_
             s_slot_row[n] = (int16_t)slot[i];
             c.slot_of[(size_t)m * c.N + n] = (int16_t)slot[i];
             if (slot[i] >= 0) {
+                atomicOr(&s_rowmask[n], 1u << m);
                 c.sel[(size_t)m * c.k_groups + slot[i]] = n;
                 if (groups_tap) groups_tap[(size_t)m * c.k_groups + slot[i]] = n;
             }
@@ -236,8 +244,8 @@ __global__ void __launch_bounds__(kRouteThreads)
                        float* __restrict__ gate_tap) {
     __shared__ int16_t s_slot[kRouteFusedMaxM][kMaxGroups];
     __shared__ float s_val[kRouteThreads / 32][kMaxGroups];
-    __shared__ int s_count[kMaxGroups];
-    __shared__ int s_offset[kMaxGroups + 1];
+    __shared__ unsigned s_rowmask[kMaxGroups];     // bit m: row m selected the group
+    __shared__ int s_warp_tot[kRouteThreads / 32];
     __shared__ float s_red[kRouteThreads / 32][8];
     __shared__ int s_last;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -287,80 +295,64 @@ __global__ void __launch_bounds__(kRouteThreads)
         if (s_last) c.state->ticket = 0;          // ready for the next call on this handle
         __threadfence();
     }
+    s_rowmask[threadIdx.x] = 0;                     // kRouteThreads == kMaxGroups
     __syncthreads();
     if (!s_last) return;
 
     // groups of every row: one warp per row
     for (int m = warp; m < c.M; m += kWarps) {
-        if (c.N <= 32) route_select_row<1>(c, forced, groups_tap, m, lane, s_val[warp], s_slot[m]);
-        else if (c.N <= 64) route_select_row<2>(c, forced, groups_tap, m, lane, s_val[warp], s_slot[m]);
-        else if (c.N <= 128) route_select_row<4>(c, forced, groups_tap, m, lane, s_val[warp], s_slot[m]);
-        else route_select_row<8>(c, forced, groups_tap, m, lane, s_val[warp], s_slot[m]);
+        if (c.N <= 32) route_select_row<1>(c, forced, groups_tap, m, lane, s_val[warp], s_slot[m], s_rowmask);
+        else if (c.N <= 64) route_select_row<2>(c, forced, groups_tap, m, lane, s_val[warp], s_slot[m], s_rowmask);
+        else if (c.N <= 128) route_select_row<4>(c, forced, groups_tap, m, lane, s_val[warp], s_slot[m], s_rowmask);
+        else route_select_row<8>(c, forced, groups_tap, m, lane, s_val[warp], s_slot[m], s_rowmask);
     }
     __syncthreads();
 
-    constexpr int kPer = kMaxGroups / 32;
-    // rows per group (M <= 32: one ballot per group)
-    for (int n = warp; n < c.N; n += kWarps) {
-        const bool in = lane < c.M && s_slot[lane][n] >= 0;
-        const unsigned bal = __ballot_sync(0xffffffffu, in);
-        if (lane == 0) s_count[n] = __popc(bal);
+    // One thread per group: rows that selected it, passes over its weights, and (by a block-wide exclusive
+    // scan of both counts, packed in one word) its place in the bucket array and in the union list.
+    const int n = threadIdx.x;
+    const unsigned mask = n < c.N ? s_rowmask[n] : 0u;
+    const int cnt = __popc(mask);
+    const int passes = cnt == 0 ? 0 : (c.pass_rows > 0 ? (cnt + c.pass_rows - 1) / c.pass_rows : 1);
+    const int packed = cnt | (passes << 16);
+    int incl = packed;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int a = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += a;
     }
-    __syncthreads();
-    if (warp == 0) {
-        // exclusive scan of the counts and numbering of the (group, pass) entries, 8 consecutive groups per lane
-        int cnt[kPer], passes[kPer], tot = 0, vtot = 0, utot = 0;
+    if (lane == 31) s_warp_tot[warp] = incl;
+    const int n_union = __syncthreads_count(cnt > 0);
+    int before = 0, total = 0;
 #pragma unroll
-        for (int i = 0; i < kPer; ++i) {
-            const int n = lane * kPer + i;
-            cnt[i] = n < c.N ? s_count[n] : 0;
-            passes[i] = cnt[i] == 0 ? 0 : (c.pass_rows > 0 ? (cnt[i] + c.pass_rows - 1) / c.pass_rows : 1);
-            tot += cnt[i];
-            vtot += passes[i];
-            utot += cnt[i] > 0;
-        }
-        int ex = tot, vex = vtot, uex = utot;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const int a = __shfl_up_sync(0xffffffffu, ex, o), b = __shfl_up_sync(0xffffffffu, vex, o);
-            const int d = __shfl_up_sync(0xffffffffu, uex, o);
-            if (lane >= o) { ex += a; vex += b; uex += d; }
-        }
-        const int all = __shfl_sync(0xffffffffu, ex, 31), vall = __shfl_sync(0xffffffffu, vex, 31);
-        const int uall = __shfl_sync(0xffffffffu, uex, 31);
-        int run = ex - tot, virt = vex - vtot;
-#pragma unroll
-        for (int i = 0; i < kPer; ++i) {
-            const int n = lane * kPer + i;
-            if (n < c.N) {
-                s_offset[n] = run;
-                c.group_offset[n] = run;
-                c.group_count[n] = cnt[i];
-                c.union_rank[n] = cnt[i] > 0 ? virt : -1;
-                for (int p = 0; p < passes[i]; ++p)
-                    if (virt + p < c.union_cap) c.union_list[virt + p] = n | (p << 16);
-                run += cnt[i];
-                virt += passes[i];
-            }
-        }
-        if (lane == 0) {
-            s_offset[c.N] = all;
-            c.group_offset[c.N] = all;
-            c.state->n_union = uall;
-            c.state->n_virtual = min(vall, c.union_cap);
+    for (int w = 0; w < kWarps; ++w) {
+        const int t = s_warp_tot[w];
+        if (w < warp) before += t;
+        total += t;
+    }
+    const int excl = before + incl - packed;
+    const int off = excl & 0xffff, virt = excl >> 16;
+    if (n < c.N) {
+        c.group_offset[n] = off;
+        c.group_count[n] = cnt;
+        c.union_rank[n] = cnt > 0 ? virt : -1;
+        for (int p = 0; p < passes; ++p)
+            if (virt + p < c.union_cap) c.union_list[virt + p] = n | (p << 16);
+        unsigned left = mask;
+        for (int pos = 0; left; ++pos) {
+            const int m = __ffs(left) - 1;
+            left &= left - 1;
+            const int sl = s_slot[m][n];
+            c.bucket_row[off + pos] = m;
+            c.bucket_slot[off + pos] = sl;
+            const int pass = c.pass_rows > 0 ? pos / c.pass_rows : 0;
+            c.slot_desc[(size_t)m * c.k_groups + sl] = ((virt + pass) << 8) | ((pos - pass * max(c.pass_rows, 1)) & 255);
         }
     }
-    __syncthreads();
-    for (int n = warp; n < c.N; n += kWarps) {
-        const int sl = lane < c.M ? (int)s_slot[lane][n] : -1;
-        const unsigned bal = __ballot_sync(0xffffffffu, sl >= 0);
-        if (sl >= 0) {
-            const int pos = __popc(bal & ((1u << lane) - 1u));
-            const int p = s_offset[n] + pos;
-            c.bucket_row[p] = lane;
-            c.bucket_slot[p] = sl;
-            c.bucket_pos[(size_t)lane * c.k_groups + sl] = pos;
-        }
+    if (threadIdx.x == 0) {
+        c.group_offset[c.N] = total & 0xffff;
+        c.state->n_union = n_union;
+        c.state->n_virtual = min(total >> 16, c.union_cap);
     }
 }
 
