@@ -271,7 +271,7 @@ def main():
     k_bytes = float(np.mean([u * cfg.v * cfg.H * 2 + cfg.M * cfg.H * 2 for u in ktouched]))
     k_ms = float(np.mean(kms))
     achieved = k_bytes / (k_ms * 1e-3) / 1e9
-    roofline = {"bound": "hbm", "kernel": "head_simt_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
+    roofline = {"bound": "hbm", "kernel": "head_stream_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
                 "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "traffic": None,
                 "avg_launch_us": k_ms * 1e3, "algorithmic_bytes_per_launch": k_bytes}
 

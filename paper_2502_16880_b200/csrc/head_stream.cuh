@@ -390,8 +390,9 @@ __global__ void __launch_bounds__(kStreamThreads, 1) head_stream_kernel(CallView
 
 // Merge for the streaming path: block per row.  The pieces of row m, slot s are the partials that the CTAs
 // overlapping that slot's (group, pass) wrote for the row's position in the pass.  Every piece holds a
-// sorted top-k list, so the largest of the pieces' k-th values is a lower bound of the row's k-th value:
-// only candidates at or above it are kept, and those few are ranked by counting.
+// sorted top-k list, so two lower bounds of the row's k-th value are at hand: the largest of the pieces'
+// k-th entries, and the k-th largest of the pieces' first entries.  Only candidates at or above the better
+// bound are kept, and those few are ranked by counting.
 constexpr int kMergeStreamThreads = 256;
 constexpr int kMergeMaxPieces = 1024;         // >= grid + 2 * k_groups for every supported shape
 constexpr int kMergeRankMax = 256;            // survivors ranked by counting; more fall back to k rounds
@@ -411,6 +412,8 @@ __global__ void __launch_bounds__(kMergeStreamThreads) merge_stream_kernel(CallV
     __shared__ int s_n;
     __shared__ int s_first[kMaxGroups], s_base[kMaxGroups + 1], s_rpos[kMaxGroups], s_j[kMaxGroups];
     __shared__ int s_piece[kMergeMaxPieces];
+    __shared__ float s_head[kMergeMaxPieces];
+    __shared__ float s_thr2;
 
     // The router's outputs were complete before the streaming kernel let this grid start.
     const int n_items = c.state->n_virtual * g.T;
@@ -425,7 +428,7 @@ __global__ void __launch_bounds__(kMergeStreamThreads) merge_stream_kernel(CallV
         s_j[s] = j;
         s_rpos[s] = desc & 255;
     }
-    if (threadIdx.x == 0) s_n = 0;
+    if (threadIdx.x == 0) { s_n = 0; s_thr2 = kNegInf; }
     __syncthreads();
     if (threadIdx.x == 0) {
         int run = 0;
@@ -445,12 +448,24 @@ __global__ void __launch_bounds__(kMergeStreamThreads) merge_stream_kernel(CallV
 
     pdl_wait();                   // partials of the streaming kernel are complete from here on
 
-    // pass 1 over the pieces: joint log-sum-exp and the candidate threshold
+    // pass 1 over the pieces (each thread owns up to kOwnPieces of them; all loads issued together):
+    // joint log-sum-exp and the candidate threshold
+    constexpr int kOwnPieces = kMergeMaxPieces / kMergeStreamThreads;
+    float pm[kOwnPieces], ps[kOwnPieces];
     float mx = kNegInf, thr = kNegInf;
-    for (int q = threadIdx.x; q < P; q += kMergeStreamThreads) {
-        const size_t p = (size_t)s_piece[q];
-        mx = fmaxf(mx, pp.pmax[p]);
-        thr = fmaxf(thr, pp.pval[p * c.k_tokens + c.k_tokens - 1]);
+#pragma unroll
+    for (int u = 0; u < kOwnPieces; ++u) {
+        const int q = threadIdx.x + u * kMergeStreamThreads;
+        pm[u] = kNegInf;
+        ps[u] = 0.f;
+        if (q < P) {
+            const size_t p = (size_t)s_piece[q];
+            pm[u] = pp.pmax[p];
+            ps[u] = pp.psum[p];
+            thr = fmaxf(thr, pp.pval[p * c.k_tokens + c.k_tokens - 1]);
+            s_head[q] = pp.pval[p * c.k_tokens];
+            mx = fmaxf(mx, pm[u]);
+        }
     }
     mx = warp_max(mx);
     thr = warp_max(thr);
@@ -460,30 +475,46 @@ __global__ void __launch_bounds__(kMergeStreamThreads) merge_stream_kernel(CallV
     thr = s_t[0];
 #pragma unroll
     for (int w = 1; w < kWarps; ++w) { mx = fmaxf(mx, s_f[w]); thr = fmaxf(thr, s_t[w]); }
-    __syncthreads();
-    float sum = 0.f;
+    // k-th largest first entry: the piece whose head is beaten by exactly k_tokens - 1 others (index breaks ties)
     for (int q = threadIdx.x; q < P; q += kMergeStreamThreads) {
-        const int p = s_piece[q];
-        sum += pp.psum[p] * expf(pp.pmax[p] - mx);
+        const float hq = s_head[q];
+        int rank = 0;
+        for (int i = 0; i < P; ++i) rank += better(s_head[i], i, hq, q) ? 1 : 0;
+        if (rank == c.k_tokens - 1) s_thr2 = hq;
     }
+    __syncthreads();
+    thr = fmaxf(thr, s_thr2);
+    float sum = 0.f;
+#pragma unroll
+    for (int u = 0; u < kOwnPieces; ++u) sum += ps[u] * expf(pm[u] - mx);     // exp(-inf) = 0 for unowned slots
     sum = warp_sum(sum);
     if (lane == 0) s_f[warp] = sum;
 
     // pass 2: keep the candidates at or above the threshold (order of arrival does not matter: the
-    // ranking below is by the total order (value desc, token id asc))
+    // ranking below is by the total order (value desc, token id asc)).  A warp reads four lists at a time.
     const int C = P * c.k_tokens;
     const int cap = (C <= smem_cands) ? smem_cands : cand_cap;
     float* cv = (C <= smem_cands) ? reinterpret_cast<float*>(msm) : cand_val_scratch + (size_t)m * cand_cap;
     int32_t* ci = (C <= smem_cands) ? reinterpret_cast<int32_t*>(msm + sizeof(float) * smem_cands)
                                     : cand_id_scratch + (size_t)m * cand_cap;
-    for (int q = warp; q < P; q += kWarps) {
-        const size_t p = (size_t)s_piece[q];
-        if (lane < c.k_tokens) {
-            const float v = pp.pval[p * c.k_tokens + lane];
-            const int id = pp.pid[p * c.k_tokens + lane];
-            if (id != kNoToken && v >= thr) {
+    for (int q0 = warp * 4; q0 < P; q0 += kWarps * 4) {
+        float v[4];
+        int id[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            v[u] = kNegInf;
+            id[u] = kNoToken;
+            if (q0 + u < P && lane < c.k_tokens) {
+                const size_t p = (size_t)s_piece[q0 + u];
+                v[u] = pp.pval[p * c.k_tokens + lane];
+                id[u] = pp.pid[p * c.k_tokens + lane];
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            if (id[u] != kNoToken && v[u] >= thr) {
                 const int at = atomicAdd(&s_n, 1);
-                if (at < cap) { cv[at] = v; ci[at] = id; }
+                if (at < cap) { cv[at] = v[u]; ci[at] = id[u]; }
             }
         }
     }
