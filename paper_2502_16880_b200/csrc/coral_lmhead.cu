@@ -116,7 +116,7 @@ Layout make_layout(const coral_lmhead_config& c) {
     L.T16 = (L.v + 15) / 16;
     L.kc = (c.H % 512 == 0) ? 512 : (c.H % 256 == 0) ? 256 : c.H;
     L.kstages = c.H / L.kc;
-    L.swz = (L.kc % 64 == 0) ? 1 : 0;
+    L.swz = 0;
     L.packed_bytes = (size_t)c.n_groups * L.T16 * 16 * H * 2;
     return L;
 }

@@ -197,7 +197,7 @@ __device__ __forceinline__ void stream_segment_mma(const CallView& c, const Stre
                 const uint32_t sp = ring + (uint32_t)stage * g.stage_bytes;
 #pragma unroll
                 for (int i = 0; i < KBW; ++i) {
-                    const uint32_t cb = ((uint32_t)(col0 + i * 32) * 2) ^ ((uint32_t)(gq & 1) << 6);   // chunk swizzle
+                    const uint32_t cb = ((uint32_t)(col0 + i * 32) * 2) ^ (c.swz ? ((uint32_t)(gq & 1) << 6) : 0u);   // chunk swizzle
                     const uint4 wg = lds128(sp + gq * g.row_stride + cb);
                     const uint4 wh = lds128(sp + (gq + 8) * g.row_stride + cb);
 #pragma unroll
