@@ -10,6 +10,7 @@
 #include "common.cuh"
 #include "head_simt.cuh"
 #include "head_stream.cuh"
+#include "head_tc.cuh"
 #include "merge.cuh"
 #include "route.cuh"
 
@@ -24,10 +25,12 @@ inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 struct Layout {
     size_t w_gate, group_tokens, state, gate, sel, slot_of, group_count, group_offset, bucket_row, bucket_slot,
         slot_desc, union_list, union_rank, part_max, part_sum, part_val, part_id, sp_max, sp_sum, sp_val, sp_id,
-        cand_val, cand_id, stage_hidden, stage_ids, stage_logprobs, total;
+        cand_val, cand_id, tc_hg, tc_max, tc_sum, tc_val, tc_id, stage_hidden, stage_ids, stage_logprobs, total;
     size_t packed_bytes, cand_cap;
     int v, T;
     int kc, kstages, swz, T16;   // packed layout (see packed_chunk_offset)
+    int tc_tiles, tc_vcap;       // tensor-core path: sub-tiles per group, capacity in (group, pass) entries
+    size_t tc_rows;              // rows of the gathered hidden matrix (0: path not provisioned)
 };
 
 bool config_ok(const coral_lmhead_config* c) {
@@ -109,6 +112,16 @@ Layout make_layout(const coral_lmhead_config& c) {
     L.part_sum = take(M * kg * T * 4);
     L.part_val = take(M * kg * T * kt * 4);
     L.part_id = take(M * kg * T * kt * 4);
+    // tensor-core path (only provisioned when calls can exceed the streaming path's row limit)
+    L.tc_tiles = (L.v + kTcSub - 1) / kTcSub;
+    L.tc_rows = M > (size_t)kStreamMaxM ? M * kg : 0;
+    L.tc_vcap = L.tc_rows ? (int)(N + (M * kg + kTcPassRows - 1) / kTcPassRows) : 0;
+    const size_t tcp = (size_t)L.tc_vcap * L.tc_tiles * kTcPassRows;
+    L.tc_hg = take(L.tc_rows * H * 2);
+    L.tc_max = take(tcp * 4);
+    L.tc_sum = take(tcp * 4);
+    L.tc_val = take(tcp * kt * 4);
+    L.tc_id = take(tcp * kt * 4);
     L.stage_hidden = take(M * H * 2);
     L.stage_ids = take(M * kt * 4);
     L.stage_logprobs = take(M * kt * 4);
@@ -144,6 +157,9 @@ struct coral_lmhead_s {
     int simt_smem;
     StreamGeom sg;
     int stream_smem;     // 0 if the streaming path is not available for this shape/device
+    bool tc_ok;          // tensor-core path available (maps encoded)
+    CUtensorMap map_w, map_h;
+    int sms;
     cudaEvent_t ev_head0, ev_head1;   // around the weight-streaming kernel when kernel timing is on
     cudaEvent_t ev_begin, ev_end;     // before the router stage / after the merge
     bool timing;
@@ -200,15 +216,64 @@ cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t s
     return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
 }
 
+// cuTensorMapEncodeTiled, looked up through the runtime so that the library does not link against libcuda.
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn() {
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) != cudaSuccess ||
+        q != cudaDriverEntryPointSuccess)
+        return nullptr;
+    return reinterpret_cast<EncodeTiledFn>(fn);
+}
+
+// Tensor maps of the tensor-core path: the packed weights as a 5-d tensor (column in slab, row in item, slab,
+// item, group) read in boxes of 64 columns x 128 rows (8 items), and the gathered hidden rows as a matrix
+// read in boxes of 64 columns x 128 rows; both land in shared memory with the 128-byte swizzle.
+bool make_tc_maps(coral_lmhead_s* h) {
+    EncodeTiledFn enc = encode_tiled_fn();
+    if (!enc) return false;
+    const Layout& L = h->L;
+    const cuuint64_t kc = (cuuint64_t)L.kc;
+    const cuuint64_t wdim[5] = {kc, 16, (cuuint64_t)L.kstages, (cuuint64_t)L.T16, (cuuint64_t)h->cfg.n_groups};
+    const cuuint64_t wstr[4] = {kc * 2, 16 * kc * 2, (cuuint64_t)L.kstages * 16 * kc * 2,
+                                (cuuint64_t)L.T16 * L.kstages * 16 * kc * 2};
+    const cuuint32_t wbox[5] = {(cuuint32_t)kTcK, 16, 1, 8, 1};
+    const cuuint32_t ones[5] = {1, 1, 1, 1, 1};
+    if (enc(&h->map_w, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, h->packed, wdim, wstr, wbox, ones,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return false;
+    const cuuint64_t hdim[2] = {(cuuint64_t)h->cfg.H, (cuuint64_t)L.tc_rows};
+    const cuuint64_t hstr[1] = {(cuuint64_t)h->cfg.H * 2};
+    const cuuint32_t hbox[2] = {(cuuint32_t)kTcK, (cuuint32_t)kTcBlockRows};
+    if (enc(&h->map_h, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, h->ws + L.tc_hg, hdim, hstr, hbox, ones,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return false;
+    return true;
+}
+
+constexpr size_t kTcSmemBytes = 1024 + (size_t)kTcStages * kTcStageBytes + 256;
+
 bool stream_ok(const coral_lmhead_s* h, int M) { return h->stream_smem > 0 && M <= kStreamMaxM; }
 
 // CORAL_PATH_STREAM: streaming kernel (M <= 128, H a multiple of 256, <= 4096); CORAL_PATH_SIMT_PLAIN: any shape.  Returns 0 if the
 // forced path cannot run this call.
+bool tc_usable(const coral_lmhead_s* h, int M, int kg) {
+    return h->tc_ok && (size_t)M * kg <= h->L.tc_rows && kg * h->L.tc_tiles <= kMergeMaxPieces &&
+           kg * h->L.tc_tiles * h->cfg.max_k_tokens <= kMergeSmemCands;
+}
+
 int choose_path(const coral_lmhead_s* h, int M, int kg) {
-    (void)kg;
     if (h->forced_path == CORAL_PATH_STREAM) return stream_ok(h, M) ? CORAL_PATH_STREAM : 0;
+    if (h->forced_path == CORAL_PATH_TCGEN05) return tc_usable(h, M, kg) ? CORAL_PATH_TCGEN05 : 0;
     if (h->forced_path != CORAL_PATH_AUTO) return h->forced_path;
-    return stream_ok(h, M) ? CORAL_PATH_STREAM : CORAL_PATH_SIMT_PLAIN;
+    if (stream_ok(h, M)) return CORAL_PATH_STREAM;
+    return tc_usable(h, M, kg) ? CORAL_PATH_TCGEN05 : CORAL_PATH_SIMT_PLAIN;
 }
 
 }  // namespace
@@ -299,6 +364,11 @@ int coral_lmhead_create(coral_lmhead_handle* out, const coral_lmhead_config* cfg
             cudaSuccess) { rc = CORAL_ERR_CUDA; break; }
         int sms = 0;
         if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) { rc = CORAL_ERR_CUDA; break; }
+        h->sms = sms;
+        h->tc_ok = false;
+        if (h->L.tc_rows > 0 && h->L.tc_vcap <= cfg->n_groups * kStreamMaxPasses && cfg->H >= kTcK && cfg->H % 8 == 0 && (int)kTcSmemBytes <= smem_optin &&
+            cudaFuncSetAttribute(head_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTcSmemBytes) == cudaSuccess)
+            h->tc_ok = make_tc_maps(h);
         h->sg = make_stream_geom(*cfg, sms, smem_optin);
         h->stream_smem = 0;
         if (cfg->H <= kStreamMaxH && cfg->H % 256 == 0 && sms >= kStreamGridMin && h->sg.n_stages >= 2) {
@@ -315,6 +385,7 @@ int coral_lmhead_create(coral_lmhead_handle* out, const coral_lmhead_config* cfg
         if (cudaMemcpyAsync(h->ws + h->L.w_gate, W_gate_dev, (size_t)N * cfg->H * 2, cudaMemcpyDeviceToDevice, st) !=
             cudaSuccess) { rc = CORAL_ERR_CUDA; break; }
         if (cudaMemsetAsync(h->ws + h->L.state, 0, sizeof(DeviceState), st) != cudaSuccess) { rc = CORAL_ERR_CUDA; break; }
+        if (cudaMemsetAsync(h->packed, 0, h->L.packed_bytes, st) != cudaSuccess) { rc = CORAL_ERR_CUDA; break; }
         pack_rows_kernel<<<V, 128, 0, st>>>(static_cast<const uint16_t*>(W_vocab_dev),
                                             reinterpret_cast<const int32_t*>(h->ws + h->L.group_tokens),
                                             reinterpret_cast<uint16_t*>(h->packed), cfg->H, v, h->L.kc, h->L.kstages,
@@ -344,7 +415,6 @@ int coral_lmhead_destroy(coral_lmhead_handle h) {
 
 int coral_lmhead_set_path(coral_lmhead_handle h, int path) {
     if (!h || path < CORAL_PATH_AUTO || path > CORAL_PATH_SIMT_PLAIN) return CORAL_ERR_INVALID;
-    if (path == CORAL_PATH_TCGEN05) return CORAL_ERR_INVALID;   // not built yet
     h->forced_path = path;
     return CORAL_OK;
 }
@@ -364,7 +434,8 @@ int coral_lmhead_draft_ex(coral_lmhead_handle h, const void* hidden_dev, int M, 
     CallView c = make_view(h, hidden_dev, M, k_groups, k_tokens);
     const int path = choose_path(h, M, k_groups);
     if (path == 0) return CORAL_ERR_INVALID;   // the forced path does not support this call
-    c.pass_rows = path == CORAL_PATH_STREAM ? kStreamPassRows : 0;
+    c.pass_rows = path == CORAL_PATH_STREAM ? kStreamPassRows : path == CORAL_PATH_TCGEN05 ? kTcPassRows : 0;
+    if (path == CORAL_PATH_TCGEN05) c.union_cap = h->L.tc_vcap;
     int launches = 0;
 
     if (h->timing) cudaEventRecord(h->ev_begin, st);
@@ -390,6 +461,24 @@ int coral_lmhead_draft_ex(coral_lmhead_handle h, const void* hidden_dev, int M, 
         ++launches;
         if (h->timing) cudaEventRecord(h->ev_head1, st);
         launch_pdl(merge_stream_kernel, dim3(M), dim3(kMergeStreamThreads), (size_t)kMergeSmemCands * 8, st, c, h->sg, pp,
+                   reinterpret_cast<float*>(h->ws + L.cand_val), reinterpret_cast<int32_t*>(h->ws + L.cand_id),
+                   (int)L.cand_cap, (int)kMergeSmemCands, out_ids_dev, out_logprobs_dev, out_lse_dev);
+        ++launches;
+    } else if (path == CORAL_PATH_TCGEN05) {
+        const Layout& L = h->L;
+        TcGeom tg{h->sms, L.tc_tiles, (cfg.H + kTcK - 1) / kTcK, L.kc};
+        TcPartials tp{reinterpret_cast<float*>(h->ws + L.tc_max), reinterpret_cast<float*>(h->ws + L.tc_sum),
+                      reinterpret_cast<float*>(h->ws + L.tc_val), reinterpret_cast<int32_t*>(h->ws + L.tc_id)};
+        tc_gather_kernel<<<M * k_groups, 128, 0, st>>>(c, reinterpret_cast<uint16_t*>(h->ws + L.tc_hg));
+        ++launches;
+        head_tc_kernel<<<tg.grid, kTcThreads, kTcSmemBytes, st>>>(c, tg, tp, h->map_w, h->map_h, out_logits_dev);
+        ++launches;
+        if (h->timing) cudaEventRecord(h->ev_head1, st);
+        StreamGeom mg = h->sg;
+        mg.tc_tiles = L.tc_tiles;
+        mg.T = L.tc_tiles;
+        StreamPartials pp{tp.pmax, tp.psum, tp.pval, tp.pid};
+        launch_pdl(merge_stream_kernel, dim3(M), dim3(kMergeStreamThreads), (size_t)kMergeSmemCands * 8, st, c, mg, pp,
                    reinterpret_cast<float*>(h->ws + L.cand_val), reinterpret_cast<int32_t*>(h->ws + L.cand_id),
                    (int)L.cand_cap, (int)kMergeSmemCands, out_ids_dev, out_logprobs_dev, out_lse_dev);
         ++launches;

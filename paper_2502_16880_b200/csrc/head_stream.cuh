@@ -45,6 +45,8 @@ struct StreamGeom {
     int T;            // items per group = ceil(v / kStreamTile)
     int row_stride;   // bytes between slab rows = kc * 2
     int stage_bytes;  // kStreamTile * row_stride: one slab, contiguous in the packed copy
+    int tc_tiles;     // 0: partials come from the streaming kernel; > 0: from the tensor-core kernel, which
+                      // writes one partial per (pass, sub-tile, row) with this many sub-tiles per pass
 };
 
 // One partial per (CTA, segment, hidden row of the pass).
@@ -417,12 +419,12 @@ __global__ void __launch_bounds__(kMergeStreamThreads) merge_stream_kernel(CallV
 
     // The router's outputs were complete before the streaming kernel let this grid start.
     const int n_items = c.state->n_virtual * g.T;
-    const int per = (n_items + g.grid - 1) / g.grid;
+    const int per = max(1, (n_items + g.grid - 1) / g.grid);
     for (int s = threadIdx.x; s < c.k_groups; s += kMergeStreamThreads) {
         const int desc = c.slot_desc[(size_t)m * c.k_groups + s];
         const int j = desc >> 8;
-        const int fb = (j * g.T) / per;
-        const int lb = ((j + 1) * g.T - 1) / per;
+        const int fb = g.tc_tiles > 0 ? j * g.tc_tiles : (j * g.T) / per;
+        const int lb = g.tc_tiles > 0 ? fb + g.tc_tiles - 1 : ((j + 1) * g.T - 1) / per;
         s_first[s] = fb;
         s_base[s] = lb - fb + 1;       // piece count, turned into an exclusive prefix below
         s_j[s] = j;
@@ -441,8 +443,12 @@ __global__ void __launch_bounds__(kMergeStreamThreads) merge_stream_kernel(CallV
         int s = 0;
         while (s + 1 < c.k_groups && s_base[s + 1] <= q) ++s;
         const int b = s_first[s] + (q - s_base[s]);
-        const int seg = s_j[s] - (b * per) / g.T;
-        s_piece[q] = (int)(((size_t)b * g.seg_max + seg) * kStreamPassRows + s_rpos[s]);
+        if (g.tc_tiles > 0) {
+            s_piece[q] = b * 256 + s_rpos[s];             // (pass * tiles + sub-tile) * rows per pass + row
+        } else {
+            const int seg = s_j[s] - (b * per) / g.T;
+            s_piece[q] = (int)(((size_t)b * g.seg_max + seg) * kStreamPassRows + s_rpos[s]);
+        }
     }
     __syncthreads();
 

@@ -1,0 +1,325 @@
+// Routed grouped GEMM for many query rows on the 5th-generation tensor cores.
+//
+// For every (group, pass) of the union list the rows that selected the group (gathered beforehand into one
+// contiguous bf16 matrix, up to 256 rows per pass) are multiplied with the group's vocab rows:
+//   D[hidden row, vocab row] = sum_k hg[row, k] * W[vocab row, k]
+// tcgen05.mma (kind::f16, bf16 x bf16 -> fp32) with M = 128 hidden rows per accumulator block (two blocks when
+// the pass has more than 128 rows) and N = 128 vocab rows per sub-tile (two sub-tiles per batch share one read
+// of the hidden rows).  Operands arrive through TMA tiled loads (128-byte swizzle) in a 3-stage ring;
+// accumulators live in tensor memory (4 x 128 columns).  The epilogue reads each thread's hidden row straight
+// from tensor memory and folds the logits into (max, sum-exp, top-k), one partial per (pass, sub-tile, row),
+// so logits never travel to HBM.  (CORAL Section 3.3: logits only for the activated groups; Appendix B: the
+// union of the rows' groups is what gets read.)
+//
+// Warp roles: warp 0 = TMA producer, warp 1 = MMA issuer and tensor-memory owner, warps 2..5 = epilogue
+// (warp w reads the 32 tensor-memory lanes of quarter w % 4).
+// Work split: all sub-tiles of all passes form one list; CTA b owns a contiguous run of it.
+#pragma once
+#include <cuda.h>
+
+#include "common.cuh"
+#include "head_stream.cuh"   // mbarrier helpers
+
+namespace coral {
+
+constexpr int kTcThreads = 192;
+constexpr int kTcSub = 128;          // vocab rows per sub-tile (MMA N)
+constexpr int kTcBlockRows = 128;    // hidden rows per accumulator block (MMA M)
+constexpr int kTcPassRows = 256;     // hidden rows per pass over a group's weights
+constexpr int kTcK = 64;             // columns per stage (one 128-byte swizzle atom of bf16)
+constexpr int kTcStages = 3;
+constexpr int kTcTileBytes = kTcBlockRows * kTcK * 2;   // 16 KiB: one 128 x 64 bf16 operand tile
+constexpr int kTcStageBytes = 4 * kTcTileBytes;         // A0, A1, B0, B1
+constexpr int kTcTmemCols = 512;
+constexpr int kTcSpin = 1 << 22;
+
+struct TcGeom {
+    int grid;
+    int tiles;        // sub-tiles per group = ceil(v / 128)
+    int ksteps;       // ceil(H / 64)
+    int kc;           // packed layout: columns per slab
+};
+
+struct TcPartials {
+    float* pmax;      // [pass][tiles][kTcPassRows]
+    float* psum;
+    float* pval;      // [...][k_tokens]
+    int32_t* pid;
+};
+
+__device__ __forceinline__ void tc_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, DeviceState* st) {
+    const int limit = *abort_flag ? 64 : kTcSpin;
+    for (int i = 0; i < limit; ++i)
+        if (mbar_try_wait(bar, parity)) return;
+    *abort_flag = 1;
+    set_status(st, -5);
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x0, int x1, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(map), "r"(x0), "r"(x1), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap* map, int x0, int x1, int x2, int x3,
+                                            int x4, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.5d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5, "
+        "%6}], [%7];"
+        ::"r"(dst), "l"(map), "r"(x0), "r"(x1), "r"(x2), "r"(x3), "r"(x4), "r"(bar) : "memory");
+}
+
+// Shared-memory matrix descriptor: K-major tile of 128-byte rows, 128-byte swizzle, 8-row groups 1024 bytes apart.
+__device__ __forceinline__ uint64_t tc_smem_desc(uint32_t saddr) {
+    return (uint64_t)((saddr >> 4) & 0x3FFF) | (1ull << 16) | (64ull << 32) | (1ull << 46) | (2ull << 61);
+}
+// Instruction descriptor: D = f32, A = B = bf16, both K-major, N = 128, M = 128.
+constexpr uint32_t kTcIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kTcSub >> 3) << 17) |
+                              ((uint32_t)(kTcBlockRows >> 4) << 24);
+
+__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(kTcIdesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+// 32 consecutive fp32 columns of this thread's tensor-memory lane.
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, float (&v)[32]) {
+    uint32_t r[32];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr));
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+// hg[p][:] = hidden[bucket_row[p]][:] for the M * k_groups (row, slot) pairs, bucket order.
+__global__ void __launch_bounds__(128) tc_gather_kernel(CallView c, uint16_t* __restrict__ hg) {
+    const int p = blockIdx.x;
+    const int m = c.bucket_row[p];
+    const uint4* src = reinterpret_cast<const uint4*>(c.hidden + (size_t)m * c.H);
+    uint4* dst = reinterpret_cast<uint4*>(hg + (size_t)p * c.H);
+    for (int ch = threadIdx.x; ch < (c.H >> 3); ch += 128) dst[ch] = __ldg(src + ch);
+}
+
+// Sorted insertion into a thread-private top-KT list (value desc, row index asc).
+template <int KT>
+__device__ __forceinline__ void tc_insert(float (&lv)[KT], int (&li)[KT], float v, int idx) {
+#pragma unroll
+    for (int j = 0; j < KT; ++j) {
+        if (better(v, idx, lv[j], li[j])) {
+            const float tv = lv[j];
+            const int ti = li[j];
+            lv[j] = v; li[j] = idx;
+            v = tv; idx = ti;
+        }
+    }
+}
+
+// Epilogue of one accumulator block for one thread (= one hidden row): fold nsub * 128 logits.
+template <int KT>
+__device__ __forceinline__ void tc_fold_row(const CallView& c, const TcPartials& pp, float* __restrict__ logits_tap,
+                                            uint32_t tmem_row, int mb, int nsub, int n, int row0, size_t pidx0,
+                                            bool row_valid, int tap_m, int tap_slot) {
+    float lv[KT];
+    int li[KT];
+#pragma unroll
+    for (int j = 0; j < KT; ++j) { lv[j] = kNegInf; li[j] = kNoToken; }
+    float mx = kNegInf, sum = 0.f;
+    for (int sub = 0; sub < nsub; ++sub) {
+        const int base = row0 + sub * kTcSub;
+        const int valid = min(kTcSub, c.v - base);
+#pragma unroll 1
+        for (int ch = 0; ch < 4; ++ch) {
+            float z[32];
+            tc_ld32(tmem_row + (uint32_t)((mb * 2 + sub) * kTcSub + ch * 32), z);
+            if (!row_valid) continue;
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+                const int col = ch * 32 + i;
+                if (col < valid) {
+                    const float v = z[i];
+                    if (logits_tap) logits_tap[((size_t)tap_m * c.k_groups + tap_slot) * c.v + base + col] = v;
+                    const float nm = fmaxf(mx, v);
+                    sum = sum * __expf(mx - nm) + __expf(v - nm);
+                    mx = nm;
+                    if (better(v, base + col, lv[KT - 1], li[KT - 1])) tc_insert<KT>(lv, li, v, base + col);
+                }
+            }
+        }
+    }
+    if (row_valid) {
+        pp.pmax[pidx0] = mx;
+        pp.psum[pidx0] = sum;
+#pragma unroll
+        for (int j = 0; j < KT; ++j) {
+            if (j < c.k_tokens) {
+                pp.pval[pidx0 * c.k_tokens + j] = lv[j];
+                pp.pid[pidx0 * c.k_tokens + j] = li[j] == kNoToken ? kNoToken : __ldg(c.group_tokens + (size_t)n * c.v + li[j]);
+            }
+        }
+    }
+}
+
+// grid = g.grid CTAs of kTcThreads threads; dynamic shared memory: 1 KiB alignment slack + kTcStages stages + barriers.
+__global__ void __launch_bounds__(kTcThreads, 1)
+    head_tc_kernel(CallView c, TcGeom g, TcPartials pp, const __grid_constant__ CUtensorMap map_w,
+                   const __grid_constant__ CUtensorMap map_h, float* __restrict__ logits_tap) {
+    extern __shared__ unsigned char tc_smem_raw[];
+    unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(tc_smem_raw) + 1023) & ~(uintptr_t)1023);
+    uint64_t* full = reinterpret_cast<uint64_t*>(smem + kTcStages * kTcStageBytes);
+    uint64_t* empty = full + kTcStages;
+    uint64_t* tmem_full = empty + kTcStages;
+    uint64_t* tmem_empty = tmem_full + 1;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tmem_empty + 1);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kTcStages; ++s) {
+            mbar_init(smem_u32(&full[s]), 1);
+            mbar_init(smem_u32(&empty[s]), 1);
+        }
+        mbar_init(smem_u32(tmem_full), 1);
+        mbar_init(smem_u32(tmem_empty), 4);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                     "r"(kTcTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    // this CTA's run of sub-tiles
+    const int n_tiles = c.state->n_virtual * g.tiles;
+    const int per = (n_tiles + g.grid - 1) / g.grid;
+    const int lo = min(n_tiles, (int)blockIdx.x * per);
+    const int hi = min(n_tiles, lo + per);
+
+    if (warp == 0) {
+        if (lane == 0) {
+            int stage = 0;
+            uint32_t phase = 0;
+            for (int pos = lo; pos < hi;) {
+                const int j = pos / g.tiles, t = pos - j * g.tiles;
+                const int nsub = (t + 1 < g.tiles && pos + 1 < hi) ? 2 : 1;
+                const int entry = c.union_list[j];
+                const int n = entry & 0xffff, pass = entry >> 16;
+                const int R = min(c.group_count[n] - pass * kTcPassRows, kTcPassRows);
+                const int nmb = R > kTcBlockRows ? 2 : 1;
+                const int hrow = c.group_offset[n] + pass * kTcPassRows;
+                const uint32_t bytes = (uint32_t)(nmb + nsub) * kTcTileBytes;
+                for (int ks = 0; ks < g.ksteps; ++ks) {
+                    tc_wait(smem_u32(&empty[stage]), phase ^ 1u, abort_flag, c.state);
+                    const uint32_t bar = smem_u32(&full[stage]);
+                    const uint32_t sb = smem_u32(smem + (size_t)stage * kTcStageBytes);
+                    mbar_expect_tx(bar, bytes);
+                    const int col = ks * kTcK;
+                    for (int mb = 0; mb < nmb; ++mb)
+                        tma_load_2d(sb + mb * kTcTileBytes, &map_h, col, hrow + mb * kTcBlockRows, bar);
+                    for (int sub = 0; sub < nsub; ++sub)
+                        tma_load_5d(sb + (2 + sub) * kTcTileBytes, &map_w, col % g.kc, 0, col / g.kc, (t + sub) * 8, n, bar);
+                    if (++stage == kTcStages) { stage = 0; phase ^= 1u; }
+                }
+                pos += nsub;
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            int stage = 0, batch = 0;
+            uint32_t phase = 0;
+            for (int pos = lo; pos < hi; ++batch) {
+                const int j = pos / g.tiles, t = pos - j * g.tiles;
+                const int nsub = (t + 1 < g.tiles && pos + 1 < hi) ? 2 : 1;
+                const int entry = c.union_list[j];
+                const int n = entry & 0xffff, pass = entry >> 16;
+                const int R = min(c.group_count[n] - pass * kTcPassRows, kTcPassRows);
+                const int nmb = R > kTcBlockRows ? 2 : 1;
+                tc_wait(smem_u32(tmem_empty), ((uint32_t)batch & 1u) ^ 1u, abort_flag, c.state);   // accumulators drained
+                tc_fence_after();
+                for (int ks = 0; ks < g.ksteps; ++ks) {
+                    tc_wait(smem_u32(&full[stage]), phase, abort_flag, c.state);
+                    tc_fence_after();
+                    const uint32_t sb = smem_u32(smem + (size_t)stage * kTcStageBytes);
+#pragma unroll
+                    for (int kk = 0; kk < kTcK / 16; ++kk) {
+                        for (int mb = 0; mb < nmb; ++mb) {
+                            const uint64_t adesc = tc_smem_desc(sb + mb * kTcTileBytes + kk * 32);
+                            for (int sub = 0; sub < nsub; ++sub) {
+                                const uint64_t bdesc = tc_smem_desc(sb + (2 + sub) * kTcTileBytes + kk * 32);
+                                tc_mma(tmem_base + (uint32_t)((mb * 2 + sub) * kTcSub), adesc, bdesc, (ks | kk) ? 1u : 0u);
+                            }
+                        }
+                    }
+                    tc_commit(smem_u32(&empty[stage]));       // the stage is free once these MMAs have read it
+                    if (++stage == kTcStages) { stage = 0; phase ^= 1u; }
+                }
+                tc_commit(smem_u32(tmem_full));               // accumulators complete
+                pos += nsub;
+            }
+        }
+    } else {
+        // epilogue: thread <-> tensor-memory lane = hidden row of the accumulator block
+        const int quarter = warp & 3;
+        const int row_in_block = quarter * 32 + lane;
+        const uint32_t tmem_row = tmem_base + ((uint32_t)(quarter * 32) << 16);
+        int batch = 0;
+        for (int pos = lo; pos < hi; ++batch) {
+            const int j = pos / g.tiles, t = pos - j * g.tiles;
+            const int nsub = (t + 1 < g.tiles && pos + 1 < hi) ? 2 : 1;
+            const int entry = c.union_list[j];
+            const int n = entry & 0xffff, pass = entry >> 16;
+            const int R = min(c.group_count[n] - pass * kTcPassRows, kTcPassRows);
+            const int nmb = R > kTcBlockRows ? 2 : 1;
+            const int hrow = c.group_offset[n] + pass * kTcPassRows;
+            tc_wait(smem_u32(tmem_full), (uint32_t)batch & 1u, abort_flag, c.state);
+            tc_fence_after();
+            for (int mb = 0; mb < nmb; ++mb) {
+                const int r = mb * kTcBlockRows + row_in_block;
+                const bool row_valid = r < R;
+                const int tap_m = row_valid ? c.bucket_row[hrow + r] : 0;
+                const int tap_slot = row_valid ? c.bucket_slot[hrow + r] : 0;
+                const size_t pidx0 = ((size_t)j * g.tiles + t) * kTcPassRows + r;
+                if (c.k_tokens <= 10)
+                    tc_fold_row<10>(c, pp, logits_tap, tmem_row, mb, nsub, n, t * kTcSub, pidx0, row_valid, tap_m, tap_slot);
+                else
+                    tc_fold_row<32>(c, pp, logits_tap, tmem_row, mb, nsub, n, t * kTcSub, pidx0, row_valid, tap_m, tap_slot);
+                if (nsub == 2 && row_valid) {            // the second sub-tile's partial is covered by the first
+                    const size_t p1 = pidx0 + kTcPassRows;
+                    pp.pmax[p1] = kNegInf;
+                    pp.psum[p1] = 0.f;
+                    for (int k = 0; k < c.k_tokens; ++k) { pp.pval[p1 * c.k_tokens + k] = kNegInf; pp.pid[p1 * c.k_tokens + k] = kNoToken; }
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(tmem_empty));
+            pos += nsub;
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTcTmemCols) : "memory");
+    }
+}
+
+}  // namespace coral

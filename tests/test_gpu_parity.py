@@ -202,3 +202,27 @@ def test_qwen_shape_group_sweep_and_dense_equivalence(path):
     same = (top.indices.cpu().numpy() == out["ids"]).mean()
     assert same > 0.99
     np.testing.assert_allclose(out["logprobs"], top.values.cpu().numpy(), atol=2e-3)
+
+
+@pytest.mark.parametrize("H,v,N,M,kg,kt", [
+    (256, 256, 16, 200, 4, 10),      # one accumulator block per pass, two sub-tiles per batch
+    (256, 256, 16, 300, 8, 10),      # groups with more than 128 rows: two accumulator blocks
+    (256, 256, 16, 600, 8, 32),      # more than 256 rows per group: second pass; long candidate lists
+    (320, 300, 6, 150, 2, 10),       # ragged group size (128 + 128 + 44) and H not a multiple of 256
+    (328, 300, 6, 150, 3, 5),        # last 64-column step only partly inside H
+])
+def test_tensor_core_path(H, v, N, M, kg, kt):
+    cfg = synth.HeadConfig("tc", H=H, V=v * N, N=N, k_groups=kg, k_tokens=kt, M=M, seed=7, w_std=0.05)
+    W, gm, Wg, hb = synth.make_all(cfg)
+    head = _head(cfg, W, gm, Wg, max_M=M, max_kg=kg, max_kt=32)
+    head.set_path(lmhead.CORAL_PATH_TCGEN05)
+    out = ph.gpu_draft_numpy(head, hb, kg, kt)
+    assert head.status() == 0
+    assert head.stats().path == lmhead.CORAL_PATH_TCGEN05
+    rows = np.unique(np.linspace(0, M - 1, 24).astype(int))
+    rep = ph.compare(W, gm, Wg, hb[rows], kg, kt, {k: a[rows] for k, a in out.items()})
+    assert rep.ok, rep.errors
+    again = ph.gpu_draft_numpy(head, hb, kg, kt)
+    for k in out:
+        assert np.array_equal(out[k], again[k]), k
+    head.close()
