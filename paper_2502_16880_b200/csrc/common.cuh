@@ -26,7 +26,7 @@ struct CallView {
     int union_cap;                 // capacity of union_list
     int pass_rows;                 // rows of a group handled per pass over its weights (0: one pass for any count)
     const uint16_t* packed;        // blocked copy of W_vocab, see packed_chunk_offset
-    int kc, kstages, swz, T16;     // packed layout: columns per slab, slabs per row, chunk swizzle, 16-row items per group
+    int KB, T16;                   // packed layout: 64-column blocks per row, 16-row items per group
     const uint16_t* w_gate;        // [N][H] bf16
     const int32_t* group_tokens;   // [N][v] global token id of packed row
     const uint16_t* hidden;        // [M][H] bf16
@@ -47,18 +47,16 @@ struct CallView {
     DeviceState* state;
 };
 
-// Packed layout of the LM head: per group, per item of 16 vocab rows (ascending token id), per slab of kc
-// columns: a contiguous [16 rows][kc] bf16 block, so that one slab is one contiguous bulk copy.  With swz
-// the 16-byte chunks of odd rows have bit 2 of their index flipped (the two 64-byte halves of every 128
-// bytes swapped), which keeps 128-bit shared-memory reads of two adjacent rows on disjoint banks.
-// Returns the offset, in 16-byte units, of logical chunk `ch` (8 columns) of row `j` of group `n`.
-__host__ __device__ __forceinline__ size_t packed_chunk_offset(int n, int j, int ch, int kc, int kstages, int swz,
-                                                               int T16) {
-    const int cpr = kc >> 3;                       // chunks per slab row
-    const int ks = ch / cpr, cc = ch - ks * cpr;
+// Packed layout of the LM head: [group][item of 16 vocab rows, ascending token id][block of 64 columns]
+// [16 rows][64 columns] bf16.  A 16-row item is contiguous (so a slab of 512 columns of an item is one
+// contiguous 16 KiB bulk copy) and every 16 x 64 block is a contiguous 2 KiB piece (so a 128-row x 64-column
+// operand tile is eight such pieces, fetched by one tiled TMA load).  Rows past the group's size and
+// columns past H are zero.
+// Returns the offset, in 16-byte units, of chunk `ch` (8 columns) of row `j` of group `n`.
+__host__ __device__ __forceinline__ size_t packed_chunk_offset(int n, int j, int ch, int KB, int T16) {
     const int item = j >> 4, r = j & 15;
-    const int phys = swz ? (cc ^ ((r & 1) << 2)) : cc;
-    return ((((size_t)n * T16 + item) * kstages + ks) * 16 + r) * cpr + phys;
+    const int kb = ch >> 3, cc = ch & 7;
+    return ((((size_t)n * T16 + item) * KB + kb) * 16 + r) * 8 + cc;
 }
 
 __device__ __forceinline__ float bf16_lo(uint32_t u) { return __uint_as_float(u << 16); }

@@ -28,7 +28,7 @@ struct Layout {
         cand_val, cand_id, tc_hg, tc_max, tc_sum, tc_val, tc_id, stage_hidden, stage_ids, stage_logprobs, total;
     size_t packed_bytes, cand_cap;
     int v, T;
-    int kc, kstages, swz, T16;   // packed layout (see packed_chunk_offset)
+    int KB, T16;                 // packed layout (see packed_chunk_offset)
     int tc_tiles, tc_vcap;       // tensor-core path: sub-tiles per group, capacity in (group, pass) entries
     size_t tc_rows;              // rows of the gathered hidden matrix (0: path not provisioned)
 };
@@ -61,8 +61,7 @@ StreamGeom make_stream_geom(const coral_lmhead_config& c, int sms, int smem_opti
     g.T = (v + kStreamTile - 1) / kStreamTile;
     g.kc = (c.H % 512 == 0) ? 512 : 256;
     g.kstages = c.H / g.kc;
-    g.row_stride = g.kc * 2;
-    g.stage_bytes = kStreamTile * g.row_stride;
+    g.stage_bytes = kStreamTile * g.kc * 2;
     const long fixed = (long)sizeof(float) * kStreamZBufs * kStreamWarps * kStreamTile * kStreamPassRows + 1024;
     long ns = ((long)smem_optin - fixed) / g.stage_bytes;
     g.n_stages = (int)(ns > 12 ? 12 : ns);
@@ -127,22 +126,20 @@ Layout make_layout(const coral_lmhead_config& c) {
     L.stage_logprobs = take(M * kt * 4);
     L.total = o;
     L.T16 = (L.v + 15) / 16;
-    L.kc = (c.H % 512 == 0) ? 512 : (c.H % 256 == 0) ? 256 : c.H;
-    L.kstages = c.H / L.kc;
-    L.swz = 0;
-    L.packed_bytes = (size_t)c.n_groups * L.T16 * 16 * H * 2;
+    L.KB = (c.H + 63) / 64;
+    L.packed_bytes = (size_t)c.n_groups * L.T16 * L.KB * 16 * 64 * 2;
     return L;
 }
 
 // Row i of group n of the packed copy = W_vocab[group_tokens[n][i]], in the blocked layout; one block per row.
 __global__ void pack_rows_kernel(const uint16_t* __restrict__ W, const int32_t* __restrict__ group_tokens,
-                                 uint16_t* __restrict__ packed, int H, int v, int kc, int kstages, int swz, int T16) {
+                                 uint16_t* __restrict__ packed, int H, int v, int KB, int T16) {
     const int row = blockIdx.x;
     const int n = row / v, j = row - n * v;
     const uint4* src = reinterpret_cast<const uint4*>(W + (size_t)group_tokens[row] * H);
     uint4* dst = reinterpret_cast<uint4*>(packed);
     for (int ch = threadIdx.x; ch < (H >> 3); ch += blockDim.x)
-        dst[packed_chunk_offset(n, j, ch, kc, kstages, swz, T16)] = __ldg(src + ch);
+        dst[packed_chunk_offset(n, j, ch, KB, T16)] = __ldg(src + ch);
 }
 
 }  // namespace
@@ -176,7 +173,7 @@ CallView make_view(const coral_lmhead_s* h, const void* hidden, int M, int kg, i
     c.M = M; c.H = h->cfg.H; c.V = h->cfg.V; c.N = h->cfg.n_groups; c.v = L.v; c.T = L.T;
     c.k_groups = kg; c.k_tokens = kt;
     c.packed = reinterpret_cast<const uint16_t*>(h->packed);
-    c.kc = L.kc; c.kstages = L.kstages; c.swz = L.swz; c.T16 = L.T16;
+    c.KB = L.KB; c.T16 = L.T16;
     c.w_gate = reinterpret_cast<const uint16_t*>(ws + L.w_gate);
     c.group_tokens = reinterpret_cast<const int32_t*>(ws + L.group_tokens);
     c.hidden = reinterpret_cast<const uint16_t*>(hidden);
@@ -230,17 +227,16 @@ EncodeTiledFn encode_tiled_fn() {
     return reinterpret_cast<EncodeTiledFn>(fn);
 }
 
-// Tensor maps of the tensor-core path: the packed weights as a 5-d tensor (column in slab, row in item, slab,
-// item, group) read in boxes of 64 columns x 128 rows (8 items), and the gathered hidden rows as a matrix
-// read in boxes of 64 columns x 128 rows; both land in shared memory with the 128-byte swizzle.
+// Tensor maps of the tensor-core path: the packed weights as a 5-d tensor (column in block, row in item,
+// 64-column block, item, group) read in boxes of 64 columns x 128 rows (8 items = eight contiguous 2 KiB
+// pieces), and the gathered hidden rows as a matrix read in boxes of 64 columns x 128 rows; both land in
+// shared memory with the 128-byte swizzle.
 bool make_tc_maps(coral_lmhead_s* h) {
     EncodeTiledFn enc = encode_tiled_fn();
     if (!enc) return false;
     const Layout& L = h->L;
-    const cuuint64_t kc = (cuuint64_t)L.kc;
-    const cuuint64_t wdim[5] = {kc, 16, (cuuint64_t)L.kstages, (cuuint64_t)L.T16, (cuuint64_t)h->cfg.n_groups};
-    const cuuint64_t wstr[4] = {kc * 2, 16 * kc * 2, (cuuint64_t)L.kstages * 16 * kc * 2,
-                                (cuuint64_t)L.T16 * L.kstages * 16 * kc * 2};
+    const cuuint64_t wdim[5] = {64, 16, (cuuint64_t)L.KB, (cuuint64_t)L.T16, (cuuint64_t)h->cfg.n_groups};
+    const cuuint64_t wstr[4] = {128, 2048, (cuuint64_t)L.KB * 2048, (cuuint64_t)L.T16 * L.KB * 2048};
     const cuuint32_t wbox[5] = {(cuuint32_t)kTcK, 16, 1, 8, 1};
     const cuuint32_t ones[5] = {1, 1, 1, 1, 1};
     if (enc(&h->map_w, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, h->packed, wdim, wstr, wbox, ones,
@@ -388,8 +384,7 @@ int coral_lmhead_create(coral_lmhead_handle* out, const coral_lmhead_config* cfg
         if (cudaMemsetAsync(h->packed, 0, h->L.packed_bytes, st) != cudaSuccess) { rc = CORAL_ERR_CUDA; break; }
         pack_rows_kernel<<<V, 128, 0, st>>>(static_cast<const uint16_t*>(W_vocab_dev),
                                             reinterpret_cast<const int32_t*>(h->ws + h->L.group_tokens),
-                                            reinterpret_cast<uint16_t*>(h->packed), cfg->H, v, h->L.kc, h->L.kstages,
-                                            h->L.swz, h->L.T16);
+                                            reinterpret_cast<uint16_t*>(h->packed), cfg->H, v, h->L.KB, h->L.T16);
         if (cudaGetLastError() != cudaSuccess) { rc = CORAL_ERR_CUDA; break; }
         if (cudaStreamSynchronize(st) != cudaSuccess) { rc = CORAL_ERR_CUDA; break; }
     } while (0);
@@ -466,7 +461,7 @@ int coral_lmhead_draft_ex(coral_lmhead_handle h, const void* hidden_dev, int M, 
         ++launches;
     } else if (path == CORAL_PATH_TCGEN05) {
         const Layout& L = h->L;
-        TcGeom tg{h->sms, L.tc_tiles, (cfg.H + kTcK - 1) / kTcK, L.kc};
+        TcGeom tg{h->sms, L.tc_tiles, L.KB};
         TcPartials tp{reinterpret_cast<float*>(h->ws + L.tc_max), reinterpret_cast<float*>(h->ws + L.tc_sum),
                       reinterpret_cast<float*>(h->ws + L.tc_val), reinterpret_cast<int32_t*>(h->ws + L.tc_id)};
         tc_gather_kernel<<<M * k_groups, 128, 0, st>>>(c, reinterpret_cast<uint16_t*>(h->ws + L.tc_hg));

@@ -43,8 +43,7 @@ struct StreamGeom {
     int n_stages;     // ring depth
     int seg_max;      // most virtual groups one CTA's run can overlap
     int T;            // items per group = ceil(v / kStreamTile)
-    int row_stride;   // bytes between slab rows = kc * 2
-    int stage_bytes;  // kStreamTile * row_stride: one slab, contiguous in the packed copy
+    int stage_bytes;  // 16 rows x kc columns: one slab, contiguous in the packed copy as kc / 64 blocks of [16][64]
     int tc_tiles;     // 0: partials come from the streaming kernel; > 0: from the tensor-core kernel, which
                       // writes one partial per (pass, sub-tile, row) with this many sub-tiles per pass
 };
@@ -199,9 +198,10 @@ __device__ __forceinline__ void stream_segment_mma(const CallView& c, const Stre
                 const uint32_t sp = ring + (uint32_t)stage * g.stage_bytes;
 #pragma unroll
                 for (int i = 0; i < KBW; ++i) {
-                    const uint32_t cb = ((uint32_t)(col0 + i * 32) * 2) ^ (c.swz ? ((uint32_t)(gq & 1) << 6) : 0u);   // chunk swizzle
-                    const uint4 wg = lds128(sp + gq * g.row_stride + cb);
-                    const uint4 wh = lds128(sp + (gq + 8) * g.row_stride + cb);
+                    const uint32_t cs = (uint32_t)(col0 + i * 32);             // column inside the slab
+                    const uint32_t at = sp + (cs >> 6) * 2048u + (uint32_t)gq * 128u + (cs & 63u) * 2u;
+                    const uint4 wg = lds128(at);
+                    const uint4 wh = lds128(at + 1024u);                        // row gq + 8
 #pragma unroll
                     for (int nt = 0; nt < NT; ++nt) {
                         const uint4 b = breg[nt][ks * KBW + i];
@@ -352,9 +352,9 @@ __global__ void __launch_bounds__(kStreamThreads, 1) head_stream_kernel(CallView
             const int seg_hi = min(sh.hi, (j + 1) * g.T);
             const int n = sh.segtab[min(j - sh.j_first, kStreamSegTab - 1)] & 0xffff;
             int t = pos - j * g.T;
-            const uint16_t* src = c.packed + ((((size_t)n * g.T + t) * g.kstages) * kStreamTile) * g.kc;
+            const uint16_t* src = c.packed + (((size_t)n * g.T + t) * g.kstages) * (size_t)(kStreamTile * g.kc);
             for (int item = pos; item < seg_hi; ++item, ++t) {
-                const uint32_t bytes = (uint32_t)min(kStreamTile, c.v - t * kStreamTile) * g.row_stride;
+                const uint32_t bytes = (uint32_t)g.stage_bytes;    // rows past the group's size are zero padding
                 for (int ks = 0; ks < g.kstages; ++ks) {
                     mbar_wait(smem_u32(&sh.empty[stage]), phase ^ 1u, sh.abort_flag, c.state);
                     const uint32_t bar = smem_u32(&sh.full[stage]);

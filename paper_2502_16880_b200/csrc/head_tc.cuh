@@ -36,8 +36,7 @@ constexpr int kTcSpin = 1 << 22;
 struct TcGeom {
     int grid;
     int tiles;        // sub-tiles per group = ceil(v / 128)
-    int ksteps;       // ceil(H / 64)
-    int kc;           // packed layout: columns per slab
+    int ksteps;       // ceil(H / 64) = 64-column blocks of the packed layout
 };
 
 struct TcPartials {
@@ -235,7 +234,7 @@ __global__ void __launch_bounds__(kTcThreads, 1)
                     for (int mb = 0; mb < nmb; ++mb)
                         tma_load_2d(sb + mb * kTcTileBytes, &map_h, col, hrow + mb * kTcBlockRows, bar);
                     for (int sub = 0; sub < nsub; ++sub)
-                        tma_load_5d(sb + (2 + sub) * kTcTileBytes, &map_w, col % g.kc, 0, col / g.kc, (t + sub) * 8, n, bar);
+                        tma_load_5d(sb + (2 + sub) * kTcTileBytes, &map_w, 0, 0, ks, (t + sub) * 8, n, bar);
                     if (++stage == kTcStages) { stage = 0; phase ^= 1u; }
                 }
                 pos += nsub;

@@ -226,3 +226,21 @@ def test_tensor_core_path(H, v, N, M, kg, kt):
     for k in out:
         assert np.array_equal(out[k], again[k]), k
     head.close()
+
+
+def test_large_m_routed_grouped_gemm():
+    """16 sequences x 60 tree nodes on the Llama3-8B shape: the tensor-core path, sampled rows against the oracle."""
+    cfg, W, gm, Wg, _ = _weights("llama3_8b")
+    M = 960
+    head = _head(cfg, W, gm, Wg, max_M=M, max_kg=cfg.k_groups, max_kt=cfg.k_tokens)
+    hb = synth.make_hidden(cfg, M)
+    ids, lps = head.draft(ph.to_dev_bf16(hb), cfg.k_groups, cfg.k_tokens)
+    torch.cuda.synchronize()
+    assert head.status() == 0
+    st = head.stats()
+    assert st.path == lmhead.CORAL_PATH_TCGEN05 and st.groups_touched == cfg.N
+    rows = np.unique(np.linspace(0, M - 1, 12).astype(int))
+    rep = ph.compare(W, gm, Wg, hb[rows], cfg.k_groups, cfg.k_tokens,
+                     {"ids": ids.cpu().numpy()[rows], "logprobs": lps.cpu().numpy()[rows]})
+    assert rep.ok, rep.errors
+    head.close()

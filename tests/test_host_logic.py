@@ -41,7 +41,7 @@ def test_error_strings_and_host_only_argument_checks(lib):
         assert lmhead.coral_lmhead_error_string(code) not in ("ok", "unknown status")
     ok = lmhead.make_config(4096, 128256, 64, 960, 8, 10)
     pb, wb = lmhead.coral_lmhead_query_sizes(ok)
-    assert pb == 64 * 126 * 16 * 4096 * 2 and wb > 0 and wb % 256 == 0   # groups x 16-row items x 16 x H x 2
+    assert pb == 64 * 126 * 16 * 4096 * 2 and wb > 0 and wb % 256 == 0   # groups x 16-row items x 64-column blocks x 16 x 64 x 2
     for bad in [lmhead.make_config(4096, 128256, 63, 8, 8, 10),     # V % N != 0
                 lmhead.make_config(4100, 128256, 64, 8, 8, 10),     # H % 8 != 0
                 lmhead.make_config(4096, 128256, 64, 0, 8, 10),
