@@ -4,15 +4,17 @@
 // contiguous bf16 matrix, up to 256 rows per pass) are multiplied with the group's vocab rows:
 //   D[hidden row, vocab row] = sum_k hg[row, k] * W[vocab row, k]
 // tcgen05.mma (kind::f16, bf16 x bf16 -> fp32) with M = 128 hidden rows per accumulator block (two blocks when
-// the pass has more than 128 rows) and N = 128 vocab rows per sub-tile (two sub-tiles per batch share one read
-// of the hidden rows).  Operands arrive through TMA tiled loads (128-byte swizzle) in a 3-stage ring;
-// accumulators live in tensor memory (4 x 128 columns).  The epilogue reads each thread's hidden row straight
-// from tensor memory and folds the logits into (max, sum-exp, top-k), one partial per (pass, sub-tile, row),
-// so logits never travel to HBM.  (CORAL Section 3.3: logits only for the activated groups; Appendix B: the
+// the pass has more than 128 rows) and N = 128 vocab rows per sub-tile.  A batch is two accumulators: two
+// sub-tiles sharing one read of the hidden rows, or one sub-tile for two row blocks.  Operands arrive through
+// TMA tiled loads (128-byte swizzle) in a 4-stage ring; accumulators live in tensor memory, double-buffered
+// (2 x 2 x 128 columns), so the epilogue of one batch runs under the MMAs of the next.  The epilogue reads
+// each thread's hidden row straight from tensor memory and folds the logits into (max, sum-exp, top-k), one
+// partial per (pass, sub-tile, row), so logits never travel to HBM.  (CORAL Section 3.3: logits only for the activated groups; Appendix B: the
 // union of the rows' groups is what gets read.)
 //
-// Warp roles: warp 0 = TMA producer, warp 1 = MMA issuer and tensor-memory owner, warps 2..5 = epilogue
-// (warp w reads the 32 tensor-memory lanes of quarter w % 4).
+// Warp roles: warp 0 = TMA producer, warp 1 = MMA issuer and tensor-memory owner, warps 2..9 = epilogue
+// (warp w reads the 32 tensor-memory lanes of quarter w % 4; warps 2..5 take the batch's first accumulator,
+// warps 6..9 the second).
 // Work split: all sub-tiles of all passes form one list; CTA b owns a contiguous run of it.
 #pragma once
 #include <cuda.h>
@@ -22,14 +24,15 @@
 
 namespace coral {
 
-constexpr int kTcThreads = 192;
+constexpr int kTcEpilogueWarps = 8;
+constexpr int kTcThreads = (2 + kTcEpilogueWarps) * 32;
 constexpr int kTcSub = 128;          // vocab rows per sub-tile (MMA N)
 constexpr int kTcBlockRows = 128;    // hidden rows per accumulator block (MMA M)
 constexpr int kTcPassRows = 256;     // hidden rows per pass over a group's weights
 constexpr int kTcK = 64;             // columns per stage (one 128-byte swizzle atom of bf16)
-constexpr int kTcStages = 3;
+constexpr int kTcStages = 4;
 constexpr int kTcTileBytes = kTcBlockRows * kTcK * 2;   // 16 KiB: one 128 x 64 bf16 operand tile
-constexpr int kTcStageBytes = 4 * kTcTileBytes;         // A0, A1, B0, B1
+constexpr int kTcStageBytes = 3 * kTcTileBytes;         // (A0, B0, B1) or (A0, A1, B0)
 constexpr int kTcTmemCols = 512;
 constexpr int kTcSpin = 1 << 22;
 
@@ -126,49 +129,78 @@ __device__ __forceinline__ void tc_insert(float (&lv)[KT], int (&li)[KT], float 
     }
 }
 
-// Epilogue of one accumulator block for one thread (= one hidden row): fold nsub * 128 logits.
+// Epilogue of one 128 x 128 accumulator for one thread (= one hidden row): fold the 128 logits of vocab rows
+// [base, base + valid) of group n into (max, sum-exp, top-k) and write the partial.
 template <int KT>
 __device__ __forceinline__ void tc_fold_row(const CallView& c, const TcPartials& pp, float* __restrict__ logits_tap,
-                                            uint32_t tmem_row, int mb, int nsub, int n, int row0, size_t pidx0,
-                                            bool row_valid, int tap_m, int tap_slot) {
+                                            uint32_t tmem_acc_row, int n, int base, size_t pidx, bool row_valid,
+                                            int tap_m, int tap_slot) {
+    constexpr float kLog2e = 1.4426950408889634f;
     float lv[KT];
     int li[KT];
 #pragma unroll
     for (int j = 0; j < KT; ++j) { lv[j] = kNegInf; li[j] = kNoToken; }
     float mx = kNegInf, sum = 0.f;
-    for (int sub = 0; sub < nsub; ++sub) {
-        const int base = row0 + sub * kTcSub;
-        const int valid = min(kTcSub, c.v - base);
+    const int valid = min(kTcSub, c.v - base);
 #pragma unroll 1
-        for (int ch = 0; ch < 4; ++ch) {
-            float z[32];
-            tc_ld32(tmem_row + (uint32_t)((mb * 2 + sub) * kTcSub + ch * 32), z);
-            if (!row_valid) continue;
+    for (int ch = 0; ch < 4; ++ch) {
+        float z[32];
+        tc_ld32(tmem_acc_row + (uint32_t)(ch * 32), z);
+        const int nv = min(32, valid - ch * 32);
+        if (!row_valid || nv <= 0) continue;
+        float cm = kNegInf;
 #pragma unroll
-            for (int i = 0; i < 32; ++i) {
-                const int col = ch * 32 + i;
-                if (col < valid) {
-                    const float v = z[i];
-                    if (logits_tap) logits_tap[((size_t)tap_m * c.k_groups + tap_slot) * c.v + base + col] = v;
-                    const float nm = fmaxf(mx, v);
-                    sum = sum * __expf(mx - nm) + __expf(v - nm);
-                    mx = nm;
-                    if (better(v, base + col, lv[KT - 1], li[KT - 1])) tc_insert<KT>(lv, li, v, base + col);
-                }
-            }
+        for (int i = 0; i < 32; ++i) cm = fmaxf(cm, i < nv ? z[i] : kNegInf);
+        const float nm = fmaxf(mx, cm);
+        float add = 0.f;
+#pragma unroll
+        for (int i = 0; i < 32; ++i) add += i < nv ? exp2f((z[i] - nm) * kLog2e) : 0.f;
+        sum = sum * exp2f((mx - nm) * kLog2e) + add;            // exp2(-inf) = 0 on the first chunk
+        mx = nm;
+        if (logits_tap) {
+            float* dst = logits_tap + ((size_t)tap_m * c.k_groups + tap_slot) * c.v + base + ch * 32;
+#pragma unroll
+            for (int i = 0; i < 32; ++i)
+                if (i < nv) dst[i] = z[i];
+        }
+        if (cm >= lv[KT - 1]) {
+#pragma unroll
+            for (int i = 0; i < 32; ++i)
+                if (i < nv && better(z[i], base + ch * 32 + i, lv[KT - 1], li[KT - 1]))
+                    tc_insert<KT>(lv, li, z[i], base + ch * 32 + i);
         }
     }
     if (row_valid) {
-        pp.pmax[pidx0] = mx;
-        pp.psum[pidx0] = sum;
+        pp.pmax[pidx] = mx;
+        pp.psum[pidx] = sum;
 #pragma unroll
         for (int j = 0; j < KT; ++j) {
             if (j < c.k_tokens) {
-                pp.pval[pidx0 * c.k_tokens + j] = lv[j];
-                pp.pid[pidx0 * c.k_tokens + j] = li[j] == kNoToken ? kNoToken : __ldg(c.group_tokens + (size_t)n * c.v + li[j]);
+                pp.pval[pidx * c.k_tokens + j] = lv[j];
+                pp.pid[pidx * c.k_tokens + j] = li[j] == kNoToken ? kNoToken : __ldg(c.group_tokens + (size_t)n * c.v + li[j]);
             }
         }
     }
+}
+
+// One batch of the run: the pass it belongs to, its first sub-tile, and how the two accumulators of the
+// batch are used: two sub-tiles of one 128-row block (nmb = 1, nsub = 2), one sub-tile of two blocks
+// (nmb = 2, nsub = 1), or a single accumulator.
+struct TcBatch {
+    int j, t, n, pass, R, nmb, nsub, hrow;
+};
+__device__ __forceinline__ TcBatch tc_batch_at(const CallView& c, const TcGeom& g, int pos, int hi) {
+    TcBatch b;
+    b.j = pos / g.tiles;
+    b.t = pos - b.j * g.tiles;
+    const int entry = c.union_list[b.j];
+    b.n = entry & 0xffff;
+    b.pass = entry >> 16;
+    b.R = min(c.group_count[b.n] - b.pass * kTcPassRows, kTcPassRows);
+    b.nmb = b.R > kTcBlockRows ? 2 : 1;
+    b.nsub = (b.nmb == 1 && b.t + 1 < g.tiles && pos + 1 < hi) ? 2 : 1;
+    b.hrow = c.group_offset[b.n] + b.pass * kTcPassRows;
+    return b;
 }
 
 // grid = g.grid CTAs of kTcThreads threads; dynamic shared memory: 1 KiB alignment slack + kTcStages stages + barriers.
@@ -179,9 +211,9 @@ __global__ void __launch_bounds__(kTcThreads, 1)
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(tc_smem_raw) + 1023) & ~(uintptr_t)1023);
     uint64_t* full = reinterpret_cast<uint64_t*>(smem + kTcStages * kTcStageBytes);
     uint64_t* empty = full + kTcStages;
-    uint64_t* tmem_full = empty + kTcStages;
-    uint64_t* tmem_empty = tmem_full + 1;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tmem_empty + 1);
+    uint64_t* tmem_full = empty + kTcStages;      // [2]
+    uint64_t* tmem_empty = tmem_full + 2;         // [2]
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tmem_empty + 2);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
@@ -190,8 +222,10 @@ __global__ void __launch_bounds__(kTcThreads, 1)
             mbar_init(smem_u32(&full[s]), 1);
             mbar_init(smem_u32(&empty[s]), 1);
         }
-        mbar_init(smem_u32(tmem_full), 1);
-        mbar_init(smem_u32(tmem_empty), 4);
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(smem_u32(&tmem_full[s]), 1);
+            mbar_init(smem_u32(&tmem_empty[s]), kTcEpilogueWarps);
+        }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -217,27 +251,21 @@ __global__ void __launch_bounds__(kTcThreads, 1)
             int stage = 0;
             uint32_t phase = 0;
             for (int pos = lo; pos < hi;) {
-                const int j = pos / g.tiles, t = pos - j * g.tiles;
-                const int nsub = (t + 1 < g.tiles && pos + 1 < hi) ? 2 : 1;
-                const int entry = c.union_list[j];
-                const int n = entry & 0xffff, pass = entry >> 16;
-                const int R = min(c.group_count[n] - pass * kTcPassRows, kTcPassRows);
-                const int nmb = R > kTcBlockRows ? 2 : 1;
-                const int hrow = c.group_offset[n] + pass * kTcPassRows;
-                const uint32_t bytes = (uint32_t)(nmb + nsub) * kTcTileBytes;
+                const TcBatch b = tc_batch_at(c, g, pos, hi);
+                const uint32_t bytes = (uint32_t)(b.nmb + b.nsub) * kTcTileBytes;
                 for (int ks = 0; ks < g.ksteps; ++ks) {
                     tc_wait(smem_u32(&empty[stage]), phase ^ 1u, abort_flag, c.state);
                     const uint32_t bar = smem_u32(&full[stage]);
                     const uint32_t sb = smem_u32(smem + (size_t)stage * kTcStageBytes);
                     mbar_expect_tx(bar, bytes);
-                    const int col = ks * kTcK;
-                    for (int mb = 0; mb < nmb; ++mb)
-                        tma_load_2d(sb + mb * kTcTileBytes, &map_h, col, hrow + mb * kTcBlockRows, bar);
-                    for (int sub = 0; sub < nsub; ++sub)
-                        tma_load_5d(sb + (2 + sub) * kTcTileBytes, &map_w, 0, 0, ks, (t + sub) * 8, n, bar);
+                    // tiles 0 and 1 of a stage are the hidden-row blocks, tiles 1/2 the weight sub-tiles
+                    for (int mb = 0; mb < b.nmb; ++mb)
+                        tma_load_2d(sb + mb * kTcTileBytes, &map_h, ks * kTcK, b.hrow + mb * kTcBlockRows, bar);
+                    for (int sub = 0; sub < b.nsub; ++sub)
+                        tma_load_5d(sb + (b.nmb + sub) * kTcTileBytes, &map_w, 0, 0, ks, (b.t + sub) * 8, b.n, bar);
                     if (++stage == kTcStages) { stage = 0; phase ^= 1u; }
                 }
-                pos += nsub;
+                pos += b.nsub;
             }
         }
     } else if (warp == 1) {
@@ -245,72 +273,62 @@ __global__ void __launch_bounds__(kTcThreads, 1)
             int stage = 0, batch = 0;
             uint32_t phase = 0;
             for (int pos = lo; pos < hi; ++batch) {
-                const int j = pos / g.tiles, t = pos - j * g.tiles;
-                const int nsub = (t + 1 < g.tiles && pos + 1 < hi) ? 2 : 1;
-                const int entry = c.union_list[j];
-                const int n = entry & 0xffff, pass = entry >> 16;
-                const int R = min(c.group_count[n] - pass * kTcPassRows, kTcPassRows);
-                const int nmb = R > kTcBlockRows ? 2 : 1;
-                tc_wait(smem_u32(tmem_empty), ((uint32_t)batch & 1u) ^ 1u, abort_flag, c.state);   // accumulators drained
+                const TcBatch b = tc_batch_at(c, g, pos, hi);
+                const int buf = batch & 1;
+                tc_wait(smem_u32(&tmem_empty[buf]), (((uint32_t)batch >> 1) & 1u) ^ 1u, abort_flag, c.state);   // drained
                 tc_fence_after();
+                const uint32_t acc = tmem_base + (uint32_t)(buf * 2 * kTcSub);
                 for (int ks = 0; ks < g.ksteps; ++ks) {
                     tc_wait(smem_u32(&full[stage]), phase, abort_flag, c.state);
                     tc_fence_after();
                     const uint32_t sb = smem_u32(smem + (size_t)stage * kTcStageBytes);
 #pragma unroll
                     for (int kk = 0; kk < kTcK / 16; ++kk) {
-                        for (int mb = 0; mb < nmb; ++mb) {
+                        for (int mb = 0; mb < b.nmb; ++mb) {
                             const uint64_t adesc = tc_smem_desc(sb + mb * kTcTileBytes + kk * 32);
-                            for (int sub = 0; sub < nsub; ++sub) {
-                                const uint64_t bdesc = tc_smem_desc(sb + (2 + sub) * kTcTileBytes + kk * 32);
-                                tc_mma(tmem_base + (uint32_t)((mb * 2 + sub) * kTcSub), adesc, bdesc, (ks | kk) ? 1u : 0u);
+                            for (int sub = 0; sub < b.nsub; ++sub) {
+                                const uint64_t bdesc = tc_smem_desc(sb + (b.nmb + sub) * kTcTileBytes + kk * 32);
+                                tc_mma(acc + (uint32_t)((mb + sub) * kTcSub), adesc, bdesc, (ks | kk) ? 1u : 0u);
                             }
                         }
                     }
                     tc_commit(smem_u32(&empty[stage]));       // the stage is free once these MMAs have read it
                     if (++stage == kTcStages) { stage = 0; phase ^= 1u; }
                 }
-                tc_commit(smem_u32(tmem_full));               // accumulators complete
-                pos += nsub;
+                tc_commit(smem_u32(&tmem_full[buf]));         // accumulators complete
+                pos += b.nsub;
             }
         }
     } else {
-        // epilogue: thread <-> tensor-memory lane = hidden row of the accumulator block
+        // epilogue: thread <-> tensor-memory lane = hidden row; the two warps of a lane quarter take one
+        // accumulator of the batch each
         const int quarter = warp & 3;
+        const int which = (warp - 2) >> 2;                    // accumulator 0 or 1 of the batch
         const int row_in_block = quarter * 32 + lane;
-        const uint32_t tmem_row = tmem_base + ((uint32_t)(quarter * 32) << 16);
         int batch = 0;
         for (int pos = lo; pos < hi; ++batch) {
-            const int j = pos / g.tiles, t = pos - j * g.tiles;
-            const int nsub = (t + 1 < g.tiles && pos + 1 < hi) ? 2 : 1;
-            const int entry = c.union_list[j];
-            const int n = entry & 0xffff, pass = entry >> 16;
-            const int R = min(c.group_count[n] - pass * kTcPassRows, kTcPassRows);
-            const int nmb = R > kTcBlockRows ? 2 : 1;
-            const int hrow = c.group_offset[n] + pass * kTcPassRows;
-            tc_wait(smem_u32(tmem_full), (uint32_t)batch & 1u, abort_flag, c.state);
+            const TcBatch b = tc_batch_at(c, g, pos, hi);
+            const int buf = batch & 1;
+            tc_wait(smem_u32(&tmem_full[buf]), ((uint32_t)batch >> 1) & 1u, abort_flag, c.state);
             tc_fence_after();
-            for (int mb = 0; mb < nmb; ++mb) {
+            if (which < b.nmb + b.nsub - 1) {
+                const int mb = b.nmb == 2 ? which : 0;
+                const int sub = b.nmb == 2 ? 0 : which;
                 const int r = mb * kTcBlockRows + row_in_block;
-                const bool row_valid = r < R;
-                const int tap_m = row_valid ? c.bucket_row[hrow + r] : 0;
-                const int tap_slot = row_valid ? c.bucket_slot[hrow + r] : 0;
-                const size_t pidx0 = ((size_t)j * g.tiles + t) * kTcPassRows + r;
+                const bool row_valid = r < b.R;
+                const int tap_m = row_valid ? c.bucket_row[b.hrow + r] : 0;
+                const int tap_slot = row_valid ? c.bucket_slot[b.hrow + r] : 0;
+                const size_t pidx = ((size_t)b.j * g.tiles + b.t + sub) * kTcPassRows + r;
+                const uint32_t acc_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)((buf * 2 + which) * kTcSub);
                 if (c.k_tokens <= 10)
-                    tc_fold_row<10>(c, pp, logits_tap, tmem_row, mb, nsub, n, t * kTcSub, pidx0, row_valid, tap_m, tap_slot);
+                    tc_fold_row<10>(c, pp, logits_tap, acc_row, b.n, (b.t + sub) * kTcSub, pidx, row_valid, tap_m, tap_slot);
                 else
-                    tc_fold_row<32>(c, pp, logits_tap, tmem_row, mb, nsub, n, t * kTcSub, pidx0, row_valid, tap_m, tap_slot);
-                if (nsub == 2 && row_valid) {            // the second sub-tile's partial is covered by the first
-                    const size_t p1 = pidx0 + kTcPassRows;
-                    pp.pmax[p1] = kNegInf;
-                    pp.psum[p1] = 0.f;
-                    for (int k = 0; k < c.k_tokens; ++k) { pp.pval[p1 * c.k_tokens + k] = kNegInf; pp.pid[p1 * c.k_tokens + k] = kNoToken; }
-                }
+                    tc_fold_row<32>(c, pp, logits_tap, acc_row, b.n, (b.t + sub) * kTcSub, pidx, row_valid, tap_m, tap_slot);
             }
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(tmem_empty));
-            pos += nsub;
+            if (lane == 0) mbar_arrive(smem_u32(&tmem_empty[buf]));
+            pos += b.nsub;
         }
     }
     tc_fence_before();
