@@ -253,7 +253,7 @@ bool make_tc_maps(coral_lmhead_s* h) {
     return true;
 }
 
-constexpr size_t kTcSmemBytes = 1024 + (size_t)kTcStages * kTcStageBytes + 256;
+constexpr size_t kTcSmemBytes = 1024 + (size_t)kTcStages * kTcStageBytes + 32 * kTcEpilogueThreads * 4 + 256;
 
 bool stream_ok(const coral_lmhead_s* h, int M) { return h->stream_smem > 0 && M <= kStreamMaxM; }
 
@@ -471,6 +471,7 @@ int coral_lmhead_draft_ex(coral_lmhead_handle h, const void* hidden_dev, int M, 
         if (h->timing) cudaEventRecord(h->ev_head1, st);
         StreamGeom mg = h->sg;
         mg.tc_tiles = L.tc_tiles;
+        mg.tc_rows = kTcPassRows;
         mg.T = L.tc_tiles;
         StreamPartials pp{tp.pmax, tp.psum, tp.pval, tp.pid};
         launch_pdl(merge_stream_kernel, dim3(M), dim3(kMergeStreamThreads), (size_t)kMergeSmemCands * 8, st, c, mg, pp,

@@ -44,6 +44,7 @@ struct StreamGeom {
     int seg_max;      // most virtual groups one CTA's run can overlap
     int T;            // items per group = ceil(v / kStreamTile)
     int stage_bytes;  // 16 rows x kc columns: one slab, contiguous in the packed copy as kc / 64 blocks of [16][64]
+    int tc_rows;      // rows per pass of the tensor-core kernel's partial layout
     int tc_tiles;     // 0: partials come from the streaming kernel; > 0: from the tensor-core kernel, which
                       // writes one partial per (pass, sub-tile, row) with this many sub-tiles per pass
 };
@@ -444,7 +445,7 @@ __global__ void __launch_bounds__(kMergeStreamThreads) merge_stream_kernel(CallV
         while (s + 1 < c.k_groups && s_base[s + 1] <= q) ++s;
         const int b = s_first[s] + (q - s_base[s]);
         if (g.tc_tiles > 0) {
-            s_piece[q] = b * 256 + s_rpos[s];             // (pass * tiles + sub-tile) * rows per pass + row
+            s_piece[q] = b * g.tc_rows + s_rpos[s];       // (pass * tiles + sub-tile) * rows per pass + row
         } else {
             const int seg = s_j[s] - (b * per) / g.T;
             s_piece[q] = (int)(((size_t)b * g.seg_max + seg) * kStreamPassRows + s_rpos[s]);

@@ -25,10 +25,13 @@
 namespace coral {
 
 constexpr int kTcEpilogueWarps = 8;
+constexpr int kTcEpilogueThreads = kTcEpilogueWarps * 32;
 constexpr int kTcThreads = (2 + kTcEpilogueWarps) * 32;
 constexpr int kTcSub = 128;          // vocab rows per sub-tile (MMA N)
 constexpr int kTcBlockRows = 128;    // hidden rows per accumulator block (MMA M)
-constexpr int kTcPassRows = 256;     // hidden rows per pass over a group's weights
+constexpr int kTcPassRows = 128;     // hidden rows per pass over a group's weights: one accumulator block, so
+                                     // that two weight sub-tiles share every read of the hidden rows (a group
+                                     // with more rows is read again; the re-read mostly hits L2)
 constexpr int kTcK = 64;             // columns per stage (one 128-byte swizzle atom of bf16)
 constexpr int kTcStages = 4;
 constexpr int kTcTileBytes = kTcBlockRows * kTcK * 2;   // 16 KiB: one 128 x 64 bf16 operand tile
@@ -134,7 +137,7 @@ __device__ __forceinline__ void tc_insert(float (&lv)[KT], int (&li)[KT], float 
 template <int KT>
 __device__ __forceinline__ void tc_fold_row(const CallView& c, const TcPartials& pp, float* __restrict__ logits_tap,
                                             uint32_t tmem_acc_row, int n, int base, size_t pidx, bool row_valid,
-                                            int tap_m, int tap_slot) {
+                                            int tap_m, int tap_slot, float* zs) {
     constexpr float kLog2e = 1.4426950408889634f;
     float lv[KT];
     int li[KT];
@@ -163,11 +166,20 @@ __device__ __forceinline__ void tc_fold_row(const CallView& c, const TcPartials&
             for (int i = 0; i < 32; ++i)
                 if (i < nv) dst[i] = z[i];
         }
-        if (cm >= lv[KT - 1]) {
+        // candidates for the top-k list: a bit per element that beats the current k-th entry; the few that do
+        // are fetched by index from a shared-memory copy of the chunk (element i of thread t at zs[i * T + t])
+        unsigned cand = 0;
 #pragma unroll
-            for (int i = 0; i < 32; ++i)
-                if (i < nv && better(z[i], base + ch * 32 + i, lv[KT - 1], li[KT - 1]))
-                    tc_insert<KT>(lv, li, z[i], base + ch * 32 + i);
+        for (int i = 0; i < 32; ++i)
+            cand |= (i < nv && z[i] >= lv[KT - 1]) ? (1u << i) : 0u;     // ties are settled by the insertion
+        if (cand) {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) zs[i * kTcEpilogueThreads] = z[i];
+            while (cand) {
+                const int i = __ffs(cand) - 1;
+                cand &= cand - 1;
+                tc_insert<KT>(lv, li, zs[i * kTcEpilogueThreads], base + ch * 32 + i);
+            }
         }
     }
     if (row_valid) {
@@ -209,7 +221,8 @@ __global__ void __launch_bounds__(kTcThreads, 1)
                    const __grid_constant__ CUtensorMap map_h, float* __restrict__ logits_tap) {
     extern __shared__ unsigned char tc_smem_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(tc_smem_raw) + 1023) & ~(uintptr_t)1023);
-    uint64_t* full = reinterpret_cast<uint64_t*>(smem + kTcStages * kTcStageBytes);
+    float* zstash = reinterpret_cast<float*>(smem + kTcStages * kTcStageBytes);          // [32][epilogue threads]
+    uint64_t* full = reinterpret_cast<uint64_t*>(smem + kTcStages * kTcStageBytes + 32 * kTcEpilogueThreads * 4);
     uint64_t* empty = full + kTcStages;
     uint64_t* tmem_full = empty + kTcStages;      // [2]
     uint64_t* tmem_empty = tmem_full + 2;         // [2]
@@ -305,6 +318,7 @@ __global__ void __launch_bounds__(kTcThreads, 1)
         const int quarter = warp & 3;
         const int which = (warp - 2) >> 2;                    // accumulator 0 or 1 of the batch
         const int row_in_block = quarter * 32 + lane;
+        float* zs = zstash + (threadIdx.x - 64);
         int batch = 0;
         for (int pos = lo; pos < hi; ++batch) {
             const TcBatch b = tc_batch_at(c, g, pos, hi);
@@ -321,9 +335,9 @@ __global__ void __launch_bounds__(kTcThreads, 1)
                 const size_t pidx = ((size_t)b.j * g.tiles + b.t + sub) * kTcPassRows + r;
                 const uint32_t acc_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)((buf * 2 + which) * kTcSub);
                 if (c.k_tokens <= 10)
-                    tc_fold_row<10>(c, pp, logits_tap, acc_row, b.n, (b.t + sub) * kTcSub, pidx, row_valid, tap_m, tap_slot);
+                    tc_fold_row<10>(c, pp, logits_tap, acc_row, b.n, (b.t + sub) * kTcSub, pidx, row_valid, tap_m, tap_slot, zs);
                 else
-                    tc_fold_row<32>(c, pp, logits_tap, acc_row, b.n, (b.t + sub) * kTcSub, pidx, row_valid, tap_m, tap_slot);
+                    tc_fold_row<32>(c, pp, logits_tap, acc_row, b.n, (b.t + sub) * kTcSub, pidx, row_valid, tap_m, tap_slot, zs);
             }
             tc_fence_before();
             __syncwarp();
