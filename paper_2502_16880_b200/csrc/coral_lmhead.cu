@@ -438,12 +438,15 @@ int coral_lmhead_draft_ex(coral_lmhead_handle h, const void* hidden_dev, int M, 
         route_fused_kernel<<<c.N, kRouteThreads, 0, st>>>(c, forced_groups_dev, out_groups_dev, out_gate_dev);
         ++launches;
     } else {
-        gate_kernel<<<dim3(c.N, (M + kGateRows - 1) / kGateRows), kGateThreads, 0, st>>>(c, out_gate_dev);
+        gate_tile_kernel<<<dim3((c.N + kGateTile - 1) / kGateTile, (M + kGateTile - 1) / kGateTile), 256, 0, st>>>(
+            c, out_gate_dev);
         ++launches;
         select_kernel<<<(M + kSelectWarps - 1) / kSelectWarps, kSelectWarps * 32, 0, st>>>(c, forced_groups_dev,
                                                                                           out_groups_dev);
         ++launches;
-        bucket_kernel<<<1, kBucketThreads, 0, st>>>(c);
+        count_groups_kernel<<<(M * k_groups + kSelectWarps * 32 - 1) / (kSelectWarps * 32), kSelectWarps * 32, 0, st>>>(c);
+        ++launches;
+        bucket_group_kernel<<<c.N, 256, 0, st>>>(c);
         ++launches;
     }
     if (h->timing) cudaEventRecord(h->ev_head0, st);

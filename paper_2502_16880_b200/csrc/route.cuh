@@ -356,4 +356,128 @@ __global__ void __launch_bounds__(kRouteThreads)
     }
 }
 
+
+// ---- router stage for many rows (M > kRouteFusedMaxM): three short kernels --------------------------------
+
+// Gate scores for a tile of 8 groups x 8 rows per block, so that every hidden row is read N/8 times and
+// every gate row M/8 times (from L2).  grid (ceil(N/8), ceil(M/8)).  Block (0,0) also clears the per-group
+// row counters that select_count_kernel accumulates.
+constexpr int kGateTile = 8;
+__global__ void __launch_bounds__(256) gate_tile_kernel(CallView c, float* __restrict__ gate_tap) {
+    __shared__ float s_red[8][kGateTile * kGateTile];
+    const int n0 = blockIdx.x * kGateTile, m0 = blockIdx.y * kGateTile;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int chunks = c.H >> 3;
+    if (blockIdx.x == 0 && blockIdx.y == 0)
+        for (int n = threadIdx.x; n < c.N; n += 256) c.group_count[n] = 0;
+    float acc[kGateTile][kGateTile];
+#pragma unroll
+    for (int g = 0; g < kGateTile; ++g)
+#pragma unroll
+        for (int r = 0; r < kGateTile; ++r) acc[g][r] = 0.f;
+    for (int ch = threadIdx.x; ch < chunks; ch += 256) {
+        float hf[kGateTile][8];
+#pragma unroll
+        for (int r = 0; r < kGateTile; ++r) {
+            const uint4 q = (m0 + r < c.M) ? __ldg(reinterpret_cast<const uint4*>(c.hidden + (size_t)(m0 + r) * c.H) + ch)
+                                           : make_uint4(0, 0, 0, 0);
+            hf[r][0] = bf16_lo(q.x); hf[r][1] = bf16_hi(q.x); hf[r][2] = bf16_lo(q.y); hf[r][3] = bf16_hi(q.y);
+            hf[r][4] = bf16_lo(q.z); hf[r][5] = bf16_hi(q.z); hf[r][6] = bf16_lo(q.w); hf[r][7] = bf16_hi(q.w);
+        }
+#pragma unroll
+        for (int g = 0; g < kGateTile; ++g) {
+            const uint4 q = (n0 + g < c.N) ? __ldg(reinterpret_cast<const uint4*>(c.w_gate + (size_t)(n0 + g) * c.H) + ch)
+                                           : make_uint4(0, 0, 0, 0);
+            const float w[8] = {bf16_lo(q.x), bf16_hi(q.x), bf16_lo(q.y), bf16_hi(q.y),
+                                bf16_lo(q.z), bf16_hi(q.z), bf16_lo(q.w), bf16_hi(q.w)};
+#pragma unroll
+            for (int r = 0; r < kGateTile; ++r)
+#pragma unroll
+                for (int e = 0; e < 8; ++e) acc[g][r] = fmaf(w[e], hf[r][e], acc[g][r]);
+        }
+    }
+#pragma unroll
+    for (int g = 0; g < kGateTile; ++g)
+#pragma unroll
+        for (int r = 0; r < kGateTile; ++r) {
+            const float sum = warp_sum(acc[g][r]);
+            if (lane == 0) s_red[warp][g * kGateTile + r] = sum;
+        }
+    __syncthreads();
+    if (threadIdx.x < kGateTile * kGateTile) {
+        const int g = threadIdx.x / kGateTile, r = threadIdx.x % kGateTile;
+        if (n0 + g < c.N && m0 + r < c.M) {
+            float sum = 0.f;
+#pragma unroll
+            for (int w = 0; w < 8; ++w) sum += s_red[w][threadIdx.x];
+            c.gate[(size_t)(m0 + r) * c.N + n0 + g] = sum;
+            if (gate_tap) gate_tap[(size_t)(m0 + r) * c.N + n0 + g] = sum;
+        }
+    }
+}
+
+// select_kernel plus per-group row counts (integer atomics: the totals do not depend on their order).
+__global__ void __launch_bounds__(kSelectWarps * 32) count_groups_kernel(CallView c) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < c.M * c.k_groups) atomicAdd(&c.group_count[c.sel[i]], 1);
+}
+
+// One block per group: the group's place in the bucket array and in the union list (prefix sums over the
+// per-group counts, recomputed by every block), then an ordered compaction of the rows that selected it.
+__global__ void __launch_bounds__(256) bucket_group_kernel(CallView c) {
+    __shared__ int s_cnt[kMaxGroups], s_pass[kMaxGroups];
+    __shared__ int s_warp[8];
+    const int n = blockIdx.x;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    {
+        const int t = threadIdx.x;
+        const int cnt = t < c.N ? c.group_count[t] : 0;
+        s_cnt[t] = cnt;
+        s_pass[t] = cnt == 0 ? 0 : (c.pass_rows > 0 ? (cnt + c.pass_rows - 1) / c.pass_rows : 1);
+    }
+    __syncthreads();
+    int off = 0, virt = 0, uni = 0, tot = 0, vtot = 0;
+    for (int t = 0; t < c.N; ++t) {           // N <= 256 shared-memory reads, same in every thread
+        if (t < n) { off += s_cnt[t]; virt += s_pass[t]; }
+        tot += s_cnt[t];
+        vtot += s_pass[t];
+        uni += s_cnt[t] > 0;
+    }
+    const int cnt = s_cnt[n], passes = s_pass[n];
+    if (threadIdx.x == 0) {
+        c.group_offset[n] = off;
+        c.union_rank[n] = cnt > 0 ? virt : -1;
+        for (int p = 0; p < passes; ++p)
+            if (virt + p < c.union_cap) c.union_list[virt + p] = n | (p << 16);
+        if (n == 0) {
+            c.group_offset[c.N] = tot;
+            c.state->n_union = uni;
+            c.state->n_virtual = min(vtot, c.union_cap);
+        }
+    }
+    int running = 0;
+    for (int m0 = 0; m0 < c.M; m0 += 256) {
+        const int m = m0 + threadIdx.x;
+        const int sl = m < c.M ? (int)c.slot_of[(size_t)m * c.N + n] : -1;
+        const unsigned bal = __ballot_sync(0xffffffffu, sl >= 0);
+        if (lane == 0) s_warp[warp] = __popc(bal);
+        __syncthreads();
+        int before = 0, all = 0;
+#pragma unroll
+        for (int w = 0; w < 8; ++w) {
+            if (w < warp) before += s_warp[w];
+            all += s_warp[w];
+        }
+        if (sl >= 0) {
+            const int pos = running + before + __popc(bal & ((1u << lane) - 1u));
+            c.bucket_row[off + pos] = m;
+            c.bucket_slot[off + pos] = sl;
+            const int pass = c.pass_rows > 0 ? pos / c.pass_rows : 0;
+            c.slot_desc[(size_t)m * c.k_groups + sl] = ((virt + pass) << 8) | ((pos - pass * max(c.pass_rows, 1)) & 255);
+        }
+        running += all;
+        __syncthreads();
+    }
+}
+
 }  // namespace coral
