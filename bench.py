@@ -341,6 +341,57 @@ def main():
             "torch_matmul_logsoftmax_topk_us": float(np.mean(tms)) * 1e3,
             "grouped_vs_dense_speedup": float(np.mean(ms_d)) / (tot_ms / args.steps),
         }
+        # large-M routed grouped GEMM (16 sequences x 60 tree nodes) on the tensor-core path, next to a dense
+        # 960 x V x H bf16 GEMM by torch (comparator only)
+        M_big = 960
+        big = lmhead.LMHead(Wd, torch.from_numpy(gm), dev_bf16(Wg), max_M=M_big, max_k_groups=cfg.k_groups,
+                            max_k_tokens=cfg.k_tokens)
+        hbig = [dev_bf16(synth.make_hidden(cfg, M_big, batch=100 + b)) for b in range(2)]
+        ids_b = torch.empty((M_big, cfg.k_tokens), dtype=torch.int32, device=dev)
+        lps_b = torch.empty((M_big, cfg.k_tokens), dtype=torch.float32, device=dev)
+        lmhead.coral_lmhead_set_kernel_timing(big.handle, True)
+        t_step, t_head = [], []
+        for i in range(13):
+            flush_l2(i)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            lmhead.coral_lmhead_draft(big.handle, hbig[i & 1], cfg.k_groups, cfg.k_tokens, ids_b, lps_b, stream)
+            b.record()
+            torch.cuda.synchronize()
+            if i >= 3:
+                t_step.append(a.elapsed_time(b))
+                t_head.append(lmhead.coral_lmhead_stage_ms(big.handle)[1])
+        assert big.status() == 0
+        st_big = big.stats()
+        flops = 2.0 * cfg.H * (M_big * cfg.N + M_big * cfg.k_groups * cfg.v)
+        pk = {}
+        if os.path.exists(os.path.join(ROOT, "MEASURED_PEAKS.json")):
+            with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+                pk = json.load(f)
+        tf_sust = float(pk.get("bf16_tflops_sustained", 1400.0))
+        tg = []
+        for i in range(8):
+            flush_l2(i)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            torch.matmul(hbig[0], Wd.T)
+            b.record()
+            torch.cuda.synchronize()
+            if i >= 3:
+                tg.append(a.elapsed_time(b))
+        head_us = float(np.mean(t_head)) * 1e3
+        out["large_m"] = {
+            "M": M_big, "path": int(st_big.path), "groups_touched": int(st_big.groups_touched),
+            "us_per_step": float(np.mean(t_step)) * 1e3, "grouped_gemm_stage_us": head_us,
+            "GBps_whole_step": st_big.algorithmic_bytes / (float(np.mean(t_step)) * 1e-3) / 1e9,
+            "GBps_grouped_gemm": st_big.weight_bytes / (head_us * 1e-6) / 1e9,
+            "hbm_frac_grouped_gemm": st_big.weight_bytes / (head_us * 1e-6) / 1e9 / peak,
+            "algorithmic_tflops_grouped_gemm": flops / (head_us * 1e-6) / 1e12,
+            "tensor_frac_of_sustained_peak": flops / (head_us * 1e-6) / 1e12 / tf_sust,
+            "tensor_frac_ceiling_at_hbm_roofline": flops / (st_big.weight_bytes / (peak * 1e9)) / 1e12 / tf_sust,
+            "torch_dense_gemm_960xVxH_us": float(np.mean(tg)) * 1e3,
+        }
+        big.close()
         out["clocks"] = sampler.stop()
         # CPU oracle on the host cores: whole steps of the same workload, bounded
         o_steps = 3

@@ -76,6 +76,7 @@ size_t stream_smem_bytes(const StreamGeom& g) {
            sizeof(int) * kStreamSegTab + 16;
 }
 
+constexpr int kTcMinRows = 96;          // above this many rows the tensor-core path is the faster one (measured)
 constexpr int kMergeSmemCands = 4096;   // candidates the streaming merge keeps in shared memory
 
 Layout make_layout(const coral_lmhead_config& c) {
@@ -113,7 +114,7 @@ Layout make_layout(const coral_lmhead_config& c) {
     L.part_id = take(M * kg * T * kt * 4);
     // tensor-core path (only provisioned when calls can exceed the streaming path's row limit)
     L.tc_tiles = (L.v + kTcSub - 1) / kTcSub;
-    L.tc_rows = M > (size_t)kStreamMaxM ? M * kg : 0;
+    L.tc_rows = M > (size_t)kTcMinRows ? M * kg : 0;
     L.tc_vcap = L.tc_rows ? (int)(N + (M * kg + kTcPassRows - 1) / kTcPassRows) : 0;
     const size_t tcp = (size_t)L.tc_vcap * L.tc_tiles * kTcPassRows;
     L.tc_hg = take(L.tc_rows * H * 2);
@@ -268,6 +269,7 @@ int choose_path(const coral_lmhead_s* h, int M, int kg) {
     if (h->forced_path == CORAL_PATH_STREAM) return stream_ok(h, M) ? CORAL_PATH_STREAM : 0;
     if (h->forced_path == CORAL_PATH_TCGEN05) return tc_usable(h, M, kg) ? CORAL_PATH_TCGEN05 : 0;
     if (h->forced_path != CORAL_PATH_AUTO) return h->forced_path;
+    if (M > kTcMinRows && tc_usable(h, M, kg)) return CORAL_PATH_TCGEN05;
     if (stream_ok(h, M)) return CORAL_PATH_STREAM;
     return tc_usable(h, M, kg) ? CORAL_PATH_TCGEN05 : CORAL_PATH_SIMT_PLAIN;
 }
