@@ -176,6 +176,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--rows", type=int, default=8, help="M of the headline workload")
     ap.add_argument("--quick", action="store_true", help="headline only: skip the other M, dense and CPU legs")
+    ap.add_argument("--large-m-only", type=int, default=0, metavar="M",
+                    help="run only the tensor-core leg with M rows (a short run for profilers) and print its line")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
@@ -204,6 +206,27 @@ def main():
         return torch.from_numpy(bits.view(np.int16)).to(dev).view(torch.bfloat16)
 
     Wd = dev_bf16(W)
+    if args.large_m_only:
+        Mb = args.large_m_only
+        big = lmhead.LMHead(Wd, torch.from_numpy(gm), dev_bf16(Wg), max_M=Mb, max_k_groups=cfg.k_groups,
+                            max_k_tokens=cfg.k_tokens)
+        hb = dev_bf16(synth.make_hidden(cfg, Mb, batch=100))
+        ids_b = torch.empty((Mb, cfg.k_tokens), dtype=torch.int32, device=dev)
+        lps_b = torch.empty((Mb, cfg.k_tokens), dtype=torch.float32, device=dev)
+        ts = []
+        for i in range(args.warmup + args.steps):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            lmhead.coral_lmhead_draft(big.handle, hb, cfg.k_groups, cfg.k_tokens, ids_b, lps_b)
+            b.record()
+            torch.cuda.synchronize()
+            if i >= args.warmup:
+                ts.append(a.elapsed_time(b))
+        st = big.stats()
+        print(json.dumps({"large_m_only": Mb, "path": int(st.path), "us_per_step": float(np.mean(ts)) * 1e3,
+                          "status": big.status()}))
+        big.close()
+        return
     head = lmhead.LMHead(Wd, torch.from_numpy(gm), dev_bf16(Wg), max_M=64, max_k_groups=cfg.N, max_k_tokens=cfg.k_tokens)
     flush = torch.empty(FLUSH_BYTES // 8, dtype=torch.int64, device=dev)
     stream = torch.cuda.current_stream()
