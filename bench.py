@@ -37,6 +37,10 @@ METRIC = "grouped LM-head draft-step HBM GB/s (algorithmic bytes of touched grou
 UNIT = "GB/s"
 WORKLOAD = "llama3_8b"
 N_BATCHES = 8            # distinct hidden batches rotated through the steps
+# DRAM bytes per algorithmic byte of the dominant kernel, from the ncu capture summarised in
+# profiles/head_stream_kernel_llama3_M8.md ((read + write) / weight bytes of the touched groups, two launches).
+# Set to None whenever that kernel changes until the capture is redone.
+STREAM_TRAFFIC_RATIO = 1.016
 FLUSH_BYTES = 512 << 20  # > 2x the 126 MB L2: written, then read back, between timed steps
 
 
@@ -295,7 +299,8 @@ def main():
     k_ms = float(np.mean(kms))
     achieved = k_bytes / (k_ms * 1e-3) / 1e9
     roofline = {"bound": "hbm", "kernel": "head_stream_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "traffic": None,
+                "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
+                "traffic": None if STREAM_TRAFFIC_RATIO is None else STREAM_TRAFFIC_RATIO * k_bytes,
                 "avg_launch_us": k_ms * 1e3, "algorithmic_bytes_per_launch": k_bytes}
 
     # end to end through the host-buffer entry point (pinned host memory; copies inside the timed region)
