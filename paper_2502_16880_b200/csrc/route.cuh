@@ -101,73 +101,6 @@ __global__ void __launch_bounds__(kSelectWarps * 32) select_kernel(CallView c, c
     }
 }
 
-// One block.  Counting sort of the (row, slot) pairs by group: group_count,
-// group_offset (exclusive scan), bucket_row / bucket_slot with the rows of each
-// group in ascending order, and the union size.
-constexpr int kBucketThreads = 1024;
-__global__ void __launch_bounds__(kBucketThreads) bucket_kernel(CallView c) {
-    __shared__ int s_count[kMaxGroups];
-    __shared__ int s_offset[kMaxGroups + 1];
-    __shared__ int s_rank[kMaxGroups];
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    constexpr int kWarps = kBucketThreads / 32;
-    for (int n = warp; n < c.N; n += kWarps) {
-        int cnt = 0;
-        for (int m0 = 0; m0 < c.M; m0 += 32) {
-            const int m = m0 + lane;
-            const bool in = m < c.M && c.slot_of[(size_t)m * c.N + n] >= 0;
-            cnt += __popc(__ballot_sync(0xffffffffu, in));
-        }
-        if (lane == 0) s_count[n] = cnt;
-    }
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        int run = 0, uni = 0, virt = 0;
-        for (int n = 0; n < c.N; ++n) {
-            s_offset[n] = run;
-            run += s_count[n];
-            s_rank[n] = virt;
-            if (c.union_rank) c.union_rank[n] = s_count[n] > 0 ? virt : -1;
-            if (s_count[n] > 0) {
-                const int passes = c.pass_rows > 0 ? (s_count[n] + c.pass_rows - 1) / c.pass_rows : 1;
-                for (int p = 0; p < passes; ++p)
-                    if (c.union_list && virt + p < c.union_cap) c.union_list[virt + p] = n | (p << 16);
-                virt += passes;
-                ++uni;
-            }
-        }
-        s_offset[c.N] = run;
-        c.state->n_union = uni;
-        c.state->n_virtual = min(virt, c.union_cap);
-    }
-    __syncthreads();
-    for (int n = threadIdx.x; n <= c.N; n += kBucketThreads) {
-        c.group_offset[n] = s_offset[n];
-        if (n < c.N) c.group_count[n] = s_count[n];
-    }
-    for (int n = warp; n < c.N; n += kWarps) {
-        int pos = s_offset[n];
-        for (int m0 = 0; m0 < c.M; m0 += 32) {
-            const int m = m0 + lane;
-            const int sl = (m < c.M) ? (int)c.slot_of[(size_t)m * c.N + n] : -1;
-            const unsigned bal = __ballot_sync(0xffffffffu, sl >= 0);
-            if (sl >= 0) {
-                const int p = pos + __popc(bal & ((1u << lane) - 1u));
-                c.bucket_row[p] = m;
-                c.bucket_slot[p] = sl;
-                if (c.slot_desc) {
-                    const int pos_in_group = p - s_offset[n];
-                    const int pass = c.pass_rows > 0 ? pos_in_group / c.pass_rows : 0;
-                    c.slot_desc[(size_t)m * c.k_groups + sl] =
-                        ((s_rank[n] + pass) << 8) | ((pos_in_group - pass * max(c.pass_rows, 1)) & 255);
-                }
-            }
-            pos += __popc(bal);
-        }
-    }
-}
-
-
 // Groups of row m by one warp (NPER = groups per lane).  Rank selection: slot of a group = number of groups
 // that beat it (higher score, or equal score and lower index).  Forced groups take their listed order.
 template <int NPER>

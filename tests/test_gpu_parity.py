@@ -244,3 +244,27 @@ def test_large_m_routed_grouped_gemm():
                      {"ids": ids.cpu().numpy()[rows], "logprobs": lps.cpu().numpy()[rows]})
     assert rep.ok, rep.errors
     head.close()
+
+
+def test_draft_is_capturable_in_a_cuda_graph():
+    """The draft call enqueues kernels only (no allocation, no host synchronisation): it can be captured once
+    and replayed, and the replay gives the same bits as the direct call."""
+    cfg, W, gm, Wg, head = _weights("tiny")
+    head.set_path(lmhead.CORAL_PATH_AUTO)
+    h = ph.to_dev_bf16(synth.make_hidden(cfg, 6))
+    ids = torch.empty((6, 10), dtype=torch.int32, device="cuda")
+    lps = torch.empty((6, 10), dtype=torch.float32, device="cuda")
+    lmhead.coral_lmhead_draft(head.handle, h, 4, 10, ids, lps)
+    torch.cuda.synchronize()
+    want_ids, want_lps = ids.clone(), lps.clone()
+    ids.zero_()
+    lps.zero_()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        lmhead.coral_lmhead_draft(head.handle, h, 4, 10, ids, lps)
+    for _ in range(2):
+        ids.zero_()
+        g.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(ids, want_ids) and torch.equal(lps, want_lps)
+    assert head.status() == 0
