@@ -50,6 +50,10 @@ extern "C" {
 #define CORAL_PATH_TCGEN05 2       /* routed grouped GEMM on tcgen05 / TMEM tiles */
 #define CORAL_PATH_SIMT_PLAIN 3    /* gathered GEMV with plain 128-bit loads, any M */
 
+/* Output modes (coral_lmhead_set_output_mode). */
+#define CORAL_OUTPUT_JOINT 0       /* log-softmax over all active logits of the row (default) */
+#define CORAL_OUTPUT_FACTORISED 1  /* Eq. 8: log p_router(n) + log p_group(x), p_router = Softmax over all N groups */
+
 typedef struct coral_lmhead_s *coral_lmhead_handle;
 
 typedef struct coral_lmhead_config {
@@ -147,6 +151,24 @@ int coral_lmhead_draft_ex(coral_lmhead_handle h, const void *hidden_dev, int M, 
  */
 int coral_lmhead_draft_host(coral_lmhead_handle h, const void *hidden_host, int M, int k_groups, int k_tokens,
                             int32_t *out_ids_host, float *out_logprobs_host, void *stream);
+
+/*
+ * Output mode of later draft calls.  CORAL_OUTPUT_FACTORISED emits the paper's final distribution (Section
+ * 3.3, Eq. 8): p(x) = p_router(n) * p_group(x^n), where p_router is the softmax of the row's N router scores
+ * (Eq. 7) and p_group the softmax inside group n, independent of the other groups; candidates are ranked by
+ * that log-probability (equal -> lower token id).  The emitted log-probabilities of a row sum, over its active
+ * vocabulary, to the router mass of its selected groups.  out_lse_dev keeps reporting the joint log-sum-exp.
+ * Not available on CORAL_PATH_SIMT_PLAIN (the draft call then returns CORAL_ERR_INVALID).
+ */
+int coral_lmhead_set_output_mode(coral_lmhead_handle h, int mode);
+
+/*
+ * Two-layer router of the paper's Eq. 7: scores = W2 (act(W1 h) + h), with W2 the W_gate given at create, W1
+ * [H x H] bf16 (device, 16-byte aligned; copied into library-owned memory, the call synchronises `stream`) and
+ * act = SiLU (the paper does not name the activation).  act(W1 h) + h is kept in fp32.  W1_dev = NULL returns
+ * to the single-matrix gate.  Allocates (cudaMalloc) H*H*2 + max_M*H*4 bytes on first use.
+ */
+int coral_lmhead_set_router_mlp(coral_lmhead_handle h, const void *W1_dev, void *stream);
 
 /*
  * Force an execution path (CORAL_PATH_*) for later draft calls; AUTO restores the default choice.

@@ -30,6 +30,7 @@ struct CallView {
     const uint16_t* w_gate;        // [N][H] bf16
     const int32_t* group_tokens;   // [N][v] global token id of packed row
     const uint16_t* hidden;        // [M][H] bf16
+    const float* router_in;        // [M][H] fp32 router input act(W1 h) + h (Eq. 7), or null: the gate reads `hidden`
     float* gate;                   // [M][N]
     int32_t* sel;                  // [M][k_groups]
     int16_t* slot_of;              // [M][N] slot of group n in row m, -1 if not selected

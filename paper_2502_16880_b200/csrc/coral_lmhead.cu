@@ -156,6 +156,9 @@ struct coral_lmhead_s {
     StreamGeom sg;
     int stream_smem;     // 0 if the streaming path is not available for this shape/device
     bool tc_ok;          // tensor-core path available (maps encoded)
+    int out_mode;        // CORAL_OUTPUT_*
+    uint16_t* w1;        // [H][H] bf16 first router layer (Eq. 7), library-owned, or null
+    float* router_u;     // [max_M][H] fp32 act(W1 h) + h, library-owned
     CUtensorMap map_w, map_h;
     int sms;
     cudaEvent_t ev_head0, ev_head1;   // around the weight-streaming kernel when kernel timing is on
@@ -178,6 +181,7 @@ CallView make_view(const coral_lmhead_s* h, const void* hidden, int M, int kg, i
     c.w_gate = reinterpret_cast<const uint16_t*>(ws + L.w_gate);
     c.group_tokens = reinterpret_cast<const int32_t*>(ws + L.group_tokens);
     c.hidden = reinterpret_cast<const uint16_t*>(hidden);
+    c.router_in = h->w1 ? h->router_u : nullptr;
     c.gate = reinterpret_cast<float*>(ws + L.gate);
     c.sel = reinterpret_cast<int32_t*>(ws + L.sel);
     c.slot_of = reinterpret_cast<int16_t*>(ws + L.slot_of);
@@ -402,6 +406,8 @@ int coral_lmhead_destroy(coral_lmhead_handle h) {
     if (!h) return CORAL_OK;
     if (h->own_packed && h->packed) cudaFree(h->packed);
     if (h->own_ws && h->ws) cudaFree(h->ws);
+    if (h->w1) cudaFree(h->w1);
+    if (h->router_u) cudaFree(h->router_u);
     if (h->ev_head0) cudaEventDestroy(h->ev_head0);
     if (h->ev_head1) cudaEventDestroy(h->ev_head1);
     if (h->ev_begin) cudaEventDestroy(h->ev_begin);
@@ -431,12 +437,26 @@ int coral_lmhead_draft_ex(coral_lmhead_handle h, const void* hidden_dev, int M, 
     CallView c = make_view(h, hidden_dev, M, k_groups, k_tokens);
     const int path = choose_path(h, M, k_groups);
     if (path == 0) return CORAL_ERR_INVALID;   // the forced path does not support this call
+    if (h->out_mode == CORAL_OUTPUT_FACTORISED && path == CORAL_PATH_SIMT_PLAIN) return CORAL_ERR_INVALID;
     c.pass_rows = path == CORAL_PATH_STREAM ? kStreamPassRows : path == CORAL_PATH_TCGEN05 ? kTcPassRows : 0;
     if (path == CORAL_PATH_TCGEN05) c.union_cap = h->L.tc_vcap;
     int launches = 0;
 
     if (h->timing) cudaEventRecord(h->ev_begin, st);
-    if (M <= kRouteFusedMaxM) {
+    if (h->w1) {
+        router_hidden_kernel<<<dim3((cfg.H + kGateTile - 1) / kGateTile, (M + kGateTile - 1) / kGateTile), 256, 0, st>>>(
+            c, h->w1, h->router_u);
+        ++launches;
+        gate_f32_kernel<<<dim3(c.N, (M + kGateRows - 1) / kGateRows), kGateThreads, 0, st>>>(c, out_gate_dev);
+        ++launches;
+        select_kernel<<<(M + kSelectWarps - 1) / kSelectWarps, kSelectWarps * 32, 0, st>>>(c, forced_groups_dev,
+                                                                                          out_groups_dev);
+        ++launches;
+        count_groups_kernel<<<(M * k_groups + kSelectWarps * 32 - 1) / (kSelectWarps * 32), kSelectWarps * 32, 0, st>>>(c);
+        ++launches;
+        bucket_group_kernel<<<c.N, 256, 0, st>>>(c);
+        ++launches;
+    } else if (M <= kRouteFusedMaxM) {
         route_fused_kernel<<<c.N, kRouteThreads, 0, st>>>(c, forced_groups_dev, out_groups_dev, out_gate_dev);
         ++launches;
     } else {
@@ -462,7 +482,8 @@ int coral_lmhead_draft_ex(coral_lmhead_handle h, const void* hidden_dev, int M, 
         if (h->timing) cudaEventRecord(h->ev_head1, st);
         launch_pdl(merge_stream_kernel, dim3(M), dim3(kMergeStreamThreads), (size_t)kMergeSmemCands * 8, st, c, h->sg, pp,
                    reinterpret_cast<float*>(h->ws + L.cand_val), reinterpret_cast<int32_t*>(h->ws + L.cand_id),
-                   (int)L.cand_cap, (int)kMergeSmemCands, out_ids_dev, out_logprobs_dev, out_lse_dev);
+                   (int)L.cand_cap, (int)kMergeSmemCands, (int)(h->out_mode == CORAL_OUTPUT_FACTORISED), out_ids_dev,
+                   out_logprobs_dev, out_lse_dev);
         ++launches;
     } else if (path == CORAL_PATH_TCGEN05) {
         const Layout& L = h->L;
@@ -481,7 +502,8 @@ int coral_lmhead_draft_ex(coral_lmhead_handle h, const void* hidden_dev, int M, 
         StreamPartials pp{tp.pmax, tp.psum, tp.pval, tp.pid};
         launch_pdl(merge_stream_kernel, dim3(M), dim3(kMergeStreamThreads), (size_t)kMergeSmemCands * 8, st, c, mg, pp,
                    reinterpret_cast<float*>(h->ws + L.cand_val), reinterpret_cast<int32_t*>(h->ws + L.cand_id),
-                   (int)L.cand_cap, (int)kMergeSmemCands, out_ids_dev, out_logprobs_dev, out_lse_dev);
+                   (int)L.cand_cap, (int)kMergeSmemCands, (int)(h->out_mode == CORAL_OUTPUT_FACTORISED), out_ids_dev,
+                   out_logprobs_dev, out_lse_dev);
         ++launches;
     } else {
         head_simt_kernel<<<dim3(c.T, c.N), kSimtThreads, h->simt_smem, st>>>(c, out_logits_dev);
@@ -520,6 +542,35 @@ int coral_lmhead_draft_host(coral_lmhead_handle h, const void* hidden_host, int 
         return CORAL_ERR_CUDA;
     if (cudaMemcpyAsync(out_logprobs_host, d_lp, (size_t)M * k_tokens * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess)
         return CORAL_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return CORAL_ERR_CUDA;
+    return CORAL_OK;
+}
+
+int coral_lmhead_set_output_mode(coral_lmhead_handle h, int mode) {
+    if (!h || (mode != CORAL_OUTPUT_JOINT && mode != CORAL_OUTPUT_FACTORISED)) return CORAL_ERR_INVALID;
+    h->out_mode = mode;
+    return CORAL_OK;
+}
+
+int coral_lmhead_set_router_mlp(coral_lmhead_handle h, const void* W1_dev, void* stream) {
+    if (!h) return CORAL_ERR_INVALID;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (!W1_dev) {                       // back to the single-matrix gate
+        if (cudaStreamSynchronize(st) != cudaSuccess) return CORAL_ERR_CUDA;
+        if (h->w1) cudaFree(h->w1);
+        if (h->router_u) cudaFree(h->router_u);
+        h->w1 = nullptr;
+        h->router_u = nullptr;
+        return CORAL_OK;
+    }
+    if (reinterpret_cast<uintptr_t>(W1_dev) & 15) return CORAL_ERR_INVALID;
+    const size_t H = h->cfg.H;
+    if (!h->w1 && cudaMalloc(&h->w1, H * H * 2) != cudaSuccess) { h->w1 = nullptr; return CORAL_ERR_NOMEM; }
+    if (!h->router_u && cudaMalloc(&h->router_u, (size_t)h->cfg.max_M * H * 4) != cudaSuccess) {
+        h->router_u = nullptr;
+        return CORAL_ERR_NOMEM;
+    }
+    if (cudaMemcpyAsync(h->w1, W1_dev, H * H * 2, cudaMemcpyDeviceToDevice, st) != cudaSuccess) return CORAL_ERR_CUDA;
     if (cudaStreamSynchronize(st) != cudaSuccess) return CORAL_ERR_CUDA;
     return CORAL_OK;
 }

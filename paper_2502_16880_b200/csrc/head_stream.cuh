@@ -391,18 +391,22 @@ __global__ void __launch_bounds__(kStreamThreads, 1) head_stream_kernel(CallView
     }
 }
 
-// Merge for the streaming path: block per row.  The pieces of row m, slot s are the partials that the CTAs
-// overlapping that slot's (group, pass) wrote for the row's position in the pass.  Every piece holds a
-// sorted top-k list, so two lower bounds of the row's k-th value are at hand: the largest of the pieces'
-// k-th entries, and the k-th largest of the pieces' first entries.  Only candidates at or above the better
-// bound are kept, and those few are ranked by counting.
+// Merge for the streaming and tensor-core paths: block per row.  The pieces of row m, slot s are the partials
+// that the CTAs overlapping that slot's (group, pass) wrote for the row's position in the pass.  Every piece
+// holds a sorted top-k list, so two lower bounds of the row's k-th value are at hand: the largest of the
+// pieces' k-th entries, and the k-th largest of the pieces' first entries.  Only candidates at or above the
+// better bound are kept, and those few are ranked by counting.
+// Output modes: joint (log-softmax over all active logits of the row) adds -LSE_row to every logit;
+// factorised (CORAL Eq. 8, p(x) = p_router(n) p_group(x)) adds log p_router(n) - LSE_group(n), a per-slot
+// offset, where p_router is the softmax of the row's N gate scores (Eq. 7).  Adding a per-slot constant
+// keeps every piece's list sorted, so both modes share the selection code.
 constexpr int kMergeStreamThreads = 256;
 constexpr int kMergeMaxPieces = 1024;         // >= grid + 2 * k_groups for every supported shape
 constexpr int kMergeRankMax = 256;            // survivors ranked by counting; more fall back to k rounds
 __global__ void __launch_bounds__(kMergeStreamThreads) merge_stream_kernel(CallView c, StreamGeom g, StreamPartials pp,
                                                                            float* __restrict__ cand_val_scratch,
                                                                            int32_t* __restrict__ cand_id_scratch,
-                                                                           int cand_cap, int smem_cands,
+                                                                           int cand_cap, int smem_cands, int factorised,
                                                                            int32_t* __restrict__ out_ids,
                                                                            float* __restrict__ out_logprobs,
                                                                            float* __restrict__ lse_tap) {
@@ -411,12 +415,13 @@ __global__ void __launch_bounds__(kMergeStreamThreads) merge_stream_kernel(CallV
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     constexpr int kWarps = kMergeStreamThreads / 32;
     __shared__ float s_f[kWarps], s_t[kWarps];
-    __shared__ float s_lse;
+    __shared__ float s_lse, s_glse, s_thr2;
     __shared__ int s_n;
     __shared__ int s_first[kMaxGroups], s_base[kMaxGroups + 1], s_rpos[kMaxGroups], s_j[kMaxGroups];
+    __shared__ float s_off[kMaxGroups];           // per slot: what is added to a logit to give the emitted log-prob
     __shared__ int s_piece[kMergeMaxPieces];
-    __shared__ float s_head[kMergeMaxPieces];
-    __shared__ float s_thr2;
+    __shared__ unsigned char s_pslot[kMergeMaxPieces];
+    __shared__ float s_pm[kMergeMaxPieces], s_ps[kMergeMaxPieces], s_last[kMergeMaxPieces], s_head[kMergeMaxPieces];
 
     // The router's outputs were complete before the streaming kernel let this grid start.
     const int n_items = c.state->n_virtual * g.T;
@@ -430,8 +435,27 @@ __global__ void __launch_bounds__(kMergeStreamThreads) merge_stream_kernel(CallV
         s_base[s] = lb - fb + 1;       // piece count, turned into an exclusive prefix below
         s_j[s] = j;
         s_rpos[s] = desc & 255;
+        s_off[s] = factorised ? c.gate[(size_t)m * c.N + c.sel[(size_t)m * c.k_groups + s]] : 0.f;
     }
     if (threadIdx.x == 0) { s_n = 0; s_thr2 = kNegInf; }
+    if (factorised) {                 // log-sum-exp of the row's N gate scores (kMergeStreamThreads >= N)
+        const float gv = threadIdx.x < c.N ? c.gate[(size_t)m * c.N + threadIdx.x] : kNegInf;
+        const float wm = warp_max(gv);
+        if (lane == 0) s_f[warp] = wm;
+        __syncthreads();
+        float gm = s_f[0];
+#pragma unroll
+        for (int w = 1; w < kWarps; ++w) gm = fmaxf(gm, s_f[w]);
+        const float ws = warp_sum(threadIdx.x < c.N ? expf(gv - gm) : 0.f);
+        if (lane == 0) s_t[warp] = ws;
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            float tot = 0.f;
+#pragma unroll
+            for (int w = 0; w < kWarps; ++w) tot += s_t[w];
+            s_glse = gm + logf(tot);
+        }
+    }
     __syncthreads();
     if (threadIdx.x == 0) {
         int run = 0;
@@ -444,6 +468,7 @@ __global__ void __launch_bounds__(kMergeStreamThreads) merge_stream_kernel(CallV
         int s = 0;
         while (s + 1 < c.k_groups && s_base[s + 1] <= q) ++s;
         const int b = s_first[s] + (q - s_base[s]);
+        s_pslot[q] = (unsigned char)s;
         if (g.tc_tiles > 0) {
             s_piece[q] = b * g.tc_rows + s_rpos[s];       // (pass * tiles + sub-tile) * rows per pass + row
         } else {
@@ -455,33 +480,60 @@ __global__ void __launch_bounds__(kMergeStreamThreads) merge_stream_kernel(CallV
 
     pdl_wait();                   // partials of the streaming kernel are complete from here on
 
-    // pass 1 over the pieces (each thread owns up to kOwnPieces of them; all loads issued together):
-    // joint log-sum-exp and the candidate threshold
-    constexpr int kOwnPieces = kMergeMaxPieces / kMergeStreamThreads;
-    float pm[kOwnPieces], ps[kOwnPieces];
-    float mx = kNegInf, thr = kNegInf;
-#pragma unroll
-    for (int u = 0; u < kOwnPieces; ++u) {
-        const int q = threadIdx.x + u * kMergeStreamThreads;
-        pm[u] = kNegInf;
-        ps[u] = 0.f;
-        if (q < P) {
-            const size_t p = (size_t)s_piece[q];
-            pm[u] = pp.pmax[p];
-            ps[u] = pp.psum[p];
-            thr = fmaxf(thr, pp.pval[p * c.k_tokens + c.k_tokens - 1]);
-            s_head[q] = pp.pval[p * c.k_tokens];
-            mx = fmaxf(mx, pm[u]);
-        }
+    // pass 1 over the pieces (all loads of a thread's pieces issued together)
+    float mx = kNegInf;
+    for (int q = threadIdx.x; q < P; q += kMergeStreamThreads) {
+        const size_t p = (size_t)s_piece[q];
+        const float a = pp.pmax[p], b = pp.psum[p];
+        const float l = pp.pval[p * c.k_tokens + c.k_tokens - 1], h = pp.pval[p * c.k_tokens];
+        s_pm[q] = a; s_ps[q] = b; s_last[q] = l; s_head[q] = h;
+        mx = fmaxf(mx, a);
     }
     mx = warp_max(mx);
-    thr = warp_max(thr);
-    if (lane == 0) { s_f[warp] = mx; s_t[warp] = thr; }
+    if (lane == 0) s_f[warp] = mx;
     __syncthreads();
     mx = s_f[0];
-    thr = s_t[0];
 #pragma unroll
-    for (int w = 1; w < kWarps; ++w) { mx = fmaxf(mx, s_f[w]); thr = fmaxf(thr, s_t[w]); }
+    for (int w = 1; w < kWarps; ++w) mx = fmaxf(mx, s_f[w]);
+    float sum = 0.f;
+    for (int q = threadIdx.x; q < P; q += kMergeStreamThreads) sum += s_ps[q] * expf(s_pm[q] - mx);
+    sum = warp_sum(sum);
+    if (lane == 0) s_t[warp] = sum;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        float tot = 0.f;
+#pragma unroll
+        for (int w = 0; w < kWarps; ++w) tot += s_t[w];
+        s_lse = mx + logf(tot);
+        if (lse_tap) lse_tap[m] = s_lse;
+    }
+    __syncthreads();
+    // per-slot offsets
+    for (int s = threadIdx.x; s < c.k_groups; s += kMergeStreamThreads) {
+        if (factorised) {
+            float sm = kNegInf;
+            for (int q = s_base[s]; q < min(s_base[s + 1], P); ++q) sm = fmaxf(sm, s_pm[q]);
+            float ss = 0.f;
+            for (int q = s_base[s]; q < min(s_base[s + 1], P); ++q) ss += s_ps[q] * expf(s_pm[q] - sm);
+            s_off[s] = (s_off[s] - s_glse) - (sm + logf(ss));
+        } else {
+            s_off[s] = -s_lse;
+        }
+    }
+    __syncthreads();
+    // thresholds on the emitted values
+    float thr = kNegInf;
+    for (int q = threadIdx.x; q < P; q += kMergeStreamThreads) {
+        const float off = s_off[s_pslot[q]];
+        thr = fmaxf(thr, s_last[q] + off);
+        s_head[q] += off;
+    }
+    thr = warp_max(thr);
+    if (lane == 0) s_f[warp] = thr;
+    __syncthreads();
+    thr = s_f[0];
+#pragma unroll
+    for (int w = 1; w < kWarps; ++w) thr = fmaxf(thr, s_f[w]);
     // k-th largest first entry: the piece whose head is beaten by exactly k_tokens - 1 others (index breaks ties)
     for (int q = threadIdx.x; q < P; q += kMergeStreamThreads) {
         const float hq = s_head[q];
@@ -491,11 +543,6 @@ __global__ void __launch_bounds__(kMergeStreamThreads) merge_stream_kernel(CallV
     }
     __syncthreads();
     thr = fmaxf(thr, s_thr2);
-    float sum = 0.f;
-#pragma unroll
-    for (int u = 0; u < kOwnPieces; ++u) sum += ps[u] * expf(pm[u] - mx);     // exp(-inf) = 0 for unowned slots
-    sum = warp_sum(sum);
-    if (lane == 0) s_f[warp] = sum;
 
     // pass 2: keep the candidates at or above the threshold (order of arrival does not matter: the
     // ranking below is by the total order (value desc, token id asc)).  A warp reads four lists at a time.
@@ -513,7 +560,7 @@ __global__ void __launch_bounds__(kMergeStreamThreads) merge_stream_kernel(CallV
             id[u] = kNoToken;
             if (q0 + u < P && lane < c.k_tokens) {
                 const size_t p = (size_t)s_piece[q0 + u];
-                v[u] = pp.pval[p * c.k_tokens + lane];
+                v[u] = pp.pval[p * c.k_tokens + lane] + s_off[s_pslot[q0 + u]];
                 id[u] = pp.pid[p * c.k_tokens + lane];
             }
         }
@@ -526,15 +573,6 @@ __global__ void __launch_bounds__(kMergeStreamThreads) merge_stream_kernel(CallV
         }
     }
     __syncthreads();
-    if (threadIdx.x == 0) {
-        float tot = 0.f;
-#pragma unroll
-        for (int w = 0; w < kWarps; ++w) tot += s_f[w];
-        s_lse = mx + logf(tot);
-        if (lse_tap) lse_tap[m] = s_lse;
-    }
-    __syncthreads();
-    const float lse = s_lse;
     const int S = min(s_n, cap);
 
     if (S <= kMergeRankMax) {
@@ -546,7 +584,7 @@ __global__ void __launch_bounds__(kMergeStreamThreads) merge_stream_kernel(CallV
             for (int i = 0; i < S; ++i) rank += better(cv[i], ci[i], v, id) ? 1 : 0;
             if (rank < c.k_tokens) {
                 out_ids[(size_t)m * c.k_tokens + rank] = id;
-                out_logprobs[(size_t)m * c.k_tokens + rank] = v - lse;
+                out_logprobs[(size_t)m * c.k_tokens + rank] = v;
             }
         }
         return;
@@ -574,7 +612,7 @@ __global__ void __launch_bounds__(kMergeStreamThreads) merge_stream_kernel(CallV
             if (better(s_f[w], s_i[w], bv, bk)) { bv = s_f[w]; bk = s_i[w]; }
         if (threadIdx.x == 0) {
             out_ids[(size_t)m * c.k_tokens + k] = bk;
-            out_logprobs[(size_t)m * c.k_tokens + k] = bv - lse;
+            out_logprobs[(size_t)m * c.k_tokens + k] = bv;
         }
         last_v = bv;
         last_id = bk;

@@ -413,4 +413,106 @@ __global__ void __launch_bounds__(256) bucket_group_kernel(CallView c) {
     }
 }
 
+
+// ---- two-layer router of the paper's Eq. 7: scores = W2 (act(W1 h) + h), act = SiLU ---------------------------
+
+// u[m][i] = SiLU(W1[i] . h[m]) + h[m][i] in fp32, for a tile of 8 output columns x 8 rows per block.
+// grid (ceil(H/8), ceil(M/8)).
+__global__ void __launch_bounds__(256) router_hidden_kernel(CallView c, const uint16_t* __restrict__ W1,
+                                                            float* __restrict__ u) {
+    __shared__ float s_red[8][kGateTile * kGateTile];
+    const int i0 = blockIdx.x * kGateTile, m0 = blockIdx.y * kGateTile;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int chunks = c.H >> 3;
+    float acc[kGateTile][kGateTile];
+#pragma unroll
+    for (int g = 0; g < kGateTile; ++g)
+#pragma unroll
+        for (int r = 0; r < kGateTile; ++r) acc[g][r] = 0.f;
+    for (int ch = threadIdx.x; ch < chunks; ch += 256) {
+        float hf[kGateTile][8];
+#pragma unroll
+        for (int r = 0; r < kGateTile; ++r) {
+            const uint4 q = (m0 + r < c.M) ? __ldg(reinterpret_cast<const uint4*>(c.hidden + (size_t)(m0 + r) * c.H) + ch)
+                                           : make_uint4(0, 0, 0, 0);
+            hf[r][0] = bf16_lo(q.x); hf[r][1] = bf16_hi(q.x); hf[r][2] = bf16_lo(q.y); hf[r][3] = bf16_hi(q.y);
+            hf[r][4] = bf16_lo(q.z); hf[r][5] = bf16_hi(q.z); hf[r][6] = bf16_lo(q.w); hf[r][7] = bf16_hi(q.w);
+        }
+#pragma unroll
+        for (int g = 0; g < kGateTile; ++g) {
+            const uint4 q = (i0 + g < c.H) ? __ldg(reinterpret_cast<const uint4*>(W1 + (size_t)(i0 + g) * c.H) + ch)
+                                           : make_uint4(0, 0, 0, 0);
+            const float w[8] = {bf16_lo(q.x), bf16_hi(q.x), bf16_lo(q.y), bf16_hi(q.y),
+                                bf16_lo(q.z), bf16_hi(q.z), bf16_lo(q.w), bf16_hi(q.w)};
+#pragma unroll
+            for (int r = 0; r < kGateTile; ++r)
+#pragma unroll
+                for (int e = 0; e < 8; ++e) acc[g][r] = fmaf(w[e], hf[r][e], acc[g][r]);
+        }
+    }
+#pragma unroll
+    for (int g = 0; g < kGateTile; ++g)
+#pragma unroll
+        for (int r = 0; r < kGateTile; ++r) {
+            const float sum = warp_sum(acc[g][r]);
+            if (lane == 0) s_red[warp][g * kGateTile + r] = sum;
+        }
+    __syncthreads();
+    if (threadIdx.x < kGateTile * kGateTile) {
+        const int g = threadIdx.x / kGateTile, r = threadIdx.x % kGateTile;
+        if (i0 + g < c.H && m0 + r < c.M) {
+            float a = 0.f;
+#pragma unroll
+            for (int w = 0; w < 8; ++w) a += s_red[w][threadIdx.x];
+            const float hv = __uint_as_float((uint32_t)c.hidden[(size_t)(m0 + r) * c.H + i0 + g] << 16);
+            u[(size_t)(m0 + r) * c.H + i0 + g] = a / (1.f + expf(-a)) + hv;
+        }
+    }
+}
+
+// g[m][n] = W_gate[n] . u[m] with u in fp32.  grid (N, ceil(M/8)); block (0,0) clears the per-group counters.
+__global__ void __launch_bounds__(kGateThreads) gate_f32_kernel(CallView c, float* __restrict__ gate_tap) {
+    const int n = blockIdx.x;
+    const int m0 = blockIdx.y * kGateRows;
+    const int rows = min(kGateRows, c.M - m0);
+    const int chunks = c.H >> 3;
+    if (blockIdx.x == 0 && blockIdx.y == 0)
+        for (int t = threadIdx.x; t < c.N; t += kGateThreads) c.group_count[t] = 0;
+    const uint4* __restrict__ wg = reinterpret_cast<const uint4*>(c.w_gate + (size_t)n * c.H);
+    float acc[kGateRows];
+#pragma unroll
+    for (int r = 0; r < kGateRows; ++r) acc[r] = 0.f;
+    for (int ch = threadIdx.x; ch < chunks; ch += kGateThreads) {
+        const uint4 q = __ldg(wg + ch);
+        const float w[8] = {bf16_lo(q.x), bf16_hi(q.x), bf16_lo(q.y), bf16_hi(q.y),
+                            bf16_lo(q.z), bf16_hi(q.z), bf16_lo(q.w), bf16_hi(q.w)};
+#pragma unroll
+        for (int r = 0; r < kGateRows; ++r) {
+            if (r < rows) {
+                const float4* up = reinterpret_cast<const float4*>(c.router_in + (size_t)(m0 + r) * c.H) + 2 * ch;
+                const float4 a = __ldg(up), b = __ldg(up + 1);
+                acc[r] = fmaf(w[0], a.x, acc[r]); acc[r] = fmaf(w[1], a.y, acc[r]);
+                acc[r] = fmaf(w[2], a.z, acc[r]); acc[r] = fmaf(w[3], a.w, acc[r]);
+                acc[r] = fmaf(w[4], b.x, acc[r]); acc[r] = fmaf(w[5], b.y, acc[r]);
+                acc[r] = fmaf(w[6], b.z, acc[r]); acc[r] = fmaf(w[7], b.w, acc[r]);
+            }
+        }
+    }
+    __shared__ float red[kGateThreads / 32][kGateRows];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+    for (int r = 0; r < kGateRows; ++r) {
+        const float sum = warp_sum(acc[r]);
+        if (lane == 0) red[warp][r] = sum;
+    }
+    __syncthreads();
+    if (threadIdx.x < rows) {
+        float sum = 0.f;
+#pragma unroll
+        for (int w = 0; w < kGateThreads / 32; ++w) sum += red[w][threadIdx.x];
+        c.gate[(size_t)(m0 + threadIdx.x) * c.N + n] = sum;
+        if (gate_tap) gate_tap[(size_t)(m0 + threadIdx.x) * c.N + n] = sum;
+    }
+}
+
 }  // namespace coral

@@ -25,6 +25,7 @@ CORAL_ERR_TIMEOUT = -5
 CORAL_ERR_BOUNDS = -6
 CORAL_ERR_TOO_LARGE = -7
 CORAL_ROUTE_STATIC_MAX_ROWS = 64
+CORAL_OUTPUT_JOINT, CORAL_OUTPUT_FACTORISED = 0, 1
 CORAL_PATH_AUTO, CORAL_PATH_STREAM, CORAL_PATH_TCGEN05, CORAL_PATH_SIMT_PLAIN = 0, 1, 2, 3
 
 
@@ -53,6 +54,8 @@ _SIGNATURES = {
     "coral_lmhead_draft_ex": (_i, [_vp, _vp, _i, _i, _i, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "coral_lmhead_draft_host": (_i, [_vp, _vp, _i, _i, _i, _vp, _vp, _vp]),
     "coral_lmhead_set_path": (_i, [_vp, _i]),
+    "coral_lmhead_set_output_mode": (_i, [_vp, _i]),
+    "coral_lmhead_set_router_mlp": (_i, [_vp, _vp, _vp]),
     "coral_lmhead_set_kernel_timing": (_i, [_vp, _i]),
     "coral_lmhead_head_kernel_ms": (_i, [_vp, ctypes.POINTER(ctypes.c_float)]),
     "coral_lmhead_stage_ms": (_i, [_vp] + [ctypes.POINTER(ctypes.c_float)] * 3),
@@ -173,6 +176,16 @@ def coral_lmhead_draft_host(handle, hidden_host, k_groups, k_tokens, out_ids_hos
         handle, ctypes.c_void_p(hidden_host.data_ptr()), M, int(k_groups), int(k_tokens),
         ctypes.c_void_p(out_ids_host.data_ptr()), ctypes.c_void_p(out_logprobs_host.data_ptr()),
         _stream_ptr(stream)), "coral_lmhead_draft_host")
+
+
+def coral_lmhead_set_output_mode(handle, mode: int) -> None:
+    _check(load_library().coral_lmhead_set_output_mode(handle, int(mode)), "coral_lmhead_set_output_mode")
+
+
+def coral_lmhead_set_router_mlp(handle, W1=None, stream=None) -> None:
+    """W1: CUDA bf16 [H, H] tensor of Eq. 7's first router layer, or None for the single-matrix gate."""
+    _check(load_library().coral_lmhead_set_router_mlp(handle, _dev_ptr(W1, torch.bfloat16), _stream_ptr(stream)),
+           "coral_lmhead_set_router_mlp")
 
 
 def coral_lmhead_set_path(handle, path: int) -> None:

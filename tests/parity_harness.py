@@ -49,14 +49,16 @@ class ParityReport:
         return not self.errors
 
 
-def compare(W, gm, Wg, hidden_bits, k_groups, k_tokens, gpu, forced_groups=None, max_errors=10) -> ParityReport:
+def compare(W, gm, Wg, hidden_bits, k_groups, k_tokens, gpu, forced_groups=None, max_errors=10, W1=None,
+            factorised=False) -> ParityReport:
     """gpu: dict of numpy arrays from LMHead.draft(taps=True) ('groups','gate','logits','lse','ids','logprobs'),
     or just 'ids'/'logprobs' (taps missing are skipped).  forced_groups: the groups the caller forced, if any."""
     rep = ParityReport()
     M = hidden_bits.shape[0]
     rep.rows = M
     g_groups = gpu.get("groups")
-    ref = orc.draft(W, gm, Wg, hidden_bits, k_groups, k_tokens, forced_groups=forced_groups)
+    ref = orc.draft(W, gm, Wg, hidden_bits, k_groups, k_tokens, forced_groups=forced_groups, W1=W1,
+                    factorised=factorised)
     forced = None
     if g_groups is not None:
         for m in range(M):
@@ -74,7 +76,8 @@ def compare(W, gm, Wg, hidden_bits, k_groups, k_tokens, gpu, forced_groups=None,
                 rep.tie_resolved_rows += 1
                 forced = g_groups
         if forced is not None and not rep.errors:
-            ref = orc.draft(W, gm, Wg, hidden_bits, k_groups, k_tokens, forced_groups=np.ascontiguousarray(forced))
+            ref = orc.draft(W, gm, Wg, hidden_bits, k_groups, k_tokens, forced_groups=np.ascontiguousarray(forced),
+                            W1=W1, factorised=factorised)
     if rep.errors:
         return rep
 
@@ -97,7 +100,13 @@ def compare(W, gm, Wg, hidden_bits, k_groups, k_tokens, gpu, forced_groups=None,
 
     ids, lps = gpu["ids"], gpu["logprobs"]
     for m in range(M):
-        zmap = dict(zip(ref.logit_tokens[m].ravel().tolist(), ref.logits[m].ravel().tolist()))
+        # the emitted log-probability of every active token: joint = z - LSE(row); factorised (Eq. 8) =
+        # log p_router(group) + z - LSE(group)
+        if factorised:
+            score = ref.log_router[m, ref.groups[m]][:, None] + ref.logits[m] - ref.group_lse[m][:, None]
+        else:
+            score = ref.logits[m] - ref.lse[m]
+        zmap = dict(zip(ref.logit_tokens[m].ravel().tolist(), score.ravel().tolist()))
         if len(set(ids[m].tolist())) != k_tokens:
             rep.errors.append(f"row {m}: duplicate ids {ids[m].tolist()}")
             continue
@@ -110,10 +119,10 @@ def compare(W, gm, Wg, hidden_bits, k_groups, k_tokens, gpu, forced_groups=None,
                 if close(zmap[t], zmap[int(ref.ids[m, i])]):
                     rep.tie_resolved_ids += 1
                 else:
-                    rep.errors.append(f"row {m} pos {i}: id {t} (z={zmap[t]}) != oracle {int(ref.ids[m, i])} "
-                                      f"(z={zmap[int(ref.ids[m, i])]})")
+                    rep.errors.append(f"row {m} pos {i}: id {t} (score={zmap[t]}) != oracle {int(ref.ids[m, i])} "
+                                      f"(score={zmap[int(ref.ids[m, i])]})")
                     break
-            want = zmap[t] - ref.lse[m]
+            want = zmap[t]
             err = abs(float(lps[m, i]) - want)
             rep.max_logprob_err = max(rep.max_logprob_err, err)
             if not close(float(lps[m, i]), want):

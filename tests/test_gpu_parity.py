@@ -268,3 +268,49 @@ def test_draft_is_capturable_in_a_cuda_graph():
         torch.cuda.synchronize()
         assert torch.equal(ids, want_ids) and torch.equal(lps, want_lps)
     assert head.status() == 0
+
+
+@pytest.mark.parametrize("path,M,kg", [(lmhead.CORAL_PATH_STREAM, 5, 4), (lmhead.CORAL_PATH_STREAM, 40, 16),
+                                       (lmhead.CORAL_PATH_TCGEN05, 200, 4)])
+def test_factorised_distribution_eq8(path, M, kg):
+    """p(x) = p_router(n) * p_group(x): per-group softmax times the softmax of the router scores (Eq. 7, Eq. 8)."""
+    cfg = synth.CONFIGS["tiny"]
+    W, gm, Wg = synth.make_w_vocab(cfg), synth.make_group_map(cfg), synth.make_w_gate(cfg)
+    hb = synth.make_hidden(cfg, M)
+    head = _head(cfg, W, gm, Wg, max_M=M, max_kg=kg, max_kt=32)
+    head.set_path(path)
+    lmhead.coral_lmhead_set_output_mode(head.handle, lmhead.CORAL_OUTPUT_FACTORISED)
+    out = ph.gpu_draft_numpy(head, hb, kg, 10)
+    assert head.status() == 0
+    rows = np.unique(np.linspace(0, M - 1, 16).astype(int))
+    rep = ph.compare(W, gm, Wg, hb[rows], kg, 10, {k: a[rows] for k, a in out.items()}, factorised=True)
+    assert rep.ok, rep.errors
+    # back to the joint mode on the same handle
+    lmhead.coral_lmhead_set_output_mode(head.handle, lmhead.CORAL_OUTPUT_JOINT)
+    out = ph.gpu_draft_numpy(head, hb, kg, 10)
+    rep = ph.compare(W, gm, Wg, hb[rows], kg, 10, {k: a[rows] for k, a in out.items()})
+    assert rep.ok, rep.errors
+    head.close()
+
+
+@pytest.mark.parametrize("M", [3, 50])
+def test_two_layer_router_eq7(M):
+    """scores = W2 (SiLU(W1 h) + h): groups, gate scores and the final Eq. 8 distribution against the oracle."""
+    cfg = synth.CONFIGS["tiny"]
+    W, gm, Wg = synth.make_w_vocab(cfg), synth.make_group_map(cfg), synth.make_w_gate(cfg)
+    W1 = synth._normal_bf16(np.random.default_rng(21), cfg.H, cfg.H, 0.05)
+    hb = synth.make_hidden(cfg, M)
+    head = _head(cfg, W, gm, Wg, max_M=M, max_kg=4, max_kt=10)
+    lmhead.coral_lmhead_set_router_mlp(head.handle, ph.to_dev_bf16(W1))
+    for factorised in (False, True):
+        lmhead.coral_lmhead_set_output_mode(head.handle, int(factorised))
+        out = ph.gpu_draft_numpy(head, hb, 4, 10)
+        assert head.status() == 0
+        rep = ph.compare(W, gm, Wg, hb, 4, 10, out, W1=W1, factorised=factorised)
+        assert rep.ok, rep.errors
+    lmhead.coral_lmhead_set_router_mlp(head.handle, None)
+    lmhead.coral_lmhead_set_output_mode(head.handle, lmhead.CORAL_OUTPUT_JOINT)
+    out = ph.gpu_draft_numpy(head, hb, 4, 10)
+    rep = ph.compare(W, gm, Wg, hb, 4, 10, out)
+    assert rep.ok, rep.errors
+    head.close()
