@@ -37,7 +37,7 @@ extern "C" {
 #define CORAL_ERR_NOMEM (-4)       /* host or device allocation failed */
 #define CORAL_ERR_TIMEOUT (-5)     /* a bounded device-side wait gave up (device status word) */
 #define CORAL_ERR_BOUNDS (-6)      /* a device-side index check failed (device status word) */
-#define CORAL_ERR_TOO_LARGE (-7)   /* request exceeds the fixed scratch of coral_lmhead_route_static */
+#define CORAL_ERR_TOO_LARGE (-7)   /* request exceeds a built-in size limit (coral_lmhead_route_static, coral_tree_expand) */
 
 /* Limits of this build. */
 #define CORAL_MAX_GROUPS 256       /* n_groups <= 256 */
@@ -239,6 +239,23 @@ int coral_lmhead_last_stats(coral_lmhead_handle h, coral_lmhead_stats *out, void
  */
 int coral_lmhead_route_static(const void *W_gate_dev, const void *hidden_dev, int M, int H, int n_groups,
                               int k_groups, int32_t *out_groups_dev, float *out_gate_dev, void *stream);
+
+/*
+ * Tree-expansion score step on the outputs of coral_lmhead_draft (Section 2.2: multiple candidates per
+ * timestep form a tree of drafts; Section 4.1: tree depth 6, 60 candidate tokens; Appendix B: top 10 candidates
+ * per node).  For each of n_seq sequences with `nodes` rows:
+ *   child score = parent_scores[node] + cand_logprobs[node][i]      (one fp32 addition)
+ * and the K best children (descending score; equal -> lower node * k_tokens + i) are returned, sorted:
+ *   out_parent [n_seq x K] node index inside the sequence, out_token [n_seq x K] = cand_ids of the child,
+ *   out_score [n_seq x K].
+ * With cand_logprobs_dev = NULL and k_tokens = 1 the call re-ranks the nodes themselves (e.g. the final choice
+ * of the best 60 nodes); cand_ids_dev may be NULL (the flat child index is returned as token).
+ * All pointers device; asynchronous on `stream`; no scratch memory.  CORAL_ERR_TOO_LARGE if nodes * k_tokens
+ * exceeds 2048; CORAL_ERR_INVALID for NULL outputs, sizes < 1, K > min(256, nodes * k_tokens).
+ */
+int coral_tree_expand(const float *parent_scores_dev, const int32_t *cand_ids_dev, const float *cand_logprobs_dev,
+                      int n_seq, int nodes, int k_tokens, int K, int32_t *out_parent_dev, int32_t *out_token_dev,
+                      float *out_score_dev, void *stream);
 
 /* Static, NUL-terminated description of a status code. */
 const char *coral_lmhead_error_string(int code);

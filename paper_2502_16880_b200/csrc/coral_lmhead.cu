@@ -13,6 +13,7 @@
 #include "head_tc.cuh"
 #include "merge.cuh"
 #include "route.cuh"
+#include "tree.cuh"
 
 using namespace coral;
 
@@ -293,7 +294,7 @@ const char* coral_lmhead_error_string(int code) {
         case CORAL_ERR_NOMEM: return "out of memory";
         case CORAL_ERR_TIMEOUT: return "device-side wait timed out";
         case CORAL_ERR_BOUNDS: return "device-side index check failed";
-        case CORAL_ERR_TOO_LARGE: return "size exceeds the built-in scratch of the no-allocation entry point";
+        case CORAL_ERR_TOO_LARGE: return "size exceeds a built-in limit (fixed scratch of the no-allocation entry point, tree step)";
         default: return "unknown status";
     }
 }
@@ -544,6 +545,20 @@ int coral_lmhead_draft_host(coral_lmhead_handle h, const void* hidden_host, int 
         return CORAL_ERR_CUDA;
     if (cudaStreamSynchronize(st) != cudaSuccess) return CORAL_ERR_CUDA;
     return CORAL_OK;
+}
+
+int coral_tree_expand(const float* parent_scores_dev, const int32_t* cand_ids_dev, const float* cand_logprobs_dev,
+                      int n_seq, int nodes, int k_tokens, int K, int32_t* out_parent_dev, int32_t* out_token_dev,
+                      float* out_score_dev, void* stream) {
+    if (!parent_scores_dev || !out_parent_dev || !out_token_dev || !out_score_dev) return CORAL_ERR_INVALID;
+    if (n_seq < 1 || nodes < 1 || k_tokens < 1) return CORAL_ERR_INVALID;
+    if ((long long)nodes * k_tokens > kTreeMaxCand) return CORAL_ERR_TOO_LARGE;
+    if (K < 1 || K > kTreeMaxK || K > nodes * k_tokens) return CORAL_ERR_INVALID;
+    if (!cand_logprobs_dev && k_tokens != 1) return CORAL_ERR_INVALID;
+    tree_expand_kernel<<<n_seq, kTreeThreads, 0, static_cast<cudaStream_t>(stream)>>>(
+        parent_scores_dev, cand_ids_dev, cand_logprobs_dev, nodes, k_tokens, K, out_parent_dev, out_token_dev,
+        out_score_dev);
+    return cudaGetLastError() == cudaSuccess ? CORAL_OK : CORAL_ERR_CUDA;
 }
 
 int coral_lmhead_set_output_mode(coral_lmhead_handle h, int mode) {

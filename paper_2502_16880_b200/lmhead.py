@@ -62,6 +62,7 @@ _SIGNATURES = {
     "coral_lmhead_status": (_i, [_vp, _vp]),
     "coral_lmhead_last_stats": (_i, [_vp, ctypes.POINTER(coral_lmhead_stats), _vp]),
     "coral_lmhead_route_static": (_i, [_vp, _vp, _i, _i, _i, _i, _vp, _vp, _vp]),
+    "coral_tree_expand": (_i, [_vp, _vp, _vp, _i, _i, _i, _i, _vp, _vp, _vp, _vp]),
     "coral_lmhead_error_string": (ctypes.c_char_p, [_i]),
     "coral_lmhead_destroy": (_i, [_vp]),
 }
@@ -231,6 +232,16 @@ def coral_lmhead_route_static(W_gate, hidden, k_groups, out_groups, out_gate=Non
         _dev_ptr(W_gate, torch.bfloat16, False), _dev_ptr(hidden, torch.bfloat16, False), M, H, N, int(k_groups),
         _dev_ptr(out_groups, torch.int32, False), _dev_ptr(out_gate, torch.float32), _stream_ptr(stream)),
         "coral_lmhead_route_static")
+
+
+def coral_tree_expand(parent_scores, cand_ids, cand_logprobs, K, out_parent, out_token, out_score, stream=None):
+    """parent_scores [n_seq, nodes] f32; cand_ids / cand_logprobs [n_seq, nodes, k_tokens] (or None); outputs [n_seq, K]."""
+    n_seq, nodes = parent_scores.shape
+    k_tokens = 1 if cand_logprobs is None else cand_logprobs.shape[-1]
+    _check(load_library().coral_tree_expand(
+        _dev_ptr(parent_scores, torch.float32, False), _dev_ptr(cand_ids, torch.int32), _dev_ptr(cand_logprobs, torch.float32),
+        n_seq, nodes, k_tokens, int(K), _dev_ptr(out_parent, torch.int32, False), _dev_ptr(out_token, torch.int32, False),
+        _dev_ptr(out_score, torch.float32, False), _stream_ptr(stream)), "coral_tree_expand")
 
 
 def coral_lmhead_destroy(handle) -> None:
