@@ -242,9 +242,9 @@ def main():
         flush.fill_(i)
         torch.sum(flush)
 
-    def time_steps(M, k_groups, steps, warmup, batches, kernel_timing=False):
+    def time_steps(M, k_groups, steps, warmup, batches, kernel_timing=False, rho=0.0):
         """Per-step CUDA-event times (ms) with an L2 flush before every step, outside the event pair."""
-        hb_bits = [synth.make_hidden(cfg, M, batch=b) for b in batches]
+        hb_bits = [synth.make_hidden(cfg.with_(rho=rho), M, batch=b) for b in batches]
         hds = [dev_bf16(b) for b in hb_bits]
         ids = torch.empty((M, cfg.k_tokens), dtype=torch.int32, device=dev)
         lps = torch.empty((M, cfg.k_tokens), dtype=torch.float32, device=dev)
@@ -348,6 +348,13 @@ def main():
             also.append({"M": M, "us_per_step": us, "GBps": b_m / us / 1e3, "hbm_frac": b_m / us / 1e3 / peak,
                          "groups_touched_mean": float(np.mean(t_m))})
         out["other_M"] = also
+        # extra (not a workload of the list): rows correlated like tree siblings of one parent, where the union
+        # of selected groups no longer saturates (Appendix B: the worst case is unlikely in practice)
+        ms_c, _, t_c, _, _ = time_steps(60, cfg.k_groups, extra_steps, 3, my_batches, rho=0.3)
+        b_c = float(np.mean([algorithmic_bytes(cfg.with_(M=60), u, 60) for u in t_c]))
+        out["correlated_rows_M60_rho0.3"] = {"us_per_step": float(np.mean(ms_c)) * 1e3,
+                                             "groups_touched_mean": float(np.mean(t_c)),
+                                             "GBps": b_c / (float(np.mean(ms_c)) * 1e-3) / 1e9}
         # dense head on the same GPU: (i) this library with every group active, (ii) torch bf16 matmul comparator
         ms_d, _, t_d, _, _ = time_steps(cfg.M, cfg.N, extra_steps, 3, my_batches)
         dense_bytes = algorithmic_bytes(cfg, cfg.N, cfg.M)
