@@ -461,8 +461,11 @@ int coral_lmhead_draft_ex(coral_lmhead_handle h, const void* hidden_dev, int M, 
         route_fused_kernel<<<c.N, kRouteThreads, 0, st>>>(c, forced_groups_dev, out_groups_dev, out_gate_dev);
         ++launches;
     } else {
-        gate_tile_kernel<<<dim3((c.N + kGateTile - 1) / kGateTile, (M + kGateTile - 1) / kGateTile), 256, 0, st>>>(
-            c, out_gate_dev);
+        if (cfg.H % 32 == 0)
+            gate_mma_kernel<<<dim3((c.N + 15) / 16, (M + 7) / 8), 256, 0, st>>>(c, out_gate_dev);
+        else
+            gate_tile_kernel<<<dim3((c.N + kGateTile - 1) / kGateTile, (M + kGateTile - 1) / kGateTile), 256, 0, st>>>(
+                c, out_gate_dev);
         ++launches;
         select_kernel<<<(M + kSelectWarps - 1) / kSelectWarps, kSelectWarps * 32, 0, st>>>(c, forced_groups_dev,
                                                                                           out_groups_dev);

@@ -349,6 +349,56 @@ __global__ void __launch_bounds__(256) gate_tile_kernel(CallView c, float* __res
     }
 }
 
+// Gate scores on the warp-level tensor cores for many rows: a block computes a 16-group x 8-row tile, its 8 warps
+// splitting H in blocks of 32 columns (mma.sync m16n8k16, bf16 x bf16 -> fp32; groups on the M axis, rows on N).
+// Every lane loads 16 bytes of two gate rows and of one hidden row per block of 32 columns; the column order
+// inside a block is permuted the same way for both operands, which leaves the dot products unchanged.
+// grid (ceil(N/16), ceil(M/8)), H a multiple of 32.  Block (0,0) also clears the per-group row counters.
+__global__ void __launch_bounds__(256) gate_mma_kernel(CallView c, float* __restrict__ gate_tap) {
+    __shared__ float s_part[8][16 * 8];
+    const int n0 = blockIdx.x * 16, m0 = blockIdx.y * 8;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int gq = lane >> 2, tq = lane & 3;
+    if (blockIdx.x == 0 && blockIdx.y == 0)
+        for (int n = threadIdx.x; n < c.N; n += 256) c.group_count[n] = 0;
+    const bool a_lo = n0 + gq < c.N, a_hi = n0 + gq + 8 < c.N, b_ok = m0 + gq < c.M;
+    const uint16_t* wlo = c.w_gate + (size_t)(a_lo ? n0 + gq : 0) * c.H + tq * 8;
+    const uint16_t* whi = c.w_gate + (size_t)(a_hi ? n0 + gq + 8 : 0) * c.H + tq * 8;
+    const uint16_t* hb = c.hidden + (size_t)(b_ok ? m0 + gq : 0) * c.H + tq * 8;
+    float acc0[4] = {0.f, 0.f, 0.f, 0.f}, acc1[4] = {0.f, 0.f, 0.f, 0.f};
+    const int kblocks = c.H >> 5;
+    const uint4 zero = make_uint4(0, 0, 0, 0);
+#pragma unroll 4
+    for (int kb = warp; kb < kblocks; kb += 8) {
+        const uint4 a = a_lo ? __ldg(reinterpret_cast<const uint4*>(wlo + kb * 32)) : zero;
+        const uint4 b = a_hi ? __ldg(reinterpret_cast<const uint4*>(whi + kb * 32)) : zero;
+        const uint4 h = b_ok ? __ldg(reinterpret_cast<const uint4*>(hb + kb * 32)) : zero;
+        asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+                     : "+f"(acc0[0]), "+f"(acc0[1]), "+f"(acc0[2]), "+f"(acc0[3])
+                     : "r"(a.x), "r"(b.x), "r"(a.y), "r"(b.y), "r"(h.x), "r"(h.y));
+        asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+                     : "+f"(acc1[0]), "+f"(acc1[1]), "+f"(acc1[2]), "+f"(acc1[3])
+                     : "r"(a.z), "r"(b.z), "r"(a.w), "r"(b.w), "r"(h.z), "r"(h.w));
+    }
+    // accumulator layout: [0],[1] = group gq, rows 2*tq, 2*tq+1; [2],[3] = group gq + 8
+    float* sp = s_part[warp];
+    sp[gq * 8 + 2 * tq] = acc0[0] + acc1[0];
+    sp[gq * 8 + 2 * tq + 1] = acc0[1] + acc1[1];
+    sp[(gq + 8) * 8 + 2 * tq] = acc0[2] + acc1[2];
+    sp[(gq + 8) * 8 + 2 * tq + 1] = acc0[3] + acc1[3];
+    __syncthreads();
+    if (threadIdx.x < 128) {
+        const int g = threadIdx.x >> 3, r = threadIdx.x & 7;
+        if (n0 + g < c.N && m0 + r < c.M) {
+            float sum = 0.f;
+#pragma unroll
+            for (int w = 0; w < 8; ++w) sum += s_part[w][threadIdx.x];
+            c.gate[(size_t)(m0 + r) * c.N + n0 + g] = sum;
+            if (gate_tap) gate_tap[(size_t)(m0 + r) * c.N + n0 + g] = sum;
+        }
+    }
+}
+
 // select_kernel plus per-group row counts (integer atomics: the totals do not depend on their order).
 __global__ void __launch_bounds__(kSelectWarps * 32) count_groups_kernel(CallView c) {
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
