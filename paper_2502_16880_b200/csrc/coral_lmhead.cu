@@ -259,6 +259,9 @@ bool make_tc_maps(coral_lmhead_s* h) {
     return true;
 }
 
+// Dynamic shared memory of merge_stream_kernel for p_cap pieces and c_cap in-smem candidates.
+inline size_t merge_smem_bytes(int p_cap, int c_cap) { return (size_t)c_cap * 8 + (size_t)p_cap * 21 + 16; }
+
 constexpr size_t kTcSmemBytes = 1024 + (size_t)kTcStages * kTcStageBytes + 32 * kTcEpilogueThreads * 4 + 256;
 
 bool stream_ok(const coral_lmhead_s* h, int M) { return h->stream_smem > 0 && M <= kStreamMaxM; }
@@ -381,7 +384,9 @@ int coral_lmhead_create(coral_lmhead_handle* out, const coral_lmhead_config* cfg
                 cudaFuncSetAttribute(head_stream_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_optin) !=
                     cudaSuccess) { rc = CORAL_ERR_CUDA; break; }
             if (cudaFuncSetAttribute(merge_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     kMergeSmemCands * 8) != cudaSuccess) { rc = CORAL_ERR_CUDA; break; }
+                                     (int)merge_smem_bytes(kMergeMaxPieces, kMergeSmemCands)) != cudaSuccess) {
+                rc = CORAL_ERR_CUDA; break;
+            }
         }
         if (cudaMemcpyAsync(h->ws + h->L.group_tokens, group_tokens.data(), (size_t)V * 4, cudaMemcpyHostToDevice, st) !=
             cudaSuccess) { rc = CORAL_ERR_CUDA; break; }
@@ -484,10 +489,14 @@ int coral_lmhead_draft_ex(coral_lmhead_handle h, const void* hidden_dev, int M, 
                    dim3(kStreamThreads), (size_t)h->stream_smem, st, c, h->sg, pp, out_logits_dev);
         ++launches;
         if (h->timing) cudaEventRecord(h->ev_head1, st);
-        launch_pdl(merge_stream_kernel, dim3(M), dim3(kMergeStreamThreads), (size_t)kMergeSmemCands * 8, st, c, h->sg, pp,
-                   reinterpret_cast<float*>(h->ws + L.cand_val), reinterpret_cast<int32_t*>(h->ws + L.cand_id),
-                   (int)L.cand_cap, (int)kMergeSmemCands, (int)(h->out_mode == CORAL_OUTPUT_FACTORISED), out_ids_dev,
-                   out_logprobs_dev, out_lse_dev);
+        {
+            const int p_cap = h->sg.grid + 2 * k_groups;
+            const int c_cap = p_cap * k_tokens < kMergeSmemCands ? p_cap * k_tokens : kMergeSmemCands;
+            launch_pdl(merge_stream_kernel, dim3(M), dim3(kMergeStreamThreads), merge_smem_bytes(p_cap, c_cap), st, c,
+                       h->sg, pp, reinterpret_cast<float*>(h->ws + L.cand_val),
+                       reinterpret_cast<int32_t*>(h->ws + L.cand_id), (int)L.cand_cap, c_cap, p_cap,
+                       (int)(h->out_mode == CORAL_OUTPUT_FACTORISED), out_ids_dev, out_logprobs_dev, out_lse_dev);
+        }
         ++launches;
     } else if (path == CORAL_PATH_TCGEN05) {
         const Layout& L = h->L;
@@ -504,10 +513,14 @@ int coral_lmhead_draft_ex(coral_lmhead_handle h, const void* hidden_dev, int M, 
         mg.tc_rows = kTcPassRows;
         mg.T = L.tc_tiles;
         StreamPartials pp{tp.pmax, tp.psum, tp.pval, tp.pid};
-        launch_pdl(merge_stream_kernel, dim3(M), dim3(kMergeStreamThreads), (size_t)kMergeSmemCands * 8, st, c, mg, pp,
-                   reinterpret_cast<float*>(h->ws + L.cand_val), reinterpret_cast<int32_t*>(h->ws + L.cand_id),
-                   (int)L.cand_cap, (int)kMergeSmemCands, (int)(h->out_mode == CORAL_OUTPUT_FACTORISED), out_ids_dev,
-                   out_logprobs_dev, out_lse_dev);
+        {
+            const int p_cap = k_groups * L.tc_tiles;
+            const int c_cap = p_cap * k_tokens;          // tc_usable() keeps this within kMergeSmemCands
+            launch_pdl(merge_stream_kernel, dim3(M), dim3(kMergeStreamThreads), merge_smem_bytes(p_cap, c_cap), st, c, mg,
+                       pp, reinterpret_cast<float*>(h->ws + L.cand_val), reinterpret_cast<int32_t*>(h->ws + L.cand_id),
+                       (int)L.cand_cap, c_cap, p_cap, (int)(h->out_mode == CORAL_OUTPUT_FACTORISED), out_ids_dev,
+                       out_logprobs_dev, out_lse_dev);
+        }
         ++launches;
     } else {
         head_simt_kernel<<<dim3(c.T, c.N), kSimtThreads, h->simt_smem, st>>>(c, out_logits_dev);

@@ -406,7 +406,7 @@ constexpr int kMergeRankMax = 256;            // survivors ranked by counting; m
 __global__ void __launch_bounds__(kMergeStreamThreads) merge_stream_kernel(CallView c, StreamGeom g, StreamPartials pp,
                                                                            float* __restrict__ cand_val_scratch,
                                                                            int32_t* __restrict__ cand_id_scratch,
-                                                                           int cand_cap, int smem_cands, int factorised,
+                                                                           int cand_cap, int smem_cands, int p_cap, int factorised,
                                                                            int32_t* __restrict__ out_ids,
                                                                            float* __restrict__ out_logprobs,
                                                                            float* __restrict__ lse_tap) {
@@ -419,9 +419,13 @@ __global__ void __launch_bounds__(kMergeStreamThreads) merge_stream_kernel(CallV
     __shared__ int s_n;
     __shared__ int s_first[kMaxGroups], s_base[kMaxGroups + 1], s_rpos[kMaxGroups], s_j[kMaxGroups];
     __shared__ float s_off[kMaxGroups];           // per slot: what is added to a logit to give the emitted log-prob
-    __shared__ int s_piece[kMergeMaxPieces];
-    __shared__ unsigned char s_pslot[kMergeMaxPieces];
-    __shared__ float s_pm[kMergeMaxPieces], s_ps[kMergeMaxPieces], s_last[kMergeMaxPieces], s_head[kMergeMaxPieces];
+    // dynamic shared memory: candidates (smem_cands values + ids), then per-piece arrays of capacity p_cap
+    float* s_pm = reinterpret_cast<float*>(msm + (size_t)smem_cands * 8);
+    float* s_ps = s_pm + p_cap;
+    float* s_last = s_ps + p_cap;
+    float* s_head = s_last + p_cap;
+    int* s_piece = reinterpret_cast<int*>(s_head + p_cap);
+    unsigned char* s_pslot = reinterpret_cast<unsigned char*>(s_piece + p_cap);
 
     // The router's outputs were complete before the streaming kernel let this grid start.
     const int n_items = c.state->n_virtual * g.T;
@@ -463,7 +467,7 @@ __global__ void __launch_bounds__(kMergeStreamThreads) merge_stream_kernel(CallV
         s_base[c.k_groups] = run;
     }
     __syncthreads();
-    const int P = min(s_base[c.k_groups], kMergeMaxPieces);
+    const int P = min(s_base[c.k_groups], p_cap);
     for (int q = threadIdx.x; q < P; q += kMergeStreamThreads) {
         int s = 0;
         while (s + 1 < c.k_groups && s_base[s + 1] <= q) ++s;
