@@ -489,7 +489,8 @@ __global__ void __launch_bounds__(kMergeStreamThreads) merge_stream_kernel(CallV
     for (int q = threadIdx.x; q < P; q += kMergeStreamThreads) {
         const size_t p = (size_t)s_piece[q];
         const float a = pp.pmax[p], b = pp.psum[p];
-        const float l = pp.pval[p * c.k_tokens + c.k_tokens - 1], h = pp.pval[p * c.k_tokens];
+        float l = pp.pval[p * c.k_tokens + c.k_tokens - 1], h = pp.pval[p * c.k_tokens];
+        if (a == kNegInf) { l = kNegInf; h = kNegInf; }      // empty piece: its candidate list was not written
         s_pm[q] = a; s_ps[q] = b; s_last[q] = l; s_head[q] = h;
         mx = fmaxf(mx, a);
     }
@@ -562,7 +563,7 @@ __global__ void __launch_bounds__(kMergeStreamThreads) merge_stream_kernel(CallV
         for (int u = 0; u < 4; ++u) {
             v[u] = kNegInf;
             id[u] = kNoToken;
-            if (q0 + u < P && lane < c.k_tokens) {
+            if (q0 + u < P && lane < c.k_tokens && s_pm[q0 + u] != kNegInf) {
                 const size_t p = (size_t)s_piece[q0 + u];
                 v[u] = pp.pval[p * c.k_tokens + lane] + s_off[s_pslot[q0 + u]];
                 id[u] = pp.pid[p * c.k_tokens + lane];

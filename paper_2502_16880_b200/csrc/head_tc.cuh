@@ -60,17 +60,38 @@ __device__ __forceinline__ void tc_wait(uint32_t bar, uint32_t parity, volatile 
     set_status(st, -5);
 }
 
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x0, int x1, uint32_t bar) {
+// L2 eviction policies for the tiled loads: the weights of a group are streamed once per pass (evict first,
+// unless a later pass reads them again), the gathered hidden rows are re-read for every pair of sub-tiles
+// (evict last), so the weight stream does not push them out of L2.
+__device__ __forceinline__ uint64_t l2_policy_evict_first() {
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+__device__ __forceinline__ uint64_t l2_policy_evict_normal() {
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_normal.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+__device__ __forceinline__ uint64_t l2_policy_evict_last() {
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x0, int x1, uint32_t bar,
+                                            uint64_t policy) {
     asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-        ::"r"(dst), "l"(map), "r"(x0), "r"(x1), "r"(bar) : "memory");
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, "
+        "%3}], [%4], %5;"
+        ::"r"(dst), "l"(map), "r"(x0), "r"(x1), "r"(bar), "l"(policy) : "memory");
 }
 __device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap* map, int x0, int x1, int x2, int x3,
-                                            int x4, uint32_t bar) {
+                                            int x4, uint32_t bar, uint64_t policy) {
     asm volatile(
-        "cp.async.bulk.tensor.5d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5, "
-        "%6}], [%7];"
-        ::"r"(dst), "l"(map), "r"(x0), "r"(x1), "r"(x2), "r"(x3), "r"(x4), "r"(bar) : "memory");
+        "cp.async.bulk.tensor.5d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, "
+        "%3, %4, %5, %6}], [%7], %8;"
+        ::"r"(dst), "l"(map), "r"(x0), "r"(x1), "r"(x2), "r"(x3), "r"(x4), "r"(bar), "l"(policy) : "memory");
 }
 
 // Shared-memory matrix descriptor: K-major tile of 128-byte rows, 128-byte swizzle, 8-row groups 1024 bytes apart.
@@ -132,18 +153,29 @@ __device__ __forceinline__ void tc_insert(float (&lv)[KT], int (&li)[KT], float 
     }
 }
 
-// Epilogue of one 128 x 128 accumulator for one thread (= one hidden row): fold the 128 logits of vocab rows
-// [base, base + valid) of group n into (max, sum-exp, top-k) and write the partial.
+// Running statistics of one hidden row over the sub-tiles one epilogue thread sees of a pass: the thread
+// keeps (max, sum-exp, top-k) in registers from sub-tile to sub-tile and writes one full partial at the
+// last of them; the other sub-tiles get an "empty" marker (max = -inf, sum = 0), which the merge skips.
 template <int KT>
-__device__ __forceinline__ void tc_fold_row(const CallView& c, const TcPartials& pp, float* __restrict__ logits_tap,
-                                            uint32_t tmem_acc_row, int n, int base, size_t pidx, bool row_valid,
-                                            int tap_m, int tap_slot, float* zs) {
-    constexpr float kLog2e = 1.4426950408889634f;
+struct TcRowState {
     float lv[KT];
     int li[KT];
+    float mx, sum;
+    __device__ __forceinline__ void reset() {
 #pragma unroll
-    for (int j = 0; j < KT; ++j) { lv[j] = kNegInf; li[j] = kNoToken; }
-    float mx = kNegInf, sum = 0.f;
+        for (int j = 0; j < KT; ++j) { lv[j] = kNegInf; li[j] = kNoToken; }
+        mx = kNegInf;
+        sum = 0.f;
+    }
+};
+
+// Epilogue of one 128 x 128 accumulator for one thread (= one hidden row): fold the 128 logits of vocab rows
+// [base, base + valid) of the group into the running (max, sum-exp, top-k).
+template <int KT>
+__device__ __forceinline__ void tc_fold_row(const CallView& c, TcRowState<KT>& st, float* __restrict__ logits_tap,
+                                            uint32_t tmem_acc_row, int base, bool row_valid, int tap_m, int tap_slot,
+                                            float* zs) {
+    constexpr float kLog2e = 1.4426950408889634f;
     const int valid = min(kTcSub, c.v - base);
 #pragma unroll 1
     for (int ch = 0; ch < 4; ++ch) {
@@ -154,43 +186,49 @@ __device__ __forceinline__ void tc_fold_row(const CallView& c, const TcPartials&
         float cm = kNegInf;
 #pragma unroll
         for (int i = 0; i < 32; ++i) cm = fmaxf(cm, i < nv ? z[i] : kNegInf);
-        const float nm = fmaxf(mx, cm);
+        const float nm = fmaxf(st.mx, cm);
         float add = 0.f;
 #pragma unroll
         for (int i = 0; i < 32; ++i) add += i < nv ? exp2f((z[i] - nm) * kLog2e) : 0.f;
-        sum = sum * exp2f((mx - nm) * kLog2e) + add;            // exp2(-inf) = 0 on the first chunk
-        mx = nm;
+        st.sum = st.sum * exp2f((st.mx - nm) * kLog2e) + add;   // exp2(-inf) = 0 on the first chunk
+        st.mx = nm;
         if (logits_tap) {
             float* dst = logits_tap + ((size_t)tap_m * c.k_groups + tap_slot) * c.v + base + ch * 32;
 #pragma unroll
             for (int i = 0; i < 32; ++i)
                 if (i < nv) dst[i] = z[i];
         }
-        // candidates for the top-k list: a bit per element that beats the current k-th entry; the few that do
+        // candidates for the top-k list: a bit per element that reaches the current k-th entry; the few that do
         // are fetched by index from a shared-memory copy of the chunk (element i of thread t at zs[i * T + t])
-        unsigned cand = 0;
+        if (cm >= st.lv[KT - 1]) {
+            unsigned cand = 0;
 #pragma unroll
-        for (int i = 0; i < 32; ++i)
-            cand |= (i < nv && z[i] >= lv[KT - 1]) ? (1u << i) : 0u;     // ties are settled by the insertion
-        if (cand) {
+            for (int i = 0; i < 32; ++i)
+                cand |= (i < nv && z[i] >= st.lv[KT - 1]) ? (1u << i) : 0u;   // ties are settled by the insertion
 #pragma unroll
             for (int i = 0; i < 32; ++i) zs[i * kTcEpilogueThreads] = z[i];
             while (cand) {
                 const int i = __ffs(cand) - 1;
                 cand &= cand - 1;
-                tc_insert<KT>(lv, li, zs[i * kTcEpilogueThreads], base + ch * 32 + i);
+                const float zi = zs[i * kTcEpilogueThreads];
+                if (zi >= st.lv[KT - 1]) tc_insert<KT>(st.lv, st.li, zi, base + ch * 32 + i);
             }
         }
     }
-    if (row_valid) {
-        pp.pmax[pidx] = mx;
-        pp.psum[pidx] = sum;
+}
+
+// Writes the thread's running partial as piece `pidx` (token ids through the group's row -> token table).
+template <int KT>
+__device__ __forceinline__ void tc_flush_row(const CallView& c, const TcPartials& pp, const TcRowState<KT>& st, int n,
+                                             size_t pidx) {
+    pp.pmax[pidx] = st.mx;
+    pp.psum[pidx] = st.sum;
 #pragma unroll
-        for (int j = 0; j < KT; ++j) {
-            if (j < c.k_tokens) {
-                pp.pval[pidx * c.k_tokens + j] = lv[j];
-                pp.pid[pidx * c.k_tokens + j] = li[j] == kNoToken ? kNoToken : __ldg(c.group_tokens + (size_t)n * c.v + li[j]);
-            }
+    for (int j = 0; j < KT; ++j) {
+        if (j < c.k_tokens) {
+            pp.pval[pidx * c.k_tokens + j] = st.lv[j];
+            pp.pid[pidx * c.k_tokens + j] =
+                st.li[j] == kNoToken ? kNoToken : __ldg(c.group_tokens + (size_t)n * c.v + st.li[j]);
         }
     }
 }
@@ -213,6 +251,59 @@ __device__ __forceinline__ TcBatch tc_batch_at(const CallView& c, const TcGeom& 
     b.nsub = (b.nmb == 1 && b.t + 1 < g.tiles && pos + 1 < hi) ? 2 : 1;
     b.hrow = c.group_offset[b.n] + b.pass * kTcPassRows;
     return b;
+}
+
+// Epilogue warps' loop over the CTA's run [lo, hi).  Of the sub-tiles of a pass inside the run, the warps of
+// accumulator `which` see every second one; they write their running partial at the last one they see.
+template <int KT>
+__device__ __forceinline__ void tc_epilogue(const CallView& c, const TcGeom& g, const TcPartials& pp,
+                                            float* __restrict__ logits_tap, uint32_t tmem_base, uint64_t* tmem_full,
+                                            uint64_t* tmem_empty, volatile int* abort_flag, float* zstash, int lo, int hi) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int quarter = warp & 3;
+    const int which = (warp - 2) >> 2;                    // accumulator 0 or 1 of the batch
+    const int row_in_block = quarter * 32 + lane;
+    float* zs = zstash + (threadIdx.x - 64);
+    TcRowState<KT> st;
+    st.reset();
+    int batch = 0;
+    for (int pos = lo; pos < hi; ++batch) {
+        const TcBatch b = tc_batch_at(c, g, pos, hi);
+        const int buf = batch & 1;
+        tc_wait(smem_u32(&tmem_full[buf]), ((uint32_t)batch >> 1) & 1u, abort_flag, c.state);
+        tc_fence_after();
+        if (which < b.nmb + b.nsub - 1) {
+            const int mb = b.nmb == 2 ? which : 0;
+            const int sub = b.nmb == 2 ? 0 : which;
+            const int r = mb * kTcBlockRows + row_in_block;
+            const bool row_valid = r < b.R;
+            const int tap_m = row_valid && logits_tap ? c.bucket_row[b.hrow + r] : 0;
+            const int tap_slot = row_valid && logits_tap ? c.bucket_slot[b.hrow + r] : 0;
+            const size_t pidx = ((size_t)b.j * g.tiles + b.t + sub) * kTcPassRows + r;
+            const uint32_t acc_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)((buf * 2 + which) * kTcSub);
+            tc_fold_row<KT>(c, st, logits_tap, acc_row, (b.t + sub) * kTcSub, row_valid, tap_m, tap_slot, zs);
+            // is this the last sub-tile of the pass that these warps see in this run?
+            const int npos = pos + b.nsub;
+            bool last = b.nmb == 2 || npos >= hi || npos / g.tiles != b.j;
+            if (!last && which == 1) {
+                const int nt = npos - b.j * g.tiles;
+                last = nt + 1 >= g.tiles || npos + 1 >= hi;       // the next batch is a single sub-tile
+            }
+            if (row_valid) {
+                if (last) {
+                    tc_flush_row<KT>(c, pp, st, b.n, pidx);
+                } else {
+                    pp.pmax[pidx] = kNegInf;
+                    pp.psum[pidx] = 0.f;
+                }
+            }
+            if (last) st.reset();
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&tmem_empty[buf]));
+        pos += b.nsub;
+    }
 }
 
 // grid = g.grid CTAs of kTcThreads threads; dynamic shared memory: 1 KiB alignment slack + kTcStages stages + barriers.
@@ -263,9 +354,13 @@ __global__ void __launch_bounds__(kTcThreads, 1)
         if (lane == 0) {
             int stage = 0;
             uint32_t phase = 0;
+            const uint64_t pol_first = l2_policy_evict_first(), pol_normal = l2_policy_evict_normal(),
+                           pol_last = l2_policy_evict_last();
             for (int pos = lo; pos < hi;) {
                 const TcBatch b = tc_batch_at(c, g, pos, hi);
                 const uint32_t bytes = (uint32_t)(b.nmb + b.nsub) * kTcTileBytes;
+                const bool read_again = c.group_count[b.n] > (b.pass + 1) * kTcPassRows;   // a later pass follows
+                const uint64_t pol_w = read_again ? pol_normal : pol_first;
                 for (int ks = 0; ks < g.ksteps; ++ks) {
                     tc_wait(smem_u32(&empty[stage]), phase ^ 1u, abort_flag, c.state);
                     const uint32_t bar = smem_u32(&full[stage]);
@@ -273,9 +368,9 @@ __global__ void __launch_bounds__(kTcThreads, 1)
                     mbar_expect_tx(bar, bytes);
                     // tiles 0 and 1 of a stage are the hidden-row blocks, tiles 1/2 the weight sub-tiles
                     for (int mb = 0; mb < b.nmb; ++mb)
-                        tma_load_2d(sb + mb * kTcTileBytes, &map_h, ks * kTcK, b.hrow + mb * kTcBlockRows, bar);
+                        tma_load_2d(sb + mb * kTcTileBytes, &map_h, ks * kTcK, b.hrow + mb * kTcBlockRows, bar, pol_last);
                     for (int sub = 0; sub < b.nsub; ++sub)
-                        tma_load_5d(sb + (b.nmb + sub) * kTcTileBytes, &map_w, 0, 0, ks, (b.t + sub) * 8, b.n, bar);
+                        tma_load_5d(sb + (b.nmb + sub) * kTcTileBytes, &map_w, 0, 0, ks, (b.t + sub) * 8, b.n, bar, pol_w);
                     if (++stage == kTcStages) { stage = 0; phase ^= 1u; }
                 }
                 pos += b.nsub;
@@ -315,35 +410,10 @@ __global__ void __launch_bounds__(kTcThreads, 1)
     } else {
         // epilogue: thread <-> tensor-memory lane = hidden row; the two warps of a lane quarter take one
         // accumulator of the batch each
-        const int quarter = warp & 3;
-        const int which = (warp - 2) >> 2;                    // accumulator 0 or 1 of the batch
-        const int row_in_block = quarter * 32 + lane;
-        float* zs = zstash + (threadIdx.x - 64);
-        int batch = 0;
-        for (int pos = lo; pos < hi; ++batch) {
-            const TcBatch b = tc_batch_at(c, g, pos, hi);
-            const int buf = batch & 1;
-            tc_wait(smem_u32(&tmem_full[buf]), ((uint32_t)batch >> 1) & 1u, abort_flag, c.state);
-            tc_fence_after();
-            if (which < b.nmb + b.nsub - 1) {
-                const int mb = b.nmb == 2 ? which : 0;
-                const int sub = b.nmb == 2 ? 0 : which;
-                const int r = mb * kTcBlockRows + row_in_block;
-                const bool row_valid = r < b.R;
-                const int tap_m = row_valid ? c.bucket_row[b.hrow + r] : 0;
-                const int tap_slot = row_valid ? c.bucket_slot[b.hrow + r] : 0;
-                const size_t pidx = ((size_t)b.j * g.tiles + b.t + sub) * kTcPassRows + r;
-                const uint32_t acc_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)((buf * 2 + which) * kTcSub);
-                if (c.k_tokens <= 10)
-                    tc_fold_row<10>(c, pp, logits_tap, acc_row, b.n, (b.t + sub) * kTcSub, pidx, row_valid, tap_m, tap_slot, zs);
-                else
-                    tc_fold_row<32>(c, pp, logits_tap, acc_row, b.n, (b.t + sub) * kTcSub, pidx, row_valid, tap_m, tap_slot, zs);
-            }
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&tmem_empty[buf]));
-            pos += b.nsub;
-        }
+        if (c.k_tokens <= 10)
+            tc_epilogue<10>(c, g, pp, logits_tap, tmem_base, tmem_full, tmem_empty, abort_flag, zstash, lo, hi);
+        else
+            tc_epilogue<32>(c, g, pp, logits_tap, tmem_base, tmem_full, tmem_empty, abort_flag, zstash, lo, hi);
     }
     tc_fence_before();
     __syncthreads();
