@@ -84,6 +84,8 @@ Layout make_layout(const coral_lmhead_config& c) {
     Layout L{};
     L.v = c.V / c.n_groups;
     L.T = (L.v + kTileRows - 1) / kTileRows;
+    L.T16 = (L.v + 15) / 16;
+    L.KB = (c.H + 63) / 64;
     const size_t M = c.max_M, N = c.n_groups, H = c.H, kg = c.max_k_groups, kt = c.max_k_tokens, T = L.T;
     size_t o = 0;
     auto take = [&](size_t bytes) { size_t at = o; o = align_up(o + bytes); return at; };
@@ -118,7 +120,7 @@ Layout make_layout(const coral_lmhead_config& c) {
     L.tc_rows = M > (size_t)kTcMinRows ? M * kg : 0;
     L.tc_vcap = L.tc_rows ? (int)(N + (M * kg + kTcPassRows - 1) / kTcPassRows) : 0;
     const size_t tcp = (size_t)L.tc_vcap * L.tc_tiles * kTcPassRows;
-    L.tc_hg = take(L.tc_rows * H * 2);
+    L.tc_hg = take((size_t)L.tc_vcap * L.KB * kTcPassRows * kTcK * 2);   // blocked: [entry][column block][128][64]
     L.tc_max = take(tcp * 4);
     L.tc_sum = take(tcp * 4);
     L.tc_val = take(tcp * kt * 4);
@@ -127,8 +129,6 @@ Layout make_layout(const coral_lmhead_config& c) {
     L.stage_ids = take(M * kt * 4);
     L.stage_logprobs = take(M * kt * 4);
     L.total = o;
-    L.T16 = (L.v + 15) / 16;
-    L.KB = (c.H + 63) / 64;
     L.packed_bytes = (size_t)c.n_groups * L.T16 * L.KB * 16 * 64 * 2;
     return L;
 }
@@ -235,8 +235,8 @@ EncodeTiledFn encode_tiled_fn() {
 
 // Tensor maps of the tensor-core path: the packed weights as a 5-d tensor (column in block, row in item,
 // 64-column block, item, group) read in boxes of 64 columns x 128 rows (8 items = eight contiguous 2 KiB
-// pieces), and the gathered hidden rows as a matrix read in boxes of 64 columns x 128 rows; both land in
-// shared memory with the 128-byte swizzle.
+// pieces), and the gathered hidden rows, stored as blocks of 128 rows x 64 columns, as a 64-column matrix
+// read one block (a contiguous 16 KiB) at a time; both land in shared memory with the 128-byte swizzle.
 bool make_tc_maps(coral_lmhead_s* h) {
     EncodeTiledFn enc = encode_tiled_fn();
     if (!enc) return false;
@@ -249,8 +249,8 @@ bool make_tc_maps(coral_lmhead_s* h) {
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
         return false;
-    const cuuint64_t hdim[2] = {(cuuint64_t)h->cfg.H, (cuuint64_t)L.tc_rows};
-    const cuuint64_t hstr[1] = {(cuuint64_t)h->cfg.H * 2};
+    const cuuint64_t hdim[2] = {(cuuint64_t)kTcK, (cuuint64_t)L.tc_vcap * L.KB * kTcPassRows};
+    const cuuint64_t hstr[1] = {(cuuint64_t)kTcK * 2};
     const cuuint32_t hbox[2] = {(cuuint32_t)kTcK, (cuuint32_t)kTcBlockRows};
     if (enc(&h->map_h, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, h->ws + L.tc_hg, hdim, hstr, hbox, ones,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,

@@ -1,12 +1,12 @@
 // Routed grouped GEMM for many query rows on the 5th-generation tensor cores.
 //
-// For every (group, pass) of the union list the rows that selected the group (gathered beforehand into one
-// contiguous bf16 matrix, up to 256 rows per pass) are multiplied with the group's vocab rows:
+// For every (group, pass) of the union list the rows that selected the group (gathered beforehand into
+// blocks of 128 rows x 64 columns, one contiguous 16 KiB block per pass and column block) are multiplied
+// with the group's vocab rows:
 //   D[hidden row, vocab row] = sum_k hg[row, k] * W[vocab row, k]
-// tcgen05.mma (kind::f16, bf16 x bf16 -> fp32) with M = 128 hidden rows per accumulator block (two blocks when
-// the pass has more than 128 rows) and N = 128 vocab rows per sub-tile.  A batch is two accumulators: two
-// sub-tiles sharing one read of the hidden rows, or one sub-tile for two row blocks.  Operands arrive through
-// TMA tiled loads (128-byte swizzle) in a 4-stage ring; accumulators live in tensor memory, double-buffered
+// tcgen05.mma (kind::f16, bf16 x bf16 -> fp32) with M = 128 hidden rows (one pass) and N = 128 vocab rows per
+// sub-tile.  A batch is two accumulators: two sub-tiles sharing one read of the hidden rows (one at the end
+// of a pass or of the CTA's run).  Operands arrive through TMA tiled loads (128-byte swizzle) in a 4-stage ring; accumulators live in tensor memory, double-buffered
 // (2 x 2 x 128 columns), so the epilogue of one batch runs under the MMAs of the next.  The epilogue reads
 // each thread's hidden row straight from tensor memory and folds the logits into (max, sum-exp, top-k), one
 // partial per (pass, sub-tile, row), so logits never travel to HBM.  (CORAL Section 3.3: logits only for the activated groups; Appendix B: the
@@ -35,7 +35,7 @@ constexpr int kTcPassRows = 128;     // hidden rows per pass over a group's weig
 constexpr int kTcK = 64;             // columns per stage (one 128-byte swizzle atom of bf16)
 constexpr int kTcStages = 4;
 constexpr int kTcTileBytes = kTcBlockRows * kTcK * 2;   // 16 KiB: one 128 x 64 bf16 operand tile
-constexpr int kTcStageBytes = 3 * kTcTileBytes;         // (A0, B0, B1) or (A0, A1, B0)
+constexpr int kTcStageBytes = 3 * kTcTileBytes;         // (A, B0, B1)
 constexpr int kTcTmemCols = 512;
 constexpr int kTcSpin = 1 << 22;
 
@@ -130,13 +130,23 @@ __device__ __forceinline__ void tc_ld32(uint32_t taddr, float (&v)[32]) {
     for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
 
-// hg[p][:] = hidden[bucket_row[p]][:] for the M * k_groups (row, slot) pairs, bucket order.
+// Gathers the hidden rows of every (group, pass) into the blocked operand layout
+//   hg[pass entry j][column block kb][row r of the pass, 128][64 columns]
+// so that the 128 x 64 operand tile of a pass is one contiguous 16 KiB block.  One thread block per
+// (row, slot) pair in bucket order; columns past H are written as zero; rows past the pass's size keep
+// whatever they held (their accumulator lanes are never read).
 __global__ void __launch_bounds__(128) tc_gather_kernel(CallView c, uint16_t* __restrict__ hg) {
     const int p = blockIdx.x;
     const int m = c.bucket_row[p];
+    const int n = c.sel[(size_t)m * c.k_groups + c.bucket_slot[p]];
+    const int rg = p - c.group_offset[n];
+    const int j = c.union_rank[n] + rg / kTcPassRows;
+    const int r = rg % kTcPassRows;
     const uint4* src = reinterpret_cast<const uint4*>(c.hidden + (size_t)m * c.H);
-    uint4* dst = reinterpret_cast<uint4*>(hg + (size_t)p * c.H);
-    for (int ch = threadIdx.x; ch < (c.H >> 3); ch += 128) dst[ch] = __ldg(src + ch);
+    uint4* dst = reinterpret_cast<uint4*>(hg) + ((size_t)j * c.KB * kTcPassRows + r) * 8;
+    const int chunks = c.H >> 3;
+    for (int ch = threadIdx.x; ch < c.KB * 8; ch += 128)
+        dst[(size_t)(ch >> 3) * kTcPassRows * 8 + (ch & 7)] = ch < chunks ? __ldg(src + ch) : make_uint4(0, 0, 0, 0);
 }
 
 // Sorted insertion into a thread-private top-KT list (value desc, row index asc).
@@ -233,11 +243,9 @@ __device__ __forceinline__ void tc_flush_row(const CallView& c, const TcPartials
     }
 }
 
-// One batch of the run: the pass it belongs to, its first sub-tile, and how the two accumulators of the
-// batch are used: two sub-tiles of one 128-row block (nmb = 1, nsub = 2), one sub-tile of two blocks
-// (nmb = 2, nsub = 1), or a single accumulator.
+// One batch of the run: the pass it belongs to, its first sub-tile, and whether it holds two sub-tiles.
 struct TcBatch {
-    int j, t, n, pass, R, nmb, nsub, hrow;
+    int j, t, n, pass, R, nsub, hrow;
 };
 __device__ __forceinline__ TcBatch tc_batch_at(const CallView& c, const TcGeom& g, int pos, int hi) {
     TcBatch b;
@@ -247,9 +255,8 @@ __device__ __forceinline__ TcBatch tc_batch_at(const CallView& c, const TcGeom& 
     b.n = entry & 0xffff;
     b.pass = entry >> 16;
     b.R = min(c.group_count[b.n] - b.pass * kTcPassRows, kTcPassRows);
-    b.nmb = b.R > kTcBlockRows ? 2 : 1;
-    b.nsub = (b.nmb == 1 && b.t + 1 < g.tiles && pos + 1 < hi) ? 2 : 1;
-    b.hrow = c.group_offset[b.n] + b.pass * kTcPassRows;
+    b.nsub = (b.t + 1 < g.tiles && pos + 1 < hi) ? 2 : 1;
+    b.hrow = c.group_offset[b.n] + b.pass * kTcPassRows;      // first bucket position of the pass
     return b;
 }
 
@@ -272,10 +279,9 @@ __device__ __forceinline__ void tc_epilogue(const CallView& c, const TcGeom& g, 
         const int buf = batch & 1;
         tc_wait(smem_u32(&tmem_full[buf]), ((uint32_t)batch >> 1) & 1u, abort_flag, c.state);
         tc_fence_after();
-        if (which < b.nmb + b.nsub - 1) {
-            const int mb = b.nmb == 2 ? which : 0;
-            const int sub = b.nmb == 2 ? 0 : which;
-            const int r = mb * kTcBlockRows + row_in_block;
+        if (which < b.nsub) {
+            const int sub = which;
+            const int r = row_in_block;
             const bool row_valid = r < b.R;
             const int tap_m = row_valid && logits_tap ? c.bucket_row[b.hrow + r] : 0;
             const int tap_slot = row_valid && logits_tap ? c.bucket_slot[b.hrow + r] : 0;
@@ -284,7 +290,7 @@ __device__ __forceinline__ void tc_epilogue(const CallView& c, const TcGeom& g, 
             tc_fold_row<KT>(c, st, logits_tap, acc_row, (b.t + sub) * kTcSub, row_valid, tap_m, tap_slot, zs);
             // is this the last sub-tile of the pass that these warps see in this run?
             const int npos = pos + b.nsub;
-            bool last = b.nmb == 2 || npos >= hi || npos / g.tiles != b.j;
+            bool last = npos >= hi || npos / g.tiles != b.j;
             if (!last && which == 1) {
                 const int nt = npos - b.j * g.tiles;
                 last = nt + 1 >= g.tiles || npos + 1 >= hi;       // the next batch is a single sub-tile
@@ -358,7 +364,7 @@ __global__ void __launch_bounds__(kTcThreads, 1)
                            pol_last = l2_policy_evict_last();
             for (int pos = lo; pos < hi;) {
                 const TcBatch b = tc_batch_at(c, g, pos, hi);
-                const uint32_t bytes = (uint32_t)(b.nmb + b.nsub) * kTcTileBytes;
+                const uint32_t bytes = (uint32_t)(1 + b.nsub) * kTcTileBytes;
                 const bool read_again = c.group_count[b.n] > (b.pass + 1) * kTcPassRows;   // a later pass follows
                 const uint64_t pol_w = read_again ? pol_normal : pol_first;
                 for (int ks = 0; ks < g.ksteps; ++ks) {
@@ -366,11 +372,10 @@ __global__ void __launch_bounds__(kTcThreads, 1)
                     const uint32_t bar = smem_u32(&full[stage]);
                     const uint32_t sb = smem_u32(smem + (size_t)stage * kTcStageBytes);
                     mbar_expect_tx(bar, bytes);
-                    // tiles 0 and 1 of a stage are the hidden-row blocks, tiles 1/2 the weight sub-tiles
-                    for (int mb = 0; mb < b.nmb; ++mb)
-                        tma_load_2d(sb + mb * kTcTileBytes, &map_h, ks * kTcK, b.hrow + mb * kTcBlockRows, bar, pol_last);
+                    // tile 0 of a stage is the pass's block of hidden rows, tiles 1 and 2 the weight sub-tiles
+                    tma_load_2d(sb, &map_h, 0, (b.j * g.ksteps + ks) * kTcPassRows, bar, pol_last);
                     for (int sub = 0; sub < b.nsub; ++sub)
-                        tma_load_5d(sb + (b.nmb + sub) * kTcTileBytes, &map_w, 0, 0, ks, (b.t + sub) * 8, b.n, bar, pol_w);
+                        tma_load_5d(sb + (1 + sub) * kTcTileBytes, &map_w, 0, 0, ks, (b.t + sub) * 8, b.n, bar, pol_w);
                     if (++stage == kTcStages) { stage = 0; phase ^= 1u; }
                 }
                 pos += b.nsub;
@@ -392,12 +397,10 @@ __global__ void __launch_bounds__(kTcThreads, 1)
                     const uint32_t sb = smem_u32(smem + (size_t)stage * kTcStageBytes);
 #pragma unroll
                     for (int kk = 0; kk < kTcK / 16; ++kk) {
-                        for (int mb = 0; mb < b.nmb; ++mb) {
-                            const uint64_t adesc = tc_smem_desc(sb + mb * kTcTileBytes + kk * 32);
-                            for (int sub = 0; sub < b.nsub; ++sub) {
-                                const uint64_t bdesc = tc_smem_desc(sb + (b.nmb + sub) * kTcTileBytes + kk * 32);
-                                tc_mma(acc + (uint32_t)((mb + sub) * kTcSub), adesc, bdesc, (ks | kk) ? 1u : 0u);
-                            }
+                        const uint64_t adesc = tc_smem_desc(sb + kk * 32);
+                        for (int sub = 0; sub < b.nsub; ++sub) {
+                            const uint64_t bdesc = tc_smem_desc(sb + (1 + sub) * kTcTileBytes + kk * 32);
+                            tc_mma(acc + (uint32_t)(sub * kTcSub), adesc, bdesc, (ks | kk) ? 1u : 0u);
                         }
                     }
                     tc_commit(smem_u32(&empty[stage]));       // the stage is free once these MMAs have read it
