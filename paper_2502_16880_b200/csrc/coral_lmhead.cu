@@ -26,7 +26,7 @@ inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 struct Layout {
     size_t w_gate, group_tokens, state, gate, sel, slot_of, group_count, group_offset, bucket_row, bucket_slot,
         slot_desc, union_list, union_rank, part_max, part_sum, part_val, part_id, sp_max, sp_sum, sp_val, sp_id,
-        cand_val, cand_id, tc_hg, tc_max, tc_sum, tc_val, tc_id, stage_hidden, stage_ids, stage_logprobs, total;
+        cand_val, cand_id, route_mid, tc_hg, tc_max, tc_sum, tc_val, tc_id, stage_hidden, stage_ids, stage_logprobs, total;
     size_t packed_bytes, cand_cap;
     int v, T;
     int KB, T16;                 // packed layout (see packed_chunk_offset)
@@ -92,6 +92,7 @@ Layout make_layout(const coral_lmhead_config& c) {
     L.w_gate = take(N * H * 2);
     L.group_tokens = take((size_t)c.V * 4);
     L.state = take(sizeof(DeviceState));
+    L.route_mid = take((kRouteMidBands + 4 * N) * 4);
     L.gate = take(M * N * 4);
     L.sel = take(M * kg * 4);
     L.slot_of = take(M * N * 2);
@@ -393,6 +394,7 @@ int coral_lmhead_create(coral_lmhead_handle* out, const coral_lmhead_config* cfg
         if (cudaMemcpyAsync(h->ws + h->L.w_gate, W_gate_dev, (size_t)N * cfg->H * 2, cudaMemcpyDeviceToDevice, st) !=
             cudaSuccess) { rc = CORAL_ERR_CUDA; break; }
         if (cudaMemsetAsync(h->ws + h->L.state, 0, sizeof(DeviceState), st) != cudaSuccess) { rc = CORAL_ERR_CUDA; break; }
+        if (cudaMemsetAsync(h->ws + h->L.route_mid, 0, (kRouteMidBands + 4 * (size_t)cfg->n_groups) * 4, st) != cudaSuccess) { rc = CORAL_ERR_CUDA; break; }
         if (cudaMemsetAsync(h->packed, 0, h->L.packed_bytes, st) != cudaSuccess) { rc = CORAL_ERR_CUDA; break; }
         pack_rows_kernel<<<V, 128, 0, st>>>(static_cast<const uint16_t*>(W_vocab_dev),
                                             reinterpret_cast<const int32_t*>(h->ws + h->L.group_tokens),
@@ -464,6 +466,10 @@ int coral_lmhead_draft_ex(coral_lmhead_handle h, const void* hidden_dev, int M, 
         ++launches;
     } else if (M <= kRouteFusedMaxM) {
         route_fused_kernel<<<c.N, kRouteThreads, 0, st>>>(c, forced_groups_dev, out_groups_dev, out_gate_dev);
+        ++launches;
+    } else if (M <= kRouteMidMaxM && M * c.N <= kRouteMidMaxCells && cfg.H % 32 == 0) {
+        route_mid_kernel<<<dim3((c.N + 15) / 16, (M + 7) / 8), 256, 0, st>>>(
+            c, forced_groups_dev, out_groups_dev, out_gate_dev, reinterpret_cast<unsigned*>(h->ws + h->L.route_mid));
         ++launches;
     } else {
         if (cfg.H % 32 == 0)

@@ -101,12 +101,12 @@ __global__ void __launch_bounds__(kSelectWarps * 32) select_kernel(CallView c, c
     }
 }
 
-// Groups of row m by one warp (NPER = groups per lane).  Rank selection: slot of a group = number of groups
+// Groups of row m by one warp (NPER = groups per lane); bit `bit` of s_rowmask[n] is set for every selected group n.  Rank selection: slot of a group = number of groups
 // that beat it (higher score, or equal score and lower index).  Forced groups take their listed order.
 template <int NPER>
 __device__ __forceinline__ void route_select_row(const CallView& c, const int32_t* __restrict__ forced,
                                                  int32_t* __restrict__ groups_tap, int m, int lane, float* s_val,
-                                                 int16_t* s_slot_row, unsigned* s_rowmask) {
+                                                 int16_t* s_slot_row, unsigned* s_rowmask, int bit) {
     int slot[NPER];
 #pragma unroll
     for (int i = 0; i < NPER; ++i) slot[i] = -1;
@@ -155,7 +155,7 @@ __device__ __forceinline__ void route_select_row(const CallView& c, const int32_
             s_slot_row[n] = (int16_t)slot[i];
             c.slot_of[(size_t)m * c.N + n] = (int16_t)slot[i];
             if (slot[i] >= 0) {
-                atomicOr(&s_rowmask[n], 1u << m);
+                atomicOr(&s_rowmask[n], 1u << bit);
                 c.sel[(size_t)m * c.k_groups + slot[i]] = n;
                 if (groups_tap) groups_tap[(size_t)m * c.k_groups + slot[i]] = n;
             }
@@ -234,10 +234,10 @@ __global__ void __launch_bounds__(kRouteThreads)
 
     // groups of every row: one warp per row
     for (int m = warp; m < c.M; m += kWarps) {
-        if (c.N <= 32) route_select_row<1>(c, forced, groups_tap, m, lane, s_val[warp], s_slot[m], s_rowmask);
-        else if (c.N <= 64) route_select_row<2>(c, forced, groups_tap, m, lane, s_val[warp], s_slot[m], s_rowmask);
-        else if (c.N <= 128) route_select_row<4>(c, forced, groups_tap, m, lane, s_val[warp], s_slot[m], s_rowmask);
-        else route_select_row<8>(c, forced, groups_tap, m, lane, s_val[warp], s_slot[m], s_rowmask);
+        if (c.N <= 32) route_select_row<1>(c, forced, groups_tap, m, lane, s_val[warp], s_slot[m], s_rowmask, m);
+        else if (c.N <= 64) route_select_row<2>(c, forced, groups_tap, m, lane, s_val[warp], s_slot[m], s_rowmask, m);
+        else if (c.N <= 128) route_select_row<4>(c, forced, groups_tap, m, lane, s_val[warp], s_slot[m], s_rowmask, m);
+        else route_select_row<8>(c, forced, groups_tap, m, lane, s_val[warp], s_slot[m], s_rowmask, m);
     }
     __syncthreads();
 
@@ -354,13 +354,10 @@ __global__ void __launch_bounds__(256) gate_tile_kernel(CallView c, float* __res
 // Every lane loads 16 bytes of two gate rows and of one hidden row per block of 32 columns; the column order
 // inside a block is permuted the same way for both operands, which leaves the dot products unchanged.
 // grid (ceil(N/16), ceil(M/8)), H a multiple of 32.  Block (0,0) also clears the per-group row counters.
-__global__ void __launch_bounds__(256) gate_mma_kernel(CallView c, float* __restrict__ gate_tap) {
-    __shared__ float s_part[8][16 * 8];
-    const int n0 = blockIdx.x * 16, m0 = blockIdx.y * 8;
+__device__ __forceinline__ void gate_mma_tile(const CallView& c, float* __restrict__ gate_tap, int n0, int m0,
+                                              float (*s_part)[16 * 8]) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int gq = lane >> 2, tq = lane & 3;
-    if (blockIdx.x == 0 && blockIdx.y == 0)
-        for (int n = threadIdx.x; n < c.N; n += 256) c.group_count[n] = 0;
     const bool a_lo = n0 + gq < c.N, a_hi = n0 + gq + 8 < c.N, b_ok = m0 + gq < c.M;
     const uint16_t* wlo = c.w_gate + (size_t)(a_lo ? n0 + gq : 0) * c.H + tq * 8;
     const uint16_t* whi = c.w_gate + (size_t)(a_hi ? n0 + gq + 8 : 0) * c.H + tq * 8;
@@ -396,6 +393,135 @@ __global__ void __launch_bounds__(256) gate_mma_kernel(CallView c, float* __rest
             c.gate[(size_t)(m0 + r) * c.N + n0 + g] = sum;
             if (gate_tap) gate_tap[(size_t)(m0 + r) * c.N + n0 + g] = sum;
         }
+    }
+}
+
+__global__ void __launch_bounds__(256) gate_mma_kernel(CallView c, float* __restrict__ gate_tap) {
+    __shared__ float s_part[8][16 * 8];
+    if (blockIdx.x == 0 && blockIdx.y == 0)
+        for (int n = threadIdx.x; n < c.N; n += 256) c.group_count[n] = 0;
+    gate_mma_tile(c, gate_tap, blockIdx.x * 16, blockIdx.y * 8, s_part);
+}
+
+// Router stage in one launch for a medium number of rows (kRouteFusedMaxM < M <= kRouteMidMaxM, M * N <=
+// kRouteMidMaxCells, H a multiple of 32).  grid (ceil(N/16), ceil(M/8)) as gate_mma_kernel.  Nobody waits for
+// anybody: the blocks of one 8-row band draw tickets from the band's counter and the last one selects the
+// groups of the band's rows (one warp per row) and ORs them into per-group row masks in global memory; these
+// band-finishers draw a second ticket and the last of them buckets the rows by group (one thread per group)
+// and writes the union list and the merge descriptors.  `scratch`: kRouteMidBands band counters, then four
+// mask words per group; all zero between calls (the last block clears what it used).
+constexpr int kRouteMidMaxM = 128;
+constexpr int kRouteMidBands = kRouteMidMaxM / 8;
+constexpr int kRouteMidMaxCells = 8192;       // M * N slots staged in shared memory by the last block
+__global__ void __launch_bounds__(256)
+    route_mid_kernel(CallView c, const int32_t* __restrict__ forced, int32_t* __restrict__ groups_tap,
+                     float* __restrict__ gate_tap, unsigned* __restrict__ scratch) {
+    __shared__ float s_part[8][16 * 8];
+    __shared__ float s_val[8][kMaxGroups];
+    __shared__ int16_t s_slot_row[8][kMaxGroups];
+    __shared__ unsigned s_mask[kMaxGroups];
+    __shared__ int16_t s_slot[kRouteMidMaxCells];
+    __shared__ int s_warp_tot[8];
+    __shared__ int s_flag;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int m0 = blockIdx.y * 8;
+    unsigned* band_ticket = scratch;
+    unsigned* rowmask = scratch + kRouteMidBands;
+    pdl_launch_dependents();      // the next kernel may set itself up; it waits for this grid before reading
+
+    gate_mma_tile(c, gate_tap, blockIdx.x * 16, m0, s_part);
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        const unsigned t = atomicAdd(&band_ticket[blockIdx.y], 1u);
+        s_flag = t == gridDim.x - 1;
+        if (s_flag) band_ticket[blockIdx.y] = 0;
+        __threadfence();
+    }
+    s_mask[threadIdx.x] = 0;                        // 256 threads == kMaxGroups
+    __syncthreads();
+    if (!s_flag) return;
+
+    // this block saw the band's last ticket: every score of rows m0 .. m0 + 7 is published
+    {
+        const int m = m0 + warp;
+        if (m < c.M) {
+            if (c.N <= 32) route_select_row<1>(c, forced, groups_tap, m, lane, s_val[warp], s_slot_row[warp], s_mask, warp);
+            else if (c.N <= 64) route_select_row<2>(c, forced, groups_tap, m, lane, s_val[warp], s_slot_row[warp], s_mask, warp);
+            else if (c.N <= 128) route_select_row<4>(c, forced, groups_tap, m, lane, s_val[warp], s_slot_row[warp], s_mask, warp);
+            else route_select_row<8>(c, forced, groups_tap, m, lane, s_val[warp], s_slot_row[warp], s_mask, warp);
+        }
+    }
+    __syncthreads();
+    if (threadIdx.x < c.N && s_mask[threadIdx.x])
+        atomicOr(&rowmask[threadIdx.x * 4 + (m0 >> 5)], s_mask[threadIdx.x] << (m0 & 31));
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        const int t = atomicAdd(&c.state->ticket, 1);
+        s_flag = t == (int)gridDim.y - 1;
+        if (s_flag) c.state->ticket = 0;
+        __threadfence();
+    }
+    __syncthreads();
+    if (!s_flag) return;
+
+    // last band-finisher: every row's selection is published.  Stage the slots, then one thread per group.
+    for (int i = threadIdx.x; i < c.M * c.N; i += 256) s_slot[i] = __ldcg(c.slot_of + i);
+    const int n = threadIdx.x;
+    unsigned mask[4] = {0u, 0u, 0u, 0u};
+    if (n < c.N) {
+#pragma unroll
+        for (int w = 0; w < 4; ++w) {
+            mask[w] = __ldcg(rowmask + n * 4 + w);
+            rowmask[n * 4 + w] = 0;                 // ready for the next call
+        }
+    }
+    const int cnt = __popc(mask[0]) + __popc(mask[1]) + __popc(mask[2]) + __popc(mask[3]);
+    const int passes = cnt == 0 ? 0 : (c.pass_rows > 0 ? (cnt + c.pass_rows - 1) / c.pass_rows : 1);
+    const int packed = cnt | (passes << 16);
+    int incl = packed;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int a = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += a;
+    }
+    if (lane == 31) s_warp_tot[warp] = incl;
+    const int n_union = __syncthreads_count(cnt > 0);
+    int before = 0, total = 0;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) {
+        const int t = s_warp_tot[w];
+        if (w < warp) before += t;
+        total += t;
+    }
+    const int excl = before + incl - packed;
+    const int off = excl & 0xffff, virt = excl >> 16;
+    if (n < c.N) {
+        c.group_offset[n] = off;
+        c.group_count[n] = cnt;
+        c.union_rank[n] = cnt > 0 ? virt : -1;
+        for (int p = 0; p < passes; ++p)
+            if (virt + p < c.union_cap) c.union_list[virt + p] = n | (p << 16);
+        int pos = 0;
+#pragma unroll
+        for (int w = 0; w < 4; ++w) {
+            unsigned left = mask[w];
+            for (; left; ++pos) {
+                const int m = w * 32 + __ffs(left) - 1;
+                left &= left - 1;
+                const int sl = s_slot[m * c.N + n];
+                c.bucket_row[off + pos] = m;
+                c.bucket_slot[off + pos] = sl;
+                const int pass = c.pass_rows > 0 ? pos / c.pass_rows : 0;
+                c.slot_desc[(size_t)m * c.k_groups + sl] = ((virt + pass) << 8) | ((pos - pass * max(c.pass_rows, 1)) & 255);
+            }
+        }
+    }
+    if (threadIdx.x == 0) {
+        c.group_offset[c.N] = total & 0xffff;
+        c.state->n_union = n_union;
+        c.state->n_virtual = min(total >> 16, c.union_cap);
     }
 }
 
