@@ -153,6 +153,37 @@ int coral_lmhead_draft_host(coral_lmhead_handle h, const void *hidden_host, int 
                             int32_t *out_ids_host, float *out_logprobs_host, void *stream);
 
 /*
+ * Vocab sharding over several GPUs (one exchange step).  Appendix B's union of groups is what a call must
+ * read; with `world` GPUs, GPU `rank` reads only the groups n with n % world == rank (Section 3.3's N equal
+ * groups dealt round-robin), so the weight bytes per GPU fall about `world`-fold.  Every GPU runs the router
+ * on all N scores (the gate matrix is small), computes logits for its own groups among each row's top-n,
+ * and coral_lmhead_draft_partial writes one record per row; the records of all GPUs are gathered (one
+ * all-gather of M x (2 + 2 k_tokens) words per GPU, the caller's collective) and
+ * coral_lmhead_merge_partials turns them into the same output coral_lmhead_draft gives on one GPU.
+ *
+ * coral_lmhead_set_group_shard: rank in [0, world), world in [1, n_groups]; world = 1 (the default) switches
+ * sharding off.  While world > 1 the handle accepts only coral_lmhead_draft_partial (a shard alone cannot
+ * normalise a row): the other draft calls return CORAL_ERR_INVALID.  The handle still holds the full packed
+ * head; sharding reduces what is read per call, not what is stored.
+ *
+ * coral_lmhead_draft_partial: arguments as coral_lmhead_draft; out_records_dev is [M][2 + 2 k_tokens] 32-bit
+ * words, per row: max of this GPU's active logits (float; -inf if none of the row's groups is local), sum of
+ * exp(logit - max) (float), the k_tokens largest logits in descending order (float; -inf where absent), their
+ * global token ids (int32; 0x7fffffff where absent).  Joint output mode only; not on the plain fallback path
+ * (CORAL_ERR_INVALID).  Asynchronous on `stream`, no allocation.
+ *
+ * coral_lmhead_merge_partials: records_dev is [world][M][2 + 2 k_tokens] words (rank-major, as an all-gather
+ * leaves them); writes out_ids_dev / out_logprobs_dev [M x k_tokens] exactly as coral_lmhead_draft defines
+ * them (log-softmax over the union of all ranks' active logits, descending, equal -> lower token id).  Needs
+ * no handle.  world * k_tokens <= 256, else CORAL_ERR_TOO_LARGE.
+ */
+int coral_lmhead_set_group_shard(coral_lmhead_handle h, int rank, int world);
+int coral_lmhead_draft_partial(coral_lmhead_handle h, const void *hidden_dev, int M, int k_groups, int k_tokens,
+                               void *out_records_dev, void *stream);
+int coral_lmhead_merge_partials(const void *records_dev, int world, int M, int k_tokens, int32_t *out_ids_dev,
+                                float *out_logprobs_dev, void *stream);
+
+/*
  * Output mode of later draft calls.  CORAL_OUTPUT_FACTORISED emits the paper's final distribution (Section
  * 3.3, Eq. 8): p(x) = p_router(n) * p_group(x^n), where p_router is the softmax of the row's N router scores
  * (Eq. 7) and p_group the softmax inside group n, independent of the other groups; candidates are ranked by

@@ -25,6 +25,7 @@ struct CallView {
     int k_groups, k_tokens;
     int union_cap;                 // capacity of union_list
     int pass_rows;                 // rows of a group handled per pass over its weights (0: one pass for any count)
+    int shard_rank, shard_world;   // vocab sharding: this call computes only the groups n with n % shard_world == shard_rank
     const uint16_t* packed;        // blocked copy of W_vocab, see packed_chunk_offset
     int KB, T16;                   // packed layout: 64-column blocks per row, 16-row items per group
     const uint16_t* w_gate;        // [N][H] bf16
@@ -110,5 +111,10 @@ __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;"
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
 __device__ __forceinline__ void set_status(DeviceState* st, int code) { atomicCAS(&st->status, 0, code); }
+
+// Vocab sharding over several GPUs: group n belongs to the GPU with rank n % world.
+__device__ __forceinline__ bool group_is_local(const CallView& c, int n) {
+    return c.shard_world <= 1 || n % c.shard_world == c.shard_rank;
+}
 
 }  // namespace coral

@@ -159,6 +159,7 @@ struct coral_lmhead_s {
     int stream_smem;     // 0 if the streaming path is not available for this shape/device
     bool tc_ok;          // tensor-core path available (maps encoded)
     int out_mode;        // CORAL_OUTPUT_*
+    int shard_rank, shard_world;   // vocab sharding (coral_lmhead_set_group_shard); world 1 = off
     uint16_t* w1;        // [H][H] bf16 first router layer (Eq. 7), library-owned, or null
     float* router_u;     // [max_M][H] fp32 act(W1 h) + h, library-owned
     CUtensorMap map_w, map_h;
@@ -195,6 +196,8 @@ CallView make_view(const coral_lmhead_s* h, const void* hidden, int M, int kg, i
     c.union_list = reinterpret_cast<int32_t*>(ws + L.union_list);
     c.union_rank = reinterpret_cast<int32_t*>(ws + L.union_rank);
     c.union_cap = h->cfg.n_groups * kStreamMaxPasses;
+    c.shard_rank = h->shard_rank;
+    c.shard_world = h->shard_world;
     c.part_max = reinterpret_cast<float*>(ws + L.part_max);
     c.part_sum = reinterpret_cast<float*>(ws + L.part_sum);
     c.part_val = reinterpret_cast<float*>(ws + L.part_val);
@@ -346,6 +349,8 @@ int coral_lmhead_create(coral_lmhead_handle* out, const coral_lmhead_config* cfg
     h->cfg = *cfg;
     h->L = make_layout(*cfg);
     h->forced_path = CORAL_PATH_AUTO;
+    h->shard_rank = 0;
+    h->shard_world = 1;
     h->packed = static_cast<unsigned char*>(packed_buf_dev);
     h->ws = static_cast<unsigned char*>(workspace_dev);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -430,11 +435,15 @@ int coral_lmhead_set_path(coral_lmhead_handle h, int path) {
     return CORAL_OK;
 }
 
-int coral_lmhead_draft_ex(coral_lmhead_handle h, const void* hidden_dev, int M, int k_groups, int k_tokens,
-                          const int32_t* forced_groups_dev, int32_t* out_groups_dev, float* out_gate_dev,
-                          float* out_logits_dev, float* out_lse_dev, int32_t* out_ids_dev, float* out_logprobs_dev,
-                          void* stream) {
-    if (!h || !hidden_dev || !out_ids_dev || !out_logprobs_dev) return CORAL_ERR_INVALID;
+// The draft step.  partial_dev != null: vocab-sharded call, the merge writes per-row records there instead of
+// out_ids / out_logprobs (which may then be null).
+static int draft_impl(coral_lmhead_handle h, const void* hidden_dev, int M, int k_groups, int k_tokens,
+                      const int32_t* forced_groups_dev, int32_t* out_groups_dev, float* out_gate_dev,
+                      float* out_logits_dev, float* out_lse_dev, int32_t* out_ids_dev, float* out_logprobs_dev,
+                      float* partial_dev, void* stream) {
+    if (!h || !hidden_dev) return CORAL_ERR_INVALID;
+    if (!partial_dev && (!out_ids_dev || !out_logprobs_dev)) return CORAL_ERR_INVALID;
+    if (!partial_dev && h->shard_world > 1) return CORAL_ERR_INVALID;   // a shard alone cannot normalise a row
     if (reinterpret_cast<uintptr_t>(hidden_dev) & 15) return CORAL_ERR_INVALID;
     const coral_lmhead_config& cfg = h->cfg;
     if (M < 1 || M > cfg.max_M) return CORAL_ERR_INVALID;
@@ -446,6 +455,9 @@ int coral_lmhead_draft_ex(coral_lmhead_handle h, const void* hidden_dev, int M, 
     const int path = choose_path(h, M, k_groups);
     if (path == 0) return CORAL_ERR_INVALID;   // the forced path does not support this call
     if (h->out_mode == CORAL_OUTPUT_FACTORISED && path == CORAL_PATH_SIMT_PLAIN) return CORAL_ERR_INVALID;
+    if (partial_dev && (path == CORAL_PATH_SIMT_PLAIN || h->out_mode != CORAL_OUTPUT_JOINT)) return CORAL_ERR_INVALID;
+    const int merge_mode = partial_dev ? kMergePartial : h->out_mode == CORAL_OUTPUT_FACTORISED ? kMergeFactorised : kMergeJoint;
+    float* merge_out = partial_dev ? partial_dev : out_logprobs_dev;
     c.pass_rows = path == CORAL_PATH_STREAM ? kStreamPassRows : path == CORAL_PATH_TCGEN05 ? kTcPassRows : 0;
     if (path == CORAL_PATH_TCGEN05) c.union_cap = h->L.tc_vcap;
     int launches = 0;
@@ -500,8 +512,8 @@ int coral_lmhead_draft_ex(coral_lmhead_handle h, const void* hidden_dev, int M, 
             const int c_cap = p_cap * k_tokens < kMergeSmemCands ? p_cap * k_tokens : kMergeSmemCands;
             launch_pdl(merge_stream_kernel, dim3(M), dim3(kMergeStreamThreads), merge_smem_bytes(p_cap, c_cap), st, c,
                        h->sg, pp, reinterpret_cast<float*>(h->ws + L.cand_val),
-                       reinterpret_cast<int32_t*>(h->ws + L.cand_id), (int)L.cand_cap, c_cap, p_cap,
-                       (int)(h->out_mode == CORAL_OUTPUT_FACTORISED), out_ids_dev, out_logprobs_dev, out_lse_dev);
+                       reinterpret_cast<int32_t*>(h->ws + L.cand_id), (int)L.cand_cap, c_cap, p_cap, merge_mode,
+                       out_ids_dev, merge_out, out_lse_dev);
         }
         ++launches;
     } else if (path == CORAL_PATH_TCGEN05) {
@@ -524,8 +536,7 @@ int coral_lmhead_draft_ex(coral_lmhead_handle h, const void* hidden_dev, int M, 
             const int c_cap = p_cap * k_tokens;          // tc_usable() keeps this within kMergeSmemCands
             launch_pdl(merge_stream_kernel, dim3(M), dim3(kMergeStreamThreads), merge_smem_bytes(p_cap, c_cap), st, c, mg,
                        pp, reinterpret_cast<float*>(h->ws + L.cand_val), reinterpret_cast<int32_t*>(h->ws + L.cand_id),
-                       (int)L.cand_cap, c_cap, p_cap, (int)(h->out_mode == CORAL_OUTPUT_FACTORISED), out_ids_dev,
-                       out_logprobs_dev, out_lse_dev);
+                       (int)L.cand_cap, c_cap, p_cap, merge_mode, out_ids_dev, merge_out, out_lse_dev);
         }
         ++launches;
     } else {
@@ -540,6 +551,38 @@ int coral_lmhead_draft_ex(coral_lmhead_handle h, const void* hidden_dev, int M, 
 
     h->last_path = path; h->last_M = M; h->last_kg = k_groups; h->last_kt = k_tokens; h->last_launches = launches;
     return CORAL_OK;
+}
+
+int coral_lmhead_draft_ex(coral_lmhead_handle h, const void* hidden_dev, int M, int k_groups, int k_tokens,
+                          const int32_t* forced_groups_dev, int32_t* out_groups_dev, float* out_gate_dev,
+                          float* out_logits_dev, float* out_lse_dev, int32_t* out_ids_dev, float* out_logprobs_dev,
+                          void* stream) {
+    return draft_impl(h, hidden_dev, M, k_groups, k_tokens, forced_groups_dev, out_groups_dev, out_gate_dev,
+                      out_logits_dev, out_lse_dev, out_ids_dev, out_logprobs_dev, nullptr, stream);
+}
+
+int coral_lmhead_set_group_shard(coral_lmhead_handle h, int rank, int world) {
+    if (!h || world < 1 || rank < 0 || rank >= world || world > h->cfg.n_groups) return CORAL_ERR_INVALID;
+    h->shard_rank = rank;
+    h->shard_world = world;
+    return CORAL_OK;
+}
+
+int coral_lmhead_draft_partial(coral_lmhead_handle h, const void* hidden_dev, int M, int k_groups, int k_tokens,
+                               void* out_records_dev, void* stream) {
+    if (!out_records_dev) return CORAL_ERR_INVALID;
+    return draft_impl(h, hidden_dev, M, k_groups, k_tokens, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr,
+                      nullptr, static_cast<float*>(out_records_dev), stream);
+}
+
+int coral_lmhead_merge_partials(const void* records_dev, int world, int M, int k_tokens, int32_t* out_ids_dev,
+                                float* out_logprobs_dev, void* stream) {
+    if (!records_dev || !out_ids_dev || !out_logprobs_dev) return CORAL_ERR_INVALID;
+    if (world < 1 || M < 1 || k_tokens < 1 || k_tokens > CORAL_MAX_K_TOKENS) return CORAL_ERR_INVALID;
+    if (world * k_tokens > kMergePartialsThreads) return CORAL_ERR_TOO_LARGE;
+    merge_partials_kernel<<<M, kMergePartialsThreads, 0, static_cast<cudaStream_t>(stream)>>>(
+        static_cast<const float*>(records_dev), world, M, k_tokens, out_ids_dev, out_logprobs_dev);
+    return cudaGetLastError() == cudaSuccess ? CORAL_OK : CORAL_ERR_CUDA;
 }
 
 int coral_lmhead_draft(coral_lmhead_handle h, const void* hidden_dev, int M, int k_groups, int k_tokens,

@@ -400,13 +400,18 @@ __global__ void __launch_bounds__(kStreamThreads, 1) head_stream_kernel(CallView
 // factorised (CORAL Eq. 8, p(x) = p_router(n) p_group(x)) adds log p_router(n) - LSE_group(n), a per-slot
 // offset, where p_router is the softmax of the row's N gate scores (Eq. 7).  Adding a per-slot constant
 // keeps every piece's list sorted, so both modes share the selection code.
+// Partial mode (vocab sharding over several GPUs): the row's record of 2 + 2 k_tokens words - max, sum of
+// exp(z - max), the k_tokens best raw logits (descending), their token ids - over the groups this GPU
+// computed, written to `out_logprobs` (as a [M][2 + 2 k_tokens] word array); slots whose group belongs to
+// another GPU have descriptor -1 and no pieces.  merge_partials_kernel combines the GPUs' records.
+constexpr int kMergeJoint = 0, kMergeFactorised = 1, kMergePartial = 2;
 constexpr int kMergeStreamThreads = 256;
 constexpr int kMergeMaxPieces = 1024;         // >= grid + 2 * k_groups for every supported shape
 constexpr int kMergeRankMax = 256;            // survivors ranked by counting; more fall back to k rounds
 __global__ void __launch_bounds__(kMergeStreamThreads) merge_stream_kernel(CallView c, StreamGeom g, StreamPartials pp,
                                                                            float* __restrict__ cand_val_scratch,
                                                                            int32_t* __restrict__ cand_id_scratch,
-                                                                           int cand_cap, int smem_cands, int p_cap, int factorised,
+                                                                           int cand_cap, int smem_cands, int p_cap, int mode,
                                                                            int32_t* __restrict__ out_ids,
                                                                            float* __restrict__ out_logprobs,
                                                                            float* __restrict__ lse_tap) {
@@ -414,6 +419,8 @@ __global__ void __launch_bounds__(kMergeStreamThreads) merge_stream_kernel(CallV
     const int m = blockIdx.x;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     constexpr int kWarps = kMergeStreamThreads / 32;
+    const bool factorised = mode == kMergeFactorised, partial = mode == kMergePartial;
+    float* rec = partial ? out_logprobs + (size_t)m * (2 + 2 * c.k_tokens) : nullptr;
     __shared__ float s_f[kWarps], s_t[kWarps];
     __shared__ float s_lse, s_glse, s_thr2;
     __shared__ int s_n;
@@ -432,11 +439,11 @@ __global__ void __launch_bounds__(kMergeStreamThreads) merge_stream_kernel(CallV
     const int per = max(1, (n_items + g.grid - 1) / g.grid);
     for (int s = threadIdx.x; s < c.k_groups; s += kMergeStreamThreads) {
         const int desc = c.slot_desc[(size_t)m * c.k_groups + s];
-        const int j = desc >> 8;
+        const int j = desc < 0 ? 0 : desc >> 8;
         const int fb = g.tc_tiles > 0 ? j * g.tc_tiles : (j * g.T) / per;
         const int lb = g.tc_tiles > 0 ? fb + g.tc_tiles - 1 : ((j + 1) * g.T - 1) / per;
         s_first[s] = fb;
-        s_base[s] = lb - fb + 1;       // piece count, turned into an exclusive prefix below
+        s_base[s] = desc < 0 ? 0 : lb - fb + 1;       // piece count, turned into an exclusive prefix below
         s_j[s] = j;
         s_rpos[s] = desc & 255;
         s_off[s] = factorised ? c.gate[(size_t)m * c.N + c.sel[(size_t)m * c.k_groups + s]] : 0.f;
@@ -468,6 +475,16 @@ __global__ void __launch_bounds__(kMergeStreamThreads) merge_stream_kernel(CallV
     }
     __syncthreads();
     const int P = min(s_base[c.k_groups], p_cap);
+    if (partial) {                 // defaults; a row none of whose groups is computed here keeps them
+        if (threadIdx.x < c.k_tokens) {
+            rec[2 + threadIdx.x] = kNegInf;
+            reinterpret_cast<int32_t*>(rec)[2 + c.k_tokens + threadIdx.x] = kNoToken;
+        }
+        if (P == 0) {
+            if (threadIdx.x == 0) { rec[0] = kNegInf; rec[1] = 0.f; }
+            return;
+        }
+    }
     for (int q = threadIdx.x; q < P; q += kMergeStreamThreads) {
         int s = 0;
         while (s + 1 < c.k_groups && s_base[s + 1] <= q) ++s;
@@ -511,6 +528,7 @@ __global__ void __launch_bounds__(kMergeStreamThreads) merge_stream_kernel(CallV
         for (int w = 0; w < kWarps; ++w) tot += s_t[w];
         s_lse = mx + logf(tot);
         if (lse_tap) lse_tap[m] = s_lse;
+        if (partial) { rec[0] = mx; rec[1] = tot; }
     }
     __syncthreads();
     // per-slot offsets
@@ -522,7 +540,7 @@ __global__ void __launch_bounds__(kMergeStreamThreads) merge_stream_kernel(CallV
             for (int q = s_base[s]; q < min(s_base[s + 1], P); ++q) ss += s_ps[q] * expf(s_pm[q] - sm);
             s_off[s] = (s_off[s] - s_glse) - (sm + logf(ss));
         } else {
-            s_off[s] = -s_lse;
+            s_off[s] = partial ? 0.f : -s_lse;
         }
     }
     __syncthreads();
@@ -588,8 +606,13 @@ __global__ void __launch_bounds__(kMergeStreamThreads) merge_stream_kernel(CallV
             int rank = 0;
             for (int i = 0; i < S; ++i) rank += better(cv[i], ci[i], v, id) ? 1 : 0;
             if (rank < c.k_tokens) {
-                out_ids[(size_t)m * c.k_tokens + rank] = id;
-                out_logprobs[(size_t)m * c.k_tokens + rank] = v;
+                if (partial) {
+                    rec[2 + rank] = v;
+                    reinterpret_cast<int32_t*>(rec)[2 + c.k_tokens + rank] = id;
+                } else {
+                    out_ids[(size_t)m * c.k_tokens + rank] = id;
+                    out_logprobs[(size_t)m * c.k_tokens + rank] = v;
+                }
             }
         }
         return;
@@ -616,11 +639,59 @@ __global__ void __launch_bounds__(kMergeStreamThreads) merge_stream_kernel(CallV
         for (int w = 1; w < kWarps; ++w)
             if (better(s_f[w], s_i[w], bv, bk)) { bv = s_f[w]; bk = s_i[w]; }
         if (threadIdx.x == 0) {
-            out_ids[(size_t)m * c.k_tokens + k] = bk;
-            out_logprobs[(size_t)m * c.k_tokens + k] = bv;
+            if (partial) {
+                rec[2 + k] = bv;
+                reinterpret_cast<int32_t*>(rec)[2 + c.k_tokens + k] = bk;
+            } else {
+                out_ids[(size_t)m * c.k_tokens + k] = bk;
+                out_logprobs[(size_t)m * c.k_tokens + k] = bv;
+            }
         }
         last_v = bv;
         last_id = bk;
+    }
+}
+
+// Combines the records that `world` GPUs wrote in partial mode (records[r][m] = record of row m from rank r,
+// 2 + 2 k_tokens words each): joint log-sum-exp over all ranks' active logits and the k_tokens best tokens
+// of the row, emitted like the single-GPU merge (log-probabilities, descending, equal -> lower token id).
+// grid M, block kMergePartialsThreads >= world * k_tokens.
+constexpr int kMergePartialsThreads = 256;
+__global__ void __launch_bounds__(kMergePartialsThreads)
+    merge_partials_kernel(const float* __restrict__ records, int world, int M, int k_tokens,
+                          int32_t* __restrict__ out_ids, float* __restrict__ out_logprobs) {
+    __shared__ float s_v[kMergePartialsThreads];
+    __shared__ int s_id[kMergePartialsThreads];
+    __shared__ float s_lse;
+    const int m = blockIdx.x;
+    const int W = 2 + 2 * k_tokens;
+    const int C = world * k_tokens;
+    if (threadIdx.x == 0) {
+        float mx = kNegInf;
+        for (int r = 0; r < world; ++r) mx = fmaxf(mx, records[((size_t)r * M + m) * W]);
+        float tot = 0.f;
+        for (int r = 0; r < world; ++r) {
+            const float* rec = records + ((size_t)r * M + m) * W;
+            if (rec[0] != kNegInf) tot += rec[1] * expf(rec[0] - mx);
+        }
+        s_lse = mx + logf(tot);
+    }
+    if (threadIdx.x < C) {
+        const int r = threadIdx.x / k_tokens, i = threadIdx.x - r * k_tokens;
+        const float* rec = records + ((size_t)r * M + m) * W;
+        s_v[threadIdx.x] = rec[2 + i];
+        s_id[threadIdx.x] = reinterpret_cast<const int32_t*>(rec)[2 + k_tokens + i];
+    }
+    __syncthreads();
+    if (threadIdx.x < C) {
+        const float v = s_v[threadIdx.x];
+        const int id = s_id[threadIdx.x];
+        int rank = 0;
+        for (int i = 0; i < C; ++i) rank += better(s_v[i], s_id[i], v, id) ? 1 : 0;
+        if (rank < k_tokens) {
+            out_ids[(size_t)m * k_tokens + rank] = id;
+            out_logprobs[(size_t)m * k_tokens + rank] = v - s_lse;
+        }
     }
 }
 

@@ -137,6 +137,7 @@ __device__ __forceinline__ void tc_ld32(uint32_t taddr, float (&v)[32]) {
 // whatever they held (their accumulator lanes are never read).
 __global__ void __launch_bounds__(128) tc_gather_kernel(CallView c, uint16_t* __restrict__ hg) {
     const int p = blockIdx.x;
+    if (p >= c.group_offset[c.N]) return;          // fewer pairs than M * k_groups when the vocab is sharded
     const int m = c.bucket_row[p];
     const int n = c.sel[(size_t)m * c.k_groups + c.bucket_slot[p]];
     const int rg = p - c.group_offset[n];

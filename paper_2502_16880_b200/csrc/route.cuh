@@ -91,6 +91,7 @@ __global__ void __launch_bounds__(kSelectWarps * 32) select_kernel(CallView c, c
         }
         if (lane == 0) {
             c.sel[(size_t)m * c.k_groups + s] = pick;
+            if (c.shard_world > 1) c.slot_desc[(size_t)m * c.k_groups + s] = -1;   // stays -1 for another GPU's group
             if (groups_tap) groups_tap[(size_t)m * c.k_groups + s] = pick;
         }
     }
@@ -157,6 +158,7 @@ __device__ __forceinline__ void route_select_row(const CallView& c, const int32_
             if (slot[i] >= 0) {
                 atomicOr(&s_rowmask[n], 1u << bit);
                 c.sel[(size_t)m * c.k_groups + slot[i]] = n;
+                if (c.shard_world > 1) c.slot_desc[(size_t)m * c.k_groups + slot[i]] = -1;   // stays -1 for another GPU's group
                 if (groups_tap) groups_tap[(size_t)m * c.k_groups + slot[i]] = n;
             }
         }
@@ -244,7 +246,7 @@ __global__ void __launch_bounds__(kRouteThreads)
     // One thread per group: rows that selected it, passes over its weights, and (by a block-wide exclusive
     // scan of both counts, packed in one word) its place in the bucket array and in the union list.
     const int n = threadIdx.x;
-    const unsigned mask = n < c.N ? s_rowmask[n] : 0u;
+    const unsigned mask = (n < c.N && group_is_local(c, n)) ? s_rowmask[n] : 0u;
     const int cnt = __popc(mask);
     const int passes = cnt == 0 ? 0 : (c.pass_rows > 0 ? (cnt + c.pass_rows - 1) / c.pass_rows : 1);
     const int packed = cnt | (passes << 16);
@@ -473,7 +475,7 @@ __global__ void __launch_bounds__(256)
     if (n < c.N) {
 #pragma unroll
         for (int w = 0; w < 4; ++w) {
-            mask[w] = __ldcg(rowmask + n * 4 + w);
+            mask[w] = group_is_local(c, n) ? __ldcg(rowmask + n * 4 + w) : 0u;
             rowmask[n * 4 + w] = 0;                 // ready for the next call
         }
     }
@@ -528,7 +530,7 @@ __global__ void __launch_bounds__(256)
 // select_kernel plus per-group row counts (integer atomics: the totals do not depend on their order).
 __global__ void __launch_bounds__(kSelectWarps * 32) count_groups_kernel(CallView c) {
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
-    if (i < c.M * c.k_groups) atomicAdd(&c.group_count[c.sel[i]], 1);
+    if (i < c.M * c.k_groups && group_is_local(c, c.sel[i])) atomicAdd(&c.group_count[c.sel[i]], 1);
 }
 
 // One block per group: the group's place in the bucket array and in the union list (prefix sums over the
@@ -567,7 +569,7 @@ __global__ void __launch_bounds__(256) bucket_group_kernel(CallView c) {
     int running = 0;
     for (int m0 = 0; m0 < c.M; m0 += 256) {
         const int m = m0 + threadIdx.x;
-        const int sl = m < c.M ? (int)c.slot_of[(size_t)m * c.N + n] : -1;
+        const int sl = (m < c.M && cnt > 0) ? (int)c.slot_of[(size_t)m * c.N + n] : -1;   // cnt = 0: not this GPU's group
         const unsigned bal = __ballot_sync(0xffffffffu, sl >= 0);
         if (lane == 0) s_warp[warp] = __popc(bal);
         __syncthreads();

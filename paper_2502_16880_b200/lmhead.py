@@ -53,6 +53,9 @@ _SIGNATURES = {
     "coral_lmhead_draft": (_i, [_vp, _vp, _i, _i, _i, _vp, _vp, _vp]),
     "coral_lmhead_draft_ex": (_i, [_vp, _vp, _i, _i, _i, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "coral_lmhead_draft_host": (_i, [_vp, _vp, _i, _i, _i, _vp, _vp, _vp]),
+    "coral_lmhead_set_group_shard": (_i, [_vp, _i, _i]),
+    "coral_lmhead_draft_partial": (_i, [_vp, _vp, _i, _i, _i, _vp, _vp]),
+    "coral_lmhead_merge_partials": (_i, [_vp, _i, _i, _i, _vp, _vp, _vp]),
     "coral_lmhead_set_path": (_i, [_vp, _i]),
     "coral_lmhead_set_output_mode": (_i, [_vp, _i]),
     "coral_lmhead_set_router_mlp": (_i, [_vp, _vp, _vp]),
@@ -177,6 +180,46 @@ def coral_lmhead_draft_host(handle, hidden_host, k_groups, k_tokens, out_ids_hos
         handle, ctypes.c_void_p(hidden_host.data_ptr()), M, int(k_groups), int(k_tokens),
         ctypes.c_void_p(out_ids_host.data_ptr()), ctypes.c_void_p(out_logprobs_host.data_ptr()),
         _stream_ptr(stream)), "coral_lmhead_draft_host")
+
+
+def coral_lmhead_set_group_shard(handle, rank: int, world: int) -> None:
+    _check(load_library().coral_lmhead_set_group_shard(handle, int(rank), int(world)), "coral_lmhead_set_group_shard")
+
+
+def coral_lmhead_draft_partial(handle, hidden, k_groups, k_tokens, out_records, stream=None):
+    """out_records: CUDA int32 tensor [M, 2 + 2 * k_tokens] (the per-row record of this GPU's groups)."""
+    M = hidden.shape[0]
+    if out_records.numel() != M * (2 + 2 * int(k_tokens)):
+        raise ValueError("out_records must hold M x (2 + 2 k_tokens) words")
+    _check(load_library().coral_lmhead_draft_partial(
+        handle, _dev_ptr(hidden, torch.bfloat16, False), M, int(k_groups), int(k_tokens),
+        _dev_ptr(out_records, torch.int32, False), _stream_ptr(stream)), "coral_lmhead_draft_partial")
+
+
+def coral_lmhead_merge_partials(records, k_tokens, out_ids, out_logprobs, stream=None):
+    """records: CUDA int32 tensor [world, M, 2 + 2 * k_tokens], rank-major as an all-gather leaves it."""
+    world, M = records.shape[0], records.shape[1]
+    _check(load_library().coral_lmhead_merge_partials(
+        _dev_ptr(records, torch.int32, False), world, M, int(k_tokens), _dev_ptr(out_ids, torch.int32, False),
+        _dev_ptr(out_logprobs, torch.float32, False), _stream_ptr(stream)), "coral_lmhead_merge_partials")
+
+
+def draft_vocab_sharded(handle, hidden, k_groups, k_tokens, out_ids, out_logprobs, group=None, records=None,
+                        gathered=None):
+    """One vocab-sharded draft step on this rank of `group` (torch.distributed): this GPU's record per row,
+    one all-gather of the records, the merge.  The handle must have been given this rank's shard with
+    coral_lmhead_set_group_shard.  `records` [M, W] and `gathered` [world, M, W] (W = 2 + 2 k_tokens, int32)
+    may be passed in to avoid allocating per call."""
+    import torch.distributed as dist
+    world = dist.get_world_size(group)
+    M, W = hidden.shape[0], 2 + 2 * int(k_tokens)
+    if records is None:
+        records = torch.empty((M, W), dtype=torch.int32, device=hidden.device)
+    if gathered is None:
+        gathered = torch.empty((world, M, W), dtype=torch.int32, device=hidden.device)
+    coral_lmhead_draft_partial(handle, hidden, k_groups, k_tokens, records)
+    dist.all_gather_into_tensor(gathered.view(world * M, W), records.view(M, W), group=group)   # rank-major rows
+    coral_lmhead_merge_partials(gathered, k_tokens, out_ids, out_logprobs)
 
 
 def coral_lmhead_set_output_mode(handle, mode: int) -> None:
