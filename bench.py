@@ -182,6 +182,9 @@ def main():
     ap.add_argument("--quick", action="store_true", help="headline only: skip the other M, dense and CPU legs")
     ap.add_argument("--large-m-only", type=int, default=0, metavar="M",
                     help="run only the tensor-core leg with M rows (a short run for profilers) and print its line")
+    ap.add_argument("--vocab-shard-only", type=int, default=0, metavar="M",
+                    help="run only the vocab-sharded step with M rows: every rank reads its own groups, one all-gather "
+                         "of the per-row records, merge (strong scaling: all ranks draft for the same rows)")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
@@ -230,6 +233,54 @@ def main():
         print(json.dumps({"large_m_only": Mb, "path": int(st.path), "us_per_step": float(np.mean(ts)) * 1e3,
                           "status": big.status()}))
         big.close()
+        return
+    if args.vocab_shard_only:
+        Ms = args.vocab_shard_only
+        sh = lmhead.LMHead(Wd, torch.from_numpy(gm), dev_bf16(Wg), max_M=Ms, max_k_groups=cfg.k_groups,
+                           max_k_tokens=cfg.k_tokens)
+        lmhead.coral_lmhead_set_group_shard(sh.handle, rank, world)
+        hs = [dev_bf16(synth.make_hidden(cfg, Ms, batch=b)) for b in range(N_BATCHES)]     # same rows on every rank
+        Wrec = 2 + 2 * cfg.k_tokens
+        rec = torch.empty((Ms, Wrec), dtype=torch.int32, device=dev)
+        gathered = torch.empty((world, Ms, Wrec), dtype=torch.int32, device=dev)
+        ids_s = torch.empty((Ms, cfg.k_tokens), dtype=torch.int32, device=dev)
+        lps_s = torch.empty((Ms, cfg.k_tokens), dtype=torch.float32, device=dev)
+        flush_s = torch.empty(FLUSH_BYTES // 8, dtype=torch.int64, device=dev)
+
+        def step(i):
+            lmhead.coral_lmhead_draft_partial(sh.handle, hs[i % len(hs)], cfg.k_groups, cfg.k_tokens, rec)
+            if world > 1:
+                dist.all_gather_into_tensor(gathered.view(world * Ms, Wrec), rec)
+            else:
+                gathered[0].copy_(rec)
+            lmhead.coral_lmhead_merge_partials(gathered, cfg.k_tokens, ids_s, lps_s)
+
+        ts, touched_s = [], []
+        for i in range(max(args.warmup, 3) + args.steps):
+            flush_s.fill_(i)
+            torch.sum(flush_s)
+            if world > 1:
+                dist.barrier()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            step(i)
+            b.record()
+            torch.cuda.synchronize()
+            if i >= max(args.warmup, 3):
+                ts.append(a.elapsed_time(b))
+                touched_s.append(sh.stats().groups_touched)
+        local_ms = float(sum(ts))
+        local_bytes = float(sum(u * cfg.v * cfg.H * 2 for u in touched_s))
+        tot_ms, tot_bytes = aggregate_over_ranks(dist if world > 1 else None, local_ms, local_bytes, dev)
+        if rank == 0:
+            print(json.dumps({"vocab_shard_only": Ms, "n_gpus": world, "scaling": "strong",
+                              "us_per_step": tot_ms / args.steps * 1e3,
+                              "GBps_all_ranks": tot_bytes / (tot_ms * 1e-3) / 1e9,
+                              "groups_touched_rank0_mean": float(np.mean(touched_s)),
+                              "exchange_bytes_per_rank": Ms * Wrec * 4, "status": sh.status()}))
+        sh.close()
+        if world > 1:
+            dist.destroy_process_group()
         return
     head = lmhead.LMHead(Wd, torch.from_numpy(gm), dev_bf16(Wg), max_M=64, max_k_groups=cfg.N, max_k_tokens=cfg.k_tokens)
     flush = torch.empty(FLUSH_BYTES // 8, dtype=torch.int64, device=dev)
