@@ -283,6 +283,7 @@ def main():
             dist.destroy_process_group()
         return
     head = lmhead.LMHead(Wd, torch.from_numpy(gm), dev_bf16(Wg), max_M=64, max_k_groups=cfg.N, max_k_tokens=cfg.k_tokens)
+    default_head = head
     flush = torch.empty(FLUSH_BYTES // 8, dtype=torch.int64, device=dev)
     stream = torch.cuda.current_stream()
 
@@ -293,9 +294,10 @@ def main():
         flush.fill_(i)
         torch.sum(flush)
 
-    def time_steps(M, k_groups, steps, warmup, batches, kernel_timing=False, rho=0.0):
+    def time_steps(M, k_groups, steps, warmup, batches, kernel_timing=False, rho=0.0, zipf_s=0.0, on=None):
         """Per-step CUDA-event times (ms) with an L2 flush before every step, outside the event pair."""
-        hb_bits = [synth.make_hidden(cfg.with_(rho=rho), M, batch=b) for b in batches]
+        head = on if on is not None else default_head
+        hb_bits = [synth.make_hidden(cfg.with_(rho=rho, zipf_s=zipf_s), M, batch=b) for b in batches]
         hds = [dev_bf16(b) for b in hb_bits]
         ids = torch.empty((M, cfg.k_tokens), dtype=torch.int32, device=dev)
         lps = torch.empty((M, cfg.k_tokens), dtype=torch.float32, device=dev)
@@ -406,6 +408,21 @@ def main():
         out["correlated_rows_M60_rho0.3"] = {"us_per_step": float(np.mean(ms_c)) * 1e3,
                                              "groups_touched_mean": float(np.mean(t_c)),
                                              "GBps": b_c / (float(np.mean(ms_c)) * 1e-3) / 1e9}
+        # extra: the paper's frequency-ordered contiguous grouping (Appendix B), modelled by a contiguous group map
+        # and a Zipf-like prior on low-index groups in the gate (synth.py), against the random map above
+        zcfg = cfg.with_(zipf_s=1.5)
+        zhead = lmhead.LMHead(Wd, torch.from_numpy(synth.make_group_map(cfg, contiguous=True)),
+                              dev_bf16(synth.make_w_gate(zcfg)), max_M=64, max_k_groups=cfg.k_groups,
+                              max_k_tokens=cfg.k_tokens)
+        zleg = []
+        for M in (8, 60):
+            ms_z, _, t_z, _, _ = time_steps(M, cfg.k_groups, extra_steps, 3, my_batches, zipf_s=1.5, on=zhead)
+            b_z = float(np.mean([algorithmic_bytes(cfg.with_(M=M), u, M) for u in t_z]))
+            zleg.append({"M": M, "us_per_step": float(np.mean(ms_z)) * 1e3, "groups_touched_mean": float(np.mean(t_z)),
+                         "GBps": b_z / (float(np.mean(ms_z)) * 1e-3) / 1e9})
+        assert zhead.status() == 0
+        zhead.close()
+        out["contiguous_groups_zipf1.5"] = zleg
         # dense head on the same GPU: (i) this library with every group active, (ii) torch bf16 matmul comparator
         ms_d, _, t_d, _, _ = time_steps(cfg.M, cfg.N, extra_steps, 3, my_batches)
         dense_bytes = algorithmic_bytes(cfg, cfg.N, cfg.M)

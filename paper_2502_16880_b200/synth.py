@@ -14,6 +14,13 @@ depend on which other tensors were drawn, nor on M):
     hidden   [M, H]  fp32 N(0, 1)       -> bf16; the first M rows of one
                      stream, so the M=1 rows are a prefix of the M=8 rows ...
 
+Extra workload (not one of the graded configs): `zipf_s > 0` together with the contiguous group map
+models the paper's frequency-ordered vocabulary, where low-index groups hold the frequent tokens and are
+routed to most often.  One fixed unit direction u is drawn; W_gate[n] += -(zipf_s * ln(n + 1) / 8) * u and
+every hidden row += 8 * u before rounding, so group n's score carries a prior of about -zipf_s * ln(n + 1)
+on top of the N(0, (w_std * sqrt(H))^2) spread.  (Only sums and a rounding: the scores themselves are still
+computed by the oracle and by the library, each on its own.)
+
 The shapes are those of the draft heads in the paper's Table 1 (hidden size,
 vocabulary) with the group counts and top-n of its Table 4 grid.
 bf16 tensors are returned as numpy uint16 arrays holding the raw bit patterns.
@@ -28,6 +35,8 @@ _TAG_W_VOCAB = 1
 _TAG_W_GATE = 2
 _TAG_PERM = 3
 _TAG_HIDDEN = 4
+_TAG_PRIOR = 5
+_PRIOR_GAIN = 8.0
 
 
 @dataclass(frozen=True)
@@ -44,6 +53,7 @@ class HeadConfig:
     seed: int = 0
     w_std: float = 0.02
     rho: float = 0.0  # correlation between rows (0 = iid rows)
+    zipf_s: float = 0.0  # strength of the frequency prior on low-index groups (0 = none)
 
     @property
     def v(self) -> int:
@@ -96,8 +106,17 @@ def make_w_vocab(cfg: HeadConfig) -> np.ndarray:
     return _normal_bf16(_rng(cfg.seed, _TAG_W_VOCAB), cfg.V, cfg.H, cfg.w_std)
 
 
+def _prior_direction(cfg: HeadConfig) -> np.ndarray:
+    u = _rng(cfg.seed, _TAG_PRIOR).standard_normal(cfg.H, dtype=np.float32)
+    return u / np.float32(np.sqrt(np.sum(u.astype(np.float64) ** 2)))
+
+
 def make_w_gate(cfg: HeadConfig) -> np.ndarray:
-    return _normal_bf16(_rng(cfg.seed, _TAG_W_GATE), cfg.N, cfg.H, cfg.w_std)
+    if cfg.zipf_s <= 0.0:
+        return _normal_bf16(_rng(cfg.seed, _TAG_W_GATE), cfg.N, cfg.H, cfg.w_std)
+    w = _rng(cfg.seed, _TAG_W_GATE).standard_normal((cfg.N, cfg.H), dtype=np.float32) * np.float32(cfg.w_std)
+    b = (-cfg.zipf_s / _PRIOR_GAIN) * np.log(np.arange(1, cfg.N + 1, dtype=np.float64))
+    return fp32_to_bf16_bits(w + b.astype(np.float32)[:, None] * _prior_direction(cfg)[None, :])
 
 
 def make_group_map(cfg: HeadConfig, contiguous: bool = False) -> np.ndarray:
@@ -124,6 +143,8 @@ def make_hidden(cfg: HeadConfig, M: int | None = None, batch: int = 0) -> np.nda
         h0 = np.random.default_rng([int(cfg.seed), _TAG_HIDDEN, int(batch), 1]).standard_normal(
             (1, cfg.H), dtype=np.float32)
         x = np.float32(np.sqrt(1.0 - cfg.rho ** 2)) * h0 + np.float32(cfg.rho) * x
+    if cfg.zipf_s > 0.0:
+        x = x + np.float32(_PRIOR_GAIN) * _prior_direction(cfg)[None, :]
     return fp32_to_bf16_bits(x)
 
 

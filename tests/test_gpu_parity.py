@@ -314,3 +314,24 @@ def test_two_layer_router_eq7(M):
     rep = ph.compare(W, gm, Wg, hb, 4, 10, out)
     assert rep.ok, rep.errors
     head.close()
+
+
+@pytest.mark.parametrize("M,path", [(8, lmhead.CORAL_PATH_STREAM), (60, lmhead.CORAL_PATH_STREAM),
+                                    (60, lmhead.CORAL_PATH_SIMT_PLAIN), (200, lmhead.CORAL_PATH_TCGEN05)])
+def test_frequency_ordered_contiguous_groups(M, path):
+    """Contiguous token-id groups with a Zipf-like prior on low-index groups (the paper's frequency-ordered
+    vocabulary): a few hot groups are selected by almost every row, so they need several passes."""
+    cfg = synth.HeadConfig("zipf", H=256, V=256 * 16, N=16, k_groups=4, k_tokens=10, M=M, seed=13, w_std=0.05,
+                           zipf_s=1.5)
+    W, Wg, hb = synth.make_w_vocab(cfg), synth.make_w_gate(cfg), synth.make_hidden(cfg)
+    gm = synth.make_group_map(cfg, contiguous=True)
+    head = _head(cfg, W, gm, Wg, max_M=M, max_kg=4)
+    head.set_path(path)
+    out = ph.gpu_draft_numpy(head, hb, 4, 10)
+    assert head.status() == 0 and head.stats().path == path
+    counts = np.bincount(out["groups"].ravel(), minlength=16)
+    assert counts[:4].sum() > counts[8:].sum()            # the prior is there: low-index groups dominate
+    rows = np.unique(np.linspace(0, M - 1, 24).astype(int))
+    rep = ph.compare(W, gm, Wg, hb[rows], 4, 10, {k: a[rows] for k, a in out.items()})
+    assert rep.ok, rep.errors
+    head.close()
