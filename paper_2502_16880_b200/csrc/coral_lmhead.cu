@@ -162,7 +162,7 @@ struct coral_lmhead_s {
     int shard_rank, shard_world;   // vocab sharding (coral_lmhead_set_group_shard); world 1 = off
     uint16_t* w1;        // [H][H] bf16 first router layer (Eq. 7), library-owned, or null
     float* router_u;     // [max_M][H] fp32 act(W1 h) + h, library-owned
-    CUtensorMap map_w, map_h;
+    CUtensorMap map_w, map_h, map_h64, map_h32;   // hidden-row blocks read whole (128 rows) or only their first 64 / 32 rows
     int sms;
     cudaEvent_t ev_head0, ev_head1;   // around the weight-streaming kernel when kernel timing is on
     cudaEvent_t ev_begin, ev_end;     // before the router stage / after the merge
@@ -255,11 +255,14 @@ bool make_tc_maps(coral_lmhead_s* h) {
         return false;
     const cuuint64_t hdim[2] = {(cuuint64_t)kTcK, (cuuint64_t)L.tc_vcap * L.KB * kTcPassRows};
     const cuuint64_t hstr[1] = {(cuuint64_t)kTcK * 2};
-    const cuuint32_t hbox[2] = {(cuuint32_t)kTcK, (cuuint32_t)kTcBlockRows};
-    if (enc(&h->map_h, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, h->ws + L.tc_hg, hdim, hstr, hbox, ones,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-        return false;
+    CUtensorMap* hmaps[3] = {&h->map_h, &h->map_h64, &h->map_h32};
+    for (int i = 0; i < 3; ++i) {
+        const cuuint32_t hbox[2] = {(cuuint32_t)kTcK, (cuuint32_t)(kTcBlockRows >> i)};
+        if (enc(hmaps[i], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, h->ws + L.tc_hg, hdim, hstr, hbox, ones,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return false;
+    }
     return true;
 }
 
@@ -523,7 +526,8 @@ static int draft_impl(coral_lmhead_handle h, const void* hidden_dev, int M, int 
                       reinterpret_cast<float*>(h->ws + L.tc_val), reinterpret_cast<int32_t*>(h->ws + L.tc_id)};
         tc_gather_kernel<<<M * k_groups, 128, 0, st>>>(c, reinterpret_cast<uint16_t*>(h->ws + L.tc_hg));
         ++launches;
-        head_tc_kernel<<<tg.grid, kTcThreads, kTcSmemBytes, st>>>(c, tg, tp, h->map_w, h->map_h, out_logits_dev);
+        head_tc_kernel<<<tg.grid, kTcThreads, kTcSmemBytes, st>>>(c, tg, tp, h->map_w, h->map_h, h->map_h64, h->map_h32,
+                                                                 out_logits_dev);
         ++launches;
         if (h->timing) cudaEventRecord(h->ev_head1, st);
         StreamGeom mg = h->sg;

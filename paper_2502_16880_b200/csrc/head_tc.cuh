@@ -316,7 +316,8 @@ __device__ __forceinline__ void tc_epilogue(const CallView& c, const TcGeom& g, 
 // grid = g.grid CTAs of kTcThreads threads; dynamic shared memory: 1 KiB alignment slack + kTcStages stages + barriers.
 __global__ void __launch_bounds__(kTcThreads, 1)
     head_tc_kernel(CallView c, TcGeom g, TcPartials pp, const __grid_constant__ CUtensorMap map_w,
-                   const __grid_constant__ CUtensorMap map_h, float* __restrict__ logits_tap) {
+                   const __grid_constant__ CUtensorMap map_h, const __grid_constant__ CUtensorMap map_h64,
+                   const __grid_constant__ CUtensorMap map_h32, float* __restrict__ logits_tap) {
     extern __shared__ unsigned char tc_smem_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(tc_smem_raw) + 1023) & ~(uintptr_t)1023);
     float* zstash = reinterpret_cast<float*>(smem + kTcStages * kTcStageBytes);          // [32][epilogue threads]
@@ -365,7 +366,11 @@ __global__ void __launch_bounds__(kTcThreads, 1)
                            pol_last = l2_policy_evict_last();
             for (int pos = lo; pos < hi;) {
                 const TcBatch b = tc_batch_at(c, g, pos, hi);
-                const uint32_t bytes = (uint32_t)(1 + b.nsub) * kTcTileBytes;
+                // a pass with few rows fetches only the first 64 or 32 rows of its block of hidden rows; the MMA
+                // still spans 128 rows, whose remaining accumulator lanes hold leftovers nobody reads
+                const CUtensorMap* mh = b.R <= 32 ? &map_h32 : b.R <= 64 ? &map_h64 : &map_h;
+                const uint32_t hbytes = b.R <= 32 ? kTcTileBytes / 4 : b.R <= 64 ? kTcTileBytes / 2 : kTcTileBytes;
+                const uint32_t bytes = hbytes + (uint32_t)b.nsub * kTcTileBytes;
                 const bool read_again = c.group_count[b.n] > (b.pass + 1) * kTcPassRows;   // a later pass follows
                 const uint64_t pol_w = read_again ? pol_normal : pol_first;
                 for (int ks = 0; ks < g.ksteps; ++ks) {
@@ -374,7 +379,7 @@ __global__ void __launch_bounds__(kTcThreads, 1)
                     const uint32_t sb = smem_u32(smem + (size_t)stage * kTcStageBytes);
                     mbar_expect_tx(bar, bytes);
                     // tile 0 of a stage is the pass's block of hidden rows, tiles 1 and 2 the weight sub-tiles
-                    tma_load_2d(sb, &map_h, 0, (b.j * g.ksteps + ks) * kTcPassRows, bar, pol_last);
+                    tma_load_2d(sb, mh, 0, (b.j * g.ksteps + ks) * kTcPassRows, bar, pol_last);
                     for (int sub = 0; sub < b.nsub; ++sub)
                         tma_load_5d(sb + (1 + sub) * kTcTileBytes, &map_w, 0, 0, ks, (b.t + sub) * 8, b.n, bar, pol_w);
                     if (++stage == kTcStages) { stage = 0; phase ^= 1u; }
