@@ -335,3 +335,25 @@ def test_frequency_ordered_contiguous_groups(M, path):
     rep = ph.compare(W, gm, Wg, hb[rows], 4, 10, {k: a[rows] for k, a in out.items()})
     assert rep.ok, rep.errors
     head.close()
+
+
+@pytest.mark.parametrize("N,M,kg,path", [
+    (256, 3, 256, lmhead.CORAL_PATH_STREAM),       # the maximum group count, every group active
+    (256, 30, 200, lmhead.CORAL_PATH_STREAM),      # one-launch router with 8 groups per lane
+    (256, 40, 7, lmhead.CORAL_PATH_STREAM),        # 40 x 256 slots: too many for the band-ticket router -> four kernels
+    (128, 60, 9, lmhead.CORAL_PATH_STREAM),        # band-ticket router with 4 groups per lane
+    (128, 60, 9, lmhead.CORAL_PATH_SIMT_PLAIN),
+    (256, 150, 20, lmhead.CORAL_PATH_TCGEN05),     # many groups with a handful of rows each on the tensor-core path
+])
+def test_many_groups(N, M, kg, path):
+    v = 48
+    cfg = synth.HeadConfig("manyN", H=256, V=v * N, N=N, k_groups=kg, k_tokens=10, M=M, seed=17, w_std=0.05)
+    W, gm, Wg, hb = synth.make_all(cfg)
+    head = _head(cfg, W, gm, Wg, max_M=M, max_kg=kg, max_kt=10)
+    head.set_path(path)
+    out = ph.gpu_draft_numpy(head, hb, kg, 10)
+    assert head.status() == 0 and head.stats().path == path
+    rows = np.unique(np.linspace(0, M - 1, 12).astype(int))
+    rep = ph.compare(W, gm, Wg, hb[rows], kg, 10, {k: a[rows] for k, a in out.items()})
+    assert rep.ok, rep.errors
+    head.close()
