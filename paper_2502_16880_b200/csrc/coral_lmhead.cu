@@ -30,6 +30,7 @@ struct Layout {
     size_t packed_bytes, cand_cap;
     int v, T;
     int KB, T16;                 // packed layout (see packed_chunk_offset)
+    size_t route_bands;
     int tc_tiles, tc_vcap;       // tensor-core path: sub-tiles per group, capacity in (group, pass) entries
     size_t tc_rows;              // rows of the gathered hidden matrix (0: path not provisioned)
 };
@@ -92,7 +93,8 @@ Layout make_layout(const coral_lmhead_config& c) {
     L.w_gate = take(N * H * 2);
     L.group_tokens = take((size_t)c.V * 4);
     L.state = take(sizeof(DeviceState));
-    L.route_mid = take((kRouteMidBands + 4 * N) * 4);
+    L.route_bands = (M + 7) / 8 > (size_t)kRouteMidBands ? (M + 7) / 8 : (size_t)kRouteMidBands;
+    L.route_mid = take((L.route_bands + 5 * N) * 4);      // band tickets, 4 mask words and one counter per group
     L.gate = take(M * N * 4);
     L.sel = take(M * kg * 4);
     L.slot_of = take(M * N * 2);
@@ -402,7 +404,7 @@ int coral_lmhead_create(coral_lmhead_handle* out, const coral_lmhead_config* cfg
         if (cudaMemcpyAsync(h->ws + h->L.w_gate, W_gate_dev, (size_t)N * cfg->H * 2, cudaMemcpyDeviceToDevice, st) !=
             cudaSuccess) { rc = CORAL_ERR_CUDA; break; }
         if (cudaMemsetAsync(h->ws + h->L.state, 0, sizeof(DeviceState), st) != cudaSuccess) { rc = CORAL_ERR_CUDA; break; }
-        if (cudaMemsetAsync(h->ws + h->L.route_mid, 0, (kRouteMidBands + 4 * (size_t)cfg->n_groups) * 4, st) != cudaSuccess) { rc = CORAL_ERR_CUDA; break; }
+        if (cudaMemsetAsync(h->ws + h->L.route_mid, 0, (h->L.route_bands + 5 * (size_t)cfg->n_groups) * 4, st) != cudaSuccess) { rc = CORAL_ERR_CUDA; break; }
         if (cudaMemsetAsync(h->packed, 0, h->L.packed_bytes, st) != cudaSuccess) { rc = CORAL_ERR_CUDA; break; }
         pack_rows_kernel<<<V, 128, 0, st>>>(static_cast<const uint16_t*>(W_vocab_dev),
                                             reinterpret_cast<const int32_t*>(h->ws + h->L.group_tokens),
@@ -464,6 +466,9 @@ static int draft_impl(coral_lmhead_handle h, const void* hidden_dev, int M, int 
     c.pass_rows = path == CORAL_PATH_STREAM ? kStreamPassRows : path == CORAL_PATH_TCGEN05 ? kTcPassRows : 0;
     if (path == CORAL_PATH_TCGEN05) c.union_cap = h->L.tc_vcap;
     int launches = 0;
+    unsigned* rt_bands = reinterpret_cast<unsigned*>(h->ws + h->L.route_mid);
+    unsigned* rt_masks = rt_bands + h->L.route_bands;
+    int* rt_counts = reinterpret_cast<int*>(rt_masks + 4 * (size_t)cfg.n_groups);
 
     if (h->timing) cudaEventRecord(h->ev_begin, st);
     if (h->w1) {
@@ -477,20 +482,23 @@ static int draft_impl(coral_lmhead_handle h, const void* hidden_dev, int M, int 
         ++launches;
         count_groups_kernel<<<(M * k_groups + kSelectWarps * 32 - 1) / (kSelectWarps * 32), kSelectWarps * 32, 0, st>>>(c);
         ++launches;
-        bucket_group_kernel<<<c.N, 256, 0, st>>>(c);
+        bucket_group_kernel<<<c.N, 256, 0, st>>>(c, nullptr);
         ++launches;
     } else if (M <= kRouteFusedMaxM) {
         route_fused_kernel<<<c.N, kRouteThreads, 0, st>>>(c, forced_groups_dev, out_groups_dev, out_gate_dev);
         ++launches;
     } else if (M <= kRouteMidMaxM && M * c.N <= kRouteMidMaxCells && cfg.H % 32 == 0) {
         route_mid_kernel<<<dim3((c.N + 15) / 16, (M + 7) / 8), 256, 0, st>>>(
-            c, forced_groups_dev, out_groups_dev, out_gate_dev, reinterpret_cast<unsigned*>(h->ws + h->L.route_mid));
+            c, forced_groups_dev, out_groups_dev, out_gate_dev, rt_bands, rt_masks, rt_counts, 1);
+        ++launches;
+    } else if (cfg.H % 32 == 0) {
+        route_mid_kernel<<<dim3((c.N + 15) / 16, (M + 7) / 8), 256, 0, st>>>(
+            c, forced_groups_dev, out_groups_dev, out_gate_dev, rt_bands, rt_masks, rt_counts, 0);
+        ++launches;
+        bucket_group_kernel<<<c.N, 256, 0, st>>>(c, rt_counts);
         ++launches;
     } else {
-        if (cfg.H % 32 == 0)
-            gate_mma_kernel<<<dim3((c.N + 15) / 16, (M + 7) / 8), 256, 0, st>>>(c, out_gate_dev);
-        else
-            gate_tile_kernel<<<dim3((c.N + kGateTile - 1) / kGateTile, (M + kGateTile - 1) / kGateTile), 256, 0, st>>>(
+        gate_tile_kernel<<<dim3((c.N + kGateTile - 1) / kGateTile, (M + kGateTile - 1) / kGateTile), 256, 0, st>>>(
                 c, out_gate_dev);
         ++launches;
         select_kernel<<<(M + kSelectWarps - 1) / kSelectWarps, kSelectWarps * 32, 0, st>>>(c, forced_groups_dev,
@@ -498,7 +506,7 @@ static int draft_impl(coral_lmhead_handle h, const void* hidden_dev, int M, int 
         ++launches;
         count_groups_kernel<<<(M * k_groups + kSelectWarps * 32 - 1) / (kSelectWarps * 32), kSelectWarps * 32, 0, st>>>(c);
         ++launches;
-        bucket_group_kernel<<<c.N, 256, 0, st>>>(c);
+        bucket_group_kernel<<<c.N, 256, 0, st>>>(c, nullptr);
         ++launches;
     }
     if (h->timing) cudaEventRecord(h->ev_head0, st);

@@ -355,7 +355,7 @@ __global__ void __launch_bounds__(256) gate_tile_kernel(CallView c, float* __res
 // splitting H in blocks of 32 columns (mma.sync m16n8k16, bf16 x bf16 -> fp32; groups on the M axis, rows on N).
 // Every lane loads 16 bytes of two gate rows and of one hidden row per block of 32 columns; the column order
 // inside a block is permuted the same way for both operands, which leaves the dot products unchanged.
-// grid (ceil(N/16), ceil(M/8)), H a multiple of 32.  Block (0,0) also clears the per-group row counters.
+// H a multiple of 32.
 __device__ __forceinline__ void gate_mma_tile(const CallView& c, float* __restrict__ gate_tap, int n0, int m0,
                                               float (*s_part)[16 * 8]) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -398,26 +398,22 @@ __device__ __forceinline__ void gate_mma_tile(const CallView& c, float* __restri
     }
 }
 
-__global__ void __launch_bounds__(256) gate_mma_kernel(CallView c, float* __restrict__ gate_tap) {
-    __shared__ float s_part[8][16 * 8];
-    if (blockIdx.x == 0 && blockIdx.y == 0)
-        for (int n = threadIdx.x; n < c.N; n += 256) c.group_count[n] = 0;
-    gate_mma_tile(c, gate_tap, blockIdx.x * 16, blockIdx.y * 8, s_part);
-}
-
 // Router stage in one launch for a medium number of rows (kRouteFusedMaxM < M <= kRouteMidMaxM, M * N <=
-// kRouteMidMaxCells, H a multiple of 32).  grid (ceil(N/16), ceil(M/8)) as gate_mma_kernel.  Nobody waits for
+// kRouteMidMaxCells, H a multiple of 32).  grid (ceil(N/16), ceil(M/8)): a block computes one 16-group x 8-row tile of scores (gate_mma_tile).  Nobody waits for
 // anybody: the blocks of one 8-row band draw tickets from the band's counter and the last one selects the
 // groups of the band's rows (one warp per row) and ORs them into per-group row masks in global memory; these
 // band-finishers draw a second ticket and the last of them buckets the rows by group (one thread per group)
-// and writes the union list and the merge descriptors.  `scratch`: kRouteMidBands band counters, then four
-// mask words per group; all zero between calls (the last block clears what it used).
+// and writes the union list and the merge descriptors.  With finish = 0 (any number of rows) the
+// band-finishers only add their rows to per-group counters and bucket_group_kernel, launched next, does the
+// bucketing.  band_ticket: one counter per 8-row band; rowmask: four mask words per group; count_acc: one
+// counter per group; all zero between calls (whoever uses them last clears them).
 constexpr int kRouteMidMaxM = 128;
 constexpr int kRouteMidBands = kRouteMidMaxM / 8;
 constexpr int kRouteMidMaxCells = 8192;       // M * N slots staged in shared memory by the last block
 __global__ void __launch_bounds__(256)
     route_mid_kernel(CallView c, const int32_t* __restrict__ forced, int32_t* __restrict__ groups_tap,
-                     float* __restrict__ gate_tap, unsigned* __restrict__ scratch) {
+                     float* __restrict__ gate_tap, unsigned* __restrict__ band_ticket, unsigned* __restrict__ rowmask,
+                     int* __restrict__ count_acc, int finish) {
     __shared__ float s_part[8][16 * 8];
     __shared__ float s_val[8][kMaxGroups];
     __shared__ int16_t s_slot_row[8][kMaxGroups];
@@ -427,8 +423,6 @@ __global__ void __launch_bounds__(256)
     __shared__ int s_flag;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int m0 = blockIdx.y * 8;
-    unsigned* band_ticket = scratch;
-    unsigned* rowmask = scratch + kRouteMidBands;
     pdl_launch_dependents();      // the next kernel may set itself up; it waits for this grid before reading
 
     gate_mma_tile(c, gate_tap, blockIdx.x * 16, m0, s_part);
@@ -455,6 +449,11 @@ __global__ void __launch_bounds__(256)
         }
     }
     __syncthreads();
+    if (!finish) {                                  // many rows: only count; bucket_group_kernel does the rest
+        if (threadIdx.x < c.N && s_mask[threadIdx.x] && group_is_local(c, threadIdx.x))
+            atomicAdd(&count_acc[threadIdx.x], __popc(s_mask[threadIdx.x]));
+        return;
+    }
     if (threadIdx.x < c.N && s_mask[threadIdx.x])
         atomicOr(&rowmask[threadIdx.x * 4 + (m0 >> 5)], s_mask[threadIdx.x] << (m0 & 31));
     __threadfence();
@@ -535,14 +534,16 @@ __global__ void __launch_bounds__(kSelectWarps * 32) count_groups_kernel(CallVie
 
 // One block per group: the group's place in the bucket array and in the union list (prefix sums over the
 // per-group counts, recomputed by every block), then an ordered compaction of the rows that selected it.
-__global__ void __launch_bounds__(256) bucket_group_kernel(CallView c) {
+__global__ void __launch_bounds__(256) bucket_group_kernel(CallView c, int* __restrict__ count_acc) {
     __shared__ int s_cnt[kMaxGroups], s_pass[kMaxGroups];
     __shared__ int s_warp[8];
     const int n = blockIdx.x;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     {
+        // counts: group_count (filled by count_groups_kernel), or the accumulators of route_mid_kernel, which
+        // the last block to have read them clears for the next call
         const int t = threadIdx.x;
-        const int cnt = t < c.N ? c.group_count[t] : 0;
+        const int cnt = t < c.N ? (count_acc ? __ldcg(count_acc + t) : c.group_count[t]) : 0;
         s_cnt[t] = cnt;
         s_pass[t] = cnt == 0 ? 0 : (c.pass_rows > 0 ? (cnt + c.pass_rows - 1) / c.pass_rows : 1);
     }
@@ -557,6 +558,14 @@ __global__ void __launch_bounds__(256) bucket_group_kernel(CallView c) {
     const int cnt = s_cnt[n], passes = s_pass[n];
     if (threadIdx.x == 0) {
         c.group_offset[n] = off;
+        if (count_acc) {
+            c.group_count[n] = cnt;
+            const int ticket = atomicAdd(&c.state->ticket, 1);     // every block has read all counters by now
+            if (ticket == (int)gridDim.x - 1) {
+                for (int t = 0; t < c.N; ++t) count_acc[t] = 0;
+                c.state->ticket = 0;
+            }
+        }
         c.union_rank[n] = cnt > 0 ? virt : -1;
         for (int p = 0; p < passes; ++p)
             if (virt + p < c.union_cap) c.union_list[virt + p] = n | (p << 16);
