@@ -5,7 +5,7 @@ What it computes (CORAL Section 2.2: several candidates per timestep form a draf
   child score = parent's cumulative log-score + candidate log-probability,
 and the K children with the highest score are kept, sorted descending, equal scores ordered by the flat
 (node, candidate) index.  The paper does not spell the rule out (it refers to EAGLE-2's dynamic tree), so the
-cumulative-log-probability ranking is this build's reading; see the design doc.  The addition is taken in fp32,
+cumulative-log-probability ranking is a reading of the paper, not a quotation.  The addition is taken in fp32,
 the precision the kernel decides in, so that the selected indices can be compared bit for bit.
 Plain numpy, a full stable sort, no shortcuts.
 """
