@@ -416,6 +416,17 @@ def main():
         out["correlated_rows_M60_rho0.3"] = {"us_per_step": float(np.mean(ms_c)) * 1e3,
                                              "groups_touched_mean": float(np.mean(t_c)),
                                              "GBps": b_c / (float(np.mean(ms_c)) * 1e-3) / 1e9}
+        # the same with the kernel chosen on the device from the rows per group (CORAL_PATH_ADAPTIVE), and what
+        # that mode costs where the streaming kernel stays the right choice (iid rows, M=60)
+        head.set_path(lmhead.CORAL_PATH_ADAPTIVE)
+        ms_ca, _, _, _, _ = time_steps(60, cfg.k_groups, extra_steps, 3, my_batches, rho=0.3)
+        took_c = int(head.stats().path)
+        ms_ia, _, _, _, _ = time_steps(60, cfg.k_groups, extra_steps, 3, my_batches)
+        took_i = int(head.stats().path)
+        head.set_path(lmhead.CORAL_PATH_AUTO)
+        out["correlated_rows_M60_rho0.3"]["adaptive_us_per_step"] = float(np.mean(ms_ca)) * 1e3
+        out["correlated_rows_M60_rho0.3"]["adaptive_path"] = took_c
+        out["adaptive_iid_M60"] = {"us_per_step": float(np.mean(ms_ia)) * 1e3, "path": took_i}
         # extra: the paper's frequency-ordered contiguous grouping (Appendix B), modelled by a contiguous group map
         # and a Zipf-like prior on low-index groups in the gate (synth.py), against the random map above
         zcfg = cfg.with_(zipf_s=1.5)
@@ -426,8 +437,13 @@ def main():
         for M in (8, 60):
             ms_z, _, t_z, _, _ = time_steps(M, cfg.k_groups, extra_steps, 3, my_batches, zipf_s=1.5, on=zhead)
             b_z = float(np.mean([algorithmic_bytes(cfg.with_(M=M), u, M) for u in t_z]))
+            zhead.set_path(lmhead.CORAL_PATH_ADAPTIVE)
+            ms_za, _, _, _, _ = time_steps(M, cfg.k_groups, extra_steps, 3, my_batches, zipf_s=1.5, on=zhead)
+            took_z = int(zhead.stats().path)
+            zhead.set_path(lmhead.CORAL_PATH_AUTO)
             zleg.append({"M": M, "us_per_step": float(np.mean(ms_z)) * 1e3, "groups_touched_mean": float(np.mean(t_z)),
-                         "GBps": b_z / (float(np.mean(ms_z)) * 1e-3) / 1e9})
+                         "GBps": b_z / (float(np.mean(ms_z)) * 1e-3) / 1e9,
+                         "adaptive_us_per_step": float(np.mean(ms_za)) * 1e3, "adaptive_path": took_z})
         assert zhead.status() == 0
         zhead.close()
         out["contiguous_groups_zipf1.5"] = zleg

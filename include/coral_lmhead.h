@@ -49,6 +49,7 @@ extern "C" {
 #define CORAL_PATH_STREAM 1        /* bulk-copy weight streaming + warp MMA (fp32 accumulate); M <= 128, H % 256 == 0, H <= 4096 */
 #define CORAL_PATH_TCGEN05 2       /* routed grouped GEMM on tcgen05 / TMEM tiles */
 #define CORAL_PATH_SIMT_PLAIN 3    /* gathered GEMV with plain 128-bit loads, any M */
+#define CORAL_PATH_ADAPTIVE 4      /* 33..128 rows: the router picks STREAM or TCGEN05 on the device from the rows per group */
 
 /* Output modes (coral_lmhead_set_output_mode). */
 #define CORAL_OUTPUT_JOINT 0       /* log-softmax over all active logits of the row (default) */
@@ -205,6 +206,12 @@ int coral_lmhead_set_router_mlp(coral_lmhead_handle h, const void *W1_dev, void 
  * Force an execution path (CORAL_PATH_*) for later draft calls; AUTO restores the default choice.
  * A draft call that the forced path cannot run (e.g. CORAL_PATH_STREAM with M > 128) returns
  * CORAL_ERR_INVALID.
+ * CORAL_PATH_ADAPTIVE: Appendix B notes that the rows of a tree seldom spread over all groups; rows then pile
+ * up on a few groups, and the streaming kernel, which reads a group once per 16 rows, reads those several
+ * times.  For calls of 33..128 rows (on a handle created with max_M > 32, H a multiple of 256) the router
+ * then compares, on the device, the reads the two kernels would need and records its choice; both kernels
+ * are launched and the one not chosen returns at once (about 4 us per call).  Other calls behave as with
+ * AUTO.  coral_lmhead_last_stats reports the kernel that ran.
  */
 int coral_lmhead_set_path(coral_lmhead_handle h, int path);
 

@@ -17,6 +17,7 @@ struct DeviceState {
     int n_union;       // groups touched by the last call
     int ticket;        // arrival counter of the fused router kernel; zero between calls
     int n_virtual;     // (group, pass) entries of the union list; equals n_union when no group needs a second pass
+    int path_choice;   // adaptive calls: 1 = streaming kernel, 2 = tensor-core kernel, chosen by the router from the row counts
 };
 
 // Per-call view of the workspace handed to the kernels.
@@ -25,6 +26,8 @@ struct CallView {
     int k_groups, k_tokens;
     int union_cap;                 // capacity of union_list
     int pass_rows;                 // rows of a group handled per pass over its weights (0: one pass for any count)
+    int adaptive;                  // 1: the router picks pass_rows (streaming) or pass_rows_tc (tensor cores) and records it
+    int pass_rows_tc, union_cap_tc;   // the tensor-core alternative of an adaptive call
     int shard_rank, shard_world;   // vocab sharding: this call computes only the groups n with n % shard_world == shard_rank
     const uint16_t* packed;        // blocked copy of W_vocab, see packed_chunk_offset
     int KB, T16;                   // packed layout: 64-column blocks per row, 16-row items per group

@@ -78,7 +78,8 @@ size_t stream_smem_bytes(const StreamGeom& g) {
            sizeof(int) * kStreamSegTab + 16;
 }
 
-constexpr int kTcMinRows = 96;          // above this many rows the tensor-core path is the faster one (measured)
+constexpr int kTcMinRows = 96;          // above this many rows the tensor-core path is the faster one (measured, iid rows)
+constexpr int kTcProvisionRows = 32;    // handles for more rows get the tensor-core workspace (adaptive calls use it from 33 rows)
 constexpr int kMergeSmemCands = 4096;   // candidates the streaming merge keeps in shared memory
 
 Layout make_layout(const coral_lmhead_config& c) {
@@ -120,7 +121,7 @@ Layout make_layout(const coral_lmhead_config& c) {
     L.part_id = take(M * kg * T * kt * 4);
     // tensor-core path (only provisioned when calls can exceed the streaming path's row limit)
     L.tc_tiles = (L.v + kTcSub - 1) / kTcSub;
-    L.tc_rows = M > (size_t)kTcMinRows ? M * kg : 0;
+    L.tc_rows = M > (size_t)kTcProvisionRows ? M * kg : 0;
     L.tc_vcap = L.tc_rows ? (int)(N + (M * kg + kTcPassRows - 1) / kTcPassRows) : 0;
     const size_t tcp = (size_t)L.tc_vcap * L.tc_tiles * kTcPassRows;
     L.tc_hg = take((size_t)L.tc_vcap * L.KB * kTcPassRows * kTcK * 2);   // blocked: [entry][column block][128][64]
@@ -285,7 +286,7 @@ bool tc_usable(const coral_lmhead_s* h, int M, int kg) {
 int choose_path(const coral_lmhead_s* h, int M, int kg) {
     if (h->forced_path == CORAL_PATH_STREAM) return stream_ok(h, M) ? CORAL_PATH_STREAM : 0;
     if (h->forced_path == CORAL_PATH_TCGEN05) return tc_usable(h, M, kg) ? CORAL_PATH_TCGEN05 : 0;
-    if (h->forced_path != CORAL_PATH_AUTO) return h->forced_path;
+    if (h->forced_path != CORAL_PATH_AUTO && h->forced_path != CORAL_PATH_ADAPTIVE) return h->forced_path;
     if (M > kTcMinRows && tc_usable(h, M, kg)) return CORAL_PATH_TCGEN05;
     if (stream_ok(h, M)) return CORAL_PATH_STREAM;
     return tc_usable(h, M, kg) ? CORAL_PATH_TCGEN05 : CORAL_PATH_SIMT_PLAIN;
@@ -435,7 +436,7 @@ int coral_lmhead_destroy(coral_lmhead_handle h) {
 }
 
 int coral_lmhead_set_path(coral_lmhead_handle h, int path) {
-    if (!h || path < CORAL_PATH_AUTO || path > CORAL_PATH_SIMT_PLAIN) return CORAL_ERR_INVALID;
+    if (!h || path < CORAL_PATH_AUTO || path > CORAL_PATH_ADAPTIVE) return CORAL_ERR_INVALID;
     h->forced_path = path;
     return CORAL_OK;
 }
@@ -457,14 +458,22 @@ static int draft_impl(coral_lmhead_handle h, const void* hidden_dev, int M, int 
         return CORAL_ERR_INVALID;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     CallView c = make_view(h, hidden_dev, M, k_groups, k_tokens);
-    const int path = choose_path(h, M, k_groups);
+    int path = choose_path(h, M, k_groups);
     if (path == 0) return CORAL_ERR_INVALID;   // the forced path does not support this call
     if (h->out_mode == CORAL_OUTPUT_FACTORISED && path == CORAL_PATH_SIMT_PLAIN) return CORAL_ERR_INVALID;
     if (partial_dev && (path == CORAL_PATH_SIMT_PLAIN || h->out_mode != CORAL_OUTPUT_JOINT)) return CORAL_ERR_INVALID;
     const int merge_mode = partial_dev ? kMergePartial : h->out_mode == CORAL_OUTPUT_FACTORISED ? kMergeFactorised : kMergeJoint;
     float* merge_out = partial_dev ? partial_dev : out_logprobs_dev;
+    // adaptive: both fast paths can take the call and the band-ticket router (which makes the choice) runs it
+    const bool adaptive = h->forced_path == CORAL_PATH_ADAPTIVE && !h->w1 && M > kRouteFusedMaxM && M <= kRouteMidMaxM &&
+                          M * cfg.n_groups <= kRouteMidMaxCells && cfg.H % 32 == 0 && stream_ok(h, M) &&
+                          tc_usable(h, M, k_groups);
+    if (adaptive) path = CORAL_PATH_STREAM;      // the launch sequence below starts from the streaming one
     c.pass_rows = path == CORAL_PATH_STREAM ? kStreamPassRows : path == CORAL_PATH_TCGEN05 ? kTcPassRows : 0;
     if (path == CORAL_PATH_TCGEN05) c.union_cap = h->L.tc_vcap;
+    c.adaptive = adaptive ? 1 : 0;
+    c.pass_rows_tc = kTcPassRows;
+    c.union_cap_tc = h->L.tc_vcap;
     int launches = 0;
     unsigned* rt_bands = reinterpret_cast<unsigned*>(h->ws + h->L.route_mid);
     unsigned* rt_masks = rt_bands + h->L.route_bands;
@@ -514,15 +523,36 @@ static int draft_impl(coral_lmhead_handle h, const void* hidden_dev, int M, int 
         const Layout& L = h->L;
         StreamPartials pp{reinterpret_cast<float*>(h->ws + L.sp_max), reinterpret_cast<float*>(h->ws + L.sp_sum),
                           reinterpret_cast<float*>(h->ws + L.sp_val), reinterpret_cast<int32_t*>(h->ws + L.sp_id)};
+        StreamPartials tpp{reinterpret_cast<float*>(h->ws + L.tc_max), reinterpret_cast<float*>(h->ws + L.tc_sum),
+                           reinterpret_cast<float*>(h->ws + L.tc_val), reinterpret_cast<int32_t*>(h->ws + L.tc_id)};
+        StreamGeom mg = h->sg;                   // geometry of the tensor-core partials, as the merge reads them
+        mg.tc_tiles = L.tc_tiles;
+        mg.tc_rows = kTcPassRows;
+        mg.T = L.tc_tiles;
+        if (adaptive) {
+            // both head kernels are launched; each reads the router's choice first and the one not chosen returns
+            TcGeom tg{h->sms, L.tc_tiles, L.KB};
+            TcPartials tp{tpp.pmax, tpp.psum, tpp.pval, tpp.pid};
+            launch_pdl(tc_gather_kernel, dim3(M * k_groups), dim3(128), (size_t)0, st, c,
+                       reinterpret_cast<uint16_t*>(h->ws + L.tc_hg));
+            ++launches;
+            head_tc_kernel<<<tg.grid, kTcThreads, kTcSmemBytes, st>>>(c, tg, tp, h->map_w, h->map_h, h->map_h64, h->map_h32,
+                                                                     out_logits_dev);
+            ++launches;
+        }
         launch_pdl(h->sg.kc == 512 ? head_stream_kernel<2> : head_stream_kernel<1>, dim3(h->sg.grid),
                    dim3(kStreamThreads), (size_t)h->stream_smem, st, c, h->sg, pp, out_logits_dev);
         ++launches;
         if (h->timing) cudaEventRecord(h->ev_head1, st);
         {
-            const int p_cap = h->sg.grid + 2 * k_groups;
-            const int c_cap = p_cap * k_tokens < kMergeSmemCands ? p_cap * k_tokens : kMergeSmemCands;
+            int p_cap = h->sg.grid + 2 * k_groups;
+            int c_cap = p_cap * k_tokens < kMergeSmemCands ? p_cap * k_tokens : kMergeSmemCands;
+            if (adaptive) {
+                p_cap = p_cap > k_groups * L.tc_tiles ? p_cap : k_groups * L.tc_tiles;
+                c_cap = c_cap > k_groups * L.tc_tiles * k_tokens ? c_cap : k_groups * L.tc_tiles * k_tokens;
+            }
             launch_pdl(merge_stream_kernel, dim3(M), dim3(kMergeStreamThreads), merge_smem_bytes(p_cap, c_cap), st, c,
-                       h->sg, pp, reinterpret_cast<float*>(h->ws + L.cand_val),
+                       h->sg, pp, mg, tpp, reinterpret_cast<float*>(h->ws + L.cand_val),
                        reinterpret_cast<int32_t*>(h->ws + L.cand_id), (int)L.cand_cap, c_cap, p_cap, merge_mode,
                        out_ids_dev, merge_out, out_lse_dev);
         }
@@ -547,7 +577,7 @@ static int draft_impl(coral_lmhead_handle h, const void* hidden_dev, int M, int 
             const int p_cap = k_groups * L.tc_tiles;
             const int c_cap = p_cap * k_tokens;          // tc_usable() keeps this within kMergeSmemCands
             launch_pdl(merge_stream_kernel, dim3(M), dim3(kMergeStreamThreads), merge_smem_bytes(p_cap, c_cap), st, c, mg,
-                       pp, reinterpret_cast<float*>(h->ws + L.cand_val), reinterpret_cast<int32_t*>(h->ws + L.cand_id),
+                       pp, mg, pp, reinterpret_cast<float*>(h->ws + L.cand_val), reinterpret_cast<int32_t*>(h->ws + L.cand_id),
                        (int)L.cand_cap, c_cap, p_cap, merge_mode, out_ids_dev, merge_out, out_lse_dev);
         }
         ++launches;
@@ -561,7 +591,7 @@ static int draft_impl(coral_lmhead_handle h, const void* hidden_dev, int M, int 
     if (h->timing) cudaEventRecord(h->ev_end, st);
     if (cudaGetLastError() != cudaSuccess) return CORAL_ERR_CUDA;
 
-    h->last_path = path; h->last_M = M; h->last_kg = k_groups; h->last_kt = k_tokens; h->last_launches = launches;
+    h->last_path = adaptive ? CORAL_PATH_ADAPTIVE : path; h->last_M = M; h->last_kg = k_groups; h->last_kt = k_tokens; h->last_launches = launches;
     return CORAL_OK;
 }
 
@@ -712,7 +742,8 @@ int coral_lmhead_last_stats(coral_lmhead_handle h, coral_lmhead_stats* out, void
     DeviceState s{};
     if (cudaMemcpyAsync(&s, h->ws + h->L.state, sizeof s, cudaMemcpyDeviceToHost, st) != cudaSuccess) return CORAL_ERR_CUDA;
     if (cudaStreamSynchronize(st) != cudaSuccess) return CORAL_ERR_CUDA;
-    out->path = h->last_path;
+    out->path = h->last_path == CORAL_PATH_ADAPTIVE ? (s.path_choice == 2 ? CORAL_PATH_TCGEN05 : CORAL_PATH_STREAM)
+                                                    : h->last_path;
     out->M = h->last_M;
     out->k_groups = h->last_kg;
     out->k_tokens = h->last_kt;

@@ -318,6 +318,7 @@ __global__ void __launch_bounds__(kStreamThreads, 1) head_stream_kernel(CallView
 
     pdl_wait();                   // the router stage's outputs are complete from here on
     pdl_launch_dependents();      // the merge kernel may start reading the router's outputs
+    if (c.adaptive && c.state->path_choice != 1) return;     // the router chose the tensor-core kernel for this call
     const int n_items = c.state->n_virtual * g.T;
     const int per = (n_items + g.grid - 1) / g.grid;
     sh.lo = min(n_items, (int)blockIdx.x * per);
@@ -408,7 +409,8 @@ constexpr int kMergeJoint = 0, kMergeFactorised = 1, kMergePartial = 2;
 constexpr int kMergeStreamThreads = 256;
 constexpr int kMergeMaxPieces = 1024;         // >= grid + 2 * k_groups for every supported shape
 constexpr int kMergeRankMax = 256;            // survivors ranked by counting; more fall back to k rounds
-__global__ void __launch_bounds__(kMergeStreamThreads) merge_stream_kernel(CallView c, StreamGeom g, StreamPartials pp,
+__global__ void __launch_bounds__(kMergeStreamThreads) merge_stream_kernel(CallView c, StreamGeom g_in, StreamPartials pp_in,
+                                                                           StreamGeom g_tc, StreamPartials pp_tc,
                                                                            float* __restrict__ cand_val_scratch,
                                                                            int32_t* __restrict__ cand_id_scratch,
                                                                            int cand_cap, int smem_cands, int p_cap, int mode,
@@ -416,6 +418,11 @@ __global__ void __launch_bounds__(kMergeStreamThreads) merge_stream_kernel(CallV
                                                                            float* __restrict__ out_logprobs,
                                                                            float* __restrict__ lse_tap) {
     extern __shared__ __align__(16) unsigned char msm[];
+    // adaptive call: the partials are those of the kernel the router chose (complete by the time this grid runs:
+    // it is launched behind the tensor-core kernel, which does not release its dependents early)
+    const bool took_tc = c.adaptive && c.state->path_choice == 2;
+    const StreamGeom g = took_tc ? g_tc : g_in;
+    const StreamPartials pp = took_tc ? pp_tc : pp_in;
     const int m = blockIdx.x;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     constexpr int kWarps = kMergeStreamThreads / 32;

@@ -137,6 +137,8 @@ __device__ __forceinline__ void tc_ld32(uint32_t taddr, float (&v)[32]) {
 // whatever they held (their accumulator lanes are never read).
 __global__ void __launch_bounds__(128) tc_gather_kernel(CallView c, uint16_t* __restrict__ hg) {
     const int p = blockIdx.x;
+    pdl_wait();                                              // (adaptive calls launch this kernel over the router's tail)
+    if (c.adaptive && c.state->path_choice != 2) return;     // the router chose the streaming kernel for this call
     if (p >= c.group_offset[c.N]) return;          // fewer pairs than M * k_groups when the vocab is sharded
     const int m = c.bucket_row[p];
     const int n = c.sel[(size_t)m * c.k_groups + c.bucket_slot[p]];
@@ -318,6 +320,7 @@ __global__ void __launch_bounds__(kTcThreads, 1)
     head_tc_kernel(CallView c, TcGeom g, TcPartials pp, const __grid_constant__ CUtensorMap map_w,
                    const __grid_constant__ CUtensorMap map_h, const __grid_constant__ CUtensorMap map_h64,
                    const __grid_constant__ CUtensorMap map_h32, float* __restrict__ logits_tap) {
+    if (c.adaptive && c.state->path_choice != 2) return;     // the router chose the streaming kernel for this call
     extern __shared__ unsigned char tc_smem_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(tc_smem_raw) + 1023) & ~(uintptr_t)1023);
     float* zstash = reinterpret_cast<float*>(smem + kTcStages * kTcStageBytes);          // [32][epilogue threads]

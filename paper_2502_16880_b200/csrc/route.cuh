@@ -479,7 +479,28 @@ __global__ void __launch_bounds__(256)
         }
     }
     const int cnt = __popc(mask[0]) + __popc(mask[1]) + __popc(mask[2]) + __popc(mask[3]);
-    const int passes = cnt == 0 ? 0 : (c.pass_rows > 0 ? (cnt + c.pass_rows - 1) / c.pass_rows : 1);
+    // Adaptive call: the streaming kernel reads a group once per pass_rows rows, the tensor-core kernel once
+    // per pass_rows_tc rows but costs more per read and has a fixed extra cost (gathering the rows, a longer
+    // tail).  Compare the two totals (cost per pass in units of 10 ns, measured on the Llama3-8B shape) and
+    // record the choice for the kernels launched after this one.
+    int pr = c.pass_rows, ucap = c.union_cap;
+    if (c.adaptive) {
+        const int ps = cnt == 0 ? 0 : (cnt + c.pass_rows - 1) / c.pass_rows;
+        const int pt = cnt == 0 ? 0 : (cnt + c.pass_rows_tc - 1) / c.pass_rows_tc;
+        int both = ps | (pt << 16);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) both += __shfl_xor_sync(0xffffffffu, both, o);
+        if (lane == 0) s_warp_tot[warp] = both;
+        __syncthreads();
+        int tot2 = 0;
+#pragma unroll
+        for (int w = 0; w < 8; ++w) tot2 += s_warp_tot[w];
+        __syncthreads();
+        const bool use_tc = (tot2 & 0xffff) * 330 > (tot2 >> 16) * 345 + 1200;
+        if (use_tc) { pr = c.pass_rows_tc; ucap = c.union_cap_tc; }
+        if (threadIdx.x == 0) c.state->path_choice = use_tc ? 2 : 1;
+    }
+    const int passes = cnt == 0 ? 0 : (pr > 0 ? (cnt + pr - 1) / pr : 1);
     const int packed = cnt | (passes << 16);
     int incl = packed;
 #pragma unroll
@@ -503,7 +524,7 @@ __global__ void __launch_bounds__(256)
         c.group_count[n] = cnt;
         c.union_rank[n] = cnt > 0 ? virt : -1;
         for (int p = 0; p < passes; ++p)
-            if (virt + p < c.union_cap) c.union_list[virt + p] = n | (p << 16);
+            if (virt + p < ucap) c.union_list[virt + p] = n | (p << 16);
         int pos = 0;
 #pragma unroll
         for (int w = 0; w < 4; ++w) {
@@ -514,15 +535,15 @@ __global__ void __launch_bounds__(256)
                 const int sl = s_slot[m * c.N + n];
                 c.bucket_row[off + pos] = m;
                 c.bucket_slot[off + pos] = sl;
-                const int pass = c.pass_rows > 0 ? pos / c.pass_rows : 0;
-                c.slot_desc[(size_t)m * c.k_groups + sl] = ((virt + pass) << 8) | ((pos - pass * max(c.pass_rows, 1)) & 255);
+                const int pass = pr > 0 ? pos / pr : 0;
+                c.slot_desc[(size_t)m * c.k_groups + sl] = ((virt + pass) << 8) | ((pos - pass * max(pr, 1)) & 255);
             }
         }
     }
     if (threadIdx.x == 0) {
         c.group_offset[c.N] = total & 0xffff;
         c.state->n_union = n_union;
-        c.state->n_virtual = min(total >> 16, c.union_cap);
+        c.state->n_virtual = min(total >> 16, ucap);
     }
 }
 

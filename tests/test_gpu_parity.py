@@ -357,3 +357,34 @@ def test_many_groups(N, M, kg, path):
     rep = ph.compare(W, gm, Wg, hb[rows], kg, 10, {k: a[rows] for k, a in out.items()})
     assert rep.ok, rep.errors
     head.close()
+
+
+@pytest.mark.parametrize("M,kg,zipf,expect", [
+    (40, 2, 0.0, lmhead.CORAL_PATH_STREAM),      # ~5 rows per group: one read per group either way -> streaming kernel
+    (60, 4, 1.5, lmhead.CORAL_PATH_TCGEN05),     # hot groups selected by most rows -> tensor-core kernel
+    (128, 8, 0.0, lmhead.CORAL_PATH_TCGEN05),    # 64 rows per group: four streaming passes against one
+    (100, 3, 0.0, None),                         # near the break-even: either choice, same results
+    (8, 4, 0.0, lmhead.CORAL_PATH_STREAM),       # outside 33..128 rows the call is an ordinary one
+])
+def test_adaptive_path_choice_on_device(M, kg, zipf, expect):
+    cfg = synth.HeadConfig("adaptive", H=256, V=256 * 16, N=16, k_groups=kg, k_tokens=10, M=M, seed=23, w_std=0.05,
+                           zipf_s=zipf)
+    W, Wg, hb = synth.make_w_vocab(cfg), synth.make_w_gate(cfg), synth.make_hidden(cfg)
+    gm = synth.make_group_map(cfg, contiguous=zipf > 0)
+    head = _head(cfg, W, gm, Wg, max_M=128, max_kg=8)
+    head.set_path(lmhead.CORAL_PATH_ADAPTIVE)
+    out = ph.gpu_draft_numpy(head, hb, kg, 10)
+    assert head.status() == 0
+    took = head.stats().path
+    assert took in (lmhead.CORAL_PATH_STREAM, lmhead.CORAL_PATH_TCGEN05)
+    if expect is not None:
+        assert took == expect
+    rows = np.unique(np.linspace(0, M - 1, 24).astype(int))
+    rep = ph.compare(W, gm, Wg, hb[rows], kg, 10, {k: a[rows] for k, a in out.items()})
+    assert rep.ok, rep.errors
+    # the same call on the path it took, forced from the host: identical bits
+    head.set_path(took)
+    again = ph.gpu_draft_numpy(head, hb, kg, 10)
+    for k in ("ids", "logprobs", "groups"):
+        assert np.array_equal(out[k], again[k]), k
+    head.close()
