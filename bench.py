@@ -353,7 +353,22 @@ def main():
     k_bytes = float(np.mean([u * cfg.v * cfg.H * 2 + cfg.M * cfg.H * 2 for u in ktouched]))
     k_ms = float(np.mean(kms))
     achieved = k_bytes / (k_ms * 1e-3) / 1e9
+    # floor for that kernel: a do-nothing bulk-copy stream of the same number of bytes of the packed head, cold L2
+    floor_bytes = int(k_bytes) // 16384 * 16384
+    fl_ms = []
+    for i in range(23):
+        flush_l2(i)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        lmhead.coral_lmhead_copy_floor(head.handle, floor_bytes, stream)
+        b.record(stream)
+        torch.cuda.synchronize()
+        if i >= 3:
+            fl_ms.append(a.elapsed_time(b))
+    assert head.status() == 0
+    copy_floor_us = float(np.mean(fl_ms)) * 1e3
     roofline = {"bound": "hbm", "kernel": "head_stream_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                "copy_floor_us_same_bytes": copy_floor_us, "frac_of_copy_floor": copy_floor_us / (k_ms * 1e3),
                 "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
                 "traffic": None if STREAM_TRAFFIC_RATIO is None else STREAM_TRAFFIC_RATIO * k_bytes,
                 "avg_launch_us": k_ms * 1e3, "algorithmic_bytes_per_launch": k_bytes}

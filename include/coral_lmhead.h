@@ -216,6 +216,15 @@ int coral_lmhead_set_router_mlp(coral_lmhead_handle h, const void *W1_dev, void 
 int coral_lmhead_set_path(coral_lmhead_handle h, int path);
 
 /*
+ * Measurement aid with no counterpart in the paper: streams the first `bytes` of the packed head into shared
+ * memory with plain contiguous 16 KiB bulk copies (one CTA per SM, eight copies in flight each) and does
+ * nothing with them.  Timed by the caller with events on `stream`, from a cold L2, it gives the floor for the
+ * weight-streaming kernel of a draft call that reads as many bytes: a one-shot read of a few hundred megabytes
+ * does not reach the bandwidth of a long copy.  bytes in [16384, packed_bytes]; asynchronous, no allocation.
+ */
+int coral_lmhead_copy_floor(coral_lmhead_handle h, long long bytes, void *stream);
+
+/*
  * Measurement aid for the dominant kernel (the one that streams the selected
  * groups' weights; Section 3.3 names the LM head as the drafter's main cost).
  * With timing on, every draft call records a CUDA event before and after that

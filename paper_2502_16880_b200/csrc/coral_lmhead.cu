@@ -11,6 +11,7 @@
 #include "head_simt.cuh"
 #include "head_stream.cuh"
 #include "head_tc.cuh"
+#include "copy_probe.cuh"
 #include "merge.cuh"
 #include "route.cuh"
 #include "tree.cuh"
@@ -270,7 +271,7 @@ bool make_tc_maps(coral_lmhead_s* h) {
 }
 
 // Dynamic shared memory of merge_stream_kernel for p_cap pieces and c_cap in-smem candidates.
-inline size_t merge_smem_bytes(int p_cap, int c_cap) { return (size_t)c_cap * 8 + (size_t)p_cap * 21 + 16; }
+inline size_t merge_smem_bytes(int p_cap, int c_cap) { return (size_t)c_cap * 8 + (size_t)p_cap * 25 + 16; }
 
 constexpr size_t kTcSmemBytes = 1024 + (size_t)kTcStages * kTcStageBytes + 32 * kTcEpilogueThreads * 4 + 256;
 
@@ -665,6 +666,16 @@ int coral_tree_expand(const float* parent_scores_dev, const int32_t* cand_ids_de
     tree_expand_kernel<<<n_seq, kTreeThreads, 0, static_cast<cudaStream_t>(stream)>>>(
         parent_scores_dev, cand_ids_dev, cand_logprobs_dev, nodes, k_tokens, K, out_parent_dev, out_token_dev,
         out_score_dev);
+    return cudaGetLastError() == cudaSuccess ? CORAL_OK : CORAL_ERR_CUDA;
+}
+
+int coral_lmhead_copy_floor(coral_lmhead_handle h, long long bytes, void* stream) {
+    if (!h || bytes < kCopyChunk || (size_t)bytes > h->L.packed_bytes) return CORAL_ERR_INVALID;
+    if (cudaFuncSetAttribute(copy_probe_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kCopyStages * kCopyChunk) !=
+        cudaSuccess) return CORAL_ERR_CUDA;
+    copy_probe_kernel<<<h->sms, 32, kCopyStages * kCopyChunk, static_cast<cudaStream_t>(stream)>>>(
+        h->packed, bytes / kCopyChunk, reinterpret_cast<DeviceState*>(h->ws + h->L.state),
+        reinterpret_cast<unsigned*>(h->ws + h->L.cand_val));
     return cudaGetLastError() == cudaSuccess ? CORAL_OK : CORAL_ERR_CUDA;
 }
 

@@ -430,7 +430,7 @@ __global__ void __launch_bounds__(kMergeStreamThreads) merge_stream_kernel(CallV
     float* rec = partial ? out_logprobs + (size_t)m * (2 + 2 * c.k_tokens) : nullptr;
     __shared__ float s_f[kWarps], s_t[kWarps];
     __shared__ float s_lse, s_glse, s_thr2;
-    __shared__ int s_n;
+    __shared__ int s_n, s_nlive;
     __shared__ int s_first[kMaxGroups], s_base[kMaxGroups + 1], s_rpos[kMaxGroups], s_j[kMaxGroups];
     __shared__ float s_off[kMaxGroups];           // per slot: what is added to a logit to give the emitted log-prob
     // dynamic shared memory: candidates (smem_cands values + ids), then per-piece arrays of capacity p_cap
@@ -439,7 +439,8 @@ __global__ void __launch_bounds__(kMergeStreamThreads) merge_stream_kernel(CallV
     float* s_last = s_ps + p_cap;
     float* s_head = s_last + p_cap;
     int* s_piece = reinterpret_cast<int*>(s_head + p_cap);
-    unsigned char* s_pslot = reinterpret_cast<unsigned char*>(s_piece + p_cap);
+    int* s_live = s_piece + p_cap;                // pieces that can hold a candidate
+    unsigned char* s_pslot = reinterpret_cast<unsigned char*>(s_live + p_cap);
 
     // The router's outputs were complete before the streaming kernel let this grid start.
     const int n_items = c.state->n_virtual * g.T;
@@ -455,7 +456,7 @@ __global__ void __launch_bounds__(kMergeStreamThreads) merge_stream_kernel(CallV
         s_rpos[s] = desc & 255;
         s_off[s] = factorised ? c.gate[(size_t)m * c.N + c.sel[(size_t)m * c.k_groups + s]] : 0.f;
     }
-    if (threadIdx.x == 0) { s_n = 0; s_thr2 = kNegInf; }
+    if (threadIdx.x == 0) { s_n = 0; s_nlive = 0; s_thr2 = kNegInf; }
     if (factorised) {                 // log-sum-exp of the row's N gate scores (kMergeStreamThreads >= N)
         const float gv = threadIdx.x < c.N ? c.gate[(size_t)m * c.N + threadIdx.x] : kNegInf;
         const float wm = warp_max(gv);
@@ -575,23 +576,30 @@ __global__ void __launch_bounds__(kMergeStreamThreads) merge_stream_kernel(CallV
     thr = fmaxf(thr, s_thr2);
 
     // pass 2: keep the candidates at or above the threshold (order of arrival does not matter: the
-    // ranking below is by the total order (value desc, token id asc)).  A warp reads four lists at a time.
+    // ranking below is by the total order (value desc, token id asc)).  Only pieces whose first entry reaches
+    // the threshold can hold one; they are listed first, then all their entries are fetched at once.
     const int C = P * c.k_tokens;
     const int cap = (C <= smem_cands) ? smem_cands : cand_cap;
     float* cv = (C <= smem_cands) ? reinterpret_cast<float*>(msm) : cand_val_scratch + (size_t)m * cand_cap;
     int32_t* ci = (C <= smem_cands) ? reinterpret_cast<int32_t*>(msm + sizeof(float) * smem_cands)
                                     : cand_id_scratch + (size_t)m * cand_cap;
-    for (int q0 = warp * 4; q0 < P; q0 += kWarps * 4) {
+    for (int q = threadIdx.x; q < P; q += kMergeStreamThreads)
+        if (s_pm[q] != kNegInf && s_head[q] >= thr) s_live[atomicAdd(&s_nlive, 1)] = q;
+    __syncthreads();
+    const int n_entries = s_nlive * c.k_tokens;
+    for (int e0 = threadIdx.x; e0 < n_entries; e0 += 4 * kMergeStreamThreads) {
         float v[4];
         int id[4];
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
+            const int e = e0 + u * kMergeStreamThreads;
             v[u] = kNegInf;
             id[u] = kNoToken;
-            if (q0 + u < P && lane < c.k_tokens && s_pm[q0 + u] != kNegInf) {
-                const size_t p = (size_t)s_piece[q0 + u];
-                v[u] = pp.pval[p * c.k_tokens + lane] + s_off[s_pslot[q0 + u]];
-                id[u] = pp.pid[p * c.k_tokens + lane];
+            if (e < n_entries) {
+                const int q = s_live[e / c.k_tokens], l = e - (e / c.k_tokens) * c.k_tokens;
+                const size_t p = (size_t)s_piece[q];
+                v[u] = pp.pval[p * c.k_tokens + l] + s_off[s_pslot[q]];
+                id[u] = pp.pid[p * c.k_tokens + l];
             }
         }
 #pragma unroll

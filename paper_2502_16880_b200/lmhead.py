@@ -56,6 +56,7 @@ _SIGNATURES = {
     "coral_lmhead_set_group_shard": (_i, [_vp, _i, _i]),
     "coral_lmhead_draft_partial": (_i, [_vp, _vp, _i, _i, _i, _vp, _vp]),
     "coral_lmhead_merge_partials": (_i, [_vp, _i, _i, _i, _vp, _vp, _vp]),
+    "coral_lmhead_copy_floor": (_i, [_vp, ctypes.c_longlong, _vp]),
     "coral_lmhead_set_path": (_i, [_vp, _i]),
     "coral_lmhead_set_output_mode": (_i, [_vp, _i]),
     "coral_lmhead_set_router_mlp": (_i, [_vp, _vp, _vp]),
@@ -230,6 +231,11 @@ def coral_lmhead_set_router_mlp(handle, W1=None, stream=None) -> None:
     """W1: CUDA bf16 [H, H] tensor of Eq. 7's first router layer, or None for the single-matrix gate."""
     _check(load_library().coral_lmhead_set_router_mlp(handle, _dev_ptr(W1, torch.bfloat16), _stream_ptr(stream)),
            "coral_lmhead_set_router_mlp")
+
+
+def coral_lmhead_copy_floor(handle, nbytes: int, stream=None) -> None:
+    """Measurement aid: a do-nothing stream of the first `nbytes` of the packed head (time it with events)."""
+    _check(load_library().coral_lmhead_copy_floor(handle, int(nbytes), _stream_ptr(stream)), "coral_lmhead_copy_floor")
 
 
 def coral_lmhead_set_path(handle, path: int) -> None:

@@ -388,3 +388,17 @@ def test_adaptive_path_choice_on_device(M, kg, zipf, expect):
     for k in ("ids", "logprobs", "groups"):
         assert np.array_equal(out[k], again[k]), k
     head.close()
+
+
+def test_copy_floor_probe_runs_and_checks_arguments():
+    cfg, W, gm, Wg, hb = (synth.CONFIGS["tiny"],) + synth.make_all(synth.CONFIGS["tiny"])
+    head = _head(cfg, W, gm, Wg)
+    lib = lmhead.load_library()
+    packed_bytes, _ = lmhead.coral_lmhead_query_sizes(head.cfg)
+    lmhead.coral_lmhead_copy_floor(head.handle, packed_bytes)
+    lmhead.coral_lmhead_copy_floor(head.handle, 16384 * 3 + 5)
+    torch.cuda.synchronize()
+    assert head.status() == 0
+    assert lib.coral_lmhead_copy_floor(head.handle, 100, None) == lmhead.CORAL_ERR_INVALID
+    assert lib.coral_lmhead_copy_floor(head.handle, packed_bytes + 16384, None) == lmhead.CORAL_ERR_INVALID
+    head.close()
