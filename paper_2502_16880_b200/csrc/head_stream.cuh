@@ -120,6 +120,7 @@ struct StreamShared {
     uint64_t* zfree;          // [kStreamZBufs] all statistics warps have read the buffer
     int* segtab;              // [kStreamSegTab] union_list entries of this CTA's run
     volatile int* abort_flag;
+    volatile int* issued;     // slabs the producer has issued so far
     int lo, hi, j_first;      // this CTA's run of items and its first virtual group
 };
 
@@ -157,18 +158,20 @@ __device__ __forceinline__ void fold_item(float zv, const int32_t* __restrict__ 
 }
 
 // MMA side of one segment: items [lo, hi) of the run, all inside virtual group j = (group n, pass) with R
-// hidden rows.  NT n-tiles of 8 hidden rows; KBW k-blocks (32 columns) per warp per slab.
+// hidden rows.  NT n-tiles of 8 hidden rows.  A slab (16 vocab rows x kc columns) belongs to ONE warp: slab ks
+// of every item to warp ks % 8, which multiplies it with its own kc columns of the hidden rows (held in
+// registers) and frees the slot by itself, so the warps never wait for each other on the ring; their partial
+// sums meet in the item's z-buffer.  KBW = 2: kc = 512, one slab per warp and item; KBW = 1: kc = 256, up to two.
 template <int NT, int KBW>
 __device__ __forceinline__ void stream_segment_mma(const CallView& c, const StreamGeom& g, const StreamShared& sh,
-                                                   int n, int pass, int R, int lo, int hi, int& stage,
-                                                   uint32_t& phase, int& it) {
-    constexpr int KSMAX = 16 / KBW;
+                                                   int n, int pass, int R, int lo, int hi, int& it) {
+    constexpr int KBS = 8 * KBW;          // 32-column blocks per slab
+    constexpr int SL = 2 / KBW;           // slabs of an item this warp can own
     const int cw = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int gq = lane >> 2, tq = lane & 3;
     const int off = c.group_offset[n] + pass * kStreamPassRows;
-    const int col0 = (cw * KBW) * 32 + tq * 8;          // first column of this lane inside a slab
 
-    // B operands: hidden row (nt*8 + gq), the lane's 8 columns of every k-block of this warp
+    // B operands: hidden row (nt*8 + gq), the lane's 8 columns of every 32-column block of this warp's slabs
     uint4 breg[NT][16];
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) {
@@ -176,12 +179,13 @@ __device__ __forceinline__ void stream_segment_mma(const CallView& c, const Stre
         const bool valid = rr < R;
         const uint16_t* hp = c.hidden + (size_t)(valid ? c.bucket_row[off + rr] : 0) * c.H;
 #pragma unroll
-        for (int ks = 0; ks < KSMAX; ++ks)
+        for (int sl = 0; sl < SL; ++sl)
 #pragma unroll
-            for (int i = 0; i < KBW; ++i) {
+            for (int i = 0; i < KBS; ++i) {
+                const int ks = cw + kStreamWarps * sl;
                 uint4 hv = make_uint4(0, 0, 0, 0);
-                if (valid && ks < g.kstages) hv = __ldg(reinterpret_cast<const uint4*>(hp + ks * g.kc + col0 + i * 32));
-                breg[nt][ks * KBW + i] = hv;
+                if (valid && ks < g.kstages) hv = __ldg(reinterpret_cast<const uint4*>(hp + ks * g.kc + i * 32 + tq * 8));
+                breg[nt][sl * KBS + i] = hv;
             }
     }
     const uint32_t ring = smem_u32(sh.ring);
@@ -193,26 +197,38 @@ __device__ __forceinline__ void stream_segment_mma(const CallView& c, const Stre
 #pragma unroll
             for (int e = 0; e < 4; ++e) { acc[nt][0][e] = 0.f; acc[nt][1][e] = 0.f; }
 #pragma unroll
-        for (int ks = 0; ks < KSMAX; ++ks) {
+        for (int sl = 0; sl < SL; ++sl) {
+            const int ks = cw + kStreamWarps * sl;
             if (ks < g.kstages) {
-                mbar_wait(smem_u32(&sh.full[stage]), phase, sh.abort_flag, c.state);
+                const int idx = it * g.kstages + ks;            // position of the slab in the CTA's stream
+                const int stage = idx % g.n_stages;
+                // A warp may run several items ahead of the slowest one, i.e. more than one turn of the ring:
+                // the parity wait below is only meaningful once the slot's barrier has entered the phase of this
+                // very slab, which the producer announces after issuing its copy.
+                {
+                    const int limit = *sh.abort_flag ? kStreamSpinAfterAbort : kStreamSpin;
+                    int i = 0;
+                    while (*sh.issued <= idx && ++i < limit) {}
+                    if (*sh.issued <= idx) { *sh.abort_flag = 1; set_status(c.state, -5); }
+                    __threadfence_block();
+                }
+                mbar_wait(smem_u32(&sh.full[stage]), (uint32_t)(idx / g.n_stages) & 1u, sh.abort_flag, c.state);
                 const uint32_t sp = ring + (uint32_t)stage * g.stage_bytes;
 #pragma unroll
-                for (int i = 0; i < KBW; ++i) {
-                    const uint32_t cs = (uint32_t)(col0 + i * 32);             // column inside the slab
+                for (int i = 0; i < KBS; ++i) {
+                    const uint32_t cs = (uint32_t)(i * 32 + tq * 8);            // column inside the slab
                     const uint32_t at = sp + (cs >> 6) * 2048u + (uint32_t)gq * 128u + (cs & 63u) * 2u;
                     const uint4 wg = lds128(at);
                     const uint4 wh = lds128(at + 1024u);                        // row gq + 8
 #pragma unroll
                     for (int nt = 0; nt < NT; ++nt) {
-                        const uint4 b = breg[nt][ks * KBW + i];
+                        const uint4 b = breg[nt][sl * KBS + i];
                         mma_bf16_16816(acc[nt][0], wg.x, wh.x, wg.y, wh.y, b.x, b.y);
                         mma_bf16_16816(acc[nt][1], wg.z, wh.z, wg.w, wh.w, b.z, b.w);
                     }
                 }
                 __syncwarp();
                 if (lane == 0) mbar_arrive(smem_u32(&sh.empty[stage]));
-                if (++stage == g.n_stages) { stage = 0; phase ^= 1u; }
             }
         }
         // this warp's partial sums over its columns: rows gq, gq+8; hidden rows nt*8 + 2*tq, +1
@@ -315,6 +331,7 @@ __global__ void __launch_bounds__(kStreamThreads, 1) head_stream_kernel(CallView
     sh.segtab = reinterpret_cast<int*>(smem_raw + o);
     o += sizeof(int) * kStreamSegTab;
     sh.abort_flag = reinterpret_cast<volatile int*>(smem_raw + o);
+    sh.issued = sh.abort_flag + 1;
 
     pdl_wait();                   // the router stage's outputs are complete from here on
     pdl_launch_dependents();      // the merge kernel may start reading the router's outputs
@@ -330,13 +347,14 @@ __global__ void __launch_bounds__(kStreamThreads, 1) head_stream_kernel(CallView
     if (threadIdx.x == 0) {
         for (int s = 0; s < g.n_stages; ++s) {
             mbar_init(smem_u32(&sh.full[s]), 1);
-            mbar_init(smem_u32(&sh.empty[s]), kStreamWarps);
+            mbar_init(smem_u32(&sh.empty[s]), 1);           // a slab is read, and its slot freed, by one warp
         }
         for (int b = 0; b < kStreamZBufs; ++b) {
             mbar_init(smem_u32(&sh.zfull[b]), kStreamWarps);
             mbar_init(smem_u32(&sh.zfree[b]), kStreamStatWarps);
         }
         *sh.abort_flag = 0;
+        *sh.issued = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
@@ -347,7 +365,7 @@ __global__ void __launch_bounds__(kStreamThreads, 1) head_stream_kernel(CallView
     if (cw == kStreamWarps + kStreamStatWarps) {
         // producer: one contiguous copy per slab; a slab's valid rows are a prefix of its 16 rows
         if (lane != 0) return;
-        int stage = 0;
+        int stage = 0, n_issued = 0;
         uint32_t phase = 0;
         for (int pos = sh.lo; pos < sh.hi;) {
             const int j = pos / g.T;
@@ -362,6 +380,8 @@ __global__ void __launch_bounds__(kStreamThreads, 1) head_stream_kernel(CallView
                     const uint32_t bar = smem_u32(&sh.full[stage]);
                     mbar_expect_tx(bar, bytes);
                     bulk_g2s(smem_u32(sh.ring + (size_t)stage * g.stage_bytes), src, bytes, bar);
+                    __threadfence_block();
+                    *sh.issued = ++n_issued;      // the slot's barrier is now in the phase of this slab
                     src += (size_t)kStreamTile * g.kc;
                     if (++stage == g.n_stages) { stage = 0; phase ^= 1u; }
                 }
@@ -373,8 +393,7 @@ __global__ void __launch_bounds__(kStreamThreads, 1) head_stream_kernel(CallView
     const bool mma_role = cw < kStreamWarps;
 
     // both roles walk the run segment by segment (one virtual group each)
-    int stage = 0, it = 0;
-    uint32_t phase = 0;
+    int it = 0;
     for (int pos = sh.lo; pos < sh.hi;) {
         const int j = pos / g.T;
         const int seg = min(j - sh.j_first, kStreamSegTab - 1);
@@ -385,9 +404,9 @@ __global__ void __launch_bounds__(kStreamThreads, 1) head_stream_kernel(CallView
         if (!mma_role)
             stream_segment_stats(c, g, sh, pp, logits_tap, n, pass, R, j, pos, seg_hi, seg, it);
         else if (R <= 8)
-            stream_segment_mma<1, KBW>(c, g, sh, n, pass, R, pos, seg_hi, stage, phase, it);
+            stream_segment_mma<1, KBW>(c, g, sh, n, pass, R, pos, seg_hi, it);
         else
-            stream_segment_mma<2, KBW>(c, g, sh, n, pass, R, pos, seg_hi, stage, phase, it);
+            stream_segment_mma<2, KBW>(c, g, sh, n, pass, R, pos, seg_hi, it);
         pos = seg_hi;
     }
 }
