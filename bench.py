@@ -40,7 +40,7 @@ N_BATCHES = 8            # distinct hidden batches rotated through the steps
 # DRAM bytes per algorithmic byte of the dominant kernel, from the ncu capture summarised in
 # profiles/head_stream_kernel_llama3_M8.md ((read + write) / weight bytes of the touched groups, two launches).
 # Set to None whenever that kernel changes until the capture is redone.
-STREAM_TRAFFIC_RATIO = 1.016
+STREAM_TRAFFIC_RATIO = 1.015
 FLUSH_BYTES = 512 << 20  # > 2x the 126 MB L2: written, then read back, between timed steps
 
 
