@@ -216,6 +216,16 @@ int coral_lmhead_set_router_mlp(coral_lmhead_handle h, const void *W1_dev, void 
 int coral_lmhead_set_path(coral_lmhead_handle h, int path);
 
 /*
+ * Failure-detection self-test with no counterpart in the paper.  Every wait inside the kernels (on a ring
+ * slot, a statistics buffer, a tensor-memory buffer) polls a bounded number of times and, when the bound
+ * runs out, writes CORAL_ERR_TIMEOUT to the handle's status word and carries on to a normal exit.  This
+ * call launches a one-warp kernel that polls the same way (with a shorter bound) on a barrier nothing
+ * completes, so a caller can check that an expired wait is reported by coral_lmhead_status and leaves
+ * the handle and the context usable.  Asynchronous on `stream`; nothing faults, traps or spins unbounded.
+ */
+int coral_lmhead_selftest_wait_expiry(coral_lmhead_handle h, void *stream);
+
+/*
  * Measurement aid with no counterpart in the paper: streams the first `bytes` of the packed head into shared
  * memory with plain contiguous 16 KiB bulk copies (one CTA per SM, eight copies in flight each) and does
  * nothing with them.  Timed by the caller with events on `stream`, from a cold L2, it gives the floor for the

@@ -53,4 +53,21 @@ __global__ void __launch_bounds__(32) copy_probe_kernel(const unsigned char* __r
     sink[blockIdx.x] = acc;
 }
 
+// Failure-detection self-test: one warp polls, with the primitive every wait in the kernels is built on
+// (mbarrier.try_wait under an iteration bound), a barrier that nothing will ever complete.  The bound runs
+// out, the status word gets CORAL_ERR_TIMEOUT and the kernel returns normally: no trap, no endless loop, the
+// context stays usable.  (A shorter bound than the kernels' own, so that the test takes milliseconds.)
+constexpr int kSelfTestSpin = 1 << 14;
+__global__ void __launch_bounds__(32) wait_expiry_kernel(DeviceState* state) {
+    __shared__ uint64_t never;
+    if (threadIdx.x == 0) {
+        mbar_init(smem_u32(&never), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncwarp();
+    for (int i = 0; i < kSelfTestSpin; ++i)
+        if (mbar_try_wait(smem_u32(&never), 0)) return;
+    set_status(state, -5);
+}
+
 }  // namespace coral

@@ -679,6 +679,12 @@ int coral_lmhead_copy_floor(coral_lmhead_handle h, long long bytes, void* stream
     return cudaGetLastError() == cudaSuccess ? CORAL_OK : CORAL_ERR_CUDA;
 }
 
+int coral_lmhead_selftest_wait_expiry(coral_lmhead_handle h, void* stream) {
+    if (!h) return CORAL_ERR_INVALID;
+    wait_expiry_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(reinterpret_cast<DeviceState*>(h->ws + h->L.state));
+    return cudaGetLastError() == cudaSuccess ? CORAL_OK : CORAL_ERR_CUDA;
+}
+
 int coral_lmhead_set_output_mode(coral_lmhead_handle h, int mode) {
     if (!h || (mode != CORAL_OUTPUT_JOINT && mode != CORAL_OUTPUT_FACTORISED)) return CORAL_ERR_INVALID;
     h->out_mode = mode;

@@ -57,6 +57,7 @@ _SIGNATURES = {
     "coral_lmhead_draft_partial": (_i, [_vp, _vp, _i, _i, _i, _vp, _vp]),
     "coral_lmhead_merge_partials": (_i, [_vp, _i, _i, _i, _vp, _vp, _vp]),
     "coral_lmhead_copy_floor": (_i, [_vp, ctypes.c_longlong, _vp]),
+    "coral_lmhead_selftest_wait_expiry": (_i, [_vp, _vp]),
     "coral_lmhead_set_path": (_i, [_vp, _i]),
     "coral_lmhead_set_output_mode": (_i, [_vp, _i]),
     "coral_lmhead_set_router_mlp": (_i, [_vp, _vp, _vp]),
@@ -236,6 +237,12 @@ def coral_lmhead_set_router_mlp(handle, W1=None, stream=None) -> None:
 def coral_lmhead_copy_floor(handle, nbytes: int, stream=None) -> None:
     """Measurement aid: a do-nothing stream of the first `nbytes` of the packed head (time it with events)."""
     _check(load_library().coral_lmhead_copy_floor(handle, int(nbytes), _stream_ptr(stream)), "coral_lmhead_copy_floor")
+
+
+def coral_lmhead_selftest_wait_expiry(handle, stream=None) -> None:
+    """Runs the kernels' bounded wait on a barrier nothing completes; coral_lmhead_status then reports a timeout."""
+    _check(load_library().coral_lmhead_selftest_wait_expiry(handle, _stream_ptr(stream)),
+           "coral_lmhead_selftest_wait_expiry")
 
 
 def coral_lmhead_set_path(handle, path: int) -> None:

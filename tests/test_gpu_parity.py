@@ -402,3 +402,19 @@ def test_copy_floor_probe_runs_and_checks_arguments():
     assert lib.coral_lmhead_copy_floor(head.handle, 100, None) == lmhead.CORAL_ERR_INVALID
     assert lib.coral_lmhead_copy_floor(head.handle, packed_bytes + 16384, None) == lmhead.CORAL_ERR_INVALID
     head.close()
+
+
+def test_expired_wait_is_reported_and_the_handle_stays_usable():
+    """Failure detection without a fault: the kernels' bounded wait runs out on a barrier nothing completes,
+    the status word says so, and the next draft call on the same handle is correct."""
+    cfg = synth.CONFIGS["tiny"]
+    W, gm, Wg, hb = synth.make_all(cfg)
+    head = _head(cfg, W, gm, Wg)
+    lmhead.coral_lmhead_selftest_wait_expiry(head.handle)
+    assert head.status() == lmhead.CORAL_ERR_TIMEOUT
+    assert head.status() == 0                          # reading the status clears it
+    out = ph.gpu_draft_numpy(head, hb, cfg.k_groups, cfg.k_tokens)
+    assert head.status() == 0
+    rep = ph.compare(W, gm, Wg, hb, cfg.k_groups, cfg.k_tokens, out)
+    assert rep.ok, rep.errors
+    head.close()
