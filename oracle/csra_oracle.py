@@ -1,0 +1,64 @@
+"""CPU oracle of the Cross-Step Representation Alignment objective.  TEST INFRASTRUCTURE: only the tests and the
+bench's CPU-baseline leg may call it; it shares no code with the CUDA library and is never a fallback for it.
+
+What it computes (CORAL Section 3.1, Eq. 2; Appendix A: temperature 0.07; the appendix on discrepancies between
+training steps uses the same quantity between the features of two steps):
+
+    q_i  : n query features (the B x S output features of the current step), k_j : m = views * n key features
+           (the features of `views` other steps and/or the targets, block s holding positions 0 .. n-1),
+    sim  : cosine similarity, so every feature is first divided by its Euclidean norm,
+    loss_i = - mean over the views s of  log [ exp(sim(q_i, k_{i + s n}) / tau) / sum_j exp(sim(q_i, k_j) / tau) ]
+           = LSE_j(sim(q_i, k_j) / tau) - mean_s sim(q_i, k_{i + s n}) / tau,
+    loss   = mean_i loss_i.
+
+Readings (the paper leaves them open): which features make up the key set F is the caller's choice (whatever
+is passed as K); the positives of query i are the keys at the same position i in every block; several positives
+are averaged; a zero feature is left at zero.  Precision: the normalised features are rounded to bf16, the
+precision in which the contraction's operands are held (bf16 inputs, as everywhere in this library); everything
+else is float64 in the order written, with a plain matmul and a plain log-sum-exp.
+
+The paper prints InfoNCE values only for trained models on its own data, so value parity with the paper is
+unpinned; the function is pinned by closed forms, a library log-softmax, invariances and brute force
+(tests/test_csra_oracle_pins.py).
+"""
+from __future__ import annotations
+
+import numpy as np
+
+
+def _widen(bits: np.ndarray) -> np.ndarray:
+    return (np.ascontiguousarray(bits, dtype=np.uint16).astype(np.uint32) << np.uint32(16)).view(np.float32).astype(np.float64)
+
+
+def _round_to_bf16(x: np.ndarray) -> np.ndarray:
+    """float64 -> nearest bf16 (ties to even), returned as float64 values."""
+    f = np.ascontiguousarray(x, dtype=np.float64).astype(np.float32)      # exact enough: |x| <= 1, 24 bits kept first
+    u = f.view(np.uint32)
+    bias = ((u >> np.uint32(16)) & np.uint32(1)) + np.uint32(0x7FFF)
+    r = ((u + bias) >> np.uint32(16)).astype(np.uint32) << np.uint32(16)
+    return r.view(np.float32).astype(np.float64)
+
+
+def normalise(bits: np.ndarray) -> np.ndarray:
+    x = _widen(bits)
+    nrm = np.sqrt((x * x).sum(axis=1, keepdims=True))
+    with np.errstate(invalid="ignore", divide="ignore"):
+        y = np.where(nrm > 0, x / nrm, 0.0)
+    return _round_to_bf16(y)
+
+
+def infonce(Q_bits: np.ndarray, K_bits: np.ndarray, views: int, tau: float = 0.07):
+    """Q_bits [n, D], K_bits [views * n, D] (bf16 bit patterns).  Returns dict(logits [n, m], lse [n], pos [n, views],
+    row_loss [n], loss)."""
+    n = Q_bits.shape[0]
+    m = K_bits.shape[0]
+    if m != views * n or views < 1:
+        raise ValueError("K must hold views * n rows")
+    qn, kn = normalise(Q_bits), normalise(K_bits)
+    logits = (qn @ kn.T) / tau
+    mx = logits.max(axis=1)
+    lse = mx + np.log(np.exp(logits - mx[:, None]).sum(axis=1))
+    idx = np.arange(n)
+    pos = np.stack([logits[idx, idx + s * n] for s in range(views)], axis=1)
+    row_loss = lse - pos.mean(axis=1)
+    return {"logits": logits, "lse": lse, "pos": pos, "row_loss": row_loss, "loss": float(row_loss.mean())}
