@@ -216,6 +216,30 @@ int coral_lmhead_set_router_mlp(coral_lmhead_handle h, const void *W1_dev, void 
 int coral_lmhead_set_path(coral_lmhead_handle h, int path);
 
 /*
+ * Cross-Step Representation Alignment objective (Section 3.1, Eq. 2; temperature 0.07 in Appendix A; the same
+ * quantity between the features of two training steps in the appendix on step discrepancies), forward only:
+ *   loss_i = LSE_j( sim(q_i, k_j) / tau ) - mean_s sim(q_i, k_{i + s n}) / tau,   loss = mean_i loss_i,
+ * sim = cosine similarity.  Q_dev [n x D] bf16 row-major are the query features (the B x S output features of
+ * the current step), K_dev [views * n x D] bf16 the key set, block s holding the features at positions 0..n-1
+ * of another step or the targets; the positives of query i are the keys at position i of every block.  Which
+ * features form the key set is the caller's choice (the paper leaves it open).  Features are divided by their
+ * norms in fp32 and rounded to bf16; the n x m contraction runs on the tensor cores with fp32 accumulation and
+ * its epilogue keeps only (max, sum-exp) per row and the positives, so the similarity matrix is not stored.
+ *
+ * coral_csra_workspace_bytes: size of the caller-owned scratch for (n, views, D).
+ * coral_csra_infonce: workspace_dev 256-byte aligned, at least that size.  out_loss_dev [1] float;
+ *   out_row_loss_dev [n] float or NULL; out_logits_dev [n x views*n] float or NULL (the scaled similarities,
+ *   for checks on small cases).  n >= 1, 1 <= views <= 8, D a multiple of 8, tau > 0, else CORAL_ERR_INVALID.
+ *   Asynchronous on `stream`; no allocation.
+ * coral_csra_status: synchronises `stream` and returns the status word of the last call that used the
+ *   workspace (0 or CORAL_ERR_TIMEOUT).
+ */
+int coral_csra_workspace_bytes(int n, int views, int D, size_t *bytes);
+int coral_csra_infonce(const void *Q_dev, const void *K_dev, int n, int views, int D, float tau, void *workspace_dev,
+                       float *out_row_loss_dev, float *out_loss_dev, float *out_logits_dev, void *stream);
+int coral_csra_status(void *workspace_dev, void *stream);
+
+/*
  * Failure-detection self-test with no counterpart in the paper.  Every wait inside the kernels (on a ring
  * slot, a statistics buffer, a tensor-memory buffer) polls a bounded number of times and, when the bound
  * runs out, writes CORAL_ERR_TIMEOUT to the handle's status word and carries on to a normal exit.  This

@@ -13,9 +13,10 @@ training steps uses the same quantity between the features of two steps):
 
 Readings (the paper leaves them open): which features make up the key set F is the caller's choice (whatever
 is passed as K); the positives of query i are the keys at the same position i in every block; several positives
-are averaged; a zero feature is left at zero.  Precision: the normalised features are rounded to bf16, the
-precision in which the contraction's operands are held (bf16 inputs, as everywhere in this library); everything
-else is float64 in the order written, with a plain matmul and a plain log-sum-exp.
+are averaged; a zero feature is left at zero.  Precision: the normalised features are rounded to bf16 (one
+rounding of the float64 quotient, nearest-even), the precision in which the contraction's operands are held
+(bf16 inputs, as everywhere in this library); everything else is float64 in the order written, with a plain
+matmul and a plain log-sum-exp.
 
 The paper prints InfoNCE values only for trained models on its own data, so value parity with the paper is
 unpinned; the function is pinned by closed forms, a library log-softmax, invariances and brute force
@@ -31,12 +32,12 @@ def _widen(bits: np.ndarray) -> np.ndarray:
 
 
 def _round_to_bf16(x: np.ndarray) -> np.ndarray:
-    """float64 -> nearest bf16 (ties to even), returned as float64 values."""
-    f = np.ascontiguousarray(x, dtype=np.float64).astype(np.float32)      # exact enough: |x| <= 1, 24 bits kept first
-    u = f.view(np.uint32)
-    bias = ((u >> np.uint32(16)) & np.uint32(1)) + np.uint32(0x7FFF)
-    r = ((u + bias) >> np.uint32(16)).astype(np.uint32) << np.uint32(16)
-    return r.view(np.float32).astype(np.float64)
+    """float64 -> nearest bf16 (ties to even) in one rounding, returned as float64 values.  bf16 keeps 7 of the
+    52 fraction bits of a double; values here lie in (2^-100, 1], far inside bf16's exponent range."""
+    u = np.ascontiguousarray(x, dtype=np.float64).view(np.uint64)
+    keep_lsb = (u >> np.uint64(45)) & np.uint64(1)
+    r = ((u + np.uint64((1 << 44) - 1) + keep_lsb) >> np.uint64(45)) << np.uint64(45)
+    return r.view(np.float64)
 
 
 def normalise(bits: np.ndarray) -> np.ndarray:

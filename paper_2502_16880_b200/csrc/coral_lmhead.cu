@@ -12,6 +12,7 @@
 #include "head_stream.cuh"
 #include "head_tc.cuh"
 #include "copy_probe.cuh"
+#include "csra.cuh"
 #include "merge.cuh"
 #include "route.cuh"
 #include "tree.cuh"
@@ -677,6 +678,102 @@ int coral_lmhead_copy_floor(coral_lmhead_handle h, long long bytes, void* stream
         h->packed, bytes / kCopyChunk, reinterpret_cast<DeviceState*>(h->ws + h->L.state),
         reinterpret_cast<unsigned*>(h->ws + h->L.cand_val));
     return cudaGetLastError() == cudaSuccess ? CORAL_OK : CORAL_ERR_CUDA;
+}
+
+// ---- CSRA objective (Eq. 2) -------------------------------------------------------------------------------
+namespace {
+struct CsraLayout {
+    size_t state, qn, kn, pmax, psum, pos, row_loss, total;
+    int RB, KT, KB;
+};
+CsraLayout csra_layout(int n, int views, int D) {
+    CsraLayout L{};
+    L.RB = (n + 127) / 128;
+    L.KT = (int)(((long long)n * views + 127) / 128);
+    L.KB = (D + 63) / 64;
+    size_t o = 0;
+    auto take = [&](size_t bytes) { size_t at = o; o = align_up(o + bytes); return at; };
+    L.state = take(sizeof(DeviceState));
+    L.qn = take((size_t)L.RB * L.KB * 128 * 64 * 2);
+    L.kn = take((size_t)L.KT * L.KB * 128 * 64 * 2);
+    L.pmax = take((size_t)L.RB * L.KT * 128 * 4);
+    L.psum = take((size_t)L.RB * L.KT * 128 * 4);
+    L.pos = take((size_t)n * views * 4);
+    L.row_loss = take((size_t)n * 4);
+    L.total = o;
+    return L;
+}
+bool csra_args_ok(int n, int views, int D) {
+    return n >= 1 && views >= 1 && views <= kCsraMaxViews && D >= 8 && D % 8 == 0 && (long long)n * views <= (1 << 24) &&
+           D <= (1 << 16);
+}
+}  // namespace
+
+int coral_csra_workspace_bytes(int n, int views, int D, size_t* bytes) {
+    if (!bytes || !csra_args_ok(n, views, D)) return CORAL_ERR_INVALID;
+    *bytes = csra_layout(n, views, D).total;
+    return CORAL_OK;
+}
+
+int coral_csra_infonce(const void* Q_dev, const void* K_dev, int n, int views, int D, float tau, void* workspace_dev,
+                       float* out_row_loss_dev, float* out_loss_dev, float* out_logits_dev, void* stream) {
+    if (!Q_dev || !K_dev || !workspace_dev || !out_loss_dev || !csra_args_ok(n, views, D) || !(tau > 0.f))
+        return CORAL_ERR_INVALID;
+    if (reinterpret_cast<uintptr_t>(workspace_dev) & 255) return CORAL_ERR_INVALID;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const CsraLayout L = csra_layout(n, views, D);
+    unsigned char* ws = static_cast<unsigned char*>(workspace_dev);
+    int dev = 0, sms = 0, smem_optin = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess)
+        return CORAL_ERR_CUDA;
+    if ((int)kTcSmemBytes > smem_optin) return CORAL_ERR_INVALID;
+    EncodeTiledFn enc = encode_tiled_fn();
+    if (!enc) return CORAL_ERR_CUDA;
+    CUtensorMap map_q, map_k;
+    {
+        const cuuint64_t qdim[2] = {(cuuint64_t)kTcK, (cuuint64_t)L.RB * L.KB * 128};
+        const cuuint64_t kdim[2] = {(cuuint64_t)kTcK, (cuuint64_t)L.KT * L.KB * 128};
+        const cuuint64_t str[1] = {(cuuint64_t)kTcK * 2};
+        const cuuint32_t box[2] = {(cuuint32_t)kTcK, 128};
+        const cuuint32_t ones[2] = {1, 1};
+        if (enc(&map_q, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, ws + L.qn, qdim, str, box, ones, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) !=
+                CUDA_SUCCESS ||
+            enc(&map_k, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, ws + L.kn, kdim, str, box, ones, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) !=
+                CUDA_SUCCESS)
+            return CORAL_ERR_CUDA;
+    }
+    if (cudaFuncSetAttribute(csra_sim_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTcSmemBytes) != cudaSuccess)
+        return CORAL_ERR_CUDA;
+    if (cudaMemsetAsync(ws + L.state, 0, sizeof(DeviceState), st) != cudaSuccess) return CORAL_ERR_CUDA;
+    CsraGeom g{};
+    g.n = n; g.views = views; g.m = n * views; g.D = D;
+    g.RB = L.RB; g.KT = L.KT; g.ksteps = L.KB; g.grid = sms; g.inv_tau = 1.0f / tau;
+    uint16_t* qn = reinterpret_cast<uint16_t*>(ws + L.qn);
+    uint16_t* kn = reinterpret_cast<uint16_t*>(ws + L.kn);
+    float* row_loss = out_row_loss_dev ? out_row_loss_dev : reinterpret_cast<float*>(ws + L.row_loss);
+    csra_normalise_kernel<<<L.RB * 128, 128, 0, st>>>(static_cast<const uint16_t*>(Q_dev), n, D, L.KB, qn);
+    csra_normalise_kernel<<<L.KT * 128, 128, 0, st>>>(static_cast<const uint16_t*>(K_dev), g.m, D, L.KB, kn);
+    csra_sim_kernel<<<g.grid, kTcThreads, kTcSmemBytes, st>>>(
+        g, map_q, map_k, reinterpret_cast<float*>(ws + L.pmax), reinterpret_cast<float*>(ws + L.psum),
+        reinterpret_cast<float*>(ws + L.pos), out_logits_dev, reinterpret_cast<DeviceState*>(ws + L.state));
+    csra_finalize_kernel<<<(n + 255) / 256, 256, 0, st>>>(g, reinterpret_cast<const float*>(ws + L.pmax),
+                                                          reinterpret_cast<const float*>(ws + L.psum),
+                                                          reinterpret_cast<const float*>(ws + L.pos), row_loss);
+    csra_mean_kernel<<<1, 1024, 0, st>>>(row_loss, n, out_loss_dev);
+    return cudaGetLastError() == cudaSuccess ? CORAL_OK : CORAL_ERR_CUDA;
+}
+
+int coral_csra_status(void* workspace_dev, void* stream) {
+    if (!workspace_dev) return CORAL_ERR_INVALID;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    DeviceState s{};
+    if (cudaMemcpyAsync(&s, workspace_dev, sizeof s, cudaMemcpyDeviceToHost, st) != cudaSuccess) return CORAL_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return CORAL_ERR_CUDA;
+    return s.status;
 }
 
 int coral_lmhead_selftest_wait_expiry(coral_lmhead_handle h, void* stream) {

@@ -1,0 +1,293 @@
+// Cross-Step Representation Alignment objective (CORAL Section 3.1, Eq. 2): InfoNCE over cosine similarities,
+//   loss_i = LSE_j( q^_i . k^_j / tau ) - mean_s ( q^_i . k^_{i + s n} / tau ),   loss = mean_i loss_i,
+// n query features, m = views * n key features, q^ and k^ the features divided by their norms.
+//
+// Three steps: (1) csra_normalise_kernel divides every feature by its norm (float64) and stores it as bf16 in
+// blocks of 128 rows x 64 columns (one contiguous 16 KiB operand tile per block); (2) csra_sim_kernel is a
+// dense n x m x D contraction on the 5th-generation tensor cores with the structure of head_tc_kernel (TMA
+// tiled loads in a 4-stage ring, tcgen05.mma with M = 128 query rows x N = 128 key rows per accumulator, two
+// key tiles per batch sharing the query tile, accumulators double-buffered in tensor memory) whose epilogue
+// folds the scaled similarities into a running (max, sum-exp) per query row and picks out the positives, so
+// the n x m similarity matrix never reaches HBM; (3) csra_finalize_kernel combines the partials per row and
+// csra_mean_kernel averages the rows in a fixed order.
+#pragma once
+#include "head_tc.cuh"
+
+namespace coral {
+
+constexpr int kCsraMaxViews = 8;
+
+struct CsraGeom {
+    int n, m, views, D;
+    int RB, KT;        // query row blocks, key tiles (of 128 rows)
+    int ksteps;        // 64-column blocks = ceil(D / 64)
+    int grid;
+    float inv_tau;
+};
+
+// One block per feature row: x / ||x||, rounded to bf16, into the blocked layout
+// out[row block][column block][128 rows][64 columns]; columns past D are zero, and the blocks past the last row
+// write zero rows, so that every operand tile is defined.  The rounding to bf16 decides which of two
+// neighbouring operand values the contraction sees, so it is taken from a float64 quotient (norm and division
+// in float64): whoever repeats it in float64 lands on the same side of the rounding boundary.
+__device__ __forceinline__ uint16_t csra_round_bf16(double y) {
+    float f = __double2float_rz(y);                     // truncate, then make the dropped bits sticky (round to odd):
+    if ((double)f != y) f = __uint_as_float(__float_as_uint(f) | 1u);   // the final rounding then sees the exact value's side
+    uint32_t u = __float_as_uint(f);
+    u = (u + 0x7FFFu + ((u >> 16) & 1u)) >> 16;         // nearest, ties to even
+    return (uint16_t)u;
+}
+
+__global__ void __launch_bounds__(128) csra_normalise_kernel(const uint16_t* __restrict__ x, int rows, int D, int KB,
+                                                             uint16_t* __restrict__ out) {
+    __shared__ double s_part[4];
+    const int row = blockIdx.x;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    double ss = 0.0;
+    if (row < rows)
+        for (int i = threadIdx.x; i < D; i += 128) {
+            const double v = (double)__uint_as_float((uint32_t)x[(size_t)row * D + i] << 16);
+            ss += v * v;
+        }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+    if (lane == 0) s_part[warp] = ss;
+    __syncthreads();
+    ss = (s_part[0] + s_part[1]) + (s_part[2] + s_part[3]);
+    const double nrm = sqrt(ss);
+    uint16_t* dst = out + ((size_t)(row >> 7) * KB * 128 + (row & 127)) * 64;
+    for (int i = threadIdx.x; i < KB * 64; i += 128) {
+        uint16_t r = 0;
+        if (row < rows && i < D && nrm > 0.0)
+            r = csra_round_bf16((double)__uint_as_float((uint32_t)x[(size_t)row * D + i] << 16) / nrm);
+        dst[(size_t)(i >> 6) * 128 * 64 + (i & 63)] = r;
+    }
+}
+
+struct CsraRowState {
+    float mx, sum;
+    __device__ __forceinline__ void reset() { mx = kNegInf; sum = 0.f; }
+};
+
+// Epilogue of one 128 x 128 accumulator for one thread (= one query row): scale by 1 / tau, fold the
+// similarities to key rows [base, base + 128) into the running (max, sum-exp), store the positives.
+__device__ __forceinline__ void csra_fold_row(const CsraGeom& g, CsraRowState& st, uint32_t tmem_acc_row, int row,
+                                              int base, bool row_valid, float* __restrict__ out_pos,
+                                              float* __restrict__ logits_tap) {
+    constexpr float kLog2e = 1.4426950408889634f;
+    const int valid = min(kTcSub, g.m - base);
+#pragma unroll 1
+    for (int ch = 0; ch < 4; ++ch) {
+        float z[32];
+        tc_ld32(tmem_acc_row + (uint32_t)(ch * 32), z);
+        const int nv = min(32, valid - ch * 32);
+        if (!row_valid || nv <= 0) continue;
+#pragma unroll
+        for (int i = 0; i < 32; ++i) z[i] *= g.inv_tau;
+        float cm = kNegInf;
+#pragma unroll
+        for (int i = 0; i < 32; ++i) cm = fmaxf(cm, i < nv ? z[i] : kNegInf);
+        const float nm = fmaxf(st.mx, cm);
+        float add = 0.f;
+#pragma unroll
+        for (int i = 0; i < 32; ++i) add += i < nv ? exp2f((z[i] - nm) * kLog2e) : 0.f;
+        st.sum = st.sum * exp2f((st.mx - nm) * kLog2e) + add;
+        st.mx = nm;
+        if (logits_tap) {
+            float* dst = logits_tap + (size_t)row * g.m + base + ch * 32;
+#pragma unroll
+            for (int i = 0; i < 32; ++i)
+                if (i < nv) dst[i] = z[i];
+        }
+        // positives of this row: key row + s * n, s = 0 .. views - 1
+        for (int s = 0; s < g.views; ++s) {
+            const int col = row + s * g.n - base - ch * 32;
+            if (col >= 0 && col < nv) {
+                float v = 0.f;
+#pragma unroll
+                for (int i = 0; i < 32; ++i) v = i == col ? z[i] : v;
+                out_pos[(size_t)row * g.views + s] = v;
+            }
+        }
+    }
+}
+
+// grid = g.grid CTAs of kTcThreads threads; the list of (row block, key tile) positions is cut into
+// contiguous runs, one per CTA.  Partials pmax / psum: [row block * KT + key tile][128 rows]; of the key
+// tiles an epilogue warp set sees of a row block inside the run, the last one carries its running partial
+// and the others an empty marker (max = -inf, sum = 0).
+__global__ void __launch_bounds__(kTcThreads, 1)
+    csra_sim_kernel(CsraGeom g, const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
+                    float* __restrict__ pmax, float* __restrict__ psum, float* __restrict__ out_pos,
+                    float* __restrict__ logits_tap, DeviceState* state) {
+    extern __shared__ unsigned char tc_smem_raw[];
+    unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(tc_smem_raw) + 1023) & ~(uintptr_t)1023);
+    uint64_t* full = reinterpret_cast<uint64_t*>(smem + kTcStages * kTcStageBytes);
+    uint64_t* empty = full + kTcStages;
+    uint64_t* tmem_full = empty + kTcStages;      // [2]
+    uint64_t* tmem_empty = tmem_full + 2;         // [2]
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tmem_empty + 2);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kTcStages; ++s) {
+            mbar_init(smem_u32(&full[s]), 1);
+            mbar_init(smem_u32(&empty[s]), 1);
+        }
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(smem_u32(&tmem_full[s]), 1);
+            mbar_init(smem_u32(&tmem_empty[s]), kTcEpilogueWarps);
+        }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                     "r"(kTcTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    const int n_pos = g.RB * g.KT;
+    const int per = (n_pos + g.grid - 1) / g.grid;
+    const int lo = min(n_pos, (int)blockIdx.x * per);
+    const int hi = min(n_pos, lo + per);
+    // a batch = two key tiles of one row block (one at the end of a row block or of the run)
+    auto nsub_at = [&](int pos) { return ((pos % g.KT) + 1 < g.KT && pos + 1 < hi) ? 2 : 1; };
+
+    if (warp == 0) {
+        if (lane == 0) {
+            int stage = 0;
+            uint32_t phase = 0;
+            const uint64_t pol_first = l2_policy_evict_first(), pol_last = l2_policy_evict_last();
+            for (int pos = lo; pos < hi;) {
+                const int rb = pos / g.KT, kt = pos - rb * g.KT, nsub = nsub_at(pos);
+                const uint32_t bytes = (uint32_t)(1 + nsub) * kTcTileBytes;
+                for (int ks = 0; ks < g.ksteps; ++ks) {
+                    tc_wait(smem_u32(&empty[stage]), phase ^ 1u, abort_flag, state);
+                    const uint32_t bar = smem_u32(&full[stage]);
+                    const uint32_t sb = smem_u32(smem + (size_t)stage * kTcStageBytes);
+                    mbar_expect_tx(bar, bytes);
+                    tma_load_2d(sb, &map_q, 0, (rb * g.ksteps + ks) * 128, bar, pol_last);
+                    for (int sub = 0; sub < nsub; ++sub)
+                        tma_load_2d(sb + (1 + sub) * kTcTileBytes, &map_k, 0, ((kt + sub) * g.ksteps + ks) * 128, bar,
+                                    pol_first);
+                    if (++stage == kTcStages) { stage = 0; phase ^= 1u; }
+                }
+                pos += nsub;
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            int stage = 0, batch = 0;
+            uint32_t phase = 0;
+            for (int pos = lo; pos < hi; ++batch) {
+                const int nsub = nsub_at(pos);
+                const int buf = batch & 1;
+                tc_wait(smem_u32(&tmem_empty[buf]), (((uint32_t)batch >> 1) & 1u) ^ 1u, abort_flag, state);
+                tc_fence_after();
+                const uint32_t acc = tmem_base + (uint32_t)(buf * 2 * kTcSub);
+                for (int ks = 0; ks < g.ksteps; ++ks) {
+                    tc_wait(smem_u32(&full[stage]), phase, abort_flag, state);
+                    tc_fence_after();
+                    const uint32_t sb = smem_u32(smem + (size_t)stage * kTcStageBytes);
+#pragma unroll
+                    for (int kk = 0; kk < kTcK / 16; ++kk) {
+                        const uint64_t adesc = tc_smem_desc(sb + kk * 32);
+                        for (int sub = 0; sub < nsub; ++sub) {
+                            const uint64_t bdesc = tc_smem_desc(sb + (1 + sub) * kTcTileBytes + kk * 32);
+                            tc_mma(acc + (uint32_t)(sub * kTcSub), adesc, bdesc, (ks | kk) ? 1u : 0u);
+                        }
+                    }
+                    tc_commit(smem_u32(&empty[stage]));
+                    if (++stage == kTcStages) { stage = 0; phase ^= 1u; }
+                }
+                tc_commit(smem_u32(&tmem_full[buf]));
+                pos += nsub;
+            }
+        }
+    } else {
+        const int quarter = warp & 3;
+        const int which = (warp - 2) >> 2;
+        const int row_in_block = quarter * 32 + lane;
+        CsraRowState st;
+        st.reset();
+        int batch = 0;
+        for (int pos = lo; pos < hi; ++batch) {
+            const int rb = pos / g.KT, kt = pos - rb * g.KT, nsub = nsub_at(pos);
+            const int buf = batch & 1;
+            tc_wait(smem_u32(&tmem_full[buf]), ((uint32_t)batch >> 1) & 1u, abort_flag, state);
+            tc_fence_after();
+            if (which < nsub) {
+                const int row = rb * 128 + row_in_block;
+                const bool row_valid = row < g.n;
+                const size_t pidx = ((size_t)rb * g.KT + kt + which) * 128 + row_in_block;
+                const uint32_t acc_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)((buf * 2 + which) * kTcSub);
+                csra_fold_row(g, st, acc_row, row, (kt + which) * kTcSub, row_valid, out_pos, logits_tap);
+                const int npos = pos + nsub;
+                bool last = npos >= hi || npos / g.KT != rb;
+                if (!last && which == 1) {
+                    const int nt = npos - rb * g.KT;
+                    last = nt + 1 >= g.KT || npos + 1 >= hi;      // the next batch is a single key tile
+                }
+                if (row_valid) {
+                    pmax[pidx] = last ? st.mx : kNegInf;
+                    psum[pidx] = last ? st.sum : 0.f;
+                }
+                if (last) st.reset();
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&tmem_empty[buf]));
+            pos += nsub;
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTcTmemCols) : "memory");
+    }
+}
+
+// One thread per query row: log-sum-exp over the row's KT partials, minus the mean of its positives.
+__global__ void __launch_bounds__(256) csra_finalize_kernel(CsraGeom g, const float* __restrict__ pmax,
+                                                            const float* __restrict__ psum,
+                                                            const float* __restrict__ pos,
+                                                            float* __restrict__ out_row_loss) {
+    const int row = blockIdx.x * 256 + threadIdx.x;
+    if (row >= g.n) return;
+    const size_t p0 = (size_t)(row >> 7) * g.KT * 128 + (row & 127);
+    float mx = kNegInf;
+    for (int t = 0; t < g.KT; ++t) mx = fmaxf(mx, pmax[p0 + (size_t)t * 128]);
+    float sum = 0.f;
+    for (int t = 0; t < g.KT; ++t) {
+        const float a = pmax[p0 + (size_t)t * 128];
+        if (a != kNegInf) sum += psum[p0 + (size_t)t * 128] * expf(a - mx);
+    }
+    float pm = 0.f;
+    for (int s = 0; s < g.views; ++s) pm += pos[(size_t)row * g.views + s];
+    out_row_loss[row] = mx + logf(sum) - pm / (float)g.views;
+}
+
+// Mean of the n row losses by one block, in a fixed order (bitwise reproducible).
+__global__ void __launch_bounds__(1024) csra_mean_kernel(const float* __restrict__ row_loss, int n, float* __restrict__ out) {
+    __shared__ float s_part[32];
+    float acc = 0.f;
+    for (int i = threadIdx.x; i < n; i += 1024) acc += row_loss[i];
+    acc = warp_sum(acc);
+    if ((threadIdx.x & 31) == 0) s_part[threadIdx.x >> 5] = acc;
+    __syncthreads();
+    if (threadIdx.x < 32) {
+        float v = s_part[threadIdx.x];
+        v = warp_sum(v);
+        if (threadIdx.x == 0) out[0] = v / (float)n;
+    }
+}
+
+}  // namespace coral

@@ -57,6 +57,9 @@ _SIGNATURES = {
     "coral_lmhead_draft_partial": (_i, [_vp, _vp, _i, _i, _i, _vp, _vp]),
     "coral_lmhead_merge_partials": (_i, [_vp, _i, _i, _i, _vp, _vp, _vp]),
     "coral_lmhead_copy_floor": (_i, [_vp, ctypes.c_longlong, _vp]),
+    "coral_csra_workspace_bytes": (_i, [_i, _i, _i, ctypes.POINTER(ctypes.c_size_t)]),
+    "coral_csra_infonce": (_i, [_vp, _vp, _i, _i, _i, ctypes.c_float, _vp, _vp, _vp, _vp, _vp]),
+    "coral_csra_status": (_i, [_vp, _vp]),
     "coral_lmhead_selftest_wait_expiry": (_i, [_vp, _vp]),
     "coral_lmhead_set_path": (_i, [_vp, _i]),
     "coral_lmhead_set_output_mode": (_i, [_vp, _i]),
@@ -237,6 +240,29 @@ def coral_lmhead_set_router_mlp(handle, W1=None, stream=None) -> None:
 def coral_lmhead_copy_floor(handle, nbytes: int, stream=None) -> None:
     """Measurement aid: a do-nothing stream of the first `nbytes` of the packed head (time it with events)."""
     _check(load_library().coral_lmhead_copy_floor(handle, int(nbytes), _stream_ptr(stream)), "coral_lmhead_copy_floor")
+
+
+def coral_csra_workspace_bytes(n: int, views: int, D: int) -> int:
+    b = ctypes.c_size_t(0)
+    _check(load_library().coral_csra_workspace_bytes(int(n), int(views), int(D), ctypes.byref(b)), "coral_csra_workspace_bytes")
+    return int(b.value)
+
+
+def coral_csra_infonce(Q, K, views, tau, workspace, out_loss, out_row_loss=None, out_logits=None, stream=None):
+    """Q [n, D], K [views * n, D] CUDA bf16; workspace: CUDA uint8 tensor of coral_csra_workspace_bytes(n, views, D);
+    out_loss [1] f32, out_row_loss [n] f32 or None, out_logits [n, views * n] f32 or None."""
+    n, D = Q.shape
+    if K.shape[0] != int(views) * n or K.shape[1] != D:
+        raise ValueError("K must be [views * n, D]")
+    _check(load_library().coral_csra_infonce(
+        _dev_ptr(Q, torch.bfloat16, False), _dev_ptr(K, torch.bfloat16, False), n, int(views), D, float(tau),
+        _dev_ptr(workspace, torch.uint8, False), _dev_ptr(out_row_loss, torch.float32),
+        _dev_ptr(out_loss, torch.float32, False), _dev_ptr(out_logits, torch.float32), _stream_ptr(stream)),
+        "coral_csra_infonce")
+
+
+def coral_csra_status(workspace, stream=None) -> int:
+    return int(load_library().coral_csra_status(_dev_ptr(workspace, torch.uint8, False), _stream_ptr(stream)))
 
 
 def coral_lmhead_selftest_wait_expiry(handle, stream=None) -> None:

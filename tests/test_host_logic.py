@@ -27,7 +27,7 @@ def lib():
 def test_library_exports_every_declared_symbol(lib):
     header = open(os.path.join(ROOT, "include", "coral_lmhead.h")).read()
     header = re.sub(r"/\*.*?\*/", "", header, flags=re.S)
-    declared = set(re.findall(r"\b(coral_(?:lmhead|tree)_[a-z0-9_]+)\s*\(", header))
+    declared = set(re.findall(r"\b(coral_(?:lmhead|tree|csra)_[a-z0-9_]+)\s*\(", header))
     assert {"coral_lmhead_create", "coral_lmhead_draft", "coral_lmhead_draft_ex", "coral_lmhead_destroy"} <= declared
     for name in declared:
         assert hasattr(lib, name), name
