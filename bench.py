@@ -534,6 +534,48 @@ def main():
             "torch_dense_gemm_960xVxH_us": float(np.mean(tg)) * 1e3,
         }
         big.close()
+        # extra (second workload, training side): the CSRA objective of Eq. 2 on synthetic features - 4096
+        # positions, keys = three other steps and the targets, D = 4096 - a tensor-bound contraction
+        n_c, v_c, D_c = 4096, 4, cfg.H
+        rng_c = np.random.default_rng([cfg.seed, 77])
+        base_c = rng_c.standard_normal((n_c, D_c), dtype=np.float32)
+        Qc = dev_bf16(synth.fp32_to_bf16_bits(0.6 * base_c + 0.8 * rng_c.standard_normal((n_c, D_c), dtype=np.float32)))
+        Kc = torch.cat([dev_bf16(synth.fp32_to_bf16_bits(0.6 * base_c + 0.8 * rng_c.standard_normal((n_c, D_c), dtype=np.float32)))
+                        for _ in range(v_c)])
+        ws_c = torch.empty(lmhead.coral_csra_workspace_bytes(n_c, v_c, D_c), dtype=torch.uint8, device=dev)
+        loss_c = torch.empty(1, dtype=torch.float32, device=dev)
+        tc_, tt_ = [], []
+        for i in range(8):
+            flush_l2(i)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            lmhead.coral_csra_infonce(Qc, Kc, v_c, 0.07, ws_c, loss_c, stream=stream)
+            b.record(stream)
+            torch.cuda.synchronize()
+            if i >= 3:
+                tc_.append(a.elapsed_time(b))
+        assert lmhead.coral_csra_status(ws_c) == 0
+        for i in range(8):          # comparator: the same objective with torch ops (bf16 matmul, fp32 softmax)
+            flush_l2(i)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            qn_ = torch.nn.functional.normalize(Qc.float(), dim=1).to(torch.bfloat16)
+            kn_ = torch.nn.functional.normalize(Kc.float(), dim=1).to(torch.bfloat16)
+            lg_ = torch.matmul(qn_, kn_.T).float() / 0.07
+            idx_ = torch.arange(n_c, device=dev)
+            pos_ = torch.stack([lg_[idx_, idx_ + s_ * n_c] for s_ in range(v_c)], 1).mean(1)
+            loss_t = (torch.logsumexp(lg_, dim=1) - pos_).mean()
+            b.record()
+            torch.cuda.synchronize()
+            if i >= 3:
+                tt_.append(a.elapsed_time(b))
+        fl_c = 2.0 * n_c * (n_c * v_c) * D_c
+        out["csra_infonce"] = {"n": n_c, "views": v_c, "D": D_c, "us": float(np.mean(tc_)) * 1e3,
+                               "tflops": fl_c / (float(np.mean(tc_)) * 1e-3) / 1e12,
+                               "tensor_frac_of_sustained_peak": fl_c / (float(np.mean(tc_)) * 1e-3) / 1e12 / tf_sust,
+                               "loss": float(loss_c.item()), "torch_ops_us": float(np.mean(tt_)) * 1e3,
+                               "torch_ops_loss": float(loss_t.item())}
+        del Qc, Kc, ws_c
         out["clocks"] = sampler.stop()
         # CPU oracle on the host cores: whole steps of the same workload, bounded
         o_steps = 3
