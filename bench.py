@@ -456,7 +456,11 @@ def main():
             ms_za, _, _, _, _ = time_steps(M, cfg.k_groups, extra_steps, 3, my_batches, zipf_s=1.5, on=zhead)
             took_z = int(zhead.stats().path)
             zhead.set_path(lmhead.CORAL_PATH_AUTO)
+            lmhead.coral_lmhead_set_hot_groups(zhead.handle, 4)     # the four most frequent groups stay in L2
+            ms_zh, _, _, _, _ = time_steps(M, cfg.k_groups, extra_steps, 3, my_batches, zipf_s=1.5, on=zhead)
+            lmhead.coral_lmhead_set_hot_groups(zhead.handle, 0)
             zleg.append({"M": M, "us_per_step": float(np.mean(ms_z)) * 1e3, "groups_touched_mean": float(np.mean(t_z)),
+                         "hot4_persisting_us_per_step": float(np.mean(ms_zh)) * 1e3,
                          "GBps": b_z / (float(np.mean(ms_z)) * 1e-3) / 1e9,
                          "adaptive_us_per_step": float(np.mean(ms_za)) * 1e3, "adaptive_path": took_z})
         assert zhead.status() == 0

@@ -165,6 +165,7 @@ struct coral_lmhead_s {
     bool tc_ok;          // tensor-core path available (maps encoded)
     int out_mode;        // CORAL_OUTPUT_*
     int shard_rank, shard_world;   // vocab sharding (coral_lmhead_set_group_shard); world 1 = off
+    int hot_groups;                // leading groups whose weights are loaded with an evict-last L2 hint (0 = off)
     uint16_t* w1;        // [H][H] bf16 first router layer (Eq. 7), library-owned, or null
     float* router_u;     // [max_M][H] fp32 act(W1 h) + h, library-owned
     CUtensorMap map_w, map_h, map_h64, map_h32;   // hidden-row blocks read whole (128 rows) or only their first 64 / 32 rows
@@ -201,6 +202,7 @@ CallView make_view(const coral_lmhead_s* h, const void* hidden, int M, int kg, i
     c.union_list = reinterpret_cast<int32_t*>(ws + L.union_list);
     c.union_rank = reinterpret_cast<int32_t*>(ws + L.union_rank);
     c.union_cap = h->cfg.n_groups * kStreamMaxPasses;
+    c.hot_groups = h->hot_groups;
     c.shard_rank = h->shard_rank;
     c.shard_world = h->shard_world;
     c.part_max = reinterpret_cast<float*>(ws + L.part_max);
@@ -359,6 +361,7 @@ int coral_lmhead_create(coral_lmhead_handle* out, const coral_lmhead_config* cfg
     h->forced_path = CORAL_PATH_AUTO;
     h->shard_rank = 0;
     h->shard_world = 1;
+    h->hot_groups = 0;
     h->packed = static_cast<unsigned char*>(packed_buf_dev);
     h->ws = static_cast<unsigned char*>(workspace_dev);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -668,6 +671,12 @@ int coral_tree_expand(const float* parent_scores_dev, const int32_t* cand_ids_de
         parent_scores_dev, cand_ids_dev, cand_logprobs_dev, nodes, k_tokens, K, out_parent_dev, out_token_dev,
         out_score_dev);
     return cudaGetLastError() == cudaSuccess ? CORAL_OK : CORAL_ERR_CUDA;
+}
+
+int coral_lmhead_set_hot_groups(coral_lmhead_handle h, int n_hot) {
+    if (!h || n_hot < 0 || n_hot > h->cfg.n_groups) return CORAL_ERR_INVALID;
+    h->hot_groups = n_hot;
+    return CORAL_OK;
 }
 
 int coral_lmhead_copy_floor(coral_lmhead_handle h, long long bytes, void* stream) {

@@ -89,6 +89,10 @@ __device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatil
     *abort_flag = 1;
     set_status(st, -5);
 }
+__device__ __forceinline__ void bulk_g2s_hint(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar, uint64_t policy) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar), "l"(policy) : "memory");
+}
 __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                  ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
@@ -367,6 +371,8 @@ __global__ void __launch_bounds__(kStreamThreads, 1) head_stream_kernel(CallView
         if (lane != 0) return;
         int stage = 0, n_issued = 0;
         uint32_t phase = 0;
+        uint64_t pol_keep = 0;
+        if (c.hot_groups > 0) asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol_keep));
         for (int pos = sh.lo; pos < sh.hi;) {
             const int j = pos / g.T;
             const int seg_hi = min(sh.hi, (j + 1) * g.T);
@@ -379,7 +385,10 @@ __global__ void __launch_bounds__(kStreamThreads, 1) head_stream_kernel(CallView
                     mbar_wait(smem_u32(&sh.empty[stage]), phase ^ 1u, sh.abort_flag, c.state);
                     const uint32_t bar = smem_u32(&sh.full[stage]);
                     mbar_expect_tx(bar, bytes);
-                    bulk_g2s(smem_u32(sh.ring + (size_t)stage * g.stage_bytes), src, bytes, bar);
+                    if (n < c.hot_groups)      // a hot group: ask L2 to keep its lines when others have to go
+                        bulk_g2s_hint(smem_u32(sh.ring + (size_t)stage * g.stage_bytes), src, bytes, bar, pol_keep);
+                    else
+                        bulk_g2s(smem_u32(sh.ring + (size_t)stage * g.stage_bytes), src, bytes, bar);
                     __threadfence_block();
                     *sh.issued = ++n_issued;      // the slot's barrier is now in the phase of this slab
                     src += (size_t)kStreamTile * g.kc;

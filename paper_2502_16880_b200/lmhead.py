@@ -57,6 +57,7 @@ _SIGNATURES = {
     "coral_lmhead_draft_partial": (_i, [_vp, _vp, _i, _i, _i, _vp, _vp]),
     "coral_lmhead_merge_partials": (_i, [_vp, _i, _i, _i, _vp, _vp, _vp]),
     "coral_lmhead_copy_floor": (_i, [_vp, ctypes.c_longlong, _vp]),
+    "coral_lmhead_set_hot_groups": (_i, [_vp, _i]),
     "coral_csra_workspace_bytes": (_i, [_i, _i, _i, ctypes.POINTER(ctypes.c_size_t)]),
     "coral_csra_infonce": (_i, [_vp, _vp, _i, _i, _i, ctypes.c_float, _vp, _vp, _vp, _vp, _vp]),
     "coral_csra_status": (_i, [_vp, _vp]),
@@ -263,6 +264,10 @@ def coral_csra_infonce(Q, K, views, tau, workspace, out_loss, out_row_loss=None,
 
 def coral_csra_status(workspace, stream=None) -> int:
     return int(load_library().coral_csra_status(_dev_ptr(workspace, torch.uint8, False), _stream_ptr(stream)))
+
+
+def coral_lmhead_set_hot_groups(handle, n_hot: int) -> None:
+    _check(load_library().coral_lmhead_set_hot_groups(handle, int(n_hot)), "coral_lmhead_set_hot_groups")
 
 
 def coral_lmhead_selftest_wait_expiry(handle, stream=None) -> None:

@@ -418,3 +418,26 @@ def test_expired_wait_is_reported_and_the_handle_stays_usable():
     rep = ph.compare(W, gm, Wg, hb, cfg.k_groups, cfg.k_tokens, out)
     assert rep.ok, rep.errors
     head.close()
+
+
+def test_hot_groups_window_changes_no_result():
+    """The persisting-L2 window over the leading groups is a cache hint: same bits with and without it."""
+    cfg = synth.HeadConfig("hot", H=256, V=256 * 16, N=16, k_groups=4, k_tokens=10, M=8, seed=29, w_std=0.05, zipf_s=1.5)
+    W, Wg, hb = synth.make_w_vocab(cfg), synth.make_w_gate(cfg), synth.make_hidden(cfg)
+    gm = synth.make_group_map(cfg, contiguous=True)
+    head = _head(cfg, W, gm, Wg, max_M=8, max_kg=4)
+    base = ph.gpu_draft_numpy(head, hb, 4, 10)
+    lmhead.coral_lmhead_set_hot_groups(head.handle, 3)
+    hot = ph.gpu_draft_numpy(head, hb, 4, 10)
+    hot2 = ph.gpu_draft_numpy(head, hb, 4, 10)
+    assert head.status() == 0
+    lmhead.coral_lmhead_set_hot_groups(head.handle, 0)
+    off = ph.gpu_draft_numpy(head, hb, 4, 10)
+    for k in base:
+        assert np.array_equal(base[k], hot[k]) and np.array_equal(base[k], hot2[k]) and np.array_equal(base[k], off[k]), k
+    lib = lmhead.load_library()
+    assert lib.coral_lmhead_set_hot_groups(head.handle, 17) == lmhead.CORAL_ERR_INVALID
+    assert lib.coral_lmhead_set_hot_groups(head.handle, -1) == lmhead.CORAL_ERR_INVALID
+    rep = ph.compare(W, gm, Wg, hb, 4, 10, hot)
+    assert rep.ok, rep.errors
+    head.close()
