@@ -737,7 +737,7 @@ int coral_csra_infonce(const void* Q_dev, const void* K_dev, int n, int views, i
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
         cudaDeviceGetAttribute(&smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess)
         return CORAL_ERR_CUDA;
-    if ((int)kTcSmemBytes > smem_optin) return CORAL_ERR_INVALID;
+    if ((int)kCsraSmemBytes > smem_optin) return CORAL_ERR_INVALID;
     EncodeTiledFn enc = encode_tiled_fn();
     if (!enc) return CORAL_ERR_CUDA;
     CUtensorMap map_q, map_k;
@@ -755,7 +755,7 @@ int coral_csra_infonce(const void* Q_dev, const void* K_dev, int n, int views, i
                 CUDA_SUCCESS)
             return CORAL_ERR_CUDA;
     }
-    if (cudaFuncSetAttribute(csra_sim_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTcSmemBytes) != cudaSuccess)
+    if (cudaFuncSetAttribute(csra_sim_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kCsraSmemBytes) != cudaSuccess)
         return CORAL_ERR_CUDA;
     if (cudaMemsetAsync(ws + L.state, 0, sizeof(DeviceState), st) != cudaSuccess) return CORAL_ERR_CUDA;
     CsraGeom g{};
@@ -766,7 +766,7 @@ int coral_csra_infonce(const void* Q_dev, const void* K_dev, int n, int views, i
     float* row_loss = out_row_loss_dev ? out_row_loss_dev : reinterpret_cast<float*>(ws + L.row_loss);
     csra_normalise_kernel<<<L.RB * 128, 128, 0, st>>>(static_cast<const uint16_t*>(Q_dev), n, D, L.KB, qn);
     csra_normalise_kernel<<<L.KT * 128, 128, 0, st>>>(static_cast<const uint16_t*>(K_dev), g.m, D, L.KB, kn);
-    csra_sim_kernel<<<g.grid, kTcThreads, kTcSmemBytes, st>>>(
+    csra_sim_kernel<<<g.grid, kTcThreads, kCsraSmemBytes, st>>>(
         g, map_q, map_k, reinterpret_cast<float*>(ws + L.pmax), reinterpret_cast<float*>(ws + L.psum),
         reinterpret_cast<float*>(ws + L.pos), out_logits_dev, reinterpret_cast<DeviceState*>(ws + L.state));
     csra_finalize_kernel<<<(n + 255) / 256, 256, 0, st>>>(g, reinterpret_cast<const float*>(ws + L.pmax),

@@ -4,9 +4,9 @@
 //
 // Three steps: (1) csra_normalise_kernel divides every feature by its norm (float64) and stores it as bf16 in
 // blocks of 128 rows x 64 columns (one contiguous 16 KiB operand tile per block); (2) csra_sim_kernel is a
-// dense n x m x D contraction on the 5th-generation tensor cores with the structure of head_tc_kernel (TMA
-// tiled loads in a 4-stage ring, tcgen05.mma with M = 128 query rows x N = 128 key rows per accumulator, two
-// key tiles per batch sharing the query tile, accumulators double-buffered in tensor memory) whose epilogue
+// dense n x m x D contraction on the 5th-generation tensor cores built from the pieces of head_tc_kernel (TMA
+// tiled loads into a ring of stages, tcgen05.mma with M = 128 query rows x N = 128 key rows per accumulator,
+// 2 x 2 accumulators per batch in tensor memory) whose epilogue
 // folds the scaled similarities into a running (max, sum-exp) per query row and picks out the positives, so
 // the n x m similarity matrix never reaches HBM; (3) csra_finalize_kernel combines the partials per row and
 // csra_mean_kernel averages the rows in a fixed order.
@@ -112,33 +112,42 @@ __device__ __forceinline__ void csra_fold_row(const CsraGeom& g, CsraRowState& s
     }
 }
 
-// grid = g.grid CTAs of kTcThreads threads; the list of (row block, key tile) positions is cut into
-// contiguous runs, one per CTA.  Partials pmax / psum: [row block * KT + key tile][128 rows]; of the key
-// tiles an epilogue warp set sees of a row block inside the run, the last one carries its running partial
-// and the others an empty marker (max = -inf, sum = 0).
+// The contraction.  A batch is a 256 x 256 block of the similarity matrix: two query row blocks x two key
+// tiles, four 128 x 128 accumulators that fill the 512 columns of tensor memory, so every operand tile that
+// enters shared memory is used twice (128 flop per byte taken in, against 85 for a 128 x 256 block; what an
+// SM can take in - about 66 GB/s - is what bounds this kernel design).  Three stages of 64 KiB (A0, A1, B0,
+// B1).  There is no second set of accumulators, so the epilogue of a batch is not hidden behind the next
+// batch's MMAs; it is short here (one exp per similarity, no top-k).
+// grid = g.grid CTAs of kTcThreads threads; the list of (row block pair, key tile pair) positions is cut into
+// contiguous runs, one per CTA.  Partials pmax / psum: [row block * KT + key tile][128 rows]; an epilogue
+// thread carries its row's running (max, sum-exp) over the batches of the run that belong to its row block
+// and writes it at the first key tile of the last of them; the other slots get an empty marker
+// (max = -inf, sum = 0).  Warps 2..5 read row block 0 of the pair, warps 6..9 row block 1.
+constexpr int kCsraStages = 3;
+constexpr int kCsraStageBytes = 4 * kTcTileBytes;
+constexpr size_t kCsraSmemBytes = 1024 + (size_t)kCsraStages * kCsraStageBytes + 256;
+
 __global__ void __launch_bounds__(kTcThreads, 1)
     csra_sim_kernel(CsraGeom g, const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                     float* __restrict__ pmax, float* __restrict__ psum, float* __restrict__ out_pos,
                     float* __restrict__ logits_tap, DeviceState* state) {
     extern __shared__ unsigned char tc_smem_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(tc_smem_raw) + 1023) & ~(uintptr_t)1023);
-    uint64_t* full = reinterpret_cast<uint64_t*>(smem + kTcStages * kTcStageBytes);
-    uint64_t* empty = full + kTcStages;
-    uint64_t* tmem_full = empty + kTcStages;      // [2]
-    uint64_t* tmem_empty = tmem_full + 2;         // [2]
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tmem_empty + 2);
+    uint64_t* full = reinterpret_cast<uint64_t*>(smem + kCsraStages * kCsraStageBytes);
+    uint64_t* empty = full + kCsraStages;
+    uint64_t* tmem_full = empty + kCsraStages;    // [1]
+    uint64_t* tmem_empty = tmem_full + 1;         // [1]
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tmem_empty + 1);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kTcStages; ++s) {
+        for (int s = 0; s < kCsraStages; ++s) {
             mbar_init(smem_u32(&full[s]), 1);
             mbar_init(smem_u32(&empty[s]), 1);
         }
-        for (int s = 0; s < 2; ++s) {
-            mbar_init(smem_u32(&tmem_full[s]), 1);
-            mbar_init(smem_u32(&tmem_empty[s]), kTcEpilogueWarps);
-        }
+        mbar_init(smem_u32(tmem_full), 1);
+        mbar_init(smem_u32(tmem_empty), kTcEpilogueWarps);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -153,98 +162,94 @@ __global__ void __launch_bounds__(kTcThreads, 1)
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
-    const int n_pos = g.RB * g.KT;
+    const int RB2 = (g.RB + 1) >> 1, KT2 = (g.KT + 1) >> 1;
+    const int n_pos = RB2 * KT2;
     const int per = (n_pos + g.grid - 1) / g.grid;
     const int lo = min(n_pos, (int)blockIdx.x * per);
     const int hi = min(n_pos, lo + per);
-    // a batch = two key tiles of one row block (one at the end of a row block or of the run)
-    auto nsub_at = [&](int pos) { return ((pos % g.KT) + 1 < g.KT && pos + 1 < hi) ? 2 : 1; };
 
     if (warp == 0) {
         if (lane == 0) {
             int stage = 0;
             uint32_t phase = 0;
-            const uint64_t pol_first = l2_policy_evict_first(), pol_last = l2_policy_evict_last();
-            for (int pos = lo; pos < hi;) {
-                const int rb = pos / g.KT, kt = pos - rb * g.KT, nsub = nsub_at(pos);
-                const uint32_t bytes = (uint32_t)(1 + nsub) * kTcTileBytes;
+            const uint64_t pol_normal = l2_policy_evict_normal();
+            for (int pos = lo; pos < hi; ++pos) {
+                const int rb2 = pos / KT2, kt2 = pos - rb2 * KT2;
                 for (int ks = 0; ks < g.ksteps; ++ks) {
                     tc_wait(smem_u32(&empty[stage]), phase ^ 1u, abort_flag, state);
                     const uint32_t bar = smem_u32(&full[stage]);
-                    const uint32_t sb = smem_u32(smem + (size_t)stage * kTcStageBytes);
-                    mbar_expect_tx(bar, bytes);
-                    tma_load_2d(sb, &map_q, 0, (rb * g.ksteps + ks) * 128, bar, pol_last);
-                    for (int sub = 0; sub < nsub; ++sub)
-                        tma_load_2d(sb + (1 + sub) * kTcTileBytes, &map_k, 0, ((kt + sub) * g.ksteps + ks) * 128, bar,
-                                    pol_first);
-                    if (++stage == kTcStages) { stage = 0; phase ^= 1u; }
+                    const uint32_t sb = smem_u32(smem + (size_t)stage * kCsraStageBytes);
+                    mbar_expect_tx(bar, (uint32_t)kCsraStageBytes);
+                    // blocks past the last row block / key tile lie outside the tensor: the copy fills zeros
+                    for (int mb = 0; mb < 2; ++mb)
+                        tma_load_2d(sb + mb * kTcTileBytes, &map_q, 0, ((rb2 * 2 + mb) * g.ksteps + ks) * 128, bar, pol_normal);
+                    for (int sub = 0; sub < 2; ++sub)
+                        tma_load_2d(sb + (2 + sub) * kTcTileBytes, &map_k, 0, ((kt2 * 2 + sub) * g.ksteps + ks) * 128, bar,
+                                    pol_normal);
+                    if (++stage == kCsraStages) { stage = 0; phase ^= 1u; }
                 }
-                pos += nsub;
             }
         }
     } else if (warp == 1) {
         if (lane == 0) {
             int stage = 0, batch = 0;
             uint32_t phase = 0;
-            for (int pos = lo; pos < hi; ++batch) {
-                const int nsub = nsub_at(pos);
-                const int buf = batch & 1;
-                tc_wait(smem_u32(&tmem_empty[buf]), (((uint32_t)batch >> 1) & 1u) ^ 1u, abort_flag, state);
+            for (int pos = lo; pos < hi; ++pos, ++batch) {
+                tc_wait(smem_u32(tmem_empty), ((uint32_t)batch & 1u) ^ 1u, abort_flag, state);   // epilogue has drained
                 tc_fence_after();
-                const uint32_t acc = tmem_base + (uint32_t)(buf * 2 * kTcSub);
                 for (int ks = 0; ks < g.ksteps; ++ks) {
                     tc_wait(smem_u32(&full[stage]), phase, abort_flag, state);
                     tc_fence_after();
-                    const uint32_t sb = smem_u32(smem + (size_t)stage * kTcStageBytes);
+                    const uint32_t sb = smem_u32(smem + (size_t)stage * kCsraStageBytes);
 #pragma unroll
                     for (int kk = 0; kk < kTcK / 16; ++kk) {
-                        const uint64_t adesc = tc_smem_desc(sb + kk * 32);
-                        for (int sub = 0; sub < nsub; ++sub) {
-                            const uint64_t bdesc = tc_smem_desc(sb + (1 + sub) * kTcTileBytes + kk * 32);
-                            tc_mma(acc + (uint32_t)(sub * kTcSub), adesc, bdesc, (ks | kk) ? 1u : 0u);
+#pragma unroll
+                        for (int mb = 0; mb < 2; ++mb) {
+                            const uint64_t adesc = tc_smem_desc(sb + mb * kTcTileBytes + kk * 32);
+#pragma unroll
+                            for (int sub = 0; sub < 2; ++sub) {
+                                const uint64_t bdesc = tc_smem_desc(sb + (2 + sub) * kTcTileBytes + kk * 32);
+                                tc_mma(tmem_base + (uint32_t)((mb * 2 + sub) * kTcSub), adesc, bdesc, (ks | kk) ? 1u : 0u);
+                            }
                         }
                     }
                     tc_commit(smem_u32(&empty[stage]));
-                    if (++stage == kTcStages) { stage = 0; phase ^= 1u; }
+                    if (++stage == kCsraStages) { stage = 0; phase ^= 1u; }
                 }
-                tc_commit(smem_u32(&tmem_full[buf]));
-                pos += nsub;
+                tc_commit(smem_u32(tmem_full));
             }
         }
     } else {
         const int quarter = warp & 3;
-        const int which = (warp - 2) >> 2;
+        const int mb = (warp - 2) >> 2;                       // row block of the pair this warp reads
         const int row_in_block = quarter * 32 + lane;
         CsraRowState st;
         st.reset();
         int batch = 0;
-        for (int pos = lo; pos < hi; ++batch) {
-            const int rb = pos / g.KT, kt = pos - rb * g.KT, nsub = nsub_at(pos);
-            const int buf = batch & 1;
-            tc_wait(smem_u32(&tmem_full[buf]), ((uint32_t)batch >> 1) & 1u, abort_flag, state);
+        for (int pos = lo; pos < hi; ++pos, ++batch) {
+            const int rb2 = pos / KT2, kt2 = pos - rb2 * KT2;
+            const int rb = rb2 * 2 + mb;
+            tc_wait(smem_u32(tmem_full), (uint32_t)batch & 1u, abort_flag, state);
             tc_fence_after();
-            if (which < nsub) {
-                const int row = rb * 128 + row_in_block;
-                const bool row_valid = row < g.n;
-                const size_t pidx = ((size_t)rb * g.KT + kt + which) * 128 + row_in_block;
-                const uint32_t acc_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)((buf * 2 + which) * kTcSub);
-                csra_fold_row(g, st, acc_row, row, (kt + which) * kTcSub, row_valid, out_pos, logits_tap);
-                const int npos = pos + nsub;
-                bool last = npos >= hi || npos / g.KT != rb;
-                if (!last && which == 1) {
-                    const int nt = npos - rb * g.KT;
-                    last = nt + 1 >= g.KT || npos + 1 >= hi;      // the next batch is a single key tile
-                }
-                if (row_valid) {
-                    pmax[pidx] = last ? st.mx : kNegInf;
-                    psum[pidx] = last ? st.sum : 0.f;
-                }
-                if (last) st.reset();
+            const int row = rb * 128 + row_in_block;
+            const bool row_valid = row < g.n;
+            for (int sub = 0; sub < 2; ++sub) {
+                const int kt = kt2 * 2 + sub;
+                if (kt >= g.KT) continue;                      // warp-uniform
+                const uint32_t acc_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)((mb * 2 + sub) * kTcSub);
+                csra_fold_row(g, st, acc_row, row, kt * kTcSub, row_valid, out_pos, logits_tap);
             }
+            const bool last = pos + 1 >= hi || (pos + 1) / KT2 != rb2;
+            if (row_valid) {
+                const size_t p0 = ((size_t)rb * g.KT + kt2 * 2) * 128 + row_in_block;
+                pmax[p0] = last ? st.mx : kNegInf;
+                psum[p0] = last ? st.sum : 0.f;
+                if (kt2 * 2 + 1 < g.KT) { pmax[p0 + 128] = kNegInf; psum[p0 + 128] = 0.f; }
+            }
+            if (last) st.reset();
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&tmem_empty[buf]));
-            pos += nsub;
+            if (lane == 0) mbar_arrive(smem_u32(tmem_empty));
         }
     }
     tc_fence_before();
