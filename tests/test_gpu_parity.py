@@ -210,6 +210,9 @@ def test_qwen_shape_group_sweep_and_dense_equivalence(path):
     (256, 256, 16, 600, 8, 32),      # more than 256 rows per group: second pass; long candidate lists
     (320, 300, 6, 150, 2, 10),       # ragged group size (128 + 128 + 44) and H not a multiple of 256
     (328, 300, 6, 150, 3, 5),        # last 64-column step only partly inside H
+    (256, 256, 16, 400, 8, 10),      # 200 rows per group: two passes for every group
+    (320, 300, 6, 400, 3, 5),        # two passes, odd number of sub-tiles, ragged group size
+    (256, 256, 16, 1200, 8, 10),     # 600 rows per group: five passes, the last one partly filled
 ])
 def test_tensor_core_path(H, v, N, M, kg, kt):
     cfg = synth.HeadConfig("tc", H=H, V=v * N, N=N, k_groups=kg, k_tokens=kt, M=M, seed=7, w_std=0.05)
