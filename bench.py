@@ -237,8 +237,7 @@ def main():
     if args.vocab_shard_only:
         Ms = args.vocab_shard_only
         sh = lmhead.LMHead(Wd, torch.from_numpy(gm), dev_bf16(Wg), max_M=Ms, max_k_groups=cfg.k_groups,
-                           max_k_tokens=cfg.k_tokens)
-        lmhead.coral_lmhead_set_group_shard(sh.handle, rank, world)
+                           max_k_tokens=cfg.k_tokens, shard=(rank, world) if world > 1 else None)   # stores its own groups only
         hs = [dev_bf16(synth.make_hidden(cfg, Ms, batch=b)) for b in range(N_BATCHES)]     # same rows on every rank
         Wrec = 2 + 2 * cfg.k_tokens
         rec = torch.empty((Ms, Wrec), dtype=torch.int32, device=dev)

@@ -45,6 +45,9 @@ extern "C" {
 #define CORAL_ROUTE_STATIC_MAX_ROWS 64 /* M <= 64 for coral_lmhead_route_static */
 
 /* Execution paths (coral_lmhead_set_path / coral_lmhead_stats.path). */
+/* config flags: a handle that stores (and computes) only the groups n with n % world == rank */
+#define CORAL_CFG_SHARD(rank, world) ((uint32_t)(((world) & 0xff) | (((rank) & 0xff) << 8)))
+
 #define CORAL_PATH_AUTO 0          /* chosen from (M, k_groups) */
 #define CORAL_PATH_STREAM 1        /* bulk-copy weight streaming + warp MMA (fp32 accumulate); M <= 128, H % 256 == 0, H <= 4096 */
 #define CORAL_PATH_TCGEN05 2       /* routed grouped GEMM on tcgen05 / TMEM tiles */
@@ -65,7 +68,7 @@ typedef struct coral_lmhead_config {
     int32_t max_M;          /* largest number of query rows per draft call */
     int32_t max_k_groups;   /* largest top-n, 1..n_groups */
     int32_t max_k_tokens;   /* largest number of candidates, 1..CORAL_MAX_K_TOKENS */
-    uint32_t flags;         /* reserved, 0 */
+    uint32_t flags;         /* 0, or CORAL_CFG_SHARD(rank, world): store only this rank's groups (see vocab sharding) */
 } coral_lmhead_config;
 
 typedef struct coral_lmhead_stats {
@@ -164,8 +167,11 @@ int coral_lmhead_draft_host(coral_lmhead_handle h, const void *hidden_host, int 
  *
  * coral_lmhead_set_group_shard: rank in [0, world), world in [1, n_groups]; world = 1 (the default) switches
  * sharding off.  While world > 1 the handle accepts only coral_lmhead_draft_partial (a shard alone cannot
- * normalise a row): the other draft calls return CORAL_ERR_INVALID.  The handle still holds the full packed
- * head; sharding reduces what is read per call, not what is stored.
+ * normalise a row): the other draft calls return CORAL_ERR_INVALID.  A handle created with flags = 0 holds the
+ * full packed head and can take any shard (set_group_shard reduces what is read per call, not what is stored);
+ * a handle created with cfg.flags = CORAL_CFG_SHARD(rank, world) packs only its own groups (packed_bytes is
+ * about 1/world of the full size; W_vocab_dev is still the full matrix, read once at create), starts with that
+ * shard set and accepts no other.
  *
  * coral_lmhead_draft_partial: arguments as coral_lmhead_draft; out_records_dev is [M][2 + 2 k_tokens] 32-bit
  * words, per row: max of this GPU's active logits (float; -inf if none of the row's groups is local), sum of

@@ -29,6 +29,7 @@ struct CallView {
     int adaptive;                  // 1: the router picks pass_rows (streaming) or pass_rows_tc (tensor cores) and records it
     int pass_rows_tc, union_cap_tc;   // the tensor-core alternative of an adaptive call
     int hot_groups;                // groups below this index are loaded with an evict-last L2 hint (kept across calls)
+    int pack_div;                  // the packed copy holds group n at index n / pack_div (1, or shard_world when only this rank's groups are stored)
     int shard_rank, shard_world;   // vocab sharding: this call computes only the groups n with n % shard_world == shard_rank
     const uint16_t* packed;        // blocked copy of W_vocab, see packed_chunk_offset
     int KB, T16;                   // packed layout: 64-column blocks per row, 16-row items per group

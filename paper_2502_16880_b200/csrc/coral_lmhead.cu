@@ -33,6 +33,7 @@ struct Layout {
     int v, T;
     int KB, T16;                 // packed layout (see packed_chunk_offset)
     size_t route_bands;
+    int packed_groups;           // groups stored in the packed copy (all, or this rank's)
     int tc_tiles, tc_vcap;       // tensor-core path: sub-tiles per group, capacity in (group, pass) entries
     size_t tc_rows;              // rows of the gathered hidden matrix (0: path not provisioned)
 };
@@ -43,8 +44,13 @@ bool config_ok(const coral_lmhead_config* c) {
     if (c->V % c->n_groups != 0) return false;
     if (c->max_M < 1 || c->max_k_groups < 1 || c->max_k_groups > c->n_groups) return false;
     if (c->max_k_tokens < 1 || c->max_k_tokens > CORAL_MAX_K_TOKENS) return false;
+    const int world = (int)(c->flags & 0xff), rank = (int)((c->flags >> 8) & 0xff);
+    if (c->flags >> 16) return false;
+    if (world == 0 ? rank != 0 : (rank >= world || world > c->n_groups)) return false;
     return true;
 }
+inline int cfg_world(const coral_lmhead_config& c) { return (c.flags & 0xff) > 1 ? (int)(c.flags & 0xff) : 1; }
+inline int cfg_rank(const coral_lmhead_config& c) { return (int)((c.flags >> 8) & 0xff); }
 
 // Geometry of the streaming path.  The workspace layout must not depend on the device (sizes are
 // queried before a device is chosen), so it is sized for any grid in [kStreamGridMin, kStreamGridCap];
@@ -135,15 +141,18 @@ Layout make_layout(const coral_lmhead_config& c) {
     L.stage_ids = take(M * kt * 4);
     L.stage_logprobs = take(M * kt * 4);
     L.total = o;
-    L.packed_bytes = (size_t)c.n_groups * L.T16 * L.KB * 16 * 64 * 2;
+    L.packed_groups = (c.n_groups - cfg_rank(c) + cfg_world(c) - 1) / cfg_world(c);   // groups n = rank, rank + world, ...
+    L.packed_bytes = (size_t)L.packed_groups * L.T16 * L.KB * 16 * 64 * 2;
     return L;
 }
 
 // Row i of group n of the packed copy = W_vocab[group_tokens[n][i]], in the blocked layout; one block per row.
 __global__ void pack_rows_kernel(const uint16_t* __restrict__ W, const int32_t* __restrict__ group_tokens,
-                                 uint16_t* __restrict__ packed, int H, int v, int KB, int T16) {
+                                 uint16_t* __restrict__ packed, int H, int v, int KB, int T16, int rank, int world) {
     const int row = blockIdx.x;
-    const int n = row / v, j = row - n * v;
+    const int ng = row / v, j = row - ng * v;
+    if (ng % world != rank) return;               // another rank's group: not stored here
+    const int n = ng / world;
     const uint4* src = reinterpret_cast<const uint4*>(W + (size_t)group_tokens[row] * H);
     uint4* dst = reinterpret_cast<uint4*>(packed);
     for (int ch = threadIdx.x; ch < (H >> 3); ch += blockDim.x)
@@ -203,6 +212,7 @@ CallView make_view(const coral_lmhead_s* h, const void* hidden, int M, int kg, i
     c.union_rank = reinterpret_cast<int32_t*>(ws + L.union_rank);
     c.union_cap = h->cfg.n_groups * kStreamMaxPasses;
     c.hot_groups = h->hot_groups;
+    c.pack_div = cfg_world(h->cfg);
     c.shard_rank = h->shard_rank;
     c.shard_world = h->shard_world;
     c.part_max = reinterpret_cast<float*>(ws + L.part_max);
@@ -252,7 +262,7 @@ bool make_tc_maps(coral_lmhead_s* h) {
     EncodeTiledFn enc = encode_tiled_fn();
     if (!enc) return false;
     const Layout& L = h->L;
-    const cuuint64_t wdim[5] = {64, 16, (cuuint64_t)L.KB, (cuuint64_t)L.T16, (cuuint64_t)h->cfg.n_groups};
+    const cuuint64_t wdim[5] = {64, 16, (cuuint64_t)L.KB, (cuuint64_t)L.T16, (cuuint64_t)L.packed_groups};
     const cuuint64_t wstr[4] = {128, 2048, (cuuint64_t)L.KB * 2048, (cuuint64_t)L.T16 * L.KB * 2048};
     const cuuint32_t wbox[5] = {(cuuint32_t)kTcK, 16, 1, 8, 1};
     const cuuint32_t ones[5] = {1, 1, 1, 1, 1};
@@ -359,8 +369,8 @@ int coral_lmhead_create(coral_lmhead_handle* out, const coral_lmhead_config* cfg
     h->cfg = *cfg;
     h->L = make_layout(*cfg);
     h->forced_path = CORAL_PATH_AUTO;
-    h->shard_rank = 0;
-    h->shard_world = 1;
+    h->shard_rank = cfg_rank(*cfg);
+    h->shard_world = cfg_world(*cfg);
     h->hot_groups = 0;
     h->packed = static_cast<unsigned char*>(packed_buf_dev);
     h->ws = static_cast<unsigned char*>(workspace_dev);
@@ -414,7 +424,8 @@ int coral_lmhead_create(coral_lmhead_handle* out, const coral_lmhead_config* cfg
         if (cudaMemsetAsync(h->packed, 0, h->L.packed_bytes, st) != cudaSuccess) { rc = CORAL_ERR_CUDA; break; }
         pack_rows_kernel<<<V, 128, 0, st>>>(static_cast<const uint16_t*>(W_vocab_dev),
                                             reinterpret_cast<const int32_t*>(h->ws + h->L.group_tokens),
-                                            reinterpret_cast<uint16_t*>(h->packed), cfg->H, v, h->L.KB, h->L.T16);
+                                            reinterpret_cast<uint16_t*>(h->packed), cfg->H, v, h->L.KB, h->L.T16,
+                                            cfg_rank(*cfg), cfg_world(*cfg));
         if (cudaGetLastError() != cudaSuccess) { rc = CORAL_ERR_CUDA; break; }
         if (cudaStreamSynchronize(st) != cudaSuccess) { rc = CORAL_ERR_CUDA; break; }
     } while (0);
@@ -610,6 +621,8 @@ int coral_lmhead_draft_ex(coral_lmhead_handle h, const void* hidden_dev, int M, 
 
 int coral_lmhead_set_group_shard(coral_lmhead_handle h, int rank, int world) {
     if (!h || world < 1 || rank < 0 || rank >= world || world > h->cfg.n_groups) return CORAL_ERR_INVALID;
+    if (cfg_world(h->cfg) > 1 && (rank != cfg_rank(h->cfg) || world != cfg_world(h->cfg)))
+        return CORAL_ERR_INVALID;                 // the handle stores one shard only
     h->shard_rank = rank;
     h->shard_world = world;
     return CORAL_OK;

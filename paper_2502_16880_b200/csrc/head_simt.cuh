@@ -70,7 +70,7 @@ __device__ __forceinline__ void simt_tile_dots(const CallView& c, int n, int row
         for (int r = 0; r < R; ++r) acc[r] = 0.f;
 #pragma unroll 4
         for (int ch = lane; ch < chunks; ch += 32) {
-            const uint4 w = __ldg(wbase + packed_chunk_offset(n, row0 + j, ch, c.KB, c.T16));
+            const uint4 w = __ldg(wbase + packed_chunk_offset(n / c.pack_div, row0 + j, ch, c.KB, c.T16));
 #pragma unroll
             for (int r = 0; r < R; ++r)
                 acc[r] = dot8(w, *reinterpret_cast<const uint4*>(hs + (size_t)r * H + ch * 8), acc[r]);

@@ -378,7 +378,7 @@ __global__ void __launch_bounds__(kStreamThreads, 1) head_stream_kernel(CallView
             const int seg_hi = min(sh.hi, (j + 1) * g.T);
             const int n = sh.segtab[min(j - sh.j_first, kStreamSegTab - 1)] & 0xffff;
             int t = pos - j * g.T;
-            const uint16_t* src = c.packed + (((size_t)n * g.T + t) * g.kstages) * (size_t)(kStreamTile * g.kc);
+            const uint16_t* src = c.packed + (((size_t)(n / c.pack_div) * g.T + t) * g.kstages) * (size_t)(kStreamTile * g.kc);
             for (int item = pos; item < seg_hi; ++item, ++t) {
                 const uint32_t bytes = (uint32_t)g.stage_bytes;    // rows past the group's size are zero padding
                 for (int ks = 0; ks < g.kstages; ++ks) {

@@ -384,7 +384,7 @@ __global__ void __launch_bounds__(kTcThreads, 1)
                     // tile 0 of a stage is the pass's block of hidden rows, tiles 1 and 2 the weight sub-tiles
                     tma_load_2d(sb, mh, 0, (b.j * g.ksteps + ks) * kTcPassRows, bar, pol_last);
                     for (int sub = 0; sub < b.nsub; ++sub)
-                        tma_load_5d(sb + (1 + sub) * kTcTileBytes, &map_w, 0, 0, ks, (b.t + sub) * 8, b.n, bar, pol_w);
+                        tma_load_5d(sb + (1 + sub) * kTcTileBytes, &map_w, 0, 0, ks, (b.t + sub) * 8, b.n / c.pack_div, bar, pol_w);
                     if (++stage == kTcStages) { stage = 0; phase ^= 1u; }
                 }
                 pos += b.nsub;

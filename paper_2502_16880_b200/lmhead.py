@@ -122,9 +122,11 @@ def _stream_ptr(stream):
     return ctypes.c_void_p(stream.cuda_stream)
 
 
-def make_config(H, V, n_groups, max_M, max_k_groups, max_k_tokens) -> coral_lmhead_config:
+def make_config(H, V, n_groups, max_M, max_k_groups, max_k_tokens, shard=None) -> coral_lmhead_config:
+    """shard = (rank, world): the handle stores and computes only the groups n with n % world == rank."""
+    flags = 0 if shard is None else (int(shard[1]) & 0xFF) | ((int(shard[0]) & 0xFF) << 8)
     return coral_lmhead_config(ctypes.sizeof(coral_lmhead_config), H, V, n_groups, max_M, max_k_groups,
-                               max_k_tokens, 0)
+                               max_k_tokens, flags)
 
 
 # ---- functions named as in the C ABI -------------------------------------------------
@@ -339,10 +341,10 @@ def coral_lmhead_destroy(handle) -> None:
 class LMHead:
     """Owns the packed weights and workspace (torch allocations) of one handle."""
 
-    def __init__(self, W_vocab, group_map_host, W_gate, max_M, max_k_groups, max_k_tokens=10):
+    def __init__(self, W_vocab, group_map_host, W_gate, max_M, max_k_groups, max_k_tokens=10, shard=None):
         V, H = W_vocab.shape
         N = W_gate.shape[0]
-        self.cfg = make_config(H, V, N, max_M, max_k_groups, max_k_tokens)
+        self.cfg = make_config(H, V, N, max_M, max_k_groups, max_k_tokens, shard)
         pb, wb = coral_lmhead_query_sizes(self.cfg)
         dev = W_vocab.device
         self.packed = torch.empty(pb, dtype=torch.uint8, device=dev)

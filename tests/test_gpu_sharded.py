@@ -128,3 +128,55 @@ def test_sharded_handle_rejects_unsharded_calls_and_bad_arguments():
     assert lib.coral_lmhead_merge_partials(lmhead._dev_ptr(rec), 9, 4, 32, lmhead._dev_ptr(ids), lmhead._dev_ptr(lps),
                                            None) == lmhead.CORAL_ERR_TOO_LARGE
     head.close()
+
+
+@pytest.mark.parametrize("M,kg,path", [(8, 4, lmhead.CORAL_PATH_STREAM), (60, 5, lmhead.CORAL_PATH_STREAM),
+                                       (200, 4, lmhead.CORAL_PATH_TCGEN05), (5, 3, lmhead.CORAL_PATH_SIMT_PLAIN)])
+@pytest.mark.parametrize("world", [2, 3])
+def test_handles_that_store_only_their_own_groups(M, kg, path, world):
+    """One handle per rank, created with CORAL_CFG_SHARD(rank, world): it packs only the groups n % world == rank
+    (about 1/world of the bytes) and produces the same records as a full handle given that shard."""
+    H, v, N, kt = 256, 300, 12, 10
+    cfg = synth.HeadConfig("shardmem", H=H, V=v * N, N=N, k_groups=kg, k_tokens=kt, M=M, seed=31, w_std=0.05)
+    W, gm, Wg, hb = synth.make_all(cfg)
+    hidden = ph.to_dev_bf16(hb)
+    full = _head(cfg, W, gm, Wg, max_M=M, max_kg=kg)
+    full_bytes, _ = lmhead.coral_lmhead_query_sizes(full.cfg)
+    if path == lmhead.CORAL_PATH_SIMT_PLAIN:
+        # the plain path has no record output; a sharded handle must still refuse cleanly
+        sh = lmhead.LMHead(ph.to_dev_bf16(W), torch.from_numpy(gm), ph.to_dev_bf16(Wg), M, kg, 32, shard=(0, world))
+        sh.set_path(path)
+        rec = torch.empty((M, 2 + 2 * kt), dtype=torch.int32, device="cuda")
+        with pytest.raises(lmhead.CoralError):
+            lmhead.coral_lmhead_draft_partial(sh.handle, hidden, kg, kt, rec)
+        sh.close()
+        full.close()
+        return
+    full.set_path(path)
+    want_ids, want_lps, _, want_rec = _sharded(full, hidden, kg, kt, world)
+    gathered = torch.empty((world, M, 2 + 2 * kt), dtype=torch.int32, device="cuda")
+    total = 0
+    for r in range(world):
+        sh = lmhead.LMHead(ph.to_dev_bf16(W), torch.from_numpy(gm), ph.to_dev_bf16(Wg), M, kg, 32, shard=(r, world))
+        b, _ = lmhead.coral_lmhead_query_sizes(sh.cfg)
+        total += b
+        assert b == full_bytes // N * len(range(r, N, world))
+        sh.set_path(path)
+        lib = lmhead.load_library()
+        assert lib.coral_lmhead_set_group_shard(sh.handle, (r + 1) % world, world) == lmhead.CORAL_ERR_INVALID
+        assert lib.coral_lmhead_set_group_shard(sh.handle, 0, 1) == lmhead.CORAL_ERR_INVALID
+        lmhead.coral_lmhead_draft_partial(sh.handle, hidden, kg, kt, gathered[r])
+        torch.cuda.synchronize()
+        assert sh.status() == 0
+        sh.close()
+    assert total == full_bytes                              # the ranks' packed copies partition the head
+    assert np.array_equal(gathered.cpu().numpy(), want_rec)  # bit-identical to the full handle's records
+    ids = torch.empty((M, kt), dtype=torch.int32, device="cuda")
+    lps = torch.empty((M, kt), dtype=torch.float32, device="cuda")
+    lmhead.coral_lmhead_merge_partials(gathered, kt, ids, lps)
+    torch.cuda.synchronize()
+    assert np.array_equal(ids.cpu().numpy(), want_ids) and np.array_equal(lps.cpu().numpy(), want_lps)
+    rows = np.unique(np.linspace(0, M - 1, 12).astype(int))
+    rep = ph.compare(W, gm, Wg, hb[rows], kg, kt, {"ids": want_ids[rows], "logprobs": want_lps[rows]})
+    assert rep.ok, rep.errors
+    full.close()
