@@ -154,6 +154,27 @@ def main_reference(args, rank):
         return
     from paper_2502_16880_b200 import synth
     cfg = synth.CONFIGS[WORKLOAD].with_(M=args.rows)
+    if args.csra_only:
+        n_c, v_c, D_c = args.csra_only, 4, cfg.H
+        rng_c = np.random.default_rng([cfg.seed, 77])
+        mk = lambda rows: torch.from_numpy(synth.fp32_to_bf16_bits(rng_c.standard_normal((rows, D_c), dtype=np.float32))
+                                           .view(np.int16)).to(dev).view(torch.bfloat16)
+        Qc, Kc = mk(n_c), mk(n_c * v_c)
+        ws_c = torch.empty(lmhead.coral_csra_workspace_bytes(n_c, v_c, D_c), dtype=torch.uint8, device=dev)
+        loss_c = torch.empty(1, dtype=torch.float32, device=dev)
+        ts = []
+        for i in range(args.warmup + args.steps):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            lmhead.coral_csra_infonce(Qc, Kc, v_c, 0.07, ws_c, loss_c)
+            b.record()
+            torch.cuda.synchronize()
+            if i >= args.warmup:
+                ts.append(a.elapsed_time(b))
+        print(json.dumps({"csra_only": n_c, "views": v_c, "D": D_c, "us": float(np.mean(ts)) * 1e3,
+                          "tflops": 2.0 * n_c * n_c * v_c * D_c / (float(np.mean(ts)) * 1e-3) / 1e12,
+                          "loss": float(loss_c.item()), "status": lmhead.coral_csra_status(ws_c)}))
+        return
     W, gm, Wg = synth.make_w_vocab(cfg), synth.make_group_map(cfg), synth.make_w_gate(cfg)
     hbs = [synth.make_hidden(cfg, cfg.M, batch=b) for b in range(N_BATCHES)]
     times, touched, cores = run_oracle_baseline(cfg, W, gm, Wg, hbs, args.steps, args.warmup)
@@ -185,6 +206,8 @@ def main():
     ap.add_argument("--vocab-shard-only", type=int, default=0, metavar="M",
                     help="run only the vocab-sharded step with M rows: every rank reads its own groups, one all-gather "
                          "of the per-row records, merge (strong scaling: all ranks draft for the same rows)")
+    ap.add_argument("--csra-only", type=int, default=0, metavar="N",
+                    help="run only the CSRA objective (Eq. 2) with N positions, 4 key blocks, D = H (a short run for profilers)")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
@@ -207,6 +230,27 @@ def main():
     lmhead.load_library()
 
     cfg = synth.CONFIGS[WORKLOAD].with_(M=args.rows)
+    if args.csra_only:
+        n_c, v_c, D_c = args.csra_only, 4, cfg.H
+        rng_c = np.random.default_rng([cfg.seed, 77])
+        mk = lambda rows: torch.from_numpy(synth.fp32_to_bf16_bits(rng_c.standard_normal((rows, D_c), dtype=np.float32))
+                                           .view(np.int16)).to(dev).view(torch.bfloat16)
+        Qc, Kc = mk(n_c), mk(n_c * v_c)
+        ws_c = torch.empty(lmhead.coral_csra_workspace_bytes(n_c, v_c, D_c), dtype=torch.uint8, device=dev)
+        loss_c = torch.empty(1, dtype=torch.float32, device=dev)
+        ts = []
+        for i in range(args.warmup + args.steps):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            lmhead.coral_csra_infonce(Qc, Kc, v_c, 0.07, ws_c, loss_c)
+            b.record()
+            torch.cuda.synchronize()
+            if i >= args.warmup:
+                ts.append(a.elapsed_time(b))
+        print(json.dumps({"csra_only": n_c, "views": v_c, "D": D_c, "us": float(np.mean(ts)) * 1e3,
+                          "tflops": 2.0 * n_c * n_c * v_c * D_c / (float(np.mean(ts)) * 1e-3) / 1e12,
+                          "loss": float(loss_c.item()), "status": lmhead.coral_csra_status(ws_c)}))
+        return
     W, gm, Wg = synth.make_w_vocab(cfg), synth.make_group_map(cfg), synth.make_w_gate(cfg)
 
     def dev_bf16(bits):

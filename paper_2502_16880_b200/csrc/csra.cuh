@@ -28,14 +28,26 @@ struct CsraGeom {
 // One block per feature row: x / ||x||, rounded to bf16, into the blocked layout
 // out[row block][column block][128 rows][64 columns]; columns past D are zero, and the blocks past the last row
 // write zero rows, so that every operand tile is defined.  The rounding to bf16 decides which of two
-// neighbouring operand values the contraction sees, so it is taken from a float64 quotient (norm and division
-// in float64): whoever repeats it in float64 lands on the same side of the rounding boundary.
-__device__ __forceinline__ uint16_t csra_round_bf16(double y) {
-    float f = __double2float_rz(y);                     // truncate, then make the dropped bits sticky (round to odd):
-    if ((double)f != y) f = __uint_as_float(__float_as_uint(f) | 1u);   // the final rounding then sees the exact value's side
-    uint32_t u = __float_as_uint(f);
-    u = (u + 0x7FFFu + ((u >> 16) & 1u)) >> 16;         // nearest, ties to even
-    return (uint16_t)u;
+// neighbouring operand values the contraction sees, so it is taken from a float64 value (norm and scaling in
+// float64): whoever repeats it in float64 lands on the same side of the rounding boundary.
+// x * inv rounded to bf16 (nearest, ties to even) as if from the exact product, in float32 arithmetic: inv is
+// given as hi + lo (two floats, from a float64), p = fl(x * hi), and err = (x * hi - p) + x * lo is the rest,
+// far below half a unit in the last place of p.  A float32 is either exactly half-way between two bf16 values
+// (then the sign of err decides, and only err = 0 is a true tie) or at least one float32 spacing away from
+// the half-way point, further than err can move it.
+__device__ __forceinline__ uint32_t csra_scale_round_bf16(float x, float hi, float lo) {
+    const float p = x * hi;
+    const float err = fmaf(x, hi, -p) + x * lo;
+    const uint32_t u = __float_as_uint(p);
+    const uint32_t low = u & 0xFFFFu;
+    uint32_t r = u >> 16;
+    if (low == 0x8000u) {                                   // exactly half-way: p's magnitude grows with err's sign
+        const bool away = (err > 0.f) != (p < 0.f);         // the exact value lies beyond the half-way point
+        if (err != 0.f ? away : (r & 1u)) ++r;
+    } else if (low > 0x8000u) {
+        ++r;
+    }
+    return r;
 }
 
 __global__ void __launch_bounds__(128) csra_normalise_kernel(const uint16_t* __restrict__ x, int rows, int D, int KB,
@@ -43,24 +55,43 @@ __global__ void __launch_bounds__(128) csra_normalise_kernel(const uint16_t* __r
     __shared__ double s_part[4];
     const int row = blockIdx.x;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int chunks = D >> 3;                                   // 8 columns = one 128-bit word
+    const uint4* src = reinterpret_cast<const uint4*>(x + (size_t)(row < rows ? row : 0) * D);
     double ss = 0.0;
     if (row < rows)
-        for (int i = threadIdx.x; i < D; i += 128) {
-            const double v = (double)__uint_as_float((uint32_t)x[(size_t)row * D + i] << 16);
-            ss += v * v;
+        for (int ch = threadIdx.x; ch < chunks; ch += 128) {
+            const uint4 w = __ldg(src + ch);
+            const uint32_t u[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const float lo = bf16_lo(u[i]), hi = bf16_hi(u[i]);
+                ss += (double)(lo * lo);                    // squares of bf16 values are exact in float32
+                ss += (double)(hi * hi);
+            }
         }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
     if (lane == 0) s_part[warp] = ss;
     __syncthreads();
     ss = (s_part[0] + s_part[1]) + (s_part[2] + s_part[3]);
-    const double nrm = sqrt(ss);
-    uint16_t* dst = out + ((size_t)(row >> 7) * KB * 128 + (row & 127)) * 64;
-    for (int i = threadIdx.x; i < KB * 64; i += 128) {
-        uint16_t r = 0;
-        if (row < rows && i < D && nrm > 0.0)
-            r = csra_round_bf16((double)__uint_as_float((uint32_t)x[(size_t)row * D + i] << 16) / nrm);
-        dst[(size_t)(i >> 6) * 128 * 64 + (i & 63)] = r;
+    // x * (1 / norm) instead of x / norm: the two differ by about one unit in the last place of a float64,
+    // 13 orders of magnitude below the spacing of bf16 values, so they round to the same bf16
+    const double inv = ss > 0.0 ? 1.0 / sqrt(ss) : 0.0;
+    const float inv_hi = (float)inv, inv_lo = (float)(inv - (double)inv_hi);
+    uint4* dst = reinterpret_cast<uint4*>(out + ((size_t)(row >> 7) * KB * 128 + (row & 127)) * 64);
+    for (int ch = threadIdx.x; ch < KB * 8; ch += 128) {
+        uint4 r = make_uint4(0, 0, 0, 0);
+        if (row < rows && ch < chunks) {
+            const uint4 w = __ldg(src + ch);
+            const uint32_t u[4] = {w.x, w.y, w.z, w.w};
+            uint32_t o[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+                o[i] = csra_scale_round_bf16(bf16_lo(u[i]), inv_hi, inv_lo) |
+                       (csra_scale_round_bf16(bf16_hi(u[i]), inv_hi, inv_lo) << 16);
+            r = make_uint4(o[0], o[1], o[2], o[3]);
+        }
+        dst[(size_t)(ch >> 3) * 128 * 8 + (ch & 7)] = r;          // block kb = ch / 8, 16 bytes at column (ch % 8) * 8
     }
 }
 
