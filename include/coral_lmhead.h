@@ -248,12 +248,13 @@ int coral_csra_status(void *workspace_dev, void *stream);
 /*
  * Ask L2 to keep the first n_hot groups of the packed head between calls (Appendix B: with a
  * frequency-ordered vocabulary the low-index groups hold the frequent tokens and are activated by almost every
- * row).  The streaming kernel then loads those groups' weights with an evict-last cache hint and everything
- * else as before, so that the traffic between two calls pushes out other lines first.  A hint, not a
- * reservation: how much survives depends on what runs in between (with 512 MiB written and read between calls,
- * four hot groups saved 4 % of the step at M=8 on the frequency-ordered workload).  No device setting is
- * changed.  Meant for contiguous, frequency-ordered group maps; n_hot = 0 (the default) switches it off.
- * Applies to calls on the streaming path.
+ * row).  The streaming kernel then loads those groups' weights with an evict-last cache hint, and up to their
+ * size of L2 is set aside for such lines (cudaLimitPersistingL2CacheSize: a setting of this process's CUDA
+ * context that takes L2 away from everything else the process runs and ends with the process; without the
+ * set-aside the hint alone changed nothing).  How much survives depends on what runs between two calls.
+ * Meant for contiguous, frequency-ordered group maps; n_hot = 0 (the default) switches it off, resets the
+ * persisting lines and returns the set-aside.  Applies to calls on the streaming path.  Synchronises nothing,
+ * but changes a context-wide limit: call it at set-up time, not between overlapping work.
  */
 int coral_lmhead_set_hot_groups(coral_lmhead_handle h, int n_hot);
 

@@ -688,6 +688,20 @@ int coral_tree_expand(const float* parent_scores_dev, const int32_t* cand_ids_de
 
 int coral_lmhead_set_hot_groups(coral_lmhead_handle h, int n_hot) {
     if (!h || n_hot < 0 || n_hot > h->cfg.n_groups) return CORAL_ERR_INVALID;
+    if (n_hot == 0) {
+        h->hot_groups = 0;
+        if (cudaCtxResetPersistingL2Cache() != cudaSuccess) return CORAL_ERR_CUDA;
+        return cudaDeviceSetLimit(cudaLimitPersistingL2CacheSize, 0) == cudaSuccess ? CORAL_OK : CORAL_ERR_CUDA;
+    }
+    // evict-last lines only outlive other traffic inside the part of L2 that is set aside for them
+    int dev = 0, max_persist = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&max_persist, cudaDevAttrMaxPersistingL2CacheSize, dev) != cudaSuccess)
+        return CORAL_ERR_CUDA;
+    if (max_persist <= 0) return CORAL_ERR_INVALID;                     // the device has no such set-aside
+    const size_t want = (size_t)n_hot * h->L.T16 * h->L.KB * 2048;      // packed bytes of the hot groups
+    const size_t carve = want < (size_t)max_persist ? want : (size_t)max_persist;
+    if (cudaDeviceSetLimit(cudaLimitPersistingL2CacheSize, carve) != cudaSuccess) return CORAL_ERR_CUDA;
     h->hot_groups = n_hot;
     return CORAL_OK;
 }
