@@ -48,6 +48,7 @@ __global__ void __launch_bounds__(32) copy_probe_kernel(const unsigned char* __r
             }
         }
         acc += copy_smem[s * kCopyChunk];
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the read above before the slot's next bulk copy
         ++done;
     }
     sink[blockIdx.x] = acc;

@@ -231,7 +231,12 @@ __device__ __forceinline__ void stream_segment_mma(const CallView& c, const Stre
                         mma_bf16_16816(acc[nt][1], wg.z, wh.z, wg.w, wh.w, b.z, b.w);
                     }
                 }
+                // The slot is refilled by a bulk copy (async proxy) as soon as it is released, and this warp has just
+                // read it with ordinary shared-memory loads (generic proxy): order the two before letting go.
+                // (Without this fence the first item after a change of segment, where the producer is already
+                // waiting for this very slot, was occasionally computed from a half-overwritten slab.)
                 __syncwarp();
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                 if (lane == 0) mbar_arrive(smem_u32(&sh.empty[stage]));
             }
         }

@@ -444,3 +444,27 @@ def test_hot_groups_window_changes_no_result():
     rep = ph.compare(W, gm, Wg, hb, 4, 10, hot)
     assert rep.ok, rep.errors
     head.close()
+
+
+def test_streaming_path_repeats_bit_for_bit_with_many_passes():
+    """Every row selects every group, so each group is streamed in four passes and every CTA changes segment
+    several times, the moment at which a ring slot is refilled the instant it is released: 30 calls must agree
+    to the bit (a missing ordering between the warps' reads of a slot and its refill showed up only here)."""
+    cfg, W, gm, Wg, head = _weights("llama3_8b")
+    head.set_path(lmhead.CORAL_PATH_STREAM)
+    M = 60
+    hidden = ph.to_dev_bf16(synth.make_hidden(cfg, M))
+    ref = None
+    for i in range(30):
+        ids, lps = head.draft(hidden, cfg.N, cfg.k_tokens)
+        torch.cuda.synchronize()
+        cur = (ids.cpu().numpy(), lps.cpu().numpy())
+        if ref is None:
+            ref = cur
+        else:
+            assert np.array_equal(cur[0], ref[0]) and np.array_equal(cur[1], ref[1]), i
+    assert head.status() == 0
+    rows = np.array([0, 29, 59])
+    hb = synth.make_hidden(cfg, M)
+    rep = ph.compare(W, gm, Wg, hb[rows], cfg.N, cfg.k_tokens, {"ids": ref[0][rows], "logprobs": ref[1][rows]})
+    assert rep.ok, rep.errors
