@@ -246,6 +246,11 @@ def test_large_m_routed_grouped_gemm():
     rep = ph.compare(W, gm, Wg, hb[rows], cfg.k_groups, cfg.k_tokens,
                      {"ids": ids.cpu().numpy()[rows], "logprobs": lps.cpu().numpy()[rows]})
     assert rep.ok, rep.errors
+    first = (ids.cpu().numpy().copy(), lps.cpu().numpy().copy())
+    for _ in range(5):                                   # the same call again: the same bits
+        ids2, lps2 = head.draft(ph.to_dev_bf16(hb), cfg.k_groups, cfg.k_tokens)
+        torch.cuda.synchronize()
+        assert np.array_equal(ids2.cpu().numpy(), first[0]) and np.array_equal(lps2.cpu().numpy(), first[1])
     head.close()
 
 
