@@ -473,3 +473,19 @@ def test_streaming_path_repeats_bit_for_bit_with_many_passes():
     hb = synth.make_hidden(cfg, M)
     rep = ph.compare(W, gm, Wg, hb[rows], cfg.N, cfg.k_tokens, {"ids": ref[0][rows], "logprobs": ref[1][rows]})
     assert rep.ok, rep.errors
+
+
+@pytest.mark.parametrize("seed", [1, 2])
+def test_other_seeds_on_the_llama2_shape(seed):
+    """The recipe's other seeds (weights, group map and hidden rows all change) on the Llama2-7B-shaped head."""
+    cfg = synth.CONFIGS["llama2_7b"].with_(seed=seed)
+    W, gm, Wg = synth.make_w_vocab(cfg), synth.make_group_map(cfg), synth.make_w_gate(cfg)
+    head = _head(cfg, W, gm, Wg, max_M=60, max_kg=cfg.k_groups, max_kt=cfg.k_tokens)
+    for M in (1, 8, 60):
+        hb = synth.make_hidden(cfg, M)
+        out = ph.gpu_draft_numpy(head, hb, cfg.k_groups, cfg.k_tokens)
+        assert head.status() == 0
+        rows = np.unique(np.linspace(0, M - 1, 6).astype(int))
+        rep = ph.compare(W, gm, Wg, hb[rows], cfg.k_groups, cfg.k_tokens, {k: v[rows] for k, v in out.items()})
+        assert rep.ok, (M, rep.errors)
+    head.close()
