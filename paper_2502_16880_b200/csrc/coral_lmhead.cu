@@ -520,7 +520,7 @@ static int draft_impl(coral_lmhead_handle h, const void* hidden_dev, int M, int 
         route_mid_kernel<<<dim3((c.N + 15) / 16, (M + 7) / 8), 256, 0, st>>>(
             c, forced_groups_dev, out_groups_dev, out_gate_dev, rt_bands, rt_masks, rt_counts, 0);
         ++launches;
-        bucket_group_kernel<<<c.N, 256, 0, st>>>(c, rt_counts);
+        launch_pdl(bucket_group_kernel, dim3(c.N), dim3(256), (size_t)0, st, c, rt_counts);
         ++launches;
     } else {
         gate_tile_kernel<<<dim3((c.N + kGateTile - 1) / kGateTile, (M + kGateTile - 1) / kGateTile), 256, 0, st>>>(
@@ -552,8 +552,8 @@ static int draft_impl(coral_lmhead_handle h, const void* hidden_dev, int M, int 
             launch_pdl(tc_gather_kernel, dim3(M * k_groups), dim3(128), (size_t)0, st, c,
                        reinterpret_cast<uint16_t*>(h->ws + L.tc_hg));
             ++launches;
-            head_tc_kernel<<<tg.grid, kTcThreads, kTcSmemBytes, st>>>(c, tg, tp, h->map_w, h->map_h, h->map_h64, h->map_h32,
-                                                                     out_logits_dev);
+            launch_pdl(head_tc_kernel, dim3(tg.grid), dim3(kTcThreads), kTcSmemBytes, st, c, tg, tp, h->map_w, h->map_h,
+                       h->map_h64, h->map_h32, out_logits_dev);
             ++launches;
         }
         launch_pdl(h->sg.kc == 512 ? head_stream_kernel<2> : head_stream_kernel<1>, dim3(h->sg.grid),
@@ -578,10 +578,11 @@ static int draft_impl(coral_lmhead_handle h, const void* hidden_dev, int M, int 
         TcGeom tg{h->sms, L.tc_tiles, L.KB};
         TcPartials tp{reinterpret_cast<float*>(h->ws + L.tc_max), reinterpret_cast<float*>(h->ws + L.tc_sum),
                       reinterpret_cast<float*>(h->ws + L.tc_val), reinterpret_cast<int32_t*>(h->ws + L.tc_id)};
-        tc_gather_kernel<<<M * k_groups, 128, 0, st>>>(c, reinterpret_cast<uint16_t*>(h->ws + L.tc_hg));
+        launch_pdl(tc_gather_kernel, dim3(M * k_groups), dim3(128), (size_t)0, st, c,
+                   reinterpret_cast<uint16_t*>(h->ws + L.tc_hg));
         ++launches;
-        head_tc_kernel<<<tg.grid, kTcThreads, kTcSmemBytes, st>>>(c, tg, tp, h->map_w, h->map_h, h->map_h64, h->map_h32,
-                                                                 out_logits_dev);
+        launch_pdl(head_tc_kernel, dim3(tg.grid), dim3(kTcThreads), kTcSmemBytes, st, c, tg, tp, h->map_w, h->map_h,
+                   h->map_h64, h->map_h32, out_logits_dev);
         ++launches;
         if (h->timing) cudaEventRecord(h->ev_head1, st);
         StreamGeom mg = h->sg;

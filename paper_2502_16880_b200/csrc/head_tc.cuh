@@ -137,7 +137,8 @@ __device__ __forceinline__ void tc_ld32(uint32_t taddr, float (&v)[32]) {
 // whatever they held (their accumulator lanes are never read).
 __global__ void __launch_bounds__(128) tc_gather_kernel(CallView c, uint16_t* __restrict__ hg) {
     const int p = blockIdx.x;
-    pdl_wait();                                              // (adaptive calls launch this kernel over the router's tail)
+    pdl_wait();                                              // launched over the tail of the router stage
+    pdl_launch_dependents();
     if (c.adaptive && c.state->path_choice != 2) return;     // the router chose the streaming kernel for this call
     if (p >= c.group_offset[c.N]) return;          // fewer pairs than M * k_groups when the vocab is sharded
     const int m = c.bucket_row[p];
@@ -320,7 +321,6 @@ __global__ void __launch_bounds__(kTcThreads, 1)
     head_tc_kernel(CallView c, TcGeom g, TcPartials pp, const __grid_constant__ CUtensorMap map_w,
                    const __grid_constant__ CUtensorMap map_h, const __grid_constant__ CUtensorMap map_h64,
                    const __grid_constant__ CUtensorMap map_h32, float* __restrict__ logits_tap) {
-    if (c.adaptive && c.state->path_choice != 2) return;     // the router chose the streaming kernel for this call
     extern __shared__ unsigned char tc_smem_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(tc_smem_raw) + 1023) & ~(uintptr_t)1023);
     float* zstash = reinterpret_cast<float*>(smem + kTcStages * kTcStageBytes);          // [32][epilogue threads]
@@ -332,6 +332,8 @@ __global__ void __launch_bounds__(kTcThreads, 1)
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
+    // The kernel may be launched while its predecessors (gather, router) still run: everything up to the
+    // dependency wait touches only this CTA's shared and tensor memory.
     if (threadIdx.x == 0) {
         for (int s = 0; s < kTcStages; ++s) {
             mbar_init(smem_u32(&full[s]), 1);
@@ -354,9 +356,12 @@ __global__ void __launch_bounds__(kTcThreads, 1)
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    pdl_wait();                                              // gathered rows and router outputs are complete from here on
+    // (no early release of the merge kernel: it reads this kernel's partials right after its own metadata)
+    const bool skip = c.adaptive && c.state->path_choice != 2;   // the router chose the streaming kernel for this call
 
     // this CTA's run of sub-tiles
-    const int n_tiles = c.state->n_virtual * g.tiles;
+    const int n_tiles = skip ? 0 : c.state->n_virtual * g.tiles;
     const int per = (n_tiles + g.grid - 1) / g.grid;
     const int lo = min(n_tiles, (int)blockIdx.x * per);
     const int hi = min(n_tiles, lo + per);

@@ -560,6 +560,8 @@ __global__ void __launch_bounds__(256) bucket_group_kernel(CallView c, int* __re
     __shared__ int s_warp[8];
     const int n = blockIdx.x;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    pdl_wait();                   // (launched over the tail of the kernel that selects and counts)
+    pdl_launch_dependents();
     {
         // counts: group_count (filled by count_groups_kernel), or the accumulators of route_mid_kernel, which
         // the last block to have read them clears for the next call
