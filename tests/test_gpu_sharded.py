@@ -180,3 +180,21 @@ def test_handles_that_store_only_their_own_groups(M, kg, path, world):
     rep = ph.compare(W, gm, Wg, hb[rows], kg, kt, {"ids": want_ids[rows], "logprobs": want_lps[rows]})
     assert rep.ok, rep.errors
     full.close()
+
+
+@pytest.mark.parametrize("zipf", [0.0, 1.5])
+def test_sharded_step_with_the_kernel_chosen_on_the_device(zipf):
+    """Vocab sharding together with CORAL_PATH_ADAPTIVE: each rank's router decides from its own groups' row
+    counts (so ranks may take different kernels); the merged result still matches the oracle."""
+    M, kg, kt, world = 60, 4, 10, 2
+    cfg = synth.HeadConfig("shard_adaptive", H=256, V=256 * 16, N=16, k_groups=kg, k_tokens=kt, M=M, seed=37,
+                           w_std=0.05, zipf_s=zipf)
+    W, Wg, hb = synth.make_w_vocab(cfg), synth.make_w_gate(cfg), synth.make_hidden(cfg)
+    gm = synth.make_group_map(cfg, contiguous=zipf > 0)
+    head = _head(cfg, W, gm, Wg, max_M=128, max_kg=kg)
+    head.set_path(lmhead.CORAL_PATH_ADAPTIVE)
+    ids, lps, touched, _ = _sharded(head, ph.to_dev_bf16(hb), kg, kt, world)
+    rows = np.unique(np.linspace(0, M - 1, 24).astype(int))
+    rep = ph.compare(W, gm, Wg, hb[rows], kg, kt, {"ids": ids[rows], "logprobs": lps[rows]})
+    assert rep.ok, rep.errors
+    head.close()
