@@ -581,6 +581,34 @@ def main():
             "torch_dense_gemm_960xVxH_us": float(np.mean(tg)) * 1e3,
         }
         big.close()
+        # supplementary points with more rows per group (240 and 480): the same path above the machine ridge
+        supp = []
+        for M_s in (1920, 3840):
+            bg = lmhead.LMHead(Wd, torch.from_numpy(gm), dev_bf16(Wg), max_M=M_s, max_k_groups=cfg.k_groups,
+                               max_k_tokens=cfg.k_tokens)
+            h_s = dev_bf16(synth.make_hidden(cfg, M_s, batch=200))
+            ids_s = torch.empty((M_s, cfg.k_tokens), dtype=torch.int32, device=dev)
+            lps_s = torch.empty((M_s, cfg.k_tokens), dtype=torch.float32, device=dev)
+            lmhead.coral_lmhead_set_kernel_timing(bg.handle, True)
+            ts_, th_ = [], []
+            for i in range(8):
+                flush_l2(i)
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record()
+                lmhead.coral_lmhead_draft(bg.handle, h_s, cfg.k_groups, cfg.k_tokens, ids_s, lps_s, stream)
+                b.record()
+                torch.cuda.synchronize()
+                if i >= 3:
+                    ts_.append(a.elapsed_time(b))
+                    th_.append(lmhead.coral_lmhead_stage_ms(bg.handle)[1])
+            assert bg.status() == 0
+            fl_s = 2.0 * cfg.H * (M_s * cfg.N + M_s * cfg.k_groups * cfg.v)
+            supp.append({"M": M_s, "us_per_step": float(np.mean(ts_)) * 1e3,
+                         "grouped_gemm_stage_us": float(np.mean(th_)) * 1e3,
+                         "tensor_frac_of_sustained_peak": fl_s / (float(np.mean(th_)) * 1e-3) / 1e12 / tf_sust})
+            bg.close()
+            del h_s, ids_s, lps_s
+        out["large_m_supplementary"] = supp
         # extra (second workload, training side): the CSRA objective of Eq. 2 on synthetic features - 4096
         # positions, keys = three other steps and the targets, D = 4096 - a tensor-bound contraction
         n_c, v_c, D_c = 4096, 4, cfg.H
