@@ -44,10 +44,10 @@ extern "C" {
 #define CORAL_MAX_K_TOKENS 32      /* k_tokens <= 32 */
 #define CORAL_ROUTE_STATIC_MAX_ROWS 64 /* M <= 64 for coral_lmhead_route_static */
 
-/* Execution paths (coral_lmhead_set_path / coral_lmhead_stats.path). */
 /* config flags: a handle that stores (and computes) only the groups n with n % world == rank */
 #define CORAL_CFG_SHARD(rank, world) ((uint32_t)(((world) & 0xff) | (((rank) & 0xff) << 8)))
 
+/* Execution paths (coral_lmhead_set_path / coral_lmhead_stats.path). */
 #define CORAL_PATH_AUTO 0          /* chosen from (M, k_groups) */
 #define CORAL_PATH_STREAM 1        /* bulk-copy weight streaming + warp MMA (fp32 accumulate); M <= 128, H % 256 == 0, H <= 4096 */
 #define CORAL_PATH_TCGEN05 2       /* routed grouped GEMM on tcgen05 / TMEM tiles */
@@ -228,9 +228,11 @@ int coral_lmhead_set_path(coral_lmhead_handle h, int path);
  * sim = cosine similarity.  Q_dev [n x D] bf16 row-major are the query features (the B x S output features of
  * the current step), K_dev [views * n x D] bf16 the key set, block s holding the features at positions 0..n-1
  * of another step or the targets; the positives of query i are the keys at position i of every block.  Which
- * features form the key set is the caller's choice (the paper leaves it open).  Features are divided by their
- * norms in fp32 and rounded to bf16; the n x m contraction runs on the tensor cores with fp32 accumulation and
- * its epilogue keeps only (max, sum-exp) per row and the positives, so the similarity matrix is not stored.
+ * features form the key set is the caller's choice (the paper leaves it open).  Every feature is divided by its
+ * norm (sum of squares, norm and scaling in float64) and the unit vector is rounded once to bf16, the operand type
+ * of the contraction: a scaled similarity can differ from Eq. 2 in real arithmetic by up to
+ * (2^-7 + 2^-16) sum_d |q_d k_d| / tau (at most 0.11 at tau = 0.07; typically 1e-3 at D = 4096).  The n x m
+ * contraction runs on the tensor cores with fp32 accumulation and its epilogue keeps only (max, sum-exp) per row and the positives, so the similarity matrix is not stored.
  *
  * coral_csra_workspace_bytes: size of the caller-owned scratch for (n, views, D).
  * coral_csra_infonce: workspace_dev 256-byte aligned, at least that size.  out_loss_dev [1] float;

@@ -42,37 +42,46 @@ def test_closed_form_all_keys_parallel_to_the_query():
     assert np.allclose(r["logits"], r["logits"][0, 0])
 
 
-def test_against_a_library_log_softmax_and_a_float32_free_path():
+def _positive_mask(n, views):
+    mask = np.zeros((n, views * n), bool)
+    for s in range(views):
+        mask[np.arange(n), np.arange(n) + s * n] = True
+    return mask
+
+
+def test_against_library_norms_and_a_library_log_softmax():
+    """The definition spelled with library routines only: numpy's vector norm, scipy's log-softmax, the positives
+    picked with a boolean mask.  Nothing of the oracle is called on the expected side."""
     n, D, views = 24, 40, 2
     Q, K = _rand(n, D, 1), _rand(views * n, D, 2)
     r = co.infonce(Q, K, views, TAU)
-    # the same definition spelled differently: cosine similarities from numpy's norms, scipy's log-softmax,
-    # the positives picked with a boolean mask
     qf = synth.bf16_bits_to_fp32(Q).astype(np.float64)
     kf = synth.bf16_bits_to_fp32(K).astype(np.float64)
     qn = qf / np.linalg.norm(qf, axis=1, keepdims=True)
     kn = kf / np.linalg.norm(kf, axis=1, keepdims=True)
-    qn = synth.bf16_bits_to_fp32(synth.fp32_to_bf16_bits(qn.astype(np.float32))).astype(np.float64)
-    kn = synth.bf16_bits_to_fp32(synth.fp32_to_bf16_bits(kn.astype(np.float32))).astype(np.float64)
+    assert np.allclose(co.normalise(Q), qn, rtol=0, atol=1e-15)
+    assert np.allclose(np.linalg.norm(co.normalise(K), axis=1), 1.0, rtol=0, atol=1e-15)
     lp = log_softmax(qn @ kn.T / TAU, axis=1)
-    mask = np.zeros((n, views * n), bool)
-    for s in range(views):
-        mask[np.arange(n), np.arange(n) + s * n] = True
-    want_rows = -(lp * mask).sum(axis=1) / views
+    want_rows = -(lp * _positive_mask(n, views)).sum(axis=1) / views
     assert np.allclose(r["row_loss"], want_rows, rtol=1e-12, atol=1e-12)
     assert abs(r["loss"] - want_rows.mean()) < 1e-12
-    # without the bf16 rounding of the unit vectors the loss moves by rounding noise only
-    exact = -(log_softmax((qf / np.linalg.norm(qf, axis=1, keepdims=True)) @
-                          (kf / np.linalg.norm(kf, axis=1, keepdims=True)).T / TAU, axis=1) * mask).sum(axis=1) / views
-    assert np.abs(exact - want_rows).max() < 5e-2
+    assert np.allclose(r["logits"], qn @ kn.T / TAU, rtol=0, atol=1e-12)
 
 
 def test_brute_force_on_a_toy():
+    """Pure-Python arithmetic from the widened inputs on: norms by math.sqrt of an exactly rounded sum of squares,
+    dot products and sums by math.fsum.  Neither numpy nor the oracle's normalise is on the expected side."""
     n, D, views = 3, 5, 2
     Q, K = _rand(n, D, 3), _rand(views * n, D, 4)
     r = co.infonce(Q, K, views, TAU)
-    qv = [[float(x) for x in row] for row in co.normalise(Q)]
-    kv = [[float(x) for x in row] for row in co.normalise(K)]
+
+    def unit(bits_row):
+        x = [float(v) for v in synth.bf16_bits_to_fp32(bits_row)]
+        nrm = math.sqrt(math.fsum(v * v for v in x))
+        return [v / nrm for v in x]
+
+    qv = [unit(row) for row in Q]
+    kv = [unit(row) for row in K]
     tot = 0.0
     for i in range(n):
         sims = [math.fsum(a * b for a, b in zip(qv[i], kv[j])) / TAU for j in range(views * n)]
@@ -81,6 +90,36 @@ def test_brute_force_on_a_toy():
         assert abs(li - r["row_loss"][i]) < 1e-10
         tot += li
     assert abs(tot / n - r["loss"]) < 1e-10
+
+
+def test_bf16_rounding_helper_is_round_to_nearest_even():
+    """round_to_bf16 (used only by the diagnostic variant) against a search over the two neighbouring bf16 values
+    built from bit patterns, and on exact half-way points."""
+    x = np.abs(np.random.default_rng(11).standard_normal(4000)) * 0.3 + 1e-3
+    got = co.round_to_bf16(x)
+    down_bits = (x.astype(np.float32).view(np.uint32) >> 16).astype(np.uint16)      # a bf16 at or just below/above x
+    cands = np.stack([synth.bf16_bits_to_fp32((down_bits.astype(np.int64) + d).astype(np.uint16)).astype(np.float64) for d in (-1, 0, 1)])
+    best = cands[np.abs(cands - x).argmin(axis=0), np.arange(x.size)]
+    assert np.array_equal(got, best)
+    # half-way between 1 and 1 + 2^-7 goes to the even neighbour 1; between 1 + 2^-7 and 1 + 2^-6 to 1 + 2^-6
+    assert co.round_to_bf16(np.array([1.0 + 2.0 ** -8]))[0] == 1.0
+    assert co.round_to_bf16(np.array([1.0 + 3 * 2.0 ** -8]))[0] == 1.0 + 2.0 ** -6
+
+
+def test_operand_rounding_moves_a_similarity_by_at_most_the_derived_bound():
+    """bf16 keeps 8 significant bits (spacing 2^-7 relative): each unit-vector element moves by at most 2^-8
+    relative, a product of two by at most 2^-7 + 2^-16, so a scaled similarity by at most
+    (2^-7 + 2^-16) sum_d |q_d k_d| / tau.  The diagnostic
+    variant must stay inside that bound of the definition (and does move: the rounding is really applied)."""
+    n, D, views = 40, 96, 2
+    Q, K = _rand(n, D, 21), _rand(views * n, D, 22)
+    exact = co.infonce(Q, K, views, TAU)
+    quant = co.infonce_bf16_operands(Q, K, views, TAU)
+    bound = (2.0 ** -7 + 2.0 ** -16) * (np.abs(co.normalise(Q)) @ np.abs(co.normalise(K)).T) / TAU
+    gap = np.abs(exact["logits"] - quant["logits"])
+    assert np.all(gap <= bound + 1e-12)
+    assert gap.max() > 1e-4
+    assert np.abs(exact["row_loss"] - quant["row_loss"]).max() <= 2 * bound.max()
 
 
 def test_invariances_scale_and_order_of_negatives():
