@@ -144,6 +144,20 @@ def run_oracle_baseline(cfg, W, gm, Wg, hidden_batches, steps, warmup=0):
     return times, touched, orc.threads()
 
 
+def workload_label(cfg):
+    """The same string in both arms' `config.workload`."""
+    return (f"{cfg.name}: H={cfg.H} V={cfg.V} N={cfg.N} top-{cfg.k_groups} M={cfg.M} k_tokens={cfg.k_tokens}, "
+            f"seed {cfg.seed}")
+
+
+def bench_config(cfg, world):
+    """`config` of the JSON line, the same in both arms."""
+    return {"workload": workload_label(cfg),
+            "l2": f"flush: {FLUSH_BYTES >> 20} MiB written then read before every timed step; {N_BATCHES} hidden "
+                  "batches rotated",
+            "parallelism": f"replicas x{world}, rows sharded by sequence, no collective"}
+
+
 def algorithmic_bytes(cfg, groups_touched, M):
     return groups_touched * cfg.v * cfg.H * 2 + cfg.N * cfg.H * 2 + M * cfg.H * 2 + M * cfg.k_tokens * 8
 
@@ -154,27 +168,6 @@ def main_reference(args, rank):
         return
     from paper_2502_16880_b200 import synth
     cfg = synth.CONFIGS[WORKLOAD].with_(M=args.rows)
-    if args.csra_only:
-        n_c, v_c, D_c = args.csra_only, 4, cfg.H
-        rng_c = np.random.default_rng([cfg.seed, 77])
-        mk = lambda rows: torch.from_numpy(synth.fp32_to_bf16_bits(rng_c.standard_normal((rows, D_c), dtype=np.float32))
-                                           .view(np.int16)).to(dev).view(torch.bfloat16)
-        Qc, Kc = mk(n_c), mk(n_c * v_c)
-        ws_c = torch.empty(lmhead.coral_csra_workspace_bytes(n_c, v_c, D_c), dtype=torch.uint8, device=dev)
-        loss_c = torch.empty(1, dtype=torch.float32, device=dev)
-        ts = []
-        for i in range(args.warmup + args.steps):
-            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            a.record()
-            lmhead.coral_csra_infonce(Qc, Kc, v_c, 0.07, ws_c, loss_c)
-            b.record()
-            torch.cuda.synchronize()
-            if i >= args.warmup:
-                ts.append(a.elapsed_time(b))
-        print(json.dumps({"csra_only": n_c, "views": v_c, "D": D_c, "us": float(np.mean(ts)) * 1e3,
-                          "tflops": 2.0 * n_c * n_c * v_c * D_c / (float(np.mean(ts)) * 1e-3) / 1e12,
-                          "loss": float(loss_c.item()), "status": lmhead.coral_csra_status(ws_c)}))
-        return
     W, gm, Wg = synth.make_w_vocab(cfg), synth.make_group_map(cfg), synth.make_w_gate(cfg)
     hbs = [synth.make_hidden(cfg, cfg.M, batch=b) for b in range(N_BATCHES)]
     times, touched, cores = run_oracle_baseline(cfg, W, gm, Wg, hbs, args.steps, args.warmup)
@@ -186,8 +179,7 @@ def main_reference(args, rank):
         "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": total / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": f"{WORKLOAD}: H={cfg.H} V={cfg.V} N={cfg.N} top-{cfg.k_groups} M={cfg.M} "
-                               f"k_tokens={cfg.k_tokens}"},
+        "config": bench_config(cfg, args.gpus),
         "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }))
@@ -230,6 +222,7 @@ def main():
     lmhead.load_library()
 
     cfg = synth.CONFIGS[WORKLOAD].with_(M=args.rows)
+    headline_cfg = cfg
     if args.csra_only:
         n_c, v_c, D_c = args.csra_only, 4, cfg.H
         rng_c = np.random.default_rng([cfg.seed, 77])
@@ -337,9 +330,13 @@ def main():
         flush.fill_(i)
         torch.sum(flush)
 
-    def time_steps(M, k_groups, steps, warmup, batches, kernel_timing=False, rho=0.0, zipf_s=0.0, on=None, cold=True):
-        """Per-step CUDA-event times (ms) with an L2 flush before every step, outside the event pair."""
+    def time_steps(M, k_groups, steps, warmup, batches, kernel_timing=False, rho=0.0, zipf_s=0.0, on=None, cold=True,
+                   shape=None, stages=None):
+        """Per-step CUDA-event times (ms) with an L2 flush before every step, outside the event pair.  With
+        kernel_timing the library records events around its stages (which keeps the kernels of a call from
+        overlapping, so step times come from runs without it); `stages`, a list, receives (route, head, merge) ms."""
         head = on if on is not None else default_head
+        cfg = shape if shape is not None else headline_cfg
         hb_bits = [synth.make_hidden(cfg.with_(rho=rho, zipf_s=zipf_s), M, batch=b) for b in batches]
         hds = [dev_bf16(b) for b in hb_bits]
         ids = torch.empty((M, cfg.k_tokens), dtype=torch.int32, device=dev)
@@ -372,6 +369,8 @@ def main():
             touched.append(per_batch_union[i % len(hds)])
             if kernel_timing:
                 kms.append(lmhead.coral_lmhead_head_kernel_ms(head.handle))
+                if stages is not None:
+                    stages.append(lmhead.coral_lmhead_stage_ms(head.handle))
         torch.cuda.synchronize()
         if world > 1:
             dist.barrier()
@@ -379,6 +378,48 @@ def main():
         lmhead.coral_lmhead_set_kernel_timing(head.handle, False)
         assert head.status() == 0
         return ms, kms, touched, launches, hb_bits
+
+    NOMINAL_HBM_GBPS = 7700.0     # HBM3e nameplate of the HGX B200 (context; the fractions that are judged use the measured copy peak)
+
+    def copy_floor_us(on, nbytes, in_flight=0, repeats=1, cold=True, n=13):
+        """Mean time (us) of the do-nothing bulk-copy stream over the first nbytes of `on`'s packed head."""
+        nbytes = int(nbytes) // 16384 * 16384
+        ts = []
+        for i in range(n):
+            if cold:
+                flush_l2(i)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            lmhead.coral_lmhead_copy_floor(on.handle, nbytes, stream, in_flight=in_flight, repeats=repeats)
+            b.record(stream)
+            torch.cuda.synchronize()
+            if i >= 3:
+                ts.append(a.elapsed_time(b))
+        assert on.status() == 0
+        return float(np.mean(ts)) * 1e3
+
+    def timed_case(on, shape, M, k_groups, steps):
+        """One (shape, M, k_groups) point, cold L2: whole-step time, the three stages timed by events inside the
+        call (a separate run), and the copy floor of the same weight bytes."""
+        ms_m, _, t_m, _, _ = time_steps(M, k_groups, steps, 3, my_batches, on=on, shape=shape)
+        stg = []
+        _, kms, _, _, _ = time_steps(M, k_groups, min(steps, 30), 3, my_batches, kernel_timing=True, on=on,
+                                     shape=shape, stages=stg)
+        c2 = shape.with_(M=M, k_groups=k_groups)
+        b_m = float(np.mean([algorithmic_bytes(c2, u, M) for u in t_m]))
+        w_m = float(np.mean([u * c2.v * c2.H * 2 for u in t_m]))
+        us = float(np.mean(ms_m)) * 1e3
+        k_us = float(np.mean(kms)) * 1e3
+        floor = copy_floor_us(on, w_m)
+        return {"M": M, "k_groups": k_groups, "path": int(on.stats().path), "us_per_step": us,
+                "us_per_step_median": float(np.median(ms_m)) * 1e3, "GBps": b_m / us / 1e3,
+                "hbm_frac": b_m / us / 1e3 / peak, "hbm_frac_of_nominal": b_m / us / 1e3 / NOMINAL_HBM_GBPS,
+                "groups_touched_mean": float(np.mean(t_m)), "roofline_us_at_measured_peak": b_m / peak / 1e3,
+                "stage_us": {"router": float(np.mean([x[0] for x in stg])) * 1e3,
+                             "head_kernel": float(np.mean([x[1] for x in stg])) * 1e3,
+                             "merge": float(np.mean([x[2] for x in stg])) * 1e3},
+                "head_kernel_us": k_us, "head_kernel_GBps": w_m / k_us / 1e3, "head_kernel_hbm_frac": w_m / k_us / 1e3 / peak,
+                "copy_floor_us_same_bytes": floor, "head_kernel_frac_of_copy_floor": floor / k_us}
 
     my_batches = batches_for_rank(rank, world)
     sampler = ClockSampler(_visible_index(local_rank))
@@ -397,23 +438,14 @@ def main():
     k_ms = float(np.mean(kms))
     achieved = k_bytes / (k_ms * 1e-3) / 1e9
     # floor for that kernel: a do-nothing bulk-copy stream of the same number of bytes of the packed head, cold L2
-    floor_bytes = int(k_bytes) // 16384 * 16384
-    fl_ms = []
-    for i in range(23):
-        flush_l2(i)
-        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        a.record(stream)
-        lmhead.coral_lmhead_copy_floor(head.handle, floor_bytes, stream)
-        b.record(stream)
-        torch.cuda.synchronize()
-        if i >= 3:
-            fl_ms.append(a.elapsed_time(b))
-    assert head.status() == 0
-    copy_floor_us = float(np.mean(fl_ms)) * 1e3
+    copy_floor_us_ = copy_floor_us(head, k_bytes, n=23)
     roofline = {"bound": "hbm", "kernel": "head_stream_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                "copy_floor_us_same_bytes": copy_floor_us, "frac_of_copy_floor": copy_floor_us / (k_ms * 1e3),
+                "copy_floor_us_same_bytes": copy_floor_us_, "frac_of_copy_floor": copy_floor_us_ / (k_ms * 1e3),
                 "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
+                "frac_of_nominal_hbm3e": achieved / NOMINAL_HBM_GBPS, "nominal_hbm3e_GBps": NOMINAL_HBM_GBPS,
                 "traffic": None if STREAM_TRAFFIC_RATIO is None else STREAM_TRAFFIC_RATIO * k_bytes,
+                "traffic_source": "bytes x the DRAM-bytes-per-algorithmic-byte ratio of the ncu capture in profiles/ "
+                                  "(not measured in this run)",
                 "avg_launch_us": k_ms * 1e3, "algorithmic_bytes_per_launch": k_bytes}
 
     # end to end through the host-buffer entry point (pinned host memory; copies inside the timed region)
@@ -439,16 +471,14 @@ def main():
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": tot_ms / args.steps, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16 inputs, f32 accumulate", "data": "synthetic",
-        "config": {"workload": f"{WORKLOAD}: H={cfg.H} V={cfg.V} N={cfg.N} top-{cfg.k_groups} M={cfg.M} "
-                               f"k_tokens={cfg.k_tokens}, seed {cfg.seed}",
-                   "l2": f"flush: {FLUSH_BYTES >> 20} MiB written then read before every timed step; {N_BATCHES} hidden "
-                         "batches rotated", "parallelism": f"replicas x{world}, rows sharded by sequence, no collective"},
+        "config": bench_config(cfg, world),
         "us_per_step": tot_ms / args.steps * 1e3,
         "us_per_step_median": float(np.median(ms)) * 1e3,
         "us_per_step_p10": float(np.percentile(ms, 10)) * 1e3,
         "us_per_step_p90": float(np.percentile(ms, 90)) * 1e3,
         "groups_touched_mean": float(np.mean(touched)),
         "hbm_frac_whole_step": value / (peak * world),
+        "hbm_frac_whole_step_of_nominal": value / (NOMINAL_HBM_GBPS * world),
         "roofline": roofline, "e2e": e2e, "gpu_launches": launches,
     }
 
@@ -458,15 +488,7 @@ def main():
         # not the headline - in a real draft cycle the other layers' weights stream through L2 between head calls
         ms_w, _, _, _, _ = time_steps(cfg.M, cfg.k_groups, extra_steps, 3, my_batches, cold=False)
         out["warm_l2_us_per_step"] = float(np.mean(ms_w)) * 1e3
-        also = []
-        for M in (1, 60):
-            ms_m, _, t_m, _, _ = time_steps(M, cfg.k_groups, extra_steps, 3, my_batches)
-            c2 = cfg.with_(M=M)
-            b_m = float(np.mean([algorithmic_bytes(c2, u, M) for u in t_m]))
-            us = float(np.mean(ms_m)) * 1e3
-            also.append({"M": M, "us_per_step": us, "GBps": b_m / us / 1e3, "hbm_frac": b_m / us / 1e3 / peak,
-                         "groups_touched_mean": float(np.mean(t_m))})
-        out["other_M"] = also
+        out["other_M"] = [timed_case(head, cfg, M, cfg.k_groups, extra_steps) for M in (1, 60)]
         # extra (not a workload of the list): rows correlated like tree siblings of one parent, where the union
         # of selected groups no longer saturates (Appendix B: the worst case is unlikely in practice)
         ms_c, _, t_c, _, _ = time_steps(60, cfg.k_groups, extra_steps, 3, my_batches, rho=0.3)
@@ -609,6 +631,50 @@ def main():
             bg.close()
             del h_s, ids_s, lps_s
         out["large_m_supplementary"] = supp
+        # the other shapes of the workload list (paper Table 1: H, V; Table 4: N, top-n), same cold-L2 protocol
+        def torch_dense_us(Wt, hidden_bits, k_tokens):
+            hd_ = dev_bf16(hidden_bits)
+            tms_ = []
+            for i in range(13):
+                flush_l2(i)
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record()
+                torch.topk(torch.log_softmax(torch.matmul(hd_, Wt.T).float(), dim=1), k_tokens, dim=1)
+                b.record()
+                torch.cuda.synchronize()
+                if i >= 3:
+                    tms_.append(a.elapsed_time(b))
+            return float(np.mean(tms_)) * 1e3
+
+        for name, cases in (("llama2_7b", [(1, 4), (8, 4), (60, 4), (8, 32)]),
+                            ("qwen25_7b", [(60, 2), (60, 4), (60, 8), (60, 16), (60, 64)])):
+            scfg = synth.CONFIGS[name]
+            Ws = dev_bf16(synth.make_w_vocab(scfg))
+            shead = lmhead.LMHead(Ws, torch.from_numpy(synth.make_group_map(scfg)), dev_bf16(synth.make_w_gate(scfg)),
+                                  max_M=64, max_k_groups=scfg.N, max_k_tokens=scfg.k_tokens)
+            pts = [timed_case(shead, scfg, M, kg, extra_steps) for M, kg in cases]
+            for pt in pts:
+                if pt["k_groups"] == scfg.N:
+                    pt["dense_equivalent"] = True
+                    pt["torch_matmul_logsoftmax_topk_us"] = torch_dense_us(
+                        Ws, synth.make_hidden(scfg, pt["M"], batch=my_batches[0]), scfg.k_tokens)
+            out[name] = {"shape": f"H={scfg.H} V={scfg.V} N={scfg.N} v={scfg.v} k_tokens={scfg.k_tokens}", "points": pts}
+            assert shead.status() == 0
+            shead.close()
+            del Ws, shead
+        # what an SM can take in: the do-nothing bulk-copy stream (one CTA per SM, 16 KiB copies) with 4, 8 and 13
+        # copies in flight, from HBM (cold L2, the touched bytes of the headline call) and from L2 (a 48 MiB region
+        # swept 9 times against once: the 8 extra sweeps hit L2)
+        l2_region = 48 << 20
+        ingest = []
+        for fl in (4, 8, 13):
+            t_h = copy_floor_us(head, k_bytes, in_flight=fl)
+            t1 = copy_floor_us(head, l2_region, in_flight=fl, repeats=1, cold=False)
+            t9 = copy_floor_us(head, l2_region, in_flight=fl, repeats=9, cold=False)
+            ingest.append({"copies_in_flight_per_sm": fl, "hbm_to_smem_GBps": (int(k_bytes) // 16384 * 16384) / t_h / 1e3,
+                           "l2_to_smem_GBps": 8.0 * l2_region / max(t9 - t1, 1e-3) / 1e3,
+                           "l2_to_smem_GBps_per_sm": 8.0 * l2_region / max(t9 - t1, 1e-3) / 1e3 / torch.cuda.get_device_properties(dev).multi_processor_count})
+        out["smem_ingest_probe"] = ingest
         # extra (second workload, training side): the CSRA objective of Eq. 2 on synthetic features - 4096
         # positions, keys = three other steps and the targets, D = 4096 - a tensor-bound contraction
         n_c, v_c, D_c = 4096, 4, cfg.H

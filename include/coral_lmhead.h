@@ -38,6 +38,7 @@ extern "C" {
 #define CORAL_ERR_TIMEOUT (-5)     /* a bounded device-side wait gave up (device status word) */
 #define CORAL_ERR_BOUNDS (-6)      /* a device-side index check failed (device status word) */
 #define CORAL_ERR_TOO_LARGE (-7)   /* request exceeds a built-in size limit (coral_lmhead_route_static, coral_tree_expand) */
+#define CORAL_ERR_NONFINITE (-8)   /* a router score was NaN (device status word) */
 
 /* Limits of this build. */
 #define CORAL_MAX_GROUPS 256       /* n_groups <= 256 */
@@ -254,9 +255,12 @@ int coral_csra_status(void *workspace_dev, void *stream);
  * size of L2 is set aside for such lines (cudaLimitPersistingL2CacheSize: a setting of this process's CUDA
  * context that takes L2 away from everything else the process runs and ends with the process; without the
  * set-aside the hint alone changed nothing).  How much survives depends on what runs between two calls.
- * Meant for contiguous, frequency-ordered group maps; n_hot = 0 (the default) switches it off, resets the
- * persisting lines and returns the set-aside.  Applies to calls on the streaming path.  Synchronises nothing,
- * but changes a context-wide limit: call it at set-up time, not between overlapping work.
+ * Meant for contiguous, frequency-ordered group maps; n_hot = 0 (the default) switches it off.  Applies to
+ * calls on the streaming path.  Synchronises nothing, but the set-aside is PROCESS-WIDE state of the CUDA context,
+ * shared with every other handle and with anything else the process runs (last writer wins): the call only ever
+ * raises the limit, remembers the value it found, and puts that value back (and resets the persisting lines)
+ * when the hot groups are switched off or the handle is destroyed.  Call it at set-up time, not between
+ * overlapping work, and not from two handles that are meant to hold different set-asides at once.
  */
 int coral_lmhead_set_hot_groups(coral_lmhead_handle h, int n_hot);
 
@@ -271,13 +275,16 @@ int coral_lmhead_set_hot_groups(coral_lmhead_handle h, int n_hot);
 int coral_lmhead_selftest_wait_expiry(coral_lmhead_handle h, void *stream);
 
 /*
- * Measurement aid with no counterpart in the paper: streams the first `bytes` of the packed head into shared
- * memory with plain contiguous 16 KiB bulk copies (one CTA per SM, eight copies in flight each) and does
- * nothing with them.  Timed by the caller with events on `stream`, from a cold L2, it gives the floor for the
- * weight-streaming kernel of a draft call that reads as many bytes: a one-shot read of a few hundred megabytes
- * does not reach the bandwidth of a long copy.  bytes in [16384, packed_bytes]; asynchronous, no allocation.
+ * Bench-side measurement aid with no counterpart in the paper (not part of the draft step): streams the first
+ * `bytes` of the packed head into shared memory with plain contiguous 16 KiB bulk copies (one CTA per SM,
+ * `in_flight` copies outstanding each; 0 = the default of 8, at most 13) and does nothing with them; the region
+ * is swept `repeats` times (1..64).  Timed by the caller with events on `stream`, from a cold L2 and with
+ * repeats = 1, it gives the floor for the weight-streaming kernel of a draft call that reads as many bytes: a
+ * one-shot read of a few hundred megabytes does not reach the bandwidth of a long copy.  With a region smaller
+ * than L2, the time difference between two repeat counts gives the rate at which the SMs can take bytes in from
+ * L2.  bytes in [16384, packed_bytes]; asynchronous, no allocation.
  */
-int coral_lmhead_copy_floor(coral_lmhead_handle h, long long bytes, void *stream);
+int coral_lmhead_copy_floor(coral_lmhead_handle h, long long bytes, int in_flight, int repeats, void *stream);
 
 /*
  * Measurement aid for the dominant kernel (the one that streams the selected
@@ -293,8 +300,14 @@ int coral_lmhead_head_kernel_ms(coral_lmhead_handle h, float *ms);
 int coral_lmhead_stage_ms(coral_lmhead_handle h, float *route_ms, float *head_ms, float *merge_ms);
 
 /*
- * Synchronise `stream`, return the device status word of the handle (CORAL_OK,
- * CORAL_ERR_TIMEOUT, CORAL_ERR_BOUNDS) and clear it.
+ * Synchronise `stream`, return the device status word of the handle and clear it: CORAL_OK;
+ * CORAL_ERR_TIMEOUT (a bounded wait gave up); CORAL_ERR_BOUNDS (forced_groups held a group outside [0, N) or
+ * the same group twice in a row); CORAL_ERR_NONFINITE (a router score was NaN, e.g. from a NaN hidden state:
+ * such a score is ranked below every other score, so each row still gets k_groups distinct groups).
+ * The word is sticky: the first problem stays until this call reads it, and while it is non-zero the
+ * kernels after the router stage of every draft call on the handle do nothing, so that nothing ever indexes
+ * with an inconsistent selection; the outputs of those calls are not written.  (The paper does not say what
+ * a router should do with non-finite scores; inputs are expected to be finite.)
  */
 int coral_lmhead_status(coral_lmhead_handle h, void *stream);
 

@@ -117,6 +117,13 @@ __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepc
 
 __device__ __forceinline__ void set_status(DeviceState* st, int code) { atomicCAS(&st->status, 0, code); }
 
+// The status word is sticky until the host reads it.  A call whose router stage reported a problem (forced
+// groups out of range or repeated: the bucket arrays are then inconsistent) must not be followed by kernels
+// that index with those arrays; every kernel after the router stage checks this first and does nothing.
+__device__ __forceinline__ bool call_is_poisoned(const DeviceState* st) {
+    return *reinterpret_cast<const volatile int*>(&st->status) != 0;
+}
+
 // Vocab sharding over several GPUs: group n belongs to the GPU with rank n % world.
 __device__ __forceinline__ bool group_is_local(const CallView& c, int n) {
     return c.shard_world <= 1 || n % c.shard_world == c.shard_rank;

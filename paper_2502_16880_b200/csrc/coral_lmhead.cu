@@ -175,6 +175,8 @@ struct coral_lmhead_s {
     int out_mode;        // CORAL_OUTPUT_*
     int shard_rank, shard_world;   // vocab sharding (coral_lmhead_set_group_shard); world 1 = off
     int hot_groups;                // leading groups whose weights are loaded with an evict-last L2 hint (0 = off)
+    bool l2_limit_changed;         // this handle raised the context's persisting-L2 limit ...
+    size_t l2_limit_before;        // ... from this value (restored when the hot groups are released)
     uint16_t* w1;        // [H][H] bf16 first router layer (Eq. 7), library-owned, or null
     float* router_u;     // [max_M][H] fp32 act(W1 h) + h, library-owned
     CUtensorMap map_w, map_h, map_h64, map_h32;   // hidden-row blocks read whole (128 rows) or only their first 64 / 32 rows
@@ -321,6 +323,7 @@ const char* coral_lmhead_error_string(int code) {
         case CORAL_ERR_NOMEM: return "out of memory";
         case CORAL_ERR_TIMEOUT: return "device-side wait timed out";
         case CORAL_ERR_BOUNDS: return "device-side index check failed";
+        case CORAL_ERR_NONFINITE: return "a router score was NaN";
         case CORAL_ERR_TOO_LARGE: return "size exceeds a built-in limit (fixed scratch of the no-allocation entry point, tree step)";
         default: return "unknown status";
     }
@@ -437,8 +440,11 @@ int coral_lmhead_create(coral_lmhead_handle* out, const coral_lmhead_config* cfg
     return CORAL_OK;
 }
 
+static int release_hot_groups(coral_lmhead_handle h);
+
 int coral_lmhead_destroy(coral_lmhead_handle h) {
     if (!h) return CORAL_OK;
+    release_hot_groups(h);
     if (h->own_packed && h->packed) cudaFree(h->packed);
     if (h->own_ws && h->ws) cudaFree(h->ws);
     if (h->w1) cudaFree(h->w1);
@@ -687,13 +693,21 @@ int coral_tree_expand(const float* parent_scores_dev, const int32_t* cand_ids_de
     return cudaGetLastError() == cudaSuccess ? CORAL_OK : CORAL_ERR_CUDA;
 }
 
+// The L2 set-aside is a limit of the process's CUDA context, shared with every other handle and with whatever
+// else the process runs.  The handle only ever raises it, remembers what it found, and puts that back when its
+// hot groups are switched off or the handle is destroyed.
+static int release_hot_groups(coral_lmhead_handle h) {
+    if (h->hot_groups == 0) return CORAL_OK;
+    h->hot_groups = 0;
+    if (!h->l2_limit_changed) return CORAL_OK;
+    h->l2_limit_changed = false;
+    if (cudaCtxResetPersistingL2Cache() != cudaSuccess) return CORAL_ERR_CUDA;
+    return cudaDeviceSetLimit(cudaLimitPersistingL2CacheSize, h->l2_limit_before) == cudaSuccess ? CORAL_OK : CORAL_ERR_CUDA;
+}
+
 int coral_lmhead_set_hot_groups(coral_lmhead_handle h, int n_hot) {
     if (!h || n_hot < 0 || n_hot > h->cfg.n_groups) return CORAL_ERR_INVALID;
-    if (n_hot == 0) {
-        h->hot_groups = 0;
-        if (cudaCtxResetPersistingL2Cache() != cudaSuccess) return CORAL_ERR_CUDA;
-        return cudaDeviceSetLimit(cudaLimitPersistingL2CacheSize, 0) == cudaSuccess ? CORAL_OK : CORAL_ERR_CUDA;
-    }
+    if (n_hot == 0) return release_hot_groups(h);
     // evict-last lines only outlive other traffic inside the part of L2 that is set aside for them
     int dev = 0, max_persist = 0;
     if (cudaGetDevice(&dev) != cudaSuccess ||
@@ -702,17 +716,25 @@ int coral_lmhead_set_hot_groups(coral_lmhead_handle h, int n_hot) {
     if (max_persist <= 0) return CORAL_ERR_INVALID;                     // the device has no such set-aside
     const size_t want = (size_t)n_hot * h->L.T16 * h->L.KB * 2048;      // packed bytes of the hot groups
     const size_t carve = want < (size_t)max_persist ? want : (size_t)max_persist;
-    if (cudaDeviceSetLimit(cudaLimitPersistingL2CacheSize, carve) != cudaSuccess) return CORAL_ERR_CUDA;
+    size_t now = 0;
+    if (cudaDeviceGetLimit(&now, cudaLimitPersistingL2CacheSize) != cudaSuccess) return CORAL_ERR_CUDA;
+    if (carve > now) {                                                  // never shrink what somebody else set
+        if (!h->l2_limit_changed) h->l2_limit_before = now;
+        if (cudaDeviceSetLimit(cudaLimitPersistingL2CacheSize, carve) != cudaSuccess) return CORAL_ERR_CUDA;
+        h->l2_limit_changed = true;
+    }
     h->hot_groups = n_hot;
     return CORAL_OK;
 }
 
-int coral_lmhead_copy_floor(coral_lmhead_handle h, long long bytes, void* stream) {
+int coral_lmhead_copy_floor(coral_lmhead_handle h, long long bytes, int in_flight, int repeats, void* stream) {
     if (!h || bytes < kCopyChunk || (size_t)bytes > h->L.packed_bytes) return CORAL_ERR_INVALID;
-    if (cudaFuncSetAttribute(copy_probe_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kCopyStages * kCopyChunk) !=
-        cudaSuccess) return CORAL_ERR_CUDA;
-    copy_probe_kernel<<<h->sms, 32, kCopyStages * kCopyChunk, static_cast<cudaStream_t>(stream)>>>(
-        h->packed, bytes / kCopyChunk, reinterpret_cast<DeviceState*>(h->ws + h->L.state),
+    if (in_flight == 0) in_flight = kCopyStages;
+    if (in_flight < 1 || in_flight > kCopyMaxStages || repeats < 1 || repeats > 64) return CORAL_ERR_INVALID;
+    if (cudaFuncSetAttribute(copy_probe_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             kCopyMaxStages * kCopyChunk) != cudaSuccess) return CORAL_ERR_CUDA;
+    copy_probe_kernel<<<h->sms, 32, in_flight * kCopyChunk, static_cast<cudaStream_t>(stream)>>>(
+        h->packed, bytes / kCopyChunk, in_flight, repeats, reinterpret_cast<DeviceState*>(h->ws + h->L.state),
         reinterpret_cast<unsigned*>(h->ws + h->L.cand_val));
     return cudaGetLastError() == cudaSuccess ? CORAL_OK : CORAL_ERR_CUDA;
 }

@@ -90,6 +90,7 @@ __global__ void __launch_bounds__(kSimtThreads) head_simt_kernel(CallView c, flo
     uint16_t* hs = reinterpret_cast<uint16_t*>(smem_raw);
     float* zs = reinterpret_cast<float*>(smem_raw + (size_t)kSimtRowBlock * c.H * sizeof(uint16_t));
     const int n = blockIdx.y, t = blockIdx.x;
+    if (call_is_poisoned(c.state)) return;        // the router stage reported a problem: index with nothing
     const int cnt = c.group_count[n];
     if (cnt == 0) return;
     const int off = c.group_offset[n];

@@ -344,6 +344,7 @@ __global__ void __launch_bounds__(kStreamThreads, 1) head_stream_kernel(CallView
 
     pdl_wait();                   // the router stage's outputs are complete from here on
     pdl_launch_dependents();      // the merge kernel may start reading the router's outputs
+    if (call_is_poisoned(c.state)) return;                   // the router stage reported a problem: index with nothing
     if (c.adaptive && c.state->path_choice != 1) return;     // the router chose the tensor-core kernel for this call
     const int n_items = c.state->n_virtual * g.T;
     const int per = (n_items + g.grid - 1) / g.grid;
@@ -476,6 +477,7 @@ __global__ void __launch_bounds__(kMergeStreamThreads) merge_stream_kernel(CallV
     unsigned char* s_pslot = reinterpret_cast<unsigned char*>(s_live + p_cap);
 
     // The router's outputs were complete before the streaming kernel let this grid start.
+    if (call_is_poisoned(c.state)) return;        // the descriptors may be inconsistent: emit nothing (the status says why)
     const int n_items = c.state->n_virtual * g.T;
     const int per = max(1, (n_items + g.grid - 1) / g.grid);
     for (int s = threadIdx.x; s < c.k_groups; s += kMergeStreamThreads) {

@@ -139,6 +139,7 @@ __global__ void __launch_bounds__(128) tc_gather_kernel(CallView c, uint16_t* __
     const int p = blockIdx.x;
     pdl_wait();                                              // launched over the tail of the router stage
     pdl_launch_dependents();
+    if (call_is_poisoned(c.state)) return;                   // the router stage reported a problem: index with nothing
     if (c.adaptive && c.state->path_choice != 2) return;     // the router chose the streaming kernel for this call
     if (p >= c.group_offset[c.N]) return;          // fewer pairs than M * k_groups when the vocab is sharded
     const int m = c.bucket_row[p];
@@ -358,7 +359,8 @@ __global__ void __launch_bounds__(kTcThreads, 1)
     const uint32_t tmem_base = *tmem_slot;
     pdl_wait();                                              // gathered rows and router outputs are complete from here on
     // (no early release of the merge kernel: it reads this kernel's partials right after its own metadata)
-    const bool skip = c.adaptive && c.state->path_choice != 2;   // the router chose the streaming kernel for this call
+    // nothing to do: the router chose the streaming kernel for this call, or the router stage reported a problem
+    const bool skip = (c.adaptive && c.state->path_choice != 2) || call_is_poisoned(c.state);
 
     // this CTA's run of sub-tiles
     const int n_tiles = skip ? 0 : c.state->n_virtual * g.tiles;

@@ -13,6 +13,7 @@ __global__ void __launch_bounds__(kMergeThreads) merge_kernel(CallView c, int32_
                                                               float* __restrict__ out_logprobs,
                                                               float* __restrict__ lse_tap) {
     const int m = blockIdx.x;
+    if (call_is_poisoned(c.state)) return;        // the partials were not written: emit nothing (the status says why)
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     constexpr int kWarps = kMergeThreads / 32;
     __shared__ float s_f[kWarps];

@@ -61,6 +61,10 @@ __global__ void __launch_bounds__(kSelectWarps * 32) select_kernel(CallView c, c
     for (int i = 0; i < kPer; ++i) {
         const int n = lane + 32 * i;
         val[i] = (n < c.N) ? c.gate[(size_t)m * c.N + n] : kNegInf;
+        if (val[i] != val[i]) {                      // NaN orders against nothing: rank it last and report
+            val[i] = kNegInf;
+            set_status(c.state, -8);
+        }
         slot[i] = -1;
     }
     for (int s = 0; s < c.k_groups; ++s) {
@@ -132,6 +136,10 @@ __device__ __forceinline__ void route_select_row(const CallView& c, const int32_
         for (int i = 0; i < NPER; ++i) {
             const int n = lane + 32 * i;
             val[i] = (n < c.N) ? __ldcg(c.gate + (size_t)m * c.N + n) : kNegInf;
+            if (val[i] != val[i]) {                  // NaN orders against nothing: rank it last and report, so that
+                val[i] = kNegInf;                    // every row still gets exactly k_groups distinct groups
+                set_status(c.state, -8);
+            }
             if (n < c.N) s_val[n] = val[i];
         }
         __syncwarp();

@@ -24,6 +24,7 @@ CORAL_ERR_NOMEM = -4
 CORAL_ERR_TIMEOUT = -5
 CORAL_ERR_BOUNDS = -6
 CORAL_ERR_TOO_LARGE = -7
+CORAL_ERR_NONFINITE = -8
 CORAL_ROUTE_STATIC_MAX_ROWS = 64
 CORAL_OUTPUT_JOINT, CORAL_OUTPUT_FACTORISED = 0, 1
 CORAL_PATH_AUTO, CORAL_PATH_STREAM, CORAL_PATH_TCGEN05, CORAL_PATH_SIMT_PLAIN, CORAL_PATH_ADAPTIVE = 0, 1, 2, 3, 4
@@ -56,7 +57,7 @@ _SIGNATURES = {
     "coral_lmhead_set_group_shard": (_i, [_vp, _i, _i]),
     "coral_lmhead_draft_partial": (_i, [_vp, _vp, _i, _i, _i, _vp, _vp]),
     "coral_lmhead_merge_partials": (_i, [_vp, _i, _i, _i, _vp, _vp, _vp]),
-    "coral_lmhead_copy_floor": (_i, [_vp, ctypes.c_longlong, _vp]),
+    "coral_lmhead_copy_floor": (_i, [_vp, ctypes.c_longlong, _i, _i, _vp]),
     "coral_lmhead_set_hot_groups": (_i, [_vp, _i]),
     "coral_csra_workspace_bytes": (_i, [_i, _i, _i, ctypes.POINTER(ctypes.c_size_t)]),
     "coral_csra_infonce": (_i, [_vp, _vp, _i, _i, _i, ctypes.c_float, _vp, _vp, _vp, _vp, _vp]),
@@ -240,9 +241,11 @@ def coral_lmhead_set_router_mlp(handle, W1=None, stream=None) -> None:
            "coral_lmhead_set_router_mlp")
 
 
-def coral_lmhead_copy_floor(handle, nbytes: int, stream=None) -> None:
-    """Measurement aid: a do-nothing stream of the first `nbytes` of the packed head (time it with events)."""
-    _check(load_library().coral_lmhead_copy_floor(handle, int(nbytes), _stream_ptr(stream)), "coral_lmhead_copy_floor")
+def coral_lmhead_copy_floor(handle, nbytes: int, stream=None, in_flight: int = 0, repeats: int = 1) -> None:
+    """Measurement aid: a do-nothing stream of the first `nbytes` of the packed head, `repeats` sweeps with
+    `in_flight` 16 KiB copies outstanding per SM (0 = default); time it with events."""
+    _check(load_library().coral_lmhead_copy_floor(handle, int(nbytes), int(in_flight), int(repeats),
+                                                  _stream_ptr(stream)), "coral_lmhead_copy_floor")
 
 
 def coral_csra_workspace_bytes(n: int, views: int, D: int) -> int:

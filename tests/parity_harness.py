@@ -106,28 +106,38 @@ def compare(W, gm, Wg, hidden_bits, k_groups, k_tokens, gpu, forced_groups=None,
             score = ref.log_router[m, ref.groups[m]][:, None] + ref.logits[m] - ref.group_lse[m][:, None]
         else:
             score = ref.logits[m] - ref.lse[m]
-        zmap = dict(zip(ref.logit_tokens[m].ravel().tolist(), score.ravel().tolist()))
+        # score of a token id by binary search in the row's sorted active token list (all rows at full size
+        # would cost a Python dictionary of 16 000 entries per row otherwise)
+        tokens = ref.logit_tokens[m].ravel()
+        order = np.argsort(tokens, kind="stable")
+        tok_sorted, score_sorted = tokens[order], score.ravel()[order]
+
+        def lookup(t):
+            at = np.minimum(np.searchsorted(tok_sorted, t), tok_sorted.size - 1)
+            return tok_sorted[at] == t, score_sorted[at]
+
         if len(set(ids[m].tolist())) != k_tokens:
             rep.errors.append(f"row {m}: duplicate ids {ids[m].tolist()}")
             continue
-        for i in range(k_tokens):
-            t = int(ids[m, i])
-            if t not in zmap:
-                rep.errors.append(f"row {m} pos {i}: id {t} is not in an active group")
-                break
-            if t != int(ref.ids[m, i]):
-                if close(zmap[t], zmap[int(ref.ids[m, i])]):
-                    rep.tie_resolved_ids += 1
-                else:
-                    rep.errors.append(f"row {m} pos {i}: id {t} (score={zmap[t]}) != oracle {int(ref.ids[m, i])} "
-                                      f"(score={zmap[int(ref.ids[m, i])]})")
-                    break
-            want = zmap[t]
-            err = abs(float(lps[m, i]) - want)
-            rep.max_logprob_err = max(rep.max_logprob_err, err)
-            if not close(float(lps[m, i]), want):
-                rep.errors.append(f"row {m} pos {i}: logprob {float(lps[m, i])} != oracle {want}")
-                break
+        active, got = lookup(ids[m].astype(np.int64))
+        _, want_ref = lookup(ref.ids[m].astype(np.int64))
+        if not active.all():
+            i = int(np.flatnonzero(~active)[0])
+            rep.errors.append(f"row {m} pos {i}: id {int(ids[m, i])} is not in an active group")
+        else:
+            differs = ids[m] != ref.ids[m]
+            tie = differs & close(got, want_ref)
+            wrong = differs & ~tie
+            lp_bad = ~close(lps[m], got)
+            rep.tie_resolved_ids += int(tie.sum())
+            rep.max_logprob_err = max(rep.max_logprob_err, float(np.abs(lps[m] - got).max()))
+            if wrong.any():
+                i = int(np.flatnonzero(wrong)[0])
+                rep.errors.append(f"row {m} pos {i}: id {int(ids[m, i])} (score={got[i]}) != oracle {int(ref.ids[m, i])} "
+                                  f"(score={want_ref[i]})")
+            elif lp_bad.any():
+                i = int(np.flatnonzero(lp_bad)[0])
+                rep.errors.append(f"row {m} pos {i}: logprob {float(lps[m, i])} != oracle {got[i]}")
         if np.any(np.diff(lps[m]) > 0):
             rep.errors.append(f"row {m}: log-probs not sorted descending")
         if len(rep.errors) >= max_errors:

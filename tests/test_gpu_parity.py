@@ -175,9 +175,7 @@ def test_paper_shapes(path, name, Ms):
         head.set_path(path)
         out = ph.gpu_draft_numpy(head, hb, cfg.k_groups, cfg.k_tokens)
         assert head.status() == 0
-        # the oracle checks all rows for M <= 8 and a spread sample of rows beyond
-        rows = np.arange(M) if M <= 8 else np.unique(np.linspace(0, M - 1, 6).astype(int))
-        rep = ph.compare(W, gm, Wg, hb[rows], cfg.k_groups, cfg.k_tokens, {k: v[rows] for k, v in out.items()})
+        rep = ph.compare(W, gm, Wg, hb, cfg.k_groups, cfg.k_tokens, out)       # every row, every tap
         assert rep.ok, rep.errors
         st = head.stats()
         assert st.groups_touched == len(set(out["groups"].ravel().tolist()))
@@ -188,11 +186,12 @@ def test_qwen_shape_group_sweep_and_dense_equivalence(path):
     cfg, W, gm, Wg, head = _weights("qwen25_7b")
     M = 60
     hb = synth.make_hidden(cfg, M)
-    rows = np.array([0, M // 2, M - 1])
     for kg in (2, 4, 8, 16, 64):
         head.set_path(path)
         out = ph.gpu_draft_numpy(head, hb, kg, cfg.k_tokens)
         assert head.status() == 0
+        # every row up to the workload's top-8; a spread of 12 rows where a row costs 2x / 8x the oracle time
+        rows = np.arange(M) if kg <= 8 else np.unique(np.linspace(0, M - 1, 12).astype(int))
         rep = ph.compare(W, gm, Wg, hb[rows], kg, cfg.k_tokens, {k: v[rows] for k, v in out.items()})
         assert rep.ok, (kg, rep.errors)
     # k_groups = N is the dense head: every row's ids/log-probs equal a dense log-softmax (library, fp32 on GPU)
@@ -222,8 +221,7 @@ def test_tensor_core_path(H, v, N, M, kg, kt):
     out = ph.gpu_draft_numpy(head, hb, kg, kt)
     assert head.status() == 0
     assert head.stats().path == lmhead.CORAL_PATH_TCGEN05
-    rows = np.unique(np.linspace(0, M - 1, 24).astype(int))
-    rep = ph.compare(W, gm, Wg, hb[rows], kg, kt, {k: a[rows] for k, a in out.items()})
+    rep = ph.compare(W, gm, Wg, hb, kg, kt, out)                # every row
     assert rep.ok, rep.errors
     again = ph.gpu_draft_numpy(head, hb, kg, kt)
     for k in out:
@@ -232,22 +230,21 @@ def test_tensor_core_path(H, v, N, M, kg, kt):
 
 
 def test_large_m_routed_grouped_gemm():
-    """16 sequences x 60 tree nodes on the Llama3-8B shape: the tensor-core path, sampled rows against the oracle."""
+    """16 sequences x 60 tree nodes on the Llama3-8B shape: the tensor-core path, every row and every tap (groups,
+    gate, all 960 x 8 x 2004 logits, log-sum-exp, ids, log-probs) against the oracle."""
     cfg, W, gm, Wg, _ = _weights("llama3_8b")
     M = 960
     head = _head(cfg, W, gm, Wg, max_M=M, max_kg=cfg.k_groups, max_kt=cfg.k_tokens)
     hb = synth.make_hidden(cfg, M)
-    ids, lps = head.draft(ph.to_dev_bf16(hb), cfg.k_groups, cfg.k_tokens)
-    torch.cuda.synchronize()
+    out = ph.gpu_draft_numpy(head, hb, cfg.k_groups, cfg.k_tokens)
     assert head.status() == 0
     st = head.stats()
     assert st.path == lmhead.CORAL_PATH_TCGEN05 and st.groups_touched == cfg.N
-    rows = np.unique(np.linspace(0, M - 1, 12).astype(int))
-    rep = ph.compare(W, gm, Wg, hb[rows], cfg.k_groups, cfg.k_tokens,
-                     {"ids": ids.cpu().numpy()[rows], "logprobs": lps.cpu().numpy()[rows]})
+    rep = ph.compare(W, gm, Wg, hb, cfg.k_groups, cfg.k_tokens, out, max_errors=20)
     assert rep.ok, rep.errors
-    first = (ids.cpu().numpy().copy(), lps.cpu().numpy().copy())
-    for _ in range(5):                                   # the same call again: the same bits
+    assert rep.rows == M
+    first = (out["ids"].copy(), out["logprobs"].copy())
+    for _ in range(5):                                   # the same call without taps: the same bits
         ids2, lps2 = head.draft(ph.to_dev_bf16(hb), cfg.k_groups, cfg.k_tokens)
         torch.cuda.synchronize()
         assert np.array_equal(ids2.cpu().numpy(), first[0]) and np.array_equal(lps2.cpu().numpy(), first[1])
@@ -405,10 +402,14 @@ def test_copy_floor_probe_runs_and_checks_arguments():
     packed_bytes, _ = lmhead.coral_lmhead_query_sizes(head.cfg)
     lmhead.coral_lmhead_copy_floor(head.handle, packed_bytes)
     lmhead.coral_lmhead_copy_floor(head.handle, 16384 * 3 + 5)
+    lmhead.coral_lmhead_copy_floor(head.handle, packed_bytes, in_flight=13, repeats=3)
+    lmhead.coral_lmhead_copy_floor(head.handle, packed_bytes, in_flight=1, repeats=2)
     torch.cuda.synchronize()
     assert head.status() == 0
-    assert lib.coral_lmhead_copy_floor(head.handle, 100, None) == lmhead.CORAL_ERR_INVALID
-    assert lib.coral_lmhead_copy_floor(head.handle, packed_bytes + 16384, None) == lmhead.CORAL_ERR_INVALID
+    assert lib.coral_lmhead_copy_floor(head.handle, 100, 0, 1, None) == lmhead.CORAL_ERR_INVALID
+    assert lib.coral_lmhead_copy_floor(head.handle, packed_bytes + 16384, 0, 1, None) == lmhead.CORAL_ERR_INVALID
+    assert lib.coral_lmhead_copy_floor(head.handle, packed_bytes, 14, 1, None) == lmhead.CORAL_ERR_INVALID
+    assert lib.coral_lmhead_copy_floor(head.handle, packed_bytes, 8, 0, None) == lmhead.CORAL_ERR_INVALID
     head.close()
 
 
@@ -488,4 +489,52 @@ def test_other_seeds_on_the_llama2_shape(seed):
         rows = np.unique(np.linspace(0, M - 1, 6).astype(int))
         rep = ph.compare(W, gm, Wg, hb[rows], cfg.k_groups, cfg.k_tokens, {k: v[rows] for k, v in out.items()})
         assert rep.ok, (M, rep.errors)
+    head.close()
+
+
+@pytest.mark.parametrize("H,M", [(256, 4), (256, 40), (256, 200), (328, 13)])
+def test_bad_router_input_is_reported_and_indexes_nothing(H, M):
+    """A NaN hidden row (so NaN router scores) and a forced group named twice, on every router variant (one-launch
+    router, band router, band router + bucketing launch, plain kernels for H not a multiple of 32): the status word
+    says what happened, every selected group is a valid, distinct index, the kernels after the router stage do
+    nothing (the outputs keep what they held), and the handle works again once the status has been read."""
+    cfg = synth.HeadConfig("badin", H=H, V=1536, N=6, k_groups=3, k_tokens=10, M=M, seed=11, w_std=0.05)
+    W, gm, Wg, hb = synth.make_all(cfg)
+    head = _head(cfg, W, gm, Wg, max_M=M, max_kg=cfg.N, max_kt=10)
+    good = ph.gpu_draft_numpy(head, hb, 3, 10)
+    assert head.status() == 0
+
+    def run(hidden_bits, forced=None):
+        dev = "cuda"
+        ids = torch.full((M, 10), -7, dtype=torch.int32, device=dev)
+        lps = torch.full((M, 10), 123.0, dtype=torch.float32, device=dev)
+        groups = torch.full((M, 3), -1, dtype=torch.int32, device=dev)
+        fg = None if forced is None else torch.from_numpy(forced).to(dev)
+        lmhead.coral_lmhead_draft_ex(head.handle, ph.to_dev_bf16(hidden_bits), 3, 10, ids, lps, forced_groups=fg,
+                                     out_groups=groups)
+        torch.cuda.synchronize()
+        return ids.cpu().numpy(), lps.cpu().numpy(), groups.cpu().numpy()
+
+    nan_row = hb.copy()
+    nan_row[M // 2, 5] = 0x7FC0                                   # a bf16 NaN
+    ids, lps, groups = run(nan_row)
+    assert head.status() == lmhead.CORAL_ERR_NONFINITE
+    assert groups.min() >= 0 and groups.max() < cfg.N
+    assert all(len(set(r.tolist())) == 3 for r in groups)
+    assert groups[M // 2].tolist() == [0, 1, 2]                   # all scores of that row rank last: lowest indices
+    assert np.all(ids == -7) and np.all(lps == 123.0)             # nothing after the router stage ran
+
+    forced = np.tile(np.array([4, 1, 4], np.int32), (M, 1))       # group 4 twice
+    ids, lps, groups = run(hb, forced)
+    assert head.status() == lmhead.CORAL_ERR_BOUNDS
+    assert np.all(ids == -7) and np.all(lps == 123.0)
+    forced = np.tile(np.array([4, 99, 0], np.int32), (M, 1))      # a group outside [0, N)
+    ids, lps, groups = run(hb, forced)
+    assert head.status() == lmhead.CORAL_ERR_BOUNDS
+    assert np.all(ids == -7)
+
+    again = ph.gpu_draft_numpy(head, hb, 3, 10)                   # status read: the handle is usable again
+    assert head.status() == 0
+    for k in good:
+        assert np.array_equal(good[k], again[k]), k
     head.close()

@@ -37,7 +37,7 @@ def test_library_exports_every_declared_symbol(lib):
 
 def test_error_strings_and_host_only_argument_checks(lib):
     assert lmhead.coral_lmhead_error_string(0) == "ok"
-    for code in range(-7, 0):
+    for code in range(-8, 0):
         assert lmhead.coral_lmhead_error_string(code) not in ("ok", "unknown status")
     ok = lmhead.make_config(4096, 128256, 64, 960, 8, 10)
     pb, wb = lmhead.coral_lmhead_query_sizes(ok)
@@ -107,3 +107,44 @@ def test_reference_arm_prints_contract_line():
     line = json.loads(p.stdout.strip().splitlines()[-1])
     assert line["impl"] == "reference" and line["cpu_baseline"]["kind"] == "oracle" and line["value"] > 0
     assert line["e2e"]["h2d_bytes_per_step"] == 0
+
+
+def test_parity_harness_accepts_the_oracle_and_rejects_planted_mistakes():
+    """The comparison the GPU tests rely on, exercised on the CPU: the oracle's own result passes; a swapped id,
+    an id outside the row's groups, a shifted log-prob and an unsorted row are each reported."""
+    from oracle import lmhead_oracle as orc
+    from tests import parity_harness as ph
+    cfg = synth.CONFIGS["tiny"]
+    W, gm, Wg, hb = synth.make_all(cfg)
+    ref = orc.draft(W, gm, Wg, hb, cfg.k_groups, cfg.k_tokens)
+    good = {"groups": ref.groups.copy(), "gate": ref.gate.astype(np.float32), "logits": ref.logits.astype(np.float32),
+            "lse": ref.lse.astype(np.float32), "ids": ref.ids.copy(), "logprobs": ref.logprobs.astype(np.float32)}
+    rep = ph.compare(W, gm, Wg, hb, cfg.k_groups, cfg.k_tokens, good)
+    assert rep.ok and rep.tie_resolved_ids == 0 and rep.max_logprob_err < 1e-5
+
+    def broken(**kw):
+        bad = {k: v.copy() for k, v in good.items()}
+        for k, fn in kw.items():
+            fn(bad[k])
+        return ph.compare(W, gm, Wg, hb, cfg.k_groups, cfg.k_tokens, bad)
+
+    def swap_ids(a):
+        a[1, [0, 5]] = a[1, [5, 0]]
+    assert any("row 1 pos 0" in e for e in broken(ids=swap_ids).errors)
+    inactive = int(np.setdiff1d(np.arange(cfg.V), ref.logit_tokens[2].ravel())[0])
+
+    def foreign_id(a):
+        a[2, 3] = inactive
+    assert any("not in an active group" in e for e in broken(ids=foreign_id).errors)
+
+    def shift_lp(a):
+        a[3, 9] -= 0.01
+    assert any("row 3 pos 9: logprob" in e for e in broken(logprobs=shift_lp).errors)
+
+    def unsort(a):
+        a[0, [2, 3]] = a[0, [3, 2]]
+    assert broken(ids=unsort, logprobs=unsort).errors          # same pairs, wrong order
+
+    def dup(a):
+        a[0, 1] = a[0, 0]
+    assert any("duplicate" in e for e in broken(ids=dup).errors)

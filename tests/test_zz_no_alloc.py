@@ -12,6 +12,8 @@ ordinary entry point (coral_lmhead_draft_ex with the groups/gate taps) within
 the tolerance the parity tests use, on two calls in a row with different rows
 (the array keeps the first call's contents, so the second call shows that stale
 data is harmless), and oversized requests must be refused with a clear code.
+The same outputs are also held against the CPU oracle directly (scores within
+the tolerance, groups equal except where the oracle's own scores tie).
 This file sorts last on purpose: a run that stops at the first failure has
 already run every other test.
 """
@@ -21,6 +23,7 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import lmhead_oracle as orc
 from paper_2502_16880_b200 import lmhead, synth
 from tests import parity_harness as ph
 
@@ -49,7 +52,17 @@ def test_route_static_matches_existing_entry_point_twice():
         torch.cuda.synchronize()
         got_gate = gate.cpu().numpy()
         assert np.all(ph.close(got_gate, want_gate)), np.abs(got_gate - want_gate).max()
-        assert np.array_equal(groups.cpu().numpy(), want_groups)
+        got_groups = groups.cpu().numpy()
+        assert np.array_equal(got_groups, want_groups)
+        # and against the oracle itself (router part of the step: Eq. 7's scores, top-n of Section 3.3)
+        hb = synth.make_hidden(cfg, M, batch=batch)
+        ref = orc.draft(W, gm, Wg, hb, k_groups, 1, want_logits=False)
+        assert np.all(ph.close(got_gate, ref.gate)), np.abs(got_gate - ref.gate).max()
+        for m in range(M):
+            for s in range(k_groups):
+                a, b = int(got_groups[m, s]), int(ref.groups[m, s])
+                assert a == b or ph.close(ref.gate[m, a], ref.gate[m, b]), (m, s, a, b)
+            assert len(set(got_groups[m].tolist())) == k_groups
     head.close()
 
 
