@@ -35,7 +35,8 @@ struct Layout {
     size_t route_bands;
     int packed_groups;           // groups stored in the packed copy (all, or this rank's)
     int tc_tiles, tc_vcap;       // tensor-core path: sub-tiles per group, capacity in (group, pass) entries
-    size_t tc_rows;              // rows of the gathered hidden matrix (0: path not provisioned)
+    size_t tc_rows;              // (row, slot) pairs the path is provisioned for (0: not provisioned)
+    int tc_hg_rows;              // rows of one column block of the gathered hidden matrix
 };
 
 bool config_ok(const coral_lmhead_config* c) {
@@ -132,7 +133,8 @@ Layout make_layout(const coral_lmhead_config& c) {
     L.tc_rows = M > (size_t)kTcProvisionRows ? M * kg : 0;
     L.tc_vcap = L.tc_rows ? (int)(N + (M * kg + kTcPassRows - 1) / kTcPassRows) : 0;
     const size_t tcp = (size_t)L.tc_vcap * L.tc_tiles * kTcPassRows;
-    L.tc_hg = take((size_t)L.tc_vcap * L.KB * kTcPassRows * kTcK * 2);   // blocked: [entry][column block][128][64]
+    L.tc_hg_rows = L.tc_rows ? (int)((L.tc_rows + 15) / 16 * 16 + 16 * (size_t)L.tc_vcap) : 0;   // see tc_entry_row
+    L.tc_hg = take((size_t)L.KB * L.tc_hg_rows * kTcK * 2);              // [column block][row][64]
     L.tc_max = take(tcp * 4);
     L.tc_sum = take(tcp * 4);
     L.tc_val = take(tcp * kt * 4);
@@ -179,7 +181,8 @@ struct coral_lmhead_s {
     size_t l2_limit_before;        // ... from this value (restored when the hot groups are released)
     uint16_t* w1;        // [H][H] bf16 first router layer (Eq. 7), library-owned, or null
     float* router_u;     // [max_M][H] fp32 act(W1 h) + h, library-owned
-    CUtensorMap map_w, map_h, map_h64, map_h32;   // hidden-row blocks read whole (128 rows) or only their first 64 / 32 rows
+    CUtensorMap map_w;   // the packed weights as a 5-d tensor, read in 128-row x 64-column boxes
+    int tc_pairs;        // CTA pairs the tensor-core kernel is launched with
     int sms;
     cudaEvent_t ev_head0, ev_head1;   // around the weight-streaming kernel when kernel timing is on
     cudaEvent_t ev_begin, ev_end;     // before the router stage / after the merge
@@ -242,6 +245,44 @@ cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t s
     return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
 }
 
+// The same for a kernel that runs as clusters of two CTAs.
+template <typename... KArgs, typename... Args>
+cudaError_t launch_pdl_pairs(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args) {
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[1].id = cudaLaunchAttributeClusterDimension;
+    attr[1].val.clusterDim.x = 2;
+    attr[1].val.clusterDim.y = 1;
+    attr[1].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 2;
+    return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
+// Clusters of two CTAs of the tensor-core kernel that the device can hold at once (0 on failure).
+int tc_max_pairs(int sms) {
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(sms / 2 * 2);
+    cfg.blockDim = dim3(kTcThreads);
+    cfg.dynamicSmemBytes = kTcSmemBytes;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, head_tc_kernel, &cfg) != cudaSuccess) { cudaGetLastError(); return 0; }
+    return n < sms / 2 ? n : sms / 2;
+}
+
 // cuTensorMapEncodeTiled, looked up through the runtime so that the library does not link against libcuda.
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -256,10 +297,9 @@ EncodeTiledFn encode_tiled_fn() {
     return reinterpret_cast<EncodeTiledFn>(fn);
 }
 
-// Tensor maps of the tensor-core path: the packed weights as a 5-d tensor (column in block, row in item,
+// Tensor map of the tensor-core path: the packed weights as a 5-d tensor (column in block, row in item,
 // 64-column block, item, group) read in boxes of 64 columns x 128 rows (8 items = eight contiguous 2 KiB
-// pieces), and the gathered hidden rows, stored as blocks of 128 rows x 64 columns, as a 64-column matrix
-// read one block (a contiguous 16 KiB) at a time; both land in shared memory with the 128-byte swizzle.
+// pieces) that land in shared memory with the 128-byte swizzle.
 bool make_tc_maps(coral_lmhead_s* h) {
     EncodeTiledFn enc = encode_tiled_fn();
     if (!enc) return false;
@@ -268,27 +308,13 @@ bool make_tc_maps(coral_lmhead_s* h) {
     const cuuint64_t wstr[4] = {128, 2048, (cuuint64_t)L.KB * 2048, (cuuint64_t)L.T16 * L.KB * 2048};
     const cuuint32_t wbox[5] = {(cuuint32_t)kTcK, 16, 1, 8, 1};
     const cuuint32_t ones[5] = {1, 1, 1, 1, 1};
-    if (enc(&h->map_w, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, h->packed, wdim, wstr, wbox, ones,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-        return false;
-    const cuuint64_t hdim[2] = {(cuuint64_t)kTcK, (cuuint64_t)L.tc_vcap * L.KB * kTcPassRows};
-    const cuuint64_t hstr[1] = {(cuuint64_t)kTcK * 2};
-    CUtensorMap* hmaps[3] = {&h->map_h, &h->map_h64, &h->map_h32};
-    for (int i = 0; i < 3; ++i) {
-        const cuuint32_t hbox[2] = {(cuuint32_t)kTcK, (cuuint32_t)(kTcBlockRows >> i)};
-        if (enc(hmaps[i], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, h->ws + L.tc_hg, hdim, hstr, hbox, ones,
-                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-            return false;
-    }
-    return true;
+    return enc(&h->map_w, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, h->packed, wdim, wstr, wbox, ones,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 // Dynamic shared memory of merge_stream_kernel for p_cap pieces and c_cap in-smem candidates.
 inline size_t merge_smem_bytes(int p_cap, int c_cap) { return (size_t)c_cap * 8 + (size_t)p_cap * 25 + 16; }
-
-constexpr size_t kTcSmemBytes = 1024 + (size_t)kTcStages * kTcStageBytes + 32 * kTcEpilogueThreads * 4 + 256;
 
 bool stream_ok(const coral_lmhead_s* h, int M) { return h->stream_smem > 0 && M <= kStreamMaxM; }
 
@@ -403,8 +429,10 @@ int coral_lmhead_create(coral_lmhead_handle* out, const coral_lmhead_config* cfg
         h->sms = sms;
         h->tc_ok = false;
         if (h->L.tc_rows > 0 && h->L.tc_vcap <= cfg->n_groups * kStreamMaxPasses && cfg->H >= kTcK && cfg->H % 8 == 0 && (int)kTcSmemBytes <= smem_optin &&
-            cudaFuncSetAttribute(head_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTcSmemBytes) == cudaSuccess)
-            h->tc_ok = make_tc_maps(h);
+            cudaFuncSetAttribute(head_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTcSmemBytes) == cudaSuccess) {
+            h->tc_pairs = tc_max_pairs(sms);
+            h->tc_ok = h->tc_pairs > 0 && make_tc_maps(h);
+        }
         h->sg = make_stream_geom(*cfg, sms, smem_optin);
         h->stream_smem = 0;
         if (cfg->H <= kStreamMaxH && cfg->H % 256 == 0 && sms >= kStreamGridMin && h->sg.n_stages >= 2) {
@@ -553,13 +581,13 @@ static int draft_impl(coral_lmhead_handle h, const void* hidden_dev, int M, int 
         mg.T = L.tc_tiles;
         if (adaptive) {
             // both head kernels are launched; each reads the router's choice first and the one not chosen returns
-            TcGeom tg{h->sms, L.tc_tiles, L.KB};
+            TcGeom tg{h->tc_pairs, L.tc_tiles, (L.tc_tiles + 1) / 2, L.KB, L.tc_hg_rows};
             TcPartials tp{tpp.pmax, tpp.psum, tpp.pval, tpp.pid};
             launch_pdl(tc_gather_kernel, dim3(M * k_groups), dim3(128), (size_t)0, st, c,
-                       reinterpret_cast<uint16_t*>(h->ws + L.tc_hg));
+                       reinterpret_cast<uint16_t*>(h->ws + L.tc_hg), L.tc_hg_rows);
             ++launches;
-            launch_pdl(head_tc_kernel, dim3(tg.grid), dim3(kTcThreads), kTcSmemBytes, st, c, tg, tp, h->map_w, h->map_h,
-                       h->map_h64, h->map_h32, out_logits_dev);
+            launch_pdl_pairs(head_tc_kernel, dim3(2 * tg.pairs), dim3(kTcThreads), kTcSmemBytes, st, c, tg, tp, h->map_w,
+                             reinterpret_cast<const uint16_t*>(h->ws + L.tc_hg), out_logits_dev);
             ++launches;
         }
         launch_pdl(h->sg.kc == 512 ? head_stream_kernel<2> : head_stream_kernel<1>, dim3(h->sg.grid),
@@ -581,14 +609,14 @@ static int draft_impl(coral_lmhead_handle h, const void* hidden_dev, int M, int 
         ++launches;
     } else if (path == CORAL_PATH_TCGEN05) {
         const Layout& L = h->L;
-        TcGeom tg{h->sms, L.tc_tiles, L.KB};
+        TcGeom tg{h->tc_pairs, L.tc_tiles, (L.tc_tiles + 1) / 2, L.KB, L.tc_hg_rows};
         TcPartials tp{reinterpret_cast<float*>(h->ws + L.tc_max), reinterpret_cast<float*>(h->ws + L.tc_sum),
                       reinterpret_cast<float*>(h->ws + L.tc_val), reinterpret_cast<int32_t*>(h->ws + L.tc_id)};
         launch_pdl(tc_gather_kernel, dim3(M * k_groups), dim3(128), (size_t)0, st, c,
-                   reinterpret_cast<uint16_t*>(h->ws + L.tc_hg));
+                   reinterpret_cast<uint16_t*>(h->ws + L.tc_hg), L.tc_hg_rows);
         ++launches;
-        launch_pdl(head_tc_kernel, dim3(tg.grid), dim3(kTcThreads), kTcSmemBytes, st, c, tg, tp, h->map_w, h->map_h,
-                   h->map_h64, h->map_h32, out_logits_dev);
+        launch_pdl_pairs(head_tc_kernel, dim3(2 * tg.pairs), dim3(kTcThreads), kTcSmemBytes, st, c, tg, tp, h->map_w,
+                         reinterpret_cast<const uint16_t*>(h->ws + L.tc_hg), out_logits_dev);
         ++launches;
         if (h->timing) cudaEventRecord(h->ev_head1, st);
         StreamGeom mg = h->sg;
