@@ -267,7 +267,17 @@ def main():
             if i >= args.warmup:
                 ts.append(a.elapsed_time(b))
         st = big.stats()
+        lmhead.coral_lmhead_set_kernel_timing(big.handle, True)      # stage split, from events inside the call
+        stg = []
+        for i in range(10):
+            lmhead.coral_lmhead_draft(big.handle, hb, cfg.k_groups, cfg.k_tokens, ids_b, lps_b)
+            torch.cuda.synchronize()
+            if i >= 3:
+                stg.append(lmhead.coral_lmhead_stage_ms(big.handle))
+        lmhead.coral_lmhead_set_kernel_timing(big.handle, False)
         print(json.dumps({"large_m_only": Mb, "path": int(st.path), "us_per_step": float(np.mean(ts)) * 1e3,
+                          "stage_us": {k: float(np.mean([x[j] for x in stg])) * 1e3
+                                       for j, k in enumerate(("router", "head_kernels", "merge"))},
                           "status": big.status()}))
         big.close()
         return

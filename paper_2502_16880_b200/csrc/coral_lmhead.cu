@@ -269,7 +269,7 @@ cudaError_t launch_pdl_pairs(void (*kernel)(KArgs...), dim3 grid, dim3 block, si
 int tc_max_pairs(int sms) {
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = dim3(sms / 2 * 2);
-    cfg.blockDim = dim3(kTcThreads);
+    cfg.blockDim = dim3(kTcHeadThreads);
     cfg.dynamicSmemBytes = kTcSmemBytes;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -586,7 +586,7 @@ static int draft_impl(coral_lmhead_handle h, const void* hidden_dev, int M, int 
             launch_pdl(tc_gather_kernel, dim3(M * k_groups), dim3(128), (size_t)0, st, c,
                        reinterpret_cast<uint16_t*>(h->ws + L.tc_hg), L.tc_hg_rows);
             ++launches;
-            launch_pdl_pairs(head_tc_kernel, dim3(2 * tg.pairs), dim3(kTcThreads), kTcSmemBytes, st, c, tg, tp, h->map_w,
+            launch_pdl_pairs(head_tc_kernel, dim3(2 * tg.pairs), dim3(kTcHeadThreads), kTcSmemBytes, st, c, tg, tp, h->map_w,
                              reinterpret_cast<const uint16_t*>(h->ws + L.tc_hg), out_logits_dev);
             ++launches;
         }
@@ -615,7 +615,7 @@ static int draft_impl(coral_lmhead_handle h, const void* hidden_dev, int M, int 
         launch_pdl(tc_gather_kernel, dim3(M * k_groups), dim3(128), (size_t)0, st, c,
                    reinterpret_cast<uint16_t*>(h->ws + L.tc_hg), L.tc_hg_rows);
         ++launches;
-        launch_pdl_pairs(head_tc_kernel, dim3(2 * tg.pairs), dim3(kTcThreads), kTcSmemBytes, st, c, tg, tp, h->map_w,
+        launch_pdl_pairs(head_tc_kernel, dim3(2 * tg.pairs), dim3(kTcHeadThreads), kTcSmemBytes, st, c, tg, tp, h->map_w,
                          reinterpret_cast<const uint16_t*>(h->ws + L.tc_hg), out_logits_dev);
         ++launches;
         if (h->timing) cudaEventRecord(h->ev_head1, st);

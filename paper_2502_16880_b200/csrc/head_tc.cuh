@@ -23,19 +23,23 @@
 // the sub-tiles the warp sees of an entry; logits never travel to HBM.  (CORAL Section 3.3: logits only for
 // the activated groups; Appendix B: the union of the rows' groups is what gets read.)
 //
-// Warp roles: warp 0 = producer (TMA tiled loads of the weights, one bulk copy of the hidden rows), warp 1 =
-// MMA issuer in the CTA of rank 0 and, in rank 1, the relay that tells rank 0 when a stage has landed;
-// warps 2..9 = epilogue, four per accumulator (with one wide accumulator: four per half of its columns).
-// Work split: the units of all entries form one list; pair p owns a contiguous run of it.
+// Warp roles: warp 0 = producer (TMA tiled loads of the weights, one bulk copy of the hidden rows); warps 1 and
+// 10 = MMA issuers in the CTA of rank 0, one per accumulator of the batch (issuing an MMA costs its thread
+// some 40 ns, which for eight MMAs per 64 columns would be the pair's critical path); warp 1 of rank 1 is the
+// relay that tells rank 0 when a stage has landed; warps 2..9 = epilogue, four per accumulator (with one wide
+// accumulator: four per half of its columns).
+// Work split: the units of all entries form one list; pair p owns a contiguous run of it, cut so that the
+// runs cost the same (a unit of a wide entry, which is a batch by itself, counts twice).
 #pragma once
 #include "tc_prims.cuh"
 
 namespace coral {
 
+constexpr int kTcHeadThreads = kTcThreads + 32;     // warp 10 issues the MMAs of a batch's second accumulator
 constexpr int kTcPassRows = 256;                    // hidden rows per pass over a group's weights (the MMA's largest N)
-constexpr int kTcStages = 4;
+constexpr int kTcStages = 5;
 constexpr int kTcStageBytes = 40 * 1024;            // two weight tiles + up to 8 KiB of hidden rows, or one + up to 16 KiB
-constexpr int kTcXchgBytes = 2 * 4 * 32 * 32 * 4;   // [accumulator][owner warp][32 vocab rows][32 hidden rows] fp32
+constexpr int kTcXchgBytes = 2 * 4 * 16 * 32 * 4;   // [accumulator][owner warp][16 vocab rows][32 hidden rows] fp32
 constexpr size_t kTcSmemBytes = 1024 + (size_t)kTcStages * kTcStageBytes + kTcXchgBytes + 256;
 
 struct TcGeom {
@@ -85,18 +89,25 @@ __global__ void __launch_bounds__(128) tc_gather_kernel(CallView c, uint16_t* __
             ch < chunks ? __ldg(src + ch) : make_uint4(0, 0, 0, 0);
 }
 
-// Sorted insertion into a thread-private top-KT list (value desc, row index asc).
+// Insertion into a thread-private top-KT list kept sorted (value desc, row index asc).  The new entry's
+// position is the number of entries that stay ahead of it - KT independent comparisons - and every slot then
+// picks its new content by itself, so the instruction stream has no chain as long as the list.
 template <int KT>
 __device__ __forceinline__ void tc_insert(float (&lv)[KT], int (&li)[KT], float v, int idx) {
+    int p0 = 0, p1 = 0;
 #pragma unroll
-    for (int j = 0; j < KT; ++j) {
-        if (better(v, idx, lv[j], li[j])) {
-            const float tv = lv[j];
-            const int ti = li[j];
-            lv[j] = v; li[j] = idx;
-            v = tv; idx = ti;
-        }
+    for (int j = 0; j < KT; j += 2) {
+        p0 += better(lv[j], li[j], v, idx) ? 1 : 0;
+        if (j + 1 < KT) p1 += better(lv[j + 1], li[j + 1], v, idx) ? 1 : 0;
     }
+    const int p = p0 + p1;
+#pragma unroll
+    for (int j = KT - 1; j >= 1; --j) {                       // descending: slot j - 1 is still the old one
+        const bool shift = j > p, here = j == p;
+        lv[j] = shift ? lv[j - 1] : (here ? v : lv[j]);
+        li[j] = shift ? li[j - 1] : (here ? idx : li[j]);
+    }
+    if (p == 0) { lv[0] = v; li[0] = idx; }
 }
 
 // Running statistics of one hidden row over the sub-tiles one epilogue thread sees of an entry.
@@ -113,39 +124,55 @@ struct TcRowState {
     }
 };
 
-// Folds the logits of 32 vocab rows [base, base + 32) of the group (nv of them real) into the running
-// statistics of one hidden row.  The values sit in a shared-memory block, element k at xb[k * 32 + (lane ^ k)].
+__device__ __forceinline__ float tc_ex2(float x) {            // 2^x for x <= 0; tiny results flush to zero
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// Folds the logits of kTcHalf vocab rows [base, base + 16) of the group (nv of them real) into the running
+// statistics of one hidden row.  The values sit in a shared-memory block, element k at xb[k * 32 + (lane ^ (k + kofs))].
+// Four independent chains for the maximum, the sum and the candidate mask keep the one thread busy.
+constexpr int kTcHalf = 16;
 template <int KT>
-__device__ __forceinline__ void tc_fold_block(const CallView& c, TcRowState<KT>& st, const float* xb, int lane, int base,
-                                              int nv, float* __restrict__ tap_row) {
+__device__ __forceinline__ void tc_fold_block(TcRowState<KT>& st, const float* xb, int lane, int kofs, int base, int nv,
+                                              float* __restrict__ tap_row) {
     constexpr float kLog2e = 1.4426950408889634f;
-    float z[32];
+    float z[kTcHalf];
 #pragma unroll
-    for (int k = 0; k < 32; ++k) z[k] = xb[k * 32 + (lane ^ k)];
-    float cm = kNegInf;
+    for (int k = 0; k < kTcHalf; ++k) z[k] = xb[k * 32 + (lane ^ (k + kofs))];
+    if (nv < kTcHalf) {                                       // ragged end of the group: rows past it do not count
 #pragma unroll
-    for (int k = 0; k < 32; ++k) cm = fmaxf(cm, k < nv ? z[k] : kNegInf);
+        for (int k = 0; k < kTcHalf; ++k) z[k] = k < nv ? z[k] : kNegInf;
+    }
+    float m[4] = {z[0], z[1], z[2], z[3]};
+#pragma unroll
+    for (int k = 4; k < kTcHalf; ++k) m[k & 3] = fmaxf(m[k & 3], z[k]);
+    const float cm = fmaxf(fmaxf(m[0], m[1]), fmaxf(m[2], m[3]));
     const float nm = fmaxf(st.mx, cm);
-    float add = 0.f;
+    const float nb = -nm * kLog2e;
+    float a[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-    for (int k = 0; k < 32; ++k) add += k < nv ? exp2f((z[k] - nm) * kLog2e) : 0.f;
-    st.sum = st.sum * exp2f((st.mx - nm) * kLog2e) + add;   // exp2(-inf) = 0 on the first block
+    for (int k = 0; k < kTcHalf; ++k) a[k & 3] += tc_ex2(fmaf(z[k], kLog2e, nb));   // 2^-inf = 0 for the rows past the end
+    st.sum = st.sum * tc_ex2((st.mx - nm) * kLog2e) + ((a[0] + a[1]) + (a[2] + a[3]));   // 2^-inf = 0 on the first block
     st.mx = nm;
     if (tap_row) {
 #pragma unroll
-        for (int k = 0; k < 32; ++k)
+        for (int k = 0; k < kTcHalf; ++k)
             if (k < nv) tap_row[base + k] = z[k];
     }
-    // candidates for the top-k list: a bit per element that reaches the current k-th entry; the few that do are
-    // fetched again by index from the block
-    if (cm >= st.lv[KT - 1]) {
-        unsigned cand = 0;
+    // candidates for the top-k list: a bit per element that reaches the current k-th entry (ties are settled by
+    // the insertion); the few that do are fetched again by index from the block
+    const float thr = st.lv[KT - 1];
+    if (cm >= thr) {
+        unsigned cb[4] = {0u, 0u, 0u, 0u};
 #pragma unroll
-        for (int k = 0; k < 32; ++k) cand |= (k < nv && z[k] >= st.lv[KT - 1]) ? (1u << k) : 0u;   // ties are settled by the insertion
+        for (int k = 0; k < kTcHalf; ++k) cb[k & 3] |= (k < nv && z[k] >= thr) ? (1u << k) : 0u;
+        unsigned cand = (cb[0] | cb[1]) | (cb[2] | cb[3]);
         while (cand) {
             const int k = __ffs(cand) - 1;
             cand &= cand - 1;
-            const float zk = xb[k * 32 + (lane ^ k)];
+            const float zk = xb[k * 32 + (lane ^ (k + kofs))];
             if (zk >= st.lv[KT - 1]) tc_insert<KT>(st.lv, st.li, zk, base + k);
         }
     }
@@ -167,26 +194,81 @@ __device__ __forceinline__ void tc_flush_row(const CallView& c, const TcPartials
     }
 }
 
-// One batch of a pair's run: its entry, first unit, rows, and whether it holds two units.
-struct TcBatch {
-    int j, u, n, R, npad, nunits, hrow, first;
-    bool read_again;
+// Walks a pair's run batch by batch.  The batches of all entries form one list: an entry with at most 128
+// padded rows ("narrow") has ceil(units / 2) batches of two units (the last may hold one), a wide one `units`
+// batches of one; every batch is one pass over the H columns, so batches cost about the same and a run is
+// simply a number of consecutive batches.
+struct TcWalk {
+    int j, b;             // entry (index in the union list) and batch inside it
+    int nb;               // batches of the entry
+    int n, R, npad, first, hrow;
+    bool wide, read_again;
+    __device__ __forceinline__ void load(const CallView& c, const TcGeom& g) {
+        const int entry = c.union_list[j];
+        n = entry & 0xffff;
+        const int pass = entry >> 16;
+        const int left = c.group_count[n] - pass * kTcPassRows;
+        R = max(1, min(left, kTcPassRows));
+        read_again = left > kTcPassRows;                      // a later pass streams the group's weights again
+        npad = (R + 15) & ~15;
+        wide = npad > kTcSub;
+        nb = wide ? g.units : (g.units + 1) >> 1;
+        first = c.group_offset[n] + pass * kTcPassRows;        // first bucket position of the entry
+        hrow = tc_entry_row(first, j);
+    }
+    __device__ __forceinline__ void start(const CallView& c, const TcGeom& g, int j0, int b0) { j = j0; b = b0; load(c, g); }
+    __device__ __forceinline__ void next(const CallView& c, const TcGeom& g, bool more) {
+        if (++b == nb) { ++j; b = 0; if (more) load(c, g); }
+    }
+    __device__ __forceinline__ int unit(const TcGeom&) const { return wide ? b : 2 * b; }                   // first unit
+    __device__ __forceinline__ int nunits(const TcGeom& g) const { return wide ? 1 : min(2, g.units - 2 * b); }
 };
-__device__ __forceinline__ TcBatch tc_batch_at(const CallView& c, const TcGeom& g, int pos, int hi) {
-    TcBatch b;
-    b.j = pos / g.units;
-    b.u = pos - b.j * g.units;
-    const int entry = c.union_list[b.j];
-    b.n = entry & 0xffff;
-    const int pass = entry >> 16;
-    const int left = c.group_count[b.n] - pass * kTcPassRows;
-    b.R = max(1, min(left, kTcPassRows));
-    b.read_again = left > kTcPassRows;                         // a later pass streams the group's weights again
-    b.npad = (b.R + 15) & ~15;
-    b.nunits = (b.npad <= kTcSub && b.u + 1 < g.units && pos + 1 < hi) ? 2 : 1;
-    b.first = c.group_offset[b.n] + pass * kTcPassRows;         // first bucket position of the entry
-    b.hrow = tc_entry_row(b.first, b.j);
-    return b;
+
+// Cuts the batch list into g.pairs runs of (almost) equal length (one warp).  out[0], out[1]: entry and batch
+// where the pair's run starts; out[2]: its number of batches.
+__device__ __forceinline__ void tc_split_runs(const CallView& c, const TcGeom& g, int n_entries, int pair, int* out) {
+    const int lane = threadIdx.x & 31;
+    int total = 0;
+    for (int j0 = 0; j0 < n_entries; j0 += 32) {
+        const int j = j0 + lane;
+        if (j < n_entries) {
+            const int entry = c.union_list[j];
+            const int left = c.group_count[entry & 0xffff] - (entry >> 16) * kTcPassRows;
+            total += min(left, kTcPassRows) > kTcSub ? g.units : (g.units + 1) >> 1;
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) total += __shfl_xor_sync(0xffffffffu, total, o);
+    const int t_lo = (int)((long long)pair * total / g.pairs), t_hi = (int)((long long)(pair + 1) * total / g.pairs);
+    int j_at = 0x7fffffff, b_at = 0, before = 0;
+    for (int j0 = 0; j0 < n_entries; j0 += 32) {
+        const int j = j0 + lane;
+        int nb = 0;
+        if (j < n_entries) {
+            const int entry = c.union_list[j];
+            const int left = c.group_count[entry & 0xffff] - (entry >> 16) * kTcPassRows;
+            nb = min(left, kTcPassRows) > kTcSub ? g.units : (g.units + 1) >> 1;
+        }
+        int incl = nb;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int v = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += v;
+        }
+        const int start = before + incl - nb;                   // list position of the entry's first batch
+        if (nb > 0 && t_lo >= start && t_lo < start + nb) { j_at = j; b_at = t_lo - start; }
+        before += __shfl_sync(0xffffffffu, incl, 31);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const int oj = __shfl_xor_sync(0xffffffffu, j_at, o), ob = __shfl_xor_sync(0xffffffffu, b_at, o);
+        if (oj < j_at) { j_at = oj; b_at = ob; }
+    }
+    if (lane == 0) {
+        out[0] = j_at == 0x7fffffff ? 0 : j_at;
+        out[1] = b_at;
+        out[2] = j_at == 0x7fffffff ? 0 : t_hi - t_lo;
+    }
 }
 
 // The four warps of accumulator `quad` meet (hardware barriers 1 and 2; barrier 0 is the block's own).
@@ -196,73 +278,79 @@ __device__ __forceinline__ void quad_sync(int quad) {
     else asm volatile("bar.sync 2, 128;" ::: "memory");
 }
 
-// Epilogue warps' loop over the pair's run [lo, hi).  `tmem_empty_at` is the (cluster) address of rank 0's
+// Epilogue warps' loop over the pair's run.  `tmem_empty_at` is the (cluster) address of rank 0's
 // "accumulators drained" barriers.
 template <int KT>
 __device__ __forceinline__ void tc_epilogue(const CallView& c, const TcGeom& g, const TcPartials& pp,
                                             float* __restrict__ logits_tap, uint32_t tmem_base, uint64_t* tmem_full,
                                             uint32_t tmem_empty_at, bool leader, volatile int* abort_flag, float* xchg,
-                                            int lo, int hi, int rank) {
+                                            const int* run, int rank) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int q = warp & 3;                                // lane quarter this warp may read = block it owns
     const int quad = (warp - 2) >> 2;                      // accumulator 0 or 1 of the batch
-    float* xq = xchg + quad * (4 * 1024);
+    float* xq = xchg + quad * (4 * kTcHalf * 32);
     TcRowState<KT> st;
     st.reset();
     long long pending = -1;                                // piece of the last sub-tile folded into `st`
     int pending_j = -1, pending_n = 0;
     bool pending_valid = false;
-    int batch = 0;
-    for (int pos = lo; pos < hi; ++batch) {
-        const TcBatch b = tc_batch_at(c, g, pos, hi);
+    const int n_batches = run[2];
+    TcWalk w;
+    if (n_batches > 0) w.start(c, g, run[0], run[1]);
+    for (int batch = 0; batch < n_batches; ++batch) {
         const int buf = batch & 1;
         tc_wait(smem_u32(&tmem_full[buf]), ((uint32_t)batch >> 1) & 1u, abort_flag, c.state);
         tc_fence_after();
-        if (pending >= 0 && pending_j != b.j) {            // the entry is behind us: its running partial goes out
+        if (pending >= 0 && pending_j != w.j) {            // the entry is behind us: its running partial goes out
             if (pending_valid) tc_flush_row<KT>(c, pp, st, pending_n, (size_t)pending);
             st.reset();
             pending = -1;
         }
-        const bool wide = b.npad > kTcSub;
-        const int t = 2 * (b.u + (wide ? 0 : quad)) + rank;                   // this quad's sub-tile
-        const bool tile_ok = (wide || quad < b.nunits) && t < g.tiles;
-        const int hbase = wide ? quad * kTcSub : 0;                            // hidden row of the quad's first column
-        const int ncols = tile_ok ? min(kTcSub, b.npad - hbase) : 0;           // columns this quad handles
+        const int t = 2 * (w.unit(g) + (w.wide ? 0 : quad)) + rank;            // this quad's sub-tile
+        const bool tile_ok = (w.wide || quad < w.nunits(g)) && t < g.tiles;
+        const int hbase = w.wide ? quad * kTcSub : 0;                          // hidden row of the quad's first column
+        const int ncols = tile_ok ? min(kTcSub, w.npad - hbase) : 0;           // columns this quad handles
         if (ncols > 0) {
             const int hrow = hbase + q * 32 + lane;                            // the hidden row this thread owns
-            const bool row_valid = hrow < b.R;
-            const size_t pidx = ((size_t)b.j * g.tiles + t) * kTcPassRows + hrow;
+            const bool row_valid = hrow < w.R;
+            const size_t pidx = ((size_t)w.j * g.tiles + t) * kTcPassRows + hrow;
             if (pending >= 0 && pending_valid) {                               // not the entry's last piece after all
                 pp.pmax[pending] = kNegInf;
                 pp.psum[pending] = 0.f;
             }
             float* tap_row = nullptr;
             if (logits_tap && row_valid)
-                tap_row = logits_tap + ((size_t)c.bucket_row[b.first + hrow] * c.k_groups + c.bucket_slot[b.first + hrow]) * c.v;
+                tap_row = logits_tap + ((size_t)c.bucket_row[w.first + hrow] * c.k_groups + c.bucket_slot[w.first + hrow]) * c.v;
             const uint32_t acc = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * 2 * kTcSub + quad * kTcSub);
             const bool own = q * 32 < ncols;
+            const int half = lane >> 4;
 #pragma unroll 1
             for (int s = 0; s < 4; ++s) {
                 const int cch = (q + s) & 3;
-                if (cch * 32 < ncols) {
-                    float z[32];
-                    tc_ld32(acc + (uint32_t)(cch * 32), z);
-                    float* xw = xq + cch * 1024 + lane * 32;
+                const bool give = cch * 32 < ncols;
+                float z[32];
+                if (give) tc_ld32(acc + (uint32_t)(cch * 32), z);
+                const int wsrc = (q - s) & 3;                                  // the warp that writes this warp's block
+#pragma unroll 1
+                for (int hf = 0; hf < 2; ++hf) {
+                    // lanes of vocab rows 16 hf .. 16 hf + 15 of the quarter hand their 32 columns over
+                    if (give && half == hf) {
+                        float* xw = xq + cch * (kTcHalf * 32) + (lane & 15) * 32;
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) xw[i ^ lane] = z[i];
+                        for (int i = 0; i < 32; ++i) xw[i ^ lane] = z[i];
+                    }
+                    quad_sync(quad);
+                    if (own && row_valid) {
+                        const int base = t * kTcSub + wsrc * 32 + hf * kTcHalf;
+                        const int nv = min(kTcHalf, c.v - base);
+                        if (nv > 0) tc_fold_block<KT>(st, xq + q * (kTcHalf * 32), lane, hf * kTcHalf, base, nv, tap_row);
+                    }
+                    quad_sync(quad);
                 }
-                quad_sync(quad);
-                if (own && row_valid) {
-                    const int w = (q - s) & 3;                                 // the warp that wrote the block
-                    const int base = t * kTcSub + w * 32;
-                    const int nv = min(32, c.v - base);
-                    if (nv > 0) tc_fold_block<KT>(c, st, xq + q * 1024, lane, base, nv, tap_row);
-                }
-                quad_sync(quad);
             }
             pending = (long long)pidx;
-            pending_j = b.j;
-            pending_n = b.n;
+            pending_j = w.j;
+            pending_n = w.n;
             pending_valid = row_valid;
         }
         tc_fence_before();
@@ -271,14 +359,14 @@ __device__ __forceinline__ void tc_epilogue(const CallView& c, const TcGeom& g, 
             if (leader) mbar_arrive(tmem_empty_at + (uint32_t)buf * 8u);
             else mbar_arrive_cluster(tmem_empty_at + (uint32_t)buf * 8u);
         }
-        pos += b.nunits;
+        w.next(c, g, batch + 1 < n_batches);
     }
     if (pending >= 0 && pending_valid) tc_flush_row<KT>(c, pp, st, pending_n, (size_t)pending);
 }
 
-// grid = 2 * g.pairs CTAs of kTcThreads threads in clusters of two; dynamic shared memory: 1 KiB alignment
+// grid = 2 * g.pairs CTAs of kTcHeadThreads threads in clusters of two; dynamic shared memory: 1 KiB alignment
 // slack + kTcStages stages + the epilogue's exchange blocks + barriers.
-__global__ void __launch_bounds__(kTcThreads, 1)
+__global__ void __launch_bounds__(kTcHeadThreads, 1)
     head_tc_kernel(CallView c, TcGeom g, TcPartials pp, const __grid_constant__ CUtensorMap map_w,
                    const uint16_t* __restrict__ hg, float* __restrict__ logits_tap) {
     extern __shared__ unsigned char tc_smem_raw[];
@@ -286,11 +374,11 @@ __global__ void __launch_bounds__(kTcThreads, 1)
     float* xchg = reinterpret_cast<float*>(smem + kTcStages * kTcStageBytes);
     uint64_t* full = reinterpret_cast<uint64_t*>(smem + kTcStages * kTcStageBytes + kTcXchgBytes);
     uint64_t* empty = full + kTcStages;
-    uint64_t* peer_full = empty + kTcStages;      // rank 0: the other CTA's copy of the stage has landed
-    uint64_t* tmem_full = peer_full + kTcStages;  // [2]
+    uint64_t* tmem_full = empty + kTcStages;      // [2]
     uint64_t* tmem_empty = tmem_full + 2;         // [2] rank 0: both CTAs' epilogue warps have drained the buffer
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tmem_empty + 2);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+    int* run = const_cast<int*>(abort_flag) + 1;  // [3] entry and batch where the pair's run starts, number of batches
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int rank = (int)cluster_ctarank();
     const bool leader = rank == 0;
@@ -299,12 +387,12 @@ __global__ void __launch_bounds__(kTcThreads, 1)
     // dependency wait touches only the pair's shared and tensor memory.
     if (threadIdx.x == 0) {
         for (int s = 0; s < kTcStages; ++s) {
-            mbar_init(smem_u32(&full[s]), 1);
-            mbar_init(smem_u32(&empty[s]), 1);
-            mbar_init(smem_u32(&peer_full[s]), 1);
+            // rank 0's "stage has landed" also counts an arrival from rank 1, sent once its own copies are in
+            mbar_init(smem_u32(&full[s]), leader ? 2 : 1);
+            mbar_init(smem_u32(&empty[s]), 2);                  // both issuers' MMAs on the stage have completed
         }
         for (int s = 0; s < 2; ++s) {
-            mbar_init(smem_u32(&tmem_full[s]), 1);
+            mbar_init(smem_u32(&tmem_full[s]), 2);
             mbar_init(smem_u32(&tmem_empty[s]), 2 * kTcEpilogueWarps);
         }
         *abort_flag = 0;
@@ -326,11 +414,10 @@ __global__ void __launch_bounds__(kTcThreads, 1)
     // nothing to do: the router chose the streaming kernel for this call, or the router stage reported a problem
     const bool skip = (c.adaptive && c.state->path_choice != 2) || call_is_poisoned(c.state);
 
-    // this pair's run of units
-    const int n_units = skip ? 0 : c.state->n_virtual * g.units;
-    const int per = (n_units + g.pairs - 1) / g.pairs;
-    const int lo = min(n_units, (int)(blockIdx.x >> 1) * per);
-    const int hi = min(n_units, lo + per);
+    // this pair's run of batches
+    if (warp == 0) tc_split_runs(c, g, skip ? 0 : c.state->n_virtual, (int)(blockIdx.x >> 1), run);
+    __syncthreads();
+    const int n_batches = run[2];
 
     if (warp == 0) {
         if (lane == 0) {
@@ -338,83 +425,85 @@ __global__ void __launch_bounds__(kTcThreads, 1)
             uint32_t phase = 0;
             const uint64_t pol_first = l2_policy_evict_first(), pol_normal = l2_policy_evict_normal(),
                            pol_last = l2_policy_evict_last();
-            for (int pos = lo; pos < hi;) {
-                const TcBatch b = tc_batch_at(c, g, pos, hi);
-                const bool wide = b.npad > kTcSub;
-                const int t0 = 2 * b.u + rank, t1 = 2 * (b.u + 1) + rank;       // this CTA's sub-tiles
-                const bool w0 = t0 < g.tiles, w1 = b.nunits == 2 && t1 < g.tiles;
-                const uint32_t hbytes = (uint32_t)(b.npad >> 1) * 128u;         // this CTA's half of the hidden rows
-                const uint32_t hoff = wide ? kTcTileBytes : 2 * kTcTileBytes;
+            TcWalk w;
+            if (n_batches > 0) w.start(c, g, run[0], run[1]);
+            for (int batch = 0; batch < n_batches; ++batch) {
+                const int u = w.unit(g), nu = w.nunits(g);
+                const int t0 = 2 * u + rank, t1 = 2 * (u + 1) + rank;           // this CTA's sub-tiles
+                const bool w0 = t0 < g.tiles, w1 = nu == 2 && t1 < g.tiles;
+                const uint32_t hbytes = (uint32_t)(w.npad >> 1) * 128u;         // this CTA's half of the hidden rows
+                const uint32_t hoff = w.wide ? kTcTileBytes : 2 * kTcTileBytes;
                 const uint32_t bytes = hbytes + (w0 ? kTcTileBytes : 0) + (w1 ? kTcTileBytes : 0);
-                const uint64_t pol_w = b.read_again ? pol_normal : pol_first;
-                const uint16_t* hsrc = hg + ((size_t)b.hrow + (size_t)rank * (b.npad >> 1)) * kTcK;
+                const uint64_t pol_w = w.read_again ? pol_normal : pol_first;
+                const uint16_t* hsrc = hg + ((size_t)w.hrow + (size_t)rank * (w.npad >> 1)) * kTcK;
+                const int gidx = w.n / c.pack_div;
                 for (int ks = 0; ks < g.ksteps; ++ks) {
                     tc_wait(smem_u32(&empty[stage]), phase ^ 1u, abort_flag, c.state);
                     const uint32_t bar = smem_u32(&full[stage]);
                     const uint32_t sb = smem_u32(smem + (size_t)stage * kTcStageBytes);
                     mbar_expect_tx(bar, bytes);
-                    if (w0) tma_load_5d(sb, &map_w, 0, 0, ks, t0 * 8, b.n / c.pack_div, bar, pol_w);
-                    if (w1) tma_load_5d(sb + kTcTileBytes, &map_w, 0, 0, ks, t1 * 8, b.n / c.pack_div, bar, pol_w);
+                    if (w0) tma_load_5d(sb, &map_w, 0, 0, ks, t0 * 8, gidx, bar, pol_w);
+                    if (w1) tma_load_5d(sb + kTcTileBytes, &map_w, 0, 0, ks, t1 * 8, gidx, bar, pol_w);
                     bulk_g2s_hint(sb + hoff, hsrc + (size_t)ks * g.hg_rows * kTcK, hbytes, bar, pol_last);
                     if (++stage == kTcStages) { stage = 0; phase ^= 1u; }
                 }
-                pos += b.nunits;
+                w.next(c, g, batch + 1 < n_batches);
             }
         }
-    } else if (warp == 1) {
+    } else if (warp == 1 || warp == 10) {
         if (lane == 0 && leader) {
-            int stage = 0, batch = 0;
+            // issuer `a` owns accumulator a of every batch; both issuers commit on every stage and every batch
+            // (a commit with nothing pending arrives at once), so the barriers always count two arrivals
+            const int a = warp == 1 ? 0 : 1;
+            int stage = 0;
             uint32_t phase = 0;
-            for (int pos = lo; pos < hi; ++batch) {
-                const TcBatch b = tc_batch_at(c, g, pos, hi);
+            const uint32_t ring_lo = tc_smem_desc_lo(smem_u32(smem)) + (uint32_t)a * (kTcTileBytes >> 4);
+            TcWalk w;
+            if (n_batches > 0) w.start(c, g, run[0], run[1]);
+            for (int batch = 0; batch < n_batches; ++batch) {
                 const int buf = batch & 1;
-                const bool wide = b.npad > kTcSub;
-                const uint32_t hoff = wide ? kTcTileBytes : 2 * kTcTileBytes;
-                const uint32_t idesc = tc_idesc(256, b.npad);
-                tc_wait_cluster(smem_u32(&tmem_empty[buf]), (((uint32_t)batch >> 1) & 1u) ^ 1u, abort_flag, c.state);   // drained
+                const uint32_t hoff_lo = ((w.wide ? kTcTileBytes : 2 * kTcTileBytes) - a * kTcTileBytes) >> 4;
+                const uint32_t idesc = tc_idesc(256, w.npad);
+                const bool mine = a < w.nunits(g);
+                tc_wait(smem_u32(&tmem_empty[buf]), (((uint32_t)batch >> 1) & 1u) ^ 1u, abort_flag, c.state);   // drained
                 tc_fence_after();
-                const uint32_t acc = tmem_base + (uint32_t)(buf * 2 * kTcSub);
+                const uint32_t acc = tmem_base + (uint32_t)(buf * 2 * kTcSub + a * kTcSub);
                 for (int ks = 0; ks < g.ksteps; ++ks) {
-                    tc_wait(smem_u32(&full[stage]), phase, abort_flag, c.state);
-                    tc_wait_cluster(smem_u32(&peer_full[stage]), phase, abort_flag, c.state);
-                    tc_fence_after();
-                    const uint32_t sb = smem_u32(smem + (size_t)stage * kTcStageBytes);
+                    // (an issuer with nothing to do in this batch waits all the same: its commits must not get
+                    // ahead of the stage they speak for)
+                    tc_wait(smem_u32(&full[stage]), phase, abort_flag, c.state);        // this CTA's copies and the other's
+                    if (mine) {
+                        tc_fence_after();
+                        const uint32_t a_lo = ring_lo + (uint32_t)stage * (kTcStageBytes >> 4);
+                        const uint32_t b_lo = a_lo + hoff_lo;
 #pragma unroll
-                    for (int kk = 0; kk < kTcK / 16; ++kk) {
-                        const uint64_t bdesc = tc_smem_desc(sb + hoff + kk * 32);
-                        for (int a = 0; a < b.nunits; ++a) {
-                            const uint64_t adesc = tc_smem_desc(sb + a * kTcTileBytes + kk * 32);
-                            tc_mma_pair(acc + (uint32_t)(a * kTcSub), adesc, bdesc, idesc, (ks | kk) ? 1u : 0u);
-                        }
+                        for (int kk = 0; kk < kTcK / 16; ++kk)               // 32 bytes (two 16-byte units) per 16 columns
+                            tc_mma_pair(acc, a_lo + 2 * kk, b_lo + 2 * kk, idesc, kk ? 1u : (ks ? 1u : 0u));
                     }
-                    tc_commit_pair(smem_u32(&empty[stage]));  // the stage is free in both CTAs once these MMAs have read it
+                    tc_commit_pair(smem_u32(&empty[stage]));  // the stage is free in both CTAs once both issuers' MMAs have read it
                     if (++stage == kTcStages) { stage = 0; phase ^= 1u; }
                 }
                 tc_commit_pair(smem_u32(&tmem_full[buf]));    // accumulators complete, in both CTAs
-                pos += b.nunits;
+                w.next(c, g, batch + 1 < n_batches);
             }
-        } else if (lane == 0) {
+        } else if (lane == 0 && warp == 1) {
             // rank 1: pass the news that a stage of this CTA has landed on to the MMA issuer in rank 0
-            const uint32_t peer_at = cluster_map_shared(smem_u32(peer_full), 0);
+            const uint32_t peer_at = cluster_map_shared(smem_u32(full), 0);
             int stage = 0;
             uint32_t phase = 0;
-            for (int pos = lo; pos < hi;) {
-                const TcBatch b = tc_batch_at(c, g, pos, hi);
-                for (int ks = 0; ks < g.ksteps; ++ks) {
-                    tc_wait(smem_u32(&full[stage]), phase, abort_flag, c.state);
-                    mbar_arrive_cluster(peer_at + (uint32_t)stage * 8u);
-                    if (++stage == kTcStages) { stage = 0; phase ^= 1u; }
-                }
-                pos += b.nunits;
+            for (int i = 0; i < n_batches * g.ksteps; ++i) {
+                tc_wait(smem_u32(&full[stage]), phase, abort_flag, c.state);
+                mbar_arrive_cluster(peer_at + (uint32_t)stage * 8u);            // counts on rank 0's barrier of the stage
+                if (++stage == kTcStages) { stage = 0; phase ^= 1u; }
             }
         }
     } else {
         // epilogue: the four warps of an accumulator exchange blocks so that every thread owns one hidden row
         const uint32_t tmem_empty_at = leader ? smem_u32(tmem_empty) : cluster_map_shared(smem_u32(tmem_empty), 0);
         if (c.k_tokens <= 10)
-            tc_epilogue<10>(c, g, pp, logits_tap, tmem_base, tmem_full, tmem_empty_at, leader, abort_flag, xchg, lo, hi, rank);
+            tc_epilogue<10>(c, g, pp, logits_tap, tmem_base, tmem_full, tmem_empty_at, leader, abort_flag, xchg, run, rank);
         else
-            tc_epilogue<32>(c, g, pp, logits_tap, tmem_base, tmem_full, tmem_empty_at, leader, abort_flag, xchg, lo, hi, rank);
+            tc_epilogue<32>(c, g, pp, logits_tap, tmem_base, tmem_full, tmem_empty_at, leader, abort_flag, xchg, run, rank);
     }
     tc_fence_before();
     cluster_sync_all();          // nothing of the other CTA is still on its way to this CTA's barriers or tensor memory

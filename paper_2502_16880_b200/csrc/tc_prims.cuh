@@ -19,6 +19,7 @@ constexpr int kTcTmemCols = 512;
 constexpr int kTcSpin = 1 << 22;     // bound of every wait
 
 __device__ __forceinline__ void tc_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, DeviceState* st) {
+    if (mbar_try_wait(bar, parity)) return;                  // the common case costs one instruction
     const int limit = *abort_flag ? 64 : kTcSpin;
     for (int i = 0; i < limit; ++i)
         if (mbar_try_wait(bar, parity)) return;
@@ -114,36 +115,30 @@ __device__ __forceinline__ uint32_t cluster_map_shared(uint32_t addr, uint32_t r
     asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
     return r;
 }
+// Arrive on a barrier of the other CTA.  What the arrival orders is work of the asynchronous units (a landed bulk
+// copy, finished tensor-memory reads), not data written by this thread, so the barrier's default semantics
+// are enough; cluster-scope release / acquire qualifiers here cost a memory fence per arrival and per wait.
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
-    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    return ok != 0;
-}
-// Bounded wait on a barrier that the other CTA of the pair arrives on.
-__device__ __forceinline__ void tc_wait_cluster(uint32_t bar, uint32_t parity, volatile int* abort_flag, DeviceState* st) {
-    const int limit = *abort_flag ? 64 : kTcSpin;
-    for (int i = 0; i < limit; ++i)
-        if (mbar_try_wait_cluster(bar, parity)) return;
-    *abort_flag = 1;
-    set_status(st, -5);
+    asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
 // All threads of both CTAs.
 __device__ __forceinline__ void cluster_sync_all() {
     asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
-__device__ __forceinline__ void tc_mma_pair(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+// The operands are given by the low words of their shared-memory descriptors (tc_smem_desc_lo); the high word
+// is the same for every tile of this layout.  The single issuing thread is the pair's critical path, so the
+// instruction stream per MMA is kept to the two register pairs and the instruction itself.
+constexpr uint32_t kTcDescHi = 64u | (1u << 14) | (2u << 29);          // bits 32..63 of tc_smem_desc
+__device__ __forceinline__ uint32_t tc_smem_desc_lo(uint32_t saddr) { return ((saddr >> 4) & 0x3FFFu) | (1u << 16); }
+__device__ __forceinline__ void tc_mma_pair(uint32_t d_tmem, uint32_t adesc_lo, uint32_t bdesc_lo, uint32_t idesc,
                                             uint32_t accumulate) {
     asm volatile(
-        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+        "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "mov.b64 da, {%1, %5};\n\t"
+        "mov.b64 db, {%2, %5};\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], da, db, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(adesc_lo), "r"(bdesc_lo), "r"(idesc), "r"(accumulate), "r"(kTcDescHi) : "memory");
 }
 // Arrives, once the pair's MMAs issued so far have completed, on the barrier at this shared-memory offset in
 // both CTAs.
