@@ -37,10 +37,42 @@ namespace coral {
 
 constexpr int kTcHeadThreads = kTcThreads + 32;     // warp 10 issues the MMAs of a batch's second accumulator
 constexpr int kTcPassRows = 256;                    // hidden rows per pass over a group's weights (the MMA's largest N)
-constexpr int kTcStages = 5;
-constexpr int kTcStageBytes = 40 * 1024;            // two weight tiles + up to 8 KiB of hidden rows, or one + up to 16 KiB
+// The operand ring is cut into slots of the size the current batch needs per 64 columns, so that the bytes in
+// flight - what hides the memory latency - stay the same whatever the batch: two weight tiles + up to 8 KiB of
+// hidden rows (40 KiB, five slots), one + up to 8 KiB (24 KiB, eight slots), one + up to 16 KiB (32 KiB, six).
+// When the kind of batch changes the producer lets the ring run empty first.
+constexpr int kTcRingBytes = 200 * 1024;
+constexpr int kTcMaxSlots = 8;
+struct TcRing {
+    int slots;            // slots of the current geometry
+    uint32_t bytes;       // their size
+    uint32_t hoff;        // offset of the hidden rows inside a slot (the weight tiles come first)
+};
+__device__ __forceinline__ TcRing tc_ring_for(bool wide, int nunits) {
+    if (wide) return TcRing{6, 32 * 1024, (uint32_t)kTcTileBytes};
+    if (nunits == 2) return TcRing{5, 40 * 1024, 2u * kTcTileBytes};
+    return TcRing{8, 24 * 1024, (uint32_t)kTcTileBytes};
+}
+// A role's place in the ring: the slot it uses next and, per slot, the parity of the slot's next use (the
+// barriers keep their history across changes of geometry; only the slot counter starts over).
+struct TcRingPos {
+    int slot = 0, kind = -1;
+    uint32_t parity = 0;
+    // true when the geometry changed (the caller then starts at slot 0 of the new one)
+    __device__ __forceinline__ bool enter(const TcRing& r) {
+        if (r.slots == kind) return false;
+        kind = r.slots;       // the three geometries differ in their slot count
+        slot = 0;
+        return true;
+    }
+    __device__ __forceinline__ uint32_t par() const { return (parity >> slot) & 1u; }
+    __device__ __forceinline__ void advance(const TcRing& r) {
+        parity ^= 1u << slot;
+        if (++slot == r.slots) slot = 0;
+    }
+};
 constexpr int kTcXchgBytes = 2 * 4 * 16 * 32 * 4;   // [accumulator][owner warp][16 vocab rows][32 hidden rows] fp32
-constexpr size_t kTcSmemBytes = 1024 + (size_t)kTcStages * kTcStageBytes + kTcXchgBytes + 256;
+constexpr size_t kTcSmemBytes = 1024 + (size_t)kTcRingBytes + kTcXchgBytes + 256;
 
 struct TcGeom {
     int pairs;        // CTA pairs launched
@@ -194,80 +226,102 @@ __device__ __forceinline__ void tc_flush_row(const CallView& c, const TcPartials
     }
 }
 
-// Walks a pair's run batch by batch.  The batches of all entries form one list: an entry with at most 128
-// padded rows ("narrow") has ceil(units / 2) batches of two units (the last may hold one), a wide one `units`
-// batches of one; every batch is one pass over the H columns, so batches cost about the same and a run is
-// simply a number of consecutive batches.
+// Walks a pair's run batch by batch.  A run is a number of consecutive units of the unit list (entry by entry,
+// unit by unit).  A batch is the next two units of the run when they belong to one entry of at most 128
+// padded rows ("narrow"), else one unit.
 struct TcWalk {
-    int j, b;             // entry (index in the union list) and batch inside it
-    int nb;               // batches of the entry
+    int j, u;             // entry (index in the union list) and unit inside it
+    int left;             // units of the run still to do, this batch included
     int n, R, npad, first, hrow;
     bool wide, read_again;
-    __device__ __forceinline__ void load(const CallView& c, const TcGeom& g) {
+    __device__ __forceinline__ void load(const CallView& c) {
         const int entry = c.union_list[j];
         n = entry & 0xffff;
         const int pass = entry >> 16;
-        const int left = c.group_count[n] - pass * kTcPassRows;
-        R = max(1, min(left, kTcPassRows));
-        read_again = left > kTcPassRows;                      // a later pass streams the group's weights again
+        const int rows = c.group_count[n] - pass * kTcPassRows;
+        R = max(1, min(rows, kTcPassRows));
+        read_again = rows > kTcPassRows;                      // a later pass streams the group's weights again
         npad = (R + 15) & ~15;
         wide = npad > kTcSub;
-        nb = wide ? g.units : (g.units + 1) >> 1;
         first = c.group_offset[n] + pass * kTcPassRows;        // first bucket position of the entry
         hrow = tc_entry_row(first, j);
     }
-    __device__ __forceinline__ void start(const CallView& c, const TcGeom& g, int j0, int b0) { j = j0; b = b0; load(c, g); }
-    __device__ __forceinline__ void next(const CallView& c, const TcGeom& g, bool more) {
-        if (++b == nb) { ++j; b = 0; if (more) load(c, g); }
+    __device__ __forceinline__ void start(const CallView& c, const int* run) {
+        j = run[0]; u = run[1]; left = run[2];
+        if (left > 0) load(c);
     }
-    __device__ __forceinline__ int unit(const TcGeom&) const { return wide ? b : 2 * b; }                   // first unit
-    __device__ __forceinline__ int nunits(const TcGeom& g) const { return wide ? 1 : min(2, g.units - 2 * b); }
+    __device__ __forceinline__ int nunits(const TcGeom& g) const { return wide ? 1 : min(2, min(g.units - u, left)); }
+    __device__ __forceinline__ void next(const CallView& c, const TcGeom& g) {
+        const int nu = nunits(g);
+        u += nu;
+        left -= nu;
+        if (u == g.units) { ++j; u = 0; if (left > 0) load(c); }
+    }
 };
 
-// Cuts the batch list into g.pairs runs of (almost) equal length (one warp).  out[0], out[1]: entry and batch
-// where the pair's run starts; out[2]: its number of batches.
+// Bytes a CTA takes in per 64 columns for one unit of an entry with `rows` rows, in 128-byte units: the weight
+// sub-tile plus its share of the hidden rows (a narrow batch's two units share one read of them).
+__device__ __forceinline__ int tc_unit_cost(int rows) {
+    const int npad = (max(1, min(rows, kTcPassRows)) + 15) & ~15;
+    return kTcSub + (npad > kTcSub ? npad >> 1 : npad >> 2);
+}
+
+// Cuts the unit list into g.pairs runs of (almost) equal cost (one warp).  out[0], out[1]: entry and unit where
+// the pair's run starts; out[2]: its number of units.  The kernel is bound by what it reads, so the cost of a
+// unit is its bytes (tc_unit_cost); run p holds the units whose cost prefix, taken at the unit's middle, lies in
+// [p, p + 1) * total / pairs.
 __device__ __forceinline__ void tc_split_runs(const CallView& c, const TcGeom& g, int n_entries, int pair, int* out) {
     const int lane = threadIdx.x & 31;
-    int total = 0;
+    long long total = 0;
     for (int j0 = 0; j0 < n_entries; j0 += 32) {
         const int j = j0 + lane;
         if (j < n_entries) {
             const int entry = c.union_list[j];
-            const int left = c.group_count[entry & 0xffff] - (entry >> 16) * kTcPassRows;
-            total += min(left, kTcPassRows) > kTcSub ? g.units : (g.units + 1) >> 1;
+            total += (long long)g.units * tc_unit_cost(c.group_count[entry & 0xffff] - (entry >> 16) * kTcPassRows);
         }
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) total += __shfl_xor_sync(0xffffffffu, total, o);
-    const int t_lo = (int)((long long)pair * total / g.pairs), t_hi = (int)((long long)(pair + 1) * total / g.pairs);
-    int j_at = 0x7fffffff, b_at = 0, before = 0;
+    const long long t_lo = pair * total / g.pairs, t_hi = (pair + 1) * total / g.pairs;
+    // global index (entry * units + unit) of the first unit whose middle reaches t_lo, and t_hi
+    const int n_units = n_entries * g.units;
+    int lo = n_units, hi = n_units;
+    long long before = 0;
     for (int j0 = 0; j0 < n_entries; j0 += 32) {
         const int j = j0 + lane;
-        int nb = 0;
+        int w = 0;
         if (j < n_entries) {
             const int entry = c.union_list[j];
-            const int left = c.group_count[entry & 0xffff] - (entry >> 16) * kTcPassRows;
-            nb = min(left, kTcPassRows) > kTcSub ? g.units : (g.units + 1) >> 1;
+            w = tc_unit_cost(c.group_count[entry & 0xffff] - (entry >> 16) * kTcPassRows);
         }
-        int incl = nb;
+        const long long cost = (long long)w * g.units;
+        long long incl = cost;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
-            const int v = __shfl_up_sync(0xffffffffu, incl, o);
+            const long long v = __shfl_up_sync(0xffffffffu, incl, o);
             if (lane >= o) incl += v;
         }
-        const int start = before + incl - nb;                   // list position of the entry's first batch
-        if (nb > 0 && t_lo >= start && t_lo < start + nb) { j_at = j; b_at = t_lo - start; }
+        const long long start = before + incl - cost;           // cost prefix of the entry's first unit
+        if (w > 0) {
+            // unit u's middle is at start + w * u + w / 2; the first u whose middle is >= t
+            const long long a_lo = 2 * (t_lo - start) - w, a_hi = 2 * (t_hi - start) - w;
+            const long long u_lo = a_lo <= 0 ? 0 : (a_lo + 2 * w - 1) / (2 * w);
+            const long long u_hi = a_hi <= 0 ? 0 : (a_hi + 2 * w - 1) / (2 * w);
+            if (u_lo < g.units) lo = min(lo, j * g.units + (int)u_lo);
+            if (u_hi < g.units) hi = min(hi, j * g.units + (int)u_hi);
+        }
         before += __shfl_sync(0xffffffffu, incl, 31);
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
-        const int oj = __shfl_xor_sync(0xffffffffu, j_at, o), ob = __shfl_xor_sync(0xffffffffu, b_at, o);
-        if (oj < j_at) { j_at = oj; b_at = ob; }
+        lo = min(lo, __shfl_xor_sync(0xffffffffu, lo, o));
+        hi = min(hi, __shfl_xor_sync(0xffffffffu, hi, o));
     }
+    if (pair == g.pairs - 1) hi = n_units;
     if (lane == 0) {
-        out[0] = j_at == 0x7fffffff ? 0 : j_at;
-        out[1] = b_at;
-        out[2] = j_at == 0x7fffffff ? 0 : t_hi - t_lo;
+        out[0] = lo / g.units;
+        out[1] = lo - (lo / g.units) * g.units;
+        out[2] = max(0, hi - lo);
     }
 }
 
@@ -294,10 +348,9 @@ __device__ __forceinline__ void tc_epilogue(const CallView& c, const TcGeom& g, 
     long long pending = -1;                                // piece of the last sub-tile folded into `st`
     int pending_j = -1, pending_n = 0;
     bool pending_valid = false;
-    const int n_batches = run[2];
     TcWalk w;
-    if (n_batches > 0) w.start(c, g, run[0], run[1]);
-    for (int batch = 0; batch < n_batches; ++batch) {
+    w.start(c, run);
+    for (int batch = 0; w.left > 0; ++batch) {
         const int buf = batch & 1;
         tc_wait(smem_u32(&tmem_full[buf]), ((uint32_t)batch >> 1) & 1u, abort_flag, c.state);
         tc_fence_after();
@@ -306,7 +359,7 @@ __device__ __forceinline__ void tc_epilogue(const CallView& c, const TcGeom& g, 
             st.reset();
             pending = -1;
         }
-        const int t = 2 * (w.unit(g) + (w.wide ? 0 : quad)) + rank;            // this quad's sub-tile
+        const int t = 2 * (w.u + (w.wide ? 0 : quad)) + rank;                  // this quad's sub-tile
         const bool tile_ok = (w.wide || quad < w.nunits(g)) && t < g.tiles;
         const int hbase = w.wide ? quad * kTcSub : 0;                          // hidden row of the quad's first column
         const int ncols = tile_ok ? min(kTcSub, w.npad - hbase) : 0;           // columns this quad handles
@@ -359,26 +412,26 @@ __device__ __forceinline__ void tc_epilogue(const CallView& c, const TcGeom& g, 
             if (leader) mbar_arrive(tmem_empty_at + (uint32_t)buf * 8u);
             else mbar_arrive_cluster(tmem_empty_at + (uint32_t)buf * 8u);
         }
-        w.next(c, g, batch + 1 < n_batches);
+        w.next(c, g);
     }
     if (pending >= 0 && pending_valid) tc_flush_row<KT>(c, pp, st, pending_n, (size_t)pending);
 }
 
 // grid = 2 * g.pairs CTAs of kTcHeadThreads threads in clusters of two; dynamic shared memory: 1 KiB alignment
-// slack + kTcStages stages + the epilogue's exchange blocks + barriers.
+// slack + the operand ring + the epilogue's exchange blocks + barriers.
 __global__ void __launch_bounds__(kTcHeadThreads, 1)
     head_tc_kernel(CallView c, TcGeom g, TcPartials pp, const __grid_constant__ CUtensorMap map_w,
                    const uint16_t* __restrict__ hg, float* __restrict__ logits_tap) {
     extern __shared__ unsigned char tc_smem_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(tc_smem_raw) + 1023) & ~(uintptr_t)1023);
-    float* xchg = reinterpret_cast<float*>(smem + kTcStages * kTcStageBytes);
-    uint64_t* full = reinterpret_cast<uint64_t*>(smem + kTcStages * kTcStageBytes + kTcXchgBytes);
-    uint64_t* empty = full + kTcStages;
-    uint64_t* tmem_full = empty + kTcStages;      // [2]
+    float* xchg = reinterpret_cast<float*>(smem + kTcRingBytes);
+    uint64_t* full = reinterpret_cast<uint64_t*>(smem + kTcRingBytes + kTcXchgBytes);
+    uint64_t* empty = full + kTcMaxSlots;
+    uint64_t* tmem_full = empty + kTcMaxSlots;    // [2]
     uint64_t* tmem_empty = tmem_full + 2;         // [2] rank 0: both CTAs' epilogue warps have drained the buffer
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tmem_empty + 2);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-    int* run = const_cast<int*>(abort_flag) + 1;  // [3] entry and batch where the pair's run starts, number of batches
+    int* run = const_cast<int*>(abort_flag) + 1;  // [3] entry and unit where the pair's run starts, number of units
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int rank = (int)cluster_ctarank();
     const bool leader = rank == 0;
@@ -386,7 +439,7 @@ __global__ void __launch_bounds__(kTcHeadThreads, 1)
     // The kernel may be launched while its predecessors (gather, router) still run: everything up to the
     // dependency wait touches only the pair's shared and tensor memory.
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kTcStages; ++s) {
+        for (int s = 0; s < kTcMaxSlots; ++s) {
             // rank 0's "stage has landed" also counts an arrival from rank 1, sent once its own copies are in
             mbar_init(smem_u32(&full[s]), leader ? 2 : 1);
             mbar_init(smem_u32(&empty[s]), 2);                  // both issuers' MMAs on the stage have completed
@@ -414,40 +467,43 @@ __global__ void __launch_bounds__(kTcHeadThreads, 1)
     // nothing to do: the router chose the streaming kernel for this call, or the router stage reported a problem
     const bool skip = (c.adaptive && c.state->path_choice != 2) || call_is_poisoned(c.state);
 
-    // this pair's run of batches
+    // this pair's run of units
     if (warp == 0) tc_split_runs(c, g, skip ? 0 : c.state->n_virtual, (int)(blockIdx.x >> 1), run);
     __syncthreads();
-    const int n_batches = run[2];
 
     if (warp == 0) {
         if (lane == 0) {
-            int stage = 0;
-            uint32_t phase = 0;
+            TcRingPos rp;
             const uint64_t pol_first = l2_policy_evict_first(), pol_normal = l2_policy_evict_normal(),
                            pol_last = l2_policy_evict_last();
             TcWalk w;
-            if (n_batches > 0) w.start(c, g, run[0], run[1]);
-            for (int batch = 0; batch < n_batches; ++batch) {
-                const int u = w.unit(g), nu = w.nunits(g);
+            w.start(c, run);
+            while (w.left > 0) {
+                const int u = w.u, nu = w.nunits(g);
                 const int t0 = 2 * u + rank, t1 = 2 * (u + 1) + rank;           // this CTA's sub-tiles
                 const bool w0 = t0 < g.tiles, w1 = nu == 2 && t1 < g.tiles;
                 const uint32_t hbytes = (uint32_t)(w.npad >> 1) * 128u;         // this CTA's half of the hidden rows
-                const uint32_t hoff = w.wide ? kTcTileBytes : 2 * kTcTileBytes;
+                const TcRing ring = tc_ring_for(w.wide, nu);
+                if (rp.enter(ring)) {
+                    // another slot size from here on: every copy issued so far must have been consumed first
+                    for (int s = 0; s < kTcMaxSlots; ++s)
+                        tc_wait(smem_u32(&empty[s]), ((rp.parity >> s) & 1u) ^ 1u, abort_flag, c.state);
+                }
                 const uint32_t bytes = hbytes + (w0 ? kTcTileBytes : 0) + (w1 ? kTcTileBytes : 0);
                 const uint64_t pol_w = w.read_again ? pol_normal : pol_first;
                 const uint16_t* hsrc = hg + ((size_t)w.hrow + (size_t)rank * (w.npad >> 1)) * kTcK;
                 const int gidx = w.n / c.pack_div;
                 for (int ks = 0; ks < g.ksteps; ++ks) {
-                    tc_wait(smem_u32(&empty[stage]), phase ^ 1u, abort_flag, c.state);
-                    const uint32_t bar = smem_u32(&full[stage]);
-                    const uint32_t sb = smem_u32(smem + (size_t)stage * kTcStageBytes);
+                    tc_wait(smem_u32(&empty[rp.slot]), rp.par() ^ 1u, abort_flag, c.state);
+                    const uint32_t bar = smem_u32(&full[rp.slot]);
+                    const uint32_t sb = smem_u32(smem) + (uint32_t)rp.slot * ring.bytes;
                     mbar_expect_tx(bar, bytes);
                     if (w0) tma_load_5d(sb, &map_w, 0, 0, ks, t0 * 8, gidx, bar, pol_w);
                     if (w1) tma_load_5d(sb + kTcTileBytes, &map_w, 0, 0, ks, t1 * 8, gidx, bar, pol_w);
-                    bulk_g2s_hint(sb + hoff, hsrc + (size_t)ks * g.hg_rows * kTcK, hbytes, bar, pol_last);
-                    if (++stage == kTcStages) { stage = 0; phase ^= 1u; }
+                    bulk_g2s_hint(sb + ring.hoff, hsrc + (size_t)ks * g.hg_rows * kTcK, hbytes, bar, pol_last);
+                    rp.advance(ring);
                 }
-                w.next(c, g, batch + 1 < n_batches);
+                w.next(c, g);
             }
         }
     } else if (warp == 1 || warp == 10) {
@@ -455,14 +511,15 @@ __global__ void __launch_bounds__(kTcHeadThreads, 1)
             // issuer `a` owns accumulator a of every batch; both issuers commit on every stage and every batch
             // (a commit with nothing pending arrives at once), so the barriers always count two arrivals
             const int a = warp == 1 ? 0 : 1;
-            int stage = 0;
-            uint32_t phase = 0;
+            TcRingPos rp;
             const uint32_t ring_lo = tc_smem_desc_lo(smem_u32(smem)) + (uint32_t)a * (kTcTileBytes >> 4);
             TcWalk w;
-            if (n_batches > 0) w.start(c, g, run[0], run[1]);
-            for (int batch = 0; batch < n_batches; ++batch) {
+            w.start(c, run);
+            for (int batch = 0; w.left > 0; ++batch) {
                 const int buf = batch & 1;
-                const uint32_t hoff_lo = ((w.wide ? kTcTileBytes : 2 * kTcTileBytes) - a * kTcTileBytes) >> 4;
+                const TcRing ring = tc_ring_for(w.wide, w.nunits(g));
+                rp.enter(ring);
+                const uint32_t hoff_lo = (ring.hoff - a * kTcTileBytes) >> 4;
                 const uint32_t idesc = tc_idesc(256, w.npad);
                 const bool mine = a < w.nunits(g);
                 tc_wait(smem_u32(&tmem_empty[buf]), (((uint32_t)batch >> 1) & 1u) ^ 1u, abort_flag, c.state);   // drained
@@ -471,30 +528,36 @@ __global__ void __launch_bounds__(kTcHeadThreads, 1)
                 for (int ks = 0; ks < g.ksteps; ++ks) {
                     // (an issuer with nothing to do in this batch waits all the same: its commits must not get
                     // ahead of the stage they speak for)
-                    tc_wait(smem_u32(&full[stage]), phase, abort_flag, c.state);        // this CTA's copies and the other's
+                    tc_wait(smem_u32(&full[rp.slot]), rp.par(), abort_flag, c.state);   // this CTA's copies and the other's
                     if (mine) {
                         tc_fence_after();
-                        const uint32_t a_lo = ring_lo + (uint32_t)stage * (kTcStageBytes >> 4);
+                        const uint32_t a_lo = ring_lo + (uint32_t)rp.slot * (ring.bytes >> 4);
                         const uint32_t b_lo = a_lo + hoff_lo;
 #pragma unroll
                         for (int kk = 0; kk < kTcK / 16; ++kk)               // 32 bytes (two 16-byte units) per 16 columns
                             tc_mma_pair(acc, a_lo + 2 * kk, b_lo + 2 * kk, idesc, kk ? 1u : (ks ? 1u : 0u));
                     }
-                    tc_commit_pair(smem_u32(&empty[stage]));  // the stage is free in both CTAs once both issuers' MMAs have read it
-                    if (++stage == kTcStages) { stage = 0; phase ^= 1u; }
+                    tc_commit_pair(smem_u32(&empty[rp.slot]));  // the slot is free in both CTAs once both issuers' MMAs have read it
+                    rp.advance(ring);
                 }
                 tc_commit_pair(smem_u32(&tmem_full[buf]));    // accumulators complete, in both CTAs
-                w.next(c, g, batch + 1 < n_batches);
+                w.next(c, g);
             }
         } else if (lane == 0 && warp == 1) {
             // rank 1: pass the news that a stage of this CTA has landed on to the MMA issuer in rank 0
             const uint32_t peer_at = cluster_map_shared(smem_u32(full), 0);
-            int stage = 0;
-            uint32_t phase = 0;
-            for (int i = 0; i < n_batches * g.ksteps; ++i) {
-                tc_wait(smem_u32(&full[stage]), phase, abort_flag, c.state);
-                mbar_arrive_cluster(peer_at + (uint32_t)stage * 8u);            // counts on rank 0's barrier of the stage
-                if (++stage == kTcStages) { stage = 0; phase ^= 1u; }
+            TcRingPos rp;
+            TcWalk w;
+            w.start(c, run);
+            while (w.left > 0) {
+                const TcRing ring = tc_ring_for(w.wide, w.nunits(g));
+                rp.enter(ring);
+                for (int ks = 0; ks < g.ksteps; ++ks) {
+                    tc_wait(smem_u32(&full[rp.slot]), rp.par(), abort_flag, c.state);
+                    mbar_arrive_cluster(peer_at + (uint32_t)rp.slot * 8u);      // counts on rank 0's barrier of the slot
+                    rp.advance(ring);
+                }
+                w.next(c, g);
             }
         }
     } else {
