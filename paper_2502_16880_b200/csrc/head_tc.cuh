@@ -259,17 +259,19 @@ struct TcWalk {
     }
 };
 
-// Bytes a CTA takes in per 64 columns for one unit of an entry with `rows` rows, in 128-byte units: the weight
-// sub-tile plus its share of the hidden rows (a narrow batch's two units share one read of them).
+// Relative time of one unit of an entry with `rows` rows.  A narrow entry's units go two to a batch and a batch
+// streams at what an SM can take in (its weight tiles plus its share of the hidden rows, in 128-byte units per
+// 64 columns); a wide entry's unit is a batch of its own and takes about as long as a narrow batch of two
+// (measured: 38-41 us against 36-40 us on the Llama3-8B shape), the MMA issue and the slot hand-over, not the
+// bytes, setting its pace.
 __device__ __forceinline__ int tc_unit_cost(int rows) {
     const int npad = (max(1, min(rows, kTcPassRows)) + 15) & ~15;
-    return kTcSub + (npad > kTcSub ? npad >> 1 : npad >> 2);
+    return npad > kTcSub ? 2 * kTcSub + (npad >> 2) : kTcSub + (npad >> 2);
 }
 
 // Cuts the unit list into g.pairs runs of (almost) equal cost (one warp).  out[0], out[1]: entry and unit where
-// the pair's run starts; out[2]: its number of units.  The kernel is bound by what it reads, so the cost of a
-// unit is its bytes (tc_unit_cost); run p holds the units whose cost prefix, taken at the unit's middle, lies in
-// [p, p + 1) * total / pairs.
+// the pair's run starts; out[2]: its number of units.  Run p holds the units whose cost prefix (tc_unit_cost),
+// taken at the unit's middle, lies in [p, p + 1) * total / pairs.
 __device__ __forceinline__ void tc_split_runs(const CallView& c, const TcGeom& g, int n_entries, int pair, int* out) {
     const int lane = threadIdx.x & 31;
     long long total = 0;
