@@ -29,7 +29,7 @@ struct Layout {
     size_t w_gate, group_tokens, state, gate, sel, slot_of, group_count, group_offset, bucket_row, bucket_slot,
         slot_desc, union_list, union_rank, part_max, part_sum, part_val, part_id, sp_max, sp_sum, sp_val, sp_id,
         cand_val, cand_id, route_mid, tc_hg, tc_max, tc_sum, tc_val, tc_id, stage_hidden, stage_ids, stage_logprobs, total;
-    size_t packed_bytes, cand_cap;
+    size_t packed_bytes, cand_cap, cand_rows;
     int v, T;
     int KB, T16;                 // packed layout (see packed_chunk_offset)
     size_t route_bands;
@@ -88,6 +88,9 @@ size_t stream_smem_bytes(const StreamGeom& g) {
 }
 
 constexpr int kTcMinRows = 96;          // above this many rows the tensor-core path is the faster one (measured, iid rows)
+constexpr int kTcMinRowsPerGroup = 8;   // ... and from this many rows per group on average (the streaming path reads a
+                                        // group once per 16 rows; measured on the three paper shapes: equal at 7.5, 1.15x-2x
+                                        // faster from 12 on)
 constexpr int kTcProvisionRows = 32;    // handles for more rows get the tensor-core workspace (adaptive calls use it from 33 rows)
 constexpr int kMergeSmemCands = 4096;   // candidates the streaming merge keeps in shared memory
 
@@ -120,8 +123,17 @@ Layout make_layout(const coral_lmhead_config& c) {
     L.sp_sum = take(sp * 4);
     L.sp_val = take(sp * kt * 4);
     L.sp_id = take(sp * kt * 4);
-    const size_t cand_rows = M < (size_t)kStreamMaxM ? M : (size_t)kStreamMaxM;
+    // candidate scratch of the merge: what does not fit its shared memory.  The streaming path has at most
+    // grid + 2 k_groups pieces per row and at most kStreamMaxM rows; the tensor-core path one piece per (slot,
+    // sub-tile), which only outgrows shared memory when very many groups are active (dense-equivalent calls)
+    size_t cand_rows = M < (size_t)kStreamMaxM ? M : (size_t)kStreamMaxM;
     L.cand_cap = ((size_t)kStreamGridCap + 2 * kg) * kt;
+    const size_t tc_cands = M > (size_t)kTcProvisionRows ? kg * (size_t)((L.v + kTcSub - 1) / kTcSub) * kt : 0;
+    if (tc_cands > (size_t)kMergeSmemCands) {
+        cand_rows = M;
+        if (tc_cands > L.cand_cap) L.cand_cap = tc_cands;
+    }
+    L.cand_rows = cand_rows;
     L.cand_val = take(cand_rows * L.cand_cap * 4);
     L.cand_id = take(cand_rows * L.cand_cap * 4);
     L.part_max = take(M * kg * T * 4);
@@ -321,15 +333,17 @@ bool stream_ok(const coral_lmhead_s* h, int M) { return h->stream_smem > 0 && M 
 // CORAL_PATH_STREAM: streaming kernel (M <= 128, H a multiple of 256, <= 4096); CORAL_PATH_SIMT_PLAIN: any shape.  Returns 0 if the
 // forced path cannot run this call.
 bool tc_usable(const coral_lmhead_s* h, int M, int kg) {
+    const size_t cands = (size_t)kg * h->L.tc_tiles * h->cfg.max_k_tokens;
     return h->tc_ok && (size_t)M * kg <= h->L.tc_rows && kg * h->L.tc_tiles <= kMergeMaxPieces &&
-           kg * h->L.tc_tiles * h->cfg.max_k_tokens <= kMergeSmemCands;
+           (cands <= (size_t)kMergeSmemCands || (cands <= h->L.cand_cap && (size_t)M <= h->L.cand_rows));
 }
 
 int choose_path(const coral_lmhead_s* h, int M, int kg) {
     if (h->forced_path == CORAL_PATH_STREAM) return stream_ok(h, M) ? CORAL_PATH_STREAM : 0;
     if (h->forced_path == CORAL_PATH_TCGEN05) return tc_usable(h, M, kg) ? CORAL_PATH_TCGEN05 : 0;
     if (h->forced_path != CORAL_PATH_AUTO && h->forced_path != CORAL_PATH_ADAPTIVE) return h->forced_path;
-    if (M > kTcMinRows && tc_usable(h, M, kg)) return CORAL_PATH_TCGEN05;
+    if ((M > kTcMinRows || (long long)M * kg >= (long long)kTcMinRowsPerGroup * h->cfg.n_groups) && tc_usable(h, M, kg))
+        return CORAL_PATH_TCGEN05;
     if (stream_ok(h, M)) return CORAL_PATH_STREAM;
     return tc_usable(h, M, kg) ? CORAL_PATH_TCGEN05 : CORAL_PATH_SIMT_PLAIN;
 }
@@ -626,7 +640,7 @@ static int draft_impl(coral_lmhead_handle h, const void* hidden_dev, int M, int 
         StreamPartials pp{tp.pmax, tp.psum, tp.pval, tp.pid};
         {
             const int p_cap = k_groups * L.tc_tiles;
-            const int c_cap = p_cap * k_tokens;          // tc_usable() keeps this within kMergeSmemCands
+            const int c_cap = p_cap * k_tokens < kMergeSmemCands ? p_cap * k_tokens : kMergeSmemCands;   // more: global scratch
             launch_pdl(merge_stream_kernel, dim3(M), dim3(kMergeStreamThreads), merge_smem_bytes(p_cap, c_cap), st, c, mg,
                        pp, mg, pp, reinterpret_cast<float*>(h->ws + L.cand_val), reinterpret_cast<int32_t*>(h->ws + L.cand_id),
                        (int)L.cand_cap, c_cap, p_cap, merge_mode, out_ids_dev, merge_out, out_lse_dev);

@@ -441,7 +441,7 @@ __global__ void __launch_bounds__(kStreamThreads, 1) head_stream_kernel(CallView
 // another GPU have descriptor -1 and no pieces.  merge_partials_kernel combines the GPUs' records.
 constexpr int kMergeJoint = 0, kMergeFactorised = 1, kMergePartial = 2;
 constexpr int kMergeStreamThreads = 256;
-constexpr int kMergeMaxPieces = 1024;         // >= grid + 2 * k_groups for every supported shape
+constexpr int kMergeMaxPieces = 2048;         // >= grid + 2 * k_groups for every supported shape
 constexpr int kMergeRankMax = 256;            // survivors ranked by counting; more fall back to k rounds
 __global__ void __launch_bounds__(kMergeStreamThreads) merge_stream_kernel(CallView c, StreamGeom g_in, StreamPartials pp_in,
                                                                            StreamGeom g_tc, StreamPartials pp_tc,
