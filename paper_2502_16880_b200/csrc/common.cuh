@@ -52,6 +52,12 @@ struct CallView {
     float* part_val;               // [M][k_groups][T][k_tokens]
     int32_t* part_id;              // [M][k_groups][T][k_tokens]
     DeviceState* state;
+    // capacities of the arrays above, for the range-checked build (CORAL_CHECK_BOUNDS)
+    int cap_pairs;                 // entries of bucket_row / bucket_slot / slot_desc / sel
+    int cap_hg_rows;               // rows of one column block of the tensor-core path's gathered hidden matrix
+    long long cap_part_stream;     // partial records of the streaming path
+    long long cap_part_tc;         // partial records of the tensor-core path
+    long long cap_packed;          // 16-byte units of the packed copy
 };
 
 // Packed layout of the LM head: [group][item of 16 vocab rows, ascending token id][block of 64 columns]
@@ -116,6 +122,25 @@ __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;"
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
 __device__ __forceinline__ void set_status(DeviceState* st, int code) { atomicCAS(&st->status, 0, code); }
+
+// Range-checked build (-DCORAL_CHECK_BOUNDS; the stand-in for a memory checker): every index the kernels
+// compute from the router's output - bucket positions, slot descriptors, union-list entries, piece indices,
+// token-table reads, offsets into the packed copy and the gathered rows - is compared with the capacity of
+// what it indexes.  A violation sets CORAL_ERR_BOUNDS in the status word; a read then takes element 0
+// instead and a write is skipped, so nothing traps and nothing outside the buffers is touched.  In the
+// normal build the macros cost nothing.
+#ifdef CORAL_CHECK_BOUNDS
+__device__ __forceinline__ bool index_ok(long long i, long long n, DeviceState* st) {
+    if (i >= 0 && i < n) return true;
+    set_status(st, -6);
+    return false;
+}
+#define CORAL_IDX(i, n, st) (::coral::index_ok((long long)(i), (long long)(n), (st)) ? (i) : 0)
+#define CORAL_IDX_OK(i, n, st) ::coral::index_ok((long long)(i), (long long)(n), (st))
+#else
+#define CORAL_IDX(i, n, st) (i)
+#define CORAL_IDX_OK(i, n, st) true
+#endif
 
 // The status word is sticky until the host reads it.  A call whose router stage reported a problem (forced
 // groups out of range or repeated: the bucket arrays are then inconsistent) must not be followed by kernels

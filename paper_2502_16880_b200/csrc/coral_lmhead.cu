@@ -237,6 +237,11 @@ CallView make_view(const coral_lmhead_s* h, const void* hidden, int M, int kg, i
     c.part_val = reinterpret_cast<float*>(ws + L.part_val);
     c.part_id = reinterpret_cast<int32_t*>(ws + L.part_id);
     c.state = reinterpret_cast<DeviceState*>(ws + L.state);
+    c.cap_pairs = (int)((size_t)h->cfg.max_M * h->cfg.max_k_groups);
+    c.cap_hg_rows = L.tc_hg_rows;
+    c.cap_part_stream = (long long)kStreamGridCap * stream_seg_max(h->cfg.n_groups, kStreamGridMin) * kStreamPassRows;
+    c.cap_part_tc = (long long)L.tc_vcap * L.tc_tiles * kTcPassRows;
+    c.cap_packed = (long long)(L.packed_bytes / 16);
     return c;
 }
 

@@ -181,7 +181,7 @@ __device__ __forceinline__ void stream_segment_mma(const CallView& c, const Stre
     for (int nt = 0; nt < NT; ++nt) {
         const int rr = nt * 8 + gq;
         const bool valid = rr < R;
-        const uint16_t* hp = c.hidden + (size_t)(valid ? c.bucket_row[off + rr] : 0) * c.H;
+        const uint16_t* hp = c.hidden + (size_t)(valid ? CORAL_IDX(c.bucket_row[CORAL_IDX(off + rr, c.cap_pairs, c.state)], c.M, c.state) : 0) * c.H;
 #pragma unroll
         for (int sl = 0; sl < SL; ++sl)
 #pragma unroll
@@ -270,14 +270,14 @@ __device__ __forceinline__ void stream_segment_stats(const CallView& c, const St
         run_max[u] = kNegInf; run_sum[u] = 0.f; lv[u] = kNegInf; lid[u] = kNoToken;
         kth[u] = kNegInf; kth_id[u] = kNoToken;
         const int r = sw + kStreamStatWarps * u;
-        my_m[u] = r < R ? c.bucket_row[off + r] : 0;
-        my_slot[u] = r < R ? c.bucket_slot[off + r] : 0;
+        my_m[u] = r < R ? CORAL_IDX(c.bucket_row[CORAL_IDX(off + r, c.cap_pairs, c.state)], c.M, c.state) : 0;
+        my_slot[u] = r < R ? CORAL_IDX(c.bucket_slot[CORAL_IDX(off + r, c.cap_pairs, c.state)], c.k_groups, c.state) : 0;
     }
     for (int item = lo; item < hi; ++item, ++it) {
         const int row0 = (item - j * g.T) * kStreamTile;
         const int rows = min(kStreamTile, c.v - row0);
         const bool have = lane < rows;
-        const int32_t* tokens = c.group_tokens + (size_t)n * c.v + row0;
+        const int32_t* tokens = c.group_tokens + CORAL_IDX((size_t)n * c.v + row0, c.V, c.state);
         const int zb = it % kStreamZBufs;
         mbar_wait(smem_u32(&sh.zfull[zb]), (uint32_t)(it / kStreamZBufs) & 1u, sh.abort_flag, c.state);
         float zv[kOwn];
@@ -310,10 +310,11 @@ __device__ __forceinline__ void stream_segment_stats(const CallView& c, const St
         const int r = sw + kStreamStatWarps * u;
         if (r < R) {
             const size_t p = ((size_t)blockIdx.x * g.seg_max + seg) * kStreamPassRows + r;
+            const bool p_ok = CORAL_IDX_OK(p, c.cap_part_stream, c.state);
             const float mx = warp_max(run_max[u]);                       // combine the lanes' online softmax states
             const float sm = warp_sum(run_sum[u] * __expf(run_max[u] - mx));
-            if (lane == 0) { pp.pmax[p] = mx; pp.psum[p] = sm; }
-            if (lane < c.k_tokens) { pp.pval[p * c.k_tokens + lane] = lv[u]; pp.pid[p * c.k_tokens + lane] = lid[u]; }
+            if (p_ok && lane == 0) { pp.pmax[p] = mx; pp.psum[p] = sm; }
+            if (p_ok && lane < c.k_tokens) { pp.pval[p * c.k_tokens + lane] = lv[u]; pp.pid[p * c.k_tokens + lane] = lid[u]; }
         }
     }
 }
@@ -385,6 +386,12 @@ __global__ void __launch_bounds__(kStreamThreads, 1) head_stream_kernel(CallView
             const int n = sh.segtab[min(j - sh.j_first, kStreamSegTab - 1)] & 0xffff;
             int t = pos - j * g.T;
             const uint16_t* src = c.packed + (((size_t)(n / c.pack_div) * g.T + t) * g.kstages) * (size_t)(kStreamTile * g.kc);
+#ifdef CORAL_CHECK_BOUNDS
+            {   // the whole run of slabs copied for this segment must lie inside the packed copy
+                const long long first16 = (src - c.packed) / 8, n16 = (long long)(seg_hi - pos) * g.kstages * (g.stage_bytes / 16);
+                if (!CORAL_IDX_OK(n, c.N, c.state) || !CORAL_IDX_OK(first16 + n16 - 1, c.cap_packed, c.state)) src = c.packed;
+            }
+#endif
             for (int item = pos; item < seg_hi; ++item, ++t) {
                 const uint32_t bytes = (uint32_t)g.stage_bytes;    // rows past the group's size are zero padding
                 for (int ks = 0; ks < g.kstages; ++ks) {
@@ -414,7 +421,7 @@ __global__ void __launch_bounds__(kStreamThreads, 1) head_stream_kernel(CallView
         const int seg = min(j - sh.j_first, kStreamSegTab - 1);
         const int seg_hi = min(sh.hi, (j + 1) * g.T);
         const int entry = sh.segtab[seg];
-        const int n = entry & 0xffff, pass = entry >> 16;
+        const int n = CORAL_IDX(entry & 0xffff, c.N, c.state), pass = entry >> 16;
         const int R = max(1, min(c.group_count[n] - pass * kStreamPassRows, kStreamPassRows));
         if (!mma_role)
             stream_segment_stats(c, g, sh, pp, logits_tap, n, pass, R, j, pos, seg_hi, seg, it);
@@ -547,6 +554,9 @@ __global__ void __launch_bounds__(kMergeStreamThreads) merge_stream_kernel(CallV
     // pass 1 over the pieces (all loads of a thread's pieces issued together)
     float mx = kNegInf;
     for (int q = threadIdx.x; q < P; q += kMergeStreamThreads) {
+#ifdef CORAL_CHECK_BOUNDS
+        if (!index_ok(s_piece[q], took_tc || g.tc_tiles > 0 ? c.cap_part_tc : c.cap_part_stream, c.state)) s_piece[q] = 0;
+#endif
         const size_t p = (size_t)s_piece[q];
         const float a = pp.pmax[p], b = pp.psum[p];
         float l = pp.pval[p * c.k_tokens + c.k_tokens - 1], h = pp.pval[p * c.k_tokens];

@@ -108,11 +108,12 @@ __global__ void __launch_bounds__(128) tc_gather_kernel(CallView c, uint16_t* __
     if (call_is_poisoned(c.state)) return;                   // the router stage reported a problem: index with nothing
     if (c.adaptive && c.state->path_choice != 2) return;     // the router chose the streaming kernel for this call
     if (p >= c.group_offset[c.N]) return;          // fewer pairs than M * k_groups when the vocab is sharded
-    const int m = c.bucket_row[p];
-    const int n = c.sel[(size_t)m * c.k_groups + c.bucket_slot[p]];
+    const int m = CORAL_IDX(c.bucket_row[p], c.M, c.state);
+    const int n = CORAL_IDX(c.sel[CORAL_IDX((size_t)m * c.k_groups + c.bucket_slot[p], c.cap_pairs, c.state)], c.N, c.state);
     const int rg = p - c.group_offset[n];
     const int pass = rg / kTcPassRows;
     const int row = tc_entry_row(c.group_offset[n] + pass * kTcPassRows, c.union_rank[n] + pass) + rg % kTcPassRows;
+    if (!CORAL_IDX_OK(row, hg_rows, c.state)) return;
     const uint4* src = reinterpret_cast<const uint4*>(c.hidden + (size_t)m * c.H);
     uint4* dst = reinterpret_cast<uint4*>(hg);
     const int chunks = c.H >> 3;
@@ -214,6 +215,7 @@ __device__ __forceinline__ void tc_fold_block(TcRowState<KT>& st, const float* x
 template <int KT>
 __device__ __forceinline__ void tc_flush_row(const CallView& c, const TcPartials& pp, const TcRowState<KT>& st, int n,
                                              size_t pidx) {
+    if (!CORAL_IDX_OK(pidx, c.cap_part_tc, c.state)) return;
     pp.pmax[pidx] = st.mx;
     pp.psum[pidx] = st.sum;
 #pragma unroll
@@ -221,7 +223,7 @@ __device__ __forceinline__ void tc_flush_row(const CallView& c, const TcPartials
         if (j < c.k_tokens) {
             pp.pval[pidx * c.k_tokens + j] = st.lv[j];
             pp.pid[pidx * c.k_tokens + j] =
-                st.li[j] == kNoToken ? kNoToken : __ldg(c.group_tokens + (size_t)n * c.v + st.li[j]);
+                st.li[j] == kNoToken ? kNoToken : __ldg(c.group_tokens + CORAL_IDX((size_t)n * c.v + st.li[j], c.V, c.state));
         }
     }
 }
@@ -235,8 +237,8 @@ struct TcWalk {
     int n, R, npad, first, hrow;
     bool wide, read_again;
     __device__ __forceinline__ void load(const CallView& c) {
-        const int entry = c.union_list[j];
-        n = entry & 0xffff;
+        const int entry = c.union_list[CORAL_IDX(j, c.union_cap, c.state)];
+        n = CORAL_IDX(entry & 0xffff, c.N, c.state);
         const int pass = entry >> 16;
         const int rows = c.group_count[n] - pass * kTcPassRows;
         R = max(1, min(rows, kTcPassRows));
@@ -245,6 +247,8 @@ struct TcWalk {
         wide = npad > kTcSub;
         first = c.group_offset[n] + pass * kTcPassRows;        // first bucket position of the entry
         hrow = tc_entry_row(first, j);
+        if (!CORAL_IDX_OK(hrow + npad - 1, c.cap_hg_rows, c.state)) hrow = 0;     // (checked build) read rows that exist
+        if (!CORAL_IDX_OK(first + R - 1, c.cap_pairs, c.state)) first = 0;
     }
     __device__ __forceinline__ void start(const CallView& c, const int* run) {
         j = run[0]; u = run[1]; left = run[2];
@@ -369,7 +373,7 @@ __device__ __forceinline__ void tc_epilogue(const CallView& c, const TcGeom& g, 
             const int hrow = hbase + q * 32 + lane;                            // the hidden row this thread owns
             const bool row_valid = hrow < w.R;
             const size_t pidx = ((size_t)w.j * g.tiles + t) * kTcPassRows + hrow;
-            if (pending >= 0 && pending_valid) {                               // not the entry's last piece after all
+            if (pending >= 0 && pending_valid && CORAL_IDX_OK(pending, c.cap_part_tc, c.state)) {   // not the entry's last piece after all
                 pp.pmax[pending] = kNegInf;
                 pp.psum[pending] = 0.f;
             }

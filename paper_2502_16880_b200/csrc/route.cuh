@@ -286,6 +286,7 @@ __global__ void __launch_bounds__(kRouteThreads)
             const int m = __ffs(left) - 1;
             left &= left - 1;
             const int sl = s_slot[m][n];
+            if (!CORAL_IDX_OK(off + pos, c.cap_pairs, c.state) || !CORAL_IDX_OK(m * c.k_groups + sl, c.cap_pairs, c.state)) continue;
             c.bucket_row[off + pos] = m;
             c.bucket_slot[off + pos] = sl;
             const int pass = c.pass_rows > 0 ? pos / c.pass_rows : 0;
@@ -541,6 +542,7 @@ __global__ void __launch_bounds__(256)
                 const int m = w * 32 + __ffs(left) - 1;
                 left &= left - 1;
                 const int sl = s_slot[m * c.N + n];
+                if (!CORAL_IDX_OK(off + pos, c.cap_pairs, c.state) || !CORAL_IDX_OK(m * c.k_groups + sl, c.cap_pairs, c.state)) continue;
                 c.bucket_row[off + pos] = m;
                 c.bucket_slot[off + pos] = sl;
                 const int pass = pr > 0 ? pos / pr : 0;
@@ -621,10 +623,12 @@ __global__ void __launch_bounds__(256) bucket_group_kernel(CallView c, int* __re
         }
         if (sl >= 0) {
             const int pos = running + before + __popc(bal & ((1u << lane) - 1u));
+            if (CORAL_IDX_OK(off + pos, c.cap_pairs, c.state) && CORAL_IDX_OK(m * c.k_groups + sl, c.cap_pairs, c.state)) {
             c.bucket_row[off + pos] = m;
             c.bucket_slot[off + pos] = sl;
             const int pass = c.pass_rows > 0 ? pos / c.pass_rows : 0;
             c.slot_desc[(size_t)m * c.k_groups + sl] = ((virt + pass) << 8) | ((pos - pass * max(c.pass_rows, 1)) & 255);
+            }
         }
         running += all;
         __syncthreads();

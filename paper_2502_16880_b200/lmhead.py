@@ -14,7 +14,8 @@ import os
 import torch
 
 _PKG = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_PKG, "libcoral_lmhead.so")
+# CORAL_LMHEAD_LIB selects another build of the same library (the range-checked one, see build.py)
+LIB_PATH = os.environ.get("CORAL_LMHEAD_LIB") or os.path.join(_PKG, "libcoral_lmhead.so")
 
 CORAL_OK = 0
 CORAL_ERR_INVALID = -1
