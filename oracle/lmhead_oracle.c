@@ -15,7 +15,11 @@
  *   4. joint mode: log-softmax over all active logits of the row;
  *      factorised mode (Eq. 8): log p(x) = log p_router(n) + log p_group(x^n),
  *      p_router = Softmax over all N scores (Eq. 7), p_group = softmax inside
- *      group n, independent of the other groups.
+ *      group n, independent of the other groups.  The paper does not say
+ *      whether p_router is renormalised over the selected groups; mode 2 is
+ *      that variant: log p(x) = log (p_router(n) / sum of p_router over the
+ *      selected groups) + log p_group(x^n), whose mass over the active
+ *      vocabulary is 1.
  *   5. the k_tokens best tokens by log-probability (descending; equal ->
  *      lower token id): the "top 10 candidates" of Appendix B, tree decoding.
  *
@@ -80,7 +84,8 @@ int coral_oracle_threads(void);
  *   W1        [H x H] bf16 or NULL (NULL: g = W_gate h)
  *   forced_groups [M x k_groups] or NULL: use these groups instead of step 2
  *   gate_override [M x N] doubles or NULL: use these scores instead of step 1
- *   factorised: 0 = joint log-softmax over the active logits, 1 = Eq. 8
+ *   factorised: 0 = joint log-softmax over the active logits, 1 = Eq. 8,
+ *               2 = Eq. 8 with p_router renormalised over the selected groups
  * Outputs (any may be NULL):
  *   out_gate [M x N], out_groups [M x k_groups] (selection order),
  *   out_logits [M x k_groups x v] and out_logit_tokens (same shape): slot s
@@ -102,6 +107,7 @@ int coral_oracle_draft(const uint16_t *W_vocab, const int32_t *group_map, const 
     const int v = V / N;
     if (k_groups < 1 || k_groups > N) return ORACLE_ERR_INVALID;
     if (k_tokens < 1 || (long)k_tokens > (long)k_groups * v) return ORACLE_ERR_INVALID;
+    if (factorised < 0 || factorised > 2) return ORACLE_ERR_INVALID;
     {
         long *cnt = (long *)calloc((size_t)N, sizeof(long));
         if (!cnt) return ORACLE_ERR_NOMEM;
@@ -128,10 +134,11 @@ int coral_oracle_draft(const uint16_t *W_vocab, const int32_t *group_map, const 
     double *z = (double *)malloc(sizeof(double) * (size_t)n_active);
     int32_t *tok = (int32_t *)malloc(sizeof(int32_t) * (size_t)n_active);
     double *group_lse = (double *)malloc(sizeof(double) * (size_t)k_groups);
+    double *z_sel = (double *)malloc(sizeof(double) * (size_t)k_groups);
     scored_t *cand = (scored_t *)malloc(sizeof(scored_t) * (size_t)n_active);
     int rc = ORACLE_OK;
     if (!h || !u || !g || !log_router || !order || !sel || !slot_of_group || !z || !tok ||
-        !group_lse || !cand) {
+        !group_lse || !z_sel || !cand) {
         rc = ORACLE_ERR_NOMEM;
         goto done;
     }
@@ -202,10 +209,15 @@ int coral_oracle_draft(const uint16_t *W_vocab, const int32_t *group_map, const 
         for (int s = 0; s < k_groups; ++s) group_lse[s] = log_sum_exp(z + (long)s * v, v);
 
         /* step 5: rank by log-probability */
+        double log_selected_mass = 0.0;     /* log of the router mass of the selected groups (mode 2) */
+        if (factorised == 2) {
+            for (int s = 0; s < k_groups; ++s) z_sel[s] = log_router[sel[s]];
+            log_selected_mass = log_sum_exp(z_sel, k_groups);
+        }
         for (long i = 0; i < n_active; ++i) {
             int s = (int)(i / v);
             cand[i].index = tok[i];
-            cand[i].score = factorised ? log_router[sel[s]] + (z[i] - group_lse[s]) : z[i] - lse;
+            cand[i].score = factorised ? log_router[sel[s]] - log_selected_mass + (z[i] - group_lse[s]) : z[i] - lse;
         }
         qsort(cand, (size_t)n_active, sizeof(scored_t), by_score_desc);
 
@@ -224,7 +236,7 @@ int coral_oracle_draft(const uint16_t *W_vocab, const int32_t *group_map, const 
 
 done:
     free(h); free(u); free(g); free(log_router); free(order); free(sel); free(slot_of_group);
-    free(z); free(tok); free(group_lse); free(cand);
+    free(z); free(tok); free(group_lse); free(z_sel); free(cand);
     return rc;
 }
 

@@ -68,7 +68,8 @@ def _ptr(a):
 
 def draft(W_vocab, group_map, W_gate, hidden, k_groups, k_tokens, *, W1=None, forced_groups=None,
           gate_override=None, factorised=False, want_logits=True, lib_path=None) -> OracleResult:
-    """Run the oracle.  bf16 tensors are uint16 bit patterns (numpy)."""
+    """Run the oracle.  bf16 tensors are uint16 bit patterns (numpy).  factorised: False/0 joint log-softmax,
+    True/1 Eq. 8, 2 Eq. 8 with p_router renormalised over the selected groups."""
     lib = _load(lib_path)
     W_vocab = np.ascontiguousarray(W_vocab, dtype=np.uint16)
     W_gate = np.ascontiguousarray(W_gate, dtype=np.uint16)
@@ -100,7 +101,7 @@ def draft(W_vocab, group_map, W_gate, hidden, k_groups, k_tokens, *, W1=None, fo
         ids=np.zeros((M, k_tokens), np.int32), logprobs=np.zeros((M, k_tokens)))
     rc = lib.coral_oracle_draft(
         _ptr(W_vocab), _ptr(group_map), _ptr(W_gate), _ptr(W1), _ptr(hidden), H, V, N, M,
-        int(k_groups), int(k_tokens), _ptr(forced_groups), _ptr(gate_override), int(bool(factorised)),
+        int(k_groups), int(k_tokens), _ptr(forced_groups), _ptr(gate_override), int(factorised),
         _ptr(res.gate), _ptr(res.groups), _ptr(res.logits), _ptr(res.logit_tokens), _ptr(res.lse),
         _ptr(res.group_lse), _ptr(res.log_router), _ptr(res.ids), _ptr(res.logprobs))
     if rc != 0:

@@ -25,8 +25,11 @@ MUTANTS = {
     "gate_transposed": ("bf16_value(W_gate[(size_t)n * H + j]) * u[j]", "bf16_value(W_gate[(size_t)j * N + n]) * u[j]"),
     "joint_uses_group_lse": (": z[i] - lse;", ": z[i] - group_lse[s];"),
     "bf16_shift": ("(uint32_t)bits << 16", "(uint32_t)bits << 15"),
-    "factorised_drops_router": ("factorised ? log_router[sel[s]] + (z[i] - group_lse[s])",
+    "factorised_drops_router": ("factorised ? log_router[sel[s]] - log_selected_mass + (z[i] - group_lse[s])",
                                 "factorised ? (z[i] - group_lse[s])"),
+    "renormalised_mass_sign": ("factorised ? log_router[sel[s]] - log_selected_mass +",
+                               "factorised ? log_router[sel[s]] + log_selected_mass +"),
+    "renormalised_over_all_groups": ("z_sel[s] = log_router[sel[s]];", "z_sel[s] = log_router[s];"),
     "selects_lowest_groups": ("sel[s] = order[s].index;", "sel[s] = order[N - 1 - s].index;"),
     "always_row_zero": ("h[j] = bf16_value(hidden[(size_t)m * H + j]);", "h[j] = bf16_value(hidden[j]);"),
     "router_softmax_not_normalised": ("log_router[n] = g[n] - l;", "log_router[n] = g[n];"),
@@ -91,6 +94,14 @@ def _battery(lib_path):
             assert np.array_equal(r.ids[m], order)
             np.testing.assert_allclose(r.logprobs[m], lp[m, order], atol=1e-11)
 
+    def p6r():
+        # renormalised variant: the probabilities of the active vocabulary sum to 1 and keep Eq. 8's order
+        r1 = orc.draft(W, gm, Wg, h, 2, 9, factorised=1, lib_path=lib_path)
+        r2 = orc.draft(W, gm, Wg, h, 2, 9, factorised=2, lib_path=lib_path)
+        assert np.array_equal(r1.ids, r2.ids)
+        mass = np.exp(r2.log_router[np.arange(cfg.M)[:, None], r2.groups]).sum(axis=1)
+        np.testing.assert_allclose(r2.logprobs, r1.logprobs - np.log(mass)[:, None], atol=1e-12)
+
     def p10():
         W1 = synth._normal_bf16(np.random.default_rng(5), cfg.H, cfg.H, 0.2)
         r = orc.draft(W, gm, Wg, h, 2, 5, W1=W1, want_logits=False, lib_path=lib_path)
@@ -98,7 +109,7 @@ def _battery(lib_path):
         g = (a / (1.0 + np.exp(-a)) + _f64(h)) @ _f64(Wg).T
         np.testing.assert_allclose(r.gate, g, atol=1e-12)
 
-    for name, fn in [("p1", p1), ("p3", p3), ("p4", p4), ("p6", p6), ("p10", p10)]:
+    for name, fn in [("p1", p1), ("p3", p3), ("p4", p4), ("p6", p6), ("p6r", p6r), ("p10", p10)]:
         check(name, fn)
     return failed
 

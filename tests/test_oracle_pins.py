@@ -229,6 +229,30 @@ def test_p6_factorised_partial_selection_mass_is_router_mass():
         np.testing.assert_allclose(r.logprobs[m], flat[order], atol=1e-13)
 
 
+def test_p6_renormalised_router_mass_is_one_over_the_active_vocabulary():
+    """Eq. 8 with p_router renormalised over the selected groups (the paper is silent on this): the active
+    vocabulary then carries probability 1, every log-probability moves by the same per-row constant
+    -log(selected router mass), so ids are those of Eq. 8; with every group selected it is Eq. 8 itself."""
+    W, gm, Wg, h = synth.make_all(TINY)
+    r1 = orc.draft(W, gm, Wg, h, 4, 10, factorised=1)
+    r2 = orc.draft(W, gm, Wg, h, 4, 10, factorised=2)
+    rows = np.arange(TINY.M)[:, None]
+    sel_lr = r2.log_router[rows, r2.groups]
+    renorm = sel_lr - logsumexp(sel_lr, axis=1)[:, None]                 # log of p_router / selected mass
+    full = renorm[:, :, None] + r2.logits - r2.group_lse[:, :, None]
+    np.testing.assert_allclose(np.exp(full).sum(axis=(1, 2)), 1.0, atol=1e-12)
+    assert np.array_equal(r1.ids, r2.ids)
+    np.testing.assert_allclose(r2.logprobs, r1.logprobs - logsumexp(sel_lr, axis=1)[:, None], atol=1e-12)
+    for m in range(TINY.M):
+        flat = full[m].ravel()
+        order = np.lexsort((r2.logit_tokens[m].ravel(), -flat))[:10]
+        np.testing.assert_allclose(r2.logprobs[m], flat[order], atol=1e-13)
+    ra = orc.draft(W, gm, Wg, h, TINY.N, 10, factorised=1)
+    rb = orc.draft(W, gm, Wg, h, TINY.N, 10, factorised=2)
+    assert np.array_equal(ra.ids, rb.ids)
+    np.testing.assert_allclose(ra.logprobs, rb.logprobs, atol=1e-12)
+
+
 # ---------------------------------------------------------------- P7
 def test_p7_group_relabelling_invariance():
     W, gm, Wg, h = synth.make_all(TINY)
