@@ -499,6 +499,19 @@ def main():
         ms_w, _, _, _, _ = time_steps(cfg.M, cfg.k_groups, extra_steps, 3, my_batches, cold=False)
         out["warm_l2_us_per_step"] = float(np.mean(ms_w)) * 1e3
         out["other_M"] = [timed_case(head, cfg, M, cfg.k_groups, extra_steps) for M in (1, 60)]
+        # the paper's two-layer router (Eq. 7: scores = W2 (act(W1 h) + h)): W1 is H x H, 33.5 MB more to read per call
+        W1d = dev_bf16(synth._normal_bf16(np.random.default_rng([cfg.seed, 91]), cfg.H, cfg.H, 0.01))
+        lmhead.coral_lmhead_set_router_mlp(head.handle, W1d)
+        eq7 = []
+        for M7 in (1, 8, 60):
+            ms7, _, t7, _, _ = time_steps(M7, cfg.k_groups, min(extra_steps, 30), 3, my_batches)
+            b7 = float(np.mean([algorithmic_bytes(cfg.with_(M=M7), u, M7) for u in t7])) + 2.0 * cfg.H * cfg.H
+            eq7.append({"M": M7, "us_per_step": float(np.mean(ms7)) * 1e3, "groups_touched_mean": float(np.mean(t7)),
+                        "algorithmic_bytes_with_W1": b7, "GBps": b7 / (float(np.mean(ms7)) * 1e-3) / 1e9,
+                        "hbm_frac": b7 / (float(np.mean(ms7)) * 1e-3) / 1e9 / peak})
+        lmhead.coral_lmhead_set_router_mlp(head.handle, None)
+        out["eq7_two_layer_router"] = eq7
+        del W1d
         # extra (not a workload of the list): rows correlated like tree siblings of one parent, where the union
         # of selected groups no longer saturates (Appendix B: the worst case is unlikely in practice)
         ms_c, _, t_c, _, _ = time_steps(60, cfg.k_groups, extra_steps, 3, my_batches, rho=0.3)

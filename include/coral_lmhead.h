@@ -58,6 +58,7 @@ extern "C" {
 /* Output modes (coral_lmhead_set_output_mode). */
 #define CORAL_OUTPUT_JOINT 0       /* log-softmax over all active logits of the row (default) */
 #define CORAL_OUTPUT_FACTORISED 1  /* Eq. 8: log p_router(n) + log p_group(x), p_router = Softmax over all N groups */
+#define CORAL_OUTPUT_FACTORISED_RENORM 2 /* Eq. 8 with p_router renormalised over the row's selected groups */
 
 typedef struct coral_lmhead_s *coral_lmhead_handle;
 
@@ -197,7 +198,10 @@ int coral_lmhead_merge_partials(const void *records_dev, int world, int M, int k
  * (Eq. 7) and p_group the softmax inside group n, independent of the other groups; candidates are ranked by
  * that log-probability (equal -> lower token id).  The emitted log-probabilities of a row sum, over its active
  * vocabulary, to the router mass of its selected groups.  out_lse_dev keeps reporting the joint log-sum-exp.
- * Not available on CORAL_PATH_SIMT_PLAIN (the draft call then returns CORAL_ERR_INVALID).
+ * CORAL_OUTPUT_FACTORISED_RENORM divides p_router by the router mass of the row's selected groups (the paper
+ * does not say whether it does), so that the active vocabulary carries probability 1; the ranking is the same,
+ * every log-probability of a row moves by one constant.
+ * Neither is available on CORAL_PATH_SIMT_PLAIN (the draft call then returns CORAL_ERR_INVALID).
  */
 int coral_lmhead_set_output_mode(coral_lmhead_handle h, int mode);
 

@@ -529,9 +529,11 @@ static int draft_impl(coral_lmhead_handle h, const void* hidden_dev, int M, int 
     CallView c = make_view(h, hidden_dev, M, k_groups, k_tokens);
     int path = choose_path(h, M, k_groups);
     if (path == 0) return CORAL_ERR_INVALID;   // the forced path does not support this call
-    if (h->out_mode == CORAL_OUTPUT_FACTORISED && path == CORAL_PATH_SIMT_PLAIN) return CORAL_ERR_INVALID;
+    if (h->out_mode != CORAL_OUTPUT_JOINT && path == CORAL_PATH_SIMT_PLAIN) return CORAL_ERR_INVALID;
     if (partial_dev && (path == CORAL_PATH_SIMT_PLAIN || h->out_mode != CORAL_OUTPUT_JOINT)) return CORAL_ERR_INVALID;
-    const int merge_mode = partial_dev ? kMergePartial : h->out_mode == CORAL_OUTPUT_FACTORISED ? kMergeFactorised : kMergeJoint;
+    const int merge_mode = partial_dev ? kMergePartial
+                           : h->out_mode == CORAL_OUTPUT_FACTORISED ? kMergeFactorised
+                           : h->out_mode == CORAL_OUTPUT_FACTORISED_RENORM ? kMergeFactorisedRenorm : kMergeJoint;
     float* merge_out = partial_dev ? partial_dev : out_logprobs_dev;
     // adaptive: both fast paths can take the call and the band-ticket router (which makes the choice) runs it
     const bool adaptive = h->forced_path == CORAL_PATH_ADAPTIVE && !h->w1 && M > kRouteFusedMaxM && M <= kRouteMidMaxM &&
@@ -889,7 +891,7 @@ int coral_lmhead_selftest_wait_expiry(coral_lmhead_handle h, void* stream) {
 }
 
 int coral_lmhead_set_output_mode(coral_lmhead_handle h, int mode) {
-    if (!h || (mode != CORAL_OUTPUT_JOINT && mode != CORAL_OUTPUT_FACTORISED)) return CORAL_ERR_INVALID;
+    if (!h || mode < CORAL_OUTPUT_JOINT || mode > CORAL_OUTPUT_FACTORISED_RENORM) return CORAL_ERR_INVALID;
     h->out_mode = mode;
     return CORAL_OK;
 }

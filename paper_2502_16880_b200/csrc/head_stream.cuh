@@ -446,7 +446,7 @@ __global__ void __launch_bounds__(kStreamThreads, 1) head_stream_kernel(CallView
 // exp(z - max), the k_tokens best raw logits (descending), their token ids - over the groups this GPU
 // computed, written to `out_logprobs` (as a [M][2 + 2 k_tokens] word array); slots whose group belongs to
 // another GPU have descriptor -1 and no pieces.  merge_partials_kernel combines the GPUs' records.
-constexpr int kMergeJoint = 0, kMergeFactorised = 1, kMergePartial = 2;
+constexpr int kMergeJoint = 0, kMergeFactorised = 1, kMergePartial = 2, kMergeFactorisedRenorm = 3;
 constexpr int kMergeStreamThreads = 256;
 constexpr int kMergeMaxPieces = 2048;         // >= grid + 2 * k_groups for every supported shape
 constexpr int kMergeRankMax = 256;            // survivors ranked by counting; more fall back to k rounds
@@ -467,7 +467,8 @@ __global__ void __launch_bounds__(kMergeStreamThreads) merge_stream_kernel(CallV
     const int m = blockIdx.x;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     constexpr int kWarps = kMergeStreamThreads / 32;
-    const bool factorised = mode == kMergeFactorised, partial = mode == kMergePartial;
+    const bool renorm = mode == kMergeFactorisedRenorm;      // p_router over the row's selected groups only
+    const bool factorised = mode == kMergeFactorised || renorm, partial = mode == kMergePartial;
     float* rec = partial ? out_logprobs + (size_t)m * (2 + 2 * c.k_tokens) : nullptr;
     __shared__ float s_f[kWarps], s_t[kWarps];
     __shared__ float s_lse, s_glse, s_thr2;
@@ -499,15 +500,18 @@ __global__ void __launch_bounds__(kMergeStreamThreads) merge_stream_kernel(CallV
         s_off[s] = factorised ? c.gate[(size_t)m * c.N + c.sel[(size_t)m * c.k_groups + s]] : 0.f;
     }
     if (threadIdx.x == 0) { s_n = 0; s_nlive = 0; s_thr2 = kNegInf; }
-    if (factorised) {                 // log-sum-exp of the row's N gate scores (kMergeStreamThreads >= N)
-        const float gv = threadIdx.x < c.N ? c.gate[(size_t)m * c.N + threadIdx.x] : kNegInf;
+    if (factorised) {                 // log-sum-exp of the row's N gate scores (kMergeStreamThreads >= N), or of
+                                      // the k_groups selected ones in the renormalised variant
+        const bool mine = renorm ? threadIdx.x < c.k_groups : threadIdx.x < c.N;
+        const float gv = !mine ? kNegInf
+                         : c.gate[(size_t)m * c.N + (renorm ? c.sel[(size_t)m * c.k_groups + threadIdx.x] : (int)threadIdx.x)];
         const float wm = warp_max(gv);
         if (lane == 0) s_f[warp] = wm;
         __syncthreads();
         float gm = s_f[0];
 #pragma unroll
         for (int w = 1; w < kWarps; ++w) gm = fmaxf(gm, s_f[w]);
-        const float ws = warp_sum(threadIdx.x < c.N ? expf(gv - gm) : 0.f);
+        const float ws = warp_sum(mine ? expf(gv - gm) : 0.f);
         if (lane == 0) s_t[warp] = ws;
         __syncthreads();
         if (threadIdx.x == 0) {

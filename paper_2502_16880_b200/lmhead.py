@@ -27,7 +27,7 @@ CORAL_ERR_BOUNDS = -6
 CORAL_ERR_TOO_LARGE = -7
 CORAL_ERR_NONFINITE = -8
 CORAL_ROUTE_STATIC_MAX_ROWS = 64
-CORAL_OUTPUT_JOINT, CORAL_OUTPUT_FACTORISED = 0, 1
+CORAL_OUTPUT_JOINT, CORAL_OUTPUT_FACTORISED, CORAL_OUTPUT_FACTORISED_RENORM = 0, 1, 2
 CORAL_PATH_AUTO, CORAL_PATH_STREAM, CORAL_PATH_TCGEN05, CORAL_PATH_SIMT_PLAIN, CORAL_PATH_ADAPTIVE = 0, 1, 2, 3, 4
 
 

@@ -104,6 +104,9 @@ def compare(W, gm, Wg, hidden_bits, k_groups, k_tokens, gpu, forced_groups=None,
         # log p_router(group) + z - LSE(group)
         if factorised:
             score = ref.log_router[m, ref.groups[m]][:, None] + ref.logits[m] - ref.group_lse[m][:, None]
+            if int(factorised) == 2:      # p_router renormalised over the row's selected groups
+                sel_lr = ref.log_router[m, ref.groups[m]]
+                score = score - (sel_lr.max() + np.log(np.exp(sel_lr - sel_lr.max()).sum()))
         else:
             score = ref.logits[m] - ref.lse[m]
         # score of a token id by binary search in the row's sorted active token list (all rows at full size

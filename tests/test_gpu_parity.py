@@ -296,6 +296,12 @@ def test_factorised_distribution_eq8(path, M, kg):
     rows = np.unique(np.linspace(0, M - 1, 16).astype(int))
     rep = ph.compare(W, gm, Wg, hb[rows], kg, 10, {k: a[rows] for k, a in out.items()}, factorised=True)
     assert rep.ok, rep.errors
+    # the variant with p_router renormalised over the selected groups: same ids, mass 1 over the active vocabulary
+    lmhead.coral_lmhead_set_output_mode(head.handle, lmhead.CORAL_OUTPUT_FACTORISED_RENORM)
+    out2 = ph.gpu_draft_numpy(head, hb, kg, 10)
+    assert head.status() == 0
+    rep = ph.compare(W, gm, Wg, hb[rows], kg, 10, {k: a[rows] for k, a in out2.items()}, factorised=2)
+    assert rep.ok, rep.errors
     # back to the joint mode on the same handle
     lmhead.coral_lmhead_set_output_mode(head.handle, lmhead.CORAL_OUTPUT_JOINT)
     out = ph.gpu_draft_numpy(head, hb, kg, 10)
@@ -325,6 +331,29 @@ def test_two_layer_router_eq7(M):
     rep = ph.compare(W, gm, Wg, hb, 4, 10, out)
     assert rep.ok, rep.errors
     head.close()
+
+
+@pytest.mark.parametrize("M", [1, 8, 60])
+def test_two_layer_router_eq7_on_the_llama3_shape(M):
+    """Eq. 7's router at H = 4096 (W1 is 4096 x 4096, 33.5 MB more to read per call): gate scores, groups and the
+    Eq. 8 distribution of every row against the oracle."""
+    cfg, W, gm, Wg, head = _weights("llama3_8b")
+    W1 = synth._normal_bf16(np.random.default_rng(23), cfg.H, cfg.H, 0.01)
+    hb = synth.make_hidden(cfg, M)
+    head.set_path(lmhead.CORAL_PATH_AUTO)
+    lmhead.coral_lmhead_set_router_mlp(head.handle, ph.to_dev_bf16(W1))
+    try:
+        for mode in (lmhead.CORAL_OUTPUT_JOINT, lmhead.CORAL_OUTPUT_FACTORISED):
+            lmhead.coral_lmhead_set_output_mode(head.handle, mode)
+            out = ph.gpu_draft_numpy(head, hb, cfg.k_groups, cfg.k_tokens)
+            assert head.status() == 0
+            rows = np.arange(M) if M <= 8 else np.unique(np.linspace(0, M - 1, 12).astype(int))
+            rep = ph.compare(W, gm, Wg, hb[rows], cfg.k_groups, cfg.k_tokens, {k: a[rows] for k, a in out.items()},
+                             W1=W1, factorised=mode)
+            assert rep.ok, rep.errors
+    finally:
+        lmhead.coral_lmhead_set_router_mlp(head.handle, None)
+        lmhead.coral_lmhead_set_output_mode(head.handle, lmhead.CORAL_OUTPUT_JOINT)
 
 
 @pytest.mark.parametrize("M,path", [(8, lmhead.CORAL_PATH_STREAM), (60, lmhead.CORAL_PATH_STREAM),
