@@ -88,9 +88,9 @@ size_t stream_smem_bytes(const StreamGeom& g) {
 }
 
 constexpr int kTcMinRows = 96;          // above this many rows the tensor-core path is the faster one (measured, iid rows)
-constexpr int kTcMinRowsPerGroup = 8;   // ... and from this many rows per group on average (the streaming path reads a
-                                        // group once per 16 rows; measured on the three paper shapes: equal at 7.5, 1.15x-2x
-                                        // faster from 12 on)
+constexpr int kTcMinRowsPerGroup = 10;  // ... and from this many rows per group on average (the streaming path reads a
+                                        // group once per 16 rows; measured on the three paper shapes: within 10 % either
+                                        // way at 7.5-8, 1.15x-2x faster from 12 on)
 constexpr int kTcProvisionRows = 32;    // handles for more rows get the tensor-core workspace (adaptive calls use it from 33 rows)
 constexpr int kMergeSmemCands = 4096;   // candidates the streaming merge keeps in shared memory
 
@@ -552,10 +552,21 @@ static int draft_impl(coral_lmhead_handle h, const void* hidden_dev, int M, int 
 
     if (h->timing) cudaEventRecord(h->ev_begin, st);
     if (h->w1) {
-        router_hidden_kernel<<<dim3((cfg.H + kGateTile - 1) / kGateTile, (M + kGateTile - 1) / kGateTile), 256, 0, st>>>(
-            c, h->w1, h->router_u);
+        if (cfg.H % 32 == 0)
+            router_hidden_mma_kernel<<<(cfg.H + 15) / 16, 256, 0, st>>>(c, h->w1, h->router_u);
+        else
+            router_hidden_kernel<<<dim3((cfg.H + kGateTile - 1) / kGateTile, (M + kGateTile - 1) / kGateTile), 256, 0, st>>>(
+                c, h->w1, h->router_u);
         ++launches;
-        gate_f32_kernel<<<dim3(c.N, (M + kGateRows - 1) / kGateRows), kGateThreads, 0, st>>>(c, out_gate_dev);
+    }
+    if (h->w1 && M <= kRouteFusedMaxM) {
+        // scores, selection and bucketing in one launch, reading the fp32 router input
+        launch_pdl(route_fused_kernel, dim3(c.N), dim3(kRouteThreads), (size_t)0, st, c, forced_groups_dev, out_groups_dev,
+                   out_gate_dev);
+        ++launches;
+    } else if (h->w1) {
+        launch_pdl(gate_f32_kernel, dim3(c.N, (M + kGateRows - 1) / kGateRows), dim3(kGateThreads), (size_t)0, st, c,
+                   out_gate_dev);
         ++launches;
         select_kernel<<<(M + kSelectWarps - 1) / kSelectWarps, kSelectWarps * 32, 0, st>>>(c, forced_groups_dev,
                                                                                           out_groups_dev);

@@ -194,6 +194,7 @@ __global__ void __launch_bounds__(kRouteThreads)
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     constexpr int kWarps = kRouteThreads / 32;
     const int chunks = c.H >> 3;
+    pdl_wait();                   // with the two-layer router this grid follows the kernel that writes router_in
     pdl_launch_dependents();      // the next kernel may set itself up; it waits for this grid before reading
 
     {
@@ -205,6 +206,24 @@ __global__ void __launch_bounds__(kRouteThreads)
             float acc[8];
 #pragma unroll
             for (int r = 0; r < 8; ++r) acc[r] = 0.f;
+            if (c.router_in) {             // Eq. 7: the gate reads act(W1 h) + h, kept in fp32
+                for (int ch = threadIdx.x; ch < chunks; ch += kRouteThreads) {
+                    const uint4 q = __ldg(wg + ch);
+                    const float w[8] = {bf16_lo(q.x), bf16_hi(q.x), bf16_lo(q.y), bf16_hi(q.y),
+                                        bf16_lo(q.z), bf16_hi(q.z), bf16_lo(q.w), bf16_hi(q.w)};
+#pragma unroll
+                    for (int r = 0; r < 8; ++r) {
+                        if (r < rows) {
+                            const float4* up = reinterpret_cast<const float4*>(c.router_in + (size_t)(m0 + r) * c.H) + 2 * ch;
+                            const float4 a = __ldcg(up), b = __ldcg(up + 1);
+                            acc[r] = fmaf(w[0], a.x, acc[r]); acc[r] = fmaf(w[1], a.y, acc[r]);
+                            acc[r] = fmaf(w[2], a.z, acc[r]); acc[r] = fmaf(w[3], a.w, acc[r]);
+                            acc[r] = fmaf(w[4], b.x, acc[r]); acc[r] = fmaf(w[5], b.y, acc[r]);
+                            acc[r] = fmaf(w[6], b.z, acc[r]); acc[r] = fmaf(w[7], b.w, acc[r]);
+                        }
+                    }
+                }
+            } else
             for (int ch = threadIdx.x; ch < chunks; ch += kRouteThreads) {
                 const uint4 w = __ldg(wg + ch);
                 uint4 hv[8];                       // all loads first, so they are in flight together
@@ -692,12 +711,87 @@ __global__ void __launch_bounds__(256) router_hidden_kernel(CallView c, const ui
     }
 }
 
+// The same on the warp-level tensor cores (H a multiple of 32): a block owns 16 columns i of u (16 rows of W1) and
+// walks over the query rows 32 at a time (four n-tiles sharing every load of W1), its 8 warps splitting H in
+// blocks of 32 columns (mma.sync m16n8k16, bf16 x bf16 -> fp32; W1 rows on the M axis, query rows on N, the same
+// column permutation in both operands).  The block's 128 KiB of W1 come from HBM once and from L1/L2 for the
+// further row tiles.  grid H / 16.
+constexpr int kRouterHiddenNT = 4;
+__global__ void __launch_bounds__(256) router_hidden_mma_kernel(CallView c, const uint16_t* __restrict__ W1,
+                                                                float* __restrict__ u) {
+    __shared__ float s_part[8][kRouterHiddenNT * 16 * 8];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int gq = lane >> 2, tq = lane & 3;
+    const int i0 = blockIdx.x * 16;
+    pdl_launch_dependents();
+    const bool a_lo = i0 + gq < c.H, a_hi = i0 + gq + 8 < c.H;
+    const uint16_t* wlo = W1 + (size_t)(a_lo ? i0 + gq : 0) * c.H + tq * 8;
+    const uint16_t* whi = W1 + (size_t)(a_hi ? i0 + gq + 8 : 0) * c.H + tq * 8;
+    const int kblocks = c.H >> 5;
+    const uint4 zero = make_uint4(0, 0, 0, 0);
+    for (int m0 = 0; m0 < c.M; m0 += 8 * kRouterHiddenNT) {
+        const uint16_t* hb[kRouterHiddenNT];
+        bool b_ok[kRouterHiddenNT];
+#pragma unroll
+        for (int t = 0; t < kRouterHiddenNT; ++t) {
+            b_ok[t] = m0 + t * 8 + gq < c.M;
+            hb[t] = c.hidden + (size_t)(b_ok[t] ? m0 + t * 8 + gq : 0) * c.H + tq * 8;
+        }
+        float acc[kRouterHiddenNT][2][4];
+#pragma unroll
+        for (int t = 0; t < kRouterHiddenNT; ++t)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) { acc[t][0][e] = 0.f; acc[t][1][e] = 0.f; }
+#pragma unroll 2
+        for (int kb = warp; kb < kblocks; kb += 8) {
+            const uint4 a = a_lo ? __ldg(reinterpret_cast<const uint4*>(wlo + kb * 32)) : zero;
+            const uint4 b = a_hi ? __ldg(reinterpret_cast<const uint4*>(whi + kb * 32)) : zero;
+            uint4 h[kRouterHiddenNT];
+#pragma unroll
+            for (int t = 0; t < kRouterHiddenNT; ++t)
+                h[t] = b_ok[t] ? __ldg(reinterpret_cast<const uint4*>(hb[t] + kb * 32)) : zero;
+#pragma unroll
+            for (int t = 0; t < kRouterHiddenNT; ++t) {
+                asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+                             : "+f"(acc[t][0][0]), "+f"(acc[t][0][1]), "+f"(acc[t][0][2]), "+f"(acc[t][0][3])
+                             : "r"(a.x), "r"(b.x), "r"(a.y), "r"(b.y), "r"(h[t].x), "r"(h[t].y));
+                asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+                             : "+f"(acc[t][1][0]), "+f"(acc[t][1][1]), "+f"(acc[t][1][2]), "+f"(acc[t][1][3])
+                             : "r"(a.z), "r"(b.z), "r"(a.w), "r"(b.w), "r"(h[t].z), "r"(h[t].w));
+            }
+        }
+        // accumulator layout: [0],[1] = W1 row gq, query rows 2*tq, 2*tq+1 of the n-tile; [2],[3] = W1 row gq + 8
+        float* sp = s_part[warp];
+#pragma unroll
+        for (int t = 0; t < kRouterHiddenNT; ++t) {
+            sp[t * 128 + gq * 8 + 2 * tq] = acc[t][0][0] + acc[t][1][0];
+            sp[t * 128 + gq * 8 + 2 * tq + 1] = acc[t][0][1] + acc[t][1][1];
+            sp[t * 128 + (gq + 8) * 8 + 2 * tq] = acc[t][0][2] + acc[t][1][2];
+            sp[t * 128 + (gq + 8) * 8 + 2 * tq + 1] = acc[t][0][3] + acc[t][1][3];
+        }
+        __syncthreads();
+        for (int e = threadIdx.x; e < kRouterHiddenNT * 128; e += 256) {
+            const int t = e >> 7, g = (e >> 3) & 15, r = e & 7;
+            const int m = m0 + t * 8 + r;
+            if (i0 + g < c.H && m < c.M) {
+                float a = 0.f;
+#pragma unroll
+                for (int w = 0; w < 8; ++w) a += s_part[w][e];
+                const float hv = __uint_as_float((uint32_t)c.hidden[(size_t)m * c.H + i0 + g] << 16);
+                u[(size_t)m * c.H + i0 + g] = a / (1.f + expf(-a)) + hv;
+            }
+        }
+        __syncthreads();
+    }
+}
+
 // g[m][n] = W_gate[n] . u[m] with u in fp32.  grid (N, ceil(M/8)); block (0,0) clears the per-group counters.
 __global__ void __launch_bounds__(kGateThreads) gate_f32_kernel(CallView c, float* __restrict__ gate_tap) {
     const int n = blockIdx.x;
     const int m0 = blockIdx.y * kGateRows;
     const int rows = min(kGateRows, c.M - m0);
     const int chunks = c.H >> 3;
+    pdl_wait();                   // router_in is complete from here on
     if (blockIdx.x == 0 && blockIdx.y == 0)
         for (int t = threadIdx.x; t < c.N; t += kGateThreads) c.group_count[t] = 0;
     const uint4* __restrict__ wg = reinterpret_cast<const uint4*>(c.w_gate + (size_t)n * c.H);
