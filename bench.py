@@ -625,6 +625,21 @@ def main():
             "tensor_frac_ceiling_at_hbm_roofline": flops / (st_big.weight_bytes / (peak * 1e9)) / 1e12 / tf_sust,
             "torch_dense_gemm_960xVxH_us": float(np.mean(tg)) * 1e3,
         }
+        # what issuing the tensor-core path's MMAs costs by itself (tcgen05.mma of a CTA pair, 256 x n x 16, four
+        # per commit as in the kernel's 64-column step, nothing loaded): ns per MMA for one and two issuing
+        # threads, next to the time the tensor pipe needs at its nominal rate
+        ns_out = torch.zeros(2, dtype=torch.int64, device=dev)
+        issue = []
+        for n_i, iss in ((32, 1), (128, 1), (256, 1), (32, 2), (128, 2), (256, 2)):
+            for _ in range(2):
+                lmhead.coral_lmhead_tc_issue_probe(big.handle, n_i, 4, iss, 2000, ns_out, stream)
+                torch.cuda.synchronize()
+            t_issue, t_done = [float(x) for x in ns_out.cpu().tolist()]
+            issue.append({"n": n_i, "issuers": iss, "mmas_per_commit": 4,
+                          "ns_per_round_of_one_issuer": t_issue / 2000.0, "ns_per_mma_over_all_issuers": t_done / 2000.0 / 4 / iss,
+                          "ns_per_mma_at_nominal_tensor_rate": 128.0 * n_i * 16 / 4096.0 / 1.965})
+        out["tc_issue_probe"] = issue
+        assert big.status() == 0
         big.close()
         # supplementary points with more rows per group (240 and 480): the same path above the machine ridge
         supp = []

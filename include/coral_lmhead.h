@@ -291,6 +291,18 @@ int coral_lmhead_selftest_wait_expiry(coral_lmhead_handle h, void *stream);
 int coral_lmhead_copy_floor(coral_lmhead_handle h, long long bytes, int in_flight, int repeats, void *stream);
 
 /*
+ * Bench-side measurement aid with no counterpart in the paper (not part of the draft step): what issuing the
+ * tensor-core path's MMAs costs by itself.  Every CTA pair of the tensor-core kernel's grid runs `rounds` rounds
+ * of `per_commit` (1..16) tcgen05.mma of 256 x n x 16 (n a multiple of 16 in [16, 256]; the instruction forms of
+ * the tensor-core path) on zeroed shared memory followed by one tcgen05.commit, from `issuers` (1 or 2) threads;
+ * nothing is loaded.  out_ns_dev[0] receives the nanoseconds the first pair's first issuer needed to issue its
+ * rounds, out_ns_dev[1] until its last MMA had completed (device memory, two 64-bit words).  Needs a handle created
+ * with max_M > 32 (CORAL_ERR_INVALID otherwise); asynchronous, no allocation; every wait is bounded.
+ */
+int coral_lmhead_tc_issue_probe(coral_lmhead_handle h, int n, int per_commit, int issuers, int rounds,
+                                unsigned long long *out_ns_dev, void *stream);
+
+/*
  * Measurement aid for the dominant kernel (the one that streams the selected
  * groups' weights; Section 3.3 names the LM head as the drafter's main cost).
  * With timing on, every draft call records a CUDA event before and after that

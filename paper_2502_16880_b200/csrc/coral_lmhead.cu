@@ -12,6 +12,7 @@
 #include "head_stream.cuh"
 #include "head_tc.cuh"
 #include "copy_probe.cuh"
+#include "tc_probe.cuh"
 #include "csra.cuh"
 #include "merge.cuh"
 #include "route.cuh"
@@ -797,6 +798,31 @@ int coral_lmhead_copy_floor(coral_lmhead_handle h, long long bytes, int in_fligh
         h->packed, bytes / kCopyChunk, in_flight, repeats, reinterpret_cast<DeviceState*>(h->ws + h->L.state),
         reinterpret_cast<unsigned*>(h->ws + h->L.cand_val));
     return cudaGetLastError() == cudaSuccess ? CORAL_OK : CORAL_ERR_CUDA;
+}
+
+int coral_lmhead_tc_issue_probe(coral_lmhead_handle h, int n, int per_commit, int issuers, int rounds,
+                                unsigned long long* out_ns_dev, void* stream) {
+    if (!h || !out_ns_dev || !h->tc_ok) return CORAL_ERR_INVALID;
+    if (n < 16 || n > 256 || n % 16 || per_commit < 1 || per_commit > 16 || issuers < 1 || issuers > 2 || rounds < 1 ||
+        rounds > (1 << 16))
+        return CORAL_ERR_INVALID;
+    const size_t smem = 1024 + kTcProbeOperandBytes + 256;
+    if (cudaFuncSetAttribute(tc_issue_probe_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+        return CORAL_ERR_CUDA;
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(2 * h->tc_pairs);
+    cfg.blockDim = dim3(128);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = static_cast<cudaStream_t>(stream);
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, tc_issue_probe_kernel, n, per_commit, rounds, issuers, out_ns_dev,
+                              reinterpret_cast<DeviceState*>(h->ws + h->L.state)) == cudaSuccess ? CORAL_OK : CORAL_ERR_CUDA;
 }
 
 // ---- CSRA objective (Eq. 2) -------------------------------------------------------------------------------

@@ -59,6 +59,7 @@ _SIGNATURES = {
     "coral_lmhead_draft_partial": (_i, [_vp, _vp, _i, _i, _i, _vp, _vp]),
     "coral_lmhead_merge_partials": (_i, [_vp, _i, _i, _i, _vp, _vp, _vp]),
     "coral_lmhead_copy_floor": (_i, [_vp, ctypes.c_longlong, _i, _i, _vp]),
+    "coral_lmhead_tc_issue_probe": (_i, [_vp, _i, _i, _i, _i, _vp, _vp]),
     "coral_lmhead_set_hot_groups": (_i, [_vp, _i]),
     "coral_csra_workspace_bytes": (_i, [_i, _i, _i, ctypes.POINTER(ctypes.c_size_t)]),
     "coral_csra_infonce": (_i, [_vp, _vp, _i, _i, _i, ctypes.c_float, _vp, _vp, _vp, _vp, _vp]),
@@ -247,6 +248,13 @@ def coral_lmhead_copy_floor(handle, nbytes: int, stream=None, in_flight: int = 0
     `in_flight` 16 KiB copies outstanding per SM (0 = default); time it with events."""
     _check(load_library().coral_lmhead_copy_floor(handle, int(nbytes), int(in_flight), int(repeats),
                                                   _stream_ptr(stream)), "coral_lmhead_copy_floor")
+
+
+def coral_lmhead_tc_issue_probe(handle, n: int, per_commit: int, issuers: int, rounds: int, out_ns, stream=None) -> None:
+    """out_ns: CUDA int64 tensor of two words (issue time, completion time in ns of the first pair's first issuer)."""
+    _check(load_library().coral_lmhead_tc_issue_probe(handle, int(n), int(per_commit), int(issuers), int(rounds),
+                                                      _dev_ptr(out_ns, torch.int64, allow_none=False),
+                                                      _stream_ptr(stream)), "coral_lmhead_tc_issue_probe")
 
 
 def coral_csra_workspace_bytes(n: int, views: int, D: int) -> int:

@@ -1,4 +1,6 @@
 """GPU parity: the CUDA path through the C ABI against the CPU oracle."""
+import ctypes
+
 import numpy as np
 import pytest
 import torch
@@ -445,6 +447,29 @@ def test_copy_floor_probe_runs_and_checks_arguments():
     assert lib.coral_lmhead_copy_floor(head.handle, packed_bytes + 16384, 0, 1, None) == lmhead.CORAL_ERR_INVALID
     assert lib.coral_lmhead_copy_floor(head.handle, packed_bytes, 14, 1, None) == lmhead.CORAL_ERR_INVALID
     assert lib.coral_lmhead_copy_floor(head.handle, packed_bytes, 8, 0, None) == lmhead.CORAL_ERR_INVALID
+    head.close()
+
+
+def test_tensor_core_issue_probe_runs_and_checks_arguments():
+    cfg = synth.HeadConfig("probe", H=256, V=256 * 16, N=16, k_groups=4, k_tokens=10, M=64, seed=3)
+    W, gm, Wg, hb = synth.make_all(cfg)
+    head = _head(cfg, W, gm, Wg, max_M=64, max_kg=4, max_kt=10)
+    lib = lmhead.load_library()
+    out = torch.zeros(2, dtype=torch.int64, device="cuda")
+    for n, iss in ((16, 1), (128, 2), (256, 1)):
+        lmhead.coral_lmhead_tc_issue_probe(head.handle, n, 4, iss, 200, out)
+        torch.cuda.synchronize()
+        t_issue, t_done = out.cpu().tolist()
+        assert 0 < t_issue <= t_done < 10_000_000
+    assert head.status() == 0
+    p = ctypes.c_void_p(out.data_ptr())
+    assert lib.coral_lmhead_tc_issue_probe(head.handle, 24, 4, 1, 10, p, None) == lmhead.CORAL_ERR_INVALID
+    assert lib.coral_lmhead_tc_issue_probe(head.handle, 128, 0, 1, 10, p, None) == lmhead.CORAL_ERR_INVALID
+    assert lib.coral_lmhead_tc_issue_probe(head.handle, 128, 4, 3, 10, p, None) == lmhead.CORAL_ERR_INVALID
+    assert lib.coral_lmhead_tc_issue_probe(head.handle, 128, 4, 1, 10, None, None) == lmhead.CORAL_ERR_INVALID
+    out2 = ph.gpu_draft_numpy(head, hb, 4, 10)                   # the handle still drafts correctly afterwards
+    rep = ph.compare(W, gm, Wg, hb[:8], 4, 10, {k: a[:8] for k, a in out2.items()})
+    assert rep.ok, rep.errors
     head.close()
 
 
