@@ -29,7 +29,7 @@ inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 struct Layout {
     size_t w_gate, group_tokens, state, gate, sel, slot_of, group_count, group_offset, bucket_row, bucket_slot,
         slot_desc, union_list, union_rank, part_max, part_sum, part_val, part_id, sp_max, sp_sum, sp_val, sp_id,
-        cand_val, cand_id, route_mid, tc_hg, tc_max, tc_sum, tc_val, tc_id, stage_hidden, stage_ids, stage_logprobs, total;
+        cand_val, cand_id, route_mid, route_part, tc_hg, tc_max, tc_sum, tc_val, tc_id, stage_hidden, stage_ids, stage_logprobs, total;
     size_t packed_bytes, cand_cap, cand_rows;
     int v, T;
     int KB, T16;                 // packed layout (see packed_chunk_offset)
@@ -109,6 +109,7 @@ Layout make_layout(const coral_lmhead_config& c) {
     L.state = take(sizeof(DeviceState));
     L.route_bands = (M + 7) / 8 > (size_t)kRouteMidBands ? (M + 7) / 8 : (size_t)kRouteMidBands;
     L.route_mid = take((L.route_bands + 5 * N) * 4);      // band tickets, 4 mask words and one counter per group
+    L.route_part = take((size_t)kRouteMidBands * kRouteMidSplitMax * ((N + 15) / 16) * 128 * 4);   // partial score tiles when H is split
     L.gate = take(M * N * 4);
     L.sel = take(M * kg * 4);
     L.slot_of = take(M * N * 2);
@@ -580,12 +581,17 @@ static int draft_impl(coral_lmhead_handle h, const void* hidden_dev, int M, int 
         route_fused_kernel<<<c.N, kRouteThreads, 0, st>>>(c, forced_groups_dev, out_groups_dev, out_gate_dev);
         ++launches;
     } else if (M <= kRouteMidMaxM && M * c.N <= kRouteMidMaxCells && cfg.H % 32 == 0) {
-        route_mid_kernel<<<dim3((c.N + 15) / 16, (M + 7) / 8), 256, 0, st>>>(
-            c, forced_groups_dev, out_groups_dev, out_gate_dev, rt_bands, rt_masks, rt_counts, 1);
+        // few tiles: split H over up to four blocks per tile, so that the GPU is filled and every block's loads
+        // are in flight at once
+        const int tiles = ((c.N + 15) / 16) * ((M + 7) / 8);
+        const int split = tiles >= 128 ? 1 : tiles >= 64 ? 2 : kRouteMidSplitMax;
+        route_mid_kernel<<<dim3((c.N + 15) / 16, (M + 7) / 8, split), 256, 0, st>>>(
+            c, forced_groups_dev, out_groups_dev, out_gate_dev, rt_bands, rt_masks, rt_counts, 1,
+            reinterpret_cast<float*>(h->ws + h->L.route_part));
         ++launches;
     } else if (cfg.H % 32 == 0) {
         route_mid_kernel<<<dim3((c.N + 15) / 16, (M + 7) / 8), 256, 0, st>>>(
-            c, forced_groups_dev, out_groups_dev, out_gate_dev, rt_bands, rt_masks, rt_counts, 0);
+            c, forced_groups_dev, out_groups_dev, out_gate_dev, rt_bands, rt_masks, rt_counts, 0, nullptr);
         ++launches;
         launch_pdl(bucket_group_kernel, dim3(c.N), dim3(256), (size_t)0, st, c, rt_counts);
         ++launches;

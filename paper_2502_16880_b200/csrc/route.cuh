@@ -111,7 +111,8 @@ __global__ void __launch_bounds__(kSelectWarps * 32) select_kernel(CallView c, c
 template <int NPER>
 __device__ __forceinline__ void route_select_row(const CallView& c, const int32_t* __restrict__ forced,
                                                  int32_t* __restrict__ groups_tap, int m, int lane, float* s_val,
-                                                 int16_t* s_slot_row, unsigned* s_rowmask, int bit) {
+                                                 int16_t* s_slot_row, unsigned* s_rowmask, int bit,
+                                                 bool from_smem = false) {
     int slot[NPER];
 #pragma unroll
     for (int i = 0; i < NPER; ++i) slot[i] = -1;
@@ -135,7 +136,7 @@ __device__ __forceinline__ void route_select_row(const CallView& c, const int32_
 #pragma unroll
         for (int i = 0; i < NPER; ++i) {
             const int n = lane + 32 * i;
-            val[i] = (n < c.N) ? __ldcg(c.gate + (size_t)m * c.N + n) : kNegInf;
+            val[i] = n >= c.N ? kNegInf : from_smem ? s_val[n] : __ldcg(c.gate + (size_t)m * c.N + n);   // s_val: the row's scores, already there
             if (val[i] != val[i]) {                  // NaN orders against nothing: rank it last and report, so that
                 val[i] = kNegInf;                    // every row still gets exactly k_groups distinct groups
                 set_status(c.state, -8);
@@ -384,8 +385,11 @@ __global__ void __launch_bounds__(256) gate_tile_kernel(CallView c, float* __res
 // Every lane loads 16 bytes of two gate rows and of one hidden row per block of 32 columns; the column order
 // inside a block is permuted the same way for both operands, which leaves the dot products unchanged.
 // H a multiple of 32.
+// With `part` set the block covers only the 32-column blocks [kb_lo, kb_hi) of H (several blocks split H between
+// them) and writes its 16 x 8 partial sums there, element (group g, row r) at part[g * 8 + r]; whoever finishes
+// the band adds the parts up in a fixed order.
 __device__ __forceinline__ void gate_mma_tile(const CallView& c, float* __restrict__ gate_tap, int n0, int m0,
-                                              float (*s_part)[16 * 8]) {
+                                              float (*s_part)[16 * 8], int kb_lo, int kb_hi, float* __restrict__ part) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int gq = lane >> 2, tq = lane & 3;
     const bool a_lo = n0 + gq < c.N, a_hi = n0 + gq + 8 < c.N, b_ok = m0 + gq < c.M;
@@ -393,10 +397,9 @@ __device__ __forceinline__ void gate_mma_tile(const CallView& c, float* __restri
     const uint16_t* whi = c.w_gate + (size_t)(a_hi ? n0 + gq + 8 : 0) * c.H + tq * 8;
     const uint16_t* hb = c.hidden + (size_t)(b_ok ? m0 + gq : 0) * c.H + tq * 8;
     float acc0[4] = {0.f, 0.f, 0.f, 0.f}, acc1[4] = {0.f, 0.f, 0.f, 0.f};
-    const int kblocks = c.H >> 5;
     const uint4 zero = make_uint4(0, 0, 0, 0);
 #pragma unroll 4
-    for (int kb = warp; kb < kblocks; kb += 8) {
+    for (int kb = kb_lo + warp; kb < kb_hi; kb += 8) {
         const uint4 a = a_lo ? __ldg(reinterpret_cast<const uint4*>(wlo + kb * 32)) : zero;
         const uint4 b = a_hi ? __ldg(reinterpret_cast<const uint4*>(whi + kb * 32)) : zero;
         const uint4 h = b_ok ? __ldg(reinterpret_cast<const uint4*>(hb + kb * 32)) : zero;
@@ -420,8 +423,12 @@ __device__ __forceinline__ void gate_mma_tile(const CallView& c, float* __restri
             float sum = 0.f;
 #pragma unroll
             for (int w = 0; w < 8; ++w) sum += s_part[w][threadIdx.x];
-            c.gate[(size_t)(m0 + r) * c.N + n0 + g] = sum;
-            if (gate_tap) gate_tap[(size_t)(m0 + r) * c.N + n0 + g] = sum;
+            if (part) {
+                part[threadIdx.x] = sum;
+            } else {
+                c.gate[(size_t)(m0 + r) * c.N + n0 + g] = sum;
+                if (gate_tap) gate_tap[(size_t)(m0 + r) * c.N + n0 + g] = sum;
+            }
         }
     }
 }
@@ -438,27 +445,33 @@ __device__ __forceinline__ void gate_mma_tile(const CallView& c, float* __restri
 constexpr int kRouteMidMaxM = 128;
 constexpr int kRouteMidBands = kRouteMidMaxM / 8;
 constexpr int kRouteMidMaxCells = 8192;       // M * N slots staged in shared memory by the last block
+constexpr int kRouteMidSplitMax = 4;          // blocks that share one tile's H
 __global__ void __launch_bounds__(256)
     route_mid_kernel(CallView c, const int32_t* __restrict__ forced, int32_t* __restrict__ groups_tap,
                      float* __restrict__ gate_tap, unsigned* __restrict__ band_ticket, unsigned* __restrict__ rowmask,
-                     int* __restrict__ count_acc, int finish) {
+                     int* __restrict__ count_acc, int finish, float* __restrict__ gate_part) {
     __shared__ float s_part[8][16 * 8];
     __shared__ float s_val[8][kMaxGroups];
     __shared__ int16_t s_slot_row[8][kMaxGroups];
     __shared__ unsigned s_mask[kMaxGroups];
-    __shared__ int16_t s_slot[kRouteMidMaxCells];
+    __shared__ int16_t s_slot[kRouteMidMaxCells];      // last finisher: every row's slot of every group
     __shared__ int s_warp_tot[8];
     __shared__ int s_flag;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int m0 = blockIdx.y * 8;
     pdl_launch_dependents();      // the next kernel may set itself up; it waits for this grid before reading
 
-    gate_mma_tile(c, gate_tap, blockIdx.x * 16, m0, s_part);
+    // gridDim.z > 1 (few rows, hence few tiles): the blocks of a tile split H between them, so that every load of
+    // a block is in flight at once, and leave partial sums for the band's finisher
+    const int KS = (int)gridDim.z, kblocks = c.H >> 5;
+    float* part = KS > 1 ? gate_part + ((((size_t)blockIdx.y * gridDim.x + blockIdx.x) * KS + blockIdx.z) << 7) : nullptr;
+    gate_mma_tile(c, gate_tap, blockIdx.x * 16, m0, s_part, (int)((long long)kblocks * blockIdx.z / KS),
+                  (int)((long long)kblocks * (blockIdx.z + 1) / KS), part);
     __threadfence();
     __syncthreads();
     if (threadIdx.x == 0) {
         const unsigned t = atomicAdd(&band_ticket[blockIdx.y], 1u);
-        s_flag = t == gridDim.x - 1;
+        s_flag = t == gridDim.x * gridDim.z - 1;
         if (s_flag) band_ticket[blockIdx.y] = 0;
         __threadfence();
     }
@@ -466,14 +479,30 @@ __global__ void __launch_bounds__(256)
     __syncthreads();
     if (!s_flag) return;
 
-    // this block saw the band's last ticket: every score of rows m0 .. m0 + 7 is published
+    // this block saw the band's last ticket: every score (or partial sum) of rows m0 .. m0 + 7 is published
+    if (KS > 1) {
+        // add the parts of every score in the order of the column ranges: the same sum whoever finishes
+        for (int e = threadIdx.x; e < 8 * c.N; e += 256) {
+            const int r = e & 7, n = e >> 3;
+            const float* p = gate_part + ((((size_t)blockIdx.y * gridDim.x + (n >> 4)) * KS) << 7) + (n & 15) * 8 + r;
+            float sum = 0.f;
+            for (int z = 0; z < KS; ++z) sum += __ldcg(p + ((size_t)z << 7));
+            s_val[r][n] = sum;
+            if (m0 + r < c.M) {
+                c.gate[(size_t)(m0 + r) * c.N + n] = sum;
+                if (gate_tap) gate_tap[(size_t)(m0 + r) * c.N + n] = sum;
+            }
+        }
+        __syncthreads();
+    }
     {
         const int m = m0 + warp;
+        const bool sm = KS > 1;
         if (m < c.M) {
-            if (c.N <= 32) route_select_row<1>(c, forced, groups_tap, m, lane, s_val[warp], s_slot_row[warp], s_mask, warp);
-            else if (c.N <= 64) route_select_row<2>(c, forced, groups_tap, m, lane, s_val[warp], s_slot_row[warp], s_mask, warp);
-            else if (c.N <= 128) route_select_row<4>(c, forced, groups_tap, m, lane, s_val[warp], s_slot_row[warp], s_mask, warp);
-            else route_select_row<8>(c, forced, groups_tap, m, lane, s_val[warp], s_slot_row[warp], s_mask, warp);
+            if (c.N <= 32) route_select_row<1>(c, forced, groups_tap, m, lane, s_val[warp], s_slot_row[warp], s_mask, warp, sm);
+            else if (c.N <= 64) route_select_row<2>(c, forced, groups_tap, m, lane, s_val[warp], s_slot_row[warp], s_mask, warp, sm);
+            else if (c.N <= 128) route_select_row<4>(c, forced, groups_tap, m, lane, s_val[warp], s_slot_row[warp], s_mask, warp, sm);
+            else route_select_row<8>(c, forced, groups_tap, m, lane, s_val[warp], s_slot_row[warp], s_mask, warp, sm);
         }
     }
     __syncthreads();
