@@ -441,6 +441,12 @@ __global__ void __launch_bounds__(kTcHeadThreads, 1)
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int rank = (int)cluster_ctarank();
     const bool leader = rank == 0;
+    if (c.adaptive) {
+        // the router decides between this kernel and the streaming one: when it is the other, leave before any
+        // set-up (every thread of both CTAs takes the same way out)
+        pdl_wait();
+        if (c.state->path_choice != 2) return;
+    }
 
     // The kernel may be launched while its predecessors (gather, router) still run: everything up to the
     // dependency wait touches only the pair's shared and tensor memory.
