@@ -49,9 +49,9 @@ extern "C" {
 #define CORAL_CFG_SHARD(rank, world) ((uint32_t)(((world) & 0xff) | (((rank) & 0xff) << 8)))
 
 /* Execution paths (coral_lmhead_set_path / coral_lmhead_stats.path). */
-#define CORAL_PATH_AUTO 0          /* chosen from (M, k_groups) */
+#define CORAL_PATH_AUTO 0          /* TCGEN05 for more than 96 rows or 10 rows per group and more on average, else STREAM, else SIMT_PLAIN */
 #define CORAL_PATH_STREAM 1        /* bulk-copy weight streaming + warp MMA (fp32 accumulate); M <= 128, H % 256 == 0, H <= 4096 */
-#define CORAL_PATH_TCGEN05 2       /* routed grouped GEMM on tcgen05 / TMEM tiles */
+#define CORAL_PATH_TCGEN05 2       /* routed grouped GEMM by CTA pairs on tcgen05 / TMEM tiles; handle created with max_M > 32 */
 #define CORAL_PATH_SIMT_PLAIN 3    /* gathered GEMV with plain 128-bit loads, any M */
 #define CORAL_PATH_ADAPTIVE 4      /* 33..128 rows: the router picks STREAM or TCGEN05 on the device from the rows per group */
 

@@ -27,8 +27,8 @@ __device__ __forceinline__ void tc_wait(uint32_t bar, uint32_t parity, volatile 
     set_status(st, -5);
 }
 
-// L2 eviction policies for the tiled loads: the weights of a group are streamed once per pass (evict first,
-// unless a later pass reads them again), the gathered hidden rows are re-read for every pair of sub-tiles
+// L2 eviction policies for the operand loads: the weights of a group are streamed once per pass (evict first,
+// unless a later pass reads them again), the gathered hidden rows are re-read for every batch of the entry
 // (evict last), so the weight stream does not push them out of L2.
 __device__ __forceinline__ uint64_t l2_policy_evict_first() {
     uint64_t p;
