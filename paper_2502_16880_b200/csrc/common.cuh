@@ -10,6 +10,12 @@ constexpr int kMaxKTokens = 32;       // CORAL_MAX_K_TOKENS
 constexpr int kMaxGroups = 256;       // CORAL_MAX_GROUPS
 constexpr float kNegInf = -__builtin_huge_valf();
 constexpr int kNoToken = 0x7fffffff;
+constexpr int kTcPassRows = 256;      // tensor-core path: hidden rows per pass over a group's weights (the MMA's largest N)
+
+// Tensor-core path: first row, in the gathered hidden matrix, of the union-list entry whose first bucket position is
+// `first` and whose index in the union list is j: entries are packed in bucket order, each starting on a multiple of
+// 16 rows (the step from one entry to the next is at least its row count rounded up to 16).
+__host__ __device__ __forceinline__ int tc_entry_row(int first, int j) { return ((first + 15) & ~15) + 16 * j; }
 
 // Device-resident per-handle state written by the kernels.
 struct DeviceState {
@@ -44,6 +50,7 @@ struct CallView {
     int32_t* group_offset;         // [N+1]
     int32_t* bucket_row;           // [M*k_groups] rows that selected a group, ascending per group
     int32_t* bucket_slot;          // [M*k_groups] the slot the group has in that row
+    int32_t* bucket_dst;           // [M*k_groups] tensor-core calls: the pair's row in the gathered hidden matrix
     int32_t* slot_desc;            // [M][k_groups] (index in union_list of the slot's (group, pass)) << 8 | row's position in the pass
     int32_t* union_list;           // [n_virtual] group | pass << 16, ascending (group, pass)
     int32_t* union_rank;           // [N] index of (group n, pass 0) in union_list, -1 if untouched

@@ -27,7 +27,7 @@ inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 // Offsets of the workspace sections (bytes from the workspace base).
 struct Layout {
-    size_t w_gate, group_tokens, state, gate, sel, slot_of, group_count, group_offset, bucket_row, bucket_slot,
+    size_t w_gate, group_tokens, state, gate, sel, slot_of, group_count, group_offset, bucket_row, bucket_slot, bucket_dst,
         slot_desc, union_list, union_rank, part_max, part_sum, part_val, part_id, sp_max, sp_sum, sp_val, sp_id,
         cand_val, cand_id, route_mid, route_part, tc_hg, tc_max, tc_sum, tc_val, tc_id, stage_hidden, stage_ids, stage_logprobs, total;
     size_t packed_bytes, cand_cap, cand_rows;
@@ -117,6 +117,7 @@ Layout make_layout(const coral_lmhead_config& c) {
     L.group_offset = take((N + 1) * 4);
     L.bucket_row = take(M * kg * 4);
     L.bucket_slot = take(M * kg * 4);
+    L.bucket_dst = take(M * kg * 4);
     L.slot_desc = take(M * kg * 4);
     L.union_list = take(N * kStreamMaxPasses * 4);
     L.union_rank = take(N * 4);
@@ -226,6 +227,7 @@ CallView make_view(const coral_lmhead_s* h, const void* hidden, int M, int kg, i
     c.group_offset = reinterpret_cast<int32_t*>(ws + L.group_offset);
     c.bucket_row = reinterpret_cast<int32_t*>(ws + L.bucket_row);
     c.bucket_slot = reinterpret_cast<int32_t*>(ws + L.bucket_slot);
+    c.bucket_dst = reinterpret_cast<int32_t*>(ws + L.bucket_dst);
     c.slot_desc = reinterpret_cast<int32_t*>(ws + L.slot_desc);
     c.union_list = reinterpret_cast<int32_t*>(ws + L.union_list);
     c.union_rank = reinterpret_cast<int32_t*>(ws + L.union_rank);
@@ -622,7 +624,7 @@ static int draft_impl(coral_lmhead_handle h, const void* hidden_dev, int M, int 
             // both head kernels are launched; each reads the router's choice first and the one not chosen returns
             TcGeom tg{h->tc_pairs, L.tc_tiles, (L.tc_tiles + 1) / 2, L.KB, L.tc_hg_rows};
             TcPartials tp{tpp.pmax, tpp.psum, tpp.pval, tpp.pid};
-            launch_pdl(tc_gather_kernel, dim3(M * k_groups), dim3(128), (size_t)0, st, c,
+            launch_pdl(tc_gather_kernel, dim3((M * k_groups + kGatherPairs - 1) / kGatherPairs), dim3(64 * kGatherPairs), (size_t)0, st, c,
                        reinterpret_cast<uint16_t*>(h->ws + L.tc_hg), L.tc_hg_rows);
             ++launches;
             launch_pdl_pairs(head_tc_kernel, dim3(2 * tg.pairs), dim3(kTcHeadThreads), kTcSmemBytes, st, c, tg, tp, h->map_w,
@@ -651,7 +653,7 @@ static int draft_impl(coral_lmhead_handle h, const void* hidden_dev, int M, int 
         TcGeom tg{h->tc_pairs, L.tc_tiles, (L.tc_tiles + 1) / 2, L.KB, L.tc_hg_rows};
         TcPartials tp{reinterpret_cast<float*>(h->ws + L.tc_max), reinterpret_cast<float*>(h->ws + L.tc_sum),
                       reinterpret_cast<float*>(h->ws + L.tc_val), reinterpret_cast<int32_t*>(h->ws + L.tc_id)};
-        launch_pdl(tc_gather_kernel, dim3(M * k_groups), dim3(128), (size_t)0, st, c,
+        launch_pdl(tc_gather_kernel, dim3((M * k_groups + kGatherPairs - 1) / kGatherPairs), dim3(64 * kGatherPairs), (size_t)0, st, c,
                    reinterpret_cast<uint16_t*>(h->ws + L.tc_hg), L.tc_hg_rows);
         ++launches;
         launch_pdl_pairs(head_tc_kernel, dim3(2 * tg.pairs), dim3(kTcHeadThreads), kTcSmemBytes, st, c, tg, tp, h->map_w,

@@ -36,7 +36,6 @@
 namespace coral {
 
 constexpr int kTcHeadThreads = kTcThreads + 32;     // warp 10 issues the MMAs of a batch's second accumulator
-constexpr int kTcPassRows = 256;                    // hidden rows per pass over a group's weights (the MMA's largest N)
 // The operand ring is cut into slots of the size the current batch needs per 64 columns, so that the bytes in
 // flight - what hides the memory latency - stay the same whatever the batch: two weight tiles + up to 8 KiB of
 // hidden rows (40 KiB, five slots), one + up to 8 KiB (24 KiB, eight slots), one + up to 16 KiB (32 KiB, six).
@@ -89,37 +88,41 @@ struct TcPartials {
     int32_t* pid;
 };
 
-// First row, in the gathered matrix, of the entry whose first bucket position is `first` and whose index in
-// the union list is j: entries are packed in bucket order, each starting on a multiple of 16 rows (the step
-// from one entry to the next is at least its row count rounded up to 16).
-__host__ __device__ __forceinline__ int tc_entry_row(int first, int j) { return ((first + 15) & ~15) + 16 * j; }
-
 // Gathers the hidden rows of every entry into the operand layout
 //   hg[column block kb][row][64 columns]     (row = tc_entry_row(...) + position in the entry)
 // with the 16-byte chunks of every 128-byte row permuted the way the 128-byte shared-memory swizzle wants
 // them (chunk c of row r at position c ^ (r & 7)), so that a plain contiguous bulk copy of n/2 rows lands in
-// shared memory as a K-major operand tile.  One thread block per (row, slot) pair in bucket order; columns
-// past H are written as zero; rows between an entry's size and its padded size keep whatever they held
-// (their accumulator columns are never read).
-__global__ void __launch_bounds__(128) tc_gather_kernel(CallView c, uint16_t* __restrict__ hg, int hg_rows) {
-    const int p = blockIdx.x;
+// shared memory as a K-major operand tile.  A block copies kGatherPairs (row, slot) pairs in bucket order, 64
+// threads each; where a pair's row comes from and goes to was written by the router stage (bucket_row,
+// bucket_dst), so one round of loads finds it.  Columns past H are written as zero; rows between an entry's
+// size and its padded size keep whatever they held (their accumulator columns are never read).
+constexpr int kGatherPairs = 4;
+__global__ void __launch_bounds__(64 * kGatherPairs) tc_gather_kernel(CallView c, uint16_t* __restrict__ hg, int hg_rows) {
+    const int p = blockIdx.x * kGatherPairs + (threadIdx.x >> 6), t = threadIdx.x & 63;
     pdl_wait();                                              // launched over the tail of the router stage
     pdl_launch_dependents();
     if (call_is_poisoned(c.state)) return;                   // the router stage reported a problem: index with nothing
     if (c.adaptive && c.state->path_choice != 2) return;     // the router chose the streaming kernel for this call
     if (p >= c.group_offset[c.N]) return;          // fewer pairs than M * k_groups when the vocab is sharded
     const int m = CORAL_IDX(c.bucket_row[p], c.M, c.state);
-    const int n = CORAL_IDX(c.sel[CORAL_IDX((size_t)m * c.k_groups + c.bucket_slot[p], c.cap_pairs, c.state)], c.N, c.state);
-    const int rg = p - c.group_offset[n];
-    const int pass = rg / kTcPassRows;
-    const int row = tc_entry_row(c.group_offset[n] + pass * kTcPassRows, c.union_rank[n] + pass) + rg % kTcPassRows;
+    const int row = c.bucket_dst[p];
     if (!CORAL_IDX_OK(row, hg_rows, c.state)) return;
     const uint4* src = reinterpret_cast<const uint4*>(c.hidden + (size_t)m * c.H);
     uint4* dst = reinterpret_cast<uint4*>(hg);
     const int chunks = c.H >> 3;
-    for (int ch = threadIdx.x; ch < c.KB * 8; ch += 128)
-        dst[((size_t)(ch >> 3) * hg_rows + row) * 8 + ((ch & 7) ^ (row & 7))] =
-            ch < chunks ? __ldg(src + ch) : make_uint4(0, 0, 0, 0);
+    for (int ch0 = 0; ch0 < c.KB * 8; ch0 += 64 * 4) {      // four loads in flight per thread
+        uint4 v[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int ch = ch0 + u * 64 + t;
+            v[u] = ch < chunks ? __ldg(src + ch) : make_uint4(0, 0, 0, 0);
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int ch = ch0 + u * 64 + t;
+            if (ch < c.KB * 8) dst[((size_t)(ch >> 3) * hg_rows + row) * 8 + ((ch & 7) ^ (row & 7))] = v[u];
+        }
+    }
 }
 
 // Insertion into a thread-private top-KT list kept sorted (value desc, row index asc).  The new entry's

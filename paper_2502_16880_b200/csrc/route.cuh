@@ -311,6 +311,8 @@ __global__ void __launch_bounds__(kRouteThreads)
             c.bucket_slot[off + pos] = sl;
             const int pass = c.pass_rows > 0 ? pos / c.pass_rows : 0;
             c.slot_desc[(size_t)m * c.k_groups + sl] = ((virt + pass) << 8) | ((pos - pass * max(c.pass_rows, 1)) & 255);
+            if (c.bucket_dst && c.pass_rows == kTcPassRows)
+                c.bucket_dst[off + pos] = tc_entry_row(off + pass * kTcPassRows, virt + pass) + pos - pass * kTcPassRows;
         }
     }
     if (threadIdx.x == 0) {
@@ -595,6 +597,8 @@ __global__ void __launch_bounds__(256)
                 c.bucket_slot[off + pos] = sl;
                 const int pass = pr > 0 ? pos / pr : 0;
                 c.slot_desc[(size_t)m * c.k_groups + sl] = ((virt + pass) << 8) | ((pos - pass * max(pr, 1)) & 255);
+                if (c.bucket_dst && pr == kTcPassRows)
+                    c.bucket_dst[off + pos] = tc_entry_row(off + pass * kTcPassRows, virt + pass) + pos - pass * kTcPassRows;
             }
         }
     }
@@ -676,6 +680,8 @@ __global__ void __launch_bounds__(256) bucket_group_kernel(CallView c, int* __re
             c.bucket_slot[off + pos] = sl;
             const int pass = c.pass_rows > 0 ? pos / c.pass_rows : 0;
             c.slot_desc[(size_t)m * c.k_groups + sl] = ((virt + pass) << 8) | ((pos - pass * max(c.pass_rows, 1)) & 255);
+            if (c.bucket_dst && c.pass_rows == kTcPassRows)
+                c.bucket_dst[off + pos] = tc_entry_row(off + pass * kTcPassRows, virt + pass) + pos - pass * kTcPassRows;
             }
         }
         running += all;
