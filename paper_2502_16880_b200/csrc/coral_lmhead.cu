@@ -109,7 +109,7 @@ Layout make_layout(const coral_lmhead_config& c) {
     L.state = take(sizeof(DeviceState));
     L.route_bands = (M + 7) / 8 > (size_t)kRouteMidBands ? (M + 7) / 8 : (size_t)kRouteMidBands;
     L.route_mid = take((L.route_bands + 5 * N) * 4);      // band tickets, 4 mask words and one counter per group
-    L.route_part = take((size_t)kRouteMidBands * kRouteMidSplitMax * ((N + 15) / 16) * 128 * 4);   // partial score tiles when H is split
+    L.route_part = take(L.route_bands * kRouteMidSplitMax * ((N + 15) / 16) * 128 * 4);   // partial score tiles when H is split
     L.gate = take(M * N * 4);
     L.sel = take(M * kg * 4);
     L.slot_of = take(M * N * 2);
@@ -592,8 +592,11 @@ static int draft_impl(coral_lmhead_handle h, const void* hidden_dev, int M, int 
             reinterpret_cast<float*>(h->ws + h->L.route_part));
         ++launches;
     } else if (cfg.H % 32 == 0) {
-        route_mid_kernel<<<dim3((c.N + 15) / 16, (M + 7) / 8), 256, 0, st>>>(
-            c, forced_groups_dev, out_groups_dev, out_gate_dev, rt_bands, rt_masks, rt_counts, 0, nullptr);
+        // (up to some 300 tiles two blocks per tile still pay: 27 -> 23 us at 256 rows; beyond, the tiles fill the GPU by themselves)
+        const int tiles = ((c.N + 15) / 16) * ((M + 7) / 8);
+        route_mid_kernel<<<dim3((c.N + 15) / 16, (M + 7) / 8, tiles < 300 ? 2 : 1), 256, 0, st>>>(
+            c, forced_groups_dev, out_groups_dev, out_gate_dev, rt_bands, rt_masks, rt_counts, 0,
+            reinterpret_cast<float*>(h->ws + h->L.route_part));
         ++launches;
         launch_pdl(bucket_group_kernel, dim3(c.N), dim3(256), (size_t)0, st, c, rt_counts);
         ++launches;
