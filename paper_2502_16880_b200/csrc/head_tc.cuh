@@ -71,7 +71,7 @@ struct TcRingPos {
     }
 };
 constexpr int kTcXchgBytes = 2 * 4 * 16 * 32 * 4;   // [accumulator][owner warp][16 vocab rows][32 hidden rows] fp32
-constexpr size_t kTcSmemBytes = 1024 + (size_t)kTcRingBytes + kTcXchgBytes + 256;
+constexpr size_t kTcSmemBytes = 1024 + (size_t)kTcRingBytes + kTcXchgBytes + 256 + 4096;   // + the run split's cost cache
 
 struct TcGeom {
     int pairs;        // CTA pairs launched
@@ -279,16 +279,24 @@ __device__ __forceinline__ int tc_unit_cost(int rows) {
 // Cuts the unit list into g.pairs runs of (almost) equal cost (one warp).  out[0], out[1]: entry and unit where
 // the pair's run starts; out[2]: its number of units.  Run p holds the units whose cost prefix (tc_unit_cost),
 // taken at the unit's middle, lies in [p, p + 1) * total / pairs.
-__device__ __forceinline__ void tc_split_runs(const CallView& c, const TcGeom& g, int n_entries, int pair, int* out) {
+// (The entries' costs are read from global memory once - two dependent loads each, all of a lane's in flight together -
+// and kept in `cost_cache` for the second pass; beyond kTcCostCache entries the second pass reads them again.)
+constexpr int kTcCostCache = 1024;
+__device__ __forceinline__ void tc_split_runs(const CallView& c, const TcGeom& g, int n_entries, int pair, int* out,
+                                              int* cost_cache) {
     const int lane = threadIdx.x & 31;
     long long total = 0;
+#pragma unroll 4
     for (int j0 = 0; j0 < n_entries; j0 += 32) {
         const int j = j0 + lane;
         if (j < n_entries) {
             const int entry = c.union_list[j];
-            total += (long long)g.units * tc_unit_cost(c.group_count[entry & 0xffff] - (entry >> 16) * kTcPassRows);
+            const int w = tc_unit_cost(c.group_count[entry & 0xffff] - (entry >> 16) * kTcPassRows);
+            if (j < kTcCostCache) cost_cache[j] = w;
+            total += (long long)g.units * w;
         }
     }
+    __syncwarp();
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) total += __shfl_xor_sync(0xffffffffu, total, o);
     const long long t_lo = pair * total / g.pairs, t_hi = (pair + 1) * total / g.pairs;
@@ -300,8 +308,12 @@ __device__ __forceinline__ void tc_split_runs(const CallView& c, const TcGeom& g
         const int j = j0 + lane;
         int w = 0;
         if (j < n_entries) {
-            const int entry = c.union_list[j];
-            w = tc_unit_cost(c.group_count[entry & 0xffff] - (entry >> 16) * kTcPassRows);
+            if (j < kTcCostCache) {
+                w = cost_cache[j];
+            } else {
+                const int entry = c.union_list[j];
+                w = tc_unit_cost(c.group_count[entry & 0xffff] - (entry >> 16) * kTcPassRows);
+            }
         }
         const long long cost = (long long)w * g.units;
         long long incl = cost;
@@ -440,6 +452,7 @@ __global__ void __launch_bounds__(kTcHeadThreads, 1)
     uint64_t* tmem_empty = tmem_full + 2;         // [2] rank 0: both CTAs' epilogue warps have drained the buffer
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tmem_empty + 2);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+    int* cost_cache = reinterpret_cast<int*>(smem + kTcRingBytes + kTcXchgBytes + 256);      // [kTcCostCache]
     int* run = const_cast<int*>(abort_flag) + 1;  // [3] entry and unit where the pair's run starts, number of units
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int rank = (int)cluster_ctarank();
@@ -483,7 +496,7 @@ __global__ void __launch_bounds__(kTcHeadThreads, 1)
     const bool skip = (c.adaptive && c.state->path_choice != 2) || call_is_poisoned(c.state);
 
     // this pair's run of units
-    if (warp == 0) tc_split_runs(c, g, skip ? 0 : c.state->n_virtual, (int)(blockIdx.x >> 1), run);
+    if (warp == 0) tc_split_runs(c, g, skip ? 0 : c.state->n_virtual, (int)(blockIdx.x >> 1), run, cost_cache);
     __syncthreads();
 
     if (warp == 0) {
