@@ -326,8 +326,15 @@ __device__ __forceinline__ void tc_split_runs(const CallView& c, const TcGeom& g
         if (w > 0) {
             // unit u's middle is at start + w * u + w / 2; the first u whose middle is >= t
             const long long a_lo = 2 * (t_lo - start) - w, a_hi = 2 * (t_hi - start) - w;
-            const long long u_lo = a_lo <= 0 ? 0 : (a_lo + 2 * w - 1) / (2 * w);
-            const long long u_hi = a_hi <= 0 ? 0 : (a_hi + 2 * w - 1) / (2 * w);
+            long long u_lo = a_lo <= 0 ? 0 : (a_lo + 2 * w - 1) / (2 * w);
+            long long u_hi = a_hi <= 0 ? 0 : (a_hi + 2 * w - 1) / (2 * w);
+            // A narrow entry with many rows is cut between its batches of two: there a batch of one unit takes about
+            // as long as a batch of two (measured at 112-128 rows: 293 against 300 us whole step), while with few
+            // rows per entry it is cheap and the finer cut balances better (60 rows: 241 against 249 us).
+            if (w < 2 * kTcSub && w >= kTcSub + 24) {
+                u_lo = (u_lo + 1) & ~1ll;
+                u_hi = (u_hi + 1) & ~1ll;
+            }
             if (u_lo < g.units) lo = min(lo, j * g.units + (int)u_lo);
             if (u_hi < g.units) hi = min(hi, j * g.units + (int)u_hi);
         }
