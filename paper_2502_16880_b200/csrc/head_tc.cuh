@@ -17,19 +17,20 @@
 //
 // Epilogue.  A tensor-memory lane holds one vocab row and a column one hidden row, and a warp reads only its
 // own quarter of the lanes; the per-row statistics need one thread per hidden row.  The four warps of an
-// accumulator therefore exchange 32 x 32 blocks through shared memory: in step s warp q reads columns
-// 32 ((q + s) mod 4) .. + 31 of its lanes and hands them to warp (q + s) mod 4, which owns those hidden rows
-// and folds the block's 32 logits per row into its running (max, sum-exp, top-k), carried in registers over
-// the sub-tiles the warp sees of an entry; logits never travel to HBM.  (CORAL Section 3.3: logits only for
+// accumulator therefore exchange blocks through shared memory: in step s warp q reads columns
+// 32 ((q + s) mod 4) .. + 31 of its lanes and hands them, 16 vocab rows at a time (16 KiB of shared memory
+// for both accumulators), to warp (q + s) mod 4, which owns those hidden rows and folds the block's 16 logits
+// per row into its running (max, sum-exp, top-k), carried in registers over the sub-tiles the warp sees of an
+// entry; logits never travel to HBM.  (CORAL Section 3.3: logits only for
 // the activated groups; Appendix B: the union of the rows' groups is what gets read.)
 //
 // Warp roles: warp 0 = producer (TMA tiled loads of the weights, one bulk copy of the hidden rows); warps 1 and
 // 10 = MMA issuers in the CTA of rank 0, one per accumulator of the batch (issuing an MMA costs its thread
-// some 40 ns, which for eight MMAs per 64 columns would be the pair's critical path); warp 1 of rank 1 is the
-// relay that tells rank 0 when a stage has landed; warps 2..9 = epilogue, four per accumulator (with one wide
+// some 50 ns, which for eight MMAs per 64 columns would be the pair's critical path); warp 1 of rank 1 is the
+// relay that tells rank 0 when a slot of the operand ring has landed; warps 2..9 = epilogue, four per accumulator (with one wide
 // accumulator: four per half of its columns).
 // Work split: the units of all entries form one list; pair p owns a contiguous run of it, cut so that the
-// runs cost the same (a unit of a wide entry, which is a batch by itself, counts twice).
+// runs cost the same (tc_unit_cost: a unit of a wide entry, which is a batch by itself, counts about twice).
 #pragma once
 #include "tc_prims.cuh"
 
