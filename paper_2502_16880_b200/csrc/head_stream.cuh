@@ -450,40 +450,32 @@ constexpr int kMergeJoint = 0, kMergeFactorised = 1, kMergePartial = 2, kMergeFa
 constexpr int kMergeStreamThreads = 256;
 constexpr int kMergeMaxPieces = 2048;         // >= grid + 2 * k_groups for every supported shape
 constexpr int kMergeRankMax = 256;            // survivors ranked by counting; more fall back to k rounds
-// Shared-memory arrays of fixed size that merge_row needs beside its candidate and per-piece arrays.
-struct MergeFixed {
-    float s_f[16], s_t[16];
-    int s_i[16];
-    float s_lse, s_glse, s_thr2;
-    int s_n, s_nlive;
-    int s_first[kMaxGroups], s_base[kMaxGroups + 1], s_rpos[kMaxGroups], s_j[kMaxGroups];
-    float s_off[kMaxGroups];           // per slot: what is added to a logit to give the emitted log-prob
-};
-
-// The merge of one row m by kMergeStreamThreads threads (threads 0 .. 255 of the calling block).  kKernel: called
-// from merge_stream_kernel (block-wide barriers, waits for the predecessor grid before reading the partials); else
-// from the tail of head_stream_kernel by the block that completed the row (hardware barrier 3 over its first 256
-// threads; the partials are complete, and they are read past L1, which may not have seen other SMs' writes).
-// msm: kMergeStreamThreads-shared scratch of merge_smem_bytes(p_cap, smem_cands) bytes.
-template <bool kKernel>
-__device__ __forceinline__ void merge_row(const CallView& c, const StreamGeom& g, const StreamPartials& pp, int m,
-                                          unsigned char* msm, MergeFixed& F, float* __restrict__ cand_val_scratch,
-                                          int32_t* __restrict__ cand_id_scratch, int cand_cap, int smem_cands, int p_cap,
-                                          int mode, int32_t* __restrict__ out_ids, float* __restrict__ out_logprobs,
-                                          float* __restrict__ lse_tap) {
-#define MSYNC() do { if (kKernel) __syncthreads(); else asm volatile("bar.sync 3, 256;" ::: "memory"); } while (0)
-#define MLD(ptr) (kKernel ? *(ptr) : __ldcg(ptr))
-    float* s_f = F.s_f; float* s_t = F.s_t; int* s_i = F.s_i;
-    float& s_lse = F.s_lse; float& s_glse = F.s_glse; float& s_thr2 = F.s_thr2;
-    int& s_n = F.s_n; int& s_nlive = F.s_nlive;
-    int* s_first = F.s_first; int* s_base = F.s_base; int* s_rpos = F.s_rpos; int* s_j = F.s_j;
-    float* s_off = F.s_off;
+__global__ void __launch_bounds__(kMergeStreamThreads) merge_stream_kernel(CallView c, StreamGeom g_in, StreamPartials pp_in,
+                                                                           StreamGeom g_tc, StreamPartials pp_tc,
+                                                                           float* __restrict__ cand_val_scratch,
+                                                                           int32_t* __restrict__ cand_id_scratch,
+                                                                           int cand_cap, int smem_cands, int p_cap, int mode,
+                                                                           int32_t* __restrict__ out_ids,
+                                                                           float* __restrict__ out_logprobs,
+                                                                           float* __restrict__ lse_tap) {
+    extern __shared__ __align__(16) unsigned char msm[];
+    // adaptive call: the partials are those of the kernel the router chose (complete by the time this grid runs:
+    // it is launched behind the tensor-core kernel, which does not release its dependents early)
+    const bool took_tc = c.adaptive && c.state->path_choice == 2;
+    const StreamGeom g = took_tc ? g_tc : g_in;
+    const StreamPartials pp = took_tc ? pp_tc : pp_in;
+    const int m = blockIdx.x;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     constexpr int kWarps = kMergeStreamThreads / 32;
     const bool renorm = mode == kMergeFactorisedRenorm;      // p_router over the row's selected groups only
     const bool factorised = mode == kMergeFactorised || renorm, partial = mode == kMergePartial;
     float* rec = partial ? out_logprobs + (size_t)m * (2 + 2 * c.k_tokens) : nullptr;
-    // scratch: candidates (smem_cands values + ids), then per-piece arrays of capacity p_cap
+    __shared__ float s_f[kWarps], s_t[kWarps];
+    __shared__ float s_lse, s_glse, s_thr2;
+    __shared__ int s_n, s_nlive;
+    __shared__ int s_first[kMaxGroups], s_base[kMaxGroups + 1], s_rpos[kMaxGroups], s_j[kMaxGroups];
+    __shared__ float s_off[kMaxGroups];           // per slot: what is added to a logit to give the emitted log-prob
+    // dynamic shared memory: candidates (smem_cands values + ids), then per-piece arrays of capacity p_cap
     float* s_pm = reinterpret_cast<float*>(msm + (size_t)smem_cands * 8);
     float* s_ps = s_pm + p_cap;
     float* s_last = s_ps + p_cap;
@@ -515,13 +507,13 @@ __device__ __forceinline__ void merge_row(const CallView& c, const StreamGeom& g
                          : c.gate[(size_t)m * c.N + (renorm ? c.sel[(size_t)m * c.k_groups + threadIdx.x] : (int)threadIdx.x)];
         const float wm = warp_max(gv);
         if (lane == 0) s_f[warp] = wm;
-        MSYNC();
+        __syncthreads();
         float gm = s_f[0];
 #pragma unroll
         for (int w = 1; w < kWarps; ++w) gm = fmaxf(gm, s_f[w]);
         const float ws = warp_sum(mine ? expf(gv - gm) : 0.f);
         if (lane == 0) s_t[warp] = ws;
-        MSYNC();
+        __syncthreads();
         if (threadIdx.x == 0) {
             float tot = 0.f;
 #pragma unroll
@@ -529,13 +521,13 @@ __device__ __forceinline__ void merge_row(const CallView& c, const StreamGeom& g
             s_glse = gm + logf(tot);
         }
     }
-    MSYNC();
+    __syncthreads();
     if (threadIdx.x == 0) {
         int run = 0;
         for (int s = 0; s < c.k_groups; ++s) { const int cnt = s_base[s]; s_base[s] = run; run += cnt; }
         s_base[c.k_groups] = run;
     }
-    MSYNC();
+    __syncthreads();
     const int P = min(s_base[c.k_groups], p_cap);
     if (partial) {                 // defaults; a row none of whose groups is computed here keeps them
         if (threadIdx.x < c.k_tokens) {
@@ -559,26 +551,26 @@ __device__ __forceinline__ void merge_row(const CallView& c, const StreamGeom& g
             s_piece[q] = (int)(((size_t)b * g.seg_max + seg) * kStreamPassRows + s_rpos[s]);
         }
     }
-    MSYNC();
+    __syncthreads();
 
-    if (kKernel) pdl_wait();      // partials of the streaming kernel are complete from here on
+    pdl_wait();                   // partials of the streaming kernel are complete from here on
 
     // pass 1 over the pieces (all loads of a thread's pieces issued together)
     float mx = kNegInf;
     for (int q = threadIdx.x; q < P; q += kMergeStreamThreads) {
 #ifdef CORAL_CHECK_BOUNDS
-        if (!index_ok(s_piece[q], g.tc_tiles > 0 ? c.cap_part_tc : c.cap_part_stream, c.state)) s_piece[q] = 0;
+        if (!index_ok(s_piece[q], took_tc || g.tc_tiles > 0 ? c.cap_part_tc : c.cap_part_stream, c.state)) s_piece[q] = 0;
 #endif
         const size_t p = (size_t)s_piece[q];
-        const float a = MLD(pp.pmax + p), b = MLD(pp.psum + p);
-        float l = MLD(pp.pval + p * c.k_tokens + c.k_tokens - 1), h = MLD(pp.pval + p * c.k_tokens);
+        const float a = pp.pmax[p], b = pp.psum[p];
+        float l = pp.pval[p * c.k_tokens + c.k_tokens - 1], h = pp.pval[p * c.k_tokens];
         if (a == kNegInf) { l = kNegInf; h = kNegInf; }      // empty piece: its candidate list was not written
         s_pm[q] = a; s_ps[q] = b; s_last[q] = l; s_head[q] = h;
         mx = fmaxf(mx, a);
     }
     mx = warp_max(mx);
     if (lane == 0) s_f[warp] = mx;
-    MSYNC();
+    __syncthreads();
     mx = s_f[0];
 #pragma unroll
     for (int w = 1; w < kWarps; ++w) mx = fmaxf(mx, s_f[w]);
@@ -586,7 +578,7 @@ __device__ __forceinline__ void merge_row(const CallView& c, const StreamGeom& g
     for (int q = threadIdx.x; q < P; q += kMergeStreamThreads) sum += s_ps[q] * expf(s_pm[q] - mx);
     sum = warp_sum(sum);
     if (lane == 0) s_t[warp] = sum;
-    MSYNC();
+    __syncthreads();
     if (threadIdx.x == 0) {
         float tot = 0.f;
 #pragma unroll
@@ -595,7 +587,7 @@ __device__ __forceinline__ void merge_row(const CallView& c, const StreamGeom& g
         if (lse_tap) lse_tap[m] = s_lse;
         if (partial) { rec[0] = mx; rec[1] = tot; }
     }
-    MSYNC();
+    __syncthreads();
     // per-slot offsets
     for (int s = threadIdx.x; s < c.k_groups; s += kMergeStreamThreads) {
         if (factorised) {
@@ -608,7 +600,7 @@ __device__ __forceinline__ void merge_row(const CallView& c, const StreamGeom& g
             s_off[s] = partial ? 0.f : -s_lse;
         }
     }
-    MSYNC();
+    __syncthreads();
     // thresholds on the emitted values
     float thr = kNegInf;
     for (int q = threadIdx.x; q < P; q += kMergeStreamThreads) {
@@ -618,7 +610,7 @@ __device__ __forceinline__ void merge_row(const CallView& c, const StreamGeom& g
     }
     thr = warp_max(thr);
     if (lane == 0) s_f[warp] = thr;
-    MSYNC();
+    __syncthreads();
     thr = s_f[0];
 #pragma unroll
     for (int w = 1; w < kWarps; ++w) thr = fmaxf(thr, s_f[w]);
@@ -629,7 +621,7 @@ __device__ __forceinline__ void merge_row(const CallView& c, const StreamGeom& g
         for (int i = 0; i < P; ++i) rank += better(s_head[i], i, hq, q) ? 1 : 0;
         if (rank == c.k_tokens - 1) s_thr2 = hq;
     }
-    MSYNC();
+    __syncthreads();
     thr = fmaxf(thr, s_thr2);
 
     // pass 2: keep the candidates at or above the threshold (order of arrival does not matter: the
@@ -642,7 +634,7 @@ __device__ __forceinline__ void merge_row(const CallView& c, const StreamGeom& g
                                     : cand_id_scratch + (size_t)m * cand_cap;
     for (int q = threadIdx.x; q < P; q += kMergeStreamThreads)
         if (s_pm[q] != kNegInf && s_head[q] >= thr) s_live[atomicAdd(&s_nlive, 1)] = q;
-    MSYNC();
+    __syncthreads();
     const int n_entries = s_nlive * c.k_tokens;
     for (int e0 = threadIdx.x; e0 < n_entries; e0 += 4 * kMergeStreamThreads) {
         float v[4];
@@ -655,8 +647,8 @@ __device__ __forceinline__ void merge_row(const CallView& c, const StreamGeom& g
             if (e < n_entries) {
                 const int q = s_live[e / c.k_tokens], l = e - (e / c.k_tokens) * c.k_tokens;
                 const size_t p = (size_t)s_piece[q];
-                v[u] = MLD(pp.pval + p * c.k_tokens + l) + s_off[s_pslot[q]];
-                id[u] = MLD(pp.pid + p * c.k_tokens + l);
+                v[u] = pp.pval[p * c.k_tokens + l] + s_off[s_pslot[q]];
+                id[u] = pp.pid[p * c.k_tokens + l];
             }
         }
 #pragma unroll
@@ -667,7 +659,7 @@ __device__ __forceinline__ void merge_row(const CallView& c, const StreamGeom& g
             }
         }
     }
-    MSYNC();
+    __syncthreads();
     const int S = min(s_n, cap);
 
     if (S <= kMergeRankMax) {
@@ -690,6 +682,7 @@ __device__ __forceinline__ void merge_row(const CallView& c, const StreamGeom& g
         return;
     }
     // many survivors (short or tied lists): k rounds of "best strictly after the last pick"
+    __shared__ int s_i[kWarps];
     float last_v = __builtin_huge_valf();
     int last_id = -1;
     for (int k = 0; k < c.k_tokens; ++k) {
@@ -702,9 +695,9 @@ __device__ __forceinline__ void merge_row(const CallView& c, const StreamGeom& g
             if (after && better(v, id, bv, bk)) { bv = v; bk = id; }
         }
         warp_argbest(bv, bk);
-        MSYNC();
+        __syncthreads();
         if (lane == 0) { s_f[warp] = bv; s_i[warp] = bk; }
-        MSYNC();
+        __syncthreads();
         bv = s_f[0]; bk = s_i[0];
 #pragma unroll
         for (int w = 1; w < kWarps; ++w)
@@ -721,25 +714,6 @@ __device__ __forceinline__ void merge_row(const CallView& c, const StreamGeom& g
         last_v = bv;
         last_id = bk;
     }
-}
-#undef MSYNC
-#undef MLD
-
-__global__ void __launch_bounds__(kMergeStreamThreads) merge_stream_kernel(CallView c, StreamGeom g_in, StreamPartials pp_in,
-                                                                           StreamGeom g_tc, StreamPartials pp_tc,
-                                                                           float* __restrict__ cand_val_scratch,
-                                                                           int32_t* __restrict__ cand_id_scratch,
-                                                                           int cand_cap, int smem_cands, int p_cap, int mode,
-                                                                           int32_t* __restrict__ out_ids,
-                                                                           float* __restrict__ out_logprobs,
-                                                                           float* __restrict__ lse_tap) {
-    extern __shared__ __align__(16) unsigned char msm[];
-    __shared__ MergeFixed fixed;
-    // adaptive call: the partials are those of the kernel the router chose (complete by the time this grid runs:
-    // it is launched behind the tensor-core kernel, which does not release its dependents early)
-    const bool took_tc = c.adaptive && c.state->path_choice == 2;
-    merge_row<true>(c, took_tc ? g_tc : g_in, took_tc ? pp_tc : pp_in, (int)blockIdx.x, msm, fixed, cand_val_scratch,
-                    cand_id_scratch, cand_cap, smem_cands, p_cap, mode, out_ids, out_logprobs, lse_tap);
 }
 
 // Combines the records that `world` GPUs wrote in partial mode (records[r][m] = record of row m from rank r,
