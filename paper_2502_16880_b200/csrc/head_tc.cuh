@@ -24,19 +24,20 @@
 // entry; logits never travel to HBM.  (CORAL Section 3.3: logits only for
 // the activated groups; Appendix B: the union of the rows' groups is what gets read.)
 //
-// Warp roles: warp 0 = producer (TMA tiled loads of the weights, one bulk copy of the hidden rows); warps 1 and
+// Warp roles: warps 0 and 11 = producers, a 64-column step each in turn (TMA tiled loads of the weights, bulk
+// copies of the hidden rows; one thread issues a step's copies in some 150 ns); warps 1 and
 // 10 = MMA issuers in the CTA of rank 0, one per accumulator of the batch (issuing an MMA costs its thread
 // some 50 ns, which for eight MMAs per 64 columns would be the pair's critical path); warp 1 of rank 1 is the
 // relay that tells rank 0 when a slot of the operand ring has landed; warps 2..9 = epilogue, four per accumulator (with one wide
 // accumulator: four per half of its columns).
 // Work split: the units of all entries form one list; pair p owns a contiguous run of it, cut so that the
-// runs cost the same (tc_unit_cost: a unit of a wide entry, which is a batch by itself, counts about twice).
+// runs cost the same (tc_unit_cost: a unit of a wide entry, which is a batch by itself, counts as 1.6 narrow ones).
 #pragma once
 #include "tc_prims.cuh"
 
 namespace coral {
 
-constexpr int kTcHeadThreads = kTcThreads + 32;     // warp 10 issues the MMAs of a batch's second accumulator
+constexpr int kTcHeadThreads = kTcThreads + 64;     // warp 10 issues the MMAs of a batch's second accumulator, warp 11 is the second producer
 // The operand ring is cut into slots of the size the current batch needs per 64 columns, so that the bytes in
 // flight - what hides the memory latency - stay the same whatever the batch: two weight tiles + up to 8 KiB of
 // hidden rows (40 KiB, five slots), one + up to 8 KiB (24 KiB, eight slots), one + up to 16 KiB (32 KiB, six).
@@ -269,12 +270,12 @@ struct TcWalk {
 
 // Relative time of one unit of an entry with `rows` rows.  A narrow entry's units go two to a batch and a batch
 // streams at what an SM can take in (its weight tiles plus its share of the hidden rows, in 128-byte units per
-// 64 columns); a wide entry's unit is a batch of its own and takes about as long as a narrow batch of two
-// (measured: 38-41 us against 36-40 us on the Llama3-8B shape), the MMA issue and the slot hand-over, not the
-// bytes, setting its pace.
+// 64 columns); a wide entry's unit is a batch of its own, whose pace the MMA issue and the slot hand-over set
+// rather than the bytes: about 0.8 of a narrow batch of two (the weight that gave the shortest whole step at
+// 960 and 1440 rows on the Llama3-8B shape; between 0.75 and 0.9 it matters by 1-2 %).
 __device__ __forceinline__ int tc_unit_cost(int rows) {
     const int npad = (max(1, min(rows, kTcPassRows)) + 15) & ~15;
-    return npad > kTcSub ? 2 * kTcSub + (npad >> 2) : kTcSub + (npad >> 2);
+    return npad > kTcSub ? kTcSub + 96 + (npad >> 2) : kTcSub + (npad >> 2);
 }
 
 // Cuts the unit list into g.pairs runs of (almost) equal cost (one warp).  out[0], out[1]: entry and unit where
@@ -330,9 +331,10 @@ __device__ __forceinline__ void tc_split_runs(const CallView& c, const TcGeom& g
             long long u_lo = a_lo <= 0 ? 0 : (a_lo + 2 * w - 1) / (2 * w);
             long long u_hi = a_hi <= 0 ? 0 : (a_hi + 2 * w - 1) / (2 * w);
             // A narrow entry with many rows is cut between its batches of two: there a batch of one unit takes about
-            // as long as a batch of two (measured at 112-128 rows: 293 against 300 us whole step), while with few
-            // rows per entry it is cheap and the finer cut balances better (60 rows: 241 against 249 us).
-            if (w < 2 * kTcSub && w >= kTcSub + 24) {
+            // as long as a batch of two (measured at 112-128 rows: 293 against 300 us whole step), while with fewer
+            // rows per entry it is cheap and the finer cut balances better (60 rows: 241 against 249 us; 96 rows:
+            // 258 against 263 us).
+            if (w <= kTcSub + (kTcSub >> 2) && w >= kTcSub + (112 >> 2)) {
                 u_lo = (u_lo + 1) & ~1ll;
                 u_hi = (u_hi + 1) & ~1ll;
             }
@@ -458,7 +460,8 @@ __global__ void __launch_bounds__(kTcHeadThreads, 1)
     uint64_t* empty = full + kTcMaxSlots;
     uint64_t* tmem_full = empty + kTcMaxSlots;    // [2]
     uint64_t* tmem_empty = tmem_full + 2;         // [2] rank 0: both CTAs' epilogue warps have drained the buffer
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tmem_empty + 2);
+    uint64_t* recut = tmem_empty + 2;             // the first producer has let the ring run empty for a new geometry
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(recut + 1);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
     int* cost_cache = reinterpret_cast<int*>(smem + kTcRingBytes + kTcXchgBytes + 256);      // [kTcCostCache]
     int* run = const_cast<int*>(abort_flag) + 1;  // [3] entry and unit where the pair's run starts, number of units
@@ -484,6 +487,7 @@ __global__ void __launch_bounds__(kTcHeadThreads, 1)
             mbar_init(smem_u32(&tmem_full[s]), 2);
             mbar_init(smem_u32(&tmem_empty[s]), 2 * kTcEpilogueWarps);
         }
+        mbar_init(smem_u32(recut), 2);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -507,8 +511,12 @@ __global__ void __launch_bounds__(kTcHeadThreads, 1)
     if (warp == 0) tc_split_runs(c, g, skip ? 0 : c.state->n_virtual, (int)(blockIdx.x >> 1), run, cost_cache);
     __syncthreads();
 
-    if (warp == 0) {
+    if (warp == 0 || warp == 11) {
         if (lane == 0) {
+            // two producers, one column step each in turn: a thread issues the copies of a step in some 150 ns,
+            // which alone would set the pace of the batches with one unit
+            const uint32_t mine = warp == 0 ? 0u : 1u;
+            uint32_t step = 0, recuts = 0;
             TcRingPos rp;
             const uint64_t pol_first = l2_policy_evict_first(), pol_normal = l2_policy_evict_normal(),
                            pol_last = l2_policy_evict_last();
@@ -526,16 +534,27 @@ __global__ void __launch_bounds__(kTcHeadThreads, 1)
                 const uint32_t hbytes = h1bytes + h2bytes;
                 const TcRing ring = tc_ring_for(w.wide, nu);
                 if (rp.enter(ring)) {
-                    // another slot size from here on: every copy issued so far must have been consumed first
-                    for (int s = 0; s < kTcMaxSlots; ++s)
-                        tc_wait(smem_u32(&empty[s]), ((rp.parity >> s) & 1u) ^ 1u, abort_flag, c.state);
+                    // another slot size from here on: every copy issued so far, by either producer, must have been
+                    // consumed first.  The first producer sees to that, then the two meet.  Its own last step is at
+                    // most one use of its slot ahead of the barrier, the other producer's last step may be two
+                    // (a parity wait cannot tell that from none): after one round over the slots everything but that
+                    // step has been consumed, the second round waits for it too.
+                    if (mine == 0) {
+                        for (int round = 0; round < 2; ++round)
+                            for (int s = 0; s < kTcMaxSlots; ++s)
+                                tc_wait(smem_u32(&empty[s]), ((rp.parity >> s) & 1u) ^ 1u, abort_flag, c.state);
+                    }
+                    mbar_arrive(smem_u32(recut));
+                    tc_wait(smem_u32(recut), recuts & 1u, abort_flag, c.state);
+                    ++recuts;
                 }
                 const uint32_t bytes = hbytes + (w0 ? kTcTileBytes : 0) + (w1 ? kTcTileBytes : 0);
                 const uint64_t pol_w = w.read_again ? pol_normal : pol_first;
                 const uint16_t* hsrc = hg + ((size_t)w.hrow + (size_t)rank * (w.wide ? kTcSub >> 1 : w.npad >> 1)) * kTcK;
                 const uint16_t* hsrc2 = hg + ((size_t)w.hrow + kTcSub + (size_t)rank * (n2 >> 1)) * kTcK;
                 const int gidx = w.n / c.pack_div;
-                for (int ks = 0; ks < g.ksteps; ++ks) {
+                for (int ks = 0; ks < g.ksteps; ++ks, ++step) {
+                    if ((step & 1u) != mine) { rp.advance(ring); continue; }
                     tc_wait(smem_u32(&empty[rp.slot]), rp.par() ^ 1u, abort_flag, c.state);
                     const uint32_t bar = smem_u32(&full[rp.slot]);
                     const uint32_t sb = smem_u32(smem) + (uint32_t)rp.slot * ring.bytes;
