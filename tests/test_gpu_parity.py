@@ -401,6 +401,30 @@ def test_many_groups(N, M, kg, path):
     head.close()
 
 
+def test_tensor_core_path_mixed_entry_kinds_with_an_odd_number_of_column_steps():
+    """Skewed routing over many small groups: every pair's run holds narrow entries, wide ones (129..256 rows) and
+    entries of groups that need several passes, so the operand ring is re-cut inside the runs; H = 320 gives five
+    64-column steps per unit, so the two producers' turns shift from unit to unit."""
+    N, v, M, kg = 200, 300, 1400, 8
+    cfg = synth.HeadConfig("mixedkinds", H=320, V=v * N, N=N, k_groups=kg, k_tokens=10, M=M, seed=29, w_std=0.05,
+                           zipf_s=1.2)
+    W, Wg, hb = synth.make_w_vocab(cfg), synth.make_w_gate(cfg), synth.make_hidden(cfg)
+    gm = synth.make_group_map(cfg, contiguous=True)
+    head = _head(cfg, W, gm, Wg, max_M=M, max_kg=kg, max_kt=10)
+    head.set_path(lmhead.CORAL_PATH_TCGEN05)
+    out = ph.gpu_draft_numpy(head, hb, kg, 10)
+    assert head.status() == 0 and head.stats().path == lmhead.CORAL_PATH_TCGEN05
+    counts = np.bincount(out["groups"].ravel(), minlength=N)
+    assert (counts > 256).any() and ((counts > 128) & (counts <= 256)).any() and ((counts > 0) & (counts <= 128)).any()
+    rows = np.unique(np.linspace(0, M - 1, 40).astype(int))
+    rep = ph.compare(W, gm, Wg, hb[rows], kg, 10, {k: a[rows] for k, a in out.items()})
+    assert rep.ok, rep.errors
+    again = ph.gpu_draft_numpy(head, hb, kg, 10)
+    for k in ("ids", "logprobs", "groups"):
+        assert np.array_equal(out[k], again[k]), k
+    head.close()
+
+
 @pytest.mark.parametrize("M,kg,zipf,expect", [
     (40, 2, 0.0, lmhead.CORAL_PATH_STREAM),      # ~5 rows per group: one read per group either way -> streaming kernel
     (60, 4, 1.5, lmhead.CORAL_PATH_TCGEN05),     # hot groups selected by most rows -> tensor-core kernel
