@@ -152,8 +152,10 @@ int coral_lmhead_draft_ex(coral_lmhead_handle h, const void *hidden_dev, int M, 
  * The same draft step for callers that hold HOST buffers (hidden_host
  * [M x H] bf16; out_ids_host / out_logprobs_host [M x k_tokens]).  Copies the
  * rows to the device, runs coral_lmhead_draft, copies the results back and
- * synchronises `stream` before returning.  Pinned host memory makes the copies
- * asynchronous up to that final synchronisation.
+ * synchronises `stream` before returning.  Pinned host memory makes the copy
+ * in asynchronous up to that final synchronisation, and pinned output buffers
+ * are written by the last kernel directly (no copies back); pageable buffers
+ * work too, staged through the workspace.
  */
 int coral_lmhead_draft_host(coral_lmhead_handle h, const void *hidden_host, int M, int k_groups, int k_tokens,
                             int32_t *out_ids_host, float *out_logprobs_host, void *stream);

@@ -204,6 +204,9 @@ struct coral_lmhead_s {
     bool timing;
     // facts about the last draft call
     int last_path, last_M, last_kg, last_kt, last_launches;
+    // coral_lmhead_draft_host: the host output buffers seen last and their device aliases (null: not pinned)
+    const void* host_seen[2] = {nullptr, nullptr};
+    void* host_alias[2] = {nullptr, nullptr};
 };
 
 namespace {
@@ -730,6 +733,23 @@ int coral_lmhead_draft(coral_lmhead_handle h, const void* hidden_dev, int M, int
                                  out_ids_dev, out_logprobs_dev, stream);
 }
 
+// The address through which kernels may write a buffer of pinned (page-locked, mapped) host memory, or null for any
+// other kind of memory.  The answer for the buffer seen last is remembered: callers reuse their buffers, and
+// the query costs about a microsecond.
+static void* pinned_alias(coral_lmhead_handle h, int which, const void* host) {
+    if (h->host_seen[which] == host) return h->host_alias[which];
+    cudaPointerAttributes attr{};
+    void* alias = nullptr;
+    if (cudaPointerGetAttributes(&attr, host) == cudaSuccess) {
+        if (attr.type == cudaMemoryTypeHost) alias = attr.devicePointer;
+    } else {
+        cudaGetLastError();              // unregistered memory is not an error of this call
+    }
+    h->host_seen[which] = host;
+    h->host_alias[which] = alias;
+    return alias;
+}
+
 int coral_lmhead_draft_host(coral_lmhead_handle h, const void* hidden_host, int M, int k_groups, int k_tokens,
                             int32_t* out_ids_host, float* out_logprobs_host, void* stream) {
     if (!h || !hidden_host || !out_ids_host || !out_logprobs_host) return CORAL_ERR_INVALID;
@@ -737,15 +757,21 @@ int coral_lmhead_draft_host(coral_lmhead_handle h, const void* hidden_host, int 
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     unsigned char* ws = h->ws;
     void* d_hidden = ws + h->L.stage_hidden;
-    int32_t* d_ids = reinterpret_cast<int32_t*>(ws + h->L.stage_ids);
-    float* d_lp = reinterpret_cast<float*>(ws + h->L.stage_logprobs);
+    // Pinned output buffers are written by the merge itself (a few hundred bytes over the host link); the two
+    // copies back, and what it costs to queue them behind the kernels, fall away.  Other memory is staged.
+    int32_t* ids_alias = static_cast<int32_t*>(pinned_alias(h, 0, out_ids_host));
+    float* lp_alias = static_cast<float*>(pinned_alias(h, 1, out_logprobs_host));
+    int32_t* d_ids = ids_alias ? ids_alias : reinterpret_cast<int32_t*>(ws + h->L.stage_ids);
+    float* d_lp = lp_alias ? lp_alias : reinterpret_cast<float*>(ws + h->L.stage_logprobs);
     if (cudaMemcpyAsync(d_hidden, hidden_host, (size_t)M * h->cfg.H * 2, cudaMemcpyHostToDevice, st) != cudaSuccess)
         return CORAL_ERR_CUDA;
     const int rc = coral_lmhead_draft(h, d_hidden, M, k_groups, k_tokens, d_ids, d_lp, stream);
     if (rc != CORAL_OK) return rc;
-    if (cudaMemcpyAsync(out_ids_host, d_ids, (size_t)M * k_tokens * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+    if (!ids_alias &&
+        cudaMemcpyAsync(out_ids_host, d_ids, (size_t)M * k_tokens * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess)
         return CORAL_ERR_CUDA;
-    if (cudaMemcpyAsync(out_logprobs_host, d_lp, (size_t)M * k_tokens * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+    if (!lp_alias &&
+        cudaMemcpyAsync(out_logprobs_host, d_lp, (size_t)M * k_tokens * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess)
         return CORAL_ERR_CUDA;
     if (cudaStreamSynchronize(st) != cudaSuccess) return CORAL_ERR_CUDA;
     return CORAL_OK;

@@ -164,6 +164,15 @@ def test_library_owned_buffers_and_host_entry():
     lmhead.coral_lmhead_draft_host(handle, hh, cfg.k_groups, 10, ids, lps)
     rep = ph.compare(W, gm, Wg, hb, cfg.k_groups, 10, {"ids": ids.numpy(), "logprobs": lps.numpy()})
     assert rep.ok, rep.errors
+    # pageable buffers take the staged way (pinned ones are written by the last kernel directly): same results
+    ids2 = torch.full((cfg.M, 10), -7, dtype=torch.int32)
+    lps2 = torch.zeros((cfg.M, 10), dtype=torch.float32)
+    lmhead.coral_lmhead_draft_host(handle, torch.from_numpy(hb.view(np.int16)).clone(), cfg.k_groups, 10, ids2, lps2)
+    assert np.array_equal(ids2.numpy(), ids.numpy()) and np.array_equal(lps2.numpy(), lps.numpy())
+    # and back to the pinned pair on the same handle
+    ids.fill_(-7)
+    lmhead.coral_lmhead_draft_host(handle, hh, cfg.k_groups, 10, ids, lps)
+    assert np.array_equal(ids2.numpy(), ids.numpy()) and np.array_equal(lps2.numpy(), lps.numpy())
     assert lmhead.coral_lmhead_status(handle) == 0
     lmhead.coral_lmhead_destroy(handle)
 
