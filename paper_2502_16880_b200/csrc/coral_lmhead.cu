@@ -344,6 +344,14 @@ bool stream_ok(const coral_lmhead_s* h, int M) { return h->stream_smem > 0 && M 
 
 // CORAL_PATH_STREAM: streaming kernel (M <= 128, H a multiple of 256, <= 4096); CORAL_PATH_SIMT_PLAIN: any shape.  Returns 0 if the
 // forced path cannot run this call.
+// The gathered hidden rows of a call (one copy per row and selected group).  Above this many bytes the pair kernel's
+// consecutive runs no longer find them in L2 (126 MB, shared with the weight stream) and the pairs take the
+// batches in turn instead.
+constexpr size_t kTcStridedHgBytes = (size_t)72 << 20;
+int tc_strided(const coral_lmhead_s* h, int M, int kg) {
+    return (size_t)M * kg * h->cfg.H * 2 > kTcStridedHgBytes ? 1 : 0;
+}
+
 bool tc_usable(const coral_lmhead_s* h, int M, int kg) {
     const size_t cands = (size_t)kg * h->L.tc_tiles * h->cfg.max_k_tokens;
     return h->tc_ok && (size_t)M * kg <= h->L.tc_rows && kg * h->L.tc_tiles <= kMergeMaxPieces &&
@@ -628,7 +636,7 @@ static int draft_impl(coral_lmhead_handle h, const void* hidden_dev, int M, int 
         mg.T = L.tc_tiles;
         if (adaptive) {
             // both head kernels are launched; each reads the router's choice first and the one not chosen returns
-            TcGeom tg{h->tc_pairs, L.tc_tiles, (L.tc_tiles + 1) / 2, L.KB, L.tc_hg_rows};
+            TcGeom tg{h->tc_pairs, L.tc_tiles, (L.tc_tiles + 1) / 2, L.KB, L.tc_hg_rows, tc_strided(h, M, k_groups)};
             TcPartials tp{tpp.pmax, tpp.psum, tpp.pval, tpp.pid};
             launch_pdl(tc_gather_kernel, dim3((M * k_groups + kGatherPairs - 1) / kGatherPairs), dim3(64 * kGatherPairs), (size_t)0, st, c,
                        reinterpret_cast<uint16_t*>(h->ws + L.tc_hg), L.tc_hg_rows);
@@ -656,7 +664,7 @@ static int draft_impl(coral_lmhead_handle h, const void* hidden_dev, int M, int 
         ++launches;
     } else if (path == CORAL_PATH_TCGEN05) {
         const Layout& L = h->L;
-        TcGeom tg{h->tc_pairs, L.tc_tiles, (L.tc_tiles + 1) / 2, L.KB, L.tc_hg_rows};
+        TcGeom tg{h->tc_pairs, L.tc_tiles, (L.tc_tiles + 1) / 2, L.KB, L.tc_hg_rows, tc_strided(h, M, k_groups)};
         TcPartials tp{reinterpret_cast<float*>(h->ws + L.tc_max), reinterpret_cast<float*>(h->ws + L.tc_sum),
                       reinterpret_cast<float*>(h->ws + L.tc_val), reinterpret_cast<int32_t*>(h->ws + L.tc_id)};
         launch_pdl(tc_gather_kernel, dim3((M * k_groups + kGatherPairs - 1) / kGatherPairs), dim3(64 * kGatherPairs), (size_t)0, st, c,

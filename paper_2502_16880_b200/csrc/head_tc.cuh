@@ -81,6 +81,7 @@ struct TcGeom {
     int units;        // units per group = ceil(tiles / 2)
     int ksteps;       // ceil(H / 64) = 64-column blocks of the packed layout
     int hg_rows;      // rows of one column block of the gathered hidden matrix
+    int strided;      // 1: the pairs take the batches of the call in turn (see tc_split_runs)
 };
 
 struct TcPartials {
@@ -233,12 +234,30 @@ __device__ __forceinline__ void tc_flush_row(const CallView& c, const TcPartials
     }
 }
 
-// Walks a pair's run batch by batch.  A run is a number of consecutive units of the unit list (entry by entry,
-// unit by unit).  A batch is the next two units of the run when they belong to one entry of at most 128
-// padded rows ("narrow"), else one unit.
+// Relative time of one unit of an entry with `rows` rows.  A narrow entry's units go two to a batch and a batch
+// streams at what an SM can take in (its weight tiles plus its share of the hidden rows, in 128-byte units per
+// 64 columns); a wide entry's unit is a batch of its own, whose pace the MMA issue and the slot hand-over set
+// rather than the bytes: about 0.8 of a narrow batch of two (the weight that gave the shortest whole step at
+// 960 and 1440 rows on the Llama3-8B shape; between 0.75 and 0.9 it matters by 1-2 %).
+__device__ __forceinline__ int tc_unit_cost(int rows) {
+    const int npad = (max(1, min(rows, kTcPassRows)) + 15) & ~15;
+    return npad > kTcSub ? kTcSub + 96 + (npad >> 2) : kTcSub + (npad >> 2);
+}
+constexpr int kTcCostNarrowMax = kTcSub + (kTcSub >> 2);      // the largest cost of a narrow entry's unit
+__device__ __forceinline__ bool tc_cost_is_wide(int cost) { return cost > kTcCostNarrowMax; }
+
+// Walks a pair's run batch by batch.  A batch is two units of one entry of at most 128 padded rows ("narrow"),
+// else one unit.  A run is either a number of consecutive units of the unit list (entry by entry, unit by unit;
+// its batches are cut from the run's first unit on), or every stride-th batch of the call's batch list (the
+// entries' batches in order, a narrow entry's being its units 0-1, 2-3, ...), found through the entries' cached
+// costs.
 struct TcWalk {
     int j, u;             // entry (index in the union list) and unit inside it
-    int left;             // units of the run still to do, this batch included
+    int left;             // consecutive: units of the run still to do, this batch included; strided: batches
+    int strided, stride;  // strided run: distance between its batches in the batch list
+    int b, bbase;         // strided run: this batch's index in the list, index of entry j's first batch
+    int n_entries;
+    const int* cost;      // the entries' unit costs (shared memory), which tell narrow from wide
     int n, R, npad, first, hrow;
     bool wide, read_again;
     __device__ __forceinline__ void load(const CallView& c) {
@@ -255,12 +274,33 @@ struct TcWalk {
         if (!CORAL_IDX_OK(hrow + npad - 1, c.cap_hg_rows, c.state)) hrow = 0;     // (checked build) read rows that exist
         if (!CORAL_IDX_OK(first + R - 1, c.cap_pairs, c.state)) first = 0;
     }
-    __device__ __forceinline__ void start(const CallView& c, const int* run) {
-        j = run[0]; u = run[1]; left = run[2];
+    __device__ __forceinline__ int batches_of(int e, const TcGeom& g) const {
+        return tc_cost_is_wide(cost[e]) ? g.units : (g.units + 1) >> 1;
+    }
+    // strided run: the entry and unit of batch b (entries are only ever passed forwards)
+    __device__ __forceinline__ void seek(const TcGeom& g) {
+        while (j + 1 < n_entries && b >= bbase + batches_of(j, g)) { bbase += batches_of(j, g); ++j; }
+        u = (b - bbase) * (tc_cost_is_wide(cost[j]) ? 1 : 2);
+    }
+    __device__ __forceinline__ void start(const CallView& c, const TcGeom& g, const int* run, const int* cost_cache) {
+        left = run[2]; strided = run[3]; n_entries = run[4];
+        cost = cost_cache;
+        if (!strided) {
+            j = run[0]; u = run[1];
+        } else {
+            b = run[0]; stride = run[1]; j = 0; bbase = 0;
+            if (left > 0) seek(g);
+        }
         if (left > 0) load(c);
     }
-    __device__ __forceinline__ int nunits(const TcGeom& g) const { return wide ? 1 : min(2, min(g.units - u, left)); }
+    __device__ __forceinline__ int nunits(const TcGeom& g) const {
+        return wide ? 1 : strided ? min(2, g.units - u) : min(2, min(g.units - u, left));
+    }
     __device__ __forceinline__ void next(const CallView& c, const TcGeom& g) {
+        if (strided) {
+            if (--left > 0) { b += stride; seek(g); load(c); }
+            return;
+        }
         const int nu = nunits(g);
         u += nu;
         left -= nu;
@@ -268,19 +308,18 @@ struct TcWalk {
     }
 };
 
-// Relative time of one unit of an entry with `rows` rows.  A narrow entry's units go two to a batch and a batch
-// streams at what an SM can take in (its weight tiles plus its share of the hidden rows, in 128-byte units per
-// 64 columns); a wide entry's unit is a batch of its own, whose pace the MMA issue and the slot hand-over set
-// rather than the bytes: about 0.8 of a narrow batch of two (the weight that gave the shortest whole step at
-// 960 and 1440 rows on the Llama3-8B shape; between 0.75 and 0.9 it matters by 1-2 %).
-__device__ __forceinline__ int tc_unit_cost(int rows) {
-    const int npad = (max(1, min(rows, kTcPassRows)) + 15) & ~15;
-    return npad > kTcSub ? kTcSub + 96 + (npad >> 2) : kTcSub + (npad >> 2);
-}
-
-// Cuts the unit list into g.pairs runs of (almost) equal cost (one warp).  out[0], out[1]: entry and unit where
-// the pair's run starts; out[2]: its number of units.  Run p holds the units whose cost prefix (tc_unit_cost),
-// taken at the unit's middle, lies in [p, p + 1) * total / pairs.
+// Gives every pair its run (one warp).
+// Consecutive (out[3] = 0): the unit list is cut into g.pairs runs of (almost) equal cost.  out[0], out[1]: entry
+// and unit where the pair's run starts; out[2]: its number of units.  Run p holds the units whose cost prefix
+// (tc_unit_cost), taken at the unit's middle, lies in [p, p + 1) * total / pairs.
+// Strided (out[3] = 1, when g.strided and the costs fit the cache): pair p takes batches p, p + pairs, ... of
+// the call's batch list; out[0] = p, out[1] = pairs, out[2] = its number of batches.  The pairs then work on
+// the same few entries at the same time, so an entry's gathered hidden rows, which every one of its batches
+// reads in full, and the weights of a group that a second pass reads again are found in L2 by all but the first
+// reader; with consecutive runs each pair sweeps its own entry's rows (2 MB at 256 rows and H = 4096) once per
+// unit, and from some 70 MB of gathered rows on those sweeps push each other out of L2 (Llama3-8B shape, 1920
+// rows: 2.11 GB from HBM for 1.05 GB of weights).
+// out[4]: entries of the call.
 // (The entries' costs are read from global memory once - two dependent loads each, all of a lane's in flight together -
 // and kept in `cost_cache` for the second pass; beyond kTcCostCache entries the second pass reads them again.)
 constexpr int kTcCostCache = 1024;
@@ -288,6 +327,7 @@ __device__ __forceinline__ void tc_split_runs(const CallView& c, const TcGeom& g
                                               int* cost_cache) {
     const int lane = threadIdx.x & 31;
     long long total = 0;
+    int batches = 0;
 #pragma unroll 4
     for (int j0 = 0; j0 < n_entries; j0 += 32) {
         const int j = j0 + lane;
@@ -296,11 +336,25 @@ __device__ __forceinline__ void tc_split_runs(const CallView& c, const TcGeom& g
             const int w = tc_unit_cost(c.group_count[entry & 0xffff] - (entry >> 16) * kTcPassRows);
             if (j < kTcCostCache) cost_cache[j] = w;
             total += (long long)g.units * w;
+            batches += tc_cost_is_wide(w) ? g.units : (g.units + 1) >> 1;
         }
     }
     __syncwarp();
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) total += __shfl_xor_sync(0xffffffffu, total, o);
+    for (int o = 16; o > 0; o >>= 1) {
+        total += __shfl_xor_sync(0xffffffffu, total, o);
+        batches += __shfl_xor_sync(0xffffffffu, batches, o);
+    }
+    if (g.strided && n_entries <= kTcCostCache) {
+        if (lane == 0) {
+            out[0] = pair;
+            out[1] = g.pairs;
+            out[2] = pair < batches ? (batches - pair + g.pairs - 1) / g.pairs : 0;
+            out[3] = 1;
+            out[4] = n_entries;
+        }
+        return;
+    }
     const long long t_lo = pair * total / g.pairs, t_hi = (pair + 1) * total / g.pairs;
     // global index (entry * units + unit) of the first unit whose middle reaches t_lo, and t_hi
     const int n_units = n_entries * g.units;
@@ -353,6 +407,8 @@ __device__ __forceinline__ void tc_split_runs(const CallView& c, const TcGeom& g
         out[0] = lo / g.units;
         out[1] = lo - (lo / g.units) * g.units;
         out[2] = max(0, hi - lo);
+        out[3] = 0;
+        out[4] = n_entries;
     }
 }
 
@@ -369,7 +425,7 @@ template <int KT>
 __device__ __forceinline__ void tc_epilogue(const CallView& c, const TcGeom& g, const TcPartials& pp,
                                             float* __restrict__ logits_tap, uint32_t tmem_base, uint64_t* tmem_full,
                                             uint32_t tmem_empty_at, bool leader, volatile int* abort_flag, float* xchg,
-                                            const int* run, int rank) {
+                                            const int* run, const int* cost_cache, int rank) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int q = warp & 3;                                // lane quarter this warp may read = block it owns
     const int quad = (warp - 2) >> 2;                      // accumulator 0 or 1 of the batch
@@ -380,7 +436,7 @@ __device__ __forceinline__ void tc_epilogue(const CallView& c, const TcGeom& g, 
     int pending_j = -1, pending_n = 0;
     bool pending_valid = false;
     TcWalk w;
-    w.start(c, run);
+    w.start(c, g, run, cost_cache);
     for (int batch = 0; w.left > 0; ++batch) {
         const int buf = batch & 1;
         tc_wait(smem_u32(&tmem_full[buf]), ((uint32_t)batch >> 1) & 1u, abort_flag, c.state);
@@ -464,7 +520,7 @@ __global__ void __launch_bounds__(kTcHeadThreads, 1)
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(recut + 1);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
     int* cost_cache = reinterpret_cast<int*>(smem + kTcRingBytes + kTcXchgBytes + 256);      // [kTcCostCache]
-    int* run = const_cast<int*>(abort_flag) + 1;  // [3] entry and unit where the pair's run starts, number of units
+    int* run = const_cast<int*>(abort_flag) + 1;  // [5] the pair's run, see tc_split_runs
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int rank = (int)cluster_ctarank();
     const bool leader = rank == 0;
@@ -521,7 +577,7 @@ __global__ void __launch_bounds__(kTcHeadThreads, 1)
             const uint64_t pol_first = l2_policy_evict_first(), pol_normal = l2_policy_evict_normal(),
                            pol_last = l2_policy_evict_last();
             TcWalk w;
-            w.start(c, run);
+            w.start(c, g, run, cost_cache);
             while (w.left > 0) {
                 const int u = w.u, nu = w.nunits(g);
                 const int t0 = 2 * u + rank, t1 = 2 * (u + 1) + rank;           // this CTA's sub-tiles
@@ -578,7 +634,7 @@ __global__ void __launch_bounds__(kTcHeadThreads, 1)
             TcRingPos rp;
             const uint32_t ring_lo = tc_smem_desc_lo(smem_u32(smem));
             TcWalk w;
-            w.start(c, run);
+            w.start(c, g, run, cost_cache);
             for (int batch = 0; w.left > 0; ++batch) {
                 const int buf = batch & 1;
                 const TcRing ring = tc_ring_for(w.wide, w.nunits(g));
@@ -613,7 +669,7 @@ __global__ void __launch_bounds__(kTcHeadThreads, 1)
             const uint32_t peer_at = cluster_map_shared(smem_u32(full), 0);
             TcRingPos rp;
             TcWalk w;
-            w.start(c, run);
+            w.start(c, g, run, cost_cache);
             while (w.left > 0) {
                 const TcRing ring = tc_ring_for(w.wide, w.nunits(g));
                 rp.enter(ring);
@@ -629,9 +685,9 @@ __global__ void __launch_bounds__(kTcHeadThreads, 1)
         // epilogue: the four warps of an accumulator exchange blocks so that every thread owns one hidden row
         const uint32_t tmem_empty_at = leader ? smem_u32(tmem_empty) : cluster_map_shared(smem_u32(tmem_empty), 0);
         if (c.k_tokens <= 10)
-            tc_epilogue<10>(c, g, pp, logits_tap, tmem_base, tmem_full, tmem_empty_at, leader, abort_flag, xchg, run, rank);
+            tc_epilogue<10>(c, g, pp, logits_tap, tmem_base, tmem_full, tmem_empty_at, leader, abort_flag, xchg, run, cost_cache, rank);
         else
-            tc_epilogue<32>(c, g, pp, logits_tap, tmem_base, tmem_full, tmem_empty_at, leader, abort_flag, xchg, run, rank);
+            tc_epilogue<32>(c, g, pp, logits_tap, tmem_base, tmem_full, tmem_empty_at, leader, abort_flag, xchg, run, cost_cache, rank);
     }
     tc_fence_before();
     cluster_sync_all();          // nothing of the other CTA is still on its way to this CTA's barriers or tensor memory
