@@ -347,7 +347,7 @@ bool stream_ok(const coral_lmhead_s* h, int M) { return h->stream_smem > 0 && M 
 // The gathered hidden rows of a call (one copy per row and selected group).  Above this many bytes the pair kernel's
 // consecutive runs no longer find them in L2 (126 MB, shared with the weight stream) and the pairs take the
 // batches in turn instead.
-constexpr size_t kTcStridedHgBytes = (size_t)72 << 20;
+constexpr size_t kTcStridedHgBytes = (size_t)96 << 20;
 int tc_strided(const coral_lmhead_s* h, int M, int kg) {
     return (size_t)M * kg * h->cfg.H * 2 > kTcStridedHgBytes ? 1 : 0;
 }
