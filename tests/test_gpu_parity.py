@@ -434,6 +434,34 @@ def test_tensor_core_path_mixed_entry_kinds_with_an_odd_number_of_column_steps()
     head.close()
 
 
+@pytest.mark.parametrize("zipf", [0.0, 1.5])
+def test_tensor_core_path_many_rows_take_the_batches_in_turn(zipf):
+    """More than 96 MB of gathered hidden rows (1600 rows x 8 groups x 8 KiB): the pairs take the call's batches
+    in turn instead of consecutive runs.  Every group needs several passes of 256 rows (its weights are read
+    again), the last tile of a group is ragged, and with the skewed routing narrow entries sit between the wide
+    ones, so the operand ring is re-cut between a pair's batches."""
+    N, v, M, kg = 16, 300, 1600, 8
+    cfg = synth.HeadConfig("turns", H=4096, V=v * N, N=N, k_groups=kg, k_tokens=10, M=M, seed=31, w_std=0.02,
+                           zipf_s=zipf)
+    W, Wg, hb = synth.make_w_vocab(cfg), synth.make_w_gate(cfg), synth.make_hidden(cfg)
+    gm = synth.make_group_map(cfg, contiguous=zipf > 0)
+    head = _head(cfg, W, gm, Wg, max_M=M, max_kg=kg, max_kt=10)
+    head.set_path(lmhead.CORAL_PATH_TCGEN05)
+    out = ph.gpu_draft_numpy(head, hb, kg, 10)
+    assert head.status() == 0 and head.stats().path == lmhead.CORAL_PATH_TCGEN05
+    counts = np.bincount(out["groups"].ravel(), minlength=N)
+    assert (counts > 256).any()
+    if zipf > 0:
+        assert ((counts % 256 > 0) & (counts % 256 <= 128)).any()      # some entry is narrow
+    rows = np.unique(np.linspace(0, M - 1, 64).astype(int))
+    rep = ph.compare(W, gm, Wg, hb[rows], kg, 10, {k: a[rows] for k, a in out.items()})
+    assert rep.ok, rep.errors
+    again = ph.gpu_draft_numpy(head, hb, kg, 10)
+    for k in ("ids", "logprobs", "groups"):
+        assert np.array_equal(out[k], again[k]), k
+    head.close()
+
+
 @pytest.mark.parametrize("M,kg,zipf,expect", [
     (40, 2, 0.0, lmhead.CORAL_PATH_STREAM),      # ~5 rows per group: one read per group either way -> streaming kernel
     (60, 4, 1.5, lmhead.CORAL_PATH_TCGEN05),     # hot groups selected by most rows -> tensor-core kernel
