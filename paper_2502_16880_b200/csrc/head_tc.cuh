@@ -582,12 +582,8 @@ __global__ void __launch_bounds__(kTcHeadThreads, 1)
                 const int u = w.u, nu = w.nunits(g);
                 const int t0 = 2 * u + rank, t1 = 2 * (u + 1) + rank;           // this CTA's sub-tiles
                 const bool w0 = t0 < g.tiles, w1 = nu == 2 && t1 < g.tiles;
-                // this CTA's half of the hidden rows; a wide entry is two column ranges of the accumulator with their
-                // own MMAs (rows 0..127 and the rest), so its half is two pieces: 64 rows of the first range, then
-                // half of the second
-                const int n2 = w.wide ? w.npad - kTcSub : 0;
-                const uint32_t h1bytes = (uint32_t)(w.wide ? kTcSub >> 1 : w.npad >> 1) * 128u, h2bytes = (uint32_t)(n2 >> 1) * 128u;
-                const uint32_t hbytes = h1bytes + h2bytes;
+                // this CTA's half of the entry's hidden rows (the first half in rank 0)
+                const uint32_t hbytes = (uint32_t)(w.npad >> 1) * 128u;
                 const TcRing ring = tc_ring_for(w.wide, nu);
                 if (rp.enter(ring)) {
                     // another slot size from here on: every copy issued so far, by either producer, must have been
@@ -606,8 +602,7 @@ __global__ void __launch_bounds__(kTcHeadThreads, 1)
                 }
                 const uint32_t bytes = hbytes + (w0 ? kTcTileBytes : 0) + (w1 ? kTcTileBytes : 0);
                 const uint64_t pol_w = w.read_again ? pol_normal : pol_first;
-                const uint16_t* hsrc = hg + ((size_t)w.hrow + (size_t)rank * (w.wide ? kTcSub >> 1 : w.npad >> 1)) * kTcK;
-                const uint16_t* hsrc2 = hg + ((size_t)w.hrow + kTcSub + (size_t)rank * (n2 >> 1)) * kTcK;
+                const uint16_t* hsrc = hg + ((size_t)w.hrow + (size_t)rank * (w.npad >> 1)) * kTcK;
                 const int gidx = w.n / c.pack_div;
                 for (int ks = 0; ks < g.ksteps; ++ks, ++step) {
                     if ((step & 1u) != mine) { rp.advance(ring); continue; }
@@ -617,8 +612,7 @@ __global__ void __launch_bounds__(kTcHeadThreads, 1)
                     mbar_expect_tx(bar, bytes);
                     if (w0) tma_load_5d(sb, &map_w, 0, 0, ks, t0 * 8, gidx, bar, pol_w);
                     if (w1) tma_load_5d(sb + kTcTileBytes, &map_w, 0, 0, ks, t1 * 8, gidx, bar, pol_w);
-                    bulk_g2s_hint(sb + ring.hoff, hsrc + (size_t)ks * g.hg_rows * kTcK, h1bytes, bar, pol_last);
-                    if (n2) bulk_g2s_hint(sb + ring.hoff + (kTcTileBytes >> 1), hsrc2 + (size_t)ks * g.hg_rows * kTcK, h2bytes, bar, pol_last);
+                    bulk_g2s_hint(sb + ring.hoff, hsrc + (size_t)ks * g.hg_rows * kTcK, hbytes, bar, pol_last);
                     rp.advance(ring);
                 }
                 w.next(c, g);
@@ -626,8 +620,9 @@ __global__ void __launch_bounds__(kTcHeadThreads, 1)
         }
     } else if (warp == 1 || warp == 10) {
         if (lane == 0 && leader) {
-            // issuer `a` owns accumulator a of a batch of two units, or of a wide entry's one unit the columns of
-            // hidden rows 128 a .. (same weight tile, the a-th piece of the hidden rows); both issuers commit on
+            // issuer `a` owns accumulator a of a batch of two units; a batch of one unit - a wide entry's, with up
+            // to 256 columns in one MMA, or a run's odd unit - is the first issuer's (splitting a wide entry's columns
+            // between the two changed nothing: 442 against 441 us at 1920 rows).  Both issuers commit on
             // every slot and every batch (a commit with nothing pending arrives at once), so the barriers always
             // count two arrivals
             const int a = warp == 1 ? 0 : 1;
@@ -640,9 +635,9 @@ __global__ void __launch_bounds__(kTcHeadThreads, 1)
                 const TcRing ring = tc_ring_for(w.wide, w.nunits(g));
                 rp.enter(ring);
                 const uint32_t aoff_lo = w.wide ? 0u : (uint32_t)a * (kTcTileBytes >> 4);
-                const uint32_t boff_lo = (ring.hoff + (w.wide ? a * (kTcTileBytes >> 1) : 0)) >> 4;
-                const uint32_t idesc = tc_idesc(256, !w.wide ? w.npad : a == 0 ? kTcSub : w.npad - kTcSub);
-                const bool mine = w.wide || a < w.nunits(g);
+                const uint32_t boff_lo = ring.hoff >> 4;
+                const uint32_t idesc = tc_idesc(256, w.npad);
+                const bool mine = a < w.nunits(g);            // (a wide entry's one unit: the first issuer's)
                 tc_wait(smem_u32(&tmem_empty[buf]), (((uint32_t)batch >> 1) & 1u) ^ 1u, abort_flag, c.state);   // drained
                 tc_fence_after();
                 const uint32_t acc = tmem_base + (uint32_t)(buf * 2 * kTcSub + a * kTcSub);
