@@ -2,7 +2,8 @@
 compute from the router's output is compared with the capacity of the array it indexes, and a violation sets
 CORAL_ERR_BOUNDS instead of touching memory.  Here the draft step runs on that build, in a process of its
 own (the library is chosen when the package is first imported), over shapes that exercise every kernel -
-all three head paths, ragged groups, several passes per group, wide tensor-core entries, forced groups, the
+all three head paths, ragged groups, several passes per group, wide tensor-core entries, the many-row mode of
+the tensor-core kernel, forced groups, the
 two-layer router, vocab sharding - and must come out with status 0 and the oracle's results."""
 import os
 import subprocess
@@ -26,6 +27,7 @@ CASES = textwrap.dedent("""
         (256, 256, 16, 200, 4, 10, lmhead.CORAL_PATH_TCGEN05), (256, 256, 16, 300, 8, 10, lmhead.CORAL_PATH_TCGEN05),
         (320, 300, 6, 400, 3, 5, lmhead.CORAL_PATH_TCGEN05), (256, 256, 16, 1200, 8, 10, lmhead.CORAL_PATH_TCGEN05),
         (256, 256, 16, 60, 16, 10, lmhead.CORAL_PATH_AUTO), (256, 256, 16, 100, 4, 10, lmhead.CORAL_PATH_ADAPTIVE),
+        (4096, 300, 16, 1600, 8, 10, lmhead.CORAL_PATH_TCGEN05),      # 105 MB of gathered rows: batches taken in turn
     ]
     for H, v, N, M, kg, kt, path in shapes:
         cfg = synth.HeadConfig("chk", H=H, V=v * N, N=N, k_groups=kg, k_tokens=kt, M=M, seed=11, w_std=0.05)
